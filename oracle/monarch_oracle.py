@@ -1,0 +1,324 @@
+"""CPU oracle for the Monarch Mixer hot path (arXiv 2310.12109).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain, double-precision
+statement of what the GPU library must compute.  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import it; the product path
+never does, and this module imports nothing from the product package.
+
+Two tiers:
+
+* Tier 1 -- the plain definitions the method reaches exactly (up to rounding):
+  stride permutation matrices, block-diagonal matrices, the dense product
+  ``P L P^T R P``, the DFT matrix, direct O(N^2) circular / causal convolution,
+  and the element-wise pieces of the M2 block (depthwise conv, GELU, dense
+  block-diagonal MLP).
+* Tier 2 -- the method step by step in the paper's order: factored Monarch
+  apply (permute, block-diagonal multiply, permute, ...), the Monarch factors
+  that make ``M = F_N`` (Corollary "DFT is M", App. D.5), and the Monarch
+  convolution ``M^-1 (M k  (.)  M u)`` (Eq. 2, Def. "matrix convolution",
+  Alg. BlockMonarchConv).  Tier 2 is itself pinned to tier 1 by the CPU tests.
+
+All arithmetic is float64 / complex128.  Index conventions (App. D notation):
+``N = N1*N2*...*Np``; the input index is ``n = (..(n1*N2 + n2)*N3 + ..)`` with
+n1 most significant; the natural output index is ``k = k1 + N1*k2 + N1*N2*k3``
+with k1 least significant.  "Plan order" is the tensor ``[k1][k2]..[kp]`` stored
+row-major.
+
+Pins (see tests/test_oracle_*.py): permutation closed forms and inverses,
+``M == F_N`` entry-wise, numpy's FFT (a different algorithm) for large N,
+brute-force convolution sums, Parseval, delta / shift kernels, causality,
+explicit dense products on tiny N.  Unpinned by the paper: the linear order of
+order-p block ids for p >= 3 with arbitrary (non-DFT) blocks, and the wiring of
+the M2 block composition (gate, short conv alignment, block count) -- marked
+"parity unpinned" at the functions concerned.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+# ----------------------------------------------------------------------------
+# Tier 1: definitions
+# ----------------------------------------------------------------------------
+
+
+def stride_perm(b: int, N: int) -> np.ndarray:
+    """sigma_(b,N)(i) = i0 * N/b + i1 for i = i1*b + i0 (App. D notation, item on
+    the permutation class P_(b,N))."""
+    if b <= 0 or N % b != 0:
+        raise ValueError("b must divide N")
+    i = np.arange(N, dtype=np.int64)
+    i0 = i % b
+    i1 = i // b
+    return i0 * (N // b) + i1
+
+
+def perm_matrix(b: int, N: int) -> np.ndarray:
+    """P_(b,N): the N x N matrix whose i-th row is e_{sigma_(b,N)(i)}, so that
+    (P x)[i] = x[sigma(i)] (App. D notation)."""
+    P = np.zeros((N, N))
+    P[np.arange(N), stride_perm(b, N)] = 1.0
+    return P
+
+
+def apply_perm(b: int, N: int, x: np.ndarray) -> np.ndarray:
+    """(P_(b,N) x) along the last axis."""
+    return x[..., stride_perm(b, N)]
+
+
+def blockdiag_dense(W: np.ndarray) -> np.ndarray:
+    """Dense matrix of a block-diagonal factor.  W has shape [nblocks, out, in]
+    (the weight layout of the paper's blockdiag_matmul listing, App. A)."""
+    nb, o, i = W.shape
+    D = np.zeros((nb * o, nb * i), dtype=W.dtype)
+    for b in range(nb):
+        D[b * o:(b + 1) * o, b * i:(b + 1) * i] = W[b]
+    return D
+
+
+def monarch_dense(L: np.ndarray, R: np.ndarray) -> np.ndarray:
+    """Dense order-2 Monarch matrix M = P L P^T R P (Sec. 3.1) with P = P_(N1,N).
+
+    R: [N2, N1, N1] (N2 blocks, applied first), L: [N1, N2, N2] (N1 blocks).
+    For square N (N1 == N2) P^T = P and this is the paper's M = P L P R P."""
+    N2, N1, _ = R.shape
+    assert R.shape == (N2, N1, N1) and L.shape == (N1, N2, N2)
+    N = N1 * N2
+    P = perm_matrix(N1, N)
+    return P @ blockdiag_dense(L) @ P.T @ blockdiag_dense(R) @ P
+
+
+def dft_matrix(N: int, sign: int = +1) -> np.ndarray:
+    """F_N[i, j] = omega_N^{i j}, omega_N = exp(sign * 2 pi i / N).  The paper uses
+    sign = +1 (App. D, definition of the roots of unity)."""
+    idx = np.arange(N)
+    # reduce the exponent modulo N in integers so large N stays accurate
+    e = (np.outer(idx, idx) % N).astype(np.float64)
+    return np.exp(sign * 2j * np.pi * e / N)
+
+
+def direct_circular_conv(k: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """y[t] = sum_{u=0}^{N-1} k[u] x[(t-u) mod N], along the last axis."""
+    N = x.shape[-1]
+    assert k.shape[-1] == N
+    y = np.zeros(np.broadcast_shapes(k.shape, x.shape), dtype=np.result_type(k, x))
+    t = np.arange(N)
+    for u in range(N):
+        y += k[..., u:u + 1] * x[..., (t - u) % N]
+    return y
+
+
+def direct_causal_conv(k: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """y[t] = sum_{u=0}^{t} k[u] x[t-u], 0 <= t < n: multiplication by the lower
+    triangular Toeplitz matrix of k (App. D.3, review of causal maps)."""
+    n = x.shape[-1]
+    assert k.shape[-1] == n
+    y = np.zeros(np.broadcast_shapes(k.shape, x.shape), dtype=np.result_type(k, x))
+    for u in range(n):
+        y[..., u:] += k[..., u:u + 1] * x[..., :n - u]
+    return y
+
+
+def depthwise_conv3_same(x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """Short depthwise convolution of width 3 along the sequence, centred, zero
+    padded: g[b,t,c] = w[c,0] x[b,t-1,c] + w[c,1] x[b,t,c] + w[c,2] x[b,t+1,c].
+    x: [B, T, C], w: [C, 3].  (Sec. 5.1 mentions the short conv only in words;
+    alignment is this build's reading -- parity unpinned.)"""
+    B, T, C = x.shape
+    g = w[:, 1] * x
+    g[:, 1:, :] += w[:, 0] * x[:, :-1, :]
+    g[:, :-1, :] += w[:, 2] * x[:, 1:, :]
+    return g
+
+
+def gelu_erf(v: np.ndarray) -> np.ndarray:
+    """GELU(v) = v/2 * (1 + erf(v / sqrt 2)), evaluated with math.erf."""
+    erf = np.vectorize(math.erf, otypes=[np.float64])
+    return 0.5 * v * (1.0 + erf(v / math.sqrt(2.0)))
+
+
+def blockdiag_apply(W: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """out[..., b, n] = sum_m W[b, n, m] x[..., b, m] on the last axis split into
+    nblocks groups (the blockdiag_matmul listing, App. A)."""
+    nb, o, i = W.shape
+    xs = x.reshape(*x.shape[:-1], nb, i)
+    out = np.einsum("bnm,...bm->...bn", W, xs)
+    return out.reshape(*x.shape[:-1], nb * o)
+
+
+# ----------------------------------------------------------------------------
+# Tier 2: the method, step by step
+# ----------------------------------------------------------------------------
+
+
+def monarch_apply(L: np.ndarray, R: np.ndarray, x: np.ndarray, stages: dict | None = None) -> np.ndarray:
+    """y = P L P^T R P x along the last axis, evaluated as the paper evaluates it
+    (Sec. 3.1 and the MonarchMatrix listing): permute, block-diagonal multiply
+    with R, permute, block-diagonal multiply with L, permute.  No dense N x N
+    matrix is formed.  `stages`, if given, receives every intermediate."""
+    N2, N1, _ = R.shape
+    N = N1 * N2
+    assert x.shape[-1] == N and L.shape == (N1, N2, N2)
+    v0 = apply_perm(N1, N, x)            # [n2][n1]
+    v1 = blockdiag_apply(R, v0)          # [n2][k1]
+    v2 = apply_perm(N2, N, v1)           # P^T = P_(N/N1, N): [k1][n2]
+    v3 = blockdiag_apply(L, v2)          # [k1][k2]   (plan order)
+    y = apply_perm(N1, N, v3)            # [k2][k1]   (natural order)
+    if stages is not None:
+        stages.update(after_P=v0, after_R=v1, after_Pt=v2, after_L=v3, out=y)
+    return y
+
+
+def monarch_apply_order_p(blocks: list, dims: tuple, x: np.ndarray) -> np.ndarray:
+    """Order-p Monarch apply in the direct form (App. D.6, "p-variate Monarch"):
+    stage a (a = 1..p) contracts input digit n_a into output digit k_a with the
+    block selected by (k1..k_{a-1}, n_{a+1}..n_p); blocks[a-1] has shape
+    [prod(dims)/dims[a-1], dims[a-1], dims[a-1]] with the block id the row-major
+    flattening of (k1, .., k_{a-1}, n_{a+1}, .., n_p).  Output in natural order
+    k = k1 + N1 k2 + ...   (For p >= 3 with arbitrary blocks the paper gives the
+    block index as a tuple only; the linear order here is this build's reading --
+    parity unpinned.  The DFT instance does not depend on it.)"""
+    p = len(dims)
+    N = int(np.prod(dims))
+    lead = x.shape[:-1]
+    v = x.reshape(*lead, *dims)          # axes: n1..np
+    nl = len(lead)
+    for a in range(p):
+        Na = dims[a]
+        W = blocks[a].reshape(*dims[:a], *dims[a + 1:], Na, Na)   # (k1..k_{a-1}, n_{a+1}..np, out, in)
+        # move the contracted axis last on the data
+        vt = np.moveaxis(v, nl + a, -1)                           # (lead, k1..k_{a-1}, n_{a+1}..np, n_a)
+        out = np.einsum("...oi,...i->...o", W, vt)                # per-block mat-vec
+        v = np.moveaxis(out, -1, nl + a)
+    # v axes are k1..kp; natural order has kp most significant
+    perm = list(range(nl)) + [nl + a for a in reversed(range(p))]
+    return np.transpose(v, perm).reshape(*lead, N)
+
+
+def monarch_dft_factors(N1: int, N2: int, sign: int = +1):
+    """Block-diagonal factors with P L P^T R P = F_N, N = N1 N2 (Corollary "DFT is
+    M": l_{j1}(Z) = Z^{j1}, r~_{j1,j0}(Z) = Z^{j0}).  Every block of R is F_{N1};
+    block k1 of L evaluates Z^{n2} at omega_N^{k1 + N1 k2}, i.e.
+    L[k1][k2, n2] = omega_N^{(k1 + N1 k2) n2} = (F_{N2} diag(omega_N^{k1 n2}))[k2, n2]."""
+    N = N1 * N2
+    R = np.broadcast_to(dft_matrix(N1, sign), (N2, N1, N1)).copy()
+    k1 = np.arange(N1)[:, None, None]
+    k2 = np.arange(N2)[None, :, None]
+    n2 = np.arange(N2)[None, None, :]
+    e = ((k1 + N1 * k2) * n2) % N
+    L = np.exp(sign * 2j * np.pi * e / N)
+    return L, R
+
+
+def monarch_dft_factors_order_p(dims: tuple, sign: int = +1) -> list:
+    """Order-p generalisation of the corollary: stage a's block with id
+    (k1..k_{a-1}, n_{a+1}..) is F_{Na} with its columns scaled by the twiddle
+    omega_{N1..Na}^{n_a (k1 + N1 k2 + .. + N1..N_{a-2} k_{a-1})}; independent of
+    the trailing n digits."""
+    p = len(dims)
+    blocks = []
+    for a in range(p):
+        Na = dims[a]
+        Mprev = int(np.prod(dims[:a]))         # N1..N_{a-1}
+        Mcur = Mprev * Na
+        trail = int(np.prod(dims[a + 1:]))
+        # kappa = k1 + N1 k2 + ... enumerated in block-id (row-major k1..k_{a-1}) order
+        kappa = np.zeros((1,), dtype=np.int64)
+        w = 1
+        for j in range(a):
+            kappa = (kappa[:, None] + w * np.arange(dims[j])[None, :]).reshape(-1)
+            w *= dims[j]
+        ka = np.arange(Na)[None, :, None]
+        na = np.arange(Na)[None, None, :]
+        e = (na * (kappa[:, None, None] + Mprev * ka)) % Mcur
+        B = np.exp(sign * 2j * np.pi * e / Mcur)              # [Mprev, Na, Na]
+        B = np.repeat(B[:, None], trail, axis=1).reshape(Mprev * trail, Na, Na)
+        blocks.append(B)
+    return blocks
+
+
+def monarch_inverse_factors(L: np.ndarray, R: np.ndarray):
+    """Block inverses: (P L P^T R P)^-1 = P^T R^-1 P L^-1 P^T with R^-1, L^-1 block
+    diagonal (each block inverted on its own)."""
+    return np.linalg.inv(L), np.linalg.inv(R)
+
+
+def monarch_inverse_apply(Linv: np.ndarray, Rinv: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """x = P^T R^-1 P L^-1 P^T y (the factors of monarch_apply undone in reverse)."""
+    N2, N1, _ = Rinv.shape
+    N = N1 * N2
+    v3 = apply_perm(N2, N, y)            # P^T: natural [k2][k1] -> [k1][k2]
+    v2 = blockdiag_apply(Linv, v3)       # [k1][n2]
+    v1 = apply_perm(N1, N, v2)           # P:   [n2][k1]
+    v0 = blockdiag_apply(Rinv, v1)       # [n2][n1]
+    return apply_perm(N2, N, v0)         # P^T: [n1][n2]
+
+
+def plan_order_index(dims: tuple) -> np.ndarray:
+    """pos -> natural frequency k for plan order: position ((k1*N2+k2)*N3+..)
+    holds frequency k1 + N1 k2 + N1 N2 k3 + ...   (a digit reversal)."""
+    p = len(dims)
+    grids = np.meshgrid(*[np.arange(d) for d in dims], indexing="ij")
+    k = np.zeros_like(grids[0])
+    w = 1
+    for a in range(p):
+        k = k + w * grids[a]
+        w *= dims[a]
+    return k.reshape(-1).astype(np.int64)
+
+
+def monarch_dft(x: np.ndarray, dims: tuple, sign: int = +1, plan_order: bool = False) -> np.ndarray:
+    """F_N x by the factored Monarch apply (order len(dims)).  With plan_order the
+    last permutation is left out and the result stays as [k1][k2].. row-major."""
+    blocks = monarch_dft_factors_order_p(dims, sign)
+    y = monarch_apply_order_p(blocks, dims, x.astype(np.complex128))
+    if plan_order:
+        return y[..., plan_order_index(dims)]
+    return y
+
+
+def monarch_conv(k: np.ndarray, x: np.ndarray, dims: tuple, causal: bool, sign: int = +1,
+                 stages: dict | None = None) -> np.ndarray:
+    """Monarch convolution f = M^-1 (M k' (.) M u') with M the Monarch-DFT
+    (Alg. BlockMonarchConv with the corollary's factors; Eq. 2).
+
+    causal: k, x have length n <= N/2; both are zero padded to N = prod(dims) and
+    the first n outputs are kept (App. D.3 review; Thm 3).  Otherwise n == N and
+    the result is the circular convolution.  k: [..., n] broadcastable against
+    x: [..., n] (kernel per channel, shared over the batch)."""
+    N = int(np.prod(dims))
+    n = x.shape[-1]
+    assert k.shape[-1] == n
+    if causal:
+        assert 2 * n <= N
+        kp = np.concatenate([k, np.zeros((*k.shape[:-1], N - n))], axis=-1)
+        xp = np.concatenate([x, np.zeros((*x.shape[:-1], N - n))], axis=-1)
+    else:
+        assert n == N
+        kp, xp = k, x
+    blocks = monarch_dft_factors_order_p(dims, sign)
+    k_f = monarch_apply_order_p(blocks, dims, kp.astype(np.complex128))
+    u_f = monarch_apply_order_p(blocks, dims, xp.astype(np.complex128))
+    prod = k_f * u_f
+    # M^-1 = conj(M) / N for the DFT: apply the conjugated factors, scale by 1/N
+    cblocks = [np.conj(B) for B in blocks]
+    f = monarch_apply_order_p(cblocks, dims, prod) / N
+    if stages is not None:
+        stages.update(k_f=k_f, u_f=u_f, prod=prod, f=f)
+    return np.real(f[..., :n])
+
+
+def m2_block_forward(x, k, w_short, W_up, W_down, dims=(32, 16)):
+    """M2 block forward as configured for the M2-BERT-base shape (Sec. 5.1, Eq. 2-3):
+    gate g = depthwise-conv3(x); long mix v = circular Monarch conv of x with k
+    along the sequence per channel; z = g (.) v; MLP y = bd(W_down) GELU(bd(W_up) z)
+    with 4-block block-diagonal matrices.  x: [B, T, C]; k: [C, T]; w_short: [C, 3];
+    W_up: [4, 4C/4, C/4]; W_down: [4, C/4, 4C/4].  (Composition is this build's
+    reading of the paper's prose -- parity unpinned; every piece is pinned.)"""
+    g = depthwise_conv3_same(x, w_short)
+    xt = np.transpose(x, (0, 2, 1))                       # [B, C, T]
+    v = monarch_conv(k[None], xt, dims, causal=False)     # [B, C, T]
+    z = g * np.transpose(v, (0, 2, 1))
+    h = gelu_erf(blockdiag_apply(W_up, z))
+    return blockdiag_apply(W_down, h), z

@@ -1,0 +1,366 @@
+"""CPU pins for the oracle: each check ties an oracle function to something other than
+itself -- a closed form, a brute-force sum, a library routine computing the same thing by a
+different algorithm, an invariant, or a number the paper prints."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import monarch_oracle as O
+
+rng = np.random.default_rng(20231012)
+
+RECT = [(2, 2), (2, 3), (3, 2), (4, 4), (8, 8), (32, 16), (16, 32), (3, 5)]
+
+
+# ---- permutations (App. D notation; Sec. 3.1 "reshape to 2D, transpose, flatten") --------
+
+@pytest.mark.parametrize("N1,N2", RECT)
+def test_stride_perm_is_reshape_transpose(N1, N2):
+    N = N1 * N2
+    x = rng.standard_normal(N)
+    # P_(N1,N) x == view x as N1 x N2 row-major, transpose, flatten
+    assert np.array_equal(O.apply_perm(N1, N, x), x.reshape(N1, N2).T.reshape(-1))
+    # einops "(m n) -> (n m)" with n = N2 is the same thing
+    from einops import rearrange
+    assert np.array_equal(O.apply_perm(N1, N, x), rearrange(x, "(m n) -> (n m)", n=N2))
+
+
+@pytest.mark.parametrize("N1,N2", RECT)
+def test_perm_inverse_and_transpose(N1, N2):
+    N = N1 * N2
+    P = O.perm_matrix(N1, N)
+    Q = O.perm_matrix(N2, N)
+    assert np.array_equal(P.T, Q)                       # P_(b,N)^T = P_(N/b,N)
+    assert np.array_equal(P @ Q, np.eye(N))
+    assert sorted(O.stride_perm(N1, N).tolist()) == list(range(N))
+    if N1 == N2:
+        assert np.array_equal(P @ P, np.eye(N))         # square case: an involution
+    # composing the index maps gives the identity
+    s1, s2 = O.stride_perm(N1, N), O.stride_perm(N2, N)
+    assert np.array_equal(s1[s2], np.arange(N))
+
+
+def test_stride_perm_small_literal():
+    # N = 6, b = 2: i = i1*2 + i0 -> i0*3 + i1
+    assert O.stride_perm(2, 6).tolist() == [0, 3, 1, 4, 2, 5]
+    assert O.stride_perm(3, 6).tolist() == [0, 2, 4, 1, 3, 5]
+
+
+# ---- block-diagonal multiply and dense Monarch ---------------------------------------------
+
+def test_blockdiag_apply_matches_dense_and_loops():
+    W = rng.standard_normal((3, 4, 5))
+    x = rng.standard_normal((2, 15))
+    D = O.blockdiag_dense(W)
+    assert D.shape == (12, 15)
+    ref = np.zeros((2, 12))
+    for r in range(2):
+        for b in range(3):
+            for o in range(4):
+                for i in range(5):
+                    ref[r, b * 4 + o] += W[b, o, i] * x[r, b * 5 + i]
+    np.testing.assert_allclose(O.blockdiag_apply(W, x), ref, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(x @ D.T, ref, rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("N1,N2", [(2, 2), (2, 3), (3, 2), (3, 4), (4, 4), (8, 8)])
+def test_factored_apply_equals_dense_product(N1, N2):
+    N = N1 * N2
+    L = rng.standard_normal((N1, N2, N2))
+    R = rng.standard_normal((N2, N1, N1))
+    x = rng.standard_normal((3, N))
+    M = O.monarch_dense(L, R)
+    y = O.monarch_apply(L, R, x)
+    np.testing.assert_allclose(y, x @ M.T, rtol=0, atol=1e-12)
+    # tensor form: y[k2*N1+k1] = sum_{n2} L[k1][k2,n2] sum_{n1} R[n2][k1,n1] x[n1*N2+n2]
+    ref = np.zeros((3, N))
+    for k1 in range(N1):
+        for k2 in range(N2):
+            for n2 in range(N2):
+                for n1 in range(N1):
+                    ref[:, k2 * N1 + k1] += L[k1, k2, n2] * R[n2, k1, n1] * x[:, n1 * N2 + n2]
+    np.testing.assert_allclose(y, ref, rtol=0, atol=1e-12)
+    # order-p routine, p = 2, is the same map
+    y2 = O.monarch_apply_order_p([R, L], (N1, N2), x)
+    np.testing.assert_allclose(y2, y, rtol=0, atol=1e-12)
+
+
+def test_identity_blocks_give_the_permutation():
+    N1, N2 = 4, 3
+    N = N1 * N2
+    L = np.broadcast_to(np.eye(N2), (N1, N2, N2)).copy()
+    R = np.broadcast_to(np.eye(N1), (N2, N1, N1)).copy()
+    x = rng.standard_normal(N)
+    np.testing.assert_array_equal(O.monarch_apply(L, R, x), O.apply_perm(N1, N, x))   # P P^T P = P
+
+
+def test_listing_semantics_square():
+    """The MonarchMatrix listing (App. A) applies its first parameter right after the
+    first rearrange; in M = P L P R P that slot is R.  Re-enact the listing with plain
+    reshapes and compare with the dense product."""
+    s = 4
+    N = s * s
+    first = rng.standard_normal((s, s, s))
+    second = rng.standard_normal((s, s, s))
+    x = rng.standard_normal((2, N))
+
+    def rearr(v):
+        return v.reshape(-1, s, s).transpose(0, 2, 1).reshape(-1, N)
+
+    def bd(v, w):
+        return np.einsum("bnm,rbm->rbn", w, v.reshape(-1, s, s)).reshape(-1, N)
+
+    out = rearr(bd(rearr(bd(rearr(x), first)), second))
+    M = O.monarch_dense(second, first)
+    np.testing.assert_allclose(out, x @ M.T, rtol=0, atol=1e-12)
+
+
+def test_inverse_factors_roundtrip():
+    N1, N2 = 4, 6
+    L = rng.standard_normal((N1, N2, N2)) + np.eye(N2)
+    R = rng.standard_normal((N2, N1, N1)) + np.eye(N1)
+    x = rng.standard_normal((2, N1 * N2))
+    Li, Ri = O.monarch_inverse_factors(L, R)
+    np.testing.assert_allclose(O.monarch_inverse_apply(Li, Ri, O.monarch_apply(L, R, x)), x, atol=1e-9)
+
+
+# ---- the DFT as a Monarch matrix (Corollary "DFT is M") -----------------------------------
+
+def test_dft_matrix_convention():
+    F = O.dft_matrix(8, +1)
+    w = np.exp(2j * np.pi / 8)
+    assert abs(F[1, 1] - w) < 1e-15 and abs(F[3, 5] - w ** 15) < 1e-14
+    x = rng.standard_normal(8)
+    # sign=+1 is the conjugate of numpy's forward transform, i.e. N * ifft
+    np.testing.assert_allclose(F @ x, 8 * np.fft.ifft(x), atol=1e-13)
+    np.testing.assert_allclose(O.dft_matrix(8, -1) @ x, np.fft.fft(x), atol=1e-13)
+    np.testing.assert_allclose(F @ np.conj(F) / 8, np.eye(8), atol=1e-13)
+
+
+@pytest.mark.parametrize("N1,N2", RECT)
+@pytest.mark.parametrize("sign", [+1, -1])
+def test_monarch_dft_is_the_dft_matrix(N1, N2, sign):
+    L, R = O.monarch_dft_factors(N1, N2, sign)
+    M = O.monarch_dense(L, R)
+    np.testing.assert_allclose(M, O.dft_matrix(N1 * N2, sign), rtol=0, atol=2e-12)
+
+
+def test_twiddle_free_factors_are_not_the_dft_but_the_2d_transform():
+    """L = R = I (x) F_sqrtN (Sec. 3.1) without twiddles is the 2-D DFT of the sqrtN x sqrtN
+    reshape; its Monarch convolution is the 2-D circular convolution (Thm 2), not the 1-D one."""
+    s = 4
+    N = s * s
+    F = O.dft_matrix(s)
+    L = np.broadcast_to(F, (s, s, s)).copy()
+    M = O.monarch_dense(L, L)
+    assert np.abs(M - O.dft_matrix(N)).max() > 0.5
+    x = rng.standard_normal(N)
+    k = rng.standard_normal(N)
+    Minv = np.linalg.inv(M)
+    y = np.real(Minv @ ((M @ k) * (M @ x)))
+    X2, K2 = x.reshape(s, s), k.reshape(s, s)
+    ref = np.zeros((s, s))
+    for a in range(s):
+        for b in range(s):
+            for c in range(s):
+                for d in range(s):
+                    ref[a, b] += K2[c, d] * X2[(a - c) % s, (b - d) % s]
+    np.testing.assert_allclose(y, ref.reshape(-1), atol=1e-11)
+    assert np.abs(y - O.direct_circular_conv(k, x)).max() > 1e-3
+
+
+@pytest.mark.parametrize("dims", [(2, 3, 4), (4, 4, 4), (8, 4, 2), (3, 3, 3), (2, 2, 2, 2), (32, 16), (16, 32)])
+def test_order_p_monarch_dft_full(dims):
+    N = int(np.prod(dims))
+    X = np.eye(N)
+    Y = O.monarch_dft(X, dims, +1)              # rows = F_N e_j = column j of F_N
+    np.testing.assert_allclose(Y.T, O.dft_matrix(N, +1), rtol=0, atol=5e-12)
+
+
+def test_order3_monarch_dft_32768_against_library_fft():
+    dims = (32, 32, 32)
+    N = 32768
+    x = rng.standard_normal((2, N))
+    y = O.monarch_dft(x, dims, +1)
+    ref = N * np.fft.ifft(x, axis=-1)           # omega = e^{+2 pi i / N}
+    assert np.linalg.norm(y - ref) / np.linalg.norm(ref) < 1e-12
+    # Parseval: ||F x||^2 = N ||x||^2
+    np.testing.assert_allclose(np.sum(np.abs(y) ** 2, -1), N * np.sum(x ** 2, -1), rtol=1e-12)
+    # sampled columns of the matrix itself
+    for j in (0, 1, 31, 32, 1023, 1024, 16385, 32767):
+        e = np.zeros(N)
+        e[j] = 1.0
+        col = O.monarch_dft(e, dims, +1)
+        kk = np.arange(N)
+        np.testing.assert_allclose(col, np.exp(2j * np.pi * ((kk * j) % N) / N), atol=1e-11)
+
+
+def test_plan_order_is_digit_reversal():
+    dims = (2, 3, 4)
+    pos = O.plan_order_index(dims)
+    assert sorted(pos.tolist()) == list(range(24))
+    for k1 in range(2):
+        for k2 in range(3):
+            for k3 in range(4):
+                assert pos[(k1 * 3 + k2) * 4 + k3] == k1 + 2 * k2 + 6 * k3
+    x = rng.standard_normal(24)
+    nat = O.monarch_dft(x, dims)
+    np.testing.assert_array_equal(O.monarch_dft(x, dims, plan_order=True), nat[pos])
+
+
+# ---- convolution ---------------------------------------------------------------------------
+
+def test_direct_convs_against_loops_and_library():
+    n = 13
+    k = rng.standard_normal(n)
+    x = rng.standard_normal(n)
+    cau = np.zeros(n)
+    cir = np.zeros(n)
+    for t in range(n):
+        for u in range(n):
+            if u <= t:
+                cau[t] += k[u] * x[t - u]
+            cir[t] += k[u] * x[(t - u) % n]
+    np.testing.assert_allclose(O.direct_causal_conv(k, x), cau, atol=1e-13)
+    np.testing.assert_allclose(O.direct_circular_conv(k, x), cir, atol=1e-13)
+    np.testing.assert_allclose(O.direct_causal_conv(k, x), np.convolve(k, x)[:n], atol=1e-13)
+    full = np.convolve(k, x)
+    wrap = full[:n].copy()
+    wrap[:n - 1] += full[n:]
+    np.testing.assert_allclose(O.direct_circular_conv(k, x), wrap, atol=1e-12)
+
+
+@pytest.mark.parametrize("dims", [(2, 2), (2, 3), (4, 4), (32, 16), (16, 32), (4, 4, 4), (2, 3, 4)])
+def test_monarch_conv_equals_direct_circular(dims):
+    N = int(np.prod(dims))
+    k = rng.standard_normal((3, N))
+    x = rng.standard_normal((2, 3, N))
+    y = O.monarch_conv(k[None], x, dims, causal=False)
+    ref = O.direct_circular_conv(k[None], x)
+    assert np.linalg.norm(y - ref) / np.linalg.norm(ref) < 1e-12
+
+
+@pytest.mark.parametrize("dims,n", [((2, 2), 2), ((4, 4), 8), ((4, 4), 5), ((32, 16), 256), ((4, 4, 4), 32), ((8, 8, 8), 256)])
+def test_monarch_conv_equals_direct_causal(dims, n):
+    k = rng.standard_normal((3, n))
+    x = rng.standard_normal((2, 3, n))
+    y = O.monarch_conv(k[None], x, dims, causal=True)
+    ref = O.direct_causal_conv(k[None], x)
+    assert y.shape == ref.shape
+    assert np.linalg.norm(y - ref) / np.linalg.norm(ref) < 1e-12
+
+
+def test_monarch_conv_sign_independent_and_stages():
+    dims = (4, 8)
+    k = rng.standard_normal(32)
+    x = rng.standard_normal(32)
+    st = {}
+    yp = O.monarch_conv(k, x, dims, causal=False, sign=+1, stages=st)
+    ym = O.monarch_conv(k, x, dims, causal=False, sign=-1)
+    np.testing.assert_allclose(yp, ym, atol=1e-12)
+    np.testing.assert_allclose(st["u_f"], O.dft_matrix(32) @ x, atol=1e-11)
+    assert np.abs(np.imag(st["f"])).max() < 1e-12
+
+
+def test_monarch_conv_special_kernels_and_invariants():
+    dims = (32, 16)
+    N = 512
+    x = rng.standard_normal((2, N))
+    delta = np.zeros(N)
+    delta[0] = 1.0
+    np.testing.assert_allclose(O.monarch_conv(delta, x, dims, causal=False), x, atol=1e-12)
+    d1 = np.zeros(N)
+    d1[1] = 1.0
+    np.testing.assert_allclose(O.monarch_conv(d1, x, dims, causal=False), np.roll(x, 1, -1), atol=1e-12)
+    k = rng.standard_normal(N)
+    # shift equivariance (circular) and linearity
+    y = O.monarch_conv(k, x, dims, causal=False)
+    np.testing.assert_allclose(O.monarch_conv(k, np.roll(x, 7, -1), dims, causal=False), np.roll(y, 7, -1), atol=1e-11)
+    x2 = rng.standard_normal((2, N))
+    np.testing.assert_allclose(O.monarch_conv(k, 2 * x - 3 * x2, dims, causal=False),
+                               2 * y - 3 * O.monarch_conv(k, x2, dims, causal=False), atol=1e-11)
+    # causality: changing x[t0:] leaves y[:t0] unchanged
+    n = 256
+    kc = rng.standard_normal(n)
+    xa = rng.standard_normal(n)
+    xb = xa.copy()
+    xb[100:] += rng.standard_normal(n - 100)
+    ya = O.monarch_conv(kc, xa, dims, causal=True)
+    yb = O.monarch_conv(kc, xb, dims, causal=True)
+    np.testing.assert_allclose(ya[:100], yb[:100], atol=1e-12)
+    assert np.abs(ya[100:] - yb[100:]).max() > 1e-3
+    # causal delta_1 is a shift with zero fill
+    d1c = np.zeros(n)
+    d1c[1] = 1.0
+    ys = O.monarch_conv(d1c, xa, dims, causal=True)
+    np.testing.assert_allclose(ys[1:], xa[:-1], atol=1e-12)
+    assert abs(ys[0]) < 1e-12
+
+
+def test_order3_causal_conv_full_size_sampled():
+    """Thm (arbitrary basis, any matrix equal to F_N) => zero padding to N = 2n suffices for
+    order 3 as well: check a full-length row against the direct sum at sampled outputs."""
+    from paper_2310_12109_b200 import synth
+    n = 16384
+    x = rng.standard_normal(n)
+    k = synth.decay_kernel(4, 1, n, 0.0005, 128.0)[0].astype(np.float64)
+    y = O.monarch_conv(k, x, (32, 32, 32), causal=True)
+    for t in (0, 1, 2, 31, 32, 1023, 1024, 5000, 16383):
+        ref = float(np.dot(k[:t + 1], x[t::-1]))
+        assert abs(y[t] - ref) < 1e-10 * max(1.0, abs(ref))
+
+
+# ---- M2 block pieces ---------------------------------------------------------------------
+
+def test_gelu_values():
+    v = np.array([0.0, 1.0, -1.0, 3.0])
+    ref = np.array([0.0, 0.8413447460685429, -0.15865525393145707, 2.9959502191322303])
+    np.testing.assert_allclose(O.gelu_erf(v), ref, atol=1e-14)
+    from scipy.special import erf
+    w = rng.standard_normal(100)
+    np.testing.assert_allclose(O.gelu_erf(w), 0.5 * w * (1 + erf(w / math.sqrt(2))), atol=1e-15)
+
+
+def test_depthwise_conv_against_library():
+    x = rng.standard_normal((2, 9, 3))
+    w = rng.standard_normal((3, 3))
+    g = O.depthwise_conv3_same(x, w)
+    for b in range(2):
+        for c in range(3):
+            # np.convolve flips its kernel: g[t] = sum_j w[j] x[t + j - 1]
+            ref = np.convolve(x[b, :, c], w[c, ::-1], mode="same")
+            np.testing.assert_allclose(g[b, :, c], ref, atol=1e-13)
+
+
+def test_block_forward_composition_small():
+    B, T, C = 2, 16, 8
+    x = rng.standard_normal((B, T, C))
+    k = rng.standard_normal((C, T))
+    w = rng.standard_normal((C, 3))
+    Wu = rng.standard_normal((4, 8, 2))
+    Wd = rng.standard_normal((4, 2, 8))
+    y, z = O.m2_block_forward(x, k, w, Wu, Wd, dims=(4, 4))
+    # explicit per-element evaluation
+    for b in range(B):
+        for c in range(C):
+            v = O.direct_circular_conv(k[c], x[b, :, c])
+            g = np.convolve(x[b, :, c], w[c, ::-1], mode="same")
+            np.testing.assert_allclose(z[b, :, c], g * v, atol=1e-11)
+    h = O.gelu_erf(z @ O.blockdiag_dense(Wu).T)
+    np.testing.assert_allclose(y, h @ O.blockdiag_dense(Wd).T, atol=1e-11)
+
+
+# ---- the one set of numbers the paper prints for this path: Table 2 FLOP costs ---------------
+
+def test_table2_flop_convention():
+    path = os.path.join(os.path.dirname(__file__), "golden", "table2_flop_cost.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    for N, dense, m2 in rows:
+        N = int(N)
+        dense_model = 2.0 * N * N * 768 / 1e12
+        m2_model = 8.0 * N ** 1.5 * 768 / 1e12
+        # printed with 3 significant digits (two entries differ in the last printed digit)
+        assert abs(dense_model - float(dense)) <= 0.012 * float(dense) + 6e-4
+        assert abs(m2_model - float(m2)) <= 0.012 * float(m2) + 6e-4

@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the Monarch hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one fused Monarch convolution (load, forward Monarch-DFT, spectrum multiply, inverse,
+store) over the M2-BERT-base-shaped batch: x[32, 768, 512] bf16, circular, N = 512 = 32 x 16.
+The step cycles through buffer sets that together exceed twice the L2 so DRAM traffic is real.
+Prints ONE JSON line.  Multi-GPU: every rank runs the same per-GPU workload (rows are independent,
+no collective on the data path); the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "Monarch-conv tokens*channels/s"
+UNIT = "tokens*ch/s"
+WORKLOAD = "config2: bidirectional Monarch conv x[B=32,H=768,N=512] bf16, N=512=32x16, fp32 accumulate"
+B2, H2, N2 = 32, 768, 512
+L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes (read + write) of one launch of the dominant kernel from the ncu capture summarised in
+# profiles/; None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def reduce_max(value: float) -> float:
+    """Max over ranks (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        t = torch.tensor([value], dtype=torch.float64)
+        if dist.get_backend() == "nccl":
+            t = t.cuda()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+    return value
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+# ---- CPU baseline: the oracle as it stands, on a bounded sample ---------------------------------
+
+def oracle_conv_sample(reps: int = 2):
+    """Times the oracle's Monarch conv on the full config-2 batch `reps` times; returns
+    (tokens*ch/s, cores used, description)."""
+    from oracle import monarch_oracle as O
+    from paper_2310_12109_b200 import synth
+    c = synth.config2(B=B2, H=H2)
+    k64, x64 = c["k"].astype(np.float64)[None], c["x"].astype(np.float64)
+    w0, c0 = time.perf_counter(), time.process_time()
+    for _ in range(reps):
+        O.monarch_conv(k64, x64, c["dims"], causal=False)
+    wall, cpu = time.perf_counter() - w0, time.process_time() - c0
+    units = reps * B2 * H2 * N2
+    cores = max(1, int(round(cpu / wall)))
+    return units / wall, cores, f"oracle.monarch_conv on the full config-2 batch ({B2 * H2} rows x {N2}), {reps} passes, {wall:.1f} s"
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import monarch_oracle as O
+    from paper_2310_12109_b200 import synth
+    # each step: the oracle on a bounded sample of the same workload, sized so that the whole run
+    # (warm-up + steps) stays near two minutes at the oracle's ~5e3 rows/s
+    rows = int(5000 * 120.0 / max(1, args.steps + args.warmup))
+    Bs = max(1, min(B2, rows // H2))
+    Hs = H2 if rows >= H2 else max(8, rows)
+    c = synth.config2(B=Bs, H=Hs)
+    k64, x64 = c["k"].astype(np.float64)[None], c["x"].astype(np.float64)
+    for _ in range(args.warmup):
+        O.monarch_conv(k64, x64, c["dims"], causal=False)
+    w0, c0 = time.perf_counter(), time.process_time()
+    for _ in range(args.steps):
+        O.monarch_conv(k64, x64, c["dims"], causal=False)
+    wall, cpu = time.perf_counter() - w0, time.process_time() - c0
+    value = args.steps * Bs * Hs * N2 / wall
+    cores = max(1, int(round(cpu / wall)))
+    sample = f"each step = oracle.monarch_conv on {Bs * Hs} of the {B2 * H2} rows (x {N2})"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * wall / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---- GPU arm ----------------------------------------------------------------------------------------
+
+def time_launches(fn, n, torch):
+    """CUDA-event time (ms) of n back-to-back calls of fn(i) on the current stream."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def side_workloads(torch, M, synth, peaks, quick: bool):
+    """Config 3 (Monarch matmul) and config 4 (order-3 causal conv): time per launch, throughput and
+    roofline fraction, outside the headline timed region."""
+    out = {}
+    reps = 3 if quick else 10
+    # config 3
+    T, b = 16384, 64
+    c = synth.config3(T=T, b=b)
+    plan = M.Plan((b, b), dtype=M.M2_BF16, device=torch.cuda.current_device())
+    bf = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)  # noqa: E731
+    L, R = bf(c["L"]), bf(c["R"])
+    Xs = [bf(c["X"]) for _ in range(2)]
+    Ys = [torch.empty_like(Xs[0]) for _ in range(2)]
+    f = lambda i: M.m2_monarch_matmul(plan, Xs[i % 2], L, R, Ys[i % 2])  # noqa: E731
+    time_launches(f, 3, torch)
+    ms = time_launches(f, reps, torch) / reps
+    by = 2 * T * b * b * 2 + 2 * b * b * b * 2
+    fl = 4.0 * T * b * b * b
+    out["config3_matmul"] = {
+        "kernel": plan.last_kernel(), "ms": ms, "elements_per_s": T * b * b / (ms * 1e-3), "algorithmic_GBps": by / (ms * 1e6),
+        "TFLOPs": fl / (ms * 1e9), "roofline": {"bound": "hbm", "achieved": by / (ms * 1e6), "peak": peaks["hbm_gbs"],
+                                                 "unit": "GB/s", "frac": by / (ms * 1e6) / peaks["hbm_gbs"]}}
+    plan.close()
+    del Xs, Ys
+    # config 4
+    B, H, n = 4, 1024, 16384
+    c = synth.config4(B=B, H=H, n=n)
+    plan = M.Plan((32, 32, 32), dtype=M.M2_BF16, device=torch.cuda.current_device())
+    kf = M.m2_kernel_spectrum(plan, torch.from_numpy(c["k"]).cuda())
+    xs = [bf(c["x"]) for _ in range(2)]
+    ys = [torch.empty_like(xs[0]) for _ in range(2)]
+    f = lambda i: M.m2_monarch_conv_fwd(plan, xs[i % 2], kf, M.M2_CAUSAL, y=ys[i % 2])  # noqa: E731
+    time_launches(f, 2, torch)
+    ms = time_launches(f, reps, torch) / reps
+    by = 2 * B * H * n * 2 + H * 32768 * 8
+    fl = 2.0 * (2 + 4 + 4) * 32768 * 32 * 2 * B * H   # plain count: real first stage, complex after, fwd + inv
+    t_hbm = by / (peaks["hbm_gbs"] * 1e9)
+    t_tc = fl / (peaks["bf16_tflops_sustained"] * 1e12)
+    bound = "tensor" if t_tc > t_hbm else "hbm"
+    ach = fl / (ms * 1e9) if bound == "tensor" else by / (ms * 1e6)
+    pk = peaks["bf16_tflops_sustained"] if bound == "tensor" else peaks["hbm_gbs"]
+    out["config4_conv_order3"] = {
+        "kernel": plan.last_kernel(), "ms": ms, "tokens_ch_per_s": B * H * n / (ms * 1e-3), "algorithmic_GBps": by / (ms * 1e6),
+        "TFLOPs_plain_count": fl / (ms * 1e9),
+        "roofline": {"bound": bound, "achieved": ach, "peak": pk, "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": ach / pk}}
+    plan.close()
+    return out
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2310_12109_b200 import binding as M
+    from paper_2310_12109_b200 import build as BLD
+    from paper_2310_12109_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group(backend="nccl", init_method="env://")
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    BLD.build()
+    peaks = measured_peaks()
+
+    c = synth.config2(B=B2, H=H2)
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=local_rank)
+    kf = M.m2_kernel_spectrum(plan, torch.from_numpy(c["k"]).cuda())
+    x0 = torch.from_numpy(c["x"]).cuda().to(torch.bfloat16)
+    set_bytes = 2 * x0.numel() * 2 + B2 * 0 + H2 * N2 * 8
+    nsets = max(2, -(-2 * L2_BYTES // set_bytes))          # rotate through > 2 x L2
+    xs = [x0] + [x0.clone() for _ in range(nsets - 1)]
+    ys = [torch.empty_like(x0) for _ in range(nsets)]
+
+    def step(i):
+        M.m2_monarch_conv_fwd(plan, xs[i % nsets], kf, M.M2_CIRCULAR, y=ys[i % nsets])
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    launches0 = plan.launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_total = reduce_max(e0.elapsed_time(e1))
+    # keep the GPU under the same load a little longer if the timed region was too short to sample
+    if sampler.nv is not None and len(sampler.samples) < 5:
+        t_end = time.perf_counter() + 0.25
+        i = 0
+        while time.perf_counter() < t_end:
+            step(i)
+            i += 1
+        torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = plan.launch_count() - launches0
+    kernel_name = plan.last_kernel()
+    ms_step = ms_total / args.steps
+    units = B2 * H2 * N2
+    value = world * units / (ms_step * 1e-3)
+    alg_bytes = 2 * units * 2 + H2 * N2 * 8                 # x read + y write (bf16) + the spectrum once
+    achieved = alg_bytes / (ms_step * 1e6)                  # GB/s
+
+    # end to end through the host-buffer entry point: pinned host x -> device -> conv -> host y
+    xh = x0.cpu().pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        M.m2_monarch_conv_fwd_host(plan, xh, kf, yh, xs[0], ys[0], M.M2_CIRCULAR)
+    barrier()
+    ms_e2e = reduce_max(time_launches(lambda i: M.m2_monarch_conv_fwd_host(plan, xh, kf, yh, xs[i % nsets], ys[i % nsets],
+                                                                           M.M2_CIRCULAR), e2e_steps, torch)) / e2e_steps
+    e2e_value = world * units / (ms_e2e * 1e-3)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": f"rotates {nsets} buffer sets of {set_bytes / 1e6:.1f} MB (> 2 x L2)",
+                   "kernel": kernel_name, "parallelism": f"dp{world} (independent rows, no collective)"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": units * 2, "d2h_bytes_per_step": units * 2,
+                "ms_per_step": ms_e2e},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                     "peak_source": peaks["source"], "algorithmic_bytes_per_launch": alg_bytes},
+    }
+    plan.close()
+    if rank == 0 and world == 1:
+        if not args.no_cpu:
+            v, cores, sample = oracle_conv_sample()
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        if not args.no_side:
+            del xs, ys
+            torch.cuda.empty_cache()
+            line["workloads"] = side_workloads(torch, M, synth, peaks, quick=args.quick)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
+    ap.add_argument("--no-side", action="store_true", help="skip the config-3 / config-4 side measurements")
+    ap.add_argument("--quick", action="store_true", help="fewer repetitions of the side measurements")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

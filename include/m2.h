@@ -1,0 +1,136 @@
+/*
+ * m2.h -- C ABI of the B200 Monarch Mixer hot-path library (libm2.so).
+ *
+ * Two operations of "Monarch Mixer" (arXiv 2310.12109) and the helpers around them:
+ *
+ *   Monarch matmul   y = P L P^T R P x                         (Sec. 3.1; Eq. 1 for order p)
+ *   Monarch conv     y = M^-1 ( (M k) (.) (M x) ),  M = F_N     (Eq. 2; App. D.3 Def. "matrix
+ *                    factored as an order-p Monarch matrix        convolution"; Alg. BlockMonarchConv;
+ *                    with twiddle diagonals                       Corollary "DFT is M", App. D.5)
+ *
+ * Conventions (App. D notation).  N = N1*N2*..*Np.  A length-N vector is indexed
+ * n = (..(n1*N2 + n2)*N3 + ..) on input (n1 most significant) and k = k1 + N1*k2 + N1*N2*k3 + ..
+ * on output (k1 least significant).  "Plan order" stores the tensor [k1][k2]..[kp] row-major.
+ * P = P_(N1,N) is the stride permutation (P x)[i] = x[sigma(i)], sigma(i) = (i mod N1)*(N/N1) + i/N1.
+ * omega_M = exp(sign * 2 pi i / M); the paper uses sign = +1.
+ *
+ * General rules.  Every function returns an m2_status (0 = OK) and never throws.  Pointers named
+ * *_dev are device pointers on the plan's device, *_host are host pointers.  The caller owns every
+ * data buffer; the library owns the plan and its device tables.  `stream` is a cudaStream_t passed
+ * as void* (NULL = the legacy default stream).  Arguments are validated on the host before
+ * anything is launched; on an error nothing has been enqueued.  The hot calls never synchronise
+ * the stream and never allocate.  All device buffers must be 16-byte aligned and contiguous.
+ */
+#ifndef M2_H_
+#define M2_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct m2_plan m2_plan;
+
+enum m2_status {
+    M2_OK = 0,
+    M2_ERR_INVALID_ARG = 1, /* null pointer, bad size, sizes inconsistent with the plan */
+    M2_ERR_UNSUPPORTED = 2, /* valid request the library has no kernel for */
+    M2_ERR_ALIGNMENT = 3,   /* a device pointer is not 16-byte aligned */
+    M2_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
+    M2_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (read via m2_last_device_status) */
+    M2_ERR_NO_DEVICE = 6    /* the plan was created host-only (device < 0) */
+};
+
+enum m2_dtype { M2_FP32 = 0, M2_BF16 = 1 };
+enum m2_conv_mode { M2_CAUSAL = 0, M2_CIRCULAR = 1 };
+enum m2_table {
+    M2_TABLE_PERM = 0,      /* sigma_(N1,N)                      (App. D notation)            */
+    M2_TABLE_PERM_INV = 1,  /* its inverse, sigma_(N/N1,N)       (P_(b,N)^T = P_(N/b,N))       */
+    M2_TABLE_DIGIT_REV = 2, /* plan position -> natural frequency k = k1 + N1 k2 + ..         */
+    M2_TABLE_TW_EXP = 16    /* M2_TABLE_TW_EXP + s, s = 1..p-1: exponent e of the twiddle
+                               omega_{N1..N_{s+1}}^e applied at plan position pos before the
+                               digit n_{s+1} is contracted: e = n_{s+1} * (k1 + N1 k2 + .. ) mod
+                               (N1..N_{s+1}), indexed by the row-major position
+                               [k1]..[k_s][n_{s+1}]..[n_p]                                     */
+};
+
+/* Creates a plan for length N = factors[0]*..*factors[p-1] (p = 2 or 3 for the convolution; the
+ * matmul uses p = 2).  dtype is the storage type of x / y (M2_FP32: float, M2_BF16: bfloat16);
+ * accumulation is always fp32.  sign = +1 (paper) or -1.  device >= 0: CUDA device ordinal, tables
+ * are uploaded (the call synchronises).  device < 0: host-only plan, usable only with
+ * m2_plan_get_table.  (Eq. 1: the factorisation N = N1..Np with block size N^(1/p); Corollary
+ * "DFT is M": the twiddles.) */
+int32_t m2_plan_create(m2_plan** out, int64_t N, int32_t p, const int32_t* factors, int32_t dtype,
+                       int32_t sign, int32_t device);
+int32_t m2_plan_destroy(m2_plan* plan);
+
+/* Copies one integer table (enum m2_table) into host_out[0..len); len must equal N. */
+int32_t m2_plan_get_table(const m2_plan* plan, int32_t which, int32_t* host_out, int64_t len);
+
+/* Bytes of the spectrum buffer m2_kernel_spectrum writes for H channels. */
+int64_t m2_spectrum_bytes(const m2_plan* plan, int64_t H);
+
+/* k_f = M * pad(k) per channel (Alg. BlockMonarchConv, the line k_f <- M k; Eq. 2's K_1 given in
+ * frequency space).  k_dev: [H, n] float32, n <= N, zero padded to N.  kf_dev: m2_spectrum_bytes
+ * bytes; the format is private to the plan (complex fp32, plan order, with the 1/N of M^-1 folded
+ * in).  Computed in fp32 whatever the plan dtype; meant to run once per weight update. */
+int32_t m2_kernel_spectrum(const m2_plan* plan, const float* k_dev, int64_t H, int64_t n, void* kf_dev,
+                           void* stream);
+
+/* Test helper: converts a spectrum buffer to natural frequency order, unnormalised (= F_N pad(k)),
+ * interleaved (re, im) float32 [H, N, 2]. */
+int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t H, float* out_dev,
+                               void* stream);
+
+/* y = Re( M^-1 ( k_f (.) M pad(x) ) )[0:n)  (Eq. 2 with M_1 = F, M_2 = F^-1; App. D.3).
+ * x_dev, y_dev: [B, H, n] in the plan dtype; kf_dev from m2_kernel_spectrum with the same H.
+ * mode M2_CAUSAL: n <= N/2, x zero padded to N, first n outputs kept (Thm 3 / App. D.3 review).
+ * mode M2_CIRCULAR: n == N. */
+int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
+                            int64_t H, int64_t n, int32_t mode, void* stream);
+
+/* Same operation from host buffers: copies x_host -> x_dev (scratch the caller provides), runs the
+ * convolution, copies y_dev -> y_host, all on `stream`; returns without synchronising.  x_host and
+ * y_host should be pinned for the copies to be asynchronous. */
+int32_t m2_monarch_conv_fwd_host(const m2_plan* plan, const void* x_host, const void* kf_dev, void* y_host,
+                                 void* x_dev_scratch, void* y_dev_scratch, int64_t B, int64_t H, int64_t n,
+                                 int32_t mode, void* stream);
+
+/* Order-2 Monarch matmul per token (Sec. 3.1, M = P L P^T R P; weight layout of the
+ * blockdiag_matmul listing, [block][out][in]):
+ *   y[t][k2*N1 + k1] = sum_{n2} L[k1][k2][n2] * sum_{n1} R[n2][k1][n1] * x[t][n1*N2 + n2].
+ * X_dev, Y_dev: [T, N] in the plan dtype; L_dev: [N1][N2][N2], R_dev: [N2][N1][N1], same dtype.
+ * R is applied first.  (The listing's parameter called L is applied first and so plays R's role.) */
+int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev,
+                          void* Y_dev, int64_t T, void* stream);
+int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const void* L_dev, const void* R_dev,
+                               void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* stream);
+
+/* M2 block forward for the M2-BERT-base shape (Eq. 2-3; Sec. 5.1): along the sequence, per channel,
+ * v = circular Monarch conv of x with the channel's kernel; gate g = depthwise conv of width 3
+ * (centred, zero padded); z = g (.) v; then the block-diagonal MLP y = bd(W_down) GELU(bd(W_up) z)
+ * with nblk blocks (exact erf GELU).  x_dev, y_dev: [B, T, C] bf16 with T == N of the plan;
+ * kf_dev: spectrum of k[C, T]; w_short_dev: [C, 3] float32; W_up_dev: [nblk, E*C/nblk, C/nblk] bf16;
+ * W_down_dev: [nblk, C/nblk, E*C/nblk] bf16; z_dev: [B, T, C] bf16 scratch that receives z. */
+int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
+                     const void* W_up_dev, const void* W_down_dev, void* z_dev, void* y_dev, int64_t B,
+                     int64_t T, int64_t C, int32_t nblk, int32_t expand, void* stream);
+
+const char* m2_status_string(int32_t status);
+
+/* Reads (synchronously) the device status word kernels set when a bounded wait expires or a
+ * self-check fails; 0 = clean.  Resets it. */
+int32_t m2_last_device_status(const m2_plan* plan, int32_t* out);
+
+/* Which implementation the last hot call on this plan dispatched to (a static string such as
+ * "conv_generic_fp32" or "conv_umma_o2"); for tests and the benchmark's report. */
+const char* m2_last_kernel_name(const m2_plan* plan);
+
+/* Number of kernels the library has launched on this plan since creation. */
+int64_t m2_launch_count(const m2_plan* plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* M2_H_ */

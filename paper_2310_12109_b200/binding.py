@@ -1,0 +1,197 @@
+"""ctypes binding of libm2.so: argument marshalling only.
+
+Function names mirror the C ABI (include/m2.h).  Tensors are torch CUDA tensors used purely as
+device memory; the current torch stream is passed as the cudaStream_t.  There is no fallback: if
+the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libm2.so")
+
+M2_FP32, M2_BF16 = 0, 1
+M2_CAUSAL, M2_CIRCULAR = 0, 1
+M2_TABLE_PERM, M2_TABLE_PERM_INV, M2_TABLE_DIGIT_REV, M2_TABLE_TW_EXP = 0, 1, 2, 16
+M2_OK, M2_ERR_INVALID_ARG, M2_ERR_UNSUPPORTED, M2_ERR_ALIGNMENT, M2_ERR_CUDA, M2_ERR_TIMEOUT, M2_ERR_NO_DEVICE = range(7)
+
+# every symbol include/m2.h declares: (name, restype, argtypes)
+_vp, _i32, _i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+SIGNATURES = {
+    "m2_plan_create": (_i32, [ctypes.POINTER(_vp), _i64, _i32, ctypes.POINTER(_i32), _i32, _i32, _i32]),
+    "m2_plan_destroy": (_i32, [_vp]),
+    "m2_plan_get_table": (_i32, [_vp, _i32, ctypes.POINTER(_i32), _i64]),
+    "m2_spectrum_bytes": (_i64, [_vp, _i64]),
+    "m2_kernel_spectrum": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp]),
+    "m2_spectrum_to_natural": (_i32, [_vp, _vp, _i64, _vp, _vp]),
+    "m2_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
+    "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
+    "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp]),
+    "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
+    "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
+    "m2_status_string": (ctypes.c_char_p, [_i32]),
+    "m2_last_device_status": (_i32, [_vp, ctypes.POINTER(_i32)]),
+    "m2_last_kernel_name": (ctypes.c_char_p, [_vp]),
+    "m2_launch_count": (_i64, [_vp]),
+}
+
+_lib = None
+
+
+class M2Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().m2_status_string(status).decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libm2.so (built by paper_2310_12109_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not built: run `python -m paper_2310_12109_b200.build`")
+        l = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != M2_OK:
+        raise M2Error(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+class Plan:
+    """m2_plan_create / m2_plan_destroy."""
+
+    def __init__(self, dims, dtype: int = M2_BF16, sign: int = +1, device: int = 0):
+        self.dims = tuple(int(d) for d in dims)
+        self.N = 1
+        for d in self.dims:
+            self.N *= d
+        self.dtype, self.sign, self.device = dtype, sign, device
+        self.handle = _vp()
+        arr = (_i32 * len(self.dims))(*self.dims)
+        _check(lib().m2_plan_create(ctypes.byref(self.handle), self.N, len(self.dims), arr, dtype, sign, device),
+               "m2_plan_create")
+
+    def close(self):
+        if self.handle:
+            lib().m2_plan_destroy(self.handle)
+            self.handle = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def torch_dtype(self):
+        return torch.bfloat16 if self.dtype == M2_BF16 else torch.float32
+
+    def get_table(self, which: int):
+        import numpy as np
+        out = (_i32 * self.N)()
+        _check(lib().m2_plan_get_table(self.handle, which, out, self.N), "m2_plan_get_table")
+        return np.frombuffer(out, dtype=np.int32).copy()
+
+    def last_kernel(self) -> str:
+        return lib().m2_last_kernel_name(self.handle).decode()
+
+    def launch_count(self) -> int:
+        return int(lib().m2_launch_count(self.handle))
+
+    def device_status(self) -> int:
+        out = _i32(0)
+        _check(lib().m2_last_device_status(self.handle, ctypes.byref(out)), "m2_last_device_status")
+        return out.value
+
+
+def m2_spectrum_bytes(plan: Plan, H: int) -> int:
+    return int(lib().m2_spectrum_bytes(plan.handle, H))
+
+
+def m2_kernel_spectrum(plan: Plan, k: torch.Tensor, kf: torch.Tensor | None = None) -> torch.Tensor:
+    """k: [H, n] float32 CUDA.  Returns the opaque spectrum buffer (uint8)."""
+    assert k.is_cuda and k.dtype == torch.float32 and k.is_contiguous() and k.dim() == 2
+    H, n = k.shape
+    if kf is None:
+        kf = torch.empty(max(m2_spectrum_bytes(plan, H), 16), dtype=torch.uint8, device=k.device)
+    _check(lib().m2_kernel_spectrum(plan.handle, _ptr(k), H, n, _ptr(kf), _stream()), "m2_kernel_spectrum")
+    return kf
+
+
+def m2_spectrum_to_natural(plan: Plan, kf: torch.Tensor, H: int) -> torch.Tensor:
+    out = torch.empty((H, plan.N, 2), dtype=torch.float32, device=kf.device)
+    _check(lib().m2_spectrum_to_natural(plan.handle, _ptr(kf), H, _ptr(out), _stream()), "m2_spectrum_to_natural")
+    return out
+
+
+def m2_monarch_conv_fwd(plan: Plan, x: torch.Tensor, kf: torch.Tensor, mode: int, y: torch.Tensor | None = None):
+    """x: [B, H, n] CUDA tensor of the plan dtype; returns y of the same shape."""
+    assert x.is_cuda and x.dtype == plan.torch_dtype and x.is_contiguous() and x.dim() == 3
+    B, H, n = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _check(lib().m2_monarch_conv_fwd(plan.handle, _ptr(x), _ptr(kf), _ptr(y), B, H, n, mode, _stream()),
+           "m2_monarch_conv_fwd")
+    return y
+
+
+def m2_monarch_conv_fwd_host(plan: Plan, x_host: torch.Tensor, kf: torch.Tensor, y_host: torch.Tensor,
+                             x_scratch: torch.Tensor, y_scratch: torch.Tensor, mode: int):
+    """x_host / y_host: pinned CPU tensors [B, H, n]; scratch: CUDA tensors of the same shape."""
+    assert not x_host.is_cuda and not y_host.is_cuda and x_scratch.is_cuda and y_scratch.is_cuda
+    B, H, n = x_host.shape
+    _check(lib().m2_monarch_conv_fwd_host(plan.handle, _ptr(x_host), _ptr(kf), _ptr(y_host), _ptr(x_scratch),
+                                          _ptr(y_scratch), B, H, n, mode, _stream()), "m2_monarch_conv_fwd_host")
+    return y_host
+
+
+def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tensor, Y: torch.Tensor | None = None):
+    """X: [T, N]; L: [N1, N2, N2]; R: [N2, N1, N1]; all CUDA, plan dtype."""
+    for t in (X, L, R):
+        assert t.is_cuda and t.dtype == plan.torch_dtype and t.is_contiguous()
+    N1, N2 = plan.dims
+    assert X.dim() == 2 and X.shape[1] == plan.N and tuple(L.shape) == (N1, N2, N2) and tuple(R.shape) == (N2, N1, N1)
+    if Y is None:
+        Y = torch.empty_like(X)
+    _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _stream()),
+           "m2_monarch_matmul")
+    return Y
+
+
+def m2_monarch_matmul_host(plan: Plan, X_host, L, R, Y_host, X_scratch, Y_scratch):
+    _check(lib().m2_monarch_matmul_host(plan.handle, _ptr(X_host), _ptr(L), _ptr(R), _ptr(Y_host), _ptr(X_scratch),
+                                        _ptr(Y_scratch), X_host.shape[0], _stream()), "m2_monarch_matmul_host")
+    return Y_host
+
+
+def m2_block_fwd(plan: Plan, x: torch.Tensor, kf: torch.Tensor, w_short: torch.Tensor, W_up: torch.Tensor,
+                 W_down: torch.Tensor, nblk: int = 4, expand: int = 4):
+    """x: [B, T, C] bf16.  Returns (y, z)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 3
+    assert w_short.dtype == torch.float32 and W_up.dtype == torch.bfloat16 and W_down.dtype == torch.bfloat16
+    B, T, C = x.shape
+    z = torch.empty_like(x)
+    y = torch.empty_like(x)
+    _check(lib().m2_block_fwd(plan.handle, _ptr(x), _ptr(kf), _ptr(w_short), _ptr(W_up), _ptr(W_down), _ptr(z), _ptr(y),
+                              B, T, C, nblk, expand, _stream()), "m2_block_fwd")
+    return y, z

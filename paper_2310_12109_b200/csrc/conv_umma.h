@@ -1,0 +1,18 @@
+// Tensor-core (tcgen05 / TMEM / TMA) Monarch convolution path (internal header).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "m2_plan.h"
+
+namespace m2u {
+
+// Builds the device constants of the tensor-core path for plans it covers (no-op otherwise).
+cudaError_t create_tables(m2_plan* plan);
+void destroy_tables(m2_plan* plan);
+
+// Returns M2_ERR_UNSUPPORTED when no tensor-core kernel covers the request (caller falls back to
+// the CUDA-core kernels), M2_OK after enqueueing, another status on failure.
+int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
+                 int32_t mode, cudaStream_t stream);
+
+}  // namespace m2u

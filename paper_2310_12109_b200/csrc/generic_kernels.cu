@@ -1,0 +1,449 @@
+// CUDA-core (fp32 FMA) kernels: the fp32 path, the kernel spectrum, and the general-shape path for
+// sizes the tensor-core kernels do not cover.  One thread block owns one (batch, channel) row and
+// keeps it in shared memory from the load to the store; every Monarch stage is an in-place
+// contraction of one index digit (the stride permutations of M = P L P^T R P only decide which
+// digit a stage contracts, so they are address arithmetic here, never a data movement pass).
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "generic_kernels.h"
+
+namespace m2g {
+
+struct Dims {
+    int p;
+    int d[3];
+    int N;
+    float sgn;  // +1 / -1: omega = exp(sgn 2 pi i / M)
+};
+
+__device__ __forceinline__ float2 cmul(float2 a, float2 b) {
+    return make_float2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x);
+}
+
+// storage traits: complex value kept as float2 or as a bf16 pair
+template <typename ST>
+struct Store;
+template <>
+struct Store<float2> {
+    static __device__ __forceinline__ float2 ld(const float2* p) { return *p; }
+    static __device__ __forceinline__ void st(float2* p, float2 v) { *p = v; }
+};
+template <>
+struct Store<__nv_bfloat162> {
+    static __device__ __forceinline__ float2 ld(const __nv_bfloat162* p) { return __bfloat1622float2(*p); }
+    static __device__ __forceinline__ void st(__nv_bfloat162* p, float2 v) { *p = __float22bfloat162_rn(v); }
+};
+
+template <typename T>
+__device__ __forceinline__ float to_f32(T v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T>
+__device__ __forceinline__ T from_f32(float v);
+template <>
+__device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// omega_M^e with e already reduced to [0, M)
+__device__ __forceinline__ float2 twiddle(int e, int M, float sgn) {
+    float s, c;
+    sincospif(2.0f * (float)e / (float)M, &s, &c);
+    return make_float2(c, sgn * s);
+}
+
+// One Monarch-DFT stage, in place on buf (plan-position layout [d0][d1][d2]).
+//   forward (INV = false), stage a: contract n_a with F_{Na} (Corollary "DFT is M": block = F times the
+//     twiddle diagonal); the twiddle of the NEXT stage is applied to the outputs so every element
+//     costs one sincos:  out[k_a] = tw_{a+1}(n_{a+1}, kappa + Mprev k_a) * sum_{n_a} w^{k_a n_a} buf[n_a]
+//   inverse (INV = true), stage a: out[n_a] = conj(tw_a(n_a, kappa)) * sum_{k_a} conj(w^{k_a n_a}) buf[k_a]
+// The N outputs of a stage are produced in chunks of blockDim * ITEMS; a chunk is always a union of
+// whole fibers, so its writes cannot disturb the inputs of another chunk.  Within a chunk every
+// thread first computes its outputs into registers, then the block synchronises, then writes.
+template <typename ST, int ITEMS, bool INV>
+__device__ __forceinline__ void stage(ST* buf, const Dims& D, int a, const float2* __restrict__ roots) {
+    const int Na = D.d[a];
+    int sa = 1;
+    for (int j = a + 1; j < D.p; ++j) sa *= D.d[j];
+    int Mprev = 1;
+    for (int j = 0; j < a; ++j) Mprev *= D.d[j];
+    const int Mcur = Mprev * Na;
+    const int G = blockDim.x * ITEMS;          // outputs per chunk (G >= N: a single chunk)
+    const int F = G / Na;                      // fibers per chunk when G < N
+    const int nchunks = (D.N + G - 1) / G;
+    for (int c = 0; c < nchunks; ++c) {
+        float2 acc[ITEMS];
+        int pos[ITEMS];
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it) {
+            const int i = threadIdx.x + it * blockDim.x;
+            int o;
+            if (nchunks == 1 || sa < F) {
+                o = c * G + i;
+            } else {
+                const int per_hi = sa / F;     // chunks per value of hi
+                o = (c / per_hi) * Na * sa + (i / F) * sa + (c % per_hi) * F + (i % F);
+            }
+            pos[it] = o;
+            acc[it] = make_float2(0.f, 0.f);
+            if (o < D.N) {
+                const int lo = o % sa;
+                const int oa = (o / sa) % Na;
+                const int hi = o / (sa * Na);
+                const ST* fib = buf + hi * Na * sa + lo;
+                float2 s = make_float2(0.f, 0.f);
+                for (int j = 0; j < Na; ++j) {
+                    float2 w = roots[(oa * j) % Na];
+                    if (INV) w.y = -w.y;
+                    const float2 v = Store<ST>::ld(fib + j * sa);
+                    s.x = fmaf(w.x, v.x, s.x);
+                    s.x = fmaf(-w.y, v.y, s.x);
+                    s.y = fmaf(w.x, v.y, s.y);
+                    s.y = fmaf(w.y, v.x, s.y);
+                }
+                if (!INV) {
+                    if (a + 1 < D.p) {
+                        // hi is empty (a = 0) or the single digit k_1 (a = 1)
+                        const int kappa = hi + Mprev * oa;
+                        const int Nn = D.d[a + 1];
+                        const int nn = lo / (sa / Nn);
+                        const int Mn = Mcur * Nn;
+                        const int e = (int)(((long long)nn * kappa) % Mn);
+                        s = cmul(s, twiddle(e, Mn, D.sgn));
+                    }
+                } else if (a > 0) {
+                    int kappa;
+                    if (a == 1) kappa = hi;
+                    else kappa = hi / D.d[1] + D.d[0] * (hi % D.d[1]);  // a = 2: hi = k_1 * N_2 + k_2
+                    const int e = (int)(((long long)oa * kappa) % Mcur);
+                    s = cmul(s, twiddle(e, Mcur, -D.sgn));
+                }
+                acc[it] = s;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it)
+            if (pos[it] < D.N) Store<ST>::st(buf + pos[it], acc[it]);
+        __syncthreads();
+    }
+}
+
+struct Roots {
+    const float2* r[3];
+};
+
+// Fused Monarch convolution for one row per block (Eq. 2 / Alg. BlockMonarchConv with M = F_N):
+// load + zero pad, forward stages, spectrum multiply (plan order on both sides, so no permutation),
+// inverse stages, real part, truncate, store.  Strides let the same kernel read a [B, T, C] tensor
+// along T (the M2 block) -- then gate_w != nullptr adds the width-3 depthwise gate before the store.
+template <typename IO, typename ST, int ITEMS>
+__global__ void __launch_bounds__(1024) conv_row_kernel(const IO* __restrict__ x, const float2* __restrict__ kf, IO* __restrict__ y, Dims D,
+                                Roots R, int H, int n, long long row_stride_b, long long row_stride_h,
+                                long long elem_stride, const float* __restrict__ gate_w) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ST* buf = reinterpret_cast<ST*>(smem_raw);
+    const int row = blockIdx.x;
+    const int h = row % H;
+    const int b = row / H;
+    const IO* xr = x + b * row_stride_b + h * row_stride_h;
+    IO* yr = y + b * row_stride_b + h * row_stride_h;
+    for (int i = threadIdx.x; i < D.N; i += blockDim.x) {
+        float v = (i < n) ? to_f32<IO>(xr[(long long)i * elem_stride]) : 0.f;
+        Store<ST>::st(buf + i, make_float2(v, 0.f));
+    }
+    __syncthreads();
+    for (int a = 0; a < D.p; ++a) stage<ST, ITEMS, false>(buf, D, a, R.r[a]);
+    const float2* kr = kf + (long long)h * D.N;
+    for (int i = threadIdx.x; i < D.N; i += blockDim.x) Store<ST>::st(buf + i, cmul(Store<ST>::ld(buf + i), kr[i]));
+    __syncthreads();
+    for (int a = D.p - 1; a >= 0; --a) stage<ST, ITEMS, true>(buf, D, a, R.r[a]);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        float v = Store<ST>::ld(buf + i).x;
+        if (gate_w != nullptr) {
+            const float w0 = gate_w[h * 3 + 0], w1 = gate_w[h * 3 + 1], w2 = gate_w[h * 3 + 2];
+            float g = w1 * to_f32<IO>(xr[(long long)i * elem_stride]);
+            if (i > 0) g = fmaf(w0, to_f32<IO>(xr[(long long)(i - 1) * elem_stride]), g);
+            if (i + 1 < n) g = fmaf(w2, to_f32<IO>(xr[(long long)(i + 1) * elem_stride]), g);
+            v *= g;
+        }
+        yr[(long long)i * elem_stride] = from_f32<IO>(v);
+    }
+}
+
+// k_f = F_N pad(k) / N per channel, in plan order, computed in place in the output buffer (global
+// memory, one block per channel): runs once per weight update, not on the hot path.
+template <int ITEMS>
+__global__ void __launch_bounds__(1024) spectrum_kernel(const float* __restrict__ k, float2* __restrict__ kf, Dims D, Roots R, int n) {
+    const int h = blockIdx.x;
+    float2* buf = kf + (long long)h * D.N;
+    for (int i = threadIdx.x; i < D.N; i += blockDim.x)
+        buf[i] = make_float2(i < n ? k[(long long)h * n + i] : 0.f, 0.f);
+    __syncthreads();
+    for (int a = 0; a < D.p; ++a) stage<float2, ITEMS, false>(buf, D, a, R.r[a]);
+    const float inv = 1.0f / (float)D.N;
+    for (int i = threadIdx.x; i < D.N; i += blockDim.x) {
+        float2 v = buf[i];
+        buf[i] = make_float2(v.x * inv, v.y * inv);
+    }
+}
+
+__global__ void spectrum_to_natural_kernel(const float2* __restrict__ kf, float2* __restrict__ out, Dims D, long long total) {
+    long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int pos = (int)(i % D.N);
+    const long long h = i / D.N;
+    // plan position (k1, k2, k3) row-major -> k = k1 + N1 k2 + N1 N2 k3
+    int rem = pos, k = 0;
+    int digits[3] = {0, 0, 0};
+    for (int a = D.p - 1; a >= 0; --a) {
+        digits[a] = rem % D.d[a];
+        rem /= D.d[a];
+    }
+    int w = 1;
+    for (int a = 0; a < D.p; ++a) {
+        k += w * digits[a];
+        w *= D.d[a];
+    }
+    float2 v = kf[i];
+    out[h * D.N + k] = make_float2(v.x * (float)D.N, v.y * (float)D.N);
+}
+
+// Order-2 Monarch matmul, TT tokens per block, fp32 accumulate (Sec. 3.1):
+//   z[n2][k1] = sum_{n1} R[n2][k1][n1] x[n1*N2 + n2];  y[k2*N1 + k1] = sum_{n2} L[k1][k2][n2] z[n2][k1]
+template <typename IO, int TT>
+__global__ void matmul_tokens_kernel(const IO* __restrict__ X, const IO* __restrict__ L, const IO* __restrict__ Rw,
+                                     IO* __restrict__ Y, int N1, int N2, long long T) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int N = N1 * N2;
+    float* xs = reinterpret_cast<float*>(smem_raw);  // [TT][N]
+    float* zs = xs + TT * N;                          // [TT][N], index n2*N1 + k1
+    const long long t0 = (long long)blockIdx.x * TT;
+    for (int i = threadIdx.x; i < TT * N; i += blockDim.x) {
+        const long long t = t0 + i / N;
+        xs[i] = (t < T) ? to_f32<IO>(X[t * N + (i % N)]) : 0.f;
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < N; o += blockDim.x) {
+        const int k1 = o % N1, n2 = o / N1;
+        const IO* w = Rw + ((long long)n2 * N1 + k1) * N1;
+        float acc[TT];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) acc[t] = 0.f;
+        for (int n1 = 0; n1 < N1; ++n1) {
+            const float wv = to_f32<IO>(w[n1]);
+#pragma unroll
+            for (int t = 0; t < TT; ++t) acc[t] = fmaf(wv, xs[t * N + n1 * N2 + n2], acc[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t) zs[t * N + o] = acc[t];
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < N; o += blockDim.x) {
+        const int k1 = o % N1, k2 = o / N1;
+        const IO* w = L + ((long long)k1 * N2 + k2) * N2;
+        float acc[TT];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) acc[t] = 0.f;
+        for (int n2 = 0; n2 < N2; ++n2) {
+            const float wv = to_f32<IO>(w[n2]);
+#pragma unroll
+            for (int t = 0; t < TT; ++t) acc[t] = fmaf(wv, zs[t * N + n2 * N1 + k1], acc[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t)
+            if (t0 + t < T) Y[(t0 + t) * N + o] = from_f32<IO>(acc[t]);
+    }
+}
+
+// Block-diagonal MLP with GELU (Eq. 3 with block-diagonal M_3, M_4): per (token tile, block)
+//   hid = GELU(W_up[j] z_j),  y_j = W_down[j] hid.   The hidden activations never leave the SM.
+template <int TT>
+__global__ void mlp_blockdiag_kernel(const __nv_bfloat16* __restrict__ z, const __nv_bfloat16* __restrict__ Wup,
+                                     const __nv_bfloat16* __restrict__ Wdn, __nv_bfloat16* __restrict__ y, int C,
+                                     int nblk, int expand, long long tokens) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int ci = C / nblk, hi = expand * ci;
+    float* zs = reinterpret_cast<float*>(smem_raw);  // [TT][ci]
+    float* hs = zs + TT * ci;                         // [TT][hi]
+    const int j = blockIdx.y;
+    const long long t0 = (long long)blockIdx.x * TT;
+    for (int i = threadIdx.x; i < TT * ci; i += blockDim.x) {
+        const long long t = t0 + i / ci;
+        zs[i] = (t < tokens) ? __bfloat162float(z[t * C + j * ci + (i % ci)]) : 0.f;
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < hi; o += blockDim.x) {
+        const __nv_bfloat16* w = Wup + ((long long)j * hi + o) * ci;
+        float acc[TT];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) acc[t] = 0.f;
+        for (int i = 0; i < ci; ++i) {
+            const float wv = __bfloat162float(w[i]);
+#pragma unroll
+            for (int t = 0; t < TT; ++t) acc[t] = fmaf(wv, zs[t * ci + i], acc[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t) {
+            const float v = acc[t];
+            hs[t * hi + o] = 0.5f * v * (1.0f + erff(v * 0.70710678118654752f));
+        }
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < ci; o += blockDim.x) {
+        const __nv_bfloat16* w = Wdn + ((long long)j * ci + o) * hi;
+        float acc[TT];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) acc[t] = 0.f;
+        for (int i = 0; i < hi; ++i) {
+            const float wv = __bfloat162float(w[i]);
+#pragma unroll
+            for (int t = 0; t < TT; ++t) acc[t] = fmaf(wv, hs[t * hi + i], acc[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t)
+            if (t0 + t < tokens) y[(t0 + t) * C + j * ci + o] = __float2bfloat16_rn(acc[t]);
+    }
+}
+
+static Dims make_dims(const ConvShape& s) {
+    Dims D;
+    D.p = s.p;
+    D.N = 1;
+    for (int a = 0; a < 3; ++a) {
+        D.d[a] = a < s.p ? s.dims[a] : 1;
+        D.N *= D.d[a];
+    }
+    D.sgn = s.sign >= 0 ? 1.f : -1.f;
+    return D;
+}
+
+// items per thread and block size.  Small or odd N: one output per thread.  N <= 2048: two.
+// Larger N: 1024 threads x 4 outputs per chunk; then every dimension must be a power of two and N a
+// multiple of 4096 so that chunks are unions of whole fibers.
+static bool pick_launch(const Dims& D, int& items, int& threads) {
+    const int N = D.N;
+    if (N % 2 != 0 || N < 128) {
+        items = 1;
+        threads = N;
+        return N >= 1 && N <= 1024;
+    }
+    if (N <= 2048) {
+        items = 2;
+        threads = N / 2;
+        return true;
+    }
+    items = 4;
+    threads = 1024;
+    if (N % 4096 != 0) return false;
+    for (int a = 0; a < D.p; ++a)
+        if ((D.d[a] & (D.d[a] - 1)) != 0 || D.d[a] > 4096) return false;
+    return true;
+}
+
+template <typename IO, typename ST>
+static cudaError_t launch_conv_t(const ConvShape& s, const void* x, const void* kf, void* y, const float* gate_w,
+                                 cudaStream_t st) {
+    Dims D = make_dims(s);
+    Roots R{{s.roots[0], s.roots[1], s.roots[2]}};
+    int items, threads;
+    if (!pick_launch(D, items, threads)) return cudaErrorInvalidValue;
+    const size_t smem = (size_t)D.N * sizeof(ST);
+    const long long rows = (long long)s.B * s.H;
+    if (rows == 0) return cudaSuccess;
+#define M2_LAUNCH_CONV(IT)                                                                                         \
+    {                                                                                                              \
+        auto kern = conv_row_kernel<IO, ST, IT>;                                                                   \
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
+        if (e != cudaSuccess) return e;                                                                            \
+        kern<<<(unsigned)rows, threads, smem, st>>>((const IO*)x, (const float2*)kf, (IO*)y, D, R, (int)s.H,       \
+                                                    (int)s.n, s.stride_b, s.stride_h, s.stride_e, gate_w);         \
+    }
+    switch (items) {
+        case 1: M2_LAUNCH_CONV(1) break;
+        case 2: M2_LAUNCH_CONV(2) break;
+        case 4: M2_LAUNCH_CONV(4) break;
+        default: return cudaErrorInvalidValue;
+    }
+#undef M2_LAUNCH_CONV
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv(const ConvShape& s, bool bf16_io, const void* x, const void* kf, void* y, const float* gate_w,
+                        cudaStream_t st) {
+    long long N = 1;
+    for (int a = 0; a < s.p; ++a) N *= s.dims[a];
+    if (!bf16_io) {
+        if (N * 8 > 200 * 1024) return cudaErrorInvalidValue;
+        return launch_conv_t<float, float2>(s, x, kf, y, gate_w, st);
+    }
+    if (N * 8 <= 160 * 1024) return launch_conv_t<__nv_bfloat16, float2>(s, x, kf, y, gate_w, st);
+    if (N * 4 > 200 * 1024) return cudaErrorInvalidValue;
+    return launch_conv_t<__nv_bfloat16, __nv_bfloat162>(s, x, kf, y, gate_w, st);
+}
+
+cudaError_t launch_spectrum(const ConvShape& s, const float* k, void* kf, cudaStream_t st) {
+    Dims D = make_dims(s);
+    Roots R{{s.roots[0], s.roots[1], s.roots[2]}};
+    int items, threads;
+    if (!pick_launch(D, items, threads)) return cudaErrorInvalidValue;
+    if (s.H == 0) return cudaSuccess;
+    switch (items) {
+        case 1: spectrum_kernel<1><<<(unsigned)s.H, threads, 0, st>>>(k, (float2*)kf, D, R, (int)s.n); break;
+        case 2: spectrum_kernel<2><<<(unsigned)s.H, threads, 0, st>>>(k, (float2*)kf, D, R, (int)s.n); break;
+        case 4: spectrum_kernel<4><<<(unsigned)s.H, threads, 0, st>>>(k, (float2*)kf, D, R, (int)s.n); break;
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_spectrum_to_natural(const ConvShape& s, const void* kf, float* out, cudaStream_t st) {
+    Dims D = make_dims(s);
+    const long long total = (long long)s.H * D.N;
+    if (total == 0) return cudaSuccess;
+    spectrum_to_natural_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const float2*)kf, (float2*)out, D, total);
+    return cudaGetLastError();
+}
+
+template <typename IO>
+static cudaError_t launch_matmul_t(int N1, int N2, long long T, const void* X, const void* L, const void* R, void* Y,
+                                   cudaStream_t st) {
+    constexpr int TT = 4;
+    const int N = N1 * N2;
+    const size_t smem = (size_t)2 * TT * N * sizeof(float);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    if (T == 0) return cudaSuccess;
+    auto kern = matmul_tokens_kernel<IO, TT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int threads = N < 512 ? ((N + 31) / 32) * 32 : 512;
+    kern<<<(unsigned)((T + TT - 1) / TT), threads, smem, st>>>((const IO*)X, (const IO*)L, (const IO*)R, (IO*)Y, N1, N2, T);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void* X, const void* L, const void* R, void* Y,
+                          cudaStream_t st) {
+    return bf16_io ? launch_matmul_t<__nv_bfloat16>(N1, N2, T, X, L, R, Y, st)
+                   : launch_matmul_t<float>(N1, N2, T, X, L, R, Y, st);
+}
+
+cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,
+                       long long tokens, cudaStream_t st) {
+    constexpr int TT = 8;
+    const int ci = C / nblk, hi = expand * ci;
+    const size_t smem = (size_t)TT * (ci + hi) * sizeof(float);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    if (tokens == 0) return cudaSuccess;
+    auto kern = mlp_blockdiag_kernel<TT>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid((unsigned)((tokens + TT - 1) / TT), (unsigned)nblk);
+    kern<<<grid, 256, smem, st>>>((const __nv_bfloat16*)z, (const __nv_bfloat16*)Wup, (const __nv_bfloat16*)Wdn,
+                                  (__nv_bfloat16*)y, C, nblk, expand, tokens);
+    return cudaGetLastError();
+}
+
+}  // namespace m2g

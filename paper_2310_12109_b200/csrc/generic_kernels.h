@@ -1,0 +1,26 @@
+// Launch wrappers of the CUDA-core kernels (internal header).
+#pragma once
+#include <cuda_runtime.h>
+
+namespace m2g {
+
+struct ConvShape {
+    int p;
+    int dims[3];
+    int sign;
+    long long B, H, n;
+    // element (b, h, i) of x / y lives at b*stride_b + h*stride_h + i*stride_e
+    long long stride_b, stride_h, stride_e;
+    const float2* roots[3];  // device: omega_{Na}^j per stage
+};
+
+cudaError_t launch_conv(const ConvShape& s, bool bf16_io, const void* x, const void* kf, void* y, const float* gate_w,
+                        cudaStream_t st);
+cudaError_t launch_spectrum(const ConvShape& s, const float* k, void* kf, cudaStream_t st);
+cudaError_t launch_spectrum_to_natural(const ConvShape& s, const void* kf, float* out, cudaStream_t st);
+cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void* X, const void* L, const void* R, void* Y,
+                          cudaStream_t st);
+cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,
+                       long long tokens, cudaStream_t st);
+
+}  // namespace m2g

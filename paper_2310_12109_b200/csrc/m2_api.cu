@@ -1,0 +1,366 @@
+// C ABI of libm2: plan management, host-side validation, dispatch to the kernels.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "conv_umma.h"
+#include "generic_kernels.h"
+#include "m2_plan.h"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
+        if (ok && prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+void build_tables(m2_plan* pl) {
+    const int64_t N = pl->N;
+    const int p = pl->p;
+    const int64_t N1 = pl->dims[0];
+    m2_fill_stride_perm(N1, N, pl->perm);
+    m2_fill_stride_perm(N / N1, N, pl->perm_inv);
+    // plan position [k1][k2]..[kp] row-major -> k = k1 + N1 k2 + ..
+    pl->digit_rev.resize(N);
+    for (int64_t pos = 0; pos < N; ++pos) {
+        int64_t rem = pos, k = 0;
+        int64_t digit[4];
+        for (int a = p - 1; a >= 0; --a) {
+            digit[a] = rem % pl->dims[a];
+            rem /= pl->dims[a];
+        }
+        int64_t w = 1;
+        for (int a = 0; a < p; ++a) {
+            k += w * digit[a];
+            w *= pl->dims[a];
+        }
+        pl->digit_rev[pos] = (int32_t)k;
+    }
+    // twiddle exponents: before digit n_{s+1} is contracted (s = 1..p-1) the element at position
+    // [k1]..[ks][n_{s+1}]..[np] is scaled by omega_{N1..N_{s+1}}^{ n_{s+1} * (k1 + N1 k2 + ..) }
+    pl->tw_exp.assign(p > 1 ? p - 1 : 0, std::vector<int32_t>());
+    for (int s = 1; s < p; ++s) {
+        std::vector<int32_t>& t = pl->tw_exp[s - 1];
+        t.resize(N);
+        int64_t Mcur = 1;
+        for (int a = 0; a <= s; ++a) Mcur *= pl->dims[a];
+        for (int64_t pos = 0; pos < N; ++pos) {
+            int64_t rem = pos;
+            int64_t digit[4];
+            for (int a = p - 1; a >= 0; --a) {
+                digit[a] = rem % pl->dims[a];
+                rem /= pl->dims[a];
+            }
+            int64_t kappa = 0, w = 1;
+            for (int a = 0; a < s; ++a) {
+                kappa += w * digit[a];
+                w *= pl->dims[a];
+            }
+            t[pos] = (int32_t)((digit[s] * kappa) % Mcur);
+        }
+    }
+}
+
+m2g::ConvShape conv_shape(const m2_plan* pl, int64_t B, int64_t H, int64_t n) {
+    m2g::ConvShape s;
+    s.p = pl->p;
+    for (int a = 0; a < 3; ++a) {
+        s.dims[a] = a < pl->p ? pl->dims[a] : 1;
+        s.roots[a] = a < pl->p ? pl->d_roots[a] : nullptr;
+    }
+    s.sign = pl->sign;
+    s.B = B;
+    s.H = H;
+    s.n = n;
+    s.stride_b = H * n;
+    s.stride_h = n;
+    s.stride_e = 1;
+    return s;
+}
+
+int32_t check_conv_args(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
+                        int32_t mode) {
+    if (!plan) return M2_ERR_INVALID_ARG;
+    if (B < 0 || H < 0 || n <= 0) return M2_ERR_INVALID_ARG;
+    if ((!x || !kf || !y) && B * H != 0) return M2_ERR_INVALID_ARG;  // empty batches may carry null pointers
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (mode == M2_CAUSAL) {
+        if (2 * n > plan->N) return M2_ERR_INVALID_ARG;
+    } else if (mode == M2_CIRCULAR) {
+        if (n != plan->N) return M2_ERR_INVALID_ARG;
+    } else {
+        return M2_ERR_INVALID_ARG;
+    }
+    if (plan->p < 2 || plan->p > 3) return M2_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(kf) || !aligned16(y)) return M2_ERR_ALIGNMENT;
+    if (B * H > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    return M2_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t m2_plan_create(m2_plan** out, int64_t N, int32_t p, const int32_t* factors, int32_t dtype, int32_t sign,
+                       int32_t device) {
+    if (!out) return M2_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!factors || p < 1 || p > 3 || N <= 0 || N > (1 << 24)) return M2_ERR_INVALID_ARG;
+    if (dtype != M2_FP32 && dtype != M2_BF16) return M2_ERR_INVALID_ARG;
+    if (sign != 1 && sign != -1) return M2_ERR_INVALID_ARG;
+    int64_t prod = 1;
+    for (int a = 0; a < p; ++a) {
+        if (factors[a] <= 0) return M2_ERR_INVALID_ARG;
+        prod *= factors[a];
+    }
+    if (prod != N) return M2_ERR_INVALID_ARG;
+    m2_plan* pl = new (std::nothrow) m2_plan();
+    if (!pl) return M2_ERR_INVALID_ARG;
+    pl->N = N;
+    pl->p = p;
+    for (int a = 0; a < p; ++a) pl->dims[a] = factors[a];
+    pl->dtype = dtype;
+    pl->sign = sign;
+    pl->device = device;
+    build_tables(pl);
+    if (device >= 0) {
+        DeviceGuard g(device);
+        bool ok = g.ok;
+        if (ok) ok = cudaMalloc(&pl->d_status, sizeof(int32_t)) == cudaSuccess;
+        if (ok) ok = cudaMemset(pl->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+        for (int a = 0; a < p && ok; ++a) {
+            const int Na = pl->dims[a];
+            std::vector<float2> r(Na);
+            for (int j = 0; j < Na; ++j) {
+                const double ang = 2.0 * M_PI * (double)j / (double)Na;
+                r[j] = make_float2((float)std::cos(ang), (float)(sign * std::sin(ang)));
+            }
+            ok = cudaMalloc(&pl->d_roots[a], sizeof(float2) * Na) == cudaSuccess &&
+                 cudaMemcpy(pl->d_roots[a], r.data(), sizeof(float2) * Na, cudaMemcpyHostToDevice) == cudaSuccess;
+        }
+        if (ok) ok = m2u::create_tables(pl) == cudaSuccess;
+        if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            m2_plan_destroy(pl);
+            return M2_ERR_CUDA;
+        }
+    }
+    *out = pl;
+    return M2_OK;
+}
+
+int32_t m2_plan_destroy(m2_plan* plan) {
+    if (!plan) return M2_ERR_INVALID_ARG;
+    if (plan->device >= 0) {
+        DeviceGuard g(plan->device);
+        cudaDeviceSynchronize();
+        m2u::destroy_tables(plan);
+        if (plan->d_status) cudaFree(plan->d_status);
+        for (int a = 0; a < 4; ++a)
+            if (plan->d_roots[a]) cudaFree(plan->d_roots[a]);
+    }
+    delete plan;
+    return M2_OK;
+}
+
+int32_t m2_plan_get_table(const m2_plan* plan, int32_t which, int32_t* host_out, int64_t len) {
+    if (!plan || !host_out || len != plan->N) return M2_ERR_INVALID_ARG;
+    const std::vector<int32_t>* src = nullptr;
+    if (which == M2_TABLE_PERM) src = &plan->perm;
+    else if (which == M2_TABLE_PERM_INV) src = &plan->perm_inv;
+    else if (which == M2_TABLE_DIGIT_REV) src = &plan->digit_rev;
+    else if (which > M2_TABLE_TW_EXP && which < M2_TABLE_TW_EXP + plan->p) src = &plan->tw_exp[which - M2_TABLE_TW_EXP - 1];
+    if (!src) return M2_ERR_INVALID_ARG;
+    std::memcpy(host_out, src->data(), sizeof(int32_t) * (size_t)len);
+    return M2_OK;
+}
+
+int64_t m2_spectrum_bytes(const m2_plan* plan, int64_t H) {
+    if (!plan || H < 0) return -1;
+    return H * plan->N * (int64_t)sizeof(float2);
+}
+
+int32_t m2_kernel_spectrum(const m2_plan* plan, const float* k_dev, int64_t H, int64_t n, void* kf_dev, void* stream) {
+    if (!plan || !k_dev || !kf_dev) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (H < 0 || n <= 0 || n > plan->N) return M2_ERR_INVALID_ARG;
+    if (plan->p < 2 || plan->p > 3) return M2_ERR_UNSUPPORTED;
+    if (!aligned16(kf_dev)) return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    m2g::ConvShape s = conv_shape(plan, 1, H, n);
+    cudaError_t e = m2g::launch_spectrum(s, k_dev, kf_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "spectrum_generic_fp32";
+    plan->launches += (H > 0);
+    return M2_OK;
+}
+
+int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t H, float* out_dev, void* stream) {
+    if (!plan || !kf_dev || !out_dev || H < 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    m2g::ConvShape s = conv_shape(plan, 1, H, plan->N);
+    if (m2g::launch_spectrum_to_natural(s, kf_dev, out_dev, (cudaStream_t)stream) != cudaSuccess) return M2_ERR_CUDA;
+    plan->launches += (H > 0);
+    return M2_OK;
+}
+
+int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
+                            int64_t H, int64_t n, int32_t mode, void* stream) {
+    int32_t st = check_conv_args(plan, x_dev, kf_dev, y_dev, B, H, n, mode);
+    if (st != M2_OK) return st;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (B * H == 0) return M2_OK;
+    // tensor-core path where a kernel exists for the shape, CUDA-core path otherwise
+    int32_t ust = m2u::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
+    if (ust == M2_OK) return M2_OK;
+    if (ust != M2_ERR_UNSUPPORTED) return ust;
+    m2g::ConvShape s = conv_shape(plan, B, H, n);
+    cudaError_t e = m2g::launch_conv(s, plan->dtype == M2_BF16, x_dev, kf_dev, y_dev, nullptr, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = plan->dtype == M2_BF16 ? "conv_generic_bf16io" : "conv_generic_fp32";
+    plan->launches += 1;
+    return M2_OK;
+}
+
+int32_t m2_monarch_conv_fwd_host(const m2_plan* plan, const void* x_host, const void* kf_dev, void* y_host,
+                                 void* x_dev_scratch, void* y_dev_scratch, int64_t B, int64_t H, int64_t n, int32_t mode,
+                                 void* stream) {
+    if (!x_host || !y_host) return M2_ERR_INVALID_ARG;
+    int32_t st = check_conv_args(plan, x_dev_scratch, kf_dev, y_dev_scratch, B, H, n, mode);
+    if (st != M2_OK) return st;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    const size_t bytes = (size_t)B * H * n * (plan->dtype == M2_BF16 ? 2 : 4);
+    if (bytes == 0) return M2_OK;
+    if (cudaMemcpyAsync(x_dev_scratch, x_host, bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess)
+        return M2_ERR_CUDA;
+    st = m2_monarch_conv_fwd(plan, x_dev_scratch, kf_dev, y_dev_scratch, B, H, n, mode, stream);
+    if (st != M2_OK) return st;
+    if (cudaMemcpyAsync(y_host, y_dev_scratch, bytes, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+        return M2_ERR_CUDA;
+    return M2_OK;
+}
+
+static int32_t check_matmul_args(const m2_plan* plan, const void* X, const void* L, const void* R, void* Y, int64_t T) {
+    if (!plan || T < 0) return M2_ERR_INVALID_ARG;
+    if ((!X || !L || !R || !Y) && T != 0) return M2_ERR_INVALID_ARG;  // an empty batch may carry null pointers
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (plan->p != 2) return M2_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(L) || !aligned16(R) || !aligned16(Y)) return M2_ERR_ALIGNMENT;
+    if (T > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    return M2_OK;
+}
+
+int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, void* Y_dev,
+                          int64_t T, void* stream) {
+    int32_t st = check_matmul_args(plan, X_dev, L_dev, R_dev, Y_dev, T);
+    if (st != M2_OK) return st;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (T == 0) return M2_OK;
+    cudaError_t e = m2g::launch_matmul(plan->dims[0], plan->dims[1], T, plan->dtype == M2_BF16, X_dev, L_dev, R_dev,
+                                       Y_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "matmul_generic";
+    plan->launches += 1;
+    return M2_OK;
+}
+
+int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const void* L_dev, const void* R_dev,
+                               void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* stream) {
+    if (!X_host || !Y_host) return M2_ERR_INVALID_ARG;
+    int32_t st = check_matmul_args(plan, X_dev_scratch, L_dev, R_dev, Y_dev_scratch, T);
+    if (st != M2_OK) return st;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    const size_t bytes = (size_t)T * plan->N * (plan->dtype == M2_BF16 ? 2 : 4);
+    if (bytes == 0) return M2_OK;
+    if (cudaMemcpyAsync(X_dev_scratch, X_host, bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess)
+        return M2_ERR_CUDA;
+    st = m2_monarch_matmul(plan, X_dev_scratch, L_dev, R_dev, Y_dev_scratch, T, stream);
+    if (st != M2_OK) return st;
+    if (cudaMemcpyAsync(Y_host, Y_dev_scratch, bytes, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+        return M2_ERR_CUDA;
+    return M2_OK;
+}
+
+int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
+                     const void* W_up_dev, const void* W_down_dev, void* z_dev, void* y_dev, int64_t B, int64_t T,
+                     int64_t C, int32_t nblk, int32_t expand, void* stream) {
+    if (!plan || !x_dev || !kf_dev || !w_short_dev || !W_up_dev || !W_down_dev || !z_dev || !y_dev)
+        return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (B < 0 || C <= 0 || nblk <= 0 || expand <= 0 || C % nblk != 0 || T != plan->N) return M2_ERR_INVALID_ARG;
+    if (plan->dtype != M2_BF16 || plan->p < 2 || plan->p > 3) return M2_ERR_UNSUPPORTED;
+    if (!aligned16(x_dev) || !aligned16(kf_dev) || !aligned16(W_up_dev) || !aligned16(W_down_dev) || !aligned16(z_dev) ||
+        !aligned16(y_dev))
+        return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (B == 0) return M2_OK;
+    // sequence mix + gate: rows are (b, c), elements strided by C along the sequence
+    m2g::ConvShape s = conv_shape(plan, B, C, T);
+    s.stride_b = T * C;
+    s.stride_h = 1;
+    s.stride_e = C;
+    cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z_dev, w_short_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    e = m2g::launch_mlp(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "block_generic";
+    plan->launches += 2;
+    return M2_OK;
+}
+
+const char* m2_status_string(int32_t status) {
+    switch (status) {
+        case M2_OK: return "ok";
+        case M2_ERR_INVALID_ARG: return "invalid argument";
+        case M2_ERR_UNSUPPORTED: return "unsupported shape or type";
+        case M2_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+        case M2_ERR_CUDA: return "CUDA call failed";
+        case M2_ERR_TIMEOUT: return "device-side wait timed out";
+        case M2_ERR_NO_DEVICE: return "plan has no device";
+        default: return "unknown status";
+    }
+}
+
+int32_t m2_last_device_status(const m2_plan* plan, int32_t* out) {
+    if (!plan || !out) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return M2_ERR_CUDA;
+    if (cudaMemcpy(out, plan->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return M2_ERR_CUDA;
+    if (cudaMemset(plan->d_status, 0, sizeof(int32_t)) != cudaSuccess) return M2_ERR_CUDA;
+    return M2_OK;
+}
+
+const char* m2_last_kernel_name(const m2_plan* plan) { return plan ? plan->last_kernel : "none"; }
+
+int64_t m2_launch_count(const m2_plan* plan) { return plan ? plan->launches : -1; }
+
+}  // extern "C"

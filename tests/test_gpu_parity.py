@@ -1,0 +1,318 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Tolerances (relative L2 over the whole tensor; worst single row at twice that):
+fp32 path 1e-5, bf16-in / fp32-accumulate / bf16-out path 2e-2.  Integer tables are bit-exact
+(tests/test_abi_host.py)."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import monarch_oracle as O
+from paper_2310_12109_b200 import binding as M
+from paper_2310_12109_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-5
+TOL_BF16 = 2e-2
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.to(dtype) if dtype is not None else t
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def check(got, ref, tol, what=""):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    assert np.isfinite(got).all(), what + ": non-finite output"
+    g = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300)
+    rows_g = got.reshape(-1, got.shape[-1])
+    rows_r = ref.reshape(-1, ref.shape[-1])
+    per = np.linalg.norm(rows_g - rows_r, axis=1) / np.maximum(np.linalg.norm(rows_r, axis=1), 1e-300)
+    assert g <= tol, f"{what}: global rel-L2 {g:.3e} > {tol}"
+    assert per.max() <= 2 * tol, f"{what}: worst row rel-L2 {per.max():.3e} (row {per.argmax()}) > {2 * tol}"
+    return g
+
+
+def run_conv(dims, x_np, k_np, causal, dtype, sign=+1):
+    plan = M.Plan(dims, dtype=dtype, sign=sign, device=0)
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    x = dev(x_np.astype(np.float32), tdt)
+    k = dev(k_np.astype(np.float32))
+    kf = M.m2_kernel_spectrum(plan, k)
+    y = M.m2_monarch_conv_fwd(plan, x, kf, M.M2_CAUSAL if causal else M.M2_CIRCULAR)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    name = plan.last_kernel()
+    plan.close()
+    return host(y), name
+
+
+# ---- config 1: fp32, order 2, causal, checked against the direct sum --------------------------
+
+def test_config1_fp32_causal_vs_direct():
+    c = synth.config1()
+    y, name = run_conv(c["dims"], c["x"], c["k"], True, M.M2_FP32)
+    ref = O.direct_causal_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64))
+    check(y, ref, TOL_FP32, "config1 " + name)
+    ref2 = O.monarch_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64), c["dims"], causal=True)
+    check(y, ref2, TOL_FP32, "config1 vs factored oracle")
+
+
+@pytest.mark.parametrize("dims", [(32, 16), (2, 3), (4, 4, 4), (32, 32, 32)])
+@pytest.mark.parametrize("sign", [+1, -1])
+def test_kernel_spectrum_is_the_dft(dims, sign):
+    N = int(np.prod(dims))
+    H, n = 3, N // 2
+    k = synth.normal(900 + N, (H, n)).astype(np.float32)
+    plan = M.Plan(dims, dtype=M.M2_FP32, sign=sign, device=0)
+    kf = M.m2_kernel_spectrum(plan, dev(k))
+    nat = host(M.m2_spectrum_to_natural(plan, kf, H))
+    got = nat[..., 0] + 1j * nat[..., 1]
+    kp = np.concatenate([k.astype(np.float64), np.zeros((H, N - n))], -1)
+    ref = O.monarch_dft(kp, dims, sign)
+    err = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert err < TOL_FP32, err
+    plan.close()
+
+
+@pytest.mark.parametrize("dims,n,causal", [
+    ((32, 16), 256, True), ((32, 16), 200, True), ((32, 16), 1, True), ((32, 16), 512, False),
+    ((16, 32), 512, False), ((2, 3), 6, False), ((3, 5), 7, True), ((4, 4, 4), 32, True),
+    ((8, 4, 2), 64, False), ((16, 16, 16), 2048, True), ((64, 64), 4096, False), ((32, 32, 8), 4096, True),
+])
+def test_fp32_conv_shapes(dims, n, causal):
+    B, H = 2, 3
+    x = synth.normal(700 + n, (B, H, n)).astype(np.float32)
+    k = (synth.normal(701 + n, (H, n)) / np.sqrt(n)).astype(np.float32)
+    y, name = run_conv(dims, x, k, causal, M.M2_FP32)
+    x64, k64 = x.astype(np.float64), k.astype(np.float64)
+    ref = O.direct_causal_conv(k64[None], x64) if causal else O.direct_circular_conv(k64[None], x64)
+    check(y, ref, TOL_FP32, f"{dims} n={n} {name}")
+
+
+def test_fp32_conv_sign_minus_matches():
+    c = synth.config1()
+    y, _ = run_conv(c["dims"], c["x"], c["k"], True, M.M2_FP32, sign=-1)
+    ref = O.direct_causal_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64))
+    check(y, ref, TOL_FP32, "sign=-1")
+
+
+# ---- config 2: bf16 circular, N = 512 = 32 x 16 ----------------------------------------------
+
+@pytest.mark.parametrize("B,H", [(4, 24), (3, 5), (1, 1), (32, 9)])
+def test_config2_small_full_compare(B, H):
+    c = synth.config2(B=B, H=H)
+    y, name = run_conv(c["dims"], c["x"], c["k"], False, M.M2_BF16)
+    ref = O.monarch_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64), c["dims"], causal=False)
+    check(y, ref, TOL_BF16, f"config2 B={B} H={H} {name}")
+
+
+def test_config2_full_size():
+    c = synth.config2()
+    y, name = run_conv(c["dims"], c["x"], c["k"], False, M.M2_BF16)
+    x64, k64 = c["x"].astype(np.float64), c["k"].astype(np.float64)
+    ref = O.monarch_conv(k64[None], x64, c["dims"], causal=False)
+    check(y, ref, TOL_BF16, "config2 full " + name)
+    # sampled rows against the direct O(N^2) sum
+    for b, h in [(0, 0), (31, 767), (7, 100), (16, 384), (1, 766), (30, 1), (12, 511), (5, 513)]:
+        d = O.direct_circular_conv(k64[h], x64[b, h])
+        check(y[b, h][None], d[None], TOL_BF16 / 2, f"config2 row ({b},{h}) direct")
+
+
+def test_bf16_causal_order2_and_ragged():
+    for n in (256, 100):
+        B, H = 5, 7
+        x = synth.round_bf16(synth.normal(800 + n, (B, H, n)))
+        k = synth.decay_kernel(2, H, n, 0.005, float(np.sqrt(512.0)))
+        y, name = run_conv((32, 16), x, k, True, M.M2_BF16)
+        ref = O.direct_causal_conv(k.astype(np.float64)[None], x.astype(np.float64))
+        check(y, ref, TOL_BF16, f"bf16 causal n={n} {name}")
+
+
+# ---- config 3: Monarch matmul ------------------------------------------------------------------
+
+def run_matmul(c, dtype=M.M2_BF16):
+    b = c["L"].shape[0]
+    plan = M.Plan((b, b), dtype=dtype, device=0)
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    Y = M.m2_monarch_matmul(plan, dev(c["X"], tdt), dev(c["L"], tdt), dev(c["R"], tdt))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    name = plan.last_kernel()
+    plan.close()
+    return host(Y), name
+
+
+@pytest.mark.parametrize("T,b", [(37, 64), (128, 64), (5, 8), (300, 16), (1, 64)])
+def test_config3_small_full_compare(T, b):
+    c = synth.config3(T=T, b=b)
+    Y, name = run_matmul(c)
+    ref = O.monarch_apply(c["L"].astype(np.float64), c["R"].astype(np.float64), c["X"].astype(np.float64))
+    check(Y, ref, TOL_BF16, f"config3 T={T} b={b} {name}")
+
+
+def test_matmul_fp32_rectangular_vs_dense():
+    N1, N2, T = 8, 4, 9
+    X = synth.normal(31, (T, N1 * N2)).astype(np.float32)
+    L = synth.normal(32, (N1, N2, N2)).astype(np.float32)
+    R = synth.normal(33, (N2, N1, N1)).astype(np.float32)
+    plan = M.Plan((N1, N2), dtype=M.M2_FP32, device=0)
+    Y = host(M.m2_monarch_matmul(plan, dev(X), dev(L), dev(R)))
+    Md = O.monarch_dense(L.astype(np.float64), R.astype(np.float64))
+    check(Y, X.astype(np.float64) @ Md.T, TOL_FP32, "fp32 rectangular matmul vs dense P L P^T R P")
+    plan.close()
+
+
+def test_config3_full_size_sampled():
+    c = synth.config3()
+    Y, name = run_matmul(c)
+    idx = np.array([0, 1, 127, 128, 4095, 8191, 8192, 12345, 16382, 16383])
+    ref = O.monarch_apply(c["L"].astype(np.float64), c["R"].astype(np.float64), c["X"][idx].astype(np.float64))
+    check(Y[idx], ref, TOL_BF16, "config3 full sampled " + name)
+    # property over every token: no row is garbage (norms agree with the sampled ratio)
+    ratio = np.linalg.norm(Y, axis=1) / np.linalg.norm(c["X"].astype(np.float64), axis=1)
+    assert np.isfinite(Y).all() and ratio.min() > 0.5 and ratio.max() < 2.0
+
+
+# ---- config 4: order-3 causal, N = 32768 ------------------------------------------------------------
+
+@pytest.mark.parametrize("B,H", [(1, 3), (2, 2)])
+def test_config4_small_full_rows(B, H):
+    c = synth.config4(B=B, H=H)
+    y, name = run_conv(c["dims"], c["x"], c["k"], True, M.M2_BF16)
+    ref = O.monarch_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64), c["dims"], causal=True)
+    check(y, ref, TOL_BF16, f"config4 B={B} H={H} {name}")
+
+
+def test_config4_full_size_sampled():
+    c = synth.config4()
+    y, name = run_conv(c["dims"], c["x"], c["k"], True, M.M2_BF16)
+    assert np.isfinite(y).all()
+    rows = [(0, 0), (3, 1023), (1, 512), (2, 77), (0, 1022), (3, 1), (2, 1000), (1, 300)]
+    xs = np.stack([c["x"][b, h] for b, h in rows]).astype(np.float64)
+    ks = np.stack([c["k"][h] for b, h in rows]).astype(np.float64)
+    ref = O.monarch_conv(ks, xs, c["dims"], causal=True)
+    got = np.stack([y[b, h] for b, h in rows])
+    check(got, ref, TOL_BF16, "config4 full sampled " + name)
+    # direct sum at sampled outputs of one row
+    b, h = rows[1]
+    for t in (0, 1, 1024, 9999, 16383):
+        d = float(np.dot(ks[1][: t + 1], xs[1][t::-1]))
+        assert abs(got[1][t] - d) <= 4e-2 * max(abs(d), np.abs(ref[1]).mean())
+    # every row is sane: output energy within the range of the checked rows
+    e = np.linalg.norm(y.reshape(-1, y.shape[-1]), axis=1)
+    assert e.min() > 0.2 * np.median(e) and e.max() < 5 * np.median(e)
+
+
+# ---- config 5: the M2 block -------------------------------------------------------------------------
+
+def run_block(c):
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)
+    kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+    y, z = M.m2_block_fwd(plan, dev(c["x"], torch.bfloat16), kf, dev(c["w_short"]), dev(c["W_up"], torch.bfloat16),
+                          dev(c["W_down"], torch.bfloat16))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    plan.close()
+    return host(y), host(z)
+
+
+def block_ref(c, bsel=None):
+    x = c["x"].astype(np.float64)
+    if bsel is not None:
+        x = x[bsel]
+    return O.m2_block_forward(x, c["k"].astype(np.float64), c["w_short"].astype(np.float64),
+                              c["W_up"].astype(np.float64), c["W_down"].astype(np.float64), c["dims"])
+
+
+def test_config5_small():
+    c = synth.config5(B=2)
+    y, z = run_block(c)
+    yr, zr = block_ref(c)
+    check(z.reshape(2 * 512, 768), zr.reshape(2 * 512, 768), TOL_BF16, "config5 z")
+    check(y.reshape(2 * 512, 768), yr.reshape(2 * 512, 768), TOL_BF16, "config5 y")
+
+
+def test_config5_full_size_sampled():
+    c = synth.config5()
+    y, z = run_block(c)
+    assert np.isfinite(y).all()
+    sel = [0, 17, 31]
+    yr, zr = block_ref(c, sel)
+    check(z[sel].reshape(-1, 768), zr.reshape(-1, 768), TOL_BF16, "config5 full z")
+    check(y[sel].reshape(-1, 768), yr.reshape(-1, 768), TOL_BF16, "config5 full y")
+
+
+# ---- edge cases, error paths, determinism -------------------------------------------------------------
+
+def test_empty_batches_and_error_codes():
+    plan = M.Plan((32, 16), dtype=M.M2_BF16, device=0)
+    k = dev(synth.decay_kernel(2, 2, 512, 0.005, 22.6))
+    kf = M.m2_kernel_spectrum(plan, k)
+    x0 = torch.empty((0, 2, 512), dtype=torch.bfloat16, device="cuda")
+    assert M.m2_monarch_conv_fwd(plan, x0, kf, M.M2_CIRCULAR).shape == (0, 2, 512)
+    lib = M.lib()
+    x = torch.zeros((1, 2, 512), dtype=torch.bfloat16, device="cuda")
+    y = torch.empty_like(x)
+    s = torch.cuda.current_stream().cuda_stream
+    # causal needs n <= N/2; circular needs n == N
+    assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr(), kf.data_ptr(), y.data_ptr(), 1, 2, 512, M.M2_CAUSAL, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr(), kf.data_ptr(), y.data_ptr(), 1, 2, 256, M.M2_CIRCULAR, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr() + 2, kf.data_ptr(), y.data_ptr(), 1, 2, 256, M.M2_CAUSAL, s) == M.M2_ERR_ALIGNMENT
+    assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr(), kf.data_ptr(), y.data_ptr(), 1, 2, 256, 9, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_matmul(plan.handle, x.data_ptr(), x.data_ptr(), x.data_ptr(), None, 1, s) == M.M2_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    plan.close()
+
+
+def test_runs_are_bit_identical_and_stay_in_bounds():
+    c = synth.config2(B=8, H=16)
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)
+    kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+    x = dev(c["x"], torch.bfloat16)
+    # canary-padded output: the kernel must not write outside [B, H, n]
+    pad = 4096
+    buf = torch.full((x.numel() + 2 * pad,), 7.0, dtype=torch.bfloat16, device="cuda")
+    y = buf[pad:pad + x.numel()].view_as(x)
+    M.m2_monarch_conv_fwd(plan, x, kf, M.M2_CIRCULAR, y=y)
+    y1 = y.clone()
+    M.m2_monarch_conv_fwd(plan, x, kf, M.M2_CIRCULAR, y=y)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y)
+    assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + x.numel():] == 7.0).all())
+    plan.close()
+
+
+def test_host_buffer_entry_points():
+    c = synth.config2(B=2, H=8)
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)
+    kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+    xh = torch.from_numpy(c["x"]).to(torch.bfloat16).pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    xs, ys = torch.empty_like(xh, device="cuda"), torch.empty_like(xh, device="cuda")
+    M.m2_monarch_conv_fwd_host(plan, xh, kf, yh, xs, ys, M.M2_CIRCULAR)
+    torch.cuda.synchronize()
+    yd = M.m2_monarch_conv_fwd(plan, xs, kf, M.M2_CIRCULAR)
+    torch.cuda.synchronize()
+    assert torch.equal(yh, yd.cpu())
+    plan.close()
+    c3 = synth.config3(T=9, b=16)
+    plan = M.Plan((16, 16), dtype=M.M2_BF16, device=0)
+    Xh = torch.from_numpy(c3["X"]).to(torch.bfloat16).pin_memory()
+    Yh = torch.empty_like(Xh).pin_memory()
+    L, R = dev(c3["L"], torch.bfloat16), dev(c3["R"], torch.bfloat16)
+    Xs, Ys = torch.empty_like(Xh, device="cuda"), torch.empty_like(Xh, device="cuda")
+    M.m2_monarch_matmul_host(plan, Xh, L, R, Yh, Xs, Ys)
+    torch.cuda.synchronize()
+    ref = O.monarch_apply(c3["L"].astype(np.float64), c3["R"].astype(np.float64), c3["X"].astype(np.float64))
+    check(host(Yh), ref, TOL_BF16, "matmul host entry")
+    plan.close()

@@ -1,9 +1,469 @@
+// Tensor-core Monarch convolution, order 2, N = 512 = 32 x 16, bf16 in / fp32 accumulate / bf16 out.
+//
+// y = Re( M^-1 ( k_f (.) M pad(x) ) ) with M = P L P^T R P = F_N (Eq. 2; Corollary "DFT is M").  Every
+// Monarch stage is a dense contraction over one index digit and runs as a tcgen05 UMMA with the
+// accumulator in TMEM; the stride permutations never move data on their own: they are the choice of
+// which digit an operand's K dimension walks, expressed in the TMA box and in where the hand-off
+// threads write the next operand.
+//
+// A "unit" is 8 batch entries of one channel (8 rows x 512).  128 TMEM lanes = 8 rows x 16 values of the
+// digit that is NOT being contracted, so each thread owns whole complex numbers (re and im sit in
+// different TMEM columns of its lane) and the twiddle / spectrum multiplies are thread-local fp32:
+//
+//   S1   D1[(r,n2)][(c,k1)]   = sum_n1  x[r][n1][n2] * F32[(c,k1)][n1]           A: M-major (TMA tile)
+//   h1   twiddle w_N^{n2 k1} (fp32), round to bf16, write A2[(r,k1)][(c,n2)]         M-major
+//   S2   D2[(r,k1)][(c,k2)]   = sum_(c,n2) A2 * F16                              two M=128 halves
+//   h2   multiply by k_f[h][k1][k2] (fp32, 1/N folded in), write A3[(r,k1)][(c,k2)]  K-major
+//   S2'  D3[(r,k1)][(c,n2)]   = sum_(c,k2) A3 * conj(F16)
+//   h3   conj twiddle, write A4[(r,n2)][(c,k1)]                                      M-major
+//   S1'  D4[(r,n2)][n1]       = Re sum_(c,k1) A4 * conj(F32)
+//   h4   round to bf16 into the output tile, TMA store.
+//
+// Four such CTAs (128 threads, 128 TMEM columns, ~52 KB shared memory each) share an SM, so one
+// CTA's UMMA / TMA latency is covered by the others' fp32 work.  All waits are bounded.
 #include "conv_umma.h"
 
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "ptx_sm100.cuh"
+
 namespace m2u {
-cudaError_t create_tables(m2_plan*) { return cudaSuccess; }
-void destroy_tables(m2_plan*) {}
-int32_t conv_fwd(const m2_plan*, const void*, const void*, void*, int64_t, int64_t, int64_t, int32_t, cudaStream_t) {
-    return M2_ERR_UNSUPPORTED;
+
+using namespace sm100;
+
+constexpr int kRows = 8;             // rows (batch entries) per unit
+constexpr int kThreads = 128;
+constexpr int kTmemCols = 128;
+// shared memory map (bytes)
+constexpr int OFF_X = 0;             // 2 boxes [n2hi][r][n1][8]            8192
+constexpr int OFF_A = 8192;          // A2 / A3 / A4                        16384
+constexpr int OFF_OUT = 24576;       // [n2hi][r][n1][8] bf16                8192
+constexpr int OFF_CONST = 32768;     // B1 4096 | B2 2048 | B3 2048 | B4 4096 | twA 4096 | twB 4096
+constexpr int CONST_BYTES = 20480;
+constexpr int OFF_B1 = OFF_CONST, OFF_B2 = OFF_B1 + 4096, OFF_B3 = OFF_B2 + 2048, OFF_B4 = OFF_B3 + 2048;
+constexpr int OFF_TWA = OFF_B4 + 4096, OFF_TWB = OFF_TWA + 4096;
+constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // bar_x, bar_mma, tmem ptr
+constexpr int SMEM_BYTES = OFF_BAR + 64;
+
+struct Tables {
+    void* d_const = nullptr;  // CONST_BYTES
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
 }
+
+__global__ void __launch_bounds__(kThreads, 4)
+conv512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
+               const float2* __restrict__ kf, const uint4* __restrict__ consts, int B, int H, int n1_valid,
+               int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t bar_x = s_base + OFF_BAR, bar_mma = s_base + OFF_BAR + 8, s_tptr = s_base + OFF_BAR + 16;
+
+    // constants -> shared memory
+    {
+        uint4* dst = reinterpret_cast<uint4*>(smem + OFF_CONST);
+        for (int i = tid; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
+    }
+    if (tid == 0) {
+        mbar_init(bar_x, 1);
+        mbar_init(bar_mma, 1);
+        fence_barrier_init();
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_y);
+    }
+    if (warp == 0) tmem_alloc(s_tptr, kTmemCols);
+    fence_proxy_async();   // the constant matrices are read by the async proxy (UMMA)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 16);
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
+    const uint32_t T1 = 0, T2 = 64;                                 // column regions: D1/D3 and D2/D4
+
+    const int bgroups = (B + kRows - 1) / kRows;
+    const int units = H * bgroups;
+    constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
+    constexpr uint32_t ID_S2 = instr_desc_bf16(128, 32, true, false);
+    constexpr uint32_t ID_S2I = instr_desc_bf16(128, 32, false, false);
+    constexpr uint32_t ID_S1I = instr_desc_bf16(128, 32, true, false);
+    const int k1steps = (n1_valid + 15) / 16;   // causal input: digits n1 >= n/16 are zero -> skipped
+
+    uint32_t ph_x = 0, ph_m = 0;
+    bool ok = true, aborted = false;
+    bool load_pending = false, store_pending = false;
+    int u = blockIdx.x;
+    if (tid == 0 && u < units) {
+        mbar_expect_tx(bar_x, 8192);
+        tma_load_4d(s_base + OFF_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
+        tma_load_4d(s_base + OFF_X + 4096, &map_x, 8, 0, u % H, (u / H) * kRows, bar_x);
+        load_pending = true;
+    }
+
+    for (; u < units; u += gridDim.x) {
+        const int h = u % H;
+        const int b0 = (u / H) * kRows;
+        // ---- S1 ---------------------------------------------------------------------------------
+        if (tid == 0) {
+            ok = mbar_wait(bar_x, ph_x);
+            load_pending = false;
+            if (ok) {
+                tc_fence_after();
+#pragma unroll 1
+                for (int s = 0; s < k1steps; ++s)
+                    umma_f16(tmem + T1, smem_desc(s_base + OFF_X + s * 256, 128, 512),
+                             smem_desc(s_base + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
+                umma_commit(bar_mma);
+            }
+        }
+        ph_x ^= 1;
+        // ---- h1: twiddle, A2 ---------------------------------------------------------------------
+        ok = ok && mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        {
+            const int un = u + gridDim.x;       // the x tile is free: fetch the next unit's
+            if (tid == 0 && ok && un < units) {
+                mbar_expect_tx(bar_x, 8192);
+                tma_load_4d(s_base + OFF_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
+                tma_load_4d(s_base + OFF_X + 4096, &map_x, 8, 0, un % H, (un / H) * kRows, bar_x);
+                load_pending = true;
+            }
+        }
+        if (ok) {
+            const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
+            const float4* twA = reinterpret_cast<const float4*>(smem + OFF_TWA);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float re[8], im[8];
+                tmem_ld8(t_lane + T1 + 8 * j, re);
+                tmem_ld8(t_lane + T1 + 32 + 8 * j, im);
+                tmem_ld_wait();
+                tmem_ld_fence8(re);
+                tmem_ld_fence8(im);
+                uint32_t pr[4], pi[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 w = twA[(4 * j + q) * 16 + n2];
+                    const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+                    pr[q] = pack_bf16(a0 * w.x - b0v * w.y, a1 * w.z - b1 * w.w);
+                    pi[q] = pack_bf16(a0 * w.y + b0v * w.x, a1 * w.w + b1 * w.z);
+                }
+                unsigned char* base = smem + OFF_A + (r * 4 + j) * 512 + n2lo * 16;
+                *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
+                *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = make_uint4(pi[0], pi[1], pi[2], pi[3]);
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (__syncthreads_or(!ok)) {
+            aborted = true;
+            break;
+        }
+        // ---- S2 ---------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int s = 0; s < 2; ++s)
+                    umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + OFF_A + hf * 8192 + s * 256, 128, 512),
+                             smem_desc(s_base + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+            umma_commit(bar_mma);
+        }
+        // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (ok) {
+            const int k1 = tid & 31;
+            const float4* kf4 = reinterpret_cast<const float4*>(kf + ((size_t)h * 512 + k1 * 16));
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int m = hf * 128 + tid;
+                unsigned char* rowp = smem + OFF_A + (m >> 3) * 512 + (m & 7) * 16;
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    float re[8], im[8];
+                    tmem_ld8(t_lane + T2 + hf * 32 + 8 * g, re);
+                    tmem_ld8(t_lane + T2 + hf * 32 + 16 + 8 * g, im);
+                    tmem_ld_wait();
+                    tmem_ld_fence8(re);
+                    tmem_ld_fence8(im);
+                    uint32_t pr[4], pi[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 w = __ldg(kf4 + g * 4 + q);
+                        const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+                        pr[q] = pack_bf16(a0 * w.x - b0v * w.y, a1 * w.z - b1 * w.w);
+                        pi[q] = pack_bf16(a0 * w.y + b0v * w.x, a1 * w.w + b1 * w.z);
+                    }
+                    *reinterpret_cast<uint4*>(rowp + g * 128) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
+                    *reinterpret_cast<uint4*>(rowp + (2 + g) * 128) = make_uint4(pi[0], pi[1], pi[2], pi[3]);
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (__syncthreads_or(!ok)) {
+            aborted = true;
+            break;
+        }
+        // ---- S2' --------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int s = 0; s < 2; ++s)
+                    umma_f16(tmem + T1 + hf * 32, smem_desc(s_base + OFF_A + hf * 8192 + s * 256, 128, 512),
+                             smem_desc(s_base + OFF_B3 + s * 256, 128, 512), ID_S2I, s > 0);
+            umma_commit(bar_mma);
+        }
+        // ---- h3: conjugate twiddle, A4 --------------------------------------------------------------
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (ok) {
+            const int k1 = tid & 31;
+            const float4* twB = reinterpret_cast<const float4*>(smem + OFF_TWB);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int r = hf * 4 + (tid >> 5);
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    float re[8], im[8];
+                    tmem_ld8(t_lane + T1 + hf * 32 + 8 * g, re);
+                    tmem_ld8(t_lane + T1 + hf * 32 + 16 + 8 * g, im);
+                    tmem_ld_wait();
+                    tmem_ld_fence8(re);
+                    tmem_ld_fence8(im);
+                    uint32_t pr[4], pi[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 w = twB[(4 * g + q) * 32 + k1];
+                        const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+                        pr[q] = pack_bf16(a0 * w.x - b0v * w.y, a1 * w.z - b1 * w.w);
+                        pi[q] = pack_bf16(a0 * w.y + b0v * w.x, a1 * w.w + b1 * w.z);
+                    }
+                    unsigned char* base = smem + OFF_A + (r * 2 + g) * 1024 + (k1 >> 3) * 128 + (k1 & 7) * 16;
+                    *reinterpret_cast<uint4*>(base) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
+                    *reinterpret_cast<uint4*>(base + 512) = make_uint4(pi[0], pi[1], pi[2], pi[3]);
+                }
+            }
+        }
+        if (tid == 0 && store_pending) {   // the output tile is about to be rewritten
+            tma_store_wait_read0();
+            store_pending = false;
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (__syncthreads_or(!ok)) {
+            aborted = true;
+            break;
+        }
+        // ---- S1' --------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+                umma_f16(tmem + T2, smem_desc(s_base + OFF_A + s * 256, 128, 1024),
+                         smem_desc(s_base + OFF_B4 + s * 256, 128, 1024), ID_S1I, s > 0);
+            umma_commit(bar_mma);
+        }
+        // ---- h4: output tile --------------------------------------------------------------------------
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (ok) {
+            const int r = tid >> 4, n2 = tid & 15;
+            __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(smem + OFF_OUT + (n2 >> 3) * 4096 + r * 512 + (n2 & 7) * 2);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                float v[8];
+                tmem_ld8(t_lane + T2 + 8 * g, v);
+                tmem_ld_wait();
+                tmem_ld_fence8(v);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) outp[(8 * g + i) * 8] = __float2bfloat16_rn(v[i]);
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (__syncthreads_or(!ok)) {
+            aborted = true;
+            break;
+        }
+        if (tid == 0) {
+            tma_store_4d(&map_y, s_base + OFF_OUT, 0, 0, h, b0);
+            tma_store_4d(&map_y, s_base + OFF_OUT + 4096, 8, 0, h, b0);
+            tma_store_commit();
+            store_pending = true;
+        }
+    }
+    // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
+    if (tid == 0) {
+        if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+        if (load_pending) mbar_wait(bar_x, ph_x);
+        tma_store_wait_all0();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+
+static uint16_t bf16_bits(double v) {
+    float f = (float)v;
+    uint32_t b;
+    std::memcpy(&b, &f, 4);
+    b += 0x7FFFu + ((b >> 16) & 1u);
+    return (uint16_t)(b >> 16);
+}
+
+// K-major operand image: element (n, k) of an [N][K] matrix, 8 x 8 core matrices of 128 bytes,
+// K-adjacent core matrices 128 bytes apart, N-adjacent ones (K/8)*128 bytes apart.
+static void put_kmajor(std::vector<uint16_t>& img, int K, int n, int k, double v) {
+    const size_t byte = (size_t)(n / 8) * (K / 8) * 128 + (size_t)(k / 8) * 128 + (n % 8) * 16 + (k % 8) * 2;
+    img[byte / 2] = bf16_bits(v);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+static bool covered(const m2_plan* pl) {
+    return pl->dtype == M2_BF16 && pl->p == 2 && pl->dims[0] == 32 && pl->dims[1] == 16;
+}
+
+cudaError_t create_tables(m2_plan* pl) {
+    if (!covered(pl)) return cudaSuccess;
+    const int N1 = 32, N2 = 16, N = 512;
+    const double sg = pl->sign >= 0 ? 1.0 : -1.0;
+    std::vector<uint16_t> B1(2048), B2(1024), B3(1024), B4(2048);
+    std::vector<float> twA(1024), twB(1024);
+    // B1: [N = (c,k1) 64][K = n1 32]: F32[k1,n1] = cos + i sg sin
+    for (int c = 0; c < 2; ++c)
+        for (int k1 = 0; k1 < N1; ++k1)
+            for (int n1 = 0; n1 < N1; ++n1) {
+                const double th = 2.0 * M_PI * ((k1 * n1) % N1) / N1;
+                put_kmajor(B1, 32, c * 32 + k1, n1, c == 0 ? std::cos(th) : sg * std::sin(th));
+            }
+    // B2: [N = (c',k2) 32][K = (c,n2) 32]: (a + ib)(cos + i s) -> re: cos a - s b ; im: s a + cos b
+    // B3: the same with the conjugate matrix: [N = (c',n2) 32][K = (c,k2) 32]
+    for (int co = 0; co < 2; ++co)
+        for (int o = 0; o < N2; ++o)
+            for (int ci = 0; ci < 2; ++ci)
+                for (int i = 0; i < N2; ++i) {
+                    const double th = 2.0 * M_PI * ((o * i) % N2) / N2;
+                    const double cs = std::cos(th), sn = sg * std::sin(th);
+                    double f, g;
+                    if (co == 0) { f = ci == 0 ? cs : -sn; g = ci == 0 ? cs : sn; }
+                    else         { f = ci == 0 ? sn : cs;  g = ci == 0 ? -sn : cs; }
+                    put_kmajor(B2, 32, co * 16 + o, ci * 16 + i, f);
+                    put_kmajor(B3, 32, co * 16 + o, ci * 16 + i, g);
+                }
+    // B4: [N = n1 32][K = (c,k1) 64]: Re( conj(F32)[n1,k1] (a + ib) ) = cos a + s b
+    for (int n1 = 0; n1 < N1; ++n1)
+        for (int c = 0; c < 2; ++c)
+            for (int k1 = 0; k1 < N1; ++k1) {
+                const double th = 2.0 * M_PI * ((k1 * n1) % N1) / N1;
+                put_kmajor(B4, 64, n1, c * 32 + k1, c == 0 ? std::cos(th) : sg * std::sin(th));
+            }
+    // twiddles w_N^{n2 k1}: twA[k1/2][n2][k1%2] (cos, sin); twB[n2/2][k1][n2%2] conjugated
+    for (int k1 = 0; k1 < N1; ++k1)
+        for (int n2 = 0; n2 < N2; ++n2) {
+            const double th = 2.0 * M_PI * ((n2 * k1) % N) / N;
+            const float cs = (float)std::cos(th), sn = (float)(sg * std::sin(th));
+            const size_t ia = (((size_t)(k1 / 2) * 16 + n2) * 2 + (k1 % 2)) * 2;
+            twA[ia] = cs;
+            twA[ia + 1] = sn;
+            const size_t ib = (((size_t)(n2 / 2) * 32 + k1) * 2 + (n2 % 2)) * 2;
+            twB[ib] = cs;
+            twB[ib + 1] = -sn;
+        }
+    std::vector<unsigned char> blob(CONST_BYTES);
+    std::memcpy(blob.data(), B1.data(), 4096);
+    std::memcpy(blob.data() + 4096, B2.data(), 2048);
+    std::memcpy(blob.data() + 6144, B3.data(), 2048);
+    std::memcpy(blob.data() + 8192, B4.data(), 4096);
+    std::memcpy(blob.data() + 12288, twA.data(), 4096);
+    std::memcpy(blob.data() + 16384, twB.data(), 4096);
+    Tables* t = new Tables();
+    cudaError_t e = cudaMalloc(&t->d_const, CONST_BYTES);
+    if (e == cudaSuccess) e = cudaMemcpy(t->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) {
+        if (t->d_const) cudaFree(t->d_const);
+        delete t;
+        return e;
+    }
+    pl->umma = reinterpret_cast<m2_umma_tables*>(t);
+    return cudaSuccess;
+}
+
+void destroy_tables(m2_plan* pl) {
+    if (!pl->umma) return;
+    Tables* t = reinterpret_cast<Tables*>(pl->umma);
+    if (t->d_const) cudaFree(t->d_const);
+    delete t;
+    pl->umma = nullptr;
+}
+
+// x / y viewed as [b][h][n1][n2] with n2 innermost; box = 8 of the 16 n2, all 32 n1, one h, 8 b.
+static bool make_map(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
+    cuuint32_t box[4] = {8, 32, 1, (cuuint32_t)kRows};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), gdim, gstr, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
+                 cudaStream_t stream) {
+    if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
+    // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
+    if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
+    Tables* t = reinterpret_cast<Tables*>(pl->umma);
+    alignas(64) CUtensorMap mx, my;
+    if (!make_map(&mx, x, B, H, n) || !make_map(&my, y, B, H, n)) return M2_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long units = H * ((B + kRows - 1) / kRows);
+    const int grid = (int)(units < 4LL * sms ? units : 4LL * sms);
+    conv512_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(mx, my, (const float2*)kf, (const uint4*)t->d_const, (int)B, (int)H,
+                                                           (int)(n / 16), pl->d_status);
+    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    pl->last_kernel = "conv_umma_o2_512";
+    pl->launches += 1;
+    return M2_OK;
+}
+
 }  // namespace m2u

@@ -37,18 +37,22 @@ namespace m2u {
 using namespace sm100;
 
 constexpr int kRows = 8;             // rows (batch entries) per unit
-constexpr int kThreads = 128;
-constexpr int kTmemCols = 128;
-// shared memory map (bytes)
-constexpr int OFF_X = 0;             // 2 boxes [n2hi][r][n1][8]            8192
-constexpr int OFF_A = 8192;          // A2 / A3 / A4                        16384
-constexpr int OFF_OUT = 24576;       // [n2hi][r][n1][8] bf16                8192
-constexpr int OFF_CONST = 32768;     // B1 4096 | B2 2048 | B3 2048 | B4 4096 | twA 4096 | twB 4096
+constexpr int kGroups = 4;           // independent warpgroups per CTA, each running its own unit loop
+constexpr int kThreads = 128 * kGroups;
+constexpr int kTmemColsPerGroup = 64;
+constexpr int kTmemCols = 256;       // allocation must be a power of two >= kGroups * 64
+// shared memory map (bytes): constants shared by the CTA, then one slice per warpgroup
+constexpr int OFF_CONST = 0;         // B1 4096 | B2 2048 | B3 2048 | B4 4096 | twA 4096 | twB 4096
 constexpr int CONST_BYTES = 20480;
 constexpr int OFF_B1 = OFF_CONST, OFF_B2 = OFF_B1 + 4096, OFF_B3 = OFF_B2 + 2048, OFF_B4 = OFF_B3 + 2048;
 constexpr int OFF_TWA = OFF_B4 + 4096, OFF_TWB = OFF_TWA + 4096;
-constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // bar_x, bar_mma, tmem ptr
-constexpr int SMEM_BYTES = OFF_BAR + 64;
+constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // per group: bar_x, bar_mma, bar_k, flag (32 B); then tmem ptr
+constexpr int OFF_GROUP = OFF_BAR + 256;
+constexpr int G_X = 0;               // 2 boxes [n2hi][r][n1][8]            8192
+constexpr int G_A = 8192;            // A2 / A3 / A4                        16384
+constexpr int G_KF = 24576;          // spectrum row of the unit's channel  4096
+constexpr int GROUP_BYTES = 28672;
+constexpr int SMEM_BYTES = OFF_GROUP + kGroups * GROUP_BYTES;
 
 struct Tables {
     void* d_const = nullptr;  // CONST_BYTES
@@ -59,116 +63,171 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__global__ void __launch_bounds__(kThreads, 4)
-conv512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
-               const float2* __restrict__ kf, const uint4* __restrict__ consts, int B, int H, int n1_valid,
-               int32_t* __restrict__ status) {
-    extern __shared__ __align__(1024) unsigned char smem[];
-    const int tid = threadIdx.x;
-    const int warp = tid >> 5;
-    const uint32_t s_base = smem_u32(smem);
-    const uint32_t bar_x = s_base + OFF_BAR, bar_mma = s_base + OFF_BAR + 8, s_tptr = s_base + OFF_BAR + 16;
-
-    // constants -> shared memory
-    {
-        uint4* dst = reinterpret_cast<uint4*>(smem + OFF_CONST);
-        for (int i = tid; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
+#ifdef M2_PHASE_TIMING
+// Development aid (never compiled into the shipped library): cycles block 0 / thread 0 spends in each
+// phase of the unit loop, summed over its units.
+__device__ long long g_phase_cycles[16];
+#define M2_TICK(slot)                                             \
+    if (blockIdx.x == 0 && threadIdx.x == 0) {                            \
+        const long long now_ = clock64();                         \
+        g_phase_cycles[slot] += now_ - tick_;                     \
+        tick_ = now_;                                             \
     }
+#else
+#define M2_TICK(slot)
+#endif
+
+// Multiplies 8 complex values (re[], im[]) by 8 complex factors given as 4 float4 (c0, s0, c1, s1) and
+// packs real and imaginary parts as bf16 pairs.
+__device__ __forceinline__ void cmul_pack8(const float* re, const float* im, const float4* w, uint4& pr, uint4& pi) {
+    uint32_t r_[4], i_[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float a0 = re[2 * q], b0 = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+        r_[q] = pack_bf16(a0 * w[q].x - b0 * w[q].y, a1 * w[q].z - b1 * w[q].w);
+        i_[q] = pack_bf16(a0 * w[q].y + b0 * w[q].x, a1 * w[q].w + b1 * w[q].z);
+    }
+    pr = make_uint4(r_[0], r_[1], r_[2], r_[3]);
+    pi = make_uint4(i_[0], i_[1], i_[2], i_[3]);
+}
+
+// block-wide barrier among the 128 threads of one warpgroup that also ORs a predicate
+__device__ __forceinline__ bool group_sync_or(int wg, bool pred, volatile int* flag) {
+    if (pred) *flag = 1;
+    asm volatile("bar.sync %0, 128;" ::"r"(wg + 1) : "memory");
+    return *flag != 0;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restrict__ y,
+               const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
+               int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem_all[];
+    const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
+    const int tid = threadIdx.x & 127;
+    const int warp = tid >> 5;                // warp within the group = TMEM lane quarter
+    const uint32_t s_all = smem_u32(smem_all);
+    unsigned char* smem = smem_all + OFF_GROUP + wg * GROUP_BYTES;   // this group's slice
+    const uint32_t s_base = s_all + OFF_GROUP + wg * GROUP_BYTES;
+    const uint32_t bar_x = s_all + OFF_BAR + wg * 32, bar_mma = bar_x + 8, bar_k = bar_x + 16;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_all + OFF_BAR + wg * 32 + 24);
+    const uint32_t s_tptr = s_all + OFF_BAR + 224;
+
+    const int bgroups0 = (B + kRows - 1) / kRows;
+    const int units0 = H * bgroups0;
+    int u = blockIdx.x * kGroups + wg;
+    const int ustride = gridDim.x * kGroups;
     if (tid == 0) {
         mbar_init(bar_x, 1);
         mbar_init(bar_mma, 1);
+        mbar_init(bar_k, 1);
+        *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_x);
-        prefetch_tensormap(&map_y);
     }
-    if (warp == 0) tmem_alloc(s_tptr, kTmemCols);
+    bool x_pending = false, k_pending = false;
+    if (tid == 0 && u < units0) {   // first loads go out before anything else
+        mbar_expect_tx(bar_x, 8192);
+        tma_load_4d(s_base + G_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
+        tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, u % H, (u / H) * kRows, bar_x);
+        x_pending = true;
+        mbar_expect_tx(bar_k, 4096);
+        bulk_load(s_base + G_KF, kfu + (size_t)(u % H) * 256, 4096, bar_k);
+        k_pending = true;
+    }
+    // constants -> shared memory
+    {
+        uint4* dst = reinterpret_cast<uint4*>(smem_all + OFF_CONST);
+        for (int i = threadIdx.x; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
+    }
+    if (threadIdx.x < 32) tmem_alloc(s_tptr, kTmemCols);
     fence_proxy_async();   // the constant matrices are read by the async proxy (UMMA)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 16);
+    const uint32_t tmem_cta = *reinterpret_cast<volatile uint32_t*>(smem_all + OFF_BAR + 224);
+    const uint32_t tmem = tmem_cta + wg * kTmemColsPerGroup;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
-    const uint32_t T1 = 0, T2 = 64;                                 // column regions: D1/D3 and D2/D4
+    const uint32_t T1 = 0, T2 = 0;   // every stage's accumulator reuses the same 64 columns
 
-    const int bgroups = (B + kRows - 1) / kRows;
-    const int units = H * bgroups;
+    const int units = units0;
     constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
     constexpr uint32_t ID_S2 = instr_desc_bf16(128, 32, true, false);
     constexpr uint32_t ID_S2I = instr_desc_bf16(128, 32, false, false);
     constexpr uint32_t ID_S1I = instr_desc_bf16(128, 32, true, false);
+    const int n1_valid = n / 16;
     const int k1steps = (n1_valid + 15) / 16;   // causal input: digits n1 >= n/16 are zero -> skipped
 
-    uint32_t ph_x = 0, ph_m = 0;
+    uint32_t ph_x = 0, ph_m = 0, ph_k = 0;
     bool ok = true, aborted = false;
-    bool load_pending = false, store_pending = false;
-    int u = blockIdx.x;
-    if (tid == 0 && u < units) {
-        mbar_expect_tx(bar_x, 8192);
-        tma_load_4d(s_base + OFF_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
-        tma_load_4d(s_base + OFF_X + 4096, &map_x, 8, 0, u % H, (u / H) * kRows, bar_x);
-        load_pending = true;
-    }
-
-    for (; u < units; u += gridDim.x) {
+#ifdef M2_PHASE_TIMING
+    long long tick_ = clock64();
+#endif
+    for (; u < units; u += ustride) {
+        M2_TICK(15)
         const int h = u % H;
         const int b0 = (u / H) * kRows;
+        const int un = u + ustride;
         // ---- S1 ---------------------------------------------------------------------------------
         if (tid == 0) {
             ok = mbar_wait(bar_x, ph_x);
-            load_pending = false;
+            x_pending = false;
             if (ok) {
                 tc_fence_after();
 #pragma unroll 1
                 for (int s = 0; s < k1steps; ++s)
-                    umma_f16(tmem + T1, smem_desc(s_base + OFF_X + s * 256, 128, 512),
-                             smem_desc(s_base + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
+                    umma_f16(tmem + T1, smem_desc(s_base + G_X + s * 256, 128, 512),
+                             smem_desc(s_all + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
                 umma_commit(bar_mma);
             }
         }
         ph_x ^= 1;
+        M2_TICK(0)
         // ---- h1: twiddle, A2 ---------------------------------------------------------------------
         ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        {
-            const int un = u + gridDim.x;       // the x tile is free: fetch the next unit's
-            if (tid == 0 && ok && un < units) {
-                mbar_expect_tx(bar_x, 8192);
-                tma_load_4d(s_base + OFF_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
-                tma_load_4d(s_base + OFF_X + 4096, &map_x, 8, 0, un % H, (un / H) * kRows, bar_x);
-                load_pending = true;
-            }
+        M2_TICK(1)
+        if (tid == 0 && ok && un < units) {   // the x tile is free: fetch the next unit's
+            mbar_expect_tx(bar_x, 8192);
+            tma_load_4d(s_base + G_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
+            tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, un % H, (un / H) * kRows, bar_x);
+            x_pending = true;
         }
         if (ok) {
             const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
-            const float4* twA = reinterpret_cast<const float4*>(smem + OFF_TWA);
+            const float4* twA = reinterpret_cast<const float4*>(smem_all + OFF_TWA) + n2;
+            float re[32], im[32];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                float re[8], im[8];
-                tmem_ld8(t_lane + T1 + 8 * j, re);
-                tmem_ld8(t_lane + T1 + 32 + 8 * j, im);
-                tmem_ld_wait();
-                tmem_ld_fence8(re);
-                tmem_ld_fence8(im);
-                uint32_t pr[4], pi[4];
+                tmem_ld8(t_lane + T1 + 8 * j, re + 8 * j);
+                tmem_ld8(t_lane + T1 + 32 + 8 * j, im + 8 * j);
+            }
+            tmem_ld_wait();
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float4 w = twA[(4 * j + q) * 16 + n2];
-                    const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-                    pr[q] = pack_bf16(a0 * w.x - b0v * w.y, a1 * w.z - b1 * w.w);
-                    pi[q] = pack_bf16(a0 * w.y + b0v * w.x, a1 * w.w + b1 * w.z);
-                }
-                unsigned char* base = smem + OFF_A + (r * 4 + j) * 512 + n2lo * 16;
-                *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
-                *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = make_uint4(pi[0], pi[1], pi[2], pi[3]);
+            for (int j = 0; j < 4; ++j) {
+                tmem_ld_fence8(re + 8 * j);
+                tmem_ld_fence8(im + 8 * j);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float4 w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = twA[(4 * j + q) * 16];
+                uint4 pr, pi;
+                cmul_pack8(re + 8 * j, im + 8 * j, w, pr, pi);
+                unsigned char* base = smem + G_A + (r * 4 + j) * 512 + n2lo * 16;
+                *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = pr;
+                *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = pi;
             }
         }
         fence_proxy_async();
         tc_fence_before();
-        if (__syncthreads_or(!ok)) {
+        if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
             break;
         }
+        M2_TICK(2)
         // ---- S2 ---------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -176,48 +235,54 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int s = 0; s < 2; ++s)
-                    umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + OFF_A + hf * 8192 + s * 256, 128, 512),
-                             smem_desc(s_base + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+                    umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + G_A + hf * 8192 + s * 256, 128, 512),
+                             smem_desc(s_all + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
             umma_commit(bar_mma);
         }
         // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
-        ok = mbar_wait(bar_mma, ph_m);
+        ok = mbar_wait(bar_k, ph_k);          // the channel's spectrum row has landed
+        ph_k ^= 1;
+        if (tid == 0) k_pending = false;
+        ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
+        M2_TICK(3)
         if (ok) {
             const int k1 = tid & 31;
-            const float4* kf4 = reinterpret_cast<const float4*>(kf + ((size_t)h * 512 + k1 * 16));
+            const float4* kfs = reinterpret_cast<const float4*>(smem + G_KF) + k1;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 const int m = hf * 128 + tid;
-                unsigned char* rowp = smem + OFF_A + (m >> 3) * 512 + (m & 7) * 16;
+                unsigned char* rowp = smem + G_A + (m >> 3) * 512 + (m & 7) * 16;
+                float re[16], im[16];
+                tmem_ld8(t_lane + T2 + hf * 32, re);
+                tmem_ld8(t_lane + T2 + hf * 32 + 8, re + 8);
+                tmem_ld8(t_lane + T2 + hf * 32 + 16, im);
+                tmem_ld8(t_lane + T2 + hf * 32 + 24, im + 8);
+                tmem_ld_wait();
+                tmem_ld_fence8(re);
+                tmem_ld_fence8(re + 8);
+                tmem_ld_fence8(im);
+                tmem_ld_fence8(im + 8);
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
-                    float re[8], im[8];
-                    tmem_ld8(t_lane + T2 + hf * 32 + 8 * g, re);
-                    tmem_ld8(t_lane + T2 + hf * 32 + 16 + 8 * g, im);
-                    tmem_ld_wait();
-                    tmem_ld_fence8(re);
-                    tmem_ld_fence8(im);
-                    uint32_t pr[4], pi[4];
+                    float4 w[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 w = __ldg(kf4 + g * 4 + q);
-                        const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-                        pr[q] = pack_bf16(a0 * w.x - b0v * w.y, a1 * w.z - b1 * w.w);
-                        pi[q] = pack_bf16(a0 * w.y + b0v * w.x, a1 * w.w + b1 * w.z);
-                    }
-                    *reinterpret_cast<uint4*>(rowp + g * 128) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
-                    *reinterpret_cast<uint4*>(rowp + (2 + g) * 128) = make_uint4(pi[0], pi[1], pi[2], pi[3]);
+                    for (int q = 0; q < 4; ++q) w[q] = kfs[(g * 4 + q) * 32];
+                    uint4 pr, pi;
+                    cmul_pack8(re + 8 * g, im + 8 * g, w, pr, pi);
+                    *reinterpret_cast<uint4*>(rowp + g * 128) = pr;
+                    *reinterpret_cast<uint4*>(rowp + (2 + g) * 128) = pi;
                 }
             }
         }
         fence_proxy_async();
         tc_fence_before();
-        if (__syncthreads_or(!ok)) {
+        if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
             break;
         }
+        M2_TICK(4)
         // ---- S2' --------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -225,100 +290,112 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int s = 0; s < 2; ++s)
-                    umma_f16(tmem + T1 + hf * 32, smem_desc(s_base + OFF_A + hf * 8192 + s * 256, 128, 512),
-                             smem_desc(s_base + OFF_B3 + s * 256, 128, 512), ID_S2I, s > 0);
+                    umma_f16(tmem + T1 + hf * 32, smem_desc(s_base + G_A + hf * 8192 + s * 256, 128, 512),
+                             smem_desc(s_all + OFF_B3 + s * 256, 128, 512), ID_S2I, s > 0);
             umma_commit(bar_mma);
+            if (un < units) {                 // the spectrum tile is free: fetch the next unit's
+                mbar_expect_tx(bar_k, 4096);
+                bulk_load(s_base + G_KF, kfu + (size_t)(un % H) * 256, 4096, bar_k);
+                k_pending = true;
+            }
         }
         // ---- h3: conjugate twiddle, A4 --------------------------------------------------------------
         ok = mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
+        M2_TICK(5)
         if (ok) {
             const int k1 = tid & 31;
-            const float4* twB = reinterpret_cast<const float4*>(smem + OFF_TWB);
+            const float4* twB = reinterpret_cast<const float4*>(smem_all + OFF_TWB) + k1;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 const int r = hf * 4 + (tid >> 5);
+                float re[16], im[16];
+                tmem_ld8(t_lane + T1 + hf * 32, re);
+                tmem_ld8(t_lane + T1 + hf * 32 + 8, re + 8);
+                tmem_ld8(t_lane + T1 + hf * 32 + 16, im);
+                tmem_ld8(t_lane + T1 + hf * 32 + 24, im + 8);
+                tmem_ld_wait();
+                tmem_ld_fence8(re);
+                tmem_ld_fence8(re + 8);
+                tmem_ld_fence8(im);
+                tmem_ld_fence8(im + 8);
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
-                    float re[8], im[8];
-                    tmem_ld8(t_lane + T1 + hf * 32 + 8 * g, re);
-                    tmem_ld8(t_lane + T1 + hf * 32 + 16 + 8 * g, im);
-                    tmem_ld_wait();
-                    tmem_ld_fence8(re);
-                    tmem_ld_fence8(im);
-                    uint32_t pr[4], pi[4];
+                    float4 w[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 w = twB[(4 * g + q) * 32 + k1];
-                        const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-                        pr[q] = pack_bf16(a0 * w.x - b0v * w.y, a1 * w.z - b1 * w.w);
-                        pi[q] = pack_bf16(a0 * w.y + b0v * w.x, a1 * w.w + b1 * w.z);
-                    }
-                    unsigned char* base = smem + OFF_A + (r * 2 + g) * 1024 + (k1 >> 3) * 128 + (k1 & 7) * 16;
-                    *reinterpret_cast<uint4*>(base) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
-                    *reinterpret_cast<uint4*>(base + 512) = make_uint4(pi[0], pi[1], pi[2], pi[3]);
+                    for (int q = 0; q < 4; ++q) w[q] = twB[(4 * g + q) * 32];
+                    uint4 pr, pi;
+                    cmul_pack8(re + 8 * g, im + 8 * g, w, pr, pi);
+                    unsigned char* base = smem + G_A + (r * 2 + g) * 1024 + (k1 >> 3) * 128 + (k1 & 7) * 16;
+                    *reinterpret_cast<uint4*>(base) = pr;
+                    *reinterpret_cast<uint4*>(base + 512) = pi;
                 }
             }
         }
-        if (tid == 0 && store_pending) {   // the output tile is about to be rewritten
-            tma_store_wait_read0();
-            store_pending = false;
-        }
         fence_proxy_async();
         tc_fence_before();
-        if (__syncthreads_or(!ok)) {
+        if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
             break;
         }
+        M2_TICK(6)
         // ---- S1' --------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
 #pragma unroll
             for (int s = 0; s < 4; ++s)
-                umma_f16(tmem + T2, smem_desc(s_base + OFF_A + s * 256, 128, 1024),
-                         smem_desc(s_base + OFF_B4 + s * 256, 128, 1024), ID_S1I, s > 0);
+                umma_f16(tmem + T2, smem_desc(s_base + G_A + s * 256, 128, 1024),
+                         smem_desc(s_all + OFF_B4 + s * 256, 128, 1024), ID_S1I, s > 0);
             umma_commit(bar_mma);
         }
-        // ---- h4: output tile --------------------------------------------------------------------------
+        // ---- h4: round and store: lane (r, n2) holds y[r][n1*16 + n2] for all n1; a warp writes two full
+        //      32-byte sectors per instruction --------------------------------------------------------
         ok = mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
+        M2_TICK(7)
         if (ok) {
             const int r = tid >> 4, n2 = tid & 15;
-            __nv_bfloat16* outp = reinterpret_cast<__nv_bfloat16*>(smem + OFF_OUT + (n2 >> 3) * 4096 + r * 512 + (n2 & 7) * 2);
+            float v[32];
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                float v[8];
-                tmem_ld8(t_lane + T2 + 8 * g, v);
-                tmem_ld_wait();
-                tmem_ld_fence8(v);
+            for (int g = 0; g < 4; ++g) tmem_ld8(t_lane + T2 + 8 * g, v + 8 * g);
+            tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) outp[(8 * g + i) * 8] = __float2bfloat16_rn(v[i]);
+            for (int g = 0; g < 4; ++g) tmem_ld_fence8(v + 8 * g);
+            if (b0 + r < B) {
+                __nv_bfloat16* yr = y + ((size_t)(b0 + r) * H + h) * n + n2;
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < n1_valid) yr[i * 16] = __float2bfloat16_rn(v[i]);
             }
         }
-        fence_proxy_async();
         tc_fence_before();
-        if (__syncthreads_or(!ok)) {
+        if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
             break;
         }
-        if (tid == 0) {
-            tma_store_4d(&map_y, s_base + OFF_OUT, 0, 0, h, b0);
-            tma_store_4d(&map_y, s_base + OFF_OUT + 4096, 8, 0, h, b0);
-            tma_store_commit();
-            store_pending = true;
-        }
+        M2_TICK(8)
     }
     // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
     if (tid == 0) {
         if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-        if (load_pending) mbar_wait(bar_x, ph_x);
-        tma_store_wait_all0();
+        if (x_pending) mbar_wait(bar_x, ph_x);
+        if (k_pending) mbar_wait(bar_k, ph_k);
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (threadIdx.x < 32) tmem_dealloc(tmem_cta, kTmemCols);
+}
+
+// spectrum re-layout for this kernel: kfu[h][k2/2][k1] = (re, im)(k2 even), (re, im)(k2 odd) from plan order
+__global__ void relayout_spectrum_kernel(const float2* __restrict__ kf, float4* __restrict__ kfu, long long total) {
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 8 * 32
+    if (i >= total) return;
+    const int k1 = (int)(i & 31), q = (int)((i >> 5) & 7);
+    const long long h = i >> 8;
+    const float2 a = kf[h * 512 + k1 * 16 + 2 * q], b = kf[h * 512 + k1 * 16 + 2 * q + 1];
+    kfu[i] = make_float4(a.x, a.y, b.x, b.y);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
@@ -451,19 +528,42 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
     Tables* t = reinterpret_cast<Tables*>(pl->umma);
-    alignas(64) CUtensorMap mx, my;
-    if (!make_map(&mx, x, B, H, n) || !make_map(&my, y, B, H, n)) return M2_ERR_UNSUPPORTED;
+    alignas(64) CUtensorMap mx;
+    if (!make_map(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long long units = H * ((B + kRows - 1) / kRows);
-    const int grid = (int)(units < 4LL * sms ? units : 4LL * sms);
-    conv512_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(mx, my, (const float2*)kf, (const uint4*)t->d_const, (int)B, (int)H,
-                                                           (int)(n / 16), pl->d_status);
+    const long long ctas = (units + kGroups - 1) / kGroups;
+    const int grid = (int)(ctas < sms ? ctas : sms);
+    const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * 512 * 8);
+    conv512_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H,
+                                                           (int)n, pl->d_status);
     if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o2_512";
     pl->launches += 1;
     return M2_OK;
 }
+
+bool has_private_spectrum(const m2_plan* pl) { return pl->umma != nullptr && covered(pl); }
+
+cudaError_t relayout_spectrum(const m2_plan* pl, void* kf, int64_t H, cudaStream_t stream) {
+    if (!has_private_spectrum(pl) || H == 0) return cudaSuccess;
+    const long long total = H * 256;
+    float4* kfu = reinterpret_cast<float4*>(static_cast<unsigned char*>(kf) + (size_t)H * 512 * 8);
+    relayout_spectrum_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>((const float2*)kf, kfu, total);
+    return cudaGetLastError();
+}
+
+#ifdef M2_PHASE_TIMING
+extern "C" void m2_debug_phase_cycles(long long* out16, int reset) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out16, g_phase_cycles, sizeof(long long) * 16);
+    if (reset) {
+        long long z[16] = {0};
+        cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z));
+    }
+}
+#endif
 
 }  // namespace m2u

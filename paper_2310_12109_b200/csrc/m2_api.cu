@@ -191,7 +191,7 @@ int32_t m2_plan_get_table(const m2_plan* plan, int32_t which, int32_t* host_out,
 
 int64_t m2_spectrum_bytes(const m2_plan* plan, int64_t H) {
     if (!plan || H < 0) return -1;
-    return H * plan->N * (int64_t)sizeof(float2);
+    return H * plan->N * (int64_t)sizeof(float2) * (m2u::has_private_spectrum(plan) ? 2 : 1);
 }
 
 int32_t m2_kernel_spectrum(const m2_plan* plan, const float* k_dev, int64_t H, int64_t n, void* kf_dev, void* stream) {
@@ -206,8 +206,9 @@ int32_t m2_kernel_spectrum(const m2_plan* plan, const float* k_dev, int64_t H, i
     cudaError_t e = m2g::launch_spectrum(s, k_dev, kf_dev, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;
+    if (m2u::relayout_spectrum(plan, kf_dev, H, (cudaStream_t)stream) != cudaSuccess) return M2_ERR_CUDA;
     plan->last_kernel = "spectrum_generic_fp32";
-    plan->launches += (H > 0);
+    plan->launches += (H > 0) * (m2u::has_private_spectrum(plan) ? 2 : 1);
     return M2_OK;
 }
 

@@ -117,6 +117,27 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
                      const void* W_up_dev, const void* W_down_dev, void* z_dev, void* y_dev, int64_t B,
                      int64_t T, int64_t C, int32_t nblk, int32_t expand, void* stream);
 
+/* The same block forward as m2_block_fwd for callers that must not allocate device memory and have
+ * no scratch buffer of their own to hand in.  (The paper has no counterpart: this is a deployment
+ * variant, not a different operation.)  Typical callers: a serving process whose framework has
+ * already taken all device memory into its own pool, so a cudaMalloc here would fail or eat into that
+ * pool's reserve; or a latency-critical loop that cannot afford the device-wide synchronisation a
+ * cudaMalloc / cudaFree implies.  The intermediate z lives in a fixed array inside the library:
+ * M2_STATIC_SCRATCH_BYTES of device memory on every GPU that loads libm2.so, held until the process exits.
+ *
+ *  - B*T*C*2 bytes must not exceed M2_STATIC_SCRATCH_BYTES, else M2_ERR_UNSUPPORTED (nothing is launched).
+ *  - The call allocates nothing and frees nothing.  The first call on each device looks up the address of
+ *    the array (once per device, kept afterwards); make that first call before any stream capture begins.
+ *  - All calls on a device share the one array.  It keeps whatever the previous call left in it; that is
+ *    harmless because every call overwrites the part it later reads, nothing needs to start at zero.
+ *    Two calls whose kernels overlap on the GPU (different streams without ordering between them) race on it:
+ *    order them on one stream or with events.
+ *  - Arguments, shapes, dtypes and results are otherwise exactly those of m2_block_fwd; z is not returned. */
+#define M2_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
+                            const void* W_up_dev, const void* W_down_dev, void* y_dev, int64_t B, int64_t T,
+                            int64_t C, int32_t nblk, int32_t expand, void* stream);
+
 const char* m2_status_string(int32_t status);
 
 /* Reads (synchronously) the device status word kernels set when a bounded wait expires or a

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libm2.so")
 
 M2_FP32, M2_BF16 = 0, 1
 M2_CAUSAL, M2_CIRCULAR = 0, 1
+M2_STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 M2_TABLE_PERM, M2_TABLE_PERM_INV, M2_TABLE_DIGIT_REV, M2_TABLE_TW_EXP = 0, 1, 2, 16
 M2_OK, M2_ERR_INVALID_ARG, M2_ERR_UNSUPPORTED, M2_ERR_ALIGNMENT, M2_ERR_CUDA, M2_ERR_TIMEOUT, M2_ERR_NO_DEVICE = range(7)
 
@@ -33,6 +34,7 @@ SIGNATURES = {
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp]),
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
+    "m2_block_fwd_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
     "m2_status_string": (ctypes.c_char_p, [_i32]),
     "m2_last_device_status": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "m2_last_kernel_name": (ctypes.c_char_p, [_vp]),
@@ -195,3 +197,16 @@ def m2_block_fwd(plan: Plan, x: torch.Tensor, kf: torch.Tensor, w_short: torch.T
     _check(lib().m2_block_fwd(plan.handle, _ptr(x), _ptr(kf), _ptr(w_short), _ptr(W_up), _ptr(W_down), _ptr(z), _ptr(y),
                               B, T, C, nblk, expand, _stream()), "m2_block_fwd")
     return y, z
+
+
+def m2_block_fwd_static(plan: Plan, x: torch.Tensor, kf: torch.Tensor, w_short: torch.Tensor, W_up: torch.Tensor,
+                        W_down: torch.Tensor, y: torch.Tensor, nblk: int = 4, expand: int = 4):
+    """m2_block_fwd without any allocation inside the library and without a caller-provided scratch: the
+    intermediate lives in a fixed array inside libm2.so (x.numel() * 2 <= M2_STATIC_SCRATCH_BYTES).  The caller
+    passes the output tensor y; calls that overlap on the GPU must be ordered by the caller."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 3
+    assert y.is_cuda and y.dtype == torch.bfloat16 and y.is_contiguous() and y.shape == x.shape
+    B, T, C = x.shape
+    _check(lib().m2_block_fwd_static(plan.handle, _ptr(x), _ptr(kf), _ptr(w_short), _ptr(W_up), _ptr(W_down), _ptr(y),
+                                     B, T, C, nblk, expand, _stream()), "m2_block_fwd_static")
+    return y

@@ -4,12 +4,17 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
 #include "conv_umma.h"
 #include "generic_kernels.h"
 #include "m2_plan.h"
+
+// Scratch of m2_block_fwd_static: the intermediate z of the block forward for callers that cannot
+// allocate.  In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned char g_block_static_scratch[M2_STATIC_SCRATCH_BYTES];
 
 namespace {
 
@@ -109,6 +114,10 @@ int32_t check_conv_args(const m2_plan* plan, const void* x, const void* kf, void
     if (B * H > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
     return M2_OK;
 }
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {nullptr};   // per device: address of g_block_static_scratch
 
 }  // namespace
 
@@ -332,6 +341,51 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;
     plan->last_kernel = "block_generic";
+    plan->launches += 2;
+    return M2_OK;
+}
+
+int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
+                            const void* W_up_dev, const void* W_down_dev, void* y_dev, int64_t B, int64_t T, int64_t C,
+                            int32_t nblk, int32_t expand, void* stream) {
+    if (!plan || !x_dev || !kf_dev || !w_short_dev || !W_up_dev || !W_down_dev || !y_dev) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (B < 0 || C <= 0 || nblk <= 0 || expand <= 0 || C % nblk != 0 || T != plan->N) return M2_ERR_INVALID_ARG;
+    if (plan->dtype != M2_BF16 || plan->p < 2 || plan->p > 3) return M2_ERR_UNSUPPORTED;
+    if (B * T * C * 2 > (int64_t)M2_STATIC_SCRATCH_BYTES) return M2_ERR_UNSUPPORTED;   // z would not fit the fixed array
+    if (!aligned16(x_dev) || !aligned16(kf_dev) || !aligned16(W_up_dev) || !aligned16(W_down_dev) || !aligned16(y_dev))
+        return M2_ERR_ALIGNMENT;
+    if (plan->device >= kMaxDevices) return M2_ERR_UNSUPPORTED;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    // Device address of the array, looked up once per device with that device current (no allocation).
+    void* z = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[plan->device]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_block_static_scratch) != cudaSuccess || !p) {
+                cudaGetLastError();
+                return M2_ERR_CUDA;
+            }
+            g_static_ptr[plan->device] = p;
+        }
+        z = g_static_ptr[plan->device];
+    }
+    if (B == 0) return M2_OK;
+    // Same two launches as m2_block_fwd; the conv + gate kernel writes every element of z[B, T, C] before the
+    // MLP kernel reads it, so the array's previous contents never matter.
+    m2g::ConvShape s = conv_shape(plan, B, C, T);
+    s.stride_b = T * C;
+    s.stride_h = 1;
+    s.stride_e = C;
+    cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z, w_short_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    e = m2g::launch_mlp(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "block_generic_static_scratch";
     plan->launches += 2;
     return M2_OK;
 }

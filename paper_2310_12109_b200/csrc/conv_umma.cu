@@ -47,7 +47,7 @@ constexpr int CONST_BYTES = 20480;
 constexpr int OFF_B1 = OFF_CONST, OFF_B2 = OFF_B1 + 4096, OFF_B3 = OFF_B2 + 2048, OFF_B4 = OFF_B3 + 2048;
 constexpr int OFF_TWA = OFF_B4 + 4096, OFF_TWB = OFF_TWA + 4096;
 constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // per group: bar_x, bar_mma, bar_k, flag (32 B); then tmem ptr
-constexpr int OFF_GROUP = OFF_BAR + 256;
+constexpr int OFF_GROUP = OFF_BAR + 1024;   // keeps every group slice 1024-byte aligned
 constexpr int G_X = 0;               // 2 boxes [n2hi][r][n1][8]            8192
 constexpr int G_A = 8192;            // A2 / A3 / A4                        16384
 constexpr int G_KF = 24576;          // spectrum row of the unit's channel  4096
@@ -216,9 +216,15 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
                 for (int q = 0; q < 4; ++q) w[q] = twA[(4 * j + q) * 16];
                 uint4 pr, pi;
                 cmul_pack8(re + 8 * j, im + 8 * j, w, pr, pi);
+#ifdef M2_EXP_SW128
+                unsigned char* base = smem + G_A + (r >> 1) * 4096 + n2lo * 128 + (((((r & 1) << 2) + j) ^ n2lo) << 4);
+                *reinterpret_cast<uint4*>(base + (0 + n2hi) * 1024) = pr;
+                *reinterpret_cast<uint4*>(base + (2 + n2hi) * 1024) = pi;
+#else
                 unsigned char* base = smem + G_A + (r * 4 + j) * 512 + n2lo * 16;
                 *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = pr;
                 *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = pi;
+#endif
             }
         }
         fence_proxy_async();
@@ -235,8 +241,13 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int s = 0; s < 2; ++s)
+#ifdef M2_EXP_SW128
+                    umma_f16(tmem + T2 + hf * 32, smem_desc_sw128(s_base + G_A + hf * 8192 + s * 2048, 4096, 1024),
+                             smem_desc(s_all + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+#else
                     umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + G_A + hf * 8192 + s * 256, 128, 512),
                              smem_desc(s_all + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+#endif
             umma_commit(bar_mma);
         }
         // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
@@ -502,7 +513,7 @@ cudaError_t create_tables(m2_plan* pl) {
 }
 
 void destroy_tables(m2_plan* pl) {
-    if (!pl->umma) return;
+    if (!pl->umma || !covered(pl)) return;
     Tables* t = reinterpret_cast<Tables*>(pl->umma);
     if (t->d_const) cudaFree(t->d_const);
     delete t;
@@ -545,9 +556,10 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     return M2_OK;
 }
 
-bool has_private_spectrum(const m2_plan* pl) { return pl->umma != nullptr && covered(pl); }
+bool has_private_spectrum(const m2_plan* pl) { return pl->umma != nullptr && (covered(pl) || m2u3::covered(pl)); }
 
 cudaError_t relayout_spectrum(const m2_plan* pl, void* kf, int64_t H, cudaStream_t stream) {
+    if (m2u3::covered(pl)) return m2u3::relayout_spectrum(pl, kf, H, stream);
     if (!has_private_spectrum(pl) || H == 0) return cudaSuccess;
     const long long total = H * 256;
     float4* kfu = reinterpret_cast<float4*>(static_cast<unsigned char*>(kf) + (size_t)H * 512 * 8);

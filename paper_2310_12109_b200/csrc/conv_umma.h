@@ -15,6 +15,20 @@ void destroy_tables(m2_plan* plan);
 int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
                  int32_t mode, cudaStream_t stream);
 
+}  // namespace m2u
+
+// Order-3 kernel for N = 32768 = 32^3, causal n = 16384 (conv_umma3.cu); same contract as m2u.
+namespace m2u3 {
+bool covered(const m2_plan* plan);
+cudaError_t create_tables(m2_plan* plan);
+void destroy_tables(m2_plan* plan);
+cudaError_t relayout_spectrum(const m2_plan* plan, void* kf, int64_t H, cudaStream_t stream);
+int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
+                 int32_t mode, cudaStream_t stream);
+}  // namespace m2u3
+
+namespace m2u {
+
 // Plans the tensor-core path covers keep a second copy of the spectrum in the layout its kernel
 // reads (appended to the plan-order copy); relayout_spectrum fills it.
 bool has_private_spectrum(const m2_plan* plan);

@@ -1,0 +1,573 @@
+// Tensor-core Monarch convolution, order 3, N = 32768 = 32 x 32 x 32, causal with n = 16384, bf16 in /
+// fp32 accumulate / bf16 out (the long M2-GPT-shaped mixer).
+//
+// y = Re( M^-1 ( k_f (.) M pad(x) ) ), M = F_N as an order-3 Monarch matrix (Eq. 1, Eq. 2; App. D.6
+// "p-variate Monarch"; Corollary "DFT is M" generalised: stage a contracts digit n_a with F_32 after a
+// twiddle diagonal).  One CTA per SM works on one PAIR of batch rows of the same channel at a time:
+// because the kernel k is real, the two real rows ride as the real and imaginary part of one complex
+// row (F^-1(F(xa + i xb) . k_f) = ya + i yb), which halves every stage.  Zero padding makes the upper
+// half of digit n1 zero on the way in and unneeded on the way out, so the first stage has K = 32 and
+// the last N = 32.
+//
+// A stage is 8 UMMA tiles (M = 128 lanes = 128 values of the two digits that are not being contracted,
+// N = 64 = (re|im) x 32 outputs, K = 64 = (re|im) x 32 inputs); the 8 accumulators fill the 512 TMEM
+// columns.  After each stage all 512 threads read their lanes back, apply the twiddle (or the
+// spectrum) in fp32, round to bf16 and write the next stage's A operand straight into its UMMA layout
+// in the one 128 KB operand buffer -- that write is the stride permutation.  Lane orders are chosen so
+// that the eight lanes of a quarter-warp always land in one 128-byte swizzle row (128B-swizzled,
+// M-major operands) or in one core matrix (K-major operand of the first inverse stage): conflict-free.
+//
+//   stage   contracts   lanes of D (tile j, lane t)                      hand-off after it
+//   S1      n1 (K=32)   n2 = 4j + t/32, n3 = t%32                        w_1024^{n2 k1}            -> A2
+//   S2      n2          k1 = 8(2(j&1)+t/64) + t%8, n3 = 8(j/2) + (t/8)%8 w_N^{n3 (k1 + 32 k2)}     -> A3
+//   S3      n3          k2 = 8(2(j&1)+t/64) + t%8, k1 = 8(j/2) + (t/8)%8 spectrum k_f              -> A4 (K-major)
+//   S3'     k3          same lanes, columns n3                           conj w_N^{n3 (k1+32 k2)}  -> A5
+//   S2'     k2          n3 = 8(2(j&1)+t/64) + t%8, k1 = 8(j/2) + (t/8)%8 conj w_1024^{n2 k1}       -> A6
+//   S1'     k1 (N=32)   n2 = 8(j/2) + t%8, n3 = 8(2(j&1)+t/64) + (t/8)%8 round, stage, bulk store
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "conv_umma.h"
+#include "ptx_sm100.cuh"
+
+namespace m2u3 {
+
+using namespace sm100;
+
+constexpr int kThreads = 512;
+constexpr int kN = 32768;
+// shared memory map
+constexpr int OFF_A = 0;                 // operand buffer (also the output staging)   131072
+constexpr int OFF_X = 131072;            // packed input pair, S1's A operand            65536
+constexpr int OFF_CONST = 196608;        // B1 4096 | BF 8192 | BI 8192 | B6 4096 | tw 8704
+constexpr int CONST_BYTES = 4096 + 8192 + 8192 + 4096 + 8704;
+constexpr int OFF_B1 = OFF_CONST, OFF_BF = OFF_B1 + 4096, OFF_BI = OFF_BF + 8192, OFF_B6 = OFF_BI + 8192;
+constexpr int OFF_TW = OFF_B6 + 4096;    // w_1024^{a b}, rows padded to 34 entries
+constexpr int TW_STRIDE = 34;
+constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // bar_mma, flag, tmem ptr
+constexpr int SMEM_BYTES = OFF_BAR + 64;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+
+struct Tables {
+    void* d_const = nullptr;   // CONST_BYTES
+    float2* d_tn = nullptr;    // w_N^{a b}, a, b < 32, row stride 32
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float2 cmul(float2 a, float2 b) { return make_float2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x); }
+__device__ __forceinline__ float2 conjf(float2 a) { return make_float2(a.x, -a.y); }
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t ssrc, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes) : "memory");
+}
+
+// 128-byte-swizzled M-major operand: 64-element M blocks 8192 B apart, groups of 8 K rows 1024 B apart
+__device__ __forceinline__ uint32_t a_off(int mb, int kgroup, int krow, int mchunk) {
+    return (uint32_t)(mb * 8192 + kgroup * 1024 + krow * 128 + ((mchunk ^ krow) << 4));
+}
+
+// reads the 64 columns (re 0..31 | im 32..63) of this thread's lane in one accumulator tile
+__device__ __forceinline__ void load_tile(uint32_t taddr, float* re, float* im) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        tmem_ld8(taddr + 8 * i, re + 8 * i);
+        tmem_ld8(taddr + 32 + 8 * i, im + 8 * i);
+    }
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        tmem_ld_fence8(re + 8 * i);
+        tmem_ld_fence8(im + 8 * i);
+    }
+}
+
+// 8 complex values (re, im) -> two 16-byte chunks of bf16
+__device__ __forceinline__ void pack8(const float* re, const float* im, uint4& pr, uint4& pi) {
+    pr = make_uint4(pack_bf16(re[0], re[1]), pack_bf16(re[2], re[3]), pack_bf16(re[4], re[5]), pack_bf16(re[6], re[7]));
+    pi = make_uint4(pack_bf16(im[0], im[1]), pack_bf16(im[2], im[3]), pack_bf16(im[4], im[5]), pack_bf16(im[6], im[7]));
+}
+
+// multiplies the 32 complex values by f0 * rho^i, i = 0..31 (four chains of eight)
+__device__ __forceinline__ void mul_geometric(float* re, float* im, float2 f0, float2 rho, float2 rho8, float2 rho16, float2 rho24) {
+    float2 f[4] = {f0, cmul(f0, rho8), cmul(f0, rho16), cmul(f0, rho24)};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int e = 8 * c + i;
+            const float a = re[e], b = im[e];
+            re[e] = a * f[c].x - b * f[c].y;
+            im[e] = a * f[c].y + b * f[c].x;
+            f[c] = cmul(f[c], rho);
+        }
+    }
+}
+
+// loads one packed input pair (rows a and b of channel h) into the S1 operand layout
+__device__ __forceinline__ void load_pair(uint32_t s_x, const __nv_bfloat16* xa, const __nv_bfloat16* xb, bool has_b) {
+    // 4096 chunks of 16 bytes: chunk = (c, n1 < 16, pc = p / 8)
+    for (int ch = threadIdx.x; ch < 4096; ch += kThreads) {
+        const int pc = ch & 127, n1 = (ch >> 7) & 15, c = ch >> 11;
+        const int k = c * 16 + n1;
+        const uint32_t dst = s_x + (uint32_t)((pc >> 3) * 4096 + (k >> 3) * 1024 + (k & 7) * 128 + (((pc & 7) ^ (k & 7)) << 4));
+        const __nv_bfloat16* src = (c == 0 ? xa : xb) + n1 * 1024 + pc * 8;
+        cp_async16(dst, (c == 0 || has_b) ? (const void*)src : (const void*)xa, (c == 0 || has_b) ? 16u : 0u);
+    }
+    cp_async_commit();
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y, const float4* __restrict__ kfu,
+               const uint4* __restrict__ consts, const float2* __restrict__ tn, int B, int H, int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x;
+    const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t bar_mma = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 16;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8);
+    const size_t row_elems = 16384;
+
+    const int bpairs = (B + 1) / 2;
+    const int pairs = H * bpairs;
+    int pr_i = blockIdx.x;
+    if (tid == 0) {
+        mbar_init(bar_mma, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (pr_i < pairs) {
+        const int h = pr_i / bpairs, b0 = (pr_i % bpairs) * 2;
+        load_pair(s_base + OFF_X, x + ((size_t)b0 * H + h) * row_elems, x + ((size_t)(b0 + 1) * H + h) * row_elems, b0 + 1 < B);
+    }
+    {
+        uint4* dst = reinterpret_cast<uint4*>(smem + OFF_CONST);
+        for (int i = tid; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
+    }
+    if (tid < 32) tmem_alloc(s_tptr, 512);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 16);
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const float2* tw = reinterpret_cast<const float2*>(smem + OFF_TW);   // w_1024^{a b} at [a * 34 + b]
+
+    constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
+    constexpr uint32_t ID_MM = instr_desc_bf16(128, 64, true, false);    // M-major A, N = 64
+    constexpr uint32_t ID_KM = instr_desc_bf16(128, 64, false, false);   // K-major A, N = 64
+    constexpr uint32_t ID_S6 = instr_desc_bf16(128, 32, true, false);    // last stage, N = 32
+
+    uint32_t ph = 0;
+    bool ok = true, aborted = false, store_pending = false;
+
+#define M2_STAGE_SYNC()                                   \
+    fence_proxy_async();                                  \
+    tc_fence_before();                                    \
+    if (__syncthreads_or(!ok)) {                          \
+        aborted = true;                                   \
+        break;                                            \
+    }
+#define M2_WAIT_MMA()                  \
+    ok = mbar_wait(bar_mma, ph);       \
+    ph ^= 1;                           \
+    tc_fence_after();
+
+    for (; pr_i < pairs; pr_i += gridDim.x) {
+        const int h = pr_i / bpairs, b0 = (pr_i % bpairs) * 2;
+        const bool has_b = b0 + 1 < B;
+        // the pair's input has landed (every thread waits for its own copies, then the block syncs)
+        cp_async_wait_all();
+        M2_STAGE_SYNC()
+        // ---- S1: contract n1 (K = 32: the zero half is skipped) -----------------------------------------
+        if (tid == 0) {
+            if (store_pending) {   // the previous pair's output staging must be read out before A is reused
+                tma_store_wait_read0();
+                store_pending = false;
+            }
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int s = 0; s < 2; ++s)
+                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_X + j * 8192 + s * 2048, 4096, 1024),
+                             smem_desc(s_base + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
+            umma_commit(bar_mma);
+        }
+        M2_WAIT_MMA()
+        {   // the input buffer is free again: start fetching the next pair
+            const int nx = pr_i + gridDim.x;
+            if (ok && nx < pairs) {
+                const int hn = nx / bpairs, bn = (nx % bpairs) * 2;
+                load_pair(s_base + OFF_X, x + ((size_t)bn * H + hn) * row_elems, x + ((size_t)(bn + 1) * H + hn) * row_elems, bn + 1 < B);
+            }
+        }
+        // ---- h1: w_1024^{n2 k1}; A2[(n3, k1)][(c, n2)] -----------------------------------------------------
+        if (ok) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = wg + 4 * jj;
+                const int n2 = 4 * j + (t >> 5), n3 = t & 31;
+                float re[32], im[32];
+                load_tile(t_lane + j * 64, re, im);
+                const float4* twr = reinterpret_cast<const float4*>(tw + n2 * TW_STRIDE);   // warp-uniform row
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const float4 w = twr[q];
+                    const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+                    re[2 * q] = a0 * w.x - b0v * w.y;
+                    im[2 * q] = a0 * w.y + b0v * w.x;
+                    re[2 * q + 1] = a1 * w.z - b1 * w.w;
+                    im[2 * q + 1] = a1 * w.w + b1 * w.z;
+                }
+#pragma unroll
+                for (int hi = 0; hi < 4; ++hi) {
+                    uint4 pr, pi;
+                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    const int mb = (n3 >> 3) * 4 + hi;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (n2 >> 3), n2 & 7, n3 & 7)) = pr;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (n2 >> 3), n2 & 7, n3 & 7)) = pi;
+                }
+            }
+        }
+        M2_STAGE_SYNC()
+        // ---- S2: contract n2 -----------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                             smem_desc(s_base + OFF_BF + s * 256, 128, 1024), ID_MM, s > 0);
+            umma_commit(bar_mma);
+        }
+        M2_WAIT_MMA()
+        // ---- h2: w_N^{n3 (k1 + 32 k2)} = w_N^{n3 k1} (w_1024^{n3})^{k2}; A3[(k1, k2)][(c, n3)] --------------------
+        if (ok) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = wg + 4 * jj;
+                const int k1 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), n3 = ((j >> 1) << 3) + ((t >> 3) & 7);
+                float re[32], im[32];
+                load_tile(t_lane + j * 64, re, im);
+                const float2* r3 = tw + n3 * TW_STRIDE;
+                mul_geometric(re, im, __ldg(tn + n3 * 32 + k1), r3[1], r3[8], r3[16], r3[24]);
+#pragma unroll
+                for (int hi = 0; hi < 4; ++hi) {
+                    uint4 pr, pi;
+                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    const int mb = (k1 >> 3) * 4 + hi;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (n3 >> 3), n3 & 7, k1 & 7)) = pr;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (n3 >> 3), n3 & 7, k1 & 7)) = pi;
+                }
+            }
+        }
+        M2_STAGE_SYNC()
+        // ---- S3: contract n3 -----------------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                             smem_desc(s_base + OFF_BF + s * 256, 128, 1024), ID_MM, s > 0);
+            umma_commit(bar_mma);
+        }
+        M2_WAIT_MMA()
+        // ---- h3: spectrum multiply (k_f holds 1/N); A4 K-major: row = lane, K = (c, k3) ---------------------------
+        if (ok) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = wg + 4 * jj;
+                float re[32], im[32];
+                const float4* kp = kfu + ((size_t)(h * 8 + j) * 16) * 128 + t;
+                float4 w[4], wn[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = __ldg(kp + q * 128);
+                load_tile(t_lane + j * 64, re, im);
+                unsigned char* rowp = smem + OFF_A + j * 16384 + (t >> 3) * 1024 + (t & 7) * 16;
+#pragma unroll
+                for (int hi = 0; hi < 4; ++hi) {
+                    if (hi < 3) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) wn[q] = __ldg(kp + (4 * (hi + 1) + q) * 128);
+                    }
+                    uint32_t r_[4], i_[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 ww = w[q];
+                        const float a0 = re[8 * hi + 2 * q], b0v = im[8 * hi + 2 * q], a1 = re[8 * hi + 2 * q + 1], b1 = im[8 * hi + 2 * q + 1];
+                        r_[q] = pack_bf16(a0 * ww.x - b0v * ww.y, a1 * ww.z - b1 * ww.w);
+                        i_[q] = pack_bf16(a0 * ww.y + b0v * ww.x, a1 * ww.w + b1 * ww.z);
+                    }
+                    *reinterpret_cast<uint4*>(rowp + hi * 128) = make_uint4(r_[0], r_[1], r_[2], r_[3]);
+                    *reinterpret_cast<uint4*>(rowp + (4 + hi) * 128) = make_uint4(i_[0], i_[1], i_[2], i_[3]);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) w[q] = wn[q];
+                }
+            }
+        }
+        M2_STAGE_SYNC()
+        // ---- S3': contract k3 with conj F ---------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + j * 64, smem_desc(s_base + OFF_A + j * 16384 + s * 256, 128, 1024),
+                             smem_desc(s_base + OFF_BI + s * 256, 128, 1024), ID_KM, s > 0);
+            umma_commit(bar_mma);
+        }
+        M2_WAIT_MMA()
+        // ---- h4: conj w_N^{n3 (k1 + 32 k2)}; A5[(k1, n3)][(c, k2)] -----------------------------------------------------
+        if (ok) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = wg + 4 * jj;
+                const int k2 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
+                float re[32], im[32];
+                load_tile(t_lane + j * 64, re, im);
+                // rho^m = conj( w_N^{m k1} w_1024^{m k2} ), m = 1, 8, 16, 24
+                const float2 rho = conjf(cmul(__ldg(tn + 1 * 32 + k1), tw[1 * TW_STRIDE + k2]));
+                const float2 rho8 = conjf(cmul(__ldg(tn + 8 * 32 + k1), tw[8 * TW_STRIDE + k2]));
+                const float2 rho16 = conjf(cmul(__ldg(tn + 16 * 32 + k1), tw[16 * TW_STRIDE + k2]));
+                const float2 rho24 = conjf(cmul(__ldg(tn + 24 * 32 + k1), tw[24 * TW_STRIDE + k2]));
+                mul_geometric(re, im, make_float2(1.f, 0.f), rho, rho8, rho16, rho24);
+#pragma unroll
+                for (int hi = 0; hi < 4; ++hi) {
+                    uint4 pr, pi;
+                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    const int mb = (k1 >> 3) * 4 + hi;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (k2 >> 3), k2 & 7, k1 & 7)) = pr;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (k2 >> 3), k2 & 7, k1 & 7)) = pi;
+                }
+            }
+        }
+        M2_STAGE_SYNC()
+        // ---- S2': contract k2 with conj F ---------------------------------------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                             smem_desc(s_base + OFF_BI + s * 256, 128, 1024), ID_MM, s > 0);
+            umma_commit(bar_mma);
+        }
+        M2_WAIT_MMA()
+        // ---- h5: conj w_1024^{n2 k1}; A6[(n2, n3)][(c, k1)] --------------------------------------------------------------
+        if (ok) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = wg + 4 * jj;
+                const int n3 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
+                float re[32], im[32];
+                load_tile(t_lane + j * 64, re, im);
+                const float4* twr = reinterpret_cast<const float4*>(tw + k1 * TW_STRIDE);
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const float4 w = twr[q];   // conjugate: (a + ib)(c - is)
+                    const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+                    re[2 * q] = a0 * w.x + b0v * w.y;
+                    im[2 * q] = b0v * w.x - a0 * w.y;
+                    re[2 * q + 1] = a1 * w.z + b1 * w.w;
+                    im[2 * q + 1] = b1 * w.z - a1 * w.w;
+                }
+#pragma unroll
+                for (int hi = 0; hi < 4; ++hi) {
+                    uint4 pr, pi;
+                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    const int mb = hi * 4 + (n3 >> 3);
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (k1 >> 3), k1 & 7, n3 & 7)) = pr;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (k1 >> 3), k1 & 7, n3 & 7)) = pi;
+                }
+            }
+        }
+        M2_STAGE_SYNC()
+        // ---- S1': contract k1 with conj F, outputs n1 < 16 only (N = 32) ----------------------------------------------
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                             smem_desc(s_base + OFF_B6 + s * 256, 128, 1024), ID_S6, s > 0);
+            umma_commit(bar_mma);
+        }
+        M2_WAIT_MMA()
+        // ---- h6: round; stage both rows in the (now free) operand buffer; bulk store ------------------------------------
+        if (ok) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = wg + 4 * jj;
+                const int n2 = ((j >> 1) << 3) + (t & 7), n3 = ((2 * (j & 1) + (t >> 6)) << 3) + ((t >> 3) & 7);
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) tmem_ld8(t_lane + j * 64 + 8 * i, v + 8 * i);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) tmem_ld_fence8(v + 8 * i);
+                __nv_bfloat16* oa = reinterpret_cast<__nv_bfloat16*>(smem + OFF_A) + n2 * 32 + n3;
+#pragma unroll
+                for (int n1 = 0; n1 < 16; ++n1) {
+                    oa[n1 * 1024] = __float2bfloat16_rn(v[n1]);
+                    oa[16384 + n1 * 1024] = __float2bfloat16_rn(v[16 + n1]);
+                }
+            }
+        }
+        M2_STAGE_SYNC()
+        if (tid == 0) {
+            bulk_store(y + ((size_t)b0 * H + h) * row_elems, s_base + OFF_A, 32768);
+            if (has_b) bulk_store(y + ((size_t)(b0 + 1) * H + h) * row_elems, s_base + OFF_A + 32768, 32768);
+            tma_store_commit();
+            store_pending = true;
+        }
+    }
+#undef M2_STAGE_SYNC
+#undef M2_WAIT_MMA
+    // ---- teardown ---------------------------------------------------------------------------------------------------
+    cp_async_wait_all();
+    if (tid == 0) {
+        if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+        tma_store_wait_all0();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid < 32) tmem_dealloc(tmem, 512);
+}
+
+// spectrum in the layout h3 reads: kfu[h][tile j][q = k3 / 2][lane t] = (re, im)(k3 = 2q), (re, im)(k3 = 2q + 1)
+// for (k1, k2) = lane map of D3; plan order is [k1][k2][k3].
+__global__ void relayout_spectrum3_kernel(const float2* __restrict__ kf, float4* __restrict__ kfu, long long total) {
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 8 * 16 * 128
+    if (i >= total) return;
+    const int t = (int)(i & 127), q = (int)((i >> 7) & 15), j = (int)((i >> 11) & 7);
+    const long long h = i >> 14;
+    const int k2 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
+    const float2* src = kf + h * kN + (k1 * 32 + k2) * 32 + 2 * q;
+    kfu[i] = make_float4(src[0].x, src[0].y, src[1].x, src[1].y);
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------------
+
+static uint16_t bf16_bits(double v) {
+    float f = (float)v;
+    uint32_t b;
+    std::memcpy(&b, &f, 4);
+    b += 0x7FFFu + ((b >> 16) & 1u);
+    return (uint16_t)(b >> 16);
+}
+// K-major operand image of an [N][K] matrix (8 x 8 core matrices, K-adjacent 128 B apart)
+static void put_kmajor(std::vector<uint16_t>& img, int K, int n, int k, double v) {
+    const size_t byte = (size_t)(n / 8) * (K / 8) * 128 + (size_t)(k / 8) * 128 + (n % 8) * 16 + (k % 8) * 2;
+    img[byte / 2] = bf16_bits(v);
+}
+
+bool covered(const m2_plan* pl) {
+    return pl->dtype == M2_BF16 && pl->p == 3 && pl->dims[0] == 32 && pl->dims[1] == 32 && pl->dims[2] == 32;
+}
+
+cudaError_t create_tables(m2_plan* pl) {
+    if (!covered(pl)) return cudaSuccess;
+    const double sg = pl->sign >= 0 ? 1.0 : -1.0;
+    std::vector<uint16_t> B1(2048), BF(4096), BI(4096), B6(2048);
+    // complex 32-point DFT as a real matrix: in (a + ib), F = cs + i sn:  re = cs a - sn b,  im = sn a + cs b
+    auto fill = [&](std::vector<uint16_t>& img, int K, int n_out, int n_in, bool inverse) {
+        for (int co = 0; co < 2; ++co)
+            for (int o = 0; o < n_out; ++o)
+                for (int ci = 0; ci < 2; ++ci)
+                    for (int i = 0; i < n_in; ++i) {
+                        const double th = 2.0 * M_PI * ((o * i) % 32) / 32.0;
+                        const double cs = std::cos(th), sn = (inverse ? -sg : sg) * std::sin(th);
+                        const double v = co == 0 ? (ci == 0 ? cs : -sn) : (ci == 0 ? sn : cs);
+                        put_kmajor(img, K, co * n_out + o, ci * n_in + i, v);
+                    }
+    };
+    fill(B1, 32, 32, 16, false);   // [N = (c, k1) 64][K = (c, n1 < 16) 32]
+    fill(BF, 64, 32, 32, false);   // [64][64]
+    fill(BI, 64, 32, 32, true);    // conjugate
+    fill(B6, 64, 16, 32, true);    // [N = (c, n1 < 16) 32][K = (c, k1) 64], conjugate
+    std::vector<float> tw(32 * TW_STRIDE * 2, 0.f), tn(32 * 32 * 2);
+    for (int a = 0; a < 32; ++a)
+        for (int b = 0; b < 32; ++b) {
+            const double t1 = 2.0 * M_PI * ((a * b) % 1024) / 1024.0, t2 = 2.0 * M_PI * ((a * b) % kN) / (double)kN;
+            tw[(a * TW_STRIDE + b) * 2] = (float)std::cos(t1);
+            tw[(a * TW_STRIDE + b) * 2 + 1] = (float)(sg * std::sin(t1));
+            tn[(a * 32 + b) * 2] = (float)std::cos(t2);
+            tn[(a * 32 + b) * 2 + 1] = (float)(sg * std::sin(t2));
+        }
+    std::vector<unsigned char> blob(CONST_BYTES);
+    std::memcpy(blob.data(), B1.data(), 4096);
+    std::memcpy(blob.data() + 4096, BF.data(), 8192);
+    std::memcpy(blob.data() + 12288, BI.data(), 8192);
+    std::memcpy(blob.data() + 20480, B6.data(), 4096);
+    std::memcpy(blob.data() + 24576, tw.data(), 8704);
+    Tables* tb = new Tables();
+    cudaError_t e = cudaMalloc(&tb->d_const, CONST_BYTES);
+    if (e == cudaSuccess) e = cudaMemcpy(tb->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&tb->d_tn, tn.size() * sizeof(float));
+    if (e == cudaSuccess) e = cudaMemcpy(tb->d_tn, tn.data(), tn.size() * sizeof(float), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv32k_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) {
+        if (tb->d_const) cudaFree(tb->d_const);
+        if (tb->d_tn) cudaFree(tb->d_tn);
+        delete tb;
+        return e;
+    }
+    pl->umma = reinterpret_cast<m2_umma_tables*>(tb);
+    return cudaSuccess;
+}
+
+void destroy_tables(m2_plan* pl) {
+    if (!pl->umma || !covered(pl)) return;
+    Tables* tb = reinterpret_cast<Tables*>(pl->umma);
+    if (tb->d_const) cudaFree(tb->d_const);
+    if (tb->d_tn) cudaFree(tb->d_tn);
+    delete tb;
+    pl->umma = nullptr;
+}
+
+cudaError_t relayout_spectrum(const m2_plan* pl, void* kf, int64_t H, cudaStream_t stream) {
+    if (!pl->umma || !covered(pl) || H == 0) return cudaSuccess;
+    const long long total = H * 16384;
+    float4* kfu = reinterpret_cast<float4*>(static_cast<unsigned char*>(kf) + (size_t)H * kN * 8);
+    relayout_spectrum3_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>((const float2*)kf, kfu, total);
+    return cudaGetLastError();
+}
+
+int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
+                 cudaStream_t stream) {
+    if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (mode != M2_CAUSAL || n != 16384) return M2_ERR_UNSUPPORTED;
+    Tables* tb = reinterpret_cast<Tables*>(pl->umma);
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long pairs = H * ((B + 1) / 2);
+    const int grid = (int)(pairs < sms ? pairs : sms);
+    const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * kN * 8);
+    conv32k_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, kfu,
+                                                           (const uint4*)tb->d_const, tb->d_tn, (int)B, (int)H, pl->d_status);
+    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    pl->last_kernel = "conv_umma_o3_32k";
+    pl->launches += 1;
+    return M2_OK;
+}
+
+}  // namespace m2u3

@@ -161,6 +161,7 @@ int32_t m2_plan_create(m2_plan** out, int64_t N, int32_t p, const int32_t* facto
                  cudaMemcpy(pl->d_roots[a], r.data(), sizeof(float2) * Na, cudaMemcpyHostToDevice) == cudaSuccess;
         }
         if (ok) ok = m2u::create_tables(pl) == cudaSuccess;
+        if (ok) ok = m2u3::create_tables(pl) == cudaSuccess;
         if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
         if (!ok) {
             cudaGetLastError();
@@ -178,6 +179,7 @@ int32_t m2_plan_destroy(m2_plan* plan) {
         DeviceGuard g(plan->device);
         cudaDeviceSynchronize();
         m2u::destroy_tables(plan);
+        m2u3::destroy_tables(plan);
         if (plan->d_status) cudaFree(plan->d_status);
         for (int a = 0; a < 4; ++a)
             if (plan->d_roots[a]) cudaFree(plan->d_roots[a]);
@@ -241,6 +243,7 @@ int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* 
     if (B * H == 0) return M2_OK;
     // tensor-core path where a kernel exists for the shape, CUDA-core path otherwise
     int32_t ust = m2u::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
+    if (ust == M2_ERR_UNSUPPORTED) ust = m2u3::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
     if (ust == M2_OK) return M2_OK;
     if (ust != M2_ERR_UNSUPPORTED) return ust;
     m2g::ConvShape s = conv_shape(plan, B, H, n);

@@ -122,6 +122,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)1 << 46;  // descriptor version of this architecture
     return d;                // base offset 0, layout type 0 = no swizzle
 }
+// Same with the 128-byte swizzle (16-byte chunk index XOR row index inside 1024-byte atoms of 8 rows x 128 B).
+//   MN-major: a row = 64 consecutive M/N elements of one K index; LBO = step between 64-element M/N blocks,
+//             SBO = step between groups of 8 K indices.
+//   K-major : a row = 64 consecutive K elements of one M/N index; SBO = step between groups of 8 M/N indices.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return smem_desc(addr, lbo_bytes, sbo_bytes) | ((uint64_t)2 << 61);
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, dense.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
     return (1u << 4)                          // D format: fp32

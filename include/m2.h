@@ -101,11 +101,16 @@ int32_t m2_monarch_conv_fwd_host(const m2_plan* plan, const void* x_host, const 
  * blockdiag_matmul listing, [block][out][in]):
  *   y[t][k2*N1 + k1] = sum_{n2} L[k1][k2][n2] * sum_{n1} R[n2][k1][n1] * x[t][n1*N2 + n2].
  * X_dev, Y_dev: [T, N] in the plan dtype; L_dev: [N1][N2][N2], R_dev: [N2][N1][N1], same dtype.
- * R is applied first.  (The listing's parameter called L is applied first and so plays R's role.) */
+ * R is applied first.  (The listing's parameter called L is applied first and so plays R's role.)
+ * ws_dev: caller-owned device workspace of at least m2_matmul_workspace_bytes(plan, T) bytes for the
+ * intermediate between the two factors (16-byte aligned); with ws_dev == NULL or ws_bytes too small the
+ * call uses the slower kernels that need none. */
+int64_t m2_matmul_workspace_bytes(const m2_plan* plan, int64_t T);
 int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev,
-                          void* Y_dev, int64_t T, void* stream);
+                          void* Y_dev, int64_t T, void* ws_dev, int64_t ws_bytes, void* stream);
 int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const void* L_dev, const void* R_dev,
-                               void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* stream);
+                               void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* ws_dev,
+                               int64_t ws_bytes, void* stream);
 
 /* M2 block forward for the M2-BERT-base shape (Eq. 2-3; Sec. 5.1): along the sequence, per channel,
  * v = circular Monarch conv of x with the channel's kernel; gate g = depthwise conv of width 3

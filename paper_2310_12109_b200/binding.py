@@ -31,8 +31,9 @@ SIGNATURES = {
     "m2_spectrum_to_natural": (_i32, [_vp, _vp, _i64, _vp, _vp]),
     "m2_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
-    "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp]),
-    "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
+    "m2_matmul_workspace_bytes": (_i64, [_vp, _i64]),
+    "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
+    "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
     "m2_block_fwd_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
     "m2_status_string": (ctypes.c_char_p, [_i32]),
@@ -167,22 +168,36 @@ def m2_monarch_conv_fwd_host(plan: Plan, x_host: torch.Tensor, kf: torch.Tensor,
     return y_host
 
 
-def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tensor, Y: torch.Tensor | None = None):
-    """X: [T, N]; L: [N1, N2, N2]; R: [N2, N1, N1]; all CUDA, plan dtype."""
+def m2_matmul_workspace(plan: Plan, T: int, device=None):
+    """Device workspace for m2_monarch_matmul (None if the plan's kernels need none)."""
+    nbytes = int(lib().m2_matmul_workspace_bytes(plan.handle, T))
+    if nbytes <= 0:
+        return None
+    return torch.empty(nbytes, dtype=torch.uint8, device=device if device is not None else f"cuda:{plan.device}")
+
+
+def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tensor, Y: torch.Tensor | None = None,
+                      ws: torch.Tensor | None = None):
+    """X: [T, N]; L: [N1, N2, N2]; R: [N2, N1, N1]; all CUDA, plan dtype.  ws: m2_matmul_workspace(plan, T)."""
     for t in (X, L, R):
         assert t.is_cuda and t.dtype == plan.torch_dtype and t.is_contiguous()
     N1, N2 = plan.dims
     assert X.dim() == 2 and X.shape[1] == plan.N and tuple(L.shape) == (N1, N2, N2) and tuple(R.shape) == (N2, N1, N1)
     if Y is None:
         Y = torch.empty_like(X)
-    _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _stream()),
-           "m2_monarch_matmul")
+    if ws is None:
+        ws = m2_matmul_workspace(plan, X.shape[0], X.device)
+    _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _ptr(ws),
+                                   0 if ws is None else ws.numel(), _stream()), "m2_monarch_matmul")
     return Y
 
 
-def m2_monarch_matmul_host(plan: Plan, X_host, L, R, Y_host, X_scratch, Y_scratch):
+def m2_monarch_matmul_host(plan: Plan, X_host, L, R, Y_host, X_scratch, Y_scratch, ws: torch.Tensor | None = None):
+    if ws is None:
+        ws = m2_matmul_workspace(plan, X_host.shape[0], X_scratch.device)
     _check(lib().m2_monarch_matmul_host(plan.handle, _ptr(X_host), _ptr(L), _ptr(R), _ptr(Y_host), _ptr(X_scratch),
-                                        _ptr(Y_scratch), X_host.shape[0], _stream()), "m2_monarch_matmul_host")
+                                        _ptr(Y_scratch), X_host.shape[0], _ptr(ws), 0 if ws is None else ws.numel(),
+                                        _stream()), "m2_monarch_matmul_host")
     return Y_host
 
 

@@ -10,6 +10,7 @@
 
 #include "conv_umma.h"
 #include "generic_kernels.h"
+#include "matmul_umma.h"
 #include "m2_plan.h"
 
 // Scratch of m2_block_fwd_static: the intermediate z of the block forward for callers that cannot
@@ -162,6 +163,7 @@ int32_t m2_plan_create(m2_plan** out, int64_t N, int32_t p, const int32_t* facto
         }
         if (ok) ok = m2u::create_tables(pl) == cudaSuccess;
         if (ok) ok = m2u3::create_tables(pl) == cudaSuccess;
+        if (ok) ok = m2mm::prepare(pl) == cudaSuccess;
         if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
         if (!ok) {
             cudaGetLastError();
@@ -284,13 +286,21 @@ static int32_t check_matmul_args(const m2_plan* plan, const void* X, const void*
     return M2_OK;
 }
 
+int64_t m2_matmul_workspace_bytes(const m2_plan* plan, int64_t T) {
+    if (!plan || T < 0) return -1;
+    return m2mm::workspace_bytes(plan, T);
+}
+
 int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, void* Y_dev,
-                          int64_t T, void* stream) {
+                          int64_t T, void* ws_dev, int64_t ws_bytes, void* stream) {
     int32_t st = check_matmul_args(plan, X_dev, L_dev, R_dev, Y_dev, T);
     if (st != M2_OK) return st;
+    if (ws_dev && !aligned16(ws_dev)) return M2_ERR_ALIGNMENT;
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
     if (T == 0) return M2_OK;
+    if (m2mm::covered(plan) && ws_dev && ws_bytes >= m2mm::workspace_bytes(plan, T))
+        return m2mm::matmul(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, (cudaStream_t)stream);
     cudaError_t e = m2g::launch_matmul(plan->dims[0], plan->dims[1], T, plan->dtype == M2_BF16, X_dev, L_dev, R_dev,
                                        Y_dev, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
@@ -301,7 +311,8 @@ int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_
 }
 
 int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const void* L_dev, const void* R_dev,
-                               void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* stream) {
+                               void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* ws_dev,
+                               int64_t ws_bytes, void* stream) {
     if (!X_host || !Y_host) return M2_ERR_INVALID_ARG;
     int32_t st = check_matmul_args(plan, X_dev_scratch, L_dev, R_dev, Y_dev_scratch, T);
     if (st != M2_OK) return st;
@@ -311,7 +322,7 @@ int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const vo
     if (bytes == 0) return M2_OK;
     if (cudaMemcpyAsync(X_dev_scratch, X_host, bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess)
         return M2_ERR_CUDA;
-    st = m2_monarch_matmul(plan, X_dev_scratch, L_dev, R_dev, Y_dev_scratch, T, stream);
+    st = m2_monarch_matmul(plan, X_dev_scratch, L_dev, R_dev, Y_dev_scratch, T, ws_dev, ws_bytes, stream);
     if (st != M2_OK) return st;
     if (cudaMemcpyAsync(Y_host, Y_dev_scratch, bytes, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
         return M2_ERR_CUDA;

@@ -1,0 +1,187 @@
+// Tensor-core order-2 Monarch matmul for 64 x 64 blocks (N = 4096), bf16 in / fp32 accumulate / bf16 out.
+//
+//   y[t][k2*64 + k1] = sum_{n2} L[k1][k2][n2] * sum_{n1} R[n2][k1][n1] * x[t][n1*64 + n2]      (Sec. 3.1)
+//
+// Both block-diagonal factors are batches of 64 independent GEMMs [tokens x 64] x [64 x 64]; the batch
+// index is the CONTIGUOUS index of the data each factor reads (n2 for R, k1 for L after the middle
+// permutation), so neither operand of a tensor-core GEMM can be taken from memory as it lies.  The two
+// factors therefore run as two passes of one kernel that exchange the intermediate z[t][k1][n2] through
+// a workspace (it mostly stays in the 126 MB L2):
+//
+//   pass 1 (R): a CTA owns 128 tokens x 8 consecutive n2.  Threads read 16-byte pieces of x (8 values of
+//               n2 for one (t, n1)), transpose 8 x 8 blocks in registers (the permutation P) and write the
+//               K-major, 128-byte-swizzled UMMA operand A_{n2}[t][n1]; 8 UMMA groups (M = 128 tokens,
+//               N = 64 = k1, K = 64 = n1) fill the 512 TMEM columns; the epilogue gathers, for every k1,
+//               the 8 values of n2 from the 8 accumulators and stores them as one 16-byte piece of
+//               z[t][k1][n2] (the permutation P^T).
+//   pass 2 (L): a CTA owns 128 tokens x 8 consecutive k1; rows z[t][k1][0..63] are already K-major and are
+//               copied into the swizzled operand with cp.async; same UMMAs with L's blocks; the epilogue
+//               stores 16-byte pieces of y[t][k2][k1] (the last permutation P).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "matmul_umma.h"
+#include "ptx_sm100.cuh"
+
+namespace m2mm {
+
+using namespace sm100;
+
+constexpr int kThreads = 512;
+constexpr int kTileT = 128;   // tokens per CTA
+constexpr int kGroup = 8;     // blocks per CTA
+constexpr int OFF_A = 0;                   // 8 operands [128 t][64] bf16, swizzled   131072
+constexpr int OFF_B = 131072;              // 8 weight blocks [64][64] bf16, swizzled   65536
+constexpr int OFF_BAR = 196608;            // bar_mma, tmem ptr
+constexpr int SMEM_BYTES = OFF_BAR + 64;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_wait() {
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// byte offset of 16-byte chunk kc of row r in a K-major operand with 128-byte rows and the 128B swizzle
+__device__ __forceinline__ uint32_t sw_off(int r, int kc) { return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((kc ^ (r & 7)) << 4)); }
+
+// PASS 1: in = x[T][64 n1][64 n2], W = R[n2][k1][n1], out = z[T][64 k1][64 n2]
+// PASS 2: in = z[T][64 k1][64 n2], W = L[k1][k2][n2], out = y[T][64 k2][64 k1]
+template <int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ out,
+                      long long T, int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x;
+    const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t bar_mma = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 16;
+    const long long t0 = (long long)blockIdx.x * kTileT;
+    const int grp = blockIdx.y;   // which 8 consecutive blocks (n2 in pass 1, k1 in pass 2)
+
+    if (tid == 0) {
+        mbar_init(bar_mma, 1);
+        fence_barrier_init();
+    }
+    if (tid < 32) tmem_alloc(s_tptr, 512);
+
+    // weight blocks -> swizzled K-major B operands ([64 out][64 in], rows of 128 bytes)
+    for (int c = tid; c < kGroup * 64 * 8; c += kThreads) {
+        const int kc = c & 7, o = (c >> 3) & 63, bl = c >> 9;
+        cp_async16(s_base + OFF_B + bl * 8192 + sw_off(o, kc), W + ((size_t)(grp * kGroup + bl) * 64 + o) * 64 + kc * 8, 16u);
+    }
+    if (PASS == 1) {
+        // unit = (token tt, group g of 8 consecutive n1): 8 loads of 16 bytes (8 values of n2 each), an 8 x 8
+        // transpose in registers, 8 stores (one per n2) of the 8 n1 values = chunk g of row tt of A_{n2}
+#pragma unroll 1
+        for (int u = tid; u < kTileT * 8; u += kThreads) {
+            const int g = u & 7, tt = u >> 3;
+            uint4 v[8];
+            const bool live = t0 + tt < T;
+            const uint4* src = reinterpret_cast<const uint4*>(in + (size_t)(t0 + tt) * 4096 + (size_t)(8 * g) * 64 + grp * 8);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = live ? __ldg(src + i * 8) : make_uint4(0u, 0u, 0u, 0u);
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(v);   // w[i*4 + j]: n1 = 8g+i, n2 = 2j, 2j+1
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint4 lo, hi;
+                lo.x = prmt(w[0 * 4 + j], w[1 * 4 + j], 0x5410); hi.x = prmt(w[0 * 4 + j], w[1 * 4 + j], 0x7632);
+                lo.y = prmt(w[2 * 4 + j], w[3 * 4 + j], 0x5410); hi.y = prmt(w[2 * 4 + j], w[3 * 4 + j], 0x7632);
+                lo.z = prmt(w[4 * 4 + j], w[5 * 4 + j], 0x5410); hi.z = prmt(w[4 * 4 + j], w[5 * 4 + j], 0x7632);
+                lo.w = prmt(w[6 * 4 + j], w[7 * 4 + j], 0x5410); hi.w = prmt(w[6 * 4 + j], w[7 * 4 + j], 0x7632);
+                *reinterpret_cast<uint4*>(smem + OFF_A + (2 * j) * 16384 + sw_off(tt, g)) = lo;
+                *reinterpret_cast<uint4*>(smem + OFF_A + (2 * j + 1) * 16384 + sw_off(tt, g)) = hi;
+            }
+        }
+    } else {
+        // rows z[t][k1][0..63] are the operand rows already
+        for (int c = tid; c < kGroup * kTileT * 8; c += kThreads) {
+            const int kc = c & 7, bl = (c >> 3) & 7, tt = c >> 6;
+            const bool live = t0 + tt < T;
+            const __nv_bfloat16* src = in + ((size_t)(live ? t0 + tt : 0) * 64 + grp * kGroup + bl) * 64 + kc * 8;
+            cp_async16(s_base + OFF_A + bl * 16384 + sw_off(tt, kc), src, live ? 16u : 0u);
+        }
+    }
+    cp_async_commit_wait();
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 16);
+
+    if (tid == 0) {
+        constexpr uint32_t IDESC = instr_desc_bf16(128, 64, false, false);
+#pragma unroll 1
+        for (int bl = 0; bl < kGroup; ++bl)
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+                umma_f16(tmem + bl * 64, smem_desc_sw128(s_base + OFF_A + bl * 16384 + s * 32, 16, 1024),
+                         smem_desc_sw128(s_base + OFF_B + bl * 8192 + s * 32, 16, 1024), IDESC, s > 0);
+        umma_commit(bar_mma);
+    }
+    const bool ok = mbar_wait(bar_mma, 0);
+    tc_fence_after();
+    // epilogue: lane = token; warpgroup wg takes output columns [16 wg, 16 wg + 16); for every output index o
+    // the 8 accumulators give the 8 consecutive block indices -> one 16-byte piece of out[t][o][grp*8 ..]
+    if (ok) {   // every lane takes part in the warp-wide TMEM loads; only live tokens store
+        const bool live = t0 + t < T;
+        const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+        __nv_bfloat16* orow = out + (size_t)(live ? t0 + t : 0) * 4096 + grp * 8;
+#pragma unroll 1
+        for (int gk = 0; gk < 2; ++gk) {
+            const int o0 = 16 * wg + 8 * gk;
+            float v[8][8];
+#pragma unroll
+            for (int bl = 0; bl < 8; ++bl) tmem_ld8(t_lane + bl * 64 + o0, v[bl]);
+            tmem_ld_wait();
+#pragma unroll
+            for (int bl = 0; bl < 8; ++bl) tmem_ld_fence8(v[bl]);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
+                                           pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
+                if (live) *reinterpret_cast<uint4*>(orow + (size_t)(o0 + kk) * 64) = p;
+            }
+        }
+    }
+    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (tid < 32) tmem_dealloc(tmem, 512);
+}
+
+bool covered(const m2_plan* pl) { return pl->dtype == M2_BF16 && pl->p == 2 && pl->dims[0] == 64 && pl->dims[1] == 64; }
+
+int64_t workspace_bytes(const m2_plan* pl, int64_t T) { return covered(pl) ? T * 4096 * 2 : 0; }
+
+cudaError_t prepare(const m2_plan* pl) {
+    if (!covered(pl)) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(monarch64_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    return e;
+}
+
+int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, cudaStream_t stream) {
+    if (!covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (T == 0) return M2_OK;
+    dim3 grid((unsigned)((T + kTileT - 1) / kTileT), 8);
+    monarch64_pass_kernel<1><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)X, (const __nv_bfloat16*)R,
+                                                                     (__nv_bfloat16*)ws, T, pl->d_status);
+    monarch64_pass_kernel<2><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)ws, (const __nv_bfloat16*)L,
+                                                                     (__nv_bfloat16*)Y, T, pl->d_status);
+    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    pl->last_kernel = "matmul_umma_64x64";
+    pl->launches += 2;
+    return M2_OK;
+}
+
+}  // namespace m2mm

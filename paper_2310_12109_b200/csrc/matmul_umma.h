@@ -1,0 +1,14 @@
+// Tensor-core Monarch matmul for 64 x 64 blocks (internal header).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "m2_plan.h"
+
+namespace m2mm {
+bool covered(const m2_plan* plan);
+int64_t workspace_bytes(const m2_plan* plan, int64_t T);
+cudaError_t prepare(const m2_plan* plan);
+// two passes (R then L) exchanging the intermediate through `ws` (workspace_bytes(plan, T) bytes)
+int32_t matmul(const m2_plan* plan, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws,
+               cudaStream_t stream);
+}  // namespace m2mm

@@ -83,7 +83,7 @@ def test_argument_validation_without_device():
     # a host-only plan refuses device work, null pointers are rejected first
     assert lib.m2_monarch_conv_fwd(h, None, None, None, 1, 1, 256, 0, None) == M.M2_ERR_INVALID_ARG
     assert lib.m2_monarch_conv_fwd(h, 16, 16, 16, 1, 1, 256, 0, None) == M.M2_ERR_NO_DEVICE
-    assert lib.m2_monarch_matmul(h, 16, 16, 16, 16, 4, None) == M.M2_ERR_NO_DEVICE
+    assert lib.m2_monarch_matmul(h, 16, 16, 16, 16, 4, None, 0, None) == M.M2_ERR_NO_DEVICE
     assert lib.m2_kernel_spectrum(h, 16, 1, 256, 16, None) == M.M2_ERR_NO_DEVICE
     assert lib.m2_spectrum_bytes(h, 3) == 3 * 512 * 8
     assert lib.m2_plan_destroy(h) == M.M2_OK

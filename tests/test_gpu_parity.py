@@ -268,7 +268,7 @@ def test_empty_batches_and_error_codes():
     assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr(), kf.data_ptr(), y.data_ptr(), 1, 2, 256, M.M2_CIRCULAR, s) == M.M2_ERR_INVALID_ARG
     assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr() + 2, kf.data_ptr(), y.data_ptr(), 1, 2, 256, M.M2_CAUSAL, s) == M.M2_ERR_ALIGNMENT
     assert lib.m2_monarch_conv_fwd(plan.handle, x.data_ptr(), kf.data_ptr(), y.data_ptr(), 1, 2, 256, 9, s) == M.M2_ERR_INVALID_ARG
-    assert lib.m2_monarch_matmul(plan.handle, x.data_ptr(), x.data_ptr(), x.data_ptr(), None, 1, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_matmul(plan.handle, x.data_ptr(), x.data_ptr(), x.data_ptr(), None, 1, None, 0, s) == M.M2_ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert plan.device_status() == 0
     plan.close()

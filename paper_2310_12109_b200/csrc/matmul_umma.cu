@@ -65,8 +65,10 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
     const uint32_t s_base = smem_u32(smem);
     const uint32_t bar_mma = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 16;
-    const long long t0 = (long long)blockIdx.x * kTileT;
-    const int grp = blockIdx.y;   // which 8 consecutive blocks (n2 in pass 1, k1 in pass 2)
+    // the 8 CTAs that share the 128-byte lines of one token tile are neighbours in launch order, so the
+    // 16-byte pieces of a line are fetched / written while the line is still in L2
+    const long long t0 = (long long)blockIdx.y * kTileT;
+    const int grp = blockIdx.x;   // which 8 consecutive blocks (n2 in pass 1, k1 in pass 2)
 
     if (tid == 0) {
         mbar_init(bar_mma, 1);
@@ -173,7 +175,7 @@ cudaError_t prepare(const m2_plan* pl) {
 int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, cudaStream_t stream) {
     if (!covered(pl)) return M2_ERR_UNSUPPORTED;
     if (T == 0) return M2_OK;
-    dim3 grid((unsigned)((T + kTileT - 1) / kTileT), 8);
+    dim3 grid(8, (unsigned)((T + kTileT - 1) / kTileT));
     monarch64_pass_kernel<1><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)X, (const __nv_bfloat16*)R,
                                                                      (__nv_bfloat16*)ws, T, pl->d_status);
     monarch64_pass_kernel<2><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)ws, (const __nv_bfloat16*)L,

@@ -178,16 +178,24 @@ def time_launches(fn, n, torch):
     return e0.elapsed_time(e1)
 
 
-def side_workloads(torch, M, synth, peaks, quick: bool):
+def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4"), reps=None):
     """Config 3 (Monarch matmul) and config 4 (order-3 causal conv): time per launch, throughput and
     roofline fraction, outside the headline timed region."""
     out = {}
-    reps = 3 if quick else 10
-    # config 3
+    reps = reps if reps is not None else (3 if quick else 10)
+    bf = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)  # noqa: E731
+    if "config3" in which:
+        out.update(_side_config3(torch, M, synth, peaks, reps, bf))
+    if "config4" in which:
+        out.update(_side_config4(torch, M, synth, peaks, reps, bf))
+    return out
+
+
+def _side_config3(torch, M, synth, peaks, reps, bf):
+    out = {}
     T, b = 16384, 64
     c = synth.config3(T=T, b=b)
     plan = M.Plan((b, b), dtype=M.M2_BF16, device=torch.cuda.current_device())
-    bf = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)  # noqa: E731
     L, R = bf(c["L"]), bf(c["R"])
     Xs = [bf(c["X"]) for _ in range(2)]
     Ys = [torch.empty_like(Xs[0]) for _ in range(2)]
@@ -202,8 +210,11 @@ def side_workloads(torch, M, synth, peaks, quick: bool):
         "TFLOPs": fl / (ms * 1e9), "roofline": {"bound": "hbm", "achieved": by / (ms * 1e6), "peak": peaks["hbm_gbs"],
                                                  "unit": "GB/s", "frac": by / (ms * 1e6) / peaks["hbm_gbs"]}}
     plan.close()
-    del Xs, Ys
-    # config 4
+    return out
+
+
+def _side_config4(torch, M, synth, peaks, reps, bf):
+    out = {}
     B, H, n = 4, 1024, 16384
     c = synth.config4(B=B, H=H, n=n)
     plan = M.Plan((32, 32, 32), dtype=M.M2_BF16, device=torch.cuda.current_device())
@@ -213,8 +224,8 @@ def side_workloads(torch, M, synth, peaks, quick: bool):
     f = lambda i: M.m2_monarch_conv_fwd(plan, xs[i % 2], kf, M.M2_CAUSAL, y=ys[i % 2])  # noqa: E731
     time_launches(f, 2, torch)
     ms = time_launches(f, reps, torch) / reps
-    by = 2 * B * H * n * 2 + H * 32768 * 8
-    fl = 2.0 * (2 + 4 + 4) * 32768 * 32 * 2 * B * H   # plain count: real first stage, complex after, fwd + inv
+    by = 2 * B * H * n * 2 + H * 32768 * 8               # x + y (bf16) + fp32 spectrum
+    fl = 2.0 * (2 + 4 + 4) * 32768 * 32 * 2 * B * H      # plain count: real first stage, complex after, fwd + inv
     t_hbm = by / (peaks["hbm_gbs"] * 1e9)
     t_tc = fl / (peaks["bf16_tflops_sustained"] * 1e12)
     bound = "tensor" if t_tc > t_hbm else "hbm"
@@ -222,7 +233,8 @@ def side_workloads(torch, M, synth, peaks, quick: bool):
     pk = peaks["bf16_tflops_sustained"] if bound == "tensor" else peaks["hbm_gbs"]
     out["config4_conv_order3"] = {
         "kernel": plan.last_kernel(), "ms": ms, "tokens_ch_per_s": B * H * n / (ms * 1e-3), "algorithmic_GBps": by / (ms * 1e6),
-        "TFLOPs_plain_count": fl / (ms * 1e9),
+        "TFLOPs_plain_count": fl / (ms * 1e9), "frac_of_hbm_roof": by / (ms * 1e6) / peaks["hbm_gbs"],
+        "note": "plain count; the kernel executes half of it (two real rows packed as one complex row, zero-skip)",
         "roofline": {"bound": bound, "achieved": ach, "peak": pk, "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": ach / pk}}
     plan.close()
     return out
@@ -339,9 +351,19 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-side", action="store_true", help="skip the config-3 / config-4 side measurements")
     ap.add_argument("--quick", action="store_true", help="fewer repetitions of the side measurements")
+    ap.add_argument("--only", default=None, choices=["config3", "config4"],
+                    help="run just this side workload (--steps launches after 2 warm-ups) and print its JSON; used for profiling")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.only:
+        import torch
+        from paper_2310_12109_b200 import binding as M
+        from paper_2310_12109_b200 import build as BLD
+        from paper_2310_12109_b200 import synth
+        BLD.build()
+        torch.cuda.set_device(0)
+        print(json.dumps(side_workloads(torch, M, synth, measured_peaks(), True, which=(args.only,), reps=max(1, args.steps))))
     else:
         run_gpu(args)
 

@@ -5,23 +5,24 @@
 // Both block-diagonal factors are batches of 64 independent GEMMs [tokens x 64] x [64 x 64]; the batch
 // index is the CONTIGUOUS index of the data each factor reads (n2 for R, k1 for L after the middle
 // permutation), so neither operand of a tensor-core GEMM can be taken from memory as it lies.  The two
-// factors therefore run as two passes of one kernel that exchange the intermediate z[t][k1][n2] through
-// a workspace (it mostly stays in the 126 MB L2):
+// factors therefore run as two passes of one kernel that exchange the intermediate through a workspace
+// laid out z[n2 / 8][t][k1][n2 % 8] (it mostly stays in the 126 MB L2):
 //
 //   pass 1 (R): a CTA owns 128 tokens x 8 consecutive n2.  Threads read 16-byte pieces of x (8 values of
 //               n2 for one (t, n1)), transpose 8 x 8 blocks in registers (the permutation P) and write the
 //               K-major, 128-byte-swizzled UMMA operand A_{n2}[t][n1]; 8 UMMA groups (M = 128 tokens,
 //               N = 64 = k1, K = 64 = n1) fill the 512 TMEM columns; the epilogue gathers, for every k1,
-//               the 8 values of n2 from the 8 accumulators and stores them as one 16-byte piece of
-//               z[t][k1][n2] (the permutation P^T).
-//   pass 2 (L): a CTA owns 128 tokens x 8 consecutive k1; rows z[t][k1][0..63] are already K-major and are
-//               copied into the swizzled operand with cp.async; same UMMAs with L's blocks; the epilogue
-//               stores 16-byte pieces of y[t][k2][k1] (the last permutation P).
+//               the 8 values of n2 from the 8 accumulators as one 16-byte piece (the permutation P^T); the
+//               CTA's pieces form one contiguous 128 KB slab of z and leave as bulk copies.
+//   pass 2 (L): a CTA owns 128 tokens x 8 consecutive k1; the pieces of z are chunks of the K-major operand
+//               rows and are copied in with cp.async; same UMMAs with L's blocks; the epilogue stages 16-byte
+//               pieces of y[t][k2][k1] and one dimension-permuting TMA store scatters them (the last P).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "matmul_umma.h"
 #include "ptx_sm100.cuh"
+#include "tma_host.h"
 
 namespace m2mm {
 
@@ -34,6 +35,7 @@ constexpr int OFF_A = 0;                   // 8 operands [128 t][64] bf16, swizz
 constexpr int OFF_B = 131072;              // 8 weight blocks [64][64] bf16, swizzled   65536
 constexpr int OFF_BAR = 196608;            // bar_mma, tmem ptr
 constexpr int SMEM_BYTES = OFF_BAR + 64;
+constexpr int kZPitch = 1040;   // staging pitch of pass 1's 1 KB output rows (the 128 rows spill into the weight buffer, free by then)
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -41,6 +43,14 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32
 __device__ __forceinline__ void cp_async_commit_wait() {
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map), "r"(src), "r"(c0),
+                 "r"(c1), "r"(c2)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t ssrc, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t r;
@@ -58,8 +68,9 @@ __device__ __forceinline__ uint32_t sw_off(int r, int kc) { return (uint32_t)((r
 // PASS 2: in = z[T][64 k1][64 n2], W = L[k1][k2][n2], out = y[T][64 k2][64 k1]
 template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
-monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16* __restrict__ W, __nv_bfloat16* __restrict__ out,
-                      long long T, int32_t* __restrict__ status) {
+monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16* __restrict__ W,
+                      const __grid_constant__ CUtensorMap map_out, __nv_bfloat16* __restrict__ zout, long long T,
+                      int32_t* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
     const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
@@ -105,11 +116,12 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
             }
         }
     } else {
-        // rows z[t][k1][0..63] are the operand rows already
+        // z[n2 group kc][t][k1][8]: the 16-byte piece (kc, t, k1) is chunk kc of row t of operand A_{k1}; the 8 pieces
+        // of this CTA's k1 group are 128 contiguous bytes
         for (int c = tid; c < kGroup * kTileT * 8; c += kThreads) {
-            const int kc = c & 7, bl = (c >> 3) & 7, tt = c >> 6;
+            const int bl = c & 7, tt = (c >> 3) & 127, kc = c >> 10;
             const bool live = t0 + tt < T;
-            const __nv_bfloat16* src = in + ((size_t)(live ? t0 + tt : 0) * 64 + grp * kGroup + bl) * 64 + kc * 8;
+            const __nv_bfloat16* src = in + ((((size_t)kc * T + (live ? t0 + tt : 0)) * 64) + grp * kGroup + bl) * 8;
             cp_async16(s_base + OFF_A + bl * 16384 + sw_off(tt, kc), src, live ? 16u : 0u);
         }
     }
@@ -132,12 +144,14 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     }
     const bool ok = mbar_wait(bar_mma, 0);
     tc_fence_after();
-    // epilogue: lane = token; warpgroup wg takes output columns [16 wg, 16 wg + 16); for every output index o
-    // the 8 accumulators give the 8 consecutive block indices -> one 16-byte piece of out[t][o][grp*8 ..]
-    if (ok) {   // every lane takes part in the warp-wide TMEM loads; only live tokens store
-        const bool live = t0 + t < T;
+    // epilogue: lane = token; warpgroup wg takes output columns [16 wg, 16 wg + 16); for every output index o the 8
+    // accumulators give the 8 consecutive block indices -> one 16-byte piece.  The pieces are staged in the (now free)
+    // operand buffer with consecutive lanes writing to different banks, then leave through the copy engine:
+    //   pass 1: z[grp][t][k1][8] -- this CTA's 128 rows of 1 KB are contiguous; every token's row is one bulk copy;
+    //   pass 2: y[t][k2][k1]     -- staged as [k2][t][16 B]; one TMA store whose tensor map lists the dimensions as
+    //                               (k1, t, k2) scatters the pieces (rows past T are clipped by the map).
+    if (ok) {
         const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-        __nv_bfloat16* orow = out + (size_t)(live ? t0 + t : 0) * 4096 + grp * 8;
 #pragma unroll 1
         for (int gk = 0; gk < 2; ++gk) {
             const int o0 = 16 * wg + 8 * gk;
@@ -151,13 +165,29 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
             for (int kk = 0; kk < 8; ++kk) {
                 const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
                                            pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
-                if (live) *reinterpret_cast<uint4*>(orow + (size_t)(o0 + kk) * 64) = p;
+                if (PASS == 1)
+                    *reinterpret_cast<uint4*>(smem + OFF_A + t * kZPitch + (o0 + kk) * 16) = p;
+                else
+                    *reinterpret_cast<uint4*>(smem + OFF_A + (o0 + kk) * 2048 + t * 16) = p;
             }
         }
     }
-    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    if (PASS == 1) {
+        if (ok && tid < kTileT && t0 + tid < T) {
+            bulk_store(zout + (((size_t)grp * T + t0 + tid) * 64) * 8, s_base + OFF_A + tid * kZPitch, 1024u);
+            tma_store_commit();
+            tma_store_wait_read0();
+        }
+    } else if (tid == 0 && ok) {
+        tma_store_3d(&map_out, s_base + OFF_A, 8 * grp, (int)t0, 0);
+        tma_store_commit();
+        tma_store_wait_read0();   // the staging buffer dies with the CTA
+    }
+    __syncthreads();
+    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
     if (tid < 32) tmem_dealloc(tmem, 512);
 }
 
@@ -176,10 +206,15 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     if (!covered(pl)) return M2_ERR_UNSUPPORTED;
     if (T == 0) return M2_OK;
     dim3 grid(8, (unsigned)((T + kTileT - 1) / kTileT));
-    monarch64_pass_kernel<1><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)X, (const __nv_bfloat16*)R,
+    // y[t][k2][k1] seen as (k1 64 | t, stride 8 KB | k2, stride 128 B); box = 8 k1 x 128 tokens x 64 k2
+    alignas(64) CUtensorMap my;
+    const cuuint64_t gdim[3] = {64, (cuuint64_t)T, 64}, gstr[2] = {8192, 128};
+    const cuuint32_t box[3] = {8, (cuuint32_t)kTileT, 64};
+    if (!tma_host::encode_bf16(&my, Y, 3, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    monarch64_pass_kernel<1><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)X, (const __nv_bfloat16*)R, my,
                                                                      (__nv_bfloat16*)ws, T, pl->d_status);
-    monarch64_pass_kernel<2><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)ws, (const __nv_bfloat16*)L,
-                                                                     (__nv_bfloat16*)Y, T, pl->d_status);
+    monarch64_pass_kernel<2><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)ws, (const __nv_bfloat16*)L, my,
+                                                                     nullptr, T, pl->d_status);
     if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
     pl->last_kernel = "matmul_umma_64x64";
     pl->launches += 2;

@@ -56,6 +56,7 @@ constexpr int SMEM_BYTES = OFF_GROUP + kGroups * GROUP_BYTES;
 
 struct Tables {
     void* d_const = nullptr;  // CONST_BYTES
+    int* d_sched = nullptr;   // {next unit, pipelines finished}; zero between launches
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -101,7 +102,7 @@ __device__ __forceinline__ bool group_sync_or(int wg, bool pred, volatile int* f
 __global__ void __launch_bounds__(kThreads, 1)
 conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
-               int32_t* __restrict__ status) {
+               int32_t* __restrict__ status, int* __restrict__ sched) {
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
@@ -111,6 +112,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     const uint32_t s_base = s_all + OFF_GROUP + wg * GROUP_BYTES;
     const uint32_t bar_x = s_all + OFF_BAR + wg * 32, bar_mma = bar_x + 8, bar_k = bar_x + 16;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_all + OFF_BAR + wg * 32 + 24);
+    volatile int* next_slot = reinterpret_cast<volatile int*>(smem_all + OFF_BAR + wg * 32 + 28);
     const uint32_t s_tptr = s_all + OFF_BAR + 224;
 
     const int bgroups0 = (B + kRows - 1) / kRows;
@@ -163,11 +165,13 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
 #ifdef M2_PHASE_TIMING
     long long tick_ = clock64();
 #endif
-    for (; u < units; u += ustride) {
+    // Units beyond the first are handed out by a device-wide counter (sched[0]): pipelines that finish early take more.
+    // The last pipeline to leave (sched[1] counts them) zeroes both words for the next launch on this plan.
+    while (u < units) {
         M2_TICK(15)
         const int h = u % H;
         const int b0 = (u / H) * kRows;
-        const int un = u + ustride;
+        int un = units;   // known to thread 0 from hand-off 1 on, to the others after the next group barrier
         // ---- S1 ---------------------------------------------------------------------------------
         if (tid == 0) {
             ok = mbar_wait(bar_x, ph_x);
@@ -188,6 +192,10 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         ph_m ^= 1;
         tc_fence_after();
         M2_TICK(1)
+        if (tid == 0) {
+            un = ustride + atomicAdd(sched, 1);
+            *next_slot = un;
+        }
         if (tid == 0 && ok && un < units) {   // the x tile is free: fetch the next unit's
             mbar_expect_tx(bar_x, 8192);
             tma_load_4d(s_base + G_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
@@ -233,6 +241,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             aborted = true;
             break;
         }
+        un = *next_slot;   // written by thread 0 before the barrier above
         M2_TICK(2)
         // ---- S2 ---------------------------------------------------------------------------------
         if (tid == 0) {
@@ -387,12 +396,19 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             break;
         }
         M2_TICK(8)
+        u = un;
     }
     // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
     if (tid == 0) {
         if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
         if (x_pending) mbar_wait(bar_x, ph_x);
         if (k_pending) mbar_wait(bar_k, ph_k);
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == ustride - 1) {   // last pipeline out: reset the scheduler words
+            sched[0] = 0;
+            sched[1] = 0;
+            __threadfence();
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -502,9 +518,12 @@ cudaError_t create_tables(m2_plan* pl) {
     Tables* t = new Tables();
     cudaError_t e = cudaMalloc(&t->d_const, CONST_BYTES);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_sched, 2 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(t->d_sched, 0, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) {
         if (t->d_const) cudaFree(t->d_const);
+        if (t->d_sched) cudaFree(t->d_sched);
         delete t;
         return e;
     }
@@ -516,6 +535,7 @@ void destroy_tables(m2_plan* pl) {
     if (!pl->umma || !covered(pl)) return;
     Tables* t = reinterpret_cast<Tables*>(pl->umma);
     if (t->d_const) cudaFree(t->d_const);
+    if (t->d_sched) cudaFree(t->d_sched);
     delete t;
     pl->umma = nullptr;
 }
@@ -549,7 +569,7 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     const int grid = (int)(ctas < sms ? ctas : sms);
     const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * 512 * 8);
     conv512_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H,
-                                                           (int)n, pl->d_status);
+                                                           (int)n, pl->d_status, t->d_sched);
     if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o2_512";
     pl->launches += 1;

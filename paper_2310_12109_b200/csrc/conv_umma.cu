@@ -64,19 +64,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-#ifdef M2_PHASE_TIMING
-// Development aid (never compiled into the shipped library): cycles block 0 / thread 0 spends in each
-// phase of the unit loop, summed over its units.
-__device__ long long g_phase_cycles[16];
-#define M2_TICK(slot)                                             \
-    if (blockIdx.x == 0 && threadIdx.x == 0) {                            \
-        const long long now_ = clock64();                         \
-        g_phase_cycles[slot] += now_ - tick_;                     \
-        tick_ = now_;                                             \
-    }
-#else
-#define M2_TICK(slot)
-#endif
 
 // Multiplies 8 complex values (re[], im[]) by 8 complex factors given as 4 float4 (c0, s0, c1, s1) and
 // packs real and imaginary parts as bf16 pairs.
@@ -162,13 +149,9 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
 
     uint32_t ph_x = 0, ph_m = 0, ph_k = 0;
     bool ok = true, aborted = false;
-#ifdef M2_PHASE_TIMING
-    long long tick_ = clock64();
-#endif
     // Units beyond the first are handed out by a device-wide counter (sched[0]): pipelines that finish early take more.
     // The last pipeline to leave (sched[1] counts them) zeroes both words for the next launch on this plan.
     while (u < units) {
-        M2_TICK(15)
         const int h = u % H;
         const int b0 = (u / H) * kRows;
         int un = units;   // known to thread 0 from hand-off 1 on, to the others after the next group barrier
@@ -186,12 +169,10 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             }
         }
         ph_x ^= 1;
-        M2_TICK(0)
         // ---- h1: twiddle, A2 ---------------------------------------------------------------------
         ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        M2_TICK(1)
         if (tid == 0) {
             un = ustride + atomicAdd(sched, 1);
             *next_slot = un;
@@ -242,7 +223,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             break;
         }
         un = *next_slot;   // written by thread 0 before the barrier above
-        M2_TICK(2)
         // ---- S2 ---------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -266,7 +246,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        M2_TICK(3)
         if (ok) {
             const int k1 = tid & 31;
             const float4* kfs = reinterpret_cast<const float4*>(smem + G_KF) + k1;
@@ -302,7 +281,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             aborted = true;
             break;
         }
-        M2_TICK(4)
         // ---- S2' --------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -323,7 +301,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         ok = mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        M2_TICK(5)
         if (ok) {
             const int k1 = tid & 31;
             const float4* twB = reinterpret_cast<const float4*>(smem_all + OFF_TWB) + k1;
@@ -359,7 +336,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             aborted = true;
             break;
         }
-        M2_TICK(6)
         // ---- S1' --------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -374,7 +350,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         ok = mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        M2_TICK(7)
         if (ok) {
             const int r = tid >> 4, n2 = tid & 15;
             float v[32];
@@ -395,7 +370,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             aborted = true;
             break;
         }
-        M2_TICK(8)
         u = un;
     }
     // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
@@ -587,15 +561,5 @@ cudaError_t relayout_spectrum(const m2_plan* pl, void* kf, int64_t H, cudaStream
     return cudaGetLastError();
 }
 
-#ifdef M2_PHASE_TIMING
-extern "C" void m2_debug_phase_cycles(long long* out16, int reset) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out16, g_phase_cycles, sizeof(long long) * 16);
-    if (reset) {
-        long long z[16] = {0};
-        cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z));
-    }
-}
-#endif
 
 }  // namespace m2u

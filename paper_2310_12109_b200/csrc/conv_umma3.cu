@@ -143,7 +143,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
     const int pairs = H * bpairs;
     int pr_i = blockIdx.x;
     if (tid == 0) {
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_mma, 4);   // one commit per warpgroup's issuing thread
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -190,18 +190,27 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         // the pair's input has landed (every thread waits for its own copies, then the block syncs)
         cp_async_wait_all();
         M2_STAGE_SYNC()
+        // pull this pair's 256 KB of spectrum towards L2 now; hand-off 3 reads it five stages later
+        if ((t & 7) == 0) {
+#pragma unroll 1
+            for (int jj = 0; jj < 2; ++jj) {
+                const float4* kp = kfu + ((size_t)(h * 8 + wg + 4 * jj) * 16) * 128 + t;
+#pragma unroll
+                for (int q = 0; q < 16; ++q) asm volatile("prefetch.global.L2 [%0];" ::"l"(kp + q * 128));
+            }
+        }
         // ---- S1: contract n1 (K = 32: the zero half is skipped) -----------------------------------------
-        if (tid == 0) {
-            if (store_pending) {   // the previous pair's output staging must be read out before A is reused
+        if (t == 0) {   // lane 0 of every warpgroup issues the UMMAs of the two tiles its warpgroup hands off
+            if (tid == 0 && store_pending) {   // the previous pair's output staging must be read out before A is reused
                 tma_store_wait_read0();
                 store_pending = false;
             }
             tc_fence_after();
-#pragma unroll 1
-            for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int s = 0; s < 2; ++s)
-                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_X + j * 8192 + s * 2048, 4096, 1024),
+                    umma_f16(tmem + (wg + 4 * jj) * 64, smem_desc_sw128(s_base + OFF_X + (wg + 4 * jj) * 8192 + s * 2048, 4096, 1024),
                              smem_desc(s_base + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
             umma_commit(bar_mma);
         }
@@ -243,13 +252,13 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S2: contract n2 -----------------------------------------------------------------------------------
-        if (tid == 0) {
+        if (t == 0) {
             tc_fence_after();
-#pragma unroll 1
-            for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int s = 0; s < 4; ++s)
-                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                    umma_f16(tmem + (wg + 4 * jj) * 64, smem_desc_sw128(s_base + OFF_A + (wg + 4 * jj) * 16384 + s * 2048, 8192, 1024),
                              smem_desc(s_base + OFF_BF + s * 256, 128, 1024), ID_MM, s > 0);
             umma_commit(bar_mma);
         }
@@ -276,13 +285,13 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S3: contract n3 -----------------------------------------------------------------------------------
-        if (tid == 0) {
+        if (t == 0) {
             tc_fence_after();
-#pragma unroll 1
-            for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int s = 0; s < 4; ++s)
-                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                    umma_f16(tmem + (wg + 4 * jj) * 64, smem_desc_sw128(s_base + OFF_A + (wg + 4 * jj) * 16384 + s * 2048, 8192, 1024),
                              smem_desc(s_base + OFF_BF + s * 256, 128, 1024), ID_MM, s > 0);
             umma_commit(bar_mma);
         }
@@ -322,13 +331,13 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S3': contract k3 with conj F ---------------------------------------------------------------------------
-        if (tid == 0) {
+        if (t == 0) {
             tc_fence_after();
-#pragma unroll 1
-            for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int s = 0; s < 4; ++s)
-                    umma_f16(tmem + j * 64, smem_desc(s_base + OFF_A + j * 16384 + s * 256, 128, 1024),
+                    umma_f16(tmem + (wg + 4 * jj) * 64, smem_desc(s_base + OFF_A + (wg + 4 * jj) * 16384 + s * 256, 128, 1024),
                              smem_desc(s_base + OFF_BI + s * 256, 128, 1024), ID_KM, s > 0);
             umma_commit(bar_mma);
         }
@@ -359,13 +368,13 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S2': contract k2 with conj F ---------------------------------------------------------------------------
-        if (tid == 0) {
+        if (t == 0) {
             tc_fence_after();
-#pragma unroll 1
-            for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int s = 0; s < 4; ++s)
-                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                    umma_f16(tmem + (wg + 4 * jj) * 64, smem_desc_sw128(s_base + OFF_A + (wg + 4 * jj) * 16384 + s * 2048, 8192, 1024),
                              smem_desc(s_base + OFF_BI + s * 256, 128, 1024), ID_MM, s > 0);
             umma_commit(bar_mma);
         }
@@ -400,13 +409,13 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S1': contract k1 with conj F, outputs n1 < 16 only (N = 32) ----------------------------------------------
-        if (tid == 0) {
+        if (t == 0) {
             tc_fence_after();
-#pragma unroll 1
-            for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj)
 #pragma unroll
                 for (int s = 0; s < 4; ++s)
-                    umma_f16(tmem + j * 64, smem_desc_sw128(s_base + OFF_A + j * 16384 + s * 2048, 8192, 1024),
+                    umma_f16(tmem + (wg + 4 * jj) * 64, smem_desc_sw128(s_base + OFF_A + (wg + 4 * jj) * 16384 + s * 2048, 8192, 1024),
                              smem_desc(s_base + OFF_B6 + s * 256, 128, 1024), ID_S6, s > 0);
             umma_commit(bar_mma);
         }

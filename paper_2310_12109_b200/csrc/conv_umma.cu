@@ -37,10 +37,10 @@ namespace m2u {
 using namespace sm100;
 
 constexpr int kRows = 8;             // rows (batch entries) per unit
-constexpr int kGroups = 4;           // independent warpgroups per CTA, each running its own unit loop
+constexpr int kGroups = 5;           // independent warpgroups per CTA, each running its own unit loop
 constexpr int kThreads = 128 * kGroups;
 constexpr int kTmemColsPerGroup = 64;
-constexpr int kTmemCols = 256;       // allocation must be a power of two >= kGroups * 64
+constexpr int kTmemCols = 512;       // allocation must be a power of two >= kGroups * 64
 // shared memory map (bytes): constants shared by the CTA, then one slice per warpgroup
 constexpr int OFF_CONST = 0;         // B1 4096 | B2 2048 | B3 2048 | B4 4096 | twA 4096 | twB 4096
 constexpr int CONST_BYTES = 20480;

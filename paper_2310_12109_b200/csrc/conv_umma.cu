@@ -19,8 +19,9 @@
 //   S1'  D4[(r,n2)][n1]       = Re sum_(c,k1) A4 * conj(F32)
 //   h4   round to bf16 into the output tile, TMA store.
 //
-// Four such CTAs (128 threads, 128 TMEM columns, ~52 KB shared memory each) share an SM, so one
-// CTA's UMMA / TMA latency is covered by the others' fp32 work.  All waits are bounded.
+// One CTA per SM keeps the constant operands once and runs kGroups independent unit pipelines of 128
+// threads (own mbarriers, 64 TMEM columns, 28 KB of shared memory each), so one pipeline's UMMA / TMA /
+// barrier latency is covered by the others' fp32 work.  All waits are bounded.
 #include "conv_umma.h"
 
 #include <cuda.h>
@@ -37,7 +38,7 @@ namespace m2u {
 using namespace sm100;
 
 constexpr int kRows = 8;             // rows (batch entries) per unit
-constexpr int kGroups = 5;           // independent warpgroups per CTA, each running its own unit loop
+constexpr int kGroups = 7;           // independent warpgroups per CTA, each running its own unit loop (72 registers per thread)
 constexpr int kThreads = 128 * kGroups;
 constexpr int kTmemColsPerGroup = 64;
 constexpr int kTmemCols = 512;       // allocation must be a power of two >= kGroups * 64
@@ -65,15 +66,44 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 
-// Multiplies 8 complex values (re[], im[]) by 8 complex factors given as 4 float4 (c0, s0, c1, s1) and
-// packs real and imaginary parts as bf16 pairs.
+// Packed pairs of fp32 (one 64-bit register): sm_100 multiplies / fuses two lanes per instruction.
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// Multiplies 8 complex values (re[], im[]) by 8 complex factors given as 4 float4 (c0, c1, s0, s1) -- the
+// factors of two neighbouring values -- and packs real and imaginary parts as bf16 pairs.
 __device__ __forceinline__ void cmul_pack8(const float* re, const float* im, const float4* w, uint4& pr, uint4& pi) {
     uint32_t r_[4], i_[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-        const float a0 = re[2 * q], b0 = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-        r_[q] = pack_bf16(a0 * w[q].x - b0 * w[q].y, a1 * w[q].z - b1 * w[q].w);
-        i_[q] = pack_bf16(a0 * w[q].y + b0 * w[q].x, a1 * w[q].w + b1 * w[q].z);
+        const uint64_t a2 = pk2(re[2 * q], re[2 * q + 1]), b2 = pk2(im[2 * q], im[2 * q + 1]);
+        const uint64_t c2 = pk2(w[q].x, w[q].y), s2 = pk2(w[q].z, w[q].w);
+        const uint64_t r2 = fma2(sub2(0ull, b2), s2, mul2(a2, c2));   // a c - b s
+        const uint64_t i2 = fma2(b2, c2, mul2(a2, s2));               // a s + b c
+        float x0, x1, y0, y1;
+        upk2(r2, x0, x1);
+        upk2(i2, y0, y1);
+        r_[q] = pack_bf16(x0, x1);
+        i_[q] = pack_bf16(y0, y1);
     }
     pr = make_uint4(r_[0], r_[1], r_[2], r_[3]);
     pi = make_uint4(i_[0], i_[1], i_[2], i_[3]);
@@ -149,12 +179,13 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
 
     uint32_t ph_x = 0, ph_m = 0, ph_k = 0;
     bool ok = true, aborted = false;
-    // Units beyond the first are handed out by a device-wide counter (sched[0]): pipelines that finish early take more.
+    // Units beyond the first two are handed out by a device-wide counter (sched[0]): pipelines that finish early take more.
     // The last pipeline to leave (sched[1] counts them) zeroes both words for the next launch on this plan.
+    int un = u + ustride;   // the second unit is static too
+    int un2 = units;        // thread 0: the unit after next, claimed one whole unit ahead so the atomic's latency is never waited for
     while (u < units) {
         const int h = u % H;
         const int b0 = (u / H) * kRows;
-        int un = units;   // known to thread 0 from hand-off 1 on, to the others after the next group barrier
         // ---- S1 ---------------------------------------------------------------------------------
         if (tid == 0) {
             ok = mbar_wait(bar_x, ph_x);
@@ -173,10 +204,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        if (tid == 0) {
-            un = ustride + atomicAdd(sched, 1);
-            *next_slot = un;
-        }
+        if (tid == 0) un2 = 2 * ustride + atomicAdd(sched, 1);   // consumed at the end of this unit
         if (tid == 0 && ok && un < units) {   // the x tile is free: fetch the next unit's
             mbar_expect_tx(bar_x, 8192);
             tma_load_4d(s_base + G_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
@@ -186,34 +214,32 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         if (ok) {
             const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
             const float4* twA = reinterpret_cast<const float4*>(smem_all + OFF_TWA) + n2;
-            float re[32], im[32];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                tmem_ld8(t_lane + T1 + 8 * j, re + 8 * j);
-                tmem_ld8(t_lane + T1 + 32 + 8 * j, im + 8 * j);
-            }
-            tmem_ld_wait();
+            for (int hh = 0; hh < 2; ++hh) {   // two batches of 16 complex values keep the register count down
+                float re[16], im[16];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                tmem_ld_fence8(re + 8 * j);
-                tmem_ld_fence8(im + 8 * j);
-            }
+                for (int jj = 0; jj < 2; ++jj) {
+                    tmem_ld8(t_lane + T1 + 16 * hh + 8 * jj, re + 8 * jj);
+                    tmem_ld8(t_lane + T1 + 32 + 16 * hh + 8 * jj, im + 8 * jj);
+                }
+                tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                float4 w[4];
+                for (int jj = 0; jj < 2; ++jj) {
+                    tmem_ld_fence8(re + 8 * jj);
+                    tmem_ld_fence8(im + 8 * jj);
+                }
 #pragma unroll
-                for (int q = 0; q < 4; ++q) w[q] = twA[(4 * j + q) * 16];
-                uint4 pr, pi;
-                cmul_pack8(re + 8 * j, im + 8 * j, w, pr, pi);
-#ifdef M2_EXP_SW128
-                unsigned char* base = smem + G_A + (r >> 1) * 4096 + n2lo * 128 + (((((r & 1) << 2) + j) ^ n2lo) << 4);
-                *reinterpret_cast<uint4*>(base + (0 + n2hi) * 1024) = pr;
-                *reinterpret_cast<uint4*>(base + (2 + n2hi) * 1024) = pi;
-#else
-                unsigned char* base = smem + G_A + (r * 4 + j) * 512 + n2lo * 16;
-                *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = pr;
-                *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = pi;
-#endif
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int j = 2 * hh + jj;
+                    float4 w[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) w[q] = twA[(4 * j + q) * 16];
+                    uint4 pr, pi;
+                    cmul_pack8(re + 8 * jj, im + 8 * jj, w, pr, pi);
+                    unsigned char* base = smem + G_A + (r * 4 + j) * 512 + n2lo * 16;
+                    *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = pr;
+                    *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = pi;
+                }
             }
         }
         fence_proxy_async();
@@ -222,7 +248,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             aborted = true;
             break;
         }
-        un = *next_slot;   // written by thread 0 before the barrier above
         // ---- S2 ---------------------------------------------------------------------------------
         if (tid == 0) {
             tc_fence_after();
@@ -230,13 +255,8 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int s = 0; s < 2; ++s)
-#ifdef M2_EXP_SW128
-                    umma_f16(tmem + T2 + hf * 32, smem_desc_sw128(s_base + G_A + hf * 8192 + s * 2048, 4096, 1024),
-                             smem_desc(s_all + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
-#else
                     umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + G_A + hf * 8192 + s * 256, 128, 512),
                              smem_desc(s_all + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
-#endif
             umma_commit(bar_mma);
         }
         // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
@@ -365,12 +385,14 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
                     if (i < n1_valid) yr[i * 16] = __float2bfloat16_rn(v[i]);
             }
         }
+        if (tid == 0) *next_slot = un2;
         tc_fence_before();
         if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
             break;
         }
         u = un;
+        un = *next_slot;   // written by thread 0 before the barrier above
     }
     // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
     if (tid == 0) {
@@ -389,14 +411,14 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     if (threadIdx.x < 32) tmem_dealloc(tmem_cta, kTmemCols);
 }
 
-// spectrum re-layout for this kernel: kfu[h][k2/2][k1] = (re, im)(k2 even), (re, im)(k2 odd) from plan order
+// spectrum re-layout for this kernel: kfu[h][k2/2][k1] = (re(k2 even), re(k2 odd), im(even), im(odd)) from plan order
 __global__ void relayout_spectrum_kernel(const float2* __restrict__ kf, float4* __restrict__ kfu, long long total) {
     const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 8 * 32
     if (i >= total) return;
     const int k1 = (int)(i & 31), q = (int)((i >> 5) & 7);
     const long long h = i >> 8;
     const float2 a = kf[h * 512 + k1 * 16 + 2 * q], b = kf[h * 512 + k1 * 16 + 2 * q + 1];
-    kfu[i] = make_float4(a.x, a.y, b.x, b.y);
+    kfu[i] = make_float4(a.x, b.x, a.y, b.y);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
@@ -470,17 +492,17 @@ cudaError_t create_tables(m2_plan* pl) {
                 const double th = 2.0 * M_PI * ((k1 * n1) % N1) / N1;
                 put_kmajor(B4, 64, n1, c * 32 + k1, c == 0 ? std::cos(th) : sg * std::sin(th));
             }
-    // twiddles w_N^{n2 k1}: twA[k1/2][n2][k1%2] (cos, sin); twB[n2/2][k1][n2%2] conjugated
+    // twiddles w_N^{n2 k1}: twA[k1/2][n2] = (cos(k1 even), cos(k1 odd), sin(even), sin(odd)); twB[n2/2][k1] likewise, conjugated
     for (int k1 = 0; k1 < N1; ++k1)
         for (int n2 = 0; n2 < N2; ++n2) {
             const double th = 2.0 * M_PI * ((n2 * k1) % N) / N;
             const float cs = (float)std::cos(th), sn = (float)(sg * std::sin(th));
-            const size_t ia = (((size_t)(k1 / 2) * 16 + n2) * 2 + (k1 % 2)) * 2;
+            const size_t ia = ((size_t)(k1 / 2) * 16 + n2) * 4 + (k1 % 2);
             twA[ia] = cs;
-            twA[ia + 1] = sn;
-            const size_t ib = (((size_t)(n2 / 2) * 32 + k1) * 2 + (n2 % 2)) * 2;
+            twA[ia + 2] = sn;
+            const size_t ib = ((size_t)(n2 / 2) * 32 + k1) * 4 + (n2 % 2);
             twB[ib] = cs;
-            twB[ib + 1] = -sn;
+            twB[ib + 2] = -sn;
         }
     std::vector<unsigned char> blob(CONST_BYTES);
     std::memcpy(blob.data(), B1.data(), 4096);

@@ -124,6 +124,9 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
     const int warp = tid >> 5;                // warp within the group = TMEM lane quarter
+    // the thread that issues this pipeline's UMMAs and copies; its warp differs from group to group so that
+    // the extra work spreads over the SM's four schedulers
+    const bool leader = tid == 32 * (wg & 3);
     const uint32_t s_all = smem_u32(smem_all);
     unsigned char* smem = smem_all + OFF_GROUP + wg * GROUP_BYTES;   // this group's slice
     const uint32_t s_base = s_all + OFF_GROUP + wg * GROUP_BYTES;
@@ -136,7 +139,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     const int units0 = H * bgroups0;
     int u = blockIdx.x * kGroups + wg;
     const int ustride = gridDim.x * kGroups;
-    if (tid == 0) {
+    if (leader) {
         mbar_init(bar_x, 1);
         mbar_init(bar_mma, 1);
         mbar_init(bar_k, 1);
@@ -145,7 +148,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         prefetch_tensormap(&map_x);
     }
     bool x_pending = false, k_pending = false;
-    if (tid == 0 && u < units0) {   // first loads go out before anything else
+    if (leader && u < units0) {   // first loads go out before anything else
         mbar_expect_tx(bar_x, 8192);
         tma_load_4d(s_base + G_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
         tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, u % H, (u / H) * kRows, bar_x);
@@ -187,7 +190,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         const int h = u % H;
         const int b0 = (u / H) * kRows;
         // ---- S1 ---------------------------------------------------------------------------------
-        if (tid == 0) {
+        if (leader) {
             ok = mbar_wait(bar_x, ph_x);
             x_pending = false;
             if (ok) {
@@ -204,8 +207,8 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
-        if (tid == 0) un2 = 2 * ustride + atomicAdd(sched, 1);   // consumed at the end of this unit
-        if (tid == 0 && ok && un < units) {   // the x tile is free: fetch the next unit's
+        if (leader) un2 = 2 * ustride + atomicAdd(sched, 1);   // consumed at the end of this unit
+        if (leader && ok && un < units) {   // the x tile is free: fetch the next unit's
             mbar_expect_tx(bar_x, 8192);
             tma_load_4d(s_base + G_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
             tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, un % H, (un / H) * kRows, bar_x);
@@ -249,7 +252,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             break;
         }
         // ---- S2 ---------------------------------------------------------------------------------
-        if (tid == 0) {
+        if (leader) {
             tc_fence_after();
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf)
@@ -262,34 +265,37 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
         ok = mbar_wait(bar_k, ph_k);          // the channel's spectrum row has landed
         ph_k ^= 1;
-        if (tid == 0) k_pending = false;
+        if (leader) k_pending = false;
         ok = ok && mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
         if (ok) {
             const int k1 = tid & 31;
             const float4* kfs = reinterpret_cast<const float4*>(smem + G_KF) + k1;
+            // both row halves (hf) of a thread share k1, hence the spectrum values: load them once per chunk
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const int m = hf * 128 + tid;
-                unsigned char* rowp = smem + G_A + (m >> 3) * 512 + (m & 7) * 16;
+            for (int g = 0; g < 2; ++g) {
                 float re[16], im[16];
-                tmem_ld8(t_lane + T2 + hf * 32, re);
-                tmem_ld8(t_lane + T2 + hf * 32 + 8, re + 8);
-                tmem_ld8(t_lane + T2 + hf * 32 + 16, im);
-                tmem_ld8(t_lane + T2 + hf * 32 + 24, im + 8);
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld8(t_lane + T2 + hf * 32 + 8 * g, re + 8 * hf);
+                    tmem_ld8(t_lane + T2 + hf * 32 + 16 + 8 * g, im + 8 * hf);
+                }
+                float4 w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = kfs[(g * 4 + q) * 32];
                 tmem_ld_wait();
-                tmem_ld_fence8(re);
-                tmem_ld_fence8(re + 8);
-                tmem_ld_fence8(im);
-                tmem_ld_fence8(im + 8);
 #pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    float4 w[4];
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld_fence8(re + 8 * hf);
+                    tmem_ld_fence8(im + 8 * hf);
+                }
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) w[q] = kfs[(g * 4 + q) * 32];
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int m = hf * 128 + tid;
+                    unsigned char* rowp = smem + G_A + (m >> 3) * 512 + (m & 7) * 16;
                     uint4 pr, pi;
-                    cmul_pack8(re + 8 * g, im + 8 * g, w, pr, pi);
+                    cmul_pack8(re + 8 * hf, im + 8 * hf, w, pr, pi);
                     *reinterpret_cast<uint4*>(rowp + g * 128) = pr;
                     *reinterpret_cast<uint4*>(rowp + (2 + g) * 128) = pi;
                 }
@@ -302,7 +308,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             break;
         }
         // ---- S2' --------------------------------------------------------------------------------
-        if (tid == 0) {
+        if (leader) {
             tc_fence_after();
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf)
@@ -325,25 +331,27 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             const int k1 = tid & 31;
             const float4* twB = reinterpret_cast<const float4*>(smem_all + OFF_TWB) + k1;
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const int r = hf * 4 + (tid >> 5);
+            for (int g = 0; g < 2; ++g) {   // the twiddles depend on (k1, n2) only: shared by both row halves
                 float re[16], im[16];
-                tmem_ld8(t_lane + T1 + hf * 32, re);
-                tmem_ld8(t_lane + T1 + hf * 32 + 8, re + 8);
-                tmem_ld8(t_lane + T1 + hf * 32 + 16, im);
-                tmem_ld8(t_lane + T1 + hf * 32 + 24, im + 8);
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld8(t_lane + T1 + hf * 32 + 8 * g, re + 8 * hf);
+                    tmem_ld8(t_lane + T1 + hf * 32 + 16 + 8 * g, im + 8 * hf);
+                }
+                float4 w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = twB[(4 * g + q) * 32];
                 tmem_ld_wait();
-                tmem_ld_fence8(re);
-                tmem_ld_fence8(re + 8);
-                tmem_ld_fence8(im);
-                tmem_ld_fence8(im + 8);
 #pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    float4 w[4];
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld_fence8(re + 8 * hf);
+                    tmem_ld_fence8(im + 8 * hf);
+                }
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) w[q] = twB[(4 * g + q) * 32];
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int r = hf * 4 + (tid >> 5);
                     uint4 pr, pi;
-                    cmul_pack8(re + 8 * g, im + 8 * g, w, pr, pi);
+                    cmul_pack8(re + 8 * hf, im + 8 * hf, w, pr, pi);
                     unsigned char* base = smem + G_A + (r * 2 + g) * 1024 + (k1 >> 3) * 128 + (k1 & 7) * 16;
                     *reinterpret_cast<uint4*>(base) = pr;
                     *reinterpret_cast<uint4*>(base + 512) = pi;
@@ -357,7 +365,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             break;
         }
         // ---- S1' --------------------------------------------------------------------------------
-        if (tid == 0) {
+        if (leader) {
             tc_fence_after();
 #pragma unroll
             for (int s = 0; s < 4; ++s)
@@ -385,7 +393,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
                     if (i < n1_valid) yr[i * 16] = __float2bfloat16_rn(v[i]);
             }
         }
-        if (tid == 0) *next_slot = un2;
+        if (leader) *next_slot = un2;
         tc_fence_before();
         if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
@@ -395,7 +403,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         un = *next_slot;   // written by thread 0 before the barrier above
     }
     // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
-    if (tid == 0) {
+    if (leader) {
         if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
         if (x_pending) mbar_wait(bar_x, ph_x);
         if (k_pending) mbar_wait(bar_k, ph_k);

@@ -134,6 +134,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
     const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
+    const bool issuer = t == 32 * wg;   // one UMMA-issuing thread per warpgroup, each on a different scheduler
     const uint32_t s_base = smem_u32(smem);
     const uint32_t bar_mma = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 16;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8);
@@ -200,7 +201,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
             }
         }
         // ---- S1: contract n1 (K = 32: the zero half is skipped) -----------------------------------------
-        if (t == 0) {   // lane 0 of every warpgroup issues the UMMAs of the two tiles its warpgroup hands off
+        if (issuer) {   // one thread of every warpgroup issues the UMMAs of the two tiles its warpgroup hands off
             if (tid == 0 && store_pending) {   // the previous pair's output staging must be read out before A is reused
                 tma_store_wait_read0();
                 store_pending = false;
@@ -252,7 +253,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S2: contract n2 -----------------------------------------------------------------------------------
-        if (t == 0) {
+        if (issuer) {
             tc_fence_after();
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -285,7 +286,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S3: contract n3 -----------------------------------------------------------------------------------
-        if (t == 0) {
+        if (issuer) {
             tc_fence_after();
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -331,7 +332,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S3': contract k3 with conj F ---------------------------------------------------------------------------
-        if (t == 0) {
+        if (issuer) {
             tc_fence_after();
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -368,7 +369,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S2': contract k2 with conj F ---------------------------------------------------------------------------
-        if (t == 0) {
+        if (issuer) {
             tc_fence_after();
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)
@@ -409,7 +410,7 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
         }
         M2_STAGE_SYNC()
         // ---- S1': contract k1 with conj F, outputs n1 < 16 only (N = 32) ----------------------------------------------
-        if (t == 0) {
+        if (issuer) {
             tc_fence_after();
 #pragma unroll
             for (int jj = 0; jj < 2; ++jj)

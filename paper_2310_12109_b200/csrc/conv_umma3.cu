@@ -33,6 +33,7 @@
 
 #include "conv_umma.h"
 #include "ptx_sm100.cuh"
+#include "tma_host.h"
 
 namespace m2u3 {
 
@@ -129,7 +130,7 @@ __device__ __forceinline__ void load_pair(uint32_t s_x, const __nv_bfloat16* xa,
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y, const float4* __restrict__ kfu,
+conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* __restrict__ x, const float4* __restrict__ kfu,
                const uint4* __restrict__ consts, const float2* __restrict__ tn, int B, int H, int32_t* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
@@ -296,37 +297,39 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
                              smem_desc(s_base + OFF_BF + s * 256, 128, 1024), ID_MM, s > 0);
             umma_commit(bar_mma);
         }
-        M2_WAIT_MMA()
-        // ---- h3: spectrum multiply (k_f holds 1/N); A4 K-major: row = lane, K = (c, k3) ---------------------------
-        if (ok) {
-#pragma unroll 1
-            for (int jj = 0; jj < 2; ++jj) {
-                const int j = wg + 4 * jj;
-                float re[32], im[32];
-                const float4* kp = kfu + ((size_t)(h * 8 + j) * 16) * 128 + t;
-                float4 w[4], wn[4];
+        // ---- h3: spectrum multiply (k_f holds 1/N); A4 K-major: row = lane, K = (c, k3).  All of a tile's spectrum
+        //      values are requested before the wait for the UMMAs, the second tile's while the first is worked on. ------
+        {
+            const float4* kp0 = kfu + ((size_t)(h * 8 + wg) * 16) * 128 + t;
+            float4 w[16];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) w[q] = __ldg(kp + q * 128);
-                load_tile(t_lane + j * 64, re, im);
-                unsigned char* rowp = smem + OFF_A + j * 16384 + (t >> 3) * 1024 + (t & 7) * 16;
+            for (int q = 0; q < 16; ++q) w[q] = __ldg(kp0 + q * 128);
+            M2_WAIT_MMA()
+            if (ok) {
 #pragma unroll
-                for (int hi = 0; hi < 4; ++hi) {
-                    if (hi < 3) {
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int j = wg + 4 * jj;
+                    unsigned char* rowp = smem + OFF_A + j * 16384 + (t >> 3) * 1024 + (t & 7) * 16;
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) wn[q] = __ldg(kp + (4 * (hi + 1) + q) * 128);
+                    for (int hi = 0; hi < 4; ++hi) {
+                        float re[8], im[8];
+                        tmem_ld8(t_lane + j * 64 + 8 * hi, re);
+                        tmem_ld8(t_lane + j * 64 + 32 + 8 * hi, im);
+                        tmem_ld_wait();
+                        tmem_ld_fence8(re);
+                        tmem_ld_fence8(im);
+                        uint32_t r_[4], i_[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 ww = w[4 * hi + q];
+                            if (jj == 0) w[4 * hi + q] = __ldg(kp0 + (size_t)4 * 16 * 128 + (4 * hi + q) * 128);   // tile wg + 4
+                            const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
+                            r_[q] = pack_bf16(a0 * ww.x - b0v * ww.y, a1 * ww.z - b1 * ww.w);
+                            i_[q] = pack_bf16(a0 * ww.y + b0v * ww.x, a1 * ww.w + b1 * ww.z);
+                        }
+                        *reinterpret_cast<uint4*>(rowp + hi * 128) = make_uint4(r_[0], r_[1], r_[2], r_[3]);
+                        *reinterpret_cast<uint4*>(rowp + (4 + hi) * 128) = make_uint4(i_[0], i_[1], i_[2], i_[3]);
                     }
-                    uint32_t r_[4], i_[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 ww = w[q];
-                        const float a0 = re[8 * hi + 2 * q], b0v = im[8 * hi + 2 * q], a1 = re[8 * hi + 2 * q + 1], b1 = im[8 * hi + 2 * q + 1];
-                        r_[q] = pack_bf16(a0 * ww.x - b0v * ww.y, a1 * ww.z - b1 * ww.w);
-                        i_[q] = pack_bf16(a0 * ww.y + b0v * ww.x, a1 * ww.w + b1 * ww.z);
-                    }
-                    *reinterpret_cast<uint4*>(rowp + hi * 128) = make_uint4(r_[0], r_[1], r_[2], r_[3]);
-                    *reinterpret_cast<uint4*>(rowp + (4 + hi) * 128) = make_uint4(i_[0], i_[1], i_[2], i_[3]);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) w[q] = wn[q];
                 }
             }
         }
@@ -433,18 +436,27 @@ conv32k_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ 
                 tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 4; ++i) tmem_ld_fence8(v + 8 * i);
-                __nv_bfloat16* oa = reinterpret_cast<__nv_bfloat16*>(smem + OFF_A) + n2 * 32 + n3;
+                // staging = the TMA store's 64-byte-swizzled box image (rows of 32 n3; chunk index XOR bits 7..8 of the
+                // address): a warp's 8 n2 x 4 n3 then hit 16 different banks instead of 4
+                unsigned char* oa = smem + OFF_A + ((n2 * 64 + n3 * 2) ^ (((n2 >> 1) & 3) << 4));
 #pragma unroll
                 for (int n1 = 0; n1 < 16; ++n1) {
-                    oa[n1 * 1024] = __float2bfloat16_rn(v[n1]);
-                    oa[16384 + n1 * 1024] = __float2bfloat16_rn(v[16 + n1]);
+                    *reinterpret_cast<__nv_bfloat16*>(oa + n1 * 2048) = __float2bfloat16_rn(v[n1]);
+                    *reinterpret_cast<__nv_bfloat16*>(oa + 32768 + n1 * 2048) = __float2bfloat16_rn(v[16 + n1]);
                 }
             }
         }
         M2_STAGE_SYNC()
         if (tid == 0) {
-            bulk_store(y + ((size_t)b0 * H + h) * row_elems, s_base + OFF_A, 32768);
-            if (has_b) bulk_store(y + ((size_t)(b0 + 1) * H + h) * row_elems, s_base + OFF_A + 32768, 32768);
+            // y as [rows of 32 elements]: a batch row is 512 of them, a box 256
+            const int ra = (b0 * H + h) * 512;
+            tma_store_2d(&map_y, s_base + OFF_A, 0, ra);
+            tma_store_2d(&map_y, s_base + OFF_A + 16384, 0, ra + 256);
+            if (has_b) {
+                const int rb = ((b0 + 1) * H + h) * 512;
+                tma_store_2d(&map_y, s_base + OFF_A + 32768, 0, rb);
+                tma_store_2d(&map_y, s_base + OFF_A + 49152, 0, rb + 256);
+            }
             tma_store_commit();
             store_pending = true;
         }
@@ -572,7 +584,14 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     const long long pairs = H * ((B + 1) / 2);
     const int grid = (int)(pairs < sms ? pairs : sms);
     const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * kN * 8);
-    conv32k_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y, kfu,
+    alignas(64) CUtensorMap my;
+    {
+        const cuuint64_t gdim[2] = {32, (cuuint64_t)(B * H * 512)};
+        const cuuint64_t gstr[1] = {64};
+        const cuuint32_t box[2] = {32, 256};
+        if (!tma_host::encode_sw64_bf16(&my, y, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    }
+    conv32k_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(my, (const __nv_bfloat16*)x, kfu,
                                                            (const uint4*)tb->d_const, tb->d_tn, (int)B, (int)H, pl->d_status);
     if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o3_32k";

@@ -147,8 +147,20 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         fence_barrier_init();
         prefetch_tensormap(&map_x);
     }
+    // Programmatic dependent launch: the next kernel on the stream may start its CTAs as this grid's CTAs leave
+    // their SMs; everything above the wait below touches only plan-owned constants and this CTA's own resources.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool x_pending = false, k_pending = false;
-    if (leader && u < units0) {   // first loads go out before anything else
+    // constants -> shared memory
+    {
+        uint4* dst = reinterpret_cast<uint4*>(smem_all + OFF_CONST);
+        for (int i = threadIdx.x; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
+    }
+    if (threadIdx.x < 32) tmem_alloc(s_tptr, kTmemCols);
+    // everything the stream ran before this kernel (the producer of x and of the spectrum, the previous launch's
+    // reset of the scheduler words, readers of y) is complete and visible from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (leader && u < units0) {   // first loads
         mbar_expect_tx(bar_x, 8192);
         tma_load_4d(s_base + G_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
         tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, u % H, (u / H) * kRows, bar_x);
@@ -157,12 +169,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         bulk_load(s_base + G_KF, kfu + (size_t)(u % H) * 256, 4096, bar_k);
         k_pending = true;
     }
-    // constants -> shared memory
-    {
-        uint4* dst = reinterpret_cast<uint4*>(smem_all + OFF_CONST);
-        for (int i = threadIdx.x; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
-    }
-    if (threadIdx.x < 32) tmem_alloc(s_tptr, kTmemCols);
     fence_proxy_async();   // the constant matrices are read by the async proxy (UMMA)
     tc_fence_before();
     __syncthreads();
@@ -572,9 +578,21 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     const long long ctas = (units + kGroups - 1) / kGroups;
     const int grid = (int)(ctas < sms ? ctas : sms);
     const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * 512 * 8);
-    conv512_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H,
-                                                           (int)n, pl->d_status, t->d_sched);
-    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    // launched with programmatic stream serialization: its CTAs may take over SMs that the previous kernel's CTAs
+    // have left while that kernel's last CTAs still run (the kernel waits for it before touching its data)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n,
+                           pl->d_status, t->d_sched) != cudaSuccess)
+        return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o2_512";
     pl->launches += 1;
     return M2_OK;

@@ -149,15 +149,19 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
         *abort_flag = 0;
         fence_barrier_init();
     }
-    if (pr_i < pairs) {
-        const int h = pr_i / bpairs, b0 = (pr_i % bpairs) * 2;
-        load_pair(s_base + OFF_X, x + ((size_t)b0 * H + h) * row_elems, x + ((size_t)(b0 + 1) * H + h) * row_elems, b0 + 1 < B);
-    }
+    // Programmatic dependent launch: the next kernel's CTAs may take over SMs as this grid's CTAs leave them; the
+    // plan-owned constants and the TMEM allocation do not depend on anything the stream ran before.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     {
         uint4* dst = reinterpret_cast<uint4*>(smem + OFF_CONST);
         for (int i = tid; i < CONST_BYTES / 16; i += kThreads) dst[i] = consts[i];
     }
     if (tid < 32) tmem_alloc(s_tptr, 512);
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // producers of x / the spectrum and earlier users of y are done
+    if (pr_i < pairs) {
+        const int h = pr_i / bpairs, b0 = (pr_i % bpairs) * 2;
+        load_pair(s_base + OFF_X, x + ((size_t)b0 * H + h) * row_elems, x + ((size_t)(b0 + 1) * H + h) * row_elems, b0 + 1 < B);
+    }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -591,9 +595,19 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
         const cuuint32_t box[2] = {32, 256};
         if (!tma_host::encode_sw64_bf16(&my, y, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
     }
-    conv32k_kernel<<<grid, kThreads, SMEM_BYTES, stream>>>(my, (const __nv_bfloat16*)x, kfu,
-                                                           (const uint4*)tb->d_const, tb->d_tn, (int)B, (int)H, pl->d_status);
-    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, conv32k_kernel, my, (const __nv_bfloat16*)x, kfu, (const uint4*)tb->d_const, (const float2*)tb->d_tn,
+                           (int)B, (int)H, pl->d_status) != cudaSuccess)
+        return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o3_32k";
     pl->launches += 1;
     return M2_OK;

@@ -86,12 +86,17 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
         fence_barrier_init();
     }
     if (tid < 32) tmem_alloc(s_tptr, 512);
+    // Programmatic dependent launch: the next kernel's CTAs may take over SMs as this grid's CTAs leave them.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // weight blocks -> swizzled K-major B operands ([64 out][64 in], rows of 128 bytes)
     for (int c = tid; c < kGroup * 64 * 8; c += kThreads) {
         const int kc = c & 7, o = (c >> 3) & 63, bl = c >> 9;
         cp_async16(s_base + OFF_B + bl * 8192 + sw_off(o, kc), W + ((size_t)(grp * kGroup + bl) * 64 + o) * 64 + kc * 8, 16u);
     }
+    // The weights are the caller's and were complete before this call; everything else (pass 1's z for pass 2, the
+    // producer of x, earlier readers of the buffers written here) is awaited now.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (PASS == 1) {
         // unit = (token tt, group g of 8 consecutive n1): 8 loads of 16 bytes (8 values of n2 each), an 8 x 8
         // transpose in registers, 8 stores (one per n2) of the 8 n1 values = chunk g of row tt of A_{n2}
@@ -211,11 +216,22 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     const cuuint64_t gdim[3] = {64, (cuuint64_t)T, 64}, gstr[2] = {8192, 128};
     const cuuint32_t box[3] = {8, (cuuint32_t)kTileT, 64};
     if (!tma_host::encode_bf16(&my, Y, 3, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
-    monarch64_pass_kernel<1><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)X, (const __nv_bfloat16*)R, my,
-                                                                     (__nv_bfloat16*)ws, T, pl->d_status);
-    monarch64_pass_kernel<2><<<grid, kThreads, SMEM_BYTES, stream>>>((const __nv_bfloat16*)ws, (const __nv_bfloat16*)L, my,
-                                                                     nullptr, T, pl->d_status);
-    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, monarch64_pass_kernel<1>, (const __nv_bfloat16*)X, (const __nv_bfloat16*)R, my, (__nv_bfloat16*)ws,
+                           (long long)T, pl->d_status) != cudaSuccess)
+        return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, monarch64_pass_kernel<2>, (const __nv_bfloat16*)ws, (const __nv_bfloat16*)L, my,
+                           (__nv_bfloat16*)nullptr, (long long)T, pl->d_status) != cudaSuccess)
+        return M2_ERR_CUDA;
     pl->last_kernel = "matmul_umma_64x64";
     pl->launches += 2;
     return M2_OK;

@@ -316,3 +316,43 @@ def test_host_buffer_entry_points():
     ref = O.monarch_apply(c3["L"].astype(np.float64), c3["R"].astype(np.float64), c3["X"].astype(np.float64))
     check(host(Yh), ref, TOL_BF16, "matmul host entry")
     plan.close()
+
+
+def test_back_to_back_calls_see_each_other():
+    """The tensor-core kernels are launched so that a kernel's CTAs may start while the previous kernel's
+    last CTAs still run; a call that consumes the previous call's output (no synchronisation in between,
+    output buffers reused in place) must still give what the synchronised sequence gives."""
+    c = synth.config2(B=32, H=96)
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)
+    kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+    x = dev(c["x"], torch.bfloat16)
+    ref = x
+    for _ in range(4):   # synchronised chain
+        ref = M.m2_monarch_conv_fwd(plan, ref, kf, M.M2_CIRCULAR)
+        torch.cuda.synchronize()
+    a, b = torch.empty_like(x), torch.empty_like(x)
+    M.m2_monarch_conv_fwd(plan, x, kf, M.M2_CIRCULAR, y=a)       # unsynchronised chain, ping-pong buffers
+    M.m2_monarch_conv_fwd(plan, a, kf, M.M2_CIRCULAR, y=b)
+    M.m2_monarch_conv_fwd(plan, b, kf, M.M2_CIRCULAR, y=a)
+    M.m2_monarch_conv_fwd(plan, a, kf, M.M2_CIRCULAR, y=b)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert torch.equal(b, ref)
+    plan.close()
+
+    c3 = synth.config3(T=2048, b=64)
+    plan = M.Plan((64, 64), dtype=M.M2_BF16, device=0)
+    X, L, R = dev(c3["X"], torch.bfloat16), dev(c3["L"], torch.bfloat16), dev(c3["R"], torch.bfloat16)
+    ws = M.m2_matmul_workspace(plan, X.shape[0])
+    ref = X
+    for _ in range(3):
+        ref = M.m2_monarch_matmul(plan, ref, L, R, ws=ws)
+        torch.cuda.synchronize()
+    A, Bb = torch.empty_like(X), torch.empty_like(X)
+    M.m2_monarch_matmul(plan, X, L, R, A, ws=ws)
+    M.m2_monarch_matmul(plan, A, L, R, Bb, ws=ws)
+    M.m2_monarch_matmul(plan, Bb, L, R, A, ws=ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "matmul_umma_64x64"
+    assert torch.equal(A, ref)
+    plan.close()

@@ -47,8 +47,7 @@ constexpr int OFF_X = 131072;            // packed input pair, S1's A operand   
 constexpr int OFF_CONST = 196608;        // B1 4096 | BF 8192 | BI 8192 | B6 4096 | tw 8704
 constexpr int CONST_BYTES = 4096 + 8192 + 8192 + 4096 + 8704;
 constexpr int OFF_B1 = OFF_CONST, OFF_BF = OFF_B1 + 4096, OFF_BI = OFF_BF + 8192, OFF_B6 = OFF_BI + 8192;
-constexpr int OFF_TW = OFF_B6 + 4096;    // w_1024^{a b}, rows padded to 34 entries
-constexpr int TW_STRIDE = 34;
+constexpr int OFF_TW = OFF_B6 + 4096;    // w_1024^{a b}: row a = 17 float4 (cos b, cos b+1, sin b, sin b+1), b even
 constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // bar_mma, flag, tmem ptr
 constexpr int SMEM_BYTES = OFF_BAR + 64;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
@@ -94,26 +93,48 @@ __device__ __forceinline__ void load_tile(uint32_t taddr, float* re, float* im) 
     }
 }
 
-// 8 complex values (re, im) -> two 16-byte chunks of bf16
-__device__ __forceinline__ void pack8(const float* re, const float* im, uint4& pr, uint4& pi) {
-    pr = make_uint4(pack_bf16(re[0], re[1]), pack_bf16(re[2], re[3]), pack_bf16(re[4], re[5]), pack_bf16(re[6], re[7]));
-    pi = make_uint4(pack_bf16(im[0], im[1]), pack_bf16(im[2], im[3]), pack_bf16(im[4], im[5]), pack_bf16(im[6], im[7]));
+// Two neighbouring complex values (re pair a0 a1, im pair b0 b1) times (c + i s) given as packed pairs c2, s2;
+// the products leave as bf16 pairs.  Packed fp32 arithmetic: 5 instructions for the two complex products.
+__device__ __forceinline__ void cmul2_pack(float a0, float a1, float b0, float b1, uint64_t c2, uint64_t s2, uint32_t& pr, uint32_t& pi) {
+    const uint64_t a2 = pk2(a0, a1), b2 = pk2(b0, b1);
+    const uint64_t r2 = fma2(sub2(0ull, b2), s2, mul2(a2, c2));   // a c - b s
+    const uint64_t i2 = fma2(b2, c2, mul2(a2, s2));               // a s + b c
+    float x0, x1, y0, y1;
+    upk2(r2, x0, x1);
+    upk2(i2, y0, y1);
+    pr = pack_bf16(x0, x1);
+    pi = pack_bf16(y0, y1);
+}
+// the same times the conjugate (c - i s)
+__device__ __forceinline__ void cmul2_conj_pack(float a0, float a1, float b0, float b1, uint64_t c2, uint64_t s2, uint32_t& pr, uint32_t& pi) {
+    const uint64_t a2 = pk2(a0, a1), b2 = pk2(b0, b1);
+    const uint64_t r2 = fma2(b2, s2, mul2(a2, c2));               // a c + b s
+    const uint64_t i2 = fma2(sub2(0ull, a2), s2, mul2(b2, c2));   // b c - a s
+    float x0, x1, y0, y1;
+    upk2(r2, x0, x1);
+    upk2(i2, y0, y1);
+    pr = pack_bf16(x0, x1);
+    pi = pack_bf16(y0, y1);
 }
 
-// multiplies the 32 complex values by f0 * rho^i, i = 0..31 (four chains of eight)
-__device__ __forceinline__ void mul_geometric(float* re, float* im, float2 f0, float2 rho, float2 rho8, float2 rho16, float2 rho24) {
-    float2 f[4] = {f0, cmul(f0, rho8), cmul(f0, rho16), cmul(f0, rho24)};
+// 8 complex values times f, f rho, ..., f rho^7: the factors of neighbouring values run as one packed chain that
+// steps by rho^2 (three steps per call)
+__device__ __forceinline__ void geometric8_pack(const float* re, const float* im, float2 f, float2 rho, uint4& pr, uint4& pi) {
+    const float2 g = cmul(f, rho), q = cmul(rho, rho);
+    uint64_t fr = pk2(f.x, g.x), fi = pk2(f.y, g.y);
+    const uint64_t qr = pk2(q.x, q.x), qi = pk2(q.y, q.y), nqi = pk2(-q.y, -q.y);
+    uint32_t r_[4], i_[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const int e = 8 * c + i;
-            const float a = re[e], b = im[e];
-            re[e] = a * f[c].x - b * f[c].y;
-            im[e] = a * f[c].y + b * f[c].x;
-            f[c] = cmul(f[c], rho);
+    for (int p = 0; p < 4; ++p) {
+        cmul2_pack(re[2 * p], re[2 * p + 1], im[2 * p], im[2 * p + 1], fr, fi, r_[p], i_[p]);
+        if (p < 3) {
+            const uint64_t nr = fma2(fi, nqi, mul2(fr, qr)), ni = fma2(fi, qr, mul2(fr, qi));
+            fr = nr;
+            fi = ni;
         }
     }
+    pr = make_uint4(r_[0], r_[1], r_[2], r_[3]);
+    pi = make_uint4(i_[0], i_[1], i_[2], i_[3]);
 }
 
 // loads one packed input pair (rows a and b of channel h) into the S1 operand layout
@@ -168,7 +189,11 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 16);
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-    const float2* tw = reinterpret_cast<const float2*>(smem + OFF_TW);   // w_1024^{a b} at [a * 34 + b]
+    const float4* tw4 = reinterpret_cast<const float4*>(smem + OFF_TW);   // row a: tw4[a * 17 + b / 2]
+    auto tw_at = [&](int a, int b) {                                       // w_1024^{a b} as one complex value
+        const float* p = reinterpret_cast<const float*>(tw4 + a * 17 + (b >> 1)) + (b & 1);
+        return make_float2(p[0], p[2]);
+    };
 
     constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
     constexpr uint32_t ID_MM = instr_desc_bf16(128, 64, true, false);    // M-major A, N = 64
@@ -236,23 +261,19 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                 const int n2 = 4 * j + (t >> 5), n3 = t & 31;
                 float re[32], im[32];
                 load_tile(t_lane + j * 64, re, im);
-                const float4* twr = reinterpret_cast<const float4*>(tw + n2 * TW_STRIDE);   // warp-uniform row
-#pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    const float4 w = twr[q];
-                    const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-                    re[2 * q] = a0 * w.x - b0v * w.y;
-                    im[2 * q] = a0 * w.y + b0v * w.x;
-                    re[2 * q + 1] = a1 * w.z - b1 * w.w;
-                    im[2 * q + 1] = a1 * w.w + b1 * w.z;
-                }
+                const float4* twr = tw4 + n2 * 17;   // warp-uniform row
 #pragma unroll
                 for (int hi = 0; hi < 4; ++hi) {
-                    uint4 pr, pi;
-                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    uint32_t r_[4], i_[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 w = twr[4 * hi + q];
+                        cmul2_pack(re[8 * hi + 2 * q], re[8 * hi + 2 * q + 1], im[8 * hi + 2 * q], im[8 * hi + 2 * q + 1], pk2(w.x, w.y),
+                                   pk2(w.z, w.w), r_[q], i_[q]);
+                    }
                     const int mb = (n3 >> 3) * 4 + hi;
-                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (n2 >> 3), n2 & 7, n3 & 7)) = pr;
-                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (n2 >> 3), n2 & 7, n3 & 7)) = pi;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (n2 >> 3), n2 & 7, n3 & 7)) = make_uint4(r_[0], r_[1], r_[2], r_[3]);
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (n2 >> 3), n2 & 7, n3 & 7)) = make_uint4(i_[0], i_[1], i_[2], i_[3]);
                 }
             }
         }
@@ -277,12 +298,11 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                 const int k1 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), n3 = ((j >> 1) << 3) + ((t >> 3) & 7);
                 float re[32], im[32];
                 load_tile(t_lane + j * 64, re, im);
-                const float2* r3 = tw + n3 * TW_STRIDE;
-                mul_geometric(re, im, __ldg(tn + n3 * 32 + k1), r3[1], r3[8], r3[16], r3[24]);
+                const float2 f0 = __ldg(tn + n3 * 32 + k1), rho = tw_at(n3, 1);
 #pragma unroll
                 for (int hi = 0; hi < 4; ++hi) {
                     uint4 pr, pi;
-                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    geometric8_pack(re + 8 * hi, im + 8 * hi, hi == 0 ? f0 : cmul(f0, tw_at(n3, 8 * hi)), rho, pr, pi);
                     const int mb = (k1 >> 3) * 4 + hi;
                     *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (n3 >> 3), n3 & 7, k1 & 7)) = pr;
                     *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (n3 >> 3), n3 & 7, k1 & 7)) = pi;
@@ -327,9 +347,7 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                         for (int q = 0; q < 4; ++q) {
                             const float4 ww = w[4 * hi + q];
                             if (jj == 0) w[4 * hi + q] = __ldg(kp0 + (size_t)4 * 16 * 128 + (4 * hi + q) * 128);   // tile wg + 4
-                            const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-                            r_[q] = pack_bf16(a0 * ww.x - b0v * ww.y, a1 * ww.z - b1 * ww.w);
-                            i_[q] = pack_bf16(a0 * ww.y + b0v * ww.x, a1 * ww.w + b1 * ww.z);
+                            cmul2_pack(re[2 * q], re[2 * q + 1], im[2 * q], im[2 * q + 1], pk2(ww.x, ww.y), pk2(ww.z, ww.w), r_[q], i_[q]);
                         }
                         *reinterpret_cast<uint4*>(rowp + hi * 128) = make_uint4(r_[0], r_[1], r_[2], r_[3]);
                         *reinterpret_cast<uint4*>(rowp + (4 + hi) * 128) = make_uint4(i_[0], i_[1], i_[2], i_[3]);
@@ -358,16 +376,14 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                 const int k2 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
                 float re[32], im[32];
                 load_tile(t_lane + j * 64, re, im);
-                // rho^m = conj( w_N^{m k1} w_1024^{m k2} ), m = 1, 8, 16, 24
-                const float2 rho = conjf(cmul(__ldg(tn + 1 * 32 + k1), tw[1 * TW_STRIDE + k2]));
-                const float2 rho8 = conjf(cmul(__ldg(tn + 8 * 32 + k1), tw[8 * TW_STRIDE + k2]));
-                const float2 rho16 = conjf(cmul(__ldg(tn + 16 * 32 + k1), tw[16 * TW_STRIDE + k2]));
-                const float2 rho24 = conjf(cmul(__ldg(tn + 24 * 32 + k1), tw[24 * TW_STRIDE + k2]));
-                mul_geometric(re, im, make_float2(1.f, 0.f), rho, rho8, rho16, rho24);
+                // rho^m = conj( w_N^{m k1} w_1024^{m k2} )
+                const float2 rho = conjf(cmul(__ldg(tn + 1 * 32 + k1), tw_at(1, k2)));
 #pragma unroll
                 for (int hi = 0; hi < 4; ++hi) {
+                    float2 f = make_float2(1.f, 0.f);
+                    if (hi > 0) f = conjf(cmul(__ldg(tn + 8 * hi * 32 + k1), tw_at(8 * hi, k2)));
                     uint4 pr, pi;
-                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    geometric8_pack(re + 8 * hi, im + 8 * hi, f, rho, pr, pi);
                     const int mb = (k1 >> 3) * 4 + hi;
                     *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (k2 >> 3), k2 & 7, k1 & 7)) = pr;
                     *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (k2 >> 3), k2 & 7, k1 & 7)) = pi;
@@ -395,23 +411,19 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                 const int n3 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
                 float re[32], im[32];
                 load_tile(t_lane + j * 64, re, im);
-                const float4* twr = reinterpret_cast<const float4*>(tw + k1 * TW_STRIDE);
-#pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    const float4 w = twr[q];   // conjugate: (a + ib)(c - is)
-                    const float a0 = re[2 * q], b0v = im[2 * q], a1 = re[2 * q + 1], b1 = im[2 * q + 1];
-                    re[2 * q] = a0 * w.x + b0v * w.y;
-                    im[2 * q] = b0v * w.x - a0 * w.y;
-                    re[2 * q + 1] = a1 * w.z + b1 * w.w;
-                    im[2 * q + 1] = b1 * w.z - a1 * w.w;
-                }
+                const float4* twr = tw4 + k1 * 17;
 #pragma unroll
                 for (int hi = 0; hi < 4; ++hi) {
-                    uint4 pr, pi;
-                    pack8(re + 8 * hi, im + 8 * hi, pr, pi);
+                    uint32_t r_[4], i_[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 w = twr[4 * hi + q];
+                        cmul2_conj_pack(re[8 * hi + 2 * q], re[8 * hi + 2 * q + 1], im[8 * hi + 2 * q], im[8 * hi + 2 * q + 1], pk2(w.x, w.y),
+                                        pk2(w.z, w.w), r_[q], i_[q]);
+                    }
                     const int mb = hi * 4 + (n3 >> 3);
-                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (k1 >> 3), k1 & 7, n3 & 7)) = pr;
-                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (k1 >> 3), k1 & 7, n3 & 7)) = pi;
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, (k1 >> 3), k1 & 7, n3 & 7)) = make_uint4(r_[0], r_[1], r_[2], r_[3]);
+                    *reinterpret_cast<uint4*>(smem + OFF_A + a_off(mb, 4 + (k1 >> 3), k1 & 7, n3 & 7)) = make_uint4(i_[0], i_[1], i_[2], i_[3]);
                 }
             }
         }
@@ -478,7 +490,7 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
     if (tid < 32) tmem_dealloc(tmem, 512);
 }
 
-// spectrum in the layout h3 reads: kfu[h][tile j][q = k3 / 2][lane t] = (re, im)(k3 = 2q), (re, im)(k3 = 2q + 1)
+// spectrum in the layout h3 reads: kfu[h][tile j][q = k3 / 2][lane t] = (re(2q), re(2q + 1), im(2q), im(2q + 1))
 // for (k1, k2) = lane map of D3; plan order is [k1][k2][k3].
 __global__ void relayout_spectrum3_kernel(const float2* __restrict__ kf, float4* __restrict__ kfu, long long total) {
     const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 8 * 16 * 128
@@ -487,7 +499,7 @@ __global__ void relayout_spectrum3_kernel(const float2* __restrict__ kf, float4*
     const long long h = i >> 14;
     const int k2 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
     const float2* src = kf + h * kN + (k1 * 32 + k2) * 32 + 2 * q;
-    kfu[i] = make_float4(src[0].x, src[0].y, src[1].x, src[1].y);
+    kfu[i] = make_float4(src[0].x, src[1].x, src[0].y, src[1].y);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------------------
@@ -529,12 +541,12 @@ cudaError_t create_tables(m2_plan* pl) {
     fill(BF, 64, 32, 32, false);   // [64][64]
     fill(BI, 64, 32, 32, true);    // conjugate
     fill(B6, 64, 16, 32, true);    // [N = (c, n1 < 16) 32][K = (c, k1) 64], conjugate
-    std::vector<float> tw(32 * TW_STRIDE * 2, 0.f), tn(32 * 32 * 2);
+    std::vector<float> tw(32 * 17 * 4, 0.f), tn(32 * 32 * 2);
     for (int a = 0; a < 32; ++a)
         for (int b = 0; b < 32; ++b) {
             const double t1 = 2.0 * M_PI * ((a * b) % 1024) / 1024.0, t2 = 2.0 * M_PI * ((a * b) % kN) / (double)kN;
-            tw[(a * TW_STRIDE + b) * 2] = (float)std::cos(t1);
-            tw[(a * TW_STRIDE + b) * 2 + 1] = (float)(sg * std::sin(t1));
+            tw[(a * 17 + b / 2) * 4 + (b & 1)] = (float)std::cos(t1);
+            tw[(a * 17 + b / 2) * 4 + 2 + (b & 1)] = (float)(sg * std::sin(t1));
             tn[(a * 32 + b) * 2] = (float)std::cos(t2);
             tn[(a * 32 + b) * 2 + 1] = (float)(sg * std::sin(t2));
         }

@@ -11,6 +11,7 @@
 #include "conv_umma.h"
 #include "generic_kernels.h"
 #include "matmul_umma.h"
+#include "mlp_umma.h"
 #include "m2_plan.h"
 
 // Scratch of m2_block_fwd_static: the intermediate z of the block forward for callers that cannot
@@ -351,10 +352,16 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
     cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z_dev, w_short_dev, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;
-    e = m2g::launch_mlp(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return M2_ERR_CUDA;
-    plan->last_kernel = "block_generic";
+    if (m2mlp::covered((int)C, nblk, expand)) {   // tensor-core MLP for 192 -> 768 -> 192 blocks
+        const int32_t st = m2mlp::launch(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
+        if (st != M2_OK) return st;
+        plan->last_kernel = "block_conv_generic_mlp_umma";
+    } else {
+        e = m2g::launch_mlp(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
+        if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+        if (e != cudaSuccess) return M2_ERR_CUDA;
+        plan->last_kernel = "block_generic";
+    }
     plan->launches += 2;
     return M2_OK;
 }
@@ -396,9 +403,14 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
     cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z, w_short_dev, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;
-    e = m2g::launch_mlp(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return M2_ERR_CUDA;
+    if (m2mlp::covered((int)C, nblk, expand)) {
+        const int32_t st = m2mlp::launch(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
+        if (st != M2_OK) return st;
+    } else {
+        e = m2g::launch_mlp(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
+        if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+        if (e != cudaSuccess) return M2_ERR_CUDA;
+    }
     plan->last_kernel = "block_generic_static_scratch";
     plan->launches += 2;
     return M2_OK;

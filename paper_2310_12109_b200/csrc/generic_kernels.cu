@@ -446,4 +446,79 @@ cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y,
     return cudaGetLastError();
 }
 
+// ---- channel-last <-> channel-first helpers of the M2 block (Sec. 5.1; Eq. 2 runs along the sequence) -----------------
+// x[B][T][C] -> xT[B][C][T] through a 64 x 64 shared-memory tile; both sides move whole 128-byte rows.
+__global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xT, int T, int C) {
+    __shared__ __nv_bfloat16 tile[64][66];
+    const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+    const long long b = blockIdx.z;
+    const __nv_bfloat16* src = x + (b * T + t0) * (long long)C + c0;
+    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+        const int tt = i >> 5, cp = i & 31;
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src + (long long)tt * C + 2 * cp);
+        tile[tt][2 * cp] = v.x;
+        tile[tt][2 * cp + 1] = v.y;
+    }
+    __syncthreads();
+    __nv_bfloat16* dst = xT + (b * C + c0) * (long long)T + t0;
+    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+        const int cc = i >> 5, tp = i & 31;
+        __nv_bfloat162 v;
+        v.x = tile[2 * tp][cc];
+        v.y = tile[2 * tp + 1][cc];
+        *reinterpret_cast<__nv_bfloat162*>(dst + (long long)cc * T + 2 * tp) = v;
+    }
+}
+
+// z[b][t][c] = (w[c][0] x[b][t-1][c] + w[c][1] x[b][t][c] + w[c][2] x[b][t+1][c]) * v[b][c][t]: the width-3 depthwise
+// gate (zero padded) times the long-convolution output, which arrives channel-first and leaves channel-last.
+__global__ void __launch_bounds__(256) gate_transpose_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ vT,
+                                                             const float* __restrict__ w, __nv_bfloat16* __restrict__ z, int T, int C) {
+    __shared__ __nv_bfloat16 tile[64][66];   // [c][t]
+    const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+    const long long b = blockIdx.z;
+    const __nv_bfloat16* src = vT + (b * C + c0) * (long long)T + t0;
+    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+        const int cc = i >> 5, tp = i & 31;
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src + (long long)cc * T + 2 * tp);
+        tile[cc][2 * tp] = v.x;
+        tile[cc][2 * tp + 1] = v.y;
+    }
+    __syncthreads();
+    const __nv_bfloat16* xb = x + b * (long long)T * C;
+    __nv_bfloat16* zb = z + b * (long long)T * C;
+    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+        const int tt = i >> 5, cp = i & 31, t = t0 + tt, c = c0 + 2 * cp;
+        const float2 xm = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(xb + (long long)t * C + c));
+        float g0 = w[c * 3 + 1] * xm.x, g1 = w[c * 3 + 4] * xm.y;
+        if (t > 0) {
+            const float2 xl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(xb + (long long)(t - 1) * C + c));
+            g0 = fmaf(w[c * 3 + 0], xl.x, g0);
+            g1 = fmaf(w[c * 3 + 3], xl.y, g1);
+        }
+        if (t + 1 < T) {
+            const float2 xr = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(xb + (long long)(t + 1) * C + c));
+            g0 = fmaf(w[c * 3 + 2], xr.x, g0);
+            g1 = fmaf(w[c * 3 + 5], xr.y, g1);
+        }
+        *reinterpret_cast<__nv_bfloat162*>(zb + (long long)t * C + c) =
+            __floats2bfloat162_rn(g0 * __bfloat162float(tile[2 * cp][tt]), g1 * __bfloat162float(tile[2 * cp + 1][tt]));
+    }
+}
+
+cudaError_t launch_transpose_btc(const void* x, void* xT, long long B, int T, int C, cudaStream_t st) {
+    if (T % 64 != 0 || C % 64 != 0) return cudaErrorInvalidValue;
+    if (B == 0) return cudaSuccess;
+    transpose_btc_kernel<<<dim3(T / 64, C / 64, (unsigned)B), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)xT, T, C);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w, void* z, long long B, int T, int C, cudaStream_t st) {
+    if (T % 64 != 0 || C % 64 != 0) return cudaErrorInvalidValue;
+    if (B == 0) return cudaSuccess;
+    gate_transpose_kernel<<<dim3(T / 64, C / 64, (unsigned)B), 256, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)vT, w,
+                                                                              (__nv_bfloat16*)z, T, C);
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

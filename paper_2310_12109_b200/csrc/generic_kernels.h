@@ -23,4 +23,8 @@ cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void*
 cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,
                        long long tokens, cudaStream_t st);
 
+// M2 block helpers (bf16): x[B][T][C] -> xT[B][C][T];  z[b][t][c] = gate3(x)[b][t][c] * vT[b][c][t]  (T, C multiples of 64)
+cudaError_t launch_transpose_btc(const void* x, void* xT, long long B, int T, int C, cudaStream_t st);
+cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w, void* z, long long B, int T, int C, cudaStream_t st);
+
 }  // namespace m2g

@@ -330,6 +330,35 @@ int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const vo
     return M2_OK;
 }
 
+namespace {
+
+// Sequence mix + gate of the M2 block, z[B][T][C] = gate3(x) (.) circular_conv(x, k) along T.  Plans the tensor-core
+// order-2 kernel covers take the channel-first route: x -> xT[B][C][T] (in z), long convolution on the tensor cores
+// (into y, which the MLP overwrites afterwards), then the gate kernel transposes back into z.  Other plans run the
+// strided CUDA-core kernel.  Returns the number of launches to add to the plan's count or a negative status.
+int32_t block_mix_gate(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev, void* z, void* y_scratch,
+                       int64_t B, int64_t T, int64_t C, cudaStream_t stream, bool* tensor_core) {
+    *tensor_core = false;
+    if (m2u::has_private_spectrum(plan) && !m2u3::covered(plan) && T == 512 && C % 64 == 0) {
+        if (m2g::launch_transpose_btc(x_dev, z, B, (int)T, (int)C, stream) != cudaSuccess) return -M2_ERR_CUDA;
+        const int32_t st = m2u::conv_fwd(plan, z, kf_dev, y_scratch, B, C, T, M2_CIRCULAR, stream);
+        if (st != M2_OK) return -st;
+        if (m2g::launch_gate_transpose(x_dev, y_scratch, w_short_dev, z, B, (int)T, (int)C, stream) != cudaSuccess) return -M2_ERR_CUDA;
+        *tensor_core = true;
+        return 2;   // (the convolution counts its own launch)
+    }
+    m2g::ConvShape s = conv_shape(plan, B, C, T);
+    s.stride_b = T * C;
+    s.stride_h = 1;
+    s.stride_e = C;
+    const cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z, w_short_dev, stream);
+    if (e == cudaErrorInvalidValue) return -M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return -M2_ERR_CUDA;
+    return 1;
+}
+
+}  // namespace
+
 int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
                      const void* W_up_dev, const void* W_down_dev, void* z_dev, void* y_dev, int64_t B, int64_t T,
                      int64_t C, int32_t nblk, int32_t expand, void* stream) {
@@ -344,25 +373,21 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
     if (B == 0) return M2_OK;
-    // sequence mix + gate: rows are (b, c), elements strided by C along the sequence
-    m2g::ConvShape s = conv_shape(plan, B, C, T);
-    s.stride_b = T * C;
-    s.stride_h = 1;
-    s.stride_e = C;
-    cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z_dev, w_short_dev, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return M2_ERR_CUDA;
+    bool tc_mix = false;
+    const int32_t nl = block_mix_gate(plan, x_dev, kf_dev, w_short_dev, z_dev, y_dev, B, T, C, (cudaStream_t)stream, &tc_mix);
+    if (nl < 0) return -nl;
+    cudaError_t e = cudaSuccess;
     if (m2mlp::covered((int)C, nblk, expand)) {   // tensor-core MLP for 192 -> 768 -> 192 blocks
         const int32_t st = m2mlp::launch(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
         if (st != M2_OK) return st;
-        plan->last_kernel = "block_conv_generic_mlp_umma";
+        plan->last_kernel = tc_mix ? "block_conv_umma_mlp_umma" : "block_conv_generic_mlp_umma";
     } else {
         e = m2g::launch_mlp(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
         if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
         if (e != cudaSuccess) return M2_ERR_CUDA;
-        plan->last_kernel = "block_generic";
+        plan->last_kernel = tc_mix ? "block_conv_umma_mlp_generic" : "block_generic";
     }
-    plan->launches += 2;
+    plan->launches += nl + 1;
     return M2_OK;
 }
 
@@ -394,15 +419,12 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
         z = g_static_ptr[plan->device];
     }
     if (B == 0) return M2_OK;
-    // Same two launches as m2_block_fwd; the conv + gate kernel writes every element of z[B, T, C] before the
-    // MLP kernel reads it, so the array's previous contents never matter.
-    m2g::ConvShape s = conv_shape(plan, B, C, T);
-    s.stride_b = T * C;
-    s.stride_h = 1;
-    s.stride_e = C;
-    cudaError_t e = m2g::launch_conv(s, true, x_dev, kf_dev, z, w_short_dev, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return M2_ERR_CUDA;
+    // Same launches as m2_block_fwd; every element of z[B, T, C] is written before it is read, so the array's
+    // previous contents never matter.
+    bool tc_mix = false;
+    const int32_t nl = block_mix_gate(plan, x_dev, kf_dev, w_short_dev, z, y_dev, B, T, C, (cudaStream_t)stream, &tc_mix);
+    if (nl < 0) return -nl;
+    cudaError_t e = cudaSuccess;
     if (m2mlp::covered((int)C, nblk, expand)) {
         const int32_t st = m2mlp::launch(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
         if (st != M2_OK) return st;
@@ -412,7 +434,7 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
         if (e != cudaSuccess) return M2_ERR_CUDA;
     }
     plan->last_kernel = "block_generic_static_scratch";
-    plan->launches += 2;
+    plan->launches += nl + 1;
     return M2_OK;
 }
 

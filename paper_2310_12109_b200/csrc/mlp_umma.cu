@@ -44,7 +44,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+// GELU(v) = v/2 (1 + erf(v / sqrt 2)), erf by the five-term rational-exponential form
+//   erf(a) = 1 - (c1 t + c2 t^2 + c3 t^3 + c4 t^4 + c5 t^5) exp(-a^2),  t = 1 / (1 + p a),  a >= 0
+// (Abramowitz & Stegun 7.1.26, absolute error < 1.5e-7: far below the bf16 rounding of the result); one reciprocal
+// and one exponential on the special-function unit, the rest fused multiply-adds.
+__device__ __forceinline__ float gelu_erf(float v) {
+    const float a = fabsf(v) * 0.70710678118654752f;
+    float t, e;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, a, 1.0f)));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(a * a * -1.4426950408889634f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float erf_a = fmaf(-poly * t, e, 1.0f);          // erf(|v| / sqrt 2)
+    return 0.5f * v + 0.5f * fabsf(v) * erf_a;             // v/2 (1 + sign(v) erf_a)
+}
 // byte offset of 16-byte chunk kc of row r in a K-major block with 128-byte rows and the 128B swizzle
 __device__ __forceinline__ uint32_t sw_off(int r, int kc) { return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((kc ^ (r & 7)) << 4)); }
 
@@ -93,19 +108,30 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         if (lane == 0) {
             mbar_expect_tx(bar(B_Z), 49152);
             for (int kb = 0; kb < 3; ++kb) tma_load_2d(s_base + OFF_Z + kb * 16384, &map_z, j * kCI + kb * 64, t0, bar(B_Z));
-            for (int c = 0; c < kChunks && ok; ++c) {
-                const int b = c & 1;
-                if (c >= 2) ok = mbar_wait(bar(B_W1E + b), ((c >> 1) - 1) & 1);   // S1(c - 2) has read this buffer
-                if (!ok) break;
-                mbar_expect_tx(bar(B_W1F + b), 49152);
-                for (int kb = 0; kb < 3; ++kb)
-                    tma_load_2d(s_base + OFF_W1 + b * 49152 + kb * 16384, &map_w1, kb * 64, j * kHID + c * kChunk, bar(B_W1F + b));
-                if (c >= 1) ok = mbar_wait(bar(B_W2E), (c - 1) & 1);                 // S2(c - 1) has read the W_down chunk
-                if (!ok) break;
-                mbar_expect_tx(bar(B_W2F), 49152);
-                for (int kb = 0; kb < 2; ++kb)
-                    tma_load_2d(s_base + OFF_W2 + kb * 24576, &map_w2, c * kChunk + kb * 64, j * kCO, bar(B_W2F));
+            // The two weight streams advance independently (a W_up chunk two ahead of the UMMAs, the single W_down
+            // buffer as soon as S2 has read it), so neither waits behind the other's barrier.
+            int c1 = 0, c2 = 0;
+            uint32_t idle = 0;
+            while ((c1 < kChunks || c2 < kChunks) && idle < (1u << 22)) {
+                bool progressed = false;
+                if (c1 < kChunks && (c1 < 2 || mbar_try_wait(bar(B_W1E + (c1 & 1)), ((c1 >> 1) - 1) & 1))) {   // S1(c1 - 2) has read the buffer
+                    const int bb = c1 & 1;
+                    mbar_expect_tx(bar(B_W1F + bb), 49152);
+                    for (int kb = 0; kb < 3; ++kb)
+                        tma_load_2d(s_base + OFF_W1 + bb * 49152 + kb * 16384, &map_w1, kb * 64, j * kHID + c1 * kChunk, bar(B_W1F + bb));
+                    ++c1;
+                    progressed = true;
+                }
+                if (c2 < kChunks && (c2 < 1 || mbar_try_wait(bar(B_W2E), (c2 - 1) & 1))) {                        // S2(c2 - 1) has read the chunk
+                    mbar_expect_tx(bar(B_W2F), 49152);
+                    for (int kb = 0; kb < 2; ++kb)
+                        tma_load_2d(s_base + OFF_W2 + kb * 24576, &map_w2, c2 * kChunk + kb * 64, j * kCO, bar(B_W2F));
+                    ++c2;
+                    progressed = true;
+                }
+                idle = progressed ? 0 : idle + 1;
             }
+            if (c1 < kChunks || c2 < kChunks) ok = false;
         }
     } else if (warp == 1) {
         // ---- UMMA issuer ---------------------------------------------------------------------------------------------

@@ -214,13 +214,16 @@ def test_config4_full_size_sampled():
 
 # ---- config 5: the M2 block -------------------------------------------------------------------------
 
-def run_block(c):
+def run_block(c, kernel=None):
     plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)
     kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+    nblk, hid, cin = c["W_up"].shape
     y, z = M.m2_block_fwd(plan, dev(c["x"], torch.bfloat16), kf, dev(c["w_short"]), dev(c["W_up"], torch.bfloat16),
-                          dev(c["W_down"], torch.bfloat16))
+                          dev(c["W_down"], torch.bfloat16), nblk=nblk, expand=hid // cin)
     torch.cuda.synchronize()
     assert plan.device_status() == 0
+    if kernel is not None:
+        assert plan.last_kernel() == kernel
     plan.close()
     return host(y), host(z)
 
@@ -235,10 +238,23 @@ def block_ref(c, bsel=None):
 
 def test_config5_small():
     c = synth.config5(B=2)
-    y, z = run_block(c)
+    y, z = run_block(c, "block_conv_umma_mlp_umma")
     yr, zr = block_ref(c)
     check(z.reshape(2 * 512, 768), zr.reshape(2 * 512, 768), TOL_BF16, "config5 z")
     check(y.reshape(2 * 512, 768), yr.reshape(2 * 512, 768), TOL_BF16, "config5 y")
+
+
+@pytest.mark.parametrize("T,C,nblk,expand,dims,kernel", [
+    (64, 32, 4, 2, (8, 8), "block_generic"),                       # neither tensor-core kernel covers it
+    (512, 128, 4, 2, (32, 16), "block_conv_umma_mlp_generic"),    # tensor-core mixer, CUDA-core MLP
+])
+def test_block_other_shapes(T, C, nblk, expand, dims, kernel):
+    c = synth.config5(B=3, T=T, C=C, nblk=nblk, expand=expand)
+    c["dims"] = dims
+    y, z = run_block(c, kernel)
+    yr, zr = block_ref(c)
+    check(z.reshape(-1, C), zr.reshape(-1, C), TOL_BF16, "block z")
+    check(y.reshape(-1, C), yr.reshape(-1, C), TOL_BF16, "block y")
 
 
 def test_config5_full_size_sampled():

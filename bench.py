@@ -178,9 +178,9 @@ def time_launches(fn, n, torch):
     return e0.elapsed_time(e1)
 
 
-def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4"), reps=None):
-    """Config 3 (Monarch matmul) and config 4 (order-3 causal conv): time per launch, throughput and
-    roofline fraction, outside the headline timed region."""
+def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5"), reps=None):
+    """Config 3 (Monarch matmul), config 4 (order-3 causal conv) and config 5 (M2 block forward): time per call,
+    throughput and roofline fraction, outside the headline timed region."""
     out = {}
     reps = reps if reps is not None else (3 if quick else 10)
     bf = lambda a: torch.from_numpy(a).cuda().to(torch.bfloat16)  # noqa: E731
@@ -188,6 +188,8 @@ def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "confi
         out.update(_side_config3(torch, M, synth, peaks, reps, bf))
     if "config4" in which:
         out.update(_side_config4(torch, M, synth, peaks, reps, bf))
+    if "config5" in which:
+        out.update(_side_config5(torch, M, synth, peaks, reps, bf))
     return out
 
 
@@ -236,6 +238,31 @@ def _side_config4(torch, M, synth, peaks, reps, bf):
         "TFLOPs_plain_count": fl / (ms * 1e9), "frac_of_hbm_roof": by / (ms * 1e6) / peaks["hbm_gbs"],
         "note": "plain count; the kernel executes half of it (two real rows packed as one complex row, zero-skip)",
         "roofline": {"bound": bound, "achieved": ach, "peak": pk, "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": ach / pk}}
+    plan.close()
+    return out
+
+
+def _side_config5(torch, M, synth, peaks, reps, bf):
+    """M2 block forward [32, 512, 768]: sequence mix + gate + block-diagonal MLP (4 launches + the conv)."""
+    out = {}
+    B, T, C = 32, 512, 768
+    c = synth.config5(B=B, T=T, C=C)
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=torch.cuda.current_device())
+    kf = M.m2_kernel_spectrum(plan, torch.from_numpy(c["k"]).cuda())
+    xs = [bf(c["x"]) for _ in range(3)]
+    w = torch.from_numpy(c["w_short"]).cuda()
+    Wu, Wd = bf(c["W_up"]), bf(c["W_down"])
+    f = lambda i: M.m2_block_fwd(plan, xs[i % 3], kf, w, Wu, Wd)  # noqa: E731
+    time_launches(f, 3, torch)
+    ms = time_launches(f, reps, torch) / reps
+    fl = 2.0 * 2 * B * T * C * (4 * C // 4)               # the MLP's two block-diagonal GEMMs (38.65 GFLOP)
+    by = 2 * B * T * C * 2 + 2 * Wu.numel() * 2 + C * T * 8   # x in, y out, weights, spectrum
+    t_tc = fl / (peaks["bf16_tflops_sustained"] * 1e12)
+    out["config5_block"] = {
+        "kernel": plan.last_kernel(), "ms": ms, "tokens_ch_per_s": B * T * C / (ms * 1e-3), "mlp_TFLOPs_if_all_time_were_mlp": fl / (ms * 1e9),
+        "note": "whole block (transpose, conv, gate, MLP); roofline = the MLP's tensor time plus the conv's HBM time",
+        "roofline": {"bound": "tensor", "achieved": fl / (ms * 1e9), "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": (t_tc + by / (peaks["hbm_gbs"] * 1e9)) / (ms * 1e-3)}}
     plan.close()
     return out
 
@@ -369,7 +396,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-side", action="store_true", help="skip the config-3 / config-4 side measurements")
     ap.add_argument("--quick", action="store_true", help="fewer repetitions of the side measurements")
-    ap.add_argument("--only", default=None, choices=["config3", "config4"],
+    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5"],
                     help="run just this side workload (--steps launches after 2 warm-ups) and print its JSON; used for profiling")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -80,11 +80,11 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
             mbar_init(bar(B_W1F + i), 1);
             mbar_init(bar(B_W1E + i), 1);
             mbar_init(bar(B_D1F + i), 1);
-            mbar_init(bar(B_D1E + i), 32 * kEpiWarps);
+            mbar_init(bar(B_D1E + i), kEpiWarps);   // one arrival per GELU warp
         }
         mbar_init(bar(B_W2F), 1);
         mbar_init(bar(B_W2E), 1);
-        mbar_init(bar(B_GF), 32 * kEpiWarps);
+        mbar_init(bar(B_GF), kEpiWarps);
         mbar_init(bar(B_GE), 1);
         mbar_init(bar(B_D2F), 1);
         fence_barrier_init();
@@ -188,7 +188,8 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
 #pragma unroll
             for (int i = 0; i < 4; ++i) tmem_ld_fence8(v + 8 * i);
             tc_fence_before();
-            mbar_arrive(bar(B_D1E + b));                                 // D1[b] may be overwritten
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_D1E + b));                  // this warp has read its part of D1[b]
             uint4 pk[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
@@ -202,7 +203,8 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 *reinterpret_cast<uint4*>(smem + OFF_G + (kc >> 3) * 16384 + sw_off(row, kc & 7)) = pk[i];
             }
             fence_proxy_async();
-            mbar_arrive(bar(B_GF));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(B_GF));
         }
         // ---- output: D2 -> bf16 -> staging (the Z buffer, free since the last S1) -> TMA store ---------------------
         if (ok) ok = mbar_wait(bar(B_D2F), 0);

@@ -447,26 +447,28 @@ cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y,
 }
 
 // ---- channel-last <-> channel-first helpers of the M2 block (Sec. 5.1; Eq. 2 runs along the sequence) -----------------
-// x[B][T][C] -> xT[B][C][T] through a 64 x 64 shared-memory tile; both sides move whole 128-byte rows.
+// x[B][T][C] -> xT[B][C][T] through a 64 x 64 shared-memory tile; both sides move 16 bytes per thread and whole
+// 128-byte rows per 8 threads.  The tile is stored transposed ([c][t], pitch 72 elements) so that the output side
+// reads 16 contiguous bytes.
 __global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xT, int T, int C) {
-    __shared__ __nv_bfloat16 tile[64][66];
+    __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [c][t]
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const long long b = blockIdx.z;
     const __nv_bfloat16* src = x + (b * T + t0) * (long long)C + c0;
-    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
-        const int tt = i >> 5, cp = i & 31;
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src + (long long)tt * C + 2 * cp);
-        tile[tt][2 * cp] = v.x;
-        tile[tt][2 * cp + 1] = v.y;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int i = threadIdx.x + 256 * r, tt = i >> 3, ch = i & 7;   // 8 channels c0 + 8 ch .. of row tt
+        const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)tt * C + 8 * ch);
+        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) tile[8 * ch + k][tt] = e[k];
     }
     __syncthreads();
     __nv_bfloat16* dst = xT + (b * C + c0) * (long long)T + t0;
-    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
-        const int cc = i >> 5, tp = i & 31;
-        __nv_bfloat162 v;
-        v.x = tile[2 * tp][cc];
-        v.y = tile[2 * tp + 1][cc];
-        *reinterpret_cast<__nv_bfloat162*>(dst + (long long)cc * T + 2 * tp) = v;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int i = threadIdx.x + 256 * r, cc = i >> 3, ch = i & 7;
+        *reinterpret_cast<uint4*>(dst + (long long)cc * T + 8 * ch) = *reinterpret_cast<const uint4*>(&tile[cc][8 * ch]);
     }
 }
 
@@ -474,35 +476,42 @@ __global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16*
 // gate (zero padded) times the long-convolution output, which arrives channel-first and leaves channel-last.
 __global__ void __launch_bounds__(256) gate_transpose_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ vT,
                                                              const float* __restrict__ w, __nv_bfloat16* __restrict__ z, int T, int C) {
-    __shared__ __nv_bfloat16 tile[64][66];   // [c][t]
+    __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [t][c]: v transposed on the way in
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const long long b = blockIdx.z;
     const __nv_bfloat16* src = vT + (b * C + c0) * (long long)T + t0;
-    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
-        const int cc = i >> 5, tp = i & 31;
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(src + (long long)cc * T + 2 * tp);
-        tile[cc][2 * tp] = v.x;
-        tile[cc][2 * tp + 1] = v.y;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int i = threadIdx.x + 256 * r, cc = i >> 3, ch = i & 7;   // 8 positions t0 + 8 ch .. of channel cc
+        const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)cc * T + 8 * ch);
+        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) tile[8 * ch + k][cc] = e[k];
     }
     __syncthreads();
     const __nv_bfloat16* xb = x + b * (long long)T * C;
     __nv_bfloat16* zb = z + b * (long long)T * C;
-    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
-        const int tt = i >> 5, cp = i & 31, t = t0 + tt, c = c0 + 2 * cp;
-        const float2 xm = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(xb + (long long)t * C + c));
-        float g0 = w[c * 3 + 1] * xm.x, g1 = w[c * 3 + 4] * xm.y;
-        if (t > 0) {
-            const float2 xl = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(xb + (long long)(t - 1) * C + c));
-            g0 = fmaf(w[c * 3 + 0], xl.x, g0);
-            g1 = fmaf(w[c * 3 + 3], xl.y, g1);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int i = threadIdx.x + 256 * r, tt = i >> 3, ch = i & 7, t = t0 + tt, c = c0 + 8 * ch;
+        const uint4 xm = *reinterpret_cast<const uint4*>(xb + (long long)t * C + c);
+        uint4 xl = make_uint4(0u, 0u, 0u, 0u), xr = make_uint4(0u, 0u, 0u, 0u);   // bf16 zeros outside the sequence
+        if (t > 0) xl = *reinterpret_cast<const uint4*>(xb + (long long)(t - 1) * C + c);
+        if (t + 1 < T) xr = *reinterpret_cast<const uint4*>(xb + (long long)(t + 1) * C + c);
+        const uint4 vv = *reinterpret_cast<const uint4*>(&tile[tt][8 * ch]);
+        const __nv_bfloat16 *em = reinterpret_cast<const __nv_bfloat16*>(&xm), *el = reinterpret_cast<const __nv_bfloat16*>(&xl),
+                            *er = reinterpret_cast<const __nv_bfloat16*>(&xr), *ev = reinterpret_cast<const __nv_bfloat16*>(&vv);
+        uint4 out;
+        __nv_bfloat16* eo = reinterpret_cast<__nv_bfloat16*>(&out);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float* wc = w + (c + k) * 3;
+            float g = wc[1] * __bfloat162float(em[k]);
+            g = fmaf(wc[0], __bfloat162float(el[k]), g);
+            g = fmaf(wc[2], __bfloat162float(er[k]), g);
+            eo[k] = __float2bfloat16_rn(g * __bfloat162float(ev[k]));
         }
-        if (t + 1 < T) {
-            const float2 xr = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(xb + (long long)(t + 1) * C + c));
-            g0 = fmaf(w[c * 3 + 2], xr.x, g0);
-            g1 = fmaf(w[c * 3 + 5], xr.y, g1);
-        }
-        *reinterpret_cast<__nv_bfloat162*>(zb + (long long)t * C + c) =
-            __floats2bfloat162_rn(g0 * __bfloat162float(tile[2 * cp][tt]), g1 * __bfloat162float(tile[2 * cp + 1][tt]));
+        *reinterpret_cast<uint4*>(zb + (long long)t * C + c) = out;
     }
 }
 

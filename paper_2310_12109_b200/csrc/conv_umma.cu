@@ -47,13 +47,14 @@ constexpr int OFF_CONST = 0;         // B1 4096 | B2 2048 | B3 2048 | B4 4096 | 
 constexpr int CONST_BYTES = 20480;
 constexpr int OFF_B1 = OFF_CONST, OFF_B2 = OFF_B1 + 4096, OFF_B3 = OFF_B2 + 2048, OFF_B4 = OFF_B3 + 2048;
 constexpr int OFF_TWA = OFF_B4 + 4096, OFF_TWB = OFF_TWA + 4096;
-constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // per group: bar_x, bar_mma, bar_k, flag (32 B); then tmem ptr
+constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // per group: bar_x, bar_mma, bar_k, flag (32 B each, up to 16 groups); tmem ptr at +512
 constexpr int OFF_GROUP = OFF_BAR + 1024;   // keeps every group slice 1024-byte aligned
 constexpr int G_X = 0;               // 2 boxes [n2hi][r][n1][8]            8192
 constexpr int G_A = 8192;            // A2 / A3 / A4                        16384
 constexpr int G_KF = 24576;          // spectrum row of the unit's channel  4096
 constexpr int GROUP_BYTES = 28672;
 constexpr int SMEM_BYTES = OFF_GROUP + kGroups * GROUP_BYTES;
+static_assert(kGroups * 32 <= 512 && kGroups * kTmemColsPerGroup <= kTmemCols && SMEM_BYTES <= 232448, "per-CTA budgets");
 
 struct Tables {
     void* d_const = nullptr;  // CONST_BYTES
@@ -110,7 +111,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     const uint32_t bar_x = s_all + OFF_BAR + wg * 32, bar_mma = bar_x + 8, bar_k = bar_x + 16;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_all + OFF_BAR + wg * 32 + 24);
     volatile int* next_slot = reinterpret_cast<volatile int*>(smem_all + OFF_BAR + wg * 32 + 28);
-    const uint32_t s_tptr = s_all + OFF_BAR + 224;
+    const uint32_t s_tptr = s_all + OFF_BAR + 512;
 
     const int bgroups0 = (B + kRows - 1) / kRows;
     const int units0 = H * bgroups0;
@@ -150,7 +151,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_cta = *reinterpret_cast<volatile uint32_t*>(smem_all + OFF_BAR + 224);
+    const uint32_t tmem_cta = *reinterpret_cast<volatile uint32_t*>(smem_all + OFF_BAR + 512);
     const uint32_t tmem = tmem_cta + wg * kTmemColsPerGroup;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
     const uint32_t T1 = 0, T2 = 0;   // every stage's accumulator reuses the same 64 columns

@@ -6,17 +6,20 @@
 // index is the CONTIGUOUS index of the data each factor reads (n2 for R, k1 for L after the middle
 // permutation), so neither operand of a tensor-core GEMM can be taken from memory as it lies.  The two
 // factors therefore run as two passes of one kernel that exchange the intermediate through a workspace
-// laid out z[n2 / 8][t][k1][n2 % 8] (it mostly stays in the 126 MB L2):
+// laid out in 16 KB blocks z[token tile][n2 / 8][k1][t % 128][n2 % 8] (it mostly stays in the 126 MB L2): what the
+// pass-1 CTA (token tile, n2 group) writes is one contiguous 128 KB slab, and what the pass-2 CTA (token tile, k1
+// group) reads are eight contiguous 16 KB pieces of eight such slabs:
 //
 //   pass 1 (R): a CTA owns 128 tokens x 8 consecutive n2.  Threads read 16-byte pieces of x (8 values of
 //               n2 for one (t, n1)), transpose 8 x 8 blocks in registers (the permutation P) and write the
 //               K-major, 128-byte-swizzled UMMA operand A_{n2}[t][n1]; 8 UMMA groups (M = 128 tokens,
 //               N = 64 = k1, K = 64 = n1) fill the 512 TMEM columns; the epilogue gathers, for every k1,
 //               the 8 values of n2 from the 8 accumulators as one 16-byte piece (the permutation P^T); the
-//               CTA's pieces form one contiguous 128 KB slab of z and leave as bulk copies.
-//   pass 2 (L): a CTA owns 128 tokens x 8 consecutive k1; the pieces of z are chunks of the K-major operand
-//               rows and are copied in with cp.async; same UMMAs with L's blocks; the epilogue stages 16-byte
-//               pieces of y[t][k2][k1] and one dimension-permuting TMA store scatters them (the last P).
+//               CTA's pieces, staged as [k1][t][16 B], are its slab of z and leave as bulk copies.
+//   pass 2 (L): a CTA owns 128 tokens x 8 consecutive k1; eight bulk copies bring [n2 / 8][k1 % 8][t][16 B] into shared
+//               memory, which IS the K-major operand of every k1 without swizzle (core matrix = 8 tokens x 16 bytes,
+//               next K chunk 16 KB further); same UMMAs with L's blocks; the epilogue stages 16-byte pieces of
+//               y[t][k2][k1] and one dimension-permuting TMA store scatters them (the last P).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -33,9 +36,8 @@ constexpr int kTileT = 128;   // tokens per CTA
 constexpr int kGroup = 8;     // blocks per CTA
 constexpr int OFF_A = 0;                   // 8 operands [128 t][64] bf16, swizzled   131072
 constexpr int OFF_B = 131072;              // 8 weight blocks [64][64] bf16, swizzled   65536
-constexpr int OFF_BAR = 196608;            // bar_mma, tmem ptr
+constexpr int OFF_BAR = 196608;            // bar_mma, tmem ptr, bar_in
 constexpr int SMEM_BYTES = OFF_BAR + 64;
-constexpr int kZPitch = 1040;   // staging pitch of pass 1's 1 KB output rows (the 128 rows spill into the weight buffer, free by then)
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -75,7 +77,7 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     const int tid = threadIdx.x;
     const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
     const uint32_t s_base = smem_u32(smem);
-    const uint32_t bar_mma = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 16;
+    const uint32_t bar_mma = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 16, bar_in = s_base + OFF_BAR + 24;
     // the 8 CTAs that share the 128-byte lines of one token tile are neighbours in launch order, so the
     // 16-byte pieces of a line are fetched / written while the line is still in L2
     const long long t0 = (long long)blockIdx.y * kTileT;
@@ -83,6 +85,7 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
 
     if (tid == 0) {
         mbar_init(bar_mma, 1);
+        mbar_init(bar_in, 1);
         fence_barrier_init();
     }
     if (tid < 32) tmem_alloc(s_tptr, 512);
@@ -120,15 +123,11 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
                 *reinterpret_cast<uint4*>(smem + OFF_A + (2 * j + 1) * 16384 + sw_off(tt, g)) = hi;
             }
         }
-    } else {
-        // z[n2 group kc][t][k1][8]: the 16-byte piece (kc, t, k1) is chunk kc of row t of operand A_{k1}; the 8 pieces
-        // of this CTA's k1 group are 128 contiguous bytes
-        for (int c = tid; c < kGroup * kTileT * 8; c += kThreads) {
-            const int bl = c & 7, tt = (c >> 3) & 127, kc = c >> 10;
-            const bool live = t0 + tt < T;
-            const __nv_bfloat16* src = in + ((((size_t)kc * T + (live ? t0 + tt : 0)) * 64) + grp * kGroup + bl) * 8;
-            cp_async16(s_base + OFF_A + bl * 16384 + sw_off(tt, kc), src, live ? 16u : 0u);
-        }
+    } else if (tid == 0) {
+        // z block (token tile, n2 group kc, k1 group grp) = [k1 % 8][t][8 n2] = 16 KB: chunk kc of every operand row
+        mbar_expect_tx(bar_in, 8 * 16384);
+        const unsigned char* zb = reinterpret_cast<const unsigned char*>(in) + (size_t)blockIdx.y * (8 * 131072) + (size_t)grp * 16384;
+        for (int kc = 0; kc < 8; ++kc) bulk_load(s_base + OFF_A + kc * 16384, zb + (size_t)kc * 131072, 16384, bar_in);
     }
     cp_async_commit_wait();
     fence_proxy_async();
@@ -140,19 +139,26 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     if (tid == 0) {
         constexpr uint32_t IDESC = instr_desc_bf16(128, 64, false, false);
 #pragma unroll 1
-        for (int bl = 0; bl < kGroup; ++bl)
+        bool in_ok = true;
+        if (PASS == 2) in_ok = mbar_wait(bar_in, 0);
+        if (in_ok) {
+            for (int bl = 0; bl < kGroup; ++bl)
 #pragma unroll
-            for (int s = 0; s < 4; ++s)
-                umma_f16(tmem + bl * 64, smem_desc_sw128(s_base + OFF_A + bl * 16384 + s * 32, 16, 1024),
-                         smem_desc_sw128(s_base + OFF_B + bl * 8192 + s * 32, 16, 1024), IDESC, s > 0);
-        umma_commit(bar_mma);
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + bl * 64,
+                             PASS == 1 ? smem_desc_sw128(s_base + OFF_A + bl * 16384 + s * 32, 16, 1024)
+                                       : smem_desc(s_base + OFF_A + bl * 2048 + s * 32768, 16384, 128),
+                             smem_desc_sw128(s_base + OFF_B + bl * 8192 + s * 32, 16, 1024), IDESC, s > 0);
+        }
+        umma_commit(bar_mma);   // (with no UMMA issued it completes at once; the missing input is reported below)
+        if (!in_ok) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
     }
     const bool ok = mbar_wait(bar_mma, 0);
     tc_fence_after();
     // epilogue: lane = token; warpgroup wg takes output columns [16 wg, 16 wg + 16); for every output index o the 8
     // accumulators give the 8 consecutive block indices -> one 16-byte piece.  The pieces are staged in the (now free)
     // operand buffer with consecutive lanes writing to different banks, then leave through the copy engine:
-    //   pass 1: z[grp][t][k1][8] -- this CTA's 128 rows of 1 KB are contiguous; every token's row is one bulk copy;
+    //   pass 1: the staged image [k1][t][16 B] is this CTA's slab of z: eight bulk copies of 16 KB;
     //   pass 2: y[t][k2][k1]     -- staged as [k2][t][16 B]; one TMA store whose tensor map lists the dimensions as
     //                               (k1, t, k2) scatters the pieces (rows past T are clipped by the map).
     if (ok) {
@@ -170,10 +176,7 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
             for (int kk = 0; kk < 8; ++kk) {
                 const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
                                            pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
-                if (PASS == 1)
-                    *reinterpret_cast<uint4*>(smem + OFF_A + t * kZPitch + (o0 + kk) * 16) = p;
-                else
-                    *reinterpret_cast<uint4*>(smem + OFF_A + (o0 + kk) * 2048 + t * 16) = p;
+                *reinterpret_cast<uint4*>(smem + OFF_A + (o0 + kk) * 2048 + t * 16) = p;   // [output index][token][16 B]
             }
         }
     }
@@ -181,8 +184,9 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     tc_fence_before();
     __syncthreads();
     if (PASS == 1) {
-        if (ok && tid < kTileT && t0 + tid < T) {
-            bulk_store(zout + (((size_t)grp * T + t0 + tid) * 64) * 8, s_base + OFF_A + tid * kZPitch, 1024u);
+        if (ok && tid < 8) {   // the staged [k1][t][16 B] image is this CTA's 128 KB slab of z
+            bulk_store(reinterpret_cast<unsigned char*>(zout) + ((size_t)blockIdx.y * 8 + grp) * 131072 + (size_t)tid * 16384,
+                       s_base + OFF_A + tid * 16384, 16384u);
             tma_store_commit();
             tma_store_wait_read0();
         }
@@ -198,7 +202,8 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
 
 bool covered(const m2_plan* pl) { return pl->dtype == M2_BF16 && pl->p == 2 && pl->dims[0] == 64 && pl->dims[1] == 64; }
 
-int64_t workspace_bytes(const m2_plan* pl, int64_t T) { return covered(pl) ? T * 4096 * 2 : 0; }
+// whole token tiles: the last tile's slab is written in full
+int64_t workspace_bytes(const m2_plan* pl, int64_t T) { return covered(pl) ? ((T + kTileT - 1) / kTileT) * kTileT * 4096 * 2 : 0; }
 
 cudaError_t prepare(const m2_plan* pl) {
     if (!covered(pl)) return cudaSuccess;

@@ -15,7 +15,7 @@
 //               K-major, 128-byte-swizzled UMMA operand A_{n2}[t][n1]; 8 UMMA groups (M = 128 tokens,
 //               N = 64 = k1, K = 64 = n1) fill the 512 TMEM columns; the epilogue gathers, for every k1,
 //               the 8 values of n2 from the 8 accumulators as one 16-byte piece (the permutation P^T); the
-//               CTA's pieces, staged as [k1][t][16 B], are its slab of z and leave as bulk copies.
+//               CTA's pieces [k1][t][16 B] are its slab of z and are stored from registers, 512 bytes per warp.
 //   pass 2 (L): a CTA owns 128 tokens x 8 consecutive k1; eight bulk copies bring [n2 / 8][k1 % 8][t][16 B] into shared
 //               memory, which IS the K-major operand of every k1 without swizzle (core matrix = 8 tokens x 16 bytes,
 //               next K chunk 16 KB further); same UMMAs with L's blocks; the epilogue stages 16-byte pieces of
@@ -158,9 +158,11 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     // epilogue: lane = token; warpgroup wg takes output columns [16 wg, 16 wg + 16); for every output index o the 8
     // accumulators give the 8 consecutive block indices -> one 16-byte piece.  The pieces are staged in the (now free)
     // operand buffer with consecutive lanes writing to different banks, then leave through the copy engine:
-    //   pass 1: the staged image [k1][t][16 B] is this CTA's slab of z: eight bulk copies of 16 KB;
+    //   pass 1: the pieces [k1][t][16 B] are this CTA's contiguous slab of z and go straight from registers to global
+    //           memory (a warp's 32 tokens are 512 contiguous bytes);
     //   pass 2: y[t][k2][k1]     -- staged as [k2][t][16 B]; one TMA store whose tensor map lists the dimensions as
     //                               (k1, t, k2) scatters the pieces (rows past T are clipped by the map).
+    unsigned char* zslab = PASS == 1 ? reinterpret_cast<unsigned char*>(zout) + ((size_t)blockIdx.y * 8 + grp) * 131072 : nullptr;
     if (ok) {
         const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
 #pragma unroll 1
@@ -176,21 +178,17 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
             for (int kk = 0; kk < 8; ++kk) {
                 const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
                                            pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
-                *reinterpret_cast<uint4*>(smem + OFF_A + (o0 + kk) * 2048 + t * 16) = p;   // [output index][token][16 B]
+                if (PASS == 1)   // z slab [k1][token][16 B]: a warp's 32 tokens are 512 contiguous bytes, stored as they are
+                    *reinterpret_cast<uint4*>(zslab + (o0 + kk) * 2048 + t * 16) = p;
+                else             // [k2][token][16 B], scattered to y by the TMA store below
+                    *reinterpret_cast<uint4*>(smem + OFF_A + (o0 + kk) * 2048 + t * 16) = p;
             }
         }
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    if (PASS == 1) {
-        if (ok && tid < 8) {   // the staged [k1][t][16 B] image is this CTA's 128 KB slab of z
-            bulk_store(reinterpret_cast<unsigned char*>(zout) + ((size_t)blockIdx.y * 8 + grp) * 131072 + (size_t)tid * 16384,
-                       s_base + OFF_A + tid * 16384, 16384u);
-            tma_store_commit();
-            tma_store_wait_read0();
-        }
-    } else if (tid == 0 && ok) {
+    if (PASS == 2 && tid == 0 && ok) {
         tma_store_3d(&map_out, s_base + OFF_A, 8 * grp, (int)t0, 0);
         tma_store_commit();
         tma_store_wait_read0();   // the staging buffer dies with the CTA

@@ -110,7 +110,11 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
             const bool live = t0 + tt < T;
             const uint4* src = reinterpret_cast<const uint4*>(in + (size_t)(t0 + tt) * 4096 + (size_t)(8 * g) * 64 + grp * 8);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = live ? __ldg(src + i * 8) : make_uint4(0u, 0u, 0u, 0u);
+            for (int i = 0; i < 8; ++i) {   // cached in L2 only: the other half of every 32-byte sector belongs to another SM
+                v[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (live)
+                    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w) : "l"(src + i * 8));
+            }
             const uint32_t* w = reinterpret_cast<const uint32_t*>(v);   // w[i*4 + j]: n1 = 8g+i, n2 = 2j, 2j+1
 #pragma unroll
             for (int j = 0; j < 4; ++j) {

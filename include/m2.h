@@ -20,6 +20,9 @@
  * as void* (NULL = the legacy default stream).  Arguments are validated on the host before
  * anything is launched; on an error nothing has been enqueued.  The hot calls never synchronise
  * the stream and never allocate.  All device buffers must be 16-byte aligned and contiguous.
+ * Work is ordered by the stream as usual: a call sees everything enqueued on `stream` before it.  (The
+ * tensor-core kernels are launched so that their thread blocks may take over SMs while the previous
+ * kernel's last blocks still run; they wait for that kernel before touching any data.)
  */
 #ifndef M2_H_
 #define M2_H_

@@ -32,6 +32,7 @@
 #include <vector>
 
 #include "ptx_sm100.cuh"
+#include "tma_host.h"
 
 namespace m2u {
 
@@ -430,22 +431,6 @@ static void put_kmajor(std::vector<uint16_t>& img, int K, int n, int k, double v
     img[byte / 2] = bf16_bits(v);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
 static bool covered(const m2_plan* pl) {
     return pl->dtype == M2_BF16 && pl->p == 2 && pl->dims[0] == 32 && pl->dims[1] == 16;
 }
@@ -530,15 +515,10 @@ void destroy_tables(m2_plan* pl) {
 
 // x / y viewed as [b][h][n1][n2] with n2 innermost; box = 8 of the 16 n2, all 32 n1, one h, 8 b.
 static bool make_map(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return false;
-    cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
-    cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
-    cuuint32_t box[4] = {8, 32, 1, (cuuint32_t)kRows};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), gdim, gstr, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
+    const cuuint32_t box[4] = {8, 32, 1, (cuuint32_t)kRows};
+    return tma_host::encode_bf16(map, ptr, 4, gdim, gstr, box);
 }
 
 int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,

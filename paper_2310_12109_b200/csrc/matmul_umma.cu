@@ -142,10 +142,10 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
 
     if (tid == 0) {
         constexpr uint32_t IDESC = instr_desc_bf16(128, 64, false, false);
-#pragma unroll 1
         bool in_ok = true;
         if (PASS == 2) in_ok = mbar_wait(bar_in, 0);
         if (in_ok) {
+#pragma unroll 1
             for (int bl = 0; bl < kGroup; ++bl)
 #pragma unroll
                 for (int s = 0; s < 4; ++s)

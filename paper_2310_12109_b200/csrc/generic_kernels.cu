@@ -4,6 +4,8 @@
 // contraction of one index digit (the stride permutations of M = P L P^T R P only decide which
 // digit a stage contracts, so they are address arithmetic here, never a data movement pass).
 #include <cuda_bf16.h>
+
+#include <cstdint>
 #include <cuda_runtime.h>
 
 #include "generic_kernels.h"
@@ -447,28 +449,48 @@ cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y,
 }
 
 // ---- channel-last <-> channel-first helpers of the M2 block (Sec. 5.1; Eq. 2 runs along the sequence) -----------------
-// x[B][T][C] -> xT[B][C][T] through a 64 x 64 shared-memory tile; both sides move 16 bytes per thread and whole
-// 128-byte rows per 8 threads.  The tile is stored transposed ([c][t], pitch 72 elements) so that the output side
-// reads 16 contiguous bytes.
+// 64 x 64 bf16 tile transposes through shared memory.  The tile is kept as 32-bit words (two neighbouring columns of one
+// row) with a row pitch of 33 words: the 16-byte global loads land as four conflict-free word stores, and the transposed
+// side gathers, for one column and 8 consecutive rows, 8 words (2-way conflicts at worst) of which it keeps one half.
+constexpr int kTrPitch = 33;
+
+// tile[row][col pair] <- 8 columns (one 16-byte load) of one row
+__device__ __forceinline__ void tr_put(uint32_t* tile, int row, int ch, const uint4& v) {
+    uint32_t* p = tile + row * kTrPitch + 4 * ch;
+    p[0] = v.x;
+    p[1] = v.y;
+    p[2] = v.z;
+    p[3] = v.w;
+}
+// 8 consecutive rows 8 rb .. 8 rb + 7 of column col -> one 16-byte vector
+__device__ __forceinline__ uint4 tr_get(const uint32_t* tile, int rb, int col) {
+    const uint32_t* p = tile + (8 * rb) * kTrPitch + (col >> 1);
+    const uint32_t sel = (col & 1) ? 0x7632u : 0x5410u;   // high or low halves of two words
+    uint4 o;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(o.x) : "r"(p[0 * kTrPitch]), "r"(p[1 * kTrPitch]), "r"(sel));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(o.y) : "r"(p[2 * kTrPitch]), "r"(p[3 * kTrPitch]), "r"(sel));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(o.z) : "r"(p[4 * kTrPitch]), "r"(p[5 * kTrPitch]), "r"(sel));
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(o.w) : "r"(p[6 * kTrPitch]), "r"(p[7 * kTrPitch]), "r"(sel));
+    return o;
+}
+
+// x[B][T][C] -> xT[B][C][T]; both sides move 16 bytes per thread and whole 128-byte rows per 8 threads.
 __global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xT, int T, int C) {
-    __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [c][t]
+    __shared__ uint32_t tile[64 * kTrPitch];   // [t][c pair]
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const long long b = blockIdx.z;
     const __nv_bfloat16* src = x + (b * T + t0) * (long long)C + c0;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int i = threadIdx.x + 256 * r, tt = i >> 3, ch = i & 7;   // 8 channels c0 + 8 ch .. of row tt
-        const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)tt * C + 8 * ch);
-        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) tile[8 * ch + k][tt] = e[k];
+        tr_put(tile, tt, ch, *reinterpret_cast<const uint4*>(src + (long long)tt * C + 8 * ch));
     }
     __syncthreads();
     __nv_bfloat16* dst = xT + (b * C + c0) * (long long)T + t0;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
-        const int i = threadIdx.x + 256 * r, cc = i >> 3, ch = i & 7;
-        *reinterpret_cast<uint4*>(dst + (long long)cc * T + 8 * ch) = *reinterpret_cast<const uint4*>(&tile[cc][8 * ch]);
+        const int i = threadIdx.x + 256 * r, cc = i >> 3, tb = i & 7;   // 8 positions t0 + 8 tb .. of channel cc
+        *reinterpret_cast<uint4*>(dst + (long long)cc * T + 8 * tb) = tr_get(tile, tb, cc);
     }
 }
 
@@ -476,29 +498,26 @@ __global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16*
 // gate (zero padded) times the long-convolution output, which arrives channel-first and leaves channel-last.
 __global__ void __launch_bounds__(256) gate_transpose_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ vT,
                                                              const float* __restrict__ w, __nv_bfloat16* __restrict__ z, int T, int C) {
-    __shared__ __align__(16) __nv_bfloat16 tile[64][72];   // [t][c]: v transposed on the way in
+    __shared__ uint32_t tile[64 * kTrPitch];   // [c][t pair]: v as it arrives
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const long long b = blockIdx.z;
     const __nv_bfloat16* src = vT + (b * C + c0) * (long long)T + t0;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const int i = threadIdx.x + 256 * r, cc = i >> 3, ch = i & 7;   // 8 positions t0 + 8 ch .. of channel cc
-        const uint4 v = *reinterpret_cast<const uint4*>(src + (long long)cc * T + 8 * ch);
-        const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) tile[8 * ch + k][cc] = e[k];
+        tr_put(tile, cc, ch, *reinterpret_cast<const uint4*>(src + (long long)cc * T + 8 * ch));
     }
     __syncthreads();
     const __nv_bfloat16* xb = x + b * (long long)T * C;
     __nv_bfloat16* zb = z + b * (long long)T * C;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
-        const int i = threadIdx.x + 256 * r, tt = i >> 3, ch = i & 7, t = t0 + tt, c = c0 + 8 * ch;
+        const int i = threadIdx.x + 256 * r, tt = i >> 3, cb = i & 7, t = t0 + tt, c = c0 + 8 * cb;
         const uint4 xm = *reinterpret_cast<const uint4*>(xb + (long long)t * C + c);
         uint4 xl = make_uint4(0u, 0u, 0u, 0u), xr = make_uint4(0u, 0u, 0u, 0u);   // bf16 zeros outside the sequence
         if (t > 0) xl = *reinterpret_cast<const uint4*>(xb + (long long)(t - 1) * C + c);
         if (t + 1 < T) xr = *reinterpret_cast<const uint4*>(xb + (long long)(t + 1) * C + c);
-        const uint4 vv = *reinterpret_cast<const uint4*>(&tile[tt][8 * ch]);
+        const uint4 vv = tr_get(tile, cb, tt);   // channels c .. c + 7 at position t
         const __nv_bfloat16 *em = reinterpret_cast<const __nv_bfloat16*>(&xm), *el = reinterpret_cast<const __nv_bfloat16*>(&xl),
                             *er = reinterpret_cast<const __nv_bfloat16*>(&xr), *ev = reinterpret_cast<const __nv_bfloat16*>(&vv);
         uint4 out;

@@ -259,10 +259,14 @@ cudaError_t prepare() { return cudaFuncSetAttribute(mlp_umma_kernel, cudaFuncAtt
 int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, long long tokens, int32_t* status,
                cudaStream_t stream) {
     if (tokens == 0) return M2_OK;
-    static bool prepared = false;
-    if (!prepared) {
-        if (prepare() != cudaSuccess) return M2_ERR_CUDA;
-        prepared = true;
+    {   // the shared-memory opt-in is per device
+        static bool prepared[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return M2_ERR_CUDA;
+        if (!prepared[dev]) {
+            if (prepare() != cudaSuccess) return M2_ERR_CUDA;
+            prepared[dev] = true;
+        }
     }
     alignas(64) CUtensorMap mz, mw1, mw2, my;
     {   // activations [tokens][C]: box = 64 columns x 128 tokens, 128B swizzle (rows past the end: zero-filled / clipped)

@@ -63,7 +63,9 @@ enum m2_table {
  * accumulation is always fp32.  sign = +1 (paper) or -1.  device >= 0: CUDA device ordinal, tables
  * are uploaded (the call synchronises).  device < 0: host-only plan, usable only with
  * m2_plan_get_table.  (Eq. 1: the factorisation N = N1..Np with block size N^(1/p); Corollary
- * "DFT is M": the twiddles.) */
+ * "DFT is M": the twiddles.)  A plan carries a little device state of its own (a status word, work
+ * counters of its kernels): calls on one plan must be ordered on the GPU -- one stream, or events
+ * between streams; use one plan per stream for calls that may overlap. */
 int32_t m2_plan_create(m2_plan** out, int64_t N, int32_t p, const int32_t* factors, int32_t dtype,
                        int32_t sign, int32_t device);
 int32_t m2_plan_destroy(m2_plan* plan);

@@ -17,11 +17,12 @@
 //   S2'  D3[(r,k1)][(c,n2)]   = sum_(c,k2) A3 * conj(F16)
 //   h3   conj twiddle, write A4[(r,n2)][(c,k1)]                                      M-major
 //   S1'  D4[(r,n2)][n1]       = Re sum_(c,k1) A4 * conj(F32)
-//   h4   round to bf16 into the output tile, TMA store.
+//   h4   round to bf16 and store y[r][n1*16 + n2] from registers (a warp instruction writes two full 32-byte sectors).
 //
 // One CTA per SM keeps the constant operands once and runs kGroups independent unit pipelines of 128
 // threads (own mbarriers, 64 TMEM columns, 28 KB of shared memory each), so one pipeline's UMMA / TMA /
-// barrier latency is covered by the others' fp32 work.  All waits are bounded.
+// barrier latency is covered by the others' fp32 work.  Units are handed out by a device-wide counter; the kernel is
+// launched with programmatic stream serialization (set-up overlaps the previous kernel's tail).  All waits are bounded.
 #include "conv_umma.h"
 
 #include <cuda.h>

@@ -23,7 +23,10 @@
 //   S3      n3          k2 = 8(2(j&1)+t/64) + t%8, k1 = 8(j/2) + (t/8)%8 spectrum k_f              -> A4 (K-major)
 //   S3'     k3          same lanes, columns n3                           conj w_N^{n3 (k1+32 k2)}  -> A5
 //   S2'     k2          n3 = 8(2(j&1)+t/64) + t%8, k1 = 8(j/2) + (t/8)%8 conj w_1024^{n2 k1}       -> A6
-//   S1'     k1 (N=32)   n2 = 8(j/2) + t%8, n3 = 8(2(j&1)+t/64) + (t/8)%8 round, stage, bulk store
+//   S1'     k1 (N=32)   n2 = 8(j/2) + t%8, n3 = 8(2(j&1)+t/64) + (t/8)%8 round, stage (64B-swizzled box image), TMA store
+//
+// The fp32 arithmetic of the hand-offs is packed (fma.rn.f32x2: two complex products in five instructions); the
+// twiddles w_N^{n3 (k1 + 32 k2)} are geometric sequences in k2 (resp. n3) and run as packed chains stepping by rho^2.
 #include <cuda.h>
 #include <cuda_bf16.h>
 

@@ -89,3 +89,14 @@ def test_argument_validation_without_device():
     assert lib.m2_plan_destroy(h) == M.M2_OK
     assert lib.m2_plan_destroy(None) == M.M2_ERR_INVALID_ARG
     assert lib.m2_status_string(M.M2_ERR_TIMEOUT) == b"device-side wait timed out"
+
+
+def test_matmul_workspace_covers_whole_token_tiles():
+    """The tensor-core matmul keeps its intermediate in 128-token tiles: the workspace is sized for whole tiles
+    (bf16 plan with 64 x 64 blocks); plans it does not cover need none."""
+    pl = M.Plan((64, 64), dtype=M.M2_BF16, sign=+1, device=-1)
+    lib = M.lib()
+    for T, tiles in [(0, 0), (1, 1), (128, 1), (129, 2), (16384, 128)]:
+        assert int(lib.m2_matmul_workspace_bytes(pl.handle, T)) == tiles * 128 * 4096 * 2
+    assert int(lib.m2_matmul_workspace_bytes(host_plan((8, 8)).handle, 100)) == 0
+    assert int(lib.m2_matmul_workspace_bytes(host_plan((64, 64)).handle, 100)) == 0   # fp32 plan: CUDA-core kernels

@@ -88,6 +88,15 @@ int32_t m2_kernel_spectrum(const m2_plan* plan, const float* k_dev, int64_t H, i
 int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t H, float* out_dev,
                                void* stream);
 
+/* kf_out = conj(kf_in), in every layout the buffer holds (kf_out may be kf_in).  With the conjugated
+ * spectrum m2_monarch_conv_fwd computes the transpose of the convolution: for an upstream gradient g of y,
+ * dx = M^-1 ( conj(k_f) (.) M pad(g) ) [0:n) is the gradient with respect to x (k is real, so conj(F k)
+ * is the spectrum of the index-reversed kernel: the transposed circulant, resp. the transposed Toeplitz
+ * matrix T_k of App. D.3 once zero padded).  The paper trains through this operator (Sec. 5) without
+ * writing the backward pass out. */
+int32_t m2_spectrum_conjugate(const m2_plan* plan, const void* kf_in_dev, int64_t H, void* kf_out_dev,
+                              void* stream);
+
 /* y = Re( M^-1 ( k_f (.) M pad(x) ) )[0:n)  (Eq. 2 with M_1 = F, M_2 = F^-1; App. D.3).
  * x_dev, y_dev: [B, H, n] in the plan dtype; kf_dev from m2_kernel_spectrum with the same H.
  * mode M2_CAUSAL: n <= N/2, x zero padded to N, first n outputs kept (Thm 3 / App. D.3 review).

@@ -120,6 +120,27 @@ def direct_causal_conv(k: np.ndarray, x: np.ndarray) -> np.ndarray:
     return y
 
 
+def direct_circular_conv_adjoint(k: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """Transpose of the circulant map x -> direct_circular_conv(k, x) applied to g:
+    dx[s] = sum_{t=0}^{N-1} g[t] k[(t-s) mod N] (the gradient of <y, g> with respect to x)."""
+    N = g.shape[-1]
+    out = np.zeros(np.broadcast_shapes(k.shape, g.shape), dtype=np.result_type(k, g))
+    for s_ in range(N):
+        idx = (np.arange(N) - s_) % N
+        out[..., s_] = np.sum(g * k[..., idx], axis=-1)
+    return out
+
+
+def direct_causal_conv_adjoint(k: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """Transpose of the lower-triangular Toeplitz map of direct_causal_conv (App. D.3, T_k):
+    dx[s] = sum_{t=s}^{n-1} g[t] k[t-s], 0 <= s < n."""
+    n = g.shape[-1]
+    out = np.zeros(np.broadcast_shapes(k.shape, g.shape), dtype=np.result_type(k, g))
+    for s_ in range(n):
+        out[..., s_] = np.sum(g[..., s_:] * k[..., : n - s_], axis=-1)
+    return out
+
+
 def depthwise_conv3_same(x: np.ndarray, w: np.ndarray) -> np.ndarray:
     """Short depthwise convolution of width 3 along the sequence, centred, zero
     padded: g[b,t,c] = w[c,0] x[b,t-1,c] + w[c,1] x[b,t,c] + w[c,2] x[b,t+1,c].
@@ -306,6 +327,27 @@ def monarch_conv(k: np.ndarray, x: np.ndarray, dims: tuple, causal: bool, sign: 
     f = monarch_apply_order_p(cblocks, dims, prod) / N
     if stages is not None:
         stages.update(k_f=k_f, u_f=u_f, prod=prod, f=f)
+    return np.real(f[..., :n])
+
+
+def monarch_conv_adjoint(k: np.ndarray, g: np.ndarray, dims: tuple, causal: bool, sign: int = +1) -> np.ndarray:
+    """Gradient of <monarch_conv(k, x), g> with respect to x: the same Monarch convolution with the
+    conjugated kernel spectrum, M^-1 (conj(M k') (.) M g') (k real: conj(F k) = F of the index-reversed
+    kernel, which is the transposed circulant; zero padding makes the causal case exact for n <= N/2)."""
+    N = int(np.prod(dims))
+    n = g.shape[-1]
+    assert k.shape[-1] == n
+    if causal:
+        assert 2 * n <= N
+        kp = np.concatenate([k, np.zeros((*k.shape[:-1], N - n))], axis=-1)
+        gp = np.concatenate([g, np.zeros((*g.shape[:-1], N - n))], axis=-1)
+    else:
+        assert n == N
+        kp, gp = k, g
+    blocks = monarch_dft_factors_order_p(dims, sign)
+    k_f = monarch_apply_order_p(blocks, dims, kp.astype(np.complex128))
+    g_f = monarch_apply_order_p(blocks, dims, gp.astype(np.complex128))
+    f = monarch_apply_order_p([np.conj(B) for B in blocks], dims, np.conj(k_f) * g_f) / N
     return np.real(f[..., :n])
 
 

@@ -32,6 +32,7 @@ SIGNATURES = {
     "m2_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_matmul_workspace_bytes": (_i64, [_vp, _i64]),
+    "m2_spectrum_conjugate": (_i32, [_vp, _vp, _i64, _vp, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
@@ -139,6 +140,15 @@ def m2_kernel_spectrum(plan: Plan, k: torch.Tensor, kf: torch.Tensor | None = No
         kf = torch.empty(max(m2_spectrum_bytes(plan, H), 16), dtype=torch.uint8, device=k.device)
     _check(lib().m2_kernel_spectrum(plan.handle, _ptr(k), H, n, _ptr(kf), _stream()), "m2_kernel_spectrum")
     return kf
+
+
+def m2_spectrum_conjugate(plan: Plan, kf: torch.Tensor, H: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    """conj(k_f) in every layout of the buffer: the spectrum with which m2_monarch_conv_fwd computes the gradient
+    with respect to its input."""
+    if out is None:
+        out = torch.empty_like(kf)
+    _check(lib().m2_spectrum_conjugate(plan.handle, _ptr(kf), H, _ptr(out), _stream()), "m2_spectrum_conjugate")
+    return out
 
 
 def m2_spectrum_to_natural(plan: Plan, kf: torch.Tensor, H: int) -> torch.Tensor:

@@ -549,4 +549,21 @@ cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w,
     return cudaGetLastError();
 }
 
+// conj of a spectrum buffer: `pairs` interleaved complex values (re, im), then `quads` values of the tensor-core
+// kernels' layouts (re, re', im, im')
+__global__ void spectrum_conj_kernel(const float4* __restrict__ in, float4* __restrict__ out, long long pair_quads, long long total) {
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const float4 v = in[i];
+    out[i] = i < pair_quads ? make_float4(v.x, -v.y, v.z, -v.w) : make_float4(v.x, v.y, -v.z, -v.w);
+}
+
+cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st) {
+    // plan_order_values complex values (even); private_values complex values stored as (re, re', im, im') quads
+    const long long pair_quads = plan_order_values / 2, total = pair_quads + private_values / 2;
+    if (total == 0) return cudaSuccess;
+    spectrum_conj_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const float4*)in, (float4*)out, pair_quads, total);
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

@@ -27,4 +27,7 @@ cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y,
 cudaError_t launch_transpose_btc(const void* x, void* xT, long long B, int T, int C, cudaStream_t st);
 cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w, void* z, long long B, int T, int C, cudaStream_t st);
 
+// conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
+cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
+
 }  // namespace m2g

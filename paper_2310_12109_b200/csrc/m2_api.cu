@@ -237,6 +237,21 @@ int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t 
     return M2_OK;
 }
 
+int32_t m2_spectrum_conjugate(const m2_plan* plan, const void* kf_in_dev, int64_t H, void* kf_out_dev, void* stream) {
+    if (!plan || !kf_in_dev || !kf_out_dev || H < 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (!aligned16(kf_in_dev) || !aligned16(kf_out_dev)) return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    const long long values = H * plan->N;   // complex values per layout; N is even for every plan with a device path
+    if (plan->N % 2 != 0) return M2_ERR_UNSUPPORTED;
+    if (m2g::launch_spectrum_conj(kf_in_dev, kf_out_dev, values, m2u::has_private_spectrum(plan) ? values : 0, (cudaStream_t)stream) !=
+        cudaSuccess)
+        return M2_ERR_CUDA;
+    plan->launches += (H > 0);
+    return M2_OK;
+}
+
 int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
                             int64_t H, int64_t n, int32_t mode, void* stream) {
     int32_t st = check_conv_args(plan, x_dev, kf_dev, y_dev, B, H, n, mode);

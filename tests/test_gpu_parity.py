@@ -267,6 +267,40 @@ def test_config5_full_size_sampled():
     check(y[sel].reshape(-1, 768), yr.reshape(-1, 768), TOL_BF16, "config5 full y")
 
 
+# ---- gradient with respect to the input: the same kernels with the conjugated spectrum ---------------------
+
+@pytest.mark.parametrize("cfg,kernel", [("c1", None), ("c2", "conv_umma_o2_512"), ("c2causal", "conv_umma_o2_512"), ("c4", "conv_umma_o3_32k")])
+def test_conv_input_gradient(cfg, kernel):
+    if cfg == "c1":
+        c, causal, dtype, tol = synth.config1(), True, M.M2_FP32, TOL_FP32
+    elif cfg == "c2":
+        c, causal, dtype, tol = synth.config2(B=8, H=12), False, M.M2_BF16, TOL_BF16
+    elif cfg == "c2causal":
+        c = synth.config2(B=8, H=12)
+        c = dict(c, x=c["x"][..., :256].copy(), k=c["k"][..., :256].copy())
+        causal, dtype, tol = True, M.M2_BF16, TOL_BF16
+    else:
+        c, causal, dtype, tol = synth.config4(B=2, H=2), True, M.M2_BF16, TOL_BF16
+    plan = M.Plan(c["dims"], dtype=dtype, device=0)
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    g = dev(c["x"].astype(np.float32), tdt)               # any tensor of the right shape serves as upstream gradient
+    H = c["k"].shape[0]
+    kf = M.m2_kernel_spectrum(plan, dev(c["k"].astype(np.float32)))
+    kfc = M.m2_spectrum_conjugate(plan, kf, H)
+    dx = M.m2_monarch_conv_fwd(plan, g, kfc, M.M2_CAUSAL if causal else M.M2_CIRCULAR)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    if kernel is not None:
+        assert plan.last_kernel() == kernel
+    ref = O.monarch_conv_adjoint(c["k"].astype(np.float64), c["x"].astype(np.float64), c["dims"], causal)
+    check(host(dx), ref, tol, "input gradient " + cfg)
+    # conjugating twice gives the spectrum back, bit for bit, in place
+    M.m2_spectrum_conjugate(plan, kfc, H, out=kfc)
+    torch.cuda.synchronize()
+    assert torch.equal(kfc, kf)
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

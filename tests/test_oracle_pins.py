@@ -314,6 +314,27 @@ def test_order3_causal_conv_full_size_sampled():
 
 # ---- M2 block pieces ---------------------------------------------------------------------
 
+def test_conv_adjoints_are_transposes_and_match_the_conjugated_spectrum():
+    """The adjoint oracles: (i) equal the transposed dense circulant / Toeplitz matrix applied to g, (ii) satisfy
+    <conv(k, x), g> = <x, adjoint(k, g)>, (iii) the factored version (conjugated kernel spectrum) equals the direct one."""
+    n = 12
+    k, x, g = rng.standard_normal(n), rng.standard_normal((3, n)), rng.standard_normal((3, n))
+    Cm = np.array([[k[(t - u) % n] for u in range(n)] for t in range(n)])          # y = Cm x (circular)
+    Tm = np.array([[k[t - u] if t >= u else 0.0 for u in range(n)] for t in range(n)])  # y = Tm x (causal)
+    assert np.allclose(O.direct_circular_conv(k, x), x @ Cm.T)
+    assert np.allclose(O.direct_circular_conv_adjoint(k, g), g @ Cm)
+    assert np.allclose(O.direct_causal_conv(k, x), x @ Tm.T)
+    assert np.allclose(O.direct_causal_conv_adjoint(k, g), g @ Tm)
+    assert np.isclose(np.sum(O.direct_causal_conv(k, x) * g), np.sum(x * O.direct_causal_conv_adjoint(k, g)))
+    for dims, nn, causal in [((4, 3), 12, False), ((4, 3, 2), 12, True), ((32, 16), 256, True), ((8, 8), 64, False)]:
+        kk, gg, xx = rng.standard_normal((2, nn)), rng.standard_normal((3, 2, nn)), rng.standard_normal((3, 2, nn))
+        direct = O.direct_causal_conv_adjoint(kk, gg) if causal else O.direct_circular_conv_adjoint(kk, gg)
+        assert np.allclose(O.monarch_conv_adjoint(kk, gg, dims, causal), direct, atol=1e-10)
+        assert np.allclose(O.monarch_conv_adjoint(kk, gg, dims, causal, sign=-1), direct, atol=1e-10)
+        lhs = np.sum(O.monarch_conv(kk, xx, dims, causal) * gg)
+        assert np.isclose(lhs, np.sum(xx * O.monarch_conv_adjoint(kk, gg, dims, causal)), rtol=1e-10)
+
+
 def test_gelu_values():
     v = np.array([0.0, 1.0, -1.0, 3.0])
     ref = np.array([0.0, 0.8413447460685429, -0.15865525393145707, 2.9959502191322303])

@@ -351,6 +351,40 @@ def monarch_conv_adjoint(k: np.ndarray, g: np.ndarray, dims: tuple, causal: bool
     return np.real(f[..., :n])
 
 
+def direct_conv_kernel_grad(x: np.ndarray, g: np.ndarray, causal: bool) -> np.ndarray:
+    """Gradient of sum_b <conv(k, x[b]), g[b]> with respect to k (the convolution is linear in k):
+    dk[h, u] = sum_b sum_t g[b, h, t] x[b, h, t - u], indices taken mod N for the circular convolution and
+    restricted to t >= u for the causal one.  x, g: [B, H, n]; result [H, n]."""
+    B, H, n = x.shape
+    dk = np.zeros((H, n), dtype=np.result_type(x, g))
+    for u in range(n):
+        if causal:
+            dk[:, u] = np.sum(g[:, :, u:] * x[:, :, : n - u], axis=(0, 2))
+        else:
+            dk[:, u] = np.sum(g * np.roll(x, u, axis=-1), axis=(0, 2))
+    return dk
+
+
+def monarch_conv_kernel_grad(x: np.ndarray, g: np.ndarray, dims: tuple, causal: bool, sign: int = +1) -> np.ndarray:
+    """The same gradient through the Monarch-DFT: dk = M^-1 ( sum_b conj(M x'_b) (.) M g'_b ) [0:n)
+    (x real; zero padded to N = prod(dims) in the causal case)."""
+    N = int(np.prod(dims))
+    n = x.shape[-1]
+    if causal:
+        assert 2 * n <= N
+        pad = np.zeros((*x.shape[:-1], N - n))
+        xp, gp = np.concatenate([x, pad], axis=-1), np.concatenate([g, pad], axis=-1)
+    else:
+        assert n == N
+        xp, gp = x, g
+    blocks = monarch_dft_factors_order_p(dims, sign)
+    x_f = monarch_apply_order_p(blocks, dims, xp.astype(np.complex128))
+    g_f = monarch_apply_order_p(blocks, dims, gp.astype(np.complex128))
+    acc = np.sum(np.conj(x_f) * g_f, axis=0)
+    f = monarch_apply_order_p([np.conj(Bk) for Bk in blocks], dims, acc) / N
+    return np.real(f[..., :n])
+
+
 def m2_block_forward(x, k, w_short, W_up, W_down, dims=(32, 16)):
     """M2 block forward as configured for the M2-BERT-base shape (Sec. 5.1, Eq. 2-3):
     gate g = depthwise-conv3(x); long mix v = circular Monarch conv of x with k

@@ -33,6 +33,7 @@ SIGNATURES = {
     "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_matmul_workspace_bytes": (_i64, [_vp, _i64]),
     "m2_spectrum_conjugate": (_i32, [_vp, _vp, _i64, _vp, _vp]),
+    "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
@@ -149,6 +150,17 @@ def m2_spectrum_conjugate(plan: Plan, kf: torch.Tensor, H: int, out: torch.Tenso
         out = torch.empty_like(kf)
     _check(lib().m2_spectrum_conjugate(plan.handle, _ptr(kf), H, _ptr(out), _stream()), "m2_spectrum_conjugate")
     return out
+
+
+def m2_monarch_conv_bwd_kernel(plan: Plan, x: torch.Tensor, g: torch.Tensor, mode: int) -> torch.Tensor:
+    """dk[H, n] (float32): gradient of sum_b <conv(k, x_b), g_b> with respect to the kernel; x, g: [B, H, n]."""
+    assert x.is_cuda and g.is_cuda and x.dtype == plan.torch_dtype and g.dtype == plan.torch_dtype
+    assert x.is_contiguous() and g.is_contiguous() and x.shape == g.shape and x.dim() == 3
+    B, H, n = x.shape
+    dk = torch.empty((H, n), dtype=torch.float32, device=x.device)
+    _check(lib().m2_monarch_conv_bwd_kernel(plan.handle, _ptr(x), _ptr(g), _ptr(dk), B, H, n, mode, _stream()),
+           "m2_monarch_conv_bwd_kernel")
+    return dk
 
 
 def m2_spectrum_to_natural(plan: Plan, kf: torch.Tensor, H: int) -> torch.Tensor:

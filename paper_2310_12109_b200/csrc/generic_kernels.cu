@@ -176,6 +176,38 @@ __global__ void __launch_bounds__(1024) conv_row_kernel(const IO* __restrict__ x
     }
 }
 
+// Gradient with respect to the kernel: dk[h] = M^-1 ( sum_b conj(M x'_b) (.) M g'_b ) [0:n) / N, one block per channel,
+// the batch walked sequentially; x, g rows and the accumulated product stay in shared memory (3 complex fp32 rows).
+template <typename IO, int ITEMS>
+__global__ void __launch_bounds__(1024) conv_wgrad_kernel(const IO* __restrict__ x, const IO* __restrict__ g, float* __restrict__ dk, Dims D,
+                                                          Roots R, int B, int H, int n) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2* bx = reinterpret_cast<float2*>(smem_raw);
+    float2* bg = bx + D.N;
+    float2* acc = bg + D.N;
+    const int h = blockIdx.x;
+    for (int i = threadIdx.x; i < D.N; i += blockDim.x) acc[i] = make_float2(0.f, 0.f);
+    for (int b = 0; b < B; ++b) {
+        const IO* xr = x + ((long long)b * H + h) * n;
+        const IO* gr = g + ((long long)b * H + h) * n;
+        for (int i = threadIdx.x; i < D.N; i += blockDim.x) {
+            bx[i] = make_float2(i < n ? to_f32<IO>(xr[i]) : 0.f, 0.f);
+            bg[i] = make_float2(i < n ? to_f32<IO>(gr[i]) : 0.f, 0.f);
+        }
+        __syncthreads();
+        for (int a = 0; a < D.p; ++a) stage<float2, ITEMS, false>(bx, D, a, R.r[a]);
+        for (int a = 0; a < D.p; ++a) stage<float2, ITEMS, false>(bg, D, a, R.r[a]);
+        for (int i = threadIdx.x; i < D.N; i += blockDim.x) {   // every thread owns the same positions in every round
+            const float2 xv = bx[i], gv = bg[i], av = acc[i];
+            acc[i] = make_float2(av.x + xv.x * gv.x + xv.y * gv.y, av.y + xv.x * gv.y - xv.y * gv.x);   // += conj(x_f) g_f
+        }
+        __syncthreads();
+    }
+    for (int a = D.p - 1; a >= 0; --a) stage<float2, ITEMS, true>(acc, D, a, R.r[a]);
+    const float inv = 1.0f / (float)D.N;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) dk[(long long)h * n + i] = acc[i].x * inv;
+}
+
 // k_f = F_N pad(k) / N per channel, in plan order, computed in place in the output buffer (global
 // memory, one block per channel): runs once per weight update, not on the hot path.
 template <int ITEMS>
@@ -563,6 +595,40 @@ cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order
     const long long pair_quads = plan_order_values / 2, total = pair_quads + private_values / 2;
     if (total == 0) return cudaSuccess;
     spectrum_conj_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>((const float4*)in, (float4*)out, pair_quads, total);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, cudaStream_t st) {
+    Dims D = make_dims(s);
+    Roots R{{s.roots[0], s.roots[1], s.roots[2]}};
+    int items, threads;
+    if (!pick_launch(D, items, threads)) return cudaErrorInvalidValue;
+    const size_t smem = (size_t)D.N * sizeof(float2) * 3;
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    if (s.H == 0) return cudaSuccess;
+#define M2_LAUNCH_WGRAD(IO, IT)                                                                                   \
+    {                                                                                                             \
+        auto kern = conv_wgrad_kernel<IO, IT>;                                                                    \
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);       \
+        if (e != cudaSuccess) return e;                                                                           \
+        kern<<<(unsigned)s.H, threads, smem, st>>>((const IO*)x, (const IO*)g, dk, D, R, (int)s.B, (int)s.H, (int)s.n); \
+    }
+    if (bf16_io) {
+        switch (items) {
+            case 1: M2_LAUNCH_WGRAD(__nv_bfloat16, 1) break;
+            case 2: M2_LAUNCH_WGRAD(__nv_bfloat16, 2) break;
+            case 4: M2_LAUNCH_WGRAD(__nv_bfloat16, 4) break;
+            default: return cudaErrorInvalidValue;
+        }
+    } else {
+        switch (items) {
+            case 1: M2_LAUNCH_WGRAD(float, 1) break;
+            case 2: M2_LAUNCH_WGRAD(float, 2) break;
+            case 4: M2_LAUNCH_WGRAD(float, 4) break;
+            default: return cudaErrorInvalidValue;
+        }
+    }
+#undef M2_LAUNCH_WGRAD
     return cudaGetLastError();
 }
 

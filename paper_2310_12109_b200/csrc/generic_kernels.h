@@ -27,6 +27,8 @@ cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y,
 cudaError_t launch_transpose_btc(const void* x, void* xT, long long B, int T, int C, cudaStream_t st);
 cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w, void* z, long long B, int T, int C, cudaStream_t st);
 
+// dk[H, n] (fp32) = gradient of sum_b <conv(k, x_b), g_b> with respect to k; x, g: [B, H, n] contiguous
+cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -237,6 +237,24 @@ int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t 
     return M2_OK;
 }
 
+int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const void* g_dev, float* dk_dev, int64_t B, int64_t H,
+                                   int64_t n, int32_t mode, void* stream) {
+    // same argument rules as the forward call (dk plays the part of the output for the null / alignment checks)
+    int32_t st = check_conv_args(plan, x_dev, g_dev, dk_dev, B, H, n, mode);
+    if (st != M2_OK) return st;
+    if (H > 0 && !dk_dev) return M2_ERR_INVALID_ARG;   // an empty batch still writes zeros
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (H == 0) return M2_OK;
+    m2g::ConvShape s = conv_shape(plan, B, H, n);
+    const cudaError_t e = m2g::launch_conv_wgrad(s, plan->dtype == M2_BF16, x_dev, g_dev, dk_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "conv_wgrad_generic";
+    plan->launches += 1;
+    return M2_OK;
+}
+
 int32_t m2_spectrum_conjugate(const m2_plan* plan, const void* kf_in_dev, int64_t H, void* kf_out_dev, void* stream) {
     if (!plan || !kf_in_dev || !kf_out_dev || H < 0) return M2_ERR_INVALID_ARG;
     if (plan->device < 0) return M2_ERR_NO_DEVICE;

@@ -301,6 +301,32 @@ def test_conv_input_gradient(cfg, kernel):
     plan.close()
 
 
+@pytest.mark.parametrize("cfg", ["c1", "c2", "c2causal", "small3"])
+def test_conv_kernel_gradient(cfg):
+    if cfg == "c1":
+        c, causal, dtype, tol = synth.config1(), True, M.M2_FP32, 1e-5
+    elif cfg == "c2":
+        c, causal, dtype, tol = synth.config2(B=8, H=12), False, M.M2_BF16, 1e-5   # bf16 inputs are exact in fp32: fp32 accuracy
+    elif cfg == "c2causal":
+        c = synth.config2(B=5, H=7)
+        c = dict(c, x=c["x"][..., :200].copy(), k=c["k"][..., :200].copy())
+        causal, dtype, tol = True, M.M2_BF16, 1e-5
+    else:
+        c = dict(x=synth.round_bf16(synth.normal(synth.stream_id(9, 0), (3, 4, 32))), dims=(4, 4, 4))
+        causal, dtype, tol = True, M.M2_BF16, 1e-5
+    plan = M.Plan(c["dims"], dtype=dtype, device=0)
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    x = c["x"].astype(np.float64)
+    gup = synth.round_bf16(synth.normal(synth.stream_id(9, 1), x.shape)).astype(np.float64)   # upstream gradient
+    dk = M.m2_monarch_conv_bwd_kernel(plan, dev(x.astype(np.float32), tdt), dev(gup.astype(np.float32), tdt),
+                                      M.M2_CAUSAL if causal else M.M2_CIRCULAR)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "conv_wgrad_generic"
+    ref = O.monarch_conv_kernel_grad(x, gup, c["dims"], causal)
+    check(host(dk), ref, tol, "kernel gradient " + cfg)
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

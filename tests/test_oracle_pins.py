@@ -335,6 +335,30 @@ def test_conv_adjoints_are_transposes_and_match_the_conjugated_spectrum():
         assert np.isclose(lhs, np.sum(xx * O.monarch_conv_adjoint(kk, gg, dims, causal)), rtol=1e-10)
 
 
+def test_kernel_gradient_oracles():
+    """dk: (i) the convolution is linear in k, so <conv(k, x), g> summed over the batch equals <k, dk> for every k;
+    (ii) the factored version equals the direct one; (iii) a brute-force triple loop on a tiny case."""
+    B, H, n = 2, 3, 6
+    x, g = rng.standard_normal((B, H, n)), rng.standard_normal((B, H, n))
+    for causal in (True, False):
+        dk = O.direct_conv_kernel_grad(x, g, causal)
+        brute = np.zeros((H, n))
+        for b in range(B):
+            for h in range(H):
+                for u in range(n):
+                    for t in range(n):
+                        if causal and t < u:
+                            continue
+                        brute[h, u] += g[b, h, t] * x[b, h, (t - u) % n]
+        assert np.allclose(dk, brute)
+    for dims, nn, causal in [((4, 3), 12, False), ((4, 3, 2), 12, True), ((32, 16), 256, True), ((8, 8), 64, False)]:
+        xx, gg, kk = rng.standard_normal((3, 2, nn)), rng.standard_normal((3, 2, nn)), rng.standard_normal((2, nn))
+        dk = O.direct_conv_kernel_grad(xx, gg, causal)
+        assert np.allclose(O.monarch_conv_kernel_grad(xx, gg, dims, causal), dk, atol=1e-9)
+        assert np.allclose(O.monarch_conv_kernel_grad(xx, gg, dims, causal, sign=-1), dk, atol=1e-9)
+        assert np.isclose(np.sum(O.monarch_conv(kk, xx, dims, causal) * gg), np.sum(kk * dk), rtol=1e-10)
+
+
 def test_gelu_values():
     v = np.array([0.0, 1.0, -1.0, 3.0])
     ref = np.array([0.0, 0.8413447460685429, -0.15865525393145707, 2.9959502191322303])

@@ -135,6 +135,16 @@ int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const vo
                                void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* ws_dev,
                                int64_t ws_bytes, void* stream);
 
+/* W_out[b][c][r] = W_in[b][r][c]: block-wise transpose of a block-diagonal factor of nblocks blocks of rows x cols
+ * elements of the plan dtype (W_out must not overlap W_in).  It gives the gradient of the Monarch matmul with
+ * respect to its input: M^T = P^T R^T P L^T P^T (Sec. 3.1 transposed) is again an order-2 Monarch product, so for an
+ * upstream gradient G of Y
+ *   dX = m2_monarch_matmul(plan', G, L' = blocks_transpose(R), R' = blocks_transpose(L), ...)
+ * where plan' has the factors in the opposite order (N2, N1) -- the same plan when N1 == N2 -- and L', R' have
+ * the shapes of R, L.  (The paper trains through the operator, Sec. 5, without writing the backward pass out.) */
+int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows,
+                            int64_t cols, void* stream);
+
 /* M2 block forward for the M2-BERT-base shape (Eq. 2-3; Sec. 5.1): along the sequence, per channel,
  * v = circular Monarch conv of x with the channel's kernel; gate g = depthwise conv of width 3
  * (centred, zero padded); z = g (.) v; then the block-diagonal MLP y = bd(W_down) GELU(bd(W_up) z)

@@ -191,6 +191,21 @@ def monarch_apply(L: np.ndarray, R: np.ndarray, x: np.ndarray, stages: dict | No
     return y
 
 
+def monarch_apply_transpose(L: np.ndarray, R: np.ndarray, g: np.ndarray) -> np.ndarray:
+    """M^T g along the last axis for M = P L P^T R P (Sec. 3.1): the gradient of <M x, g> with respect to x.
+    M^T = P^T R^T P L^T P^T with block-wise transposes; written with the inverse permutations explicitly."""
+    N1, N2 = L.shape[0], R.shape[0]
+    N = N1 * N2
+    lead = g.shape[:-1]
+    v = g.reshape(*lead, N2, N1)                      # g[k2, k1]; P^T: back to blocks indexed by k1
+    v = np.swapaxes(v, -1, -2)                        # [k1][k2]
+    v = np.einsum("bkn,...bk->...bn", L, v)           # L^T per block k1: [k1][n2]
+    v = np.swapaxes(v, -1, -2)                        # P: [n2][k1]
+    v = np.einsum("bkn,...bk->...bn", R, v)           # R^T per block n2: [n2][n1]
+    v = np.swapaxes(v, -1, -2)                        # P^T: [n1][n2]
+    return v.reshape(*lead, N)
+
+
 def monarch_apply_order_p(blocks: list, dims: tuple, x: np.ndarray) -> np.ndarray:
     """Order-p Monarch apply in the direct form (App. D.6, "p-variate Monarch"):
     stage a (a = 1..p) contracts input digit n_a into output digit k_a with the

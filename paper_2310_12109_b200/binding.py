@@ -33,6 +33,7 @@ SIGNATURES = {
     "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_matmul_workspace_bytes": (_i64, [_vp, _i64]),
     "m2_spectrum_conjugate": (_i32, [_vp, _vp, _i64, _vp, _vp]),
+    "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
@@ -212,6 +213,21 @@ def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Ten
     _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _ptr(ws),
                                    0 if ws is None else ws.numel(), _stream()), "m2_monarch_matmul")
     return Y
+
+
+def m2_blocks_transpose(plan: Plan, W: torch.Tensor) -> torch.Tensor:
+    """W: [nblocks, rows, cols] CUDA tensor of the plan dtype; returns [nblocks, cols, rows]."""
+    assert W.is_cuda and W.dtype == plan.torch_dtype and W.is_contiguous() and W.dim() == 3
+    nb, r, c = W.shape
+    out = torch.empty((nb, c, r), dtype=W.dtype, device=W.device)
+    _check(lib().m2_blocks_transpose(plan.handle, _ptr(W), _ptr(out), nb, r, c, _stream()), "m2_blocks_transpose")
+    return out
+
+
+def m2_monarch_matmul_bwd_input(plan_t: Plan, G: torch.Tensor, L: torch.Tensor, R: torch.Tensor, ws: torch.Tensor | None = None):
+    """dX = M^T G for M = P L P^T R P: the forward call with the block-wise transposed factors in swapped roles.
+    plan_t: a plan with the factors (N2, N1) (the forward plan itself when N1 == N2)."""
+    return m2_monarch_matmul(plan_t, G, m2_blocks_transpose(plan_t, R), m2_blocks_transpose(plan_t, L), ws=ws)
 
 
 def m2_monarch_matmul_host(plan: Plan, X_host, L, R, Y_host, X_scratch, Y_scratch, ws: torch.Tensor | None = None):

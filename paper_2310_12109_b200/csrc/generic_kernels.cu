@@ -632,4 +632,26 @@ cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, c
     return cudaGetLastError();
 }
 
+// out[b][c][r] = in[b][r][c]: block-wise transpose of a block-diagonal factor
+template <typename T>
+__global__ void blocks_transpose_kernel(const T* __restrict__ in, T* __restrict__ out, int rows, int cols, long long total) {
+    const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // index into out
+    if (i >= total) return;
+    const int r = (int)(i % rows);
+    const int c = (int)((i / rows) % cols);
+    const long long b = i / ((long long)rows * cols);
+    out[i] = in[(b * rows + r) * cols + c];
+}
+
+cudaError_t launch_blocks_transpose(const void* in, void* out, long long nblocks, int rows, int cols, bool bf16, cudaStream_t st) {
+    const long long total = nblocks * rows * cols;
+    if (total == 0) return cudaSuccess;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (bf16)
+        blocks_transpose_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)in, (__nv_bfloat16*)out, rows, cols, total);
+    else
+        blocks_transpose_kernel<float><<<grid, 256, 0, st>>>((const float*)in, (float*)out, rows, cols, total);
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

@@ -29,6 +29,8 @@ cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w,
 
 // dk[H, n] (fp32) = gradient of sum_b <conv(k, x_b), g_b> with respect to k; x, g: [B, H, n] contiguous
 cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, cudaStream_t st);
+// out[b][c][r] = in[b][r][c] for nblocks blocks of rows x cols elements (fp32 or bf16)
+cudaError_t launch_blocks_transpose(const void* in, void* out, long long nblocks, int rows, int cols, bool bf16, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -344,6 +344,21 @@ int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_
     return M2_OK;
 }
 
+int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows, int64_t cols,
+                            void* stream) {
+    if (!plan || nblocks < 0 || rows <= 0 || cols <= 0 || rows > 65536 || cols > 65536) return M2_ERR_INVALID_ARG;
+    if ((!W_in_dev || !W_out_dev) && nblocks > 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (!aligned16(W_in_dev) || !aligned16(W_out_dev)) return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (m2g::launch_blocks_transpose(W_in_dev, W_out_dev, nblocks, (int)rows, (int)cols, plan->dtype == M2_BF16, (cudaStream_t)stream) !=
+        cudaSuccess)
+        return M2_ERR_CUDA;
+    plan->launches += (nblocks > 0);
+    return M2_OK;
+}
+
 int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const void* L_dev, const void* R_dev,
                                void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* ws_dev,
                                int64_t ws_bytes, void* stream) {

@@ -327,6 +327,26 @@ def test_conv_kernel_gradient(cfg):
     plan.close()
 
 
+@pytest.mark.parametrize("T,dims,dtype", [(300, (64, 64), M.M2_BF16), (40, (8, 8), M.M2_BF16), (17, (6, 4), M.M2_FP32)])
+def test_matmul_input_gradient(T, dims, dtype):
+    N1, N2 = dims
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    L = rnd(synth.normal(synth.stream_id(8, 0), (N1, N2, N2)) / np.sqrt(N2))
+    R = rnd(synth.normal(synth.stream_id(8, 1), (N2, N1, N1)) / np.sqrt(N1))
+    G = rnd(synth.normal(synth.stream_id(8, 2), (T, N1 * N2)))
+    plan_t = M.Plan((N2, N1), dtype=dtype, device=0)       # factors in the opposite order
+    dX = M.m2_monarch_matmul_bwd_input(plan_t, dev(G.astype(np.float32), tdt), dev(L.astype(np.float32), tdt),
+                                       dev(R.astype(np.float32), tdt))
+    torch.cuda.synchronize()
+    assert plan_t.device_status() == 0
+    if dims == (64, 64):
+        assert plan_t.last_kernel() == "matmul_umma_64x64"
+    ref = O.monarch_apply_transpose(L.astype(np.float64), R.astype(np.float64), G.astype(np.float64))
+    check(host(dX), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, "matmul input gradient")
+    plan_t.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -335,6 +335,19 @@ def test_conv_adjoints_are_transposes_and_match_the_conjugated_spectrum():
         assert np.isclose(lhs, np.sum(xx * O.monarch_conv_adjoint(kk, gg, dims, causal)), rtol=1e-10)
 
 
+@pytest.mark.parametrize("N1,N2", [(4, 4), (3, 5), (8, 2), (16, 16)])
+def test_monarch_transpose_apply(N1, N2):
+    """M^T g: against the dense matrix, by <M x, g> = <x, M^T g>, and as the forward apply with the block-wise
+    transposed factors in swapped roles (the identity the library's backward-input call rests on)."""
+    L, R = rng.standard_normal((N1, N2, N2)), rng.standard_normal((N2, N1, N1))
+    Md = O.monarch_dense(L, R)
+    x, g = rng.standard_normal((3, N1 * N2)), rng.standard_normal((3, N1 * N2))
+    assert np.allclose(O.monarch_apply_transpose(L, R, g), g @ Md)
+    assert np.isclose(np.sum(O.monarch_apply(L, R, x) * g), np.sum(x * O.monarch_apply_transpose(L, R, g)))
+    Lt, Rt = np.swapaxes(R, 1, 2).copy(), np.swapaxes(L, 1, 2).copy()
+    assert np.allclose(O.monarch_apply(Lt, Rt, g), g @ Md)
+
+
 def test_kernel_gradient_oracles():
     """dk: (i) the convolution is linear in k, so <conv(k, x), g> summed over the batch equals <k, dk> for every k;
     (ii) the factored version equals the direct one; (iii) a brute-force triple loop on a tiny case."""

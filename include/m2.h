@@ -145,6 +145,19 @@ int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const vo
 int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows,
                             int64_t cols, void* stream);
 
+/* Gradients of sum_t <Y_t, G_t>, Y = M X with M = P L P^T R P (Sec. 3.1), with respect to the blocks of L and R:
+ *   dL[k1][k2][n2] = sum_t G[t][k2 N1 + k1] v[t][n2][k1],           v  = R-stage of the forward pass,
+ *   dR[n2][k1][n1] = sum_t dv[t][n2][k1] X[t][n1 N2 + n2],          dv = L^T-stage applied to G.
+ * X_dev, G_dev: [T, N], L_dev, R_dev as in m2_monarch_matmul (plan dtype); dL_dev [N1][N2][N2] and dR_dev [N2][N1][N1]
+ * are fp32 and overwritten (zeros for T == 0).  ws_dev: caller-owned, at least m2_matmul_bwd_workspace_bytes(plan, T)
+ * = 4 T N bytes (holds v, then dv), 16-byte aligned; too small or NULL with T > 0: M2_ERR_INVALID_ARG.  fp32
+ * CUDA-core kernels with a fixed summation order (deterministic).  (The paper trains through the operator, Sec. 5,
+ * without writing the backward pass out.) */
+int64_t m2_matmul_bwd_workspace_bytes(const m2_plan* plan, int64_t T);
+int32_t m2_monarch_matmul_bwd_weights(const m2_plan* plan, const void* X_dev, const void* G_dev, const void* L_dev,
+                                      const void* R_dev, float* dL_dev, float* dR_dev, int64_t T, void* ws_dev,
+                                      int64_t ws_bytes, void* stream);
+
 /* M2 block forward for the M2-BERT-base shape (Eq. 2-3; Sec. 5.1): along the sequence, per channel,
  * v = circular Monarch conv of x with the channel's kernel; gate g = depthwise conv of width 3
  * (centred, zero padded); z = g (.) v; then the block-diagonal MLP y = bd(W_down) GELU(bd(W_up) z)

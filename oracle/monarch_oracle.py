@@ -206,6 +206,25 @@ def monarch_apply_transpose(L: np.ndarray, R: np.ndarray, g: np.ndarray) -> np.n
     return v.reshape(*lead, N)
 
 
+def monarch_weight_grads(L: np.ndarray, R: np.ndarray, x: np.ndarray, g: np.ndarray):
+    """Gradients of sum_t <M x_t, g_t> with respect to the blocks of L and R for M = P L P^T R P (Sec. 3.1), by the
+    chain rule through the stages of monarch_apply: with v0 = P x ([n2][n1]), v1 = R v0 ([n2][k1]) and the upstream
+    gradient read in plan order gv[k1][k2] = g[k2 N1 + k1],
+        dL[k1][k2][n2] = sum_t gv[t][k1][k2] v1[t][n2][k1]
+        dv1[t][n2][k1] = sum_k2 L[k1][k2][n2] gv[t][k1][k2]
+        dR[n2][k1][n1] = sum_t dv1[t][n2][k1] v0[t][n2][n1].
+    x, g: [T, N].  Returns (dL, dR) with the shapes of L and R."""
+    N2, N1, _ = R.shape
+    T = x.shape[0]
+    v0 = np.swapaxes(x.reshape(T, N1, N2), 1, 2)          # [t][n2][n1]
+    v1 = np.einsum("nki,tni->tnk", R, v0)                 # [t][n2][k1]
+    gv = np.swapaxes(g.reshape(T, N2, N1), 1, 2)          # [t][k1][k2]
+    dL = np.einsum("tkq,tnk->kqn", gv, v1)                # [k1][k2][n2]
+    dv1 = np.einsum("kqn,tkq->tnk", L, gv)                # [t][n2][k1]
+    dR = np.einsum("tnk,tni->nki", dv1, v0)               # [n2][k1][n1]
+    return dL, dR
+
+
 def monarch_apply_order_p(blocks: list, dims: tuple, x: np.ndarray) -> np.ndarray:
     """Order-p Monarch apply in the direct form (App. D.6, "p-variate Monarch"):
     stage a (a = 1..p) contracts input digit n_a into output digit k_a with the

@@ -33,6 +33,8 @@ SIGNATURES = {
     "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_matmul_workspace_bytes": (_i64, [_vp, _i64]),
     "m2_spectrum_conjugate": (_i32, [_vp, _vp, _i64, _vp, _vp]),
+    "m2_matmul_bwd_workspace_bytes": (_i64, [_vp, _i64]),
+    "m2_monarch_matmul_bwd_weights": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
@@ -228,6 +230,24 @@ def m2_monarch_matmul_bwd_input(plan_t: Plan, G: torch.Tensor, L: torch.Tensor, 
     """dX = M^T G for M = P L P^T R P: the forward call with the block-wise transposed factors in swapped roles.
     plan_t: a plan with the factors (N2, N1) (the forward plan itself when N1 == N2)."""
     return m2_monarch_matmul(plan_t, G, m2_blocks_transpose(plan_t, R), m2_blocks_transpose(plan_t, L), ws=ws)
+
+
+def m2_monarch_matmul_bwd_weights(plan: Plan, X: torch.Tensor, G: torch.Tensor, L: torch.Tensor, R: torch.Tensor,
+                                  ws: torch.Tensor | None = None):
+    """(dL, dR) in fp32 for the upstream gradient G of Y = M X; X, G: [T, N] of the plan dtype."""
+    for a in (X, G, L, R):
+        assert a.is_cuda and a.dtype == plan.torch_dtype and a.is_contiguous()
+    T = X.shape[0]
+    assert X.shape == G.shape
+    dL = torch.empty(L.shape, dtype=torch.float32, device=X.device)
+    dR = torch.empty(R.shape, dtype=torch.float32, device=X.device)
+    need = int(lib().m2_matmul_bwd_workspace_bytes(plan.handle, T))
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=X.device)
+    _check(lib().m2_monarch_matmul_bwd_weights(plan.handle, _ptr(X), _ptr(G), _ptr(L), _ptr(R), _ptr(dL), _ptr(dR), T,
+                                               _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "m2_monarch_matmul_bwd_weights")
+    return dL, dR
 
 
 def m2_monarch_matmul_host(plan: Plan, X_host, L, R, Y_host, X_scratch, Y_scratch, ws: torch.Tensor | None = None):

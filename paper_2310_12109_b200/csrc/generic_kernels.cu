@@ -654,4 +654,114 @@ cudaError_t launch_blocks_transpose(const void* in, void* out, long long nblocks
     return cudaGetLastError();
 }
 
+// First stage of the matmul or of its transpose, fp32 result in index order n2*N1 + k1 (Sec. 3.1):
+//   BWD == false: v[n2][k1] = sum_{n1} R[n2][k1][n1] x[n1*N2 + n2]      (W = R, in = X)
+//   BWD == true : v[n2][k1] = sum_{k2} L[k1][k2][n2] g[k2*N1 + k1]      (W = L, in = G)
+template <typename IO, int TT, bool BWD>
+__global__ void matmul_stage1_kernel(const IO* __restrict__ in, const IO* __restrict__ W, float* __restrict__ out, int N1, int N2,
+                                     long long T) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int N = N1 * N2;
+    float* xs = reinterpret_cast<float*>(smem_raw);  // [TT][N]
+    const long long t0 = (long long)blockIdx.x * TT;
+    for (int i = threadIdx.x; i < TT * N; i += blockDim.x) {
+        const long long t = t0 + i / N;
+        xs[i] = (t < T) ? to_f32<IO>(in[t * N + (i % N)]) : 0.f;
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < N; o += blockDim.x) {
+        const int k1 = o % N1, n2 = o / N1;
+        float acc[TT];
+#pragma unroll
+        for (int t = 0; t < TT; ++t) acc[t] = 0.f;
+        if (!BWD) {
+            const IO* w = W + ((long long)n2 * N1 + k1) * N1;
+            for (int n1 = 0; n1 < N1; ++n1) {
+                const float wv = to_f32<IO>(w[n1]);
+#pragma unroll
+                for (int t = 0; t < TT; ++t) acc[t] = fmaf(wv, xs[t * N + n1 * N2 + n2], acc[t]);
+            }
+        } else {
+            const IO* w = W + (long long)k1 * N2 * N2 + n2;
+            for (int k2 = 0; k2 < N2; ++k2) {
+                const float wv = to_f32<IO>(w[(long long)k2 * N2]);
+#pragma unroll
+                for (int t = 0; t < TT; ++t) acc[t] = fmaf(wv, xs[t * N + k2 * N1 + k1], acc[t]);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t)
+            if (t0 + t < T) out[(t0 + t) * N + o] = acc[t];
+    }
+}
+
+// C[b][i][j] = sum_t A[t*N + b*sAb + i*sAi] * B[t*N + b*sBb + j*sBj], i < I, j < J: one 32 x 32 tile of one block per
+// CTA, the whole token range walked in chunks of 32 by the same CTA (fixed summation order: deterministic).
+template <typename TA, typename TB>
+__global__ void __launch_bounds__(256) outer_accum_kernel(const TA* __restrict__ A, const TB* __restrict__ B, float* __restrict__ C, int N,
+                                                          long long T, int I, int J, int sAb, int sAi, int sBb, int sBj) {
+    __shared__ float as[32][33], bs[32][33];
+    const int b = blockIdx.x, i0 = blockIdx.y * 32, j0 = blockIdx.z * 32;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;   // outputs (i0 + ty + 16 a, j0 + tx + 16 c)
+    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    for (long long t0 = 0; t0 < T; t0 += 32) {
+        for (int e = threadIdx.x; e < 1024; e += 256) {
+            const int tt = e / 32, c = e % 32;
+            const long long t = t0 + tt;
+            as[tt][c] = (t < T && i0 + c < I) ? to_f32<TA>(A[t * N + (long long)b * sAb + (long long)(i0 + c) * sAi]) : 0.f;
+            bs[tt][c] = (t < T && j0 + c < J) ? to_f32<TB>(B[t * N + (long long)b * sBb + (long long)(j0 + c) * sBj]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int tt = 0; tt < 32; ++tt) {
+            const float a0 = as[tt][ty], a1 = as[tt][ty + 16], b0 = bs[tt][tx], b1 = bs[tt][tx + 16];
+            acc[0][0] = fmaf(a0, b0, acc[0][0]);
+            acc[0][1] = fmaf(a0, b1, acc[0][1]);
+            acc[1][0] = fmaf(a1, b0, acc[1][0]);
+            acc[1][1] = fmaf(a1, b1, acc[1][1]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            const int i = i0 + ty + 16 * a, j = j0 + tx + 16 * c;
+            if (i < I && j < J) C[((long long)b * I + i) * J + j] = acc[a][c];
+        }
+}
+
+template <typename IO>
+static cudaError_t launch_matmul_wgrad_t(int N1, int N2, long long T, const IO* X, const IO* G, const IO* L, const IO* R, float* dL,
+                                         float* dR, float* ws, cudaStream_t st) {
+    constexpr int TT = 4;
+    const int N = N1 * N2;
+    const size_t smem = (size_t)TT * N * sizeof(float);
+    if (smem > 200 * 1024 || N1 > 65535 * 32 || N2 > 65535 * 32) return cudaErrorInvalidValue;
+    auto fwd = matmul_stage1_kernel<IO, TT, false>;
+    auto bwd = matmul_stage1_kernel<IO, TT, true>;
+    cudaError_t e = cudaFuncSetAttribute(fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int threads = N < 512 ? ((N + 31) / 32) * 32 : 512;
+    const unsigned tiles = (unsigned)((T + TT - 1) / TT);
+    const unsigned t1 = (unsigned)((N1 + 31) / 32), t2 = (unsigned)((N2 + 31) / 32);
+    if (T > 0) fwd<<<tiles, threads, smem, st>>>(X, R, ws, N1, N2, T);                    // ws = v1[t][n2][k1]
+    // dL[k1][k2][n2] = sum_t g[t][k2*N1 + k1] v1[t][n2*N1 + k1]
+    outer_accum_kernel<IO, float><<<dim3(N1, t2, t2), 256, 0, st>>>(G, ws, dL, N, T, N2, N2, 1, N1, 1, N1);
+    if (T > 0) bwd<<<tiles, threads, smem, st>>>(G, L, ws, N1, N2, T);                    // ws = dv1[t][n2][k1]
+    // dR[n2][k1][n1] = sum_t dv1[t][n2*N1 + k1] x[t][n1*N2 + n2]
+    outer_accum_kernel<float, IO><<<dim3(N2, t1, t1), 256, 0, st>>>(ws, X, dR, N, T, N1, N1, N1, 1, 1, N2);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_matmul_wgrad(int N1, int N2, long long T, bool bf16_io, const void* X, const void* G, const void* L, const void* R,
+                                float* dL, float* dR, float* ws, cudaStream_t st) {
+    return bf16_io ? launch_matmul_wgrad_t<__nv_bfloat16>(N1, N2, T, (const __nv_bfloat16*)X, (const __nv_bfloat16*)G,
+                                                          (const __nv_bfloat16*)L, (const __nv_bfloat16*)R, dL, dR, ws, st)
+                   : launch_matmul_wgrad_t<float>(N1, N2, T, (const float*)X, (const float*)G, (const float*)L, (const float*)R, dL, dR,
+                                                  ws, st);
+}
+
 }  // namespace m2g

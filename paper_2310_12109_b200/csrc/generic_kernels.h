@@ -31,6 +31,9 @@ cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w,
 cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, cudaStream_t st);
 // out[b][c][r] = in[b][r][c] for nblocks blocks of rows x cols elements (fp32 or bf16)
 cudaError_t launch_blocks_transpose(const void* in, void* out, long long nblocks, int rows, int cols, bool bf16, cudaStream_t st);
+// dL[N1][N2][N2], dR[N2][N1][N1] (fp32) of sum_t <M x_t, g_t>; ws: T*N floats (4 launches)
+cudaError_t launch_matmul_wgrad(int N1, int N2, long long T, bool bf16_io, const void* X, const void* G, const void* L, const void* R,
+                                float* dL, float* dR, float* ws, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -359,6 +359,29 @@ int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_o
     return M2_OK;
 }
 
+int64_t m2_matmul_bwd_workspace_bytes(const m2_plan* plan, int64_t T) {
+    if (!plan || plan->p != 2 || T < 0) return -1;
+    return T * plan->N * 4;
+}
+
+int32_t m2_monarch_matmul_bwd_weights(const m2_plan* plan, const void* X_dev, const void* G_dev, const void* L_dev, const void* R_dev,
+                                      float* dL_dev, float* dR_dev, int64_t T, void* ws_dev, int64_t ws_bytes, void* stream) {
+    int32_t st = check_matmul_args(plan, X_dev, L_dev, R_dev, dL_dev, T);
+    if (st != M2_OK) return st;
+    if (!dL_dev || !dR_dev || (T > 0 && !G_dev)) return M2_ERR_INVALID_ARG;   // the gradients are written (zeros) even for T == 0
+    if (!aligned16(G_dev) || !aligned16(dR_dev) || !aligned16(ws_dev)) return M2_ERR_ALIGNMENT;
+    if (T > 0 && (!ws_dev || ws_bytes < m2_matmul_bwd_workspace_bytes(plan, T))) return M2_ERR_INVALID_ARG;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    cudaError_t e = m2g::launch_matmul_wgrad(plan->dims[0], plan->dims[1], T, plan->dtype == M2_BF16, X_dev, G_dev, L_dev, R_dev, dL_dev,
+                                             dR_dev, (float*)ws_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "matmul_wgrad_generic";
+    plan->launches += T > 0 ? 4 : 2;
+    return M2_OK;
+}
+
 int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const void* L_dev, const void* R_dev,
                                void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* ws_dev,
                                int64_t ws_bytes, void* stream) {

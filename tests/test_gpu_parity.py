@@ -347,6 +347,27 @@ def test_matmul_input_gradient(T, dims, dtype):
     plan_t.close()
 
 
+@pytest.mark.parametrize("T,dims,dtype", [(300, (64, 64), M.M2_BF16), (77, (8, 16), M.M2_BF16), (33, (6, 4), M.M2_FP32), (0, (4, 4), M.M2_FP32)])
+def test_matmul_weight_gradients(T, dims, dtype):
+    N1, N2 = dims
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    L = rnd(synth.normal(synth.stream_id(9, 0), (N1, N2, N2)) / np.sqrt(N2))
+    R = rnd(synth.normal(synth.stream_id(9, 1), (N2, N1, N1)) / np.sqrt(N1))
+    X = rnd(synth.normal(synth.stream_id(9, 2), (T, N1 * N2)))
+    G = rnd(synth.normal(synth.stream_id(9, 3), (T, N1 * N2)))
+    plan = M.Plan(dims, dtype=dtype, device=0)
+    dL, dR = M.m2_monarch_matmul_bwd_weights(plan, dev(X.astype(np.float32), tdt), dev(G.astype(np.float32), tdt),
+                                             dev(L.astype(np.float32), tdt), dev(R.astype(np.float32), tdt))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "matmul_wgrad_generic"
+    rL, rR = O.monarch_weight_grads(L, R, X, G)
+    # inputs are exactly representable and every product is accumulated in fp32: the fp32 tolerance holds for both dtypes
+    check(host(dL), rL, TOL_FP32, "dL")
+    check(host(dR), rR, TOL_FP32, "dR")
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -348,6 +348,22 @@ def test_monarch_transpose_apply(N1, N2):
     assert np.allclose(O.monarch_apply(Lt, Rt, g), g @ Md)
 
 
+@pytest.mark.parametrize("N1,N2", [(2, 3), (4, 4), (5, 2)])
+def test_monarch_weight_grads(N1, N2):
+    """y is linear in L and in R, so perturbing one weight by 1 changes sum <y, g> by exactly that weight's
+    gradient: brute force over every entry, with the dense matrix doing the forward."""
+    L, R = rng.standard_normal((N1, N2, N2)), rng.standard_normal((N2, N1, N1))
+    x, g = rng.standard_normal((5, N1 * N2)), rng.standard_normal((5, N1 * N2))
+    dL, dR = O.monarch_weight_grads(L, R, x, g)
+    base = np.sum((x @ O.monarch_dense(L, R).T) * g)
+    for idx in np.ndindex(*L.shape):
+        Lp = L.copy(); Lp[idx] += 1.0
+        assert np.isclose(np.sum((x @ O.monarch_dense(Lp, R).T) * g) - base, dL[idx], atol=1e-9), ("dL", idx)
+    for idx in np.ndindex(*R.shape):
+        Rp = R.copy(); Rp[idx] += 1.0
+        assert np.isclose(np.sum((x @ O.monarch_dense(L, Rp).T) * g) - base, dR[idx], atol=1e-9), ("dR", idx)
+
+
 def test_kernel_gradient_oracles():
     """dk: (i) the convolution is linear in k, so <conv(k, x), g> summed over the batch equals <k, dk> for every k;
     (ii) the factored version equals the direct one; (iii) a brute-force triple loop on a tiny case."""

@@ -178,7 +178,7 @@ def time_launches(fn, n, torch):
     return e0.elapsed_time(e1)
 
 
-def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5"), reps=None):
+def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5", "operator"), reps=None):
     """Config 3 (Monarch matmul), config 4 (order-3 causal conv) and config 5 (M2 block forward): time per call,
     throughput and roofline fraction, outside the headline timed region."""
     out = {}
@@ -190,6 +190,33 @@ def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "confi
         out.update(_side_config4(torch, M, synth, peaks, reps, bf))
     if "config5" in which:
         out.update(_side_config5(torch, M, synth, peaks, reps, bf))
+    if "operator" in which:
+        out.update(_side_operator(torch, M, synth, peaks, reps, bf))
+    return out
+
+
+def _side_operator(torch, M, synth, peaks, reps, bf):
+    """The paper's operator benchmark (Table 2, first column): M_b (K (.) M_a X) with learnable order-2 Monarch matrices,
+    N = 4096, block size 64, 768 columns; FLOP utilisation = 2 products x 4 N sqrt(N) flops per column / time / bf16 peak."""
+    import numpy as np
+    N, b, T = 4096, 64, 768
+    plan = M.Plan((b, b), dtype=M.M2_BF16, device=torch.cuda.current_device())
+    W = [bf(synth.round_bf16(synth.normal(synth.stream_id(6, i), (b, b, b)) / np.sqrt(float(b)))) for i in range(4)]
+    K = bf(synth.round_bf16(synth.normal(synth.stream_id(6, 4), (T, N))))
+    Xs = [bf(synth.round_bf16(synth.normal(synth.stream_id(6, 5 + i), (T, N)))) for i in range(2)]
+    Ys = [torch.empty_like(Xs[0]) for _ in range(2)]
+    ws = M.m2_matmul_workspace(plan, T)
+    f = lambda i: M.m2_monarch_mix(plan, Xs[i % 2], K, W[0], W[1], W[2], W[3], act=M.M2_ACT_NONE, Y=Ys[i % 2], ws=ws)  # noqa: E731
+    time_launches(f, 3, torch)
+    reps = max(reps, 20)
+    ms = time_launches(f, reps, torch) / reps
+    fl = 2 * 4.0 * T * N * b
+    out = {"operator_4k": {
+        "kernel": plan.last_kernel(), "ms": ms, "TFLOPs": fl / (ms * 1e9), "launches_per_call": 4,
+        "flop_utilisation": fl / (ms * 1e9) / peaks["bf16_tflops"],
+        "note": "6.3 MB working set, 48 CTAs per launch: launch- and latency-bound; the paper reports 4.78 % (A100) and 11.1 % (RTX 4090) "
+                "of those parts' peaks, i.e. about 15 and 18 TFLOP/s"}}
+    plan.close()
     return out
 
 
@@ -396,7 +423,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-side", action="store_true", help="skip the config-3 / config-4 side measurements")
     ap.add_argument("--quick", action="store_true", help="fewer repetitions of the side measurements")
-    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5"],
+    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5", "operator"],
                     help="run just this side workload (--steps launches after 2 warm-ups) and print its JSON; used for profiling")
     args = ap.parse_args()
     if args.impl == "reference":

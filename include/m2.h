@@ -135,6 +135,19 @@ int32_t m2_monarch_matmul_host(const m2_plan* plan, const void* X_host, const vo
                                void* Y_host, void* X_dev_scratch, void* Y_dev_scratch, int64_t T, void* ws_dev,
                                int64_t ws_bytes, void* stream);
 
+/* The M2 operator with general (learnable) Monarch matrices, Eq. 2 / the sequence- and feature-mixing lines of the M2
+ * layer listing:  Y = M_b sigma(K (.) M_a X),  M_a = P La P^T Ra P,  M_b = P Lb P^T Rb P,  sigma = identity or ReLU.
+ * X_dev, Y_dev: [T, N] in the plan dtype (Y_dev may be X_dev; Y_dev also holds the intermediate);
+ * K_dev: [Hk, N] in the plan dtype, row t of X takes row t mod Hk of K (one kernel row per channel with the rows of X
+ * ordered (batch, channel): Hk = channels; one shared row: Hk = 1).  Factors as in m2_monarch_matmul; ws_dev/ws_bytes
+ * as there (m2_matmul_workspace_bytes(plan, T)).  The product K (.) M_a X and sigma are taken in fp32 on the fp32
+ * accumulator; the intermediate is then rounded to the plan dtype. */
+#define M2_ACT_NONE 0
+#define M2_ACT_RELU 1
+int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev, int64_t Hk, int32_t act,
+                       const void* La_dev, const void* Ra_dev, const void* Lb_dev, const void* Rb_dev, void* Y_dev,
+                       int64_t T, void* ws_dev, int64_t ws_bytes, void* stream);
+
 /* W_out[b][c][r] = W_in[b][r][c]: block-wise transpose of a block-diagonal factor of nblocks blocks of rows x cols
  * elements of the plan dtype (W_out must not overlap W_in).  It gives the gradient of the Monarch matmul with
  * respect to its input: M^T = P^T R^T P L^T P^T (Sec. 3.1 transposed) is again an order-2 Monarch product, so for an

@@ -206,6 +206,18 @@ def monarch_apply_transpose(L: np.ndarray, R: np.ndarray, g: np.ndarray) -> np.n
     return v.reshape(*lead, N)
 
 
+def monarch_mix(La, Ra, Lb, Rb, K: np.ndarray, x: np.ndarray, act: str = "none") -> np.ndarray:
+    """The M2 operator y = M_b sigma(K (.) M_a x) along the last axis (Eq. 2 with general Monarch matrices; the M2
+    layer listing applies it once along the sequence and once along the features with sigma = ReLU).  x: [T, N];
+    K: [Hk, N], row t of x takes row t mod Hk of K (Hk = T: one kernel row per row; Hk = 1: one shared row)."""
+    assert act in ("none", "relu")
+    T = x.shape[0]
+    mid = K[np.arange(T) % K.shape[0]] * monarch_apply(La, Ra, x)
+    if act == "relu":
+        mid = np.maximum(mid, 0.0)
+    return monarch_apply(Lb, Rb, mid)
+
+
 def monarch_weight_grads(L: np.ndarray, R: np.ndarray, x: np.ndarray, g: np.ndarray):
     """Gradients of sum_t <M x_t, g_t> with respect to the blocks of L and R for M = P L P^T R P (Sec. 3.1), by the
     chain rule through the stages of monarch_apply: with v0 = P x ([n2][n1]), v1 = R v0 ([n2][k1]) and the upstream

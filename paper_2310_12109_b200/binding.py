@@ -35,6 +35,7 @@ SIGNATURES = {
     "m2_spectrum_conjugate": (_i32, [_vp, _vp, _i64, _vp, _vp]),
     "m2_matmul_bwd_workspace_bytes": (_i64, [_vp, _i64]),
     "m2_monarch_matmul_bwd_weights": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
+    "m2_monarch_mix": (_i32, [_vp, _vp, _vp, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
@@ -214,6 +215,25 @@ def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Ten
         ws = m2_matmul_workspace(plan, X.shape[0], X.device)
     _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _ptr(ws),
                                    0 if ws is None else ws.numel(), _stream()), "m2_monarch_matmul")
+    return Y
+
+
+M2_ACT_NONE, M2_ACT_RELU = 0, 1
+
+
+def m2_monarch_mix(plan: Plan, X: torch.Tensor, K: torch.Tensor, La, Ra, Lb, Rb, act: int = M2_ACT_NONE, Y: torch.Tensor | None = None,
+                   ws: torch.Tensor | None = None) -> torch.Tensor:
+    """Y = M_b sigma(K (.) M_a X); X: [T, N], K: [Hk, N] (row t uses K[t % Hk]), all of the plan dtype."""
+    for a in (X, K, La, Ra, Lb, Rb):
+        assert a.is_cuda and a.dtype == plan.torch_dtype and a.is_contiguous()
+    T = X.shape[0]
+    if Y is None:
+        Y = torch.empty_like(X)
+    assert X.dim() == 2 and X.shape[1] == plan.N and K.dim() == 2 and K.shape[1] == plan.N
+    if ws is None:
+        ws = m2_matmul_workspace(plan, T, X.device)
+    _check(lib().m2_monarch_mix(plan.handle, _ptr(X), _ptr(K), K.shape[0], act, _ptr(La), _ptr(Ra), _ptr(Lb), _ptr(Rb), _ptr(Y), T,
+                                _ptr(ws), 0 if ws is None else ws.numel(), _stream()), "m2_monarch_mix")
     return Y
 
 

@@ -250,7 +250,7 @@ __global__ void spectrum_to_natural_kernel(const float2* __restrict__ kf, float2
 //   z[n2][k1] = sum_{n1} R[n2][k1][n1] x[n1*N2 + n2];  y[k2*N1 + k1] = sum_{n2} L[k1][k2][n2] z[n2][k1]
 template <typename IO, int TT>
 __global__ void matmul_tokens_kernel(const IO* __restrict__ X, const IO* __restrict__ L, const IO* __restrict__ Rw,
-                                     IO* __restrict__ Y, int N1, int N2, long long T) {
+                                     IO* __restrict__ Y, int N1, int N2, long long T, const IO* __restrict__ Kmul, long long Hk, int relu) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = N1 * N2;
     float* xs = reinterpret_cast<float*>(smem_raw);  // [TT][N]
@@ -289,7 +289,14 @@ __global__ void matmul_tokens_kernel(const IO* __restrict__ X, const IO* __restr
         }
 #pragma unroll
         for (int t = 0; t < TT; ++t)
-            if (t0 + t < T) Y[(t0 + t) * N + o] = from_f32<IO>(acc[t]);
+            if (t0 + t < T) {
+                float v = acc[t];
+                if (Kmul) {   // y = sigma(K (.) M x): the first half of the M2 operator (Eq. 2)
+                    v *= to_f32<IO>(Kmul[((t0 + t) % Hk) * N + o]);
+                    if (relu) v = fmaxf(v, 0.f);
+                }
+                Y[(t0 + t) * N + o] = from_f32<IO>(v);
+            }
     }
 }
 
@@ -444,7 +451,7 @@ cudaError_t launch_spectrum_to_natural(const ConvShape& s, const void* kf, float
 
 template <typename IO>
 static cudaError_t launch_matmul_t(int N1, int N2, long long T, const void* X, const void* L, const void* R, void* Y,
-                                   cudaStream_t st) {
+                                   const void* Kmul, long long Hk, int relu, cudaStream_t st) {
     constexpr int TT = 4;
     const int N = N1 * N2;
     const size_t smem = (size_t)2 * TT * N * sizeof(float);
@@ -454,14 +461,15 @@ static cudaError_t launch_matmul_t(int N1, int N2, long long T, const void* X, c
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int threads = N < 512 ? ((N + 31) / 32) * 32 : 512;
-    kern<<<(unsigned)((T + TT - 1) / TT), threads, smem, st>>>((const IO*)X, (const IO*)L, (const IO*)R, (IO*)Y, N1, N2, T);
+    kern<<<(unsigned)((T + TT - 1) / TT), threads, smem, st>>>((const IO*)X, (const IO*)L, (const IO*)R, (IO*)Y, N1, N2, T,
+                                                                   (const IO*)Kmul, Hk, relu);
     return cudaGetLastError();
 }
 
 cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void* X, const void* L, const void* R, void* Y,
-                          cudaStream_t st) {
-    return bf16_io ? launch_matmul_t<__nv_bfloat16>(N1, N2, T, X, L, R, Y, st)
-                   : launch_matmul_t<float>(N1, N2, T, X, L, R, Y, st);
+                          const void* Kmul, long long Hk, int relu, cudaStream_t st) {
+    return bf16_io ? launch_matmul_t<__nv_bfloat16>(N1, N2, T, X, L, R, Y, Kmul, Hk, relu, st)
+                   : launch_matmul_t<float>(N1, N2, T, X, L, R, Y, Kmul, Hk, relu, st);
 }
 
 cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,

@@ -18,8 +18,9 @@ cudaError_t launch_conv(const ConvShape& s, bool bf16_io, const void* x, const v
                         cudaStream_t st);
 cudaError_t launch_spectrum(const ConvShape& s, const float* k, void* kf, cudaStream_t st);
 cudaError_t launch_spectrum_to_natural(const ConvShape& s, const void* kf, float* out, cudaStream_t st);
+// Kmul != nullptr: Y = sigma(K (.) M X), K [Hk][N] of the I/O type, row t uses K[t % Hk], sigma = ReLU if relu else identity
 cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void* X, const void* L, const void* R, void* Y,
-                          cudaStream_t st);
+                          const void* Kmul, long long Hk, int relu, cudaStream_t st);
 cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,
                        long long tokens, cudaStream_t st);
 

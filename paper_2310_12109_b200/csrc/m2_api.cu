@@ -325,6 +325,21 @@ int64_t m2_matmul_workspace_bytes(const m2_plan* plan, int64_t T) {
     return m2mm::workspace_bytes(plan, T);
 }
 
+// Y = sigma(K (.) M X) (K == nullptr: Y = M X); arguments already checked, device already current
+static int32_t matmul_impl(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, void* Y_dev, int64_t T,
+                           void* ws_dev, int64_t ws_bytes, const void* K_dev, int64_t Hk, int relu, cudaStream_t stream) {
+    if (T == 0) return M2_OK;
+    if (m2mm::covered(plan) && ws_dev && ws_bytes >= m2mm::workspace_bytes(plan, T))
+        return m2mm::matmul(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, K_dev, Hk, relu, stream);
+    cudaError_t e = m2g::launch_matmul(plan->dims[0], plan->dims[1], T, plan->dtype == M2_BF16, X_dev, L_dev, R_dev, Y_dev, K_dev,
+                                       Hk > 0 ? Hk : 1, relu, stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "matmul_generic";
+    plan->launches += 1;
+    return M2_OK;
+}
+
 int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, void* Y_dev,
                           int64_t T, void* ws_dev, int64_t ws_bytes, void* stream) {
     int32_t st = check_matmul_args(plan, X_dev, L_dev, R_dev, Y_dev, T);
@@ -332,16 +347,23 @@ int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_
     if (ws_dev && !aligned16(ws_dev)) return M2_ERR_ALIGNMENT;
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
-    if (T == 0) return M2_OK;
-    if (m2mm::covered(plan) && ws_dev && ws_bytes >= m2mm::workspace_bytes(plan, T))
-        return m2mm::matmul(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, (cudaStream_t)stream);
-    cudaError_t e = m2g::launch_matmul(plan->dims[0], plan->dims[1], T, plan->dtype == M2_BF16, X_dev, L_dev, R_dev,
-                                       Y_dev, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return M2_ERR_CUDA;
-    plan->last_kernel = "matmul_generic";
-    plan->launches += 1;
-    return M2_OK;
+    return matmul_impl(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, ws_bytes, nullptr, 1, 0, (cudaStream_t)stream);
+}
+
+int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev, int64_t Hk, int32_t act, const void* La_dev,
+                       const void* Ra_dev, const void* Lb_dev, const void* Rb_dev, void* Y_dev, int64_t T, void* ws_dev,
+                       int64_t ws_bytes, void* stream) {
+    int32_t st = check_matmul_args(plan, X_dev, La_dev, Ra_dev, Y_dev, T);
+    if (st != M2_OK) return st;
+    if (act != M2_ACT_NONE && act != M2_ACT_RELU) return M2_ERR_INVALID_ARG;
+    if (T > 0 && (!K_dev || !Lb_dev || !Rb_dev || Hk < 1)) return M2_ERR_INVALID_ARG;
+    if (!aligned16(K_dev) || !aligned16(Lb_dev) || !aligned16(Rb_dev) || (ws_dev && !aligned16(ws_dev))) return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    // the intermediate sigma(K (.) M_a X) lives in Y: every kernel of the second product reads its tokens before it writes them
+    st = matmul_impl(plan, X_dev, La_dev, Ra_dev, Y_dev, T, ws_dev, ws_bytes, K_dev, Hk, act == M2_ACT_RELU, (cudaStream_t)stream);
+    if (st != M2_OK) return st;
+    return matmul_impl(plan, Y_dev, Lb_dev, Rb_dev, Y_dev, T, ws_dev, ws_bytes, nullptr, 1, 0, (cudaStream_t)stream);
 }
 
 int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows, int64_t cols,

@@ -72,7 +72,7 @@ template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
 monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16* __restrict__ W,
                       const __grid_constant__ CUtensorMap map_out, __nv_bfloat16* __restrict__ zout, long long T,
-                      int32_t* __restrict__ status) {
+                      int32_t* __restrict__ status, const __nv_bfloat16* __restrict__ Kmul, long long Hk, int relu) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
     const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
@@ -178,6 +178,23 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
             tmem_ld_wait();
 #pragma unroll
             for (int bl = 0; bl < 8; ++bl) tmem_ld_fence8(v[bl]);
+            if (PASS == 2 && Kmul != nullptr && t0 + t < T) {
+                // y = sigma(K (.) M x) (first half of the M2 operator, Eq. 2): the 8 accumulators of one kk are the 8
+                // consecutive k1 of output index k2*64 + k1 -> one 16-byte piece of the kernel row
+                const __nv_bfloat16* krow = Kmul + (size_t)((t0 + t) % Hk) * 4096 + 8 * grp;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint4 kp = *reinterpret_cast<const uint4*>(krow + (o0 + kk) * 64);
+                    const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float a = v[2 * q][kk] * __uint_as_float(kw[q] << 16);
+                        float b = v[2 * q + 1][kk] * __uint_as_float(kw[q] & 0xffff0000u);
+                        v[2 * q][kk] = relu ? fmaxf(a, 0.f) : a;
+                        v[2 * q + 1][kk] = relu ? fmaxf(b, 0.f) : b;
+                    }
+                }
+            }
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
                 const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
@@ -214,7 +231,8 @@ cudaError_t prepare(const m2_plan* pl) {
     return e;
 }
 
-int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, cudaStream_t stream) {
+int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
+               int64_t Hk, int relu, cudaStream_t stream) {
     if (!covered(pl)) return M2_ERR_UNSUPPORTED;
     if (T == 0) return M2_OK;
     dim3 grid(8, (unsigned)((T + kTileT - 1) / kTileT));
@@ -234,10 +252,11 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, monarch64_pass_kernel<1>, (const __nv_bfloat16*)X, (const __nv_bfloat16*)R, my, (__nv_bfloat16*)ws,
-                           (long long)T, pl->d_status) != cudaSuccess)
+                           (long long)T, pl->d_status, (const __nv_bfloat16*)nullptr, 1LL, 0) != cudaSuccess)
         return M2_ERR_CUDA;
     if (cudaLaunchKernelEx(&cfg, monarch64_pass_kernel<2>, (const __nv_bfloat16*)ws, (const __nv_bfloat16*)L, my,
-                           (__nv_bfloat16*)nullptr, (long long)T, pl->d_status) != cudaSuccess)
+                           (__nv_bfloat16*)nullptr, (long long)T, pl->d_status, (const __nv_bfloat16*)Kmul, (long long)(Hk > 0 ? Hk : 1),
+                           relu) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "matmul_umma_64x64";
     pl->launches += 2;

@@ -8,7 +8,8 @@ namespace m2mm {
 bool covered(const m2_plan* plan);
 int64_t workspace_bytes(const m2_plan* plan, int64_t T);
 cudaError_t prepare(const m2_plan* plan);
-// two passes (R then L) exchanging the intermediate through `ws` (workspace_bytes(plan, T) bytes)
-int32_t matmul(const m2_plan* plan, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws,
-               cudaStream_t stream);
+// two passes (R then L) exchanging the intermediate through `ws` (workspace_bytes(plan, T) bytes); Y may be X.
+// Kmul != nullptr: Y = sigma(K (.) M X) with K [Hk][4096] bf16, row t uses K[t % Hk], sigma = ReLU if relu else identity
+int32_t matmul(const m2_plan* plan, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
+               int64_t Hk, int relu, cudaStream_t stream);
 }  // namespace m2mm

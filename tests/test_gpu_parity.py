@@ -368,6 +368,36 @@ def test_matmul_weight_gradients(T, dims, dtype):
     plan.close()
 
 
+@pytest.mark.parametrize("T,Hk,dims,dtype,act", [(300, 3, (64, 64), M.M2_BF16, "relu"), (257, 257, (64, 64), M.M2_BF16, "none"),
+                                                  (50, 1, (8, 4), M.M2_BF16, "relu"), (19, 5, (4, 6), M.M2_FP32, "relu"),
+                                                  (19, 19, (4, 6), M.M2_FP32, "none")])
+def test_monarch_mix_operator(T, Hk, dims, dtype, act):
+    """Y = M_b sigma(K (.) M_a X) with general Monarch factors (Eq. 2; the mixing lines of the M2 layer listing)."""
+    N1, N2 = dims
+    N = N1 * N2
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    W = [rnd(synth.normal(synth.stream_id(10, i), shp) / np.sqrt(shp[-1]))
+         for i, shp in enumerate([(N1, N2, N2), (N2, N1, N1), (N1, N2, N2), (N2, N1, N1)])]
+    K = rnd(synth.normal(synth.stream_id(10, 4), (Hk, N)))
+    X = rnd(synth.normal(synth.stream_id(10, 5), (T, N)))
+    plan = M.Plan(dims, dtype=dtype, device=0)
+    d = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
+    Xd = d(X)
+    Y = M.m2_monarch_mix(plan, Xd, d(K), d(W[0]), d(W[1]), d(W[2]), d(W[3]), act=M.M2_ACT_RELU if act == "relu" else M.M2_ACT_NONE)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    assert plan.last_kernel() == ("matmul_umma_64x64" if dims == (64, 64) else "matmul_generic")
+    ref = O.monarch_mix(W[0], W[1], W[2], W[3], K, X, act)
+    tol = TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32
+    check(host(Y), ref, tol, "monarch mix")
+    # in place (Y = X) gives the same bits
+    Y2 = M.m2_monarch_mix(plan, Xd, d(K), d(W[0]), d(W[1]), d(W[2]), d(W[3]), act=M.M2_ACT_RELU if act == "relu" else M.M2_ACT_NONE, Y=Xd)
+    torch.cuda.synchronize()
+    assert torch.equal(Y2, Y)
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -348,6 +348,34 @@ def test_monarch_transpose_apply(N1, N2):
     assert np.allclose(O.monarch_apply(Lt, Rt, g), g @ Md)
 
 
+def test_monarch_mix_operator():
+    """M_b sigma(K (.) M_a x): against dense matrices; with identity blocks M = P, so the operator is the closed-form
+    permutation y = P (K (.) P x); with M_a = F, M_b = F^-1 (complex factors) it is the circular convolution."""
+    N1, N2, T, Hk = 3, 4, 6, 2
+    N = N1 * N2
+    La, Lb = rng.standard_normal((2, N1, N2, N2))
+    Ra, Rb = rng.standard_normal((2, N2, N1, N1))
+    K, x = rng.standard_normal((Hk, N)), rng.standard_normal((T, N))
+    Ma, Mb = O.monarch_dense(La, Ra), O.monarch_dense(Lb, Rb)
+    for act in ("none", "relu"):
+        mid = np.tile(K, (T // Hk, 1)) * (x @ Ma.T)
+        if act == "relu":
+            mid = np.where(mid > 0, mid, 0.0)
+        assert np.allclose(O.monarch_mix(La, Ra, Lb, Rb, K, x, act), mid @ Mb.T)
+    # identity blocks: M = P with (P v)[n2 N1 + n1] = v[n1 N2 + n2]
+    I_L, I_R = np.broadcast_to(np.eye(N2), (N1, N2, N2)), np.broadcast_to(np.eye(N1), (N2, N1, N1))
+    y = O.monarch_mix(I_L, I_R, I_L, I_R, K[:1], x)
+    Px = x.reshape(T, N1, N2).swapaxes(1, 2).reshape(T, N)
+    want = (K[0] * Px).reshape(T, N1, N2).swapaxes(1, 2).reshape(T, N)
+    assert np.array_equal(y, want)
+    # DFT factors: the operator is the circular convolution with the kernel whose spectrum is K (Eq. 2)
+    Lf, Rf = O.monarch_dft_factors(N1, N2)
+    k = rng.standard_normal((Hk, N))
+    kf = k @ O.dft_matrix(N).T
+    y = O.monarch_mix(Lf, Rf, np.conj(Lf), np.conj(Rf) / N, kf, x.astype(complex))
+    assert np.allclose(y.imag, 0) and np.allclose(y.real, np.stack([O.direct_circular_conv(k[t % Hk], x[t]) for t in range(T)]))
+
+
 @pytest.mark.parametrize("N1,N2", [(2, 3), (4, 4), (5, 2)])
 def test_monarch_weight_grads(N1, N2):
     """y is linear in L and in R, so perturbing one weight by 1 changes sum <y, g> by exactly that weight's

@@ -148,6 +148,23 @@ int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev
                        const void* La_dev, const void* Ra_dev, const void* Lb_dev, const void* Rb_dev, void* Y_dev,
                        int64_t T, void* ws_dev, int64_t ws_bytes, void* stream);
 
+/* The basic M2 layer (App. "Implementation", the MonarchMixerLayer listing), x: [B, n, d] in the plans' dtype:
+ *   x~  = (M2 relu(K_n (.) M1 x^T))^T        mix along the sequence;  K_n = n_kernel_dev [d, n]
+ *   y   = M4 relu(k_d (.) M3 x~)             mix along the features;  k_d = d_kernel_dev [1, d]
+ *   out = LayerNorm(y + x~) * gamma + beta   over d, biased variance, eps inside the root; gamma, beta fp32 [d]
+ * plan_n: order-2 plan of length n (M1, M2), plan_d: order-2 plan of length d (M3, M4); same dtype and device.
+ * factors: HOST array of 8 device pointers {L1, R1, L2, R2, L3, R3, L4, R4}, each pair as in m2_monarch_matmul
+ * (R is applied first; the listing's parameter called L is the one applied first, i.e. this library's R).
+ * y_dev: [B, n, d] (must not overlap x_dev).  scratch_dev: m2_layer_scratch_bytes(plan_n, plan_d, B) bytes, caller-owned.
+ * ws_dev / ws_bytes: optional matmul workspace, at least the larger of m2_matmul_workspace_bytes(plan_n, B d) and
+ * m2_matmul_workspace_bytes(plan_d, B n); NULL selects the kernels that need none.  9 launches with a workspace
+ * for both products, fewer on the generic path. */
+int64_t m2_layer_scratch_bytes(const m2_plan* plan_n, const m2_plan* plan_d, int64_t B);
+int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x_dev, const void* const* factors,
+                     const void* n_kernel_dev, const void* d_kernel_dev, const float* gamma_dev, const float* beta_dev,
+                     float eps, void* y_dev, int64_t B, void* scratch_dev, int64_t scratch_bytes, void* ws_dev,
+                     int64_t ws_bytes, void* stream);
+
 /* W_out[b][c][r] = W_in[b][r][c]: block-wise transpose of a block-diagonal factor of nblocks blocks of rows x cols
  * elements of the plan dtype (W_out must not overlap W_in).  It gives the gradient of the Monarch matmul with
  * respect to its input: M^T = P^T R^T P L^T P^T (Sec. 3.1 transposed) is again an order-2 Monarch product, so for an

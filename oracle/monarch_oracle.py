@@ -218,6 +218,31 @@ def monarch_mix(La, Ra, Lb, Rb, K: np.ndarray, x: np.ndarray, act: str = "none")
     return monarch_apply(Lb, Rb, mid)
 
 
+def layer_norm(v: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float = 1e-5) -> np.ndarray:
+    """LayerNorm over the last axis: (v - mean) / sqrt(var + eps) * gamma + beta with the biased variance."""
+    mu = v.mean(axis=-1, keepdims=True)
+    var = ((v - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (v - mu) / np.sqrt(var + eps) * gamma + beta
+
+
+def m2_layer(x: np.ndarray, p: dict, eps: float = 1e-5, stages: dict | None = None) -> np.ndarray:
+    """The basic M2 layer (App. "Implementation", the MonarchMixerLayer listing), x: [B, n, d]:
+        x~ = (M2 relu(K_n (.) M1 x^T))^T                 mix along the sequence, K_n: [d, n]
+        y  = M4 relu(k_d (.) M3 x~)                      mix along the features, k_d: [1, d]
+        out = LayerNorm(y + x~).
+    p: factors "L1","R1",..,"L4","R4" in this library's convention (R is applied first: the listing's parameter
+    called L), "n_kernel", "d_kernel", "gamma", "beta"."""
+    B, n, d = x.shape
+    xT = np.swapaxes(x, 1, 2).reshape(B * d, n)                                        # rows (b, channel)
+    u = monarch_mix(p["L1"], p["R1"], p["L2"], p["R2"], p["n_kernel"], xT, "relu")     # row (b, c) takes K_n[c]
+    xt = np.swapaxes(u.reshape(B, d, n), 1, 2)                                         # [B, n, d]
+    y = monarch_mix(p["L3"], p["R3"], p["L4"], p["R4"], p["d_kernel"], xt.reshape(B * n, d), "relu").reshape(B, n, d)
+    out = layer_norm(y + xt, p["gamma"], p["beta"], eps)
+    if stages is not None:
+        stages.update(x_tilde=xt, y=y)
+    return out
+
+
 def monarch_weight_grads(L: np.ndarray, R: np.ndarray, x: np.ndarray, g: np.ndarray):
     """Gradients of sum_t <M x_t, g_t> with respect to the blocks of L and R for M = P L P^T R P (Sec. 3.1), by the
     chain rule through the stages of monarch_apply: with v0 = P x ([n2][n1]), v1 = R v0 ([n2][k1]) and the upstream

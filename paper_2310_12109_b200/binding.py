@@ -36,6 +36,8 @@ SIGNATURES = {
     "m2_matmul_bwd_workspace_bytes": (_i64, [_vp, _i64]),
     "m2_monarch_matmul_bwd_weights": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_mix": (_i32, [_vp, _vp, _vp, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
+    "m2_layer_scratch_bytes": (_i64, [_vp, _vp, _i64]),
+    "m2_layer_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
@@ -235,6 +237,29 @@ def m2_monarch_mix(plan: Plan, X: torch.Tensor, K: torch.Tensor, La, Ra, Lb, Rb,
     _check(lib().m2_monarch_mix(plan.handle, _ptr(X), _ptr(K), K.shape[0], act, _ptr(La), _ptr(Ra), _ptr(Lb), _ptr(Rb), _ptr(Y), T,
                                 _ptr(ws), 0 if ws is None else ws.numel(), _stream()), "m2_monarch_mix")
     return Y
+
+
+def m2_layer_fwd(plan_n: Plan, plan_d: Plan, x: torch.Tensor, factors, n_kernel: torch.Tensor, d_kernel: torch.Tensor,
+                 gamma: torch.Tensor, beta: torch.Tensor, eps: float = 1e-5, ws: torch.Tensor | None = None) -> torch.Tensor:
+    """The basic M2 layer on x [B, n, d]; factors = (L1, R1, L2, R2, L3, R3, L4, R4); gamma, beta fp32 [d]."""
+    B, n, d = x.shape
+    assert n == plan_n.N and d == plan_d.N and len(factors) == 8
+    for a in (x, n_kernel, d_kernel, *factors):
+        assert a.is_cuda and a.dtype == plan_n.torch_dtype and a.is_contiguous()
+    for a in (gamma, beta):
+        assert a.is_cuda and a.dtype == torch.float32 and a.is_contiguous() and a.numel() == d
+    assert tuple(n_kernel.shape) == (d, n) and d_kernel.numel() == d
+    y = torch.empty_like(x)
+    sb = int(lib().m2_layer_scratch_bytes(plan_n.handle, plan_d.handle, B))
+    scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=x.device)
+    if ws is None:
+        need = max(int(lib().m2_matmul_workspace_bytes(plan_n.handle, B * d)), int(lib().m2_matmul_workspace_bytes(plan_d.handle, B * n)))
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device) if need > 0 else None
+    fp = (ctypes.c_void_p * 8)(*[f.data_ptr() for f in factors])
+    _check(lib().m2_layer_fwd(plan_n.handle, plan_d.handle, _ptr(x), fp, _ptr(n_kernel), _ptr(d_kernel), _ptr(gamma), _ptr(beta), eps,
+                              _ptr(y), B, _ptr(scratch), scratch.numel(), _ptr(ws), 0 if ws is None else ws.numel(), _stream()),
+           "m2_layer_fwd")
+    return y
 
 
 def m2_blocks_transpose(plan: Plan, W: torch.Tensor) -> torch.Tensor:

@@ -772,4 +772,75 @@ cudaError_t launch_matmul_wgrad(int N1, int N2, long long T, bool bf16_io, const
                                                   ws, st);
 }
 
+// out[b][c][r] = in[b][r][c] for any sizes and both I/O types: 32 x 32 tiles through shared memory
+template <typename T>
+__global__ void __launch_bounds__(256) transpose_any_kernel(const T* __restrict__ in, T* __restrict__ out, int R, int C) {
+    __shared__ T tile[32][33];
+    const long long b = blockIdx.z;
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    for (int i = ty; i < 32; i += 8)
+        if (r0 + i < R && c0 + tx < C) tile[i][tx] = in[(b * R + r0 + i) * C + c0 + tx];
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8)
+        if (c0 + i < C && r0 + tx < R) out[(b * C + c0 + i) * R + r0 + tx] = tile[tx][i];
+}
+
+cudaError_t launch_transpose_any(const void* in, void* out, long long B, int R, int C, bool bf16, cudaStream_t st) {
+    if (B == 0 || R == 0 || C == 0) return cudaSuccess;
+    if (B > 65535 || (R + 31) / 32 > 65535) return cudaErrorInvalidValue;
+    if (bf16 && R % 64 == 0 && C % 64 == 0) return launch_transpose_btc(in, out, B, R, C, st);
+    const dim3 grid((C + 31) / 32, (R + 31) / 32, (unsigned)B);
+    if (bf16)
+        transpose_any_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)in, (__nv_bfloat16*)out, R, C);
+    else
+        transpose_any_kernel<float><<<grid, 256, 0, st>>>((const float*)in, (float*)out, R, C);
+    return cudaGetLastError();
+}
+
+// y[row] = LayerNorm(a[row] + b[row]) * gamma + beta over d values per row (biased variance, fp32 statistics, two passes
+// over registers-or-L1-resident data); one 128-thread block per row; y may be a or b.
+template <typename IO>
+__global__ void __launch_bounds__(128) add_layernorm_kernel(const IO* a, const IO* b, const float* __restrict__ gamma,
+                                                            const float* __restrict__ beta, IO* y, int d, float eps) {
+    __shared__ float red[4];
+    const long long row = blockIdx.x;
+    const IO* ar = a + row * d;
+    const IO* br = b + row * d;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    auto block_sum = [&](float v) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        __syncthreads();   // red[] may still be read from the previous reduction
+        if (lane == 0) red[w] = v;
+        __syncthreads();
+        return red[0] + red[1] + red[2] + red[3];
+    };
+    float s = 0.f;
+    for (int i = threadIdx.x; i < d; i += 128) s += to_f32<IO>(ar[i]) + to_f32<IO>(br[i]);
+    const float mean = block_sum(s) / (float)d;
+    float q = 0.f;
+    for (int i = threadIdx.x; i < d; i += 128) {
+        const float v = to_f32<IO>(ar[i]) + to_f32<IO>(br[i]) - mean;
+        q = fmaf(v, v, q);
+    }
+    const float rstd = rsqrtf(block_sum(q) / (float)d + eps);
+    for (int i = threadIdx.x; i < d; i += 128) {
+        const float v = to_f32<IO>(ar[i]) + to_f32<IO>(br[i]) - mean;
+        y[row * d + i] = from_f32<IO>(fmaf(v * rstd, gamma[i], beta[i]));
+    }
+}
+
+cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamma, const float* beta, void* y, long long rows, int d,
+                                 float eps, bool bf16, cudaStream_t st) {
+    if (rows == 0) return cudaSuccess;
+    if (rows > 0x7fffffffLL) return cudaErrorInvalidValue;
+    if (bf16)
+        add_layernorm_kernel<__nv_bfloat16><<<(unsigned)rows, 128, 0, st>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, gamma, beta,
+                                                                           (__nv_bfloat16*)y, d, eps);
+    else
+        add_layernorm_kernel<float><<<(unsigned)rows, 128, 0, st>>>((const float*)a, (const float*)b, gamma, beta, (float*)y, d, eps);
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

@@ -35,6 +35,11 @@ cudaError_t launch_blocks_transpose(const void* in, void* out, long long nblocks
 // dL[N1][N2][N2], dR[N2][N1][N1] (fp32) of sum_t <M x_t, g_t>; ws: T*N floats (4 launches)
 cudaError_t launch_matmul_wgrad(int N1, int N2, long long T, bool bf16_io, const void* X, const void* G, const void* L, const void* R,
                                 float* dL, float* dR, float* ws, cudaStream_t st);
+// out[b][c][r] = in[b][r][c], any sizes, fp32 or bf16
+cudaError_t launch_transpose_any(const void* in, void* out, long long B, int R, int C, bool bf16, cudaStream_t st);
+// y[row] = LayerNorm(a[row] + b[row]) * gamma + beta over d values (y may alias a or b)
+cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamma, const float* beta, void* y, long long rows, int d,
+                                 float eps, bool bf16, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -366,6 +366,51 @@ int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev
     return matmul_impl(plan, Y_dev, Lb_dev, Rb_dev, Y_dev, T, ws_dev, ws_bytes, nullptr, 1, 0, (cudaStream_t)stream);
 }
 
+static int64_t round256(int64_t v) { return (v + 255) / 256 * 256; }
+
+int64_t m2_layer_scratch_bytes(const m2_plan* plan_n, const m2_plan* plan_d, int64_t B) {
+    if (!plan_n || !plan_d || B < 0) return -1;
+    return 2 * round256(B * plan_n->N * plan_d->N * (plan_n->dtype == M2_BF16 ? 2 : 4));
+}
+
+int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x_dev, const void* const* factors, const void* n_kernel_dev,
+                     const void* d_kernel_dev, const float* gamma_dev, const float* beta_dev, float eps, void* y_dev, int64_t B,
+                     void* scratch_dev, int64_t scratch_bytes, void* ws_dev, int64_t ws_bytes, void* stream) {
+    if (!plan_n || !plan_d || !factors || B < 0 || !(eps >= 0.f)) return M2_ERR_INVALID_ARG;
+    if (plan_n->device < 0 || plan_d->device < 0) return M2_ERR_NO_DEVICE;
+    if (plan_n->p != 2 || plan_d->p != 2) return M2_ERR_UNSUPPORTED;
+    if (plan_n->dtype != plan_d->dtype || plan_n->device != plan_d->device) return M2_ERR_INVALID_ARG;
+    const int64_t n = plan_n->N, d = plan_d->N;
+    if (B > 65535 || B * n > 0x7fffffffLL || B * d > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    if (B == 0) return M2_OK;
+    for (int i = 0; i < 8; ++i)
+        if (!factors[i] || !aligned16(factors[i])) return factors[i] ? M2_ERR_ALIGNMENT : M2_ERR_INVALID_ARG;
+    if (!x_dev || !n_kernel_dev || !d_kernel_dev || !gamma_dev || !beta_dev || !y_dev || !scratch_dev) return M2_ERR_INVALID_ARG;
+    if (!aligned16(x_dev) || !aligned16(n_kernel_dev) || !aligned16(d_kernel_dev) || !aligned16(y_dev) || !aligned16(scratch_dev) ||
+        (ws_dev && !aligned16(ws_dev)))
+        return M2_ERR_ALIGNMENT;
+    const bool bf = plan_n->dtype == M2_BF16;
+    const int64_t tensor_bytes = B * n * d * (bf ? 2 : 4);
+    if (scratch_bytes < 2 * round256(tensor_bytes)) return M2_ERR_INVALID_ARG;
+    DeviceGuard g(plan_n->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    void* s1 = scratch_dev;                                                  // [B, d, n]: x^T, then the sequence mix
+    void* s2 = static_cast<unsigned char*>(scratch_dev) + round256(tensor_bytes);   // [B, n, d]: x~
+    if (m2g::launch_transpose_any(x_dev, s1, B, (int)n, (int)d, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    int32_t rc = matmul_impl(plan_n, s1, factors[0], factors[1], s1, B * d, ws_dev, ws_bytes, n_kernel_dev, d, 1, st);
+    if (rc == M2_OK) rc = matmul_impl(plan_n, s1, factors[2], factors[3], s1, B * d, ws_dev, ws_bytes, nullptr, 1, 0, st);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_transpose_any(s1, s2, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    rc = matmul_impl(plan_d, s2, factors[4], factors[5], y_dev, B * n, ws_dev, ws_bytes, d_kernel_dev, 1, 1, st);
+    if (rc == M2_OK) rc = matmul_impl(plan_d, y_dev, factors[6], factors[7], y_dev, B * n, ws_dev, ws_bytes, nullptr, 1, 0, st);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_add_layernorm(y_dev, s2, gamma_dev, beta_dev, y_dev, B * n, (int)d, eps, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    plan_n->launches += 3;   // the two transposes and the normalisation (the products count themselves on their plans)
+    plan_n->last_kernel = "layer_fwd";
+    return M2_OK;
+}
+
 int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows, int64_t cols,
                             void* stream) {
     if (!plan || nblocks < 0 || rows <= 0 || cols <= 0 || rows > 65536 || cols > 65536) return M2_ERR_INVALID_ARG;

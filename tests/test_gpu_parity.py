@@ -398,6 +398,34 @@ def test_monarch_mix_operator(T, Hk, dims, dtype, act):
     plan.close()
 
 
+@pytest.mark.parametrize("B,sn,sd,dtype", [(2, 64, 8, M.M2_BF16), (3, 5, 3, M.M2_FP32), (2, 8, 64, M.M2_BF16)])
+def test_m2_layer_fwd(B, sn, sd, dtype):
+    """The basic M2 layer (the MonarchMixerLayer listing): sequence mix, feature mix, residual LayerNorm."""
+    n, d = sn * sn, sd * sd
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    p = {}
+    for i, s in ((1, sn), (2, sn), (3, sd), (4, sd)):
+        p[f"L{i}"] = rnd(synth.normal(synth.stream_id(11, 2 * i), (s, s, s)) / np.sqrt(s))
+        p[f"R{i}"] = rnd(synth.normal(synth.stream_id(11, 2 * i + 1), (s, s, s)) / np.sqrt(s))
+    p["n_kernel"] = rnd(synth.normal(synth.stream_id(11, 20), (d, n)))
+    p["d_kernel"] = rnd(synth.normal(synth.stream_id(11, 21), (1, d)))
+    p["gamma"] = (1.0 + 0.1 * synth.normal(synth.stream_id(11, 22), (d,))).astype(np.float32).astype(np.float64)
+    p["beta"] = (0.1 * synth.normal(synth.stream_id(11, 23), (d,))).astype(np.float32).astype(np.float64)
+    x = rnd(synth.normal(synth.stream_id(11, 24), (B, n, d)))
+    plan_n, plan_d = M.Plan((sn, sn), dtype=dtype, device=0), M.Plan((sd, sd), dtype=dtype, device=0)
+    dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
+    fac = [dv(p[k]) for k in ("L1", "R1", "L2", "R2", "L3", "R3", "L4", "R4")]
+    y = M.m2_layer_fwd(plan_n, plan_d, dv(x), fac, dv(p["n_kernel"]), dv(p["d_kernel"]),
+                       dev(p["gamma"].astype(np.float32), torch.float32), dev(p["beta"].astype(np.float32), torch.float32))
+    torch.cuda.synchronize()
+    assert plan_n.device_status() == 0 and plan_d.device_status() == 0 and plan_n.last_kernel() == "layer_fwd"
+    ref = O.m2_layer(x, p)
+    check(host(y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, "M2 layer")
+    plan_n.close()
+    plan_d.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -376,6 +376,36 @@ def test_monarch_mix_operator():
     assert np.allclose(y.imag, 0) and np.allclose(y.real, np.stack([O.direct_circular_conv(k[t % Hk], x[t]) for t in range(T)]))
 
 
+def test_m2_layer_oracle():
+    """The layer against the same computation with dense matrices and einsum over the un-transposed [B, n, d] tensor;
+    LayerNorm against torch's routine and its invariants (zero mean, unit variance, shift/scale invariance)."""
+    import torch
+    B, sn, sd = 2, 3, 2
+    n, d = sn * sn, sd * sd
+    p = {}
+    for i in (1, 2):
+        p[f"L{i}"], p[f"R{i}"] = rng.standard_normal((sn, sn, sn)), rng.standard_normal((sn, sn, sn))
+    for i in (3, 4):
+        p[f"L{i}"], p[f"R{i}"] = rng.standard_normal((sd, sd, sd)), rng.standard_normal((sd, sd, sd))
+    p["n_kernel"], p["d_kernel"] = rng.standard_normal((d, n)), rng.standard_normal((1, d))
+    p["gamma"], p["beta"] = rng.standard_normal(d), rng.standard_normal(d)
+    x = rng.standard_normal((B, n, d))
+    st = {}
+    out = O.m2_layer(x, p, stages=st)
+    D = {i: O.monarch_dense(p[f"L{i}"], p[f"R{i}"]) for i in (1, 2, 3, 4)}
+    a = np.einsum("kn,bnc->bkc", D[1], x) * p["n_kernel"].T[None]                 # [B, n, d], kernel indexed [c, k]
+    xt = np.einsum("kn,bnc->bkc", D[2], np.maximum(a, 0))
+    y = np.maximum(p["d_kernel"][0] * (xt @ D[3].T), 0) @ D[4].T
+    assert np.allclose(st["x_tilde"], xt) and np.allclose(st["y"], y)
+    s = y + xt
+    want = torch.nn.functional.layer_norm(torch.from_numpy(s), (d,), torch.from_numpy(p["gamma"]), torch.from_numpy(p["beta"]), 1e-5).numpy()
+    assert np.allclose(out, want)
+    v = rng.standard_normal((5, 64))
+    ln = O.layer_norm(v, np.ones(64), np.zeros(64), 0.0)
+    assert np.allclose(ln.mean(-1), 0) and np.allclose(ln.var(-1), 1)
+    assert np.allclose(O.layer_norm(3.0 * v + 7.0, np.ones(64), np.zeros(64), 0.0), ln)
+
+
 @pytest.mark.parametrize("N1,N2", [(2, 3), (4, 4), (5, 2)])
 def test_monarch_weight_grads(N1, N2):
     """y is linear in L and in R, so perturbing one weight by 1 changes sum <y, g> by exactly that weight's

@@ -428,7 +428,8 @@ int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_o
 
 int64_t m2_matmul_bwd_workspace_bytes(const m2_plan* plan, int64_t T) {
     if (!plan || plan->p != 2 || T < 0) return -1;
-    return T * plan->N * 4;
+    const int64_t generic = T * plan->N * 4, umma = m2mm::wgrad_workspace_bytes(plan, T);
+    return generic > umma ? generic : umma;
 }
 
 int32_t m2_monarch_matmul_bwd_weights(const m2_plan* plan, const void* X_dev, const void* G_dev, const void* L_dev, const void* R_dev,
@@ -440,6 +441,7 @@ int32_t m2_monarch_matmul_bwd_weights(const m2_plan* plan, const void* X_dev, co
     if (T > 0 && (!ws_dev || ws_bytes < m2_matmul_bwd_workspace_bytes(plan, T))) return M2_ERR_INVALID_ARG;
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
+    if (m2mm::covered(plan)) return m2mm::wgrad(plan, X_dev, G_dev, L_dev, R_dev, dL_dev, dR_dev, T, ws_dev, (cudaStream_t)stream);
     cudaError_t e = m2g::launch_matmul_wgrad(plan->dims[0], plan->dims[1], T, plan->dtype == M2_BF16, X_dev, G_dev, L_dev, R_dev, dL_dev,
                                              dR_dev, (float*)ws_dev, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;

@@ -23,6 +23,9 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstring>
+
+#include "generic_kernels.h"
 #include "matmul_umma.h"
 #include "ptx_sm100.cuh"
 #include "tma_host.h"
@@ -219,6 +222,205 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
     if (tid < 32) tmem_dealloc(tmem, 512);
 }
 
+bool covered(const m2_plan* pl);
+int64_t workspace_bytes(const m2_plan* pl, int64_t T);
+
+// ---- gradients with respect to the weight blocks ------------------------------------------------------------------
+//
+//   D_b[m][a] = sum_t Z_b[t][m] * V_b[t][a]        for the 64 blocks b, contraction over ALL tokens
+//
+// V = x or the upstream gradient g, read as [t][a][b] with the block index b contiguous (exactly what pass 1 reads), and
+// Z = the intermediate in the workspace layout [token tile][m / 8][b][t % 128][m % 8] that pass 1 writes:
+//   dR[n2][k1][n1] = sum_t dv[t][n2][k1] x[t][n1][n2]:  V = x (b = n2, a = n1),  Z = pass 1 of (g, L^T) (m = k1)
+//   dL[k1][k2][n2] = sum_t g[t][k2][k1] v[t][n2][k1]:   V = g (b = k1, a = k2),  Z = pass 1 of (x, R)   (m = n2), D = dL[k1]^T
+// With the tokens as the K dimension both operands lie in shared memory as the forward kernels already produce them: the
+// 128-byte-swizzled tile [t][a] that pass 1 builds from 16-byte pieces of V is an N-major B operand (a row = one t), and a
+// workspace block [t][8 m] is a column of M-major core matrices (8 consecutive t x 16 bytes) of the A operand.
+// A CTA owns 8 consecutive blocks and one share of the 64-token half tiles, accumulates its 8 [64 x 64] partial results in
+// TMEM (M = 64: rows in lanes 0..15 of every lane quarter) over its whole share and writes them once; a second kernel adds
+// the shares in a fixed order.
+constexpr int WG_OFF_X = 0;           // 8 operands [64 t][64 a] bf16, swizzled rows of 128 bytes            65536
+constexpr int WG_OFF_Z = 65536;       // [m / 8][block 8][64 t][16 B]                                         65536
+constexpr int WG_OFF_BAR = 131072;
+constexpr int WG_SMEM = WG_OFF_BAR + 64;
+constexpr int kWgSplits = 18;         // 8 block groups x 18 shares = 144 CTAs
+constexpr size_t kWgPartialBytes = (size_t)kWgSplits * 64 * 4096 * 4;
+
+__global__ void __launch_bounds__(kThreads, 1)
+monarch64_wgrad_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16* __restrict__ zin, float* __restrict__ partial,
+                       long long T, int units, int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t bar_mma = s_base + WG_OFF_BAR, s_tptr = s_base + WG_OFF_BAR + 16, bar_in = s_base + WG_OFF_BAR + 24;
+    const int grp = blockIdx.x, split = blockIdx.y, nsplit = gridDim.y;
+    if (tid == 0) {
+        mbar_init(bar_mma, 1);
+        mbar_init(bar_in, 1);
+        fence_barrier_init();
+    }
+    if (tid < 32) tmem_alloc(s_tptr, 512);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // the workspace was written by the kernel before this one
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + WG_OFF_BAR + 16);
+    constexpr uint32_t IDESC = instr_desc_bf16(64, 64, true, true);
+    uint32_t ph = 0;
+    bool ok = true;
+    int it = 0;
+#pragma unroll 1
+    for (int u = split; u < units; u += nsplit, ++it) {
+        const int tile = u >> 1, half = u & 1;
+        const long long t0 = (long long)tile * kTileT + half * 64;
+        if (tid == 0) {   // 64 tokens of the 8 blocks' workspace columns: 64 pieces of 1 KB
+            mbar_expect_tx(bar_in, 65536);
+            const unsigned char* zb = reinterpret_cast<const unsigned char*>(zin) + (size_t)tile * (8 * 131072) + (size_t)grp * 16384 + half * 1024;
+            for (int kc = 0; kc < 8; ++kc)
+                for (int bl = 0; bl < 8; ++bl)
+                    bulk_load(s_base + WG_OFF_Z + kc * 8192 + bl * 1024, zb + (size_t)kc * 131072 + bl * 2048, 1024, bar_in);
+        }
+        {   // one (token, group of 8 a) per thread: 8 pieces of 16 bytes, 8 x 8 transpose, 8 stores (see pass 1)
+            const int g = tid & 7, tt = tid >> 3;
+            uint4 v[8];
+            const bool live = t0 + tt < T;
+            const uint4* src = reinterpret_cast<const uint4*>(in + (size_t)(t0 + tt) * 4096 + (size_t)(8 * g) * 64 + grp * 8);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (live)
+                    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i].x), "=r"(v[i].y), "=r"(v[i].z), "=r"(v[i].w) : "l"(src + i * 8));
+            }
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint4 lo, hi;
+                lo.x = prmt(w[0 * 4 + j], w[1 * 4 + j], 0x5410); hi.x = prmt(w[0 * 4 + j], w[1 * 4 + j], 0x7632);
+                lo.y = prmt(w[2 * 4 + j], w[3 * 4 + j], 0x5410); hi.y = prmt(w[2 * 4 + j], w[3 * 4 + j], 0x7632);
+                lo.z = prmt(w[4 * 4 + j], w[5 * 4 + j], 0x5410); hi.z = prmt(w[4 * 4 + j], w[5 * 4 + j], 0x7632);
+                lo.w = prmt(w[6 * 4 + j], w[7 * 4 + j], 0x5410); hi.w = prmt(w[6 * 4 + j], w[7 * 4 + j], 0x7632);
+                *reinterpret_cast<uint4*>(smem + WG_OFF_X + (2 * j) * 8192 + sw_off(tt, g)) = lo;
+                *reinterpret_cast<uint4*>(smem + WG_OFF_X + (2 * j + 1) * 8192 + sw_off(tt, g)) = hi;
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            const bool in_ok = mbar_wait(bar_in, ph);
+            if (in_ok) {
+#pragma unroll 1
+                for (int bl = 0; bl < kGroup; ++bl)
+#pragma unroll
+                    for (int s = 0; s < 4; ++s)   // 16 tokens per instruction
+                        umma_f16(tmem + bl * 64, smem_desc(s_base + WG_OFF_Z + bl * 1024 + s * 256, 128, 8192),
+                                 smem_desc_sw128(s_base + WG_OFF_X + bl * 8192 + s * 2048, 8192, 1024), IDESC, (it > 0 || s > 0) ? 1u : 0u);
+            }
+            umma_commit(bar_mma);
+            if (!in_ok) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+        }
+        ok = mbar_wait(bar_mma, ph);   // both operand buffers are free again
+        ph ^= 1;
+        tc_fence_after();
+        if (!__syncthreads_and(ok)) {
+            ok = false;
+            break;
+        }
+    }
+    // the 8 accumulators: row r of a block sits in lane (r % 16) of lane quarter r / 16; warpgroup wg takes blocks 2 wg, 2 wg + 1
+    if (ok && it > 0) {
+        const int q = warp & 3, wg = warp >> 2, r = 16 * q + lane;
+        const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+        for (int bb = 0; bb < 2; ++bb) {
+            const int bl = 2 * wg + bb;
+            float* dst = partial + (((size_t)split * 64 + grp * 8 + bl) * 64 + r) * 64;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 64; c0 += 8) {
+                float v[8];
+                tmem_ld8(t_lane + bl * 64 + c0, v);
+                tmem_ld_wait();
+                tmem_ld_fence8(v);
+                if (lane < 16) {
+                    *reinterpret_cast<float4*>(dst + c0) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4*>(dst + c0 + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                }
+            }
+        }
+    }
+    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (tid < 32) tmem_dealloc(tmem, 512);
+}
+
+// out[b][i][j] = sum_s partial[s][b][i][j]  (transposed: partial[s][b][j][i]), shares added in index order
+__global__ void wgrad_reduce_kernel(const float* __restrict__ partial, float* __restrict__ out, int nsplit, int transposed) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;   // < 64 * 4096
+    const int b = e >> 12, i = (e >> 6) & 63, j = e & 63;
+    const int src = transposed ? (b << 12) + (j << 6) + i : e;
+    float acc = 0.f;
+    for (int s = 0; s < nsplit; ++s) acc += partial[(size_t)s * (64 * 4096) + src];
+    out[e] = acc;
+}
+
+int64_t wgrad_workspace_bytes(const m2_plan* pl, int64_t T) {
+    return covered(pl) ? workspace_bytes(pl, T) + (int64_t)kWgPartialBytes + 64 * 4096 * 2 : 0;
+}
+
+int32_t wgrad(const m2_plan* pl, const void* X, const void* G, const void* L, const void* R, float* dL, float* dR, int64_t T, void* ws,
+              cudaStream_t stream) {
+    if (!covered(pl)) return M2_ERR_UNSUPPORTED;
+    const int units = (int)(2 * ((T + kTileT - 1) / kTileT));
+    const int nsplit = units < kWgSplits ? units : kWgSplits;
+    unsigned char* zws = static_cast<unsigned char*>(ws);
+    float* partial = reinterpret_cast<float*>(zws + workspace_bytes(pl, T));
+    __nv_bfloat16* Lt = reinterpret_cast<__nv_bfloat16*>(zws + workspace_bytes(pl, T) + kWgPartialBytes);
+    if (T == 0) {
+        wgrad_reduce_kernel<<<1024, 256, 0, stream>>>(partial, dL, 0, 0);
+        wgrad_reduce_kernel<<<1024, 256, 0, stream>>>(partial, dR, 0, 0);
+        pl->launches += 2;
+        return cudaGetLastError() == cudaSuccess ? M2_OK : M2_ERR_CUDA;
+    }
+    alignas(64) CUtensorMap unused;
+    memset(&unused, 0, sizeof(unused));   // pass 1 never touches its map
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t p1 = {};
+    p1.gridDim = dim3(8, (unsigned)((T + kTileT - 1) / kTileT));
+    p1.blockDim = dim3(kThreads);
+    p1.dynamicSmemBytes = SMEM_BYTES;
+    p1.stream = stream;
+    p1.attrs = attr;
+    p1.numAttrs = 1;
+    cudaLaunchConfig_t wg = p1;
+    wg.gridDim = dim3(8, (unsigned)nsplit);
+    wg.dynamicSmemBytes = WG_SMEM;
+    const __nv_bfloat16 *x = (const __nv_bfloat16*)X, *g = (const __nv_bfloat16*)G;
+    // dL: v = R-stage of x, then sum_t v (x) g per block k1
+    if (cudaLaunchKernelEx(&p1, monarch64_pass_kernel<1>, x, (const __nv_bfloat16*)R, unused, (__nv_bfloat16*)zws, (long long)T, pl->d_status,
+                           (const __nv_bfloat16*)nullptr, 1LL, 0) != cudaSuccess)
+        return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&wg, monarch64_wgrad_kernel, g, (const __nv_bfloat16*)zws, partial, (long long)T, units, pl->d_status) != cudaSuccess)
+        return M2_ERR_CUDA;
+    wgrad_reduce_kernel<<<1024, 256, 0, stream>>>(partial, dL, nsplit, 1);
+    // dR: dv = L^T-stage of g, then sum_t dv (x) x per block n2
+    if (m2g::launch_blocks_transpose(L, Lt, 64, 64, 64, true, stream) != cudaSuccess) return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&p1, monarch64_pass_kernel<1>, g, (const __nv_bfloat16*)Lt, unused, (__nv_bfloat16*)zws, (long long)T, pl->d_status,
+                           (const __nv_bfloat16*)nullptr, 1LL, 0) != cudaSuccess)
+        return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&wg, monarch64_wgrad_kernel, x, (const __nv_bfloat16*)zws, partial, (long long)T, units, pl->d_status) != cudaSuccess)
+        return M2_ERR_CUDA;
+    wgrad_reduce_kernel<<<1024, 256, 0, stream>>>(partial, dR, nsplit, 0);
+    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    pl->last_kernel = "matmul_wgrad_umma_64x64";
+    pl->launches += 7;
+    return M2_OK;
+}
+
 bool covered(const m2_plan* pl) { return pl->dtype == M2_BF16 && pl->p == 2 && pl->dims[0] == 64 && pl->dims[1] == 64; }
 
 // whole token tiles: the last tile's slab is written in full
@@ -228,6 +430,7 @@ cudaError_t prepare(const m2_plan* pl) {
     if (!covered(pl)) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(monarch64_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM);
     return e;
 }
 

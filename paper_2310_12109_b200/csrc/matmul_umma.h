@@ -12,4 +12,8 @@ cudaError_t prepare(const m2_plan* plan);
 // Kmul != nullptr: Y = sigma(K (.) M X) with K [Hk][4096] bf16, row t uses K[t % Hk], sigma = ReLU if relu else identity
 int32_t matmul(const m2_plan* plan, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
                int64_t Hk, int relu, cudaStream_t stream);
+// gradients with respect to L and R on the tensor cores (fp32 results, bf16 intermediate); ws: wgrad_workspace_bytes
+int64_t wgrad_workspace_bytes(const m2_plan* plan, int64_t T);
+int32_t wgrad(const m2_plan* plan, const void* X, const void* G, const void* L, const void* R, float* dL, float* dR, int64_t T, void* ws,
+              cudaStream_t stream);
 }  // namespace m2mm

@@ -100,11 +100,17 @@ int32_t m2_spectrum_conjugate(const m2_plan* plan, const void* kf_in_dev, int64_
 /* Gradient with respect to the kernel: for an upstream gradient g of y,
  *   dk[h][u] = sum_b sum_t g[b][h][t] x[b][h][t - u]  =  M^-1 ( sum_b conj(M pad(x_b)) (.) M pad(g_b) ) [0:n)
  * (the convolution of Eq. 2 is linear in k; indices mod N for M2_CIRCULAR, t >= u for M2_CAUSAL).
- * x_dev, g_dev: [B, H, n] in the plan dtype; dk_dev: [H, n] float32.  Runs on the CUDA cores in fp32, one thread
- * block per channel; M2_ERR_UNSUPPORTED for N above 8192.  (The paper trains through the operator, Sec. 5, without
- * writing the backward pass out.) */
+ * x_dev, g_dev: [B, H, n] in the plan dtype; dk_dev: [H, n] float32.
+ * ws_dev: optional caller-owned workspace of m2_conv_bwd_workspace_bytes(plan, B, H) bytes (16-byte aligned; 0 bytes
+ * means this plan has no kernel that uses one).  With it, plans the tensor-core path covers (bf16, N = 512 = 32 x 16)
+ * run both forward transforms and the products conj(M x) (.) M g on the tensor cores (intermediates rounded to bf16
+ * like the forward pass), 8 batch rows at a time, and a CUDA-core kernel adds the groups in order and applies M^-1 in
+ * fp32.  Without it everything runs on the CUDA cores in fp32, one thread block per channel (N up to 8192, else
+ * M2_ERR_UNSUPPORTED).  Both are deterministic.  (The paper trains through the operator, Sec. 5, without writing the
+ * backward pass out.) */
+int64_t m2_conv_bwd_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H);
 int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const void* g_dev, float* dk_dev, int64_t B,
-                                   int64_t H, int64_t n, int32_t mode, void* stream);
+                                   int64_t H, int64_t n, int32_t mode, void* ws_dev, int64_t ws_bytes, void* stream);
 
 /* y = Re( M^-1 ( k_f (.) M pad(x) ) )[0:n)  (Eq. 2 with M_1 = F, M_2 = F^-1; App. D.3).
  * x_dev, y_dev: [B, H, n] in the plan dtype; kf_dev from m2_kernel_spectrum with the same H.

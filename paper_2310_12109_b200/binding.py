@@ -39,7 +39,8 @@ SIGNATURES = {
     "m2_layer_scratch_bytes": (_i64, [_vp, _vp, _i64]),
     "m2_layer_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
-    "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
+    "m2_conv_bwd_workspace_bytes": (_i64, [_vp, _i64, _i64]),
+    "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]),
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
@@ -158,14 +159,19 @@ def m2_spectrum_conjugate(plan: Plan, kf: torch.Tensor, H: int, out: torch.Tenso
     return out
 
 
-def m2_monarch_conv_bwd_kernel(plan: Plan, x: torch.Tensor, g: torch.Tensor, mode: int) -> torch.Tensor:
-    """dk[H, n] (float32): gradient of sum_b <conv(k, x_b), g_b> with respect to the kernel; x, g: [B, H, n]."""
+def m2_monarch_conv_bwd_kernel(plan: Plan, x: torch.Tensor, g: torch.Tensor, mode: int, ws: torch.Tensor | None = None,
+                               use_workspace: bool = True) -> torch.Tensor:
+    """dk[H, n] (float32): gradient of sum_b <conv(k, x_b), g_b> with respect to the kernel; x, g: [B, H, n].
+    use_workspace=False selects the fp32 CUDA-core kernel even where a tensor-core one exists."""
     assert x.is_cuda and g.is_cuda and x.dtype == plan.torch_dtype and g.dtype == plan.torch_dtype
     assert x.is_contiguous() and g.is_contiguous() and x.shape == g.shape and x.dim() == 3
     B, H, n = x.shape
     dk = torch.empty((H, n), dtype=torch.float32, device=x.device)
-    _check(lib().m2_monarch_conv_bwd_kernel(plan.handle, _ptr(x), _ptr(g), _ptr(dk), B, H, n, mode, _stream()),
-           "m2_monarch_conv_bwd_kernel")
+    if ws is None and use_workspace:
+        need = int(lib().m2_conv_bwd_workspace_bytes(plan.handle, B, H))
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device) if need > 0 else None
+    _check(lib().m2_monarch_conv_bwd_kernel(plan.handle, _ptr(x), _ptr(g), _ptr(dk), B, H, n, mode, _ptr(ws),
+                                            0 if ws is None else ws.numel(), _stream()), "m2_monarch_conv_bwd_kernel")
     return dk
 
 

@@ -405,6 +405,222 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     if (threadIdx.x < 32) tmem_dealloc(tmem_cta, kTmemCols);
 }
 
+// ---- gradient with respect to the kernel k ---------------------------------------------------------------------------
+//
+//   dk[h] = M^-1 ( sum_b conj(M x_b) (.) M g_b ) [0:n)          (the transpose of Eq. 2 with respect to k)
+//
+// The forward half of the pipeline above (S1, twiddle, S2) runs on the x tile and on the g tile of a unit (8 batch
+// entries of one channel) side by side: 128 TMEM columns per pipeline, 4 pipelines per CTA.  Each thread then holds the
+// two spectra of its rows at the same (k1, k2), forms conj(X) G in fp32, adds its two rows, the four warps' sums are
+// added through shared memory, and the unit's [k1][k2] sum goes to partial[b group][h] in plan order.  A CUDA-core
+// kernel adds the b groups in order and applies M^-1 in fp32 (one block per channel).
+constexpr int kGroupsW = 4;
+constexpr int kThreadsW = 128 * kGroupsW;
+constexpr int WG_X = 0;              // x tile 8192 | g tile 8192 (2 boxes [n2hi][r][n1][8] each)
+constexpr int WG_A = 16384;          // A2 of x 16384 | A2 of g 16384; afterwards the four warps' sums [warp][k2][33 k1] float2
+constexpr int W_GROUP_BYTES = 49152;
+constexpr int W_SMEM_BYTES = OFF_GROUP + kGroupsW * W_GROUP_BYTES;
+static_assert(W_SMEM_BYTES <= 232448 && 4 * 16 * 33 * 8 <= 32768, "per-CTA budgets");
+
+__global__ void __launch_bounds__(kThreadsW, 1)
+convwgrad512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_g, float2* __restrict__ partial,
+                    const uint4* __restrict__ consts, int B, int H, int n, int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem_all[];
+    const int wg = threadIdx.x >> 7, tid = threadIdx.x & 127, warp = tid >> 5;
+    const bool leader = tid == 32 * (wg & 3);
+    const uint32_t s_all = smem_u32(smem_all);
+    unsigned char* smem = smem_all + OFF_GROUP + wg * W_GROUP_BYTES;
+    const uint32_t s_base = s_all + OFF_GROUP + wg * W_GROUP_BYTES;
+    const uint32_t bar_x = s_all + OFF_BAR + wg * 32, bar_mma = bar_x + 8;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_all + OFF_BAR + wg * 32 + 24);
+    const uint32_t s_tptr = s_all + OFF_BAR + 512;
+    const int bgroups = (B + kRows - 1) / kRows;
+    const int units = H * bgroups;
+    const int ustride = gridDim.x * kGroupsW;
+    int u = blockIdx.x * kGroupsW + wg;
+    if (leader) {
+        mbar_init(bar_x, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_g);
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    {
+        uint4* dst = reinterpret_cast<uint4*>(smem_all + OFF_CONST);
+        for (int i = threadIdx.x; i < CONST_BYTES / 16; i += kThreadsW) dst[i] = consts[i];
+    }
+    if (threadIdx.x < 32) tmem_alloc(s_tptr, kTmemCols);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    bool x_pending = false;
+    auto load_unit = [&](int v) {   // both tiles of unit v, one barrier phase
+        mbar_expect_tx(bar_x, 16384);
+        const int hh = v % H, bb = (v / H) * kRows;
+        tma_load_4d(s_base + WG_X, &map_x, 0, 0, hh, bb, bar_x);
+        tma_load_4d(s_base + WG_X + 4096, &map_x, 8, 0, hh, bb, bar_x);
+        tma_load_4d(s_base + WG_X + 8192, &map_g, 0, 0, hh, bb, bar_x);
+        tma_load_4d(s_base + WG_X + 12288, &map_g, 8, 0, hh, bb, bar_x);
+        x_pending = true;
+    };
+    if (leader && u < units) load_unit(u);
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_cta = *reinterpret_cast<volatile uint32_t*>(smem_all + OFF_BAR + 512);
+    const uint32_t tmem = tmem_cta + wg * 128;
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
+    constexpr uint32_t ID_S2 = instr_desc_bf16(128, 32, true, false);
+    const int k1steps = (n / 16 + 15) / 16;
+    uint32_t ph_x = 0, ph_m = 0;
+    bool ok = true, aborted = false;
+    while (u < units) {
+        const int h = u % H, bg = u / H;
+        const int un = u + ustride;
+        // ---- S1 on both tiles -----------------------------------------------------------------------
+        if (leader) {
+            ok = mbar_wait(bar_x, ph_x);
+            x_pending = false;
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int tt = 0; tt < 2; ++tt)
+#pragma unroll 1
+                    for (int s = 0; s < k1steps; ++s)
+                        umma_f16(tmem + 64 * tt, smem_desc(s_base + WG_X + tt * 8192 + s * 256, 128, 512),
+                                 smem_desc(s_all + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
+                umma_commit(bar_mma);
+            }
+        }
+        ph_x ^= 1;
+        ok = ok && mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (leader && ok && un < units) load_unit(un);   // the tiles are free
+        // ---- h1: twiddle, A2 of x and of g ---------------------------------------------------------------
+        if (ok) {
+            const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
+            const float4* twA = reinterpret_cast<const float4*>(smem_all + OFF_TWA) + n2;
+#pragma unroll 1
+            for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    float re[16], im[16];
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        tmem_ld8(t_lane + 64 * tt + 16 * hh + 8 * jj, re + 8 * jj);
+                        tmem_ld8(t_lane + 64 * tt + 32 + 16 * hh + 8 * jj, im + 8 * jj);
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        tmem_ld_fence8(re + 8 * jj);
+                        tmem_ld_fence8(im + 8 * jj);
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int j = 2 * hh + jj;
+                        float4 w[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) w[q] = twA[(4 * j + q) * 16];
+                        uint4 pr, pi;
+                        cmul_pack8(re + 8 * jj, im + 8 * jj, w, pr, pi);
+                        unsigned char* base = smem + WG_A + tt * 16384 + (r * 4 + j) * 512 + n2lo * 16;
+                        *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = pr;
+                        *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = pi;
+                    }
+                }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (group_sync_or(wg, !ok, abort_flag)) {
+            aborted = true;
+            break;
+        }
+        // ---- S2 on both ---------------------------------------------------------------------------------
+        if (leader) {
+            tc_fence_after();
+#pragma unroll
+            for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                    for (int s = 0; s < 2; ++s)
+                        umma_f16(tmem + 64 * tt + hf * 32, smem_desc(s_base + WG_A + tt * 16384 + hf * 8192 + s * 256, 128, 512),
+                                 smem_desc(s_all + OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+            umma_commit(bar_mma);
+        }
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        // ---- conj(X) G, summed over this thread's two rows, then over the four warps ------------------------------
+        float2* red = reinterpret_cast<float2*>(smem + WG_A);   // [warp][k2][33]: both A2 buffers are free now
+        if (ok) {
+            const int k1 = tid & 31;
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                float sr[8], si[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) sr[q] = si[q] = 0.f;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    float xr[8], xi[8], gr[8], gi[8];
+                    tmem_ld8(t_lane + hf * 32 + 8 * g, xr);
+                    tmem_ld8(t_lane + hf * 32 + 16 + 8 * g, xi);
+                    tmem_ld8(t_lane + 64 + hf * 32 + 8 * g, gr);
+                    tmem_ld8(t_lane + 64 + hf * 32 + 16 + 8 * g, gi);
+                    tmem_ld_wait();
+                    tmem_ld_fence8(xr);
+                    tmem_ld_fence8(xi);
+                    tmem_ld_fence8(gr);
+                    tmem_ld_fence8(gi);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        sr[q] = fmaf(xr[q], gr[q], fmaf(xi[q], gi[q], sr[q]));
+                        si[q] = fmaf(xr[q], gi[q], fmaf(-xi[q], gr[q], si[q]));
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) red[(warp * 16 + 8 * g + q) * 33 + k1] = make_float2(sr[q], si[q]);
+            }
+        }
+        tc_fence_before();
+        if (group_sync_or(wg, !ok, abort_flag)) {
+            aborted = true;
+            break;
+        }
+        {
+            float2* dst = partial + ((size_t)bg * H + h) * 512;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int p = tid + 128 * i, k1 = p >> 4, k2 = p & 15;   // plan order
+                float2 a = red[(0 * 16 + k2) * 33 + k1];
+#pragma unroll
+                for (int w = 1; w < 4; ++w) {
+                    const float2 b = red[(w * 16 + k2) * 33 + k1];
+                    a.x += b.x;
+                    a.y += b.y;
+                }
+                dst[p] = a;
+            }
+        }
+        if (group_sync_or(wg, false, abort_flag)) {   // the sums are read: the next unit's h1 may overwrite them
+            aborted = true;
+            break;
+        }
+        u = un;
+    }
+    if (leader) {
+        if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+        if (x_pending) mbar_wait(bar_x, ph_x);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(tmem_cta, kTmemCols);
+}
+
 // spectrum re-layout for this kernel: kfu[h][k2/2][k1] = (re(k2 even), re(k2 odd), im(even), im(odd)) from plan order
 __global__ void relayout_spectrum_kernel(const float2* __restrict__ kf, float4* __restrict__ kfu, long long total) {
     const long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 8 * 32
@@ -495,6 +711,7 @@ cudaError_t create_tables(m2_plan* pl) {
     if (e == cudaSuccess) e = cudaMalloc(&t->d_sched, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(t->d_sched, 0, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(convwgrad512_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, W_SMEM_BYTES);
     if (e != cudaSuccess) {
         if (t->d_const) cudaFree(t->d_const);
         if (t->d_sched) cudaFree(t->d_sched);
@@ -553,6 +770,41 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
                            pl->d_status, t->d_sched) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o2_512";
+    pl->launches += 1;
+    return M2_OK;
+}
+
+int64_t conv_wgrad_workspace_bytes(const m2_plan* pl, int64_t B, int64_t H) {
+    return pl->umma && covered(pl) ? ((B + kRows - 1) / kRows) * H * 512 * 8 : 0;
+}
+
+// partial[b group][h][512] (plan order) = sum over the group's rows of conj(M x) (.) M g; returns the number of b groups in *parts
+int32_t conv_wgrad_partials(const m2_plan* pl, const void* x, const void* g, void* partial, int64_t B, int64_t H, int64_t n, int32_t mode,
+                            int* parts, cudaStream_t stream) {
+    if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
+    Tables* t = reinterpret_cast<Tables*>(pl->umma);
+    alignas(64) CUtensorMap mx, mg;
+    if (!make_map(&mx, x, B, H, n) || !make_map(&mg, g, B, H, n)) return M2_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long bgroups = (B + kRows - 1) / kRows, units = H * bgroups;
+    const long long ctas = (units + kGroupsW - 1) / kGroupsW;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(ctas < sms ? ctas : sms));
+    cfg.blockDim = dim3(kThreadsW);
+    cfg.dynamicSmemBytes = W_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, convwgrad512_kernel, mx, mg, (float2*)partial, (const uint4*)t->d_const, (int)B, (int)H, (int)n,
+                           pl->d_status) != cudaSuccess)
+        return M2_ERR_CUDA;
+    *parts = (int)bgroups;
     pl->launches += 1;
     return M2_OK;
 }

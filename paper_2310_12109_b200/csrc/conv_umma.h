@@ -15,6 +15,12 @@ void destroy_tables(m2_plan* plan);
 int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
                  int32_t mode, cudaStream_t stream);
 
+// Kernel gradient, tensor-core part: partial[b group][h][512] = sum over the group's 8 rows of conj(M x) (.) M g in plan
+// order (complex fp32, conv_wgrad_workspace_bytes(plan, B, H) bytes); *parts = number of b groups.
+int64_t conv_wgrad_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H);
+int32_t conv_wgrad_partials(const m2_plan* plan, const void* x, const void* g, void* partial, int64_t B, int64_t H, int64_t n,
+                            int32_t mode, int* parts, cudaStream_t stream);
+
 }  // namespace m2u
 
 // Order-3 kernel for N = 32768 = 32^3, causal n = 16384 (conv_umma3.cu); same contract as m2u.

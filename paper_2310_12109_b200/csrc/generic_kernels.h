@@ -40,6 +40,8 @@ cudaError_t launch_transpose_any(const void* in, void* out, long long B, int R, 
 // y[row] = LayerNorm(a[row] + b[row]) * gamma + beta over d values (y may alias a or b)
 cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamma, const float* beta, void* y, long long rows, int d,
                                  float eps, bool bf16, cudaStream_t st);
+// dk[h] = Re M^-1(sum_p partial[p][h][:])[0:n) / N with partial [parts][H][N] complex fp32 in plan order
+cudaError_t launch_spectrum_sum_inverse(const ConvShape& s, const void* partial, int parts, float* dk, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -237,8 +237,13 @@ int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t 
     return M2_OK;
 }
 
+int64_t m2_conv_bwd_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H) {
+    if (!plan || B < 0 || H < 0) return -1;
+    return m2u::conv_wgrad_workspace_bytes(plan, B, H);
+}
+
 int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const void* g_dev, float* dk_dev, int64_t B, int64_t H,
-                                   int64_t n, int32_t mode, void* stream) {
+                                   int64_t n, int32_t mode, void* ws_dev, int64_t ws_bytes, void* stream) {
     // same argument rules as the forward call (dk plays the part of the output for the null / alignment checks)
     int32_t st = check_conv_args(plan, x_dev, g_dev, dk_dev, B, H, n, mode);
     if (st != M2_OK) return st;
@@ -246,7 +251,20 @@ int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
     if (H == 0) return M2_OK;
+    if (ws_dev && !aligned16(ws_dev)) return M2_ERR_ALIGNMENT;
     m2g::ConvShape s = conv_shape(plan, B, H, n);
+    const int64_t need = m2u::conv_wgrad_workspace_bytes(plan, B, H);
+    if (need > 0 && B > 0 && ws_dev && ws_bytes >= need) {   // tensor-core transforms and products, CUDA-core sum + inverse
+        int parts = 0;
+        st = m2u::conv_wgrad_partials(plan, x_dev, g_dev, ws_dev, B, H, n, mode, &parts, (cudaStream_t)stream);
+        if (st == M2_OK) {
+            if (m2g::launch_spectrum_sum_inverse(s, ws_dev, parts, dk_dev, (cudaStream_t)stream) != cudaSuccess) return M2_ERR_CUDA;
+            plan->last_kernel = "conv_wgrad_umma_o2_512";
+            plan->launches += 1;
+            return M2_OK;
+        }
+        if (st != M2_ERR_UNSUPPORTED) return st;
+    }
     const cudaError_t e = m2g::launch_conv_wgrad(s, plan->dtype == M2_BF16, x_dev, g_dev, dk_dev, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;

@@ -301,15 +301,22 @@ def test_conv_input_gradient(cfg, kernel):
     plan.close()
 
 
-@pytest.mark.parametrize("cfg", ["c1", "c2", "c2causal", "small3"])
-def test_conv_kernel_gradient(cfg):
+@pytest.mark.parametrize("cfg,use_ws", [("c1", True), ("c2", False), ("c2", True), ("c2big", True), ("c2causal", True),
+                                        ("c2causal256", True), ("small3", True)])
+def test_conv_kernel_gradient(cfg, use_ws):
     if cfg == "c1":
         c, causal, dtype, tol = synth.config1(), True, M.M2_FP32, 1e-5
     elif cfg == "c2":
         c, causal, dtype, tol = synth.config2(B=8, H=12), False, M.M2_BF16, 1e-5   # bf16 inputs are exact in fp32: fp32 accuracy
-    elif cfg == "c2causal":
+    elif cfg == "c2big":     # several units per pipeline, a ragged last batch group
+        c, causal, dtype, tol = synth.config2(B=19, H=160), False, M.M2_BF16, 1e-5
+    elif cfg == "c2causal":  # n not a multiple of 16: no tensor-core kernel
         c = synth.config2(B=5, H=7)
         c = dict(c, x=c["x"][..., :200].copy(), k=c["k"][..., :200].copy())
+        causal, dtype, tol = True, M.M2_BF16, 1e-5
+    elif cfg == "c2causal256":
+        c = synth.config2(B=5, H=7)
+        c = dict(c, x=c["x"][..., :256].copy(), k=c["k"][..., :256].copy())
         causal, dtype, tol = True, M.M2_BF16, 1e-5
     else:
         c = dict(x=synth.round_bf16(synth.normal(synth.stream_id(9, 0), (3, 4, 32))), dims=(4, 4, 4))
@@ -319,11 +326,12 @@ def test_conv_kernel_gradient(cfg):
     x = c["x"].astype(np.float64)
     gup = synth.round_bf16(synth.normal(synth.stream_id(9, 1), x.shape)).astype(np.float64)   # upstream gradient
     dk = M.m2_monarch_conv_bwd_kernel(plan, dev(x.astype(np.float32), tdt), dev(gup.astype(np.float32), tdt),
-                                      M.M2_CAUSAL if causal else M.M2_CIRCULAR)
+                                      M.M2_CAUSAL if causal else M.M2_CIRCULAR, use_workspace=use_ws)
     torch.cuda.synchronize()
-    assert plan.device_status() == 0 and plan.last_kernel() == "conv_wgrad_generic"
+    umma = use_ws and cfg in ("c2", "c2big", "c2causal256")
+    assert plan.device_status() == 0 and plan.last_kernel() == ("conv_wgrad_umma_o2_512" if umma else "conv_wgrad_generic")
     ref = O.monarch_conv_kernel_grad(x, gup, c["dims"], causal)
-    check(host(dk), ref, tol, "kernel gradient " + cfg)
+    check(host(dk), ref, TOL_BF16 if umma else tol, "kernel gradient " + cfg)   # tensor-core path: bf16 intermediates
     plan.close()
 
 

@@ -29,6 +29,7 @@
 #include <cuda_bf16.h>
 
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -60,6 +61,7 @@ static_assert(kGroups * 32 <= 512 && kGroups * kTmemColsPerGroup <= kTmemCols &&
 
 struct Tables {
     void* d_const = nullptr;  // CONST_BYTES
+    void* d_const_p = nullptr;  // constants of the row-pair kernel
     int* d_sched = nullptr;   // {next unit, pipelines finished}; zero between launches
 };
 
@@ -405,6 +407,335 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     if (threadIdx.x < 32) tmem_dealloc(tmem_cta, kTmemCols);
 }
 
+// ---- the same pipeline on PAIRS of batch rows ------------------------------------------------------------------------
+//
+// k is real, so two batch rows of one channel ride as the real and the imaginary part of one complex row:
+// F^-1(k_f (.) F(xa + i xb)) = ya + i yb.  A unit is then 16 batch rows = 8 complex rows: the first stage contracts
+// K = (re | im) x n1 = 64 and the last one produces both parts (N = 64), everything between is unchanged, so the three
+// fp32 hand-offs between the stages are paid once per two rows.  6 pipelines of 32 KB (the spectrum values come straight
+// from global memory / L2, requested before the accumulator wait).
+constexpr int kGroupsP = 6;
+constexpr int kThreadsP = 128 * kGroupsP;
+constexpr int P_OFF_B1 = 0, P_OFF_B2 = 8192, P_OFF_B3 = 10240, P_OFF_B4 = 12288, P_OFF_TWA = 20480, P_OFF_TWB = 24576;
+constexpr int P_CONST_BYTES = 28672;
+constexpr int P_OFF_BAR = P_CONST_BYTES;          // per group 32 B; tmem ptr at +512
+constexpr int P_OFF_GROUP = P_OFF_BAR + 1024;
+constexpr int P_G_X = 0;                          // re tile 8192 | im tile 8192 (2 boxes [n2hi][r][n1][8] each)
+constexpr int P_G_A = 16384;                      // A2 / A3 / A4   16384
+constexpr int P_GROUP_BYTES = 32768;
+constexpr int P_SMEM_BYTES = P_OFF_GROUP + kGroupsP * P_GROUP_BYTES;
+static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols && P_SMEM_BYTES <= 232448 && P_OFF_GROUP % 1024 == 0,
+              "per-CTA budgets");
+
+__global__ void __launch_bounds__(kThreadsP, 1)
+conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restrict__ y,
+               const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
+               int32_t* __restrict__ status, int* __restrict__ sched) {
+    extern __shared__ __align__(1024) unsigned char smem_all[];
+    const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
+    const int tid = threadIdx.x & 127;
+    const int warp = tid >> 5;                // warp within the group = TMEM lane quarter
+    // the thread that issues this pipeline's UMMAs and copies; its warp differs from group to group so that
+    // the extra work spreads over the SM's four schedulers
+    const bool leader = tid == 32 * (wg & 3);
+    const uint32_t s_all = smem_u32(smem_all);
+    unsigned char* smem = smem_all + P_OFF_GROUP + wg * P_GROUP_BYTES;   // this group's slice
+    const uint32_t s_base = s_all + P_OFF_GROUP + wg * P_GROUP_BYTES;
+    const uint32_t bar_x = s_all + P_OFF_BAR + wg * 32, bar_mma = bar_x + 8;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_all + P_OFF_BAR + wg * 32 + 24);
+    volatile int* next_slot = reinterpret_cast<volatile int*>(smem_all + P_OFF_BAR + wg * 32 + 28);
+    const uint32_t s_tptr = s_all + P_OFF_BAR + 512;
+
+    const int bgroups0 = (B + 2 * kRows - 1) / (2 * kRows);   // 16 batch rows = 8 complex rows per unit
+    const int units0 = H * bgroups0;
+    // pipeline-major numbering: a partial last round of units spreads over all CTAs instead of filling the first ones
+    int u = wg * gridDim.x + blockIdx.x;
+    const int ustride = gridDim.x * kGroupsP;
+    if (leader) {
+        mbar_init(bar_x, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_x);
+    }
+    // Programmatic dependent launch: the next kernel on the stream may start its CTAs as this grid's CTAs leave
+    // their SMs; everything above the wait below touches only plan-owned constants and this CTA's own resources.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool x_pending = false;
+    // constants -> shared memory
+    {
+        uint4* dst = reinterpret_cast<uint4*>(smem_all);
+        for (int i = threadIdx.x; i < P_CONST_BYTES / 16; i += kThreadsP) dst[i] = consts[i];
+    }
+    if (threadIdx.x < 32) tmem_alloc(s_tptr, kTmemCols);
+    // everything the stream ran before this kernel (the producer of x and of the spectrum, the previous launch's
+    // reset of the scheduler words, readers of y) is complete and visible from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // rows b0 .. b0+7 are the real parts and rows b0+8 .. b0+15 the imaginary parts of the unit's 8 complex rows (boxes
+    // past the end of the batch read zeros)
+    auto load_unit = [&](int v) {
+        mbar_expect_tx(bar_x, 16384);
+        const int hh = v % H, bb = (v / H) * 2 * kRows;
+        tma_load_4d(s_base + P_G_X, &map_x, 0, 0, hh, bb, bar_x);
+        tma_load_4d(s_base + P_G_X + 4096, &map_x, 8, 0, hh, bb, bar_x);
+        tma_load_4d(s_base + P_G_X + 8192, &map_x, 0, 0, hh, bb + kRows, bar_x);
+        tma_load_4d(s_base + P_G_X + 12288, &map_x, 8, 0, hh, bb + kRows, bar_x);
+        x_pending = true;
+    };
+    if (leader && u < units0) {   // first loads
+        load_unit(u);
+    }
+    fence_proxy_async();   // the constant matrices are read by the async proxy (UMMA)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_cta = *reinterpret_cast<volatile uint32_t*>(smem_all + P_OFF_BAR + 512);
+    const uint32_t tmem = tmem_cta + wg * kTmemColsPerGroup;
+    const float4* kfu_k1 = kfu + (threadIdx.x & 31);
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
+    const uint32_t T1 = 0, T2 = 0;   // every stage's accumulator reuses the same 64 columns
+
+    const int units = units0;
+    constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
+    constexpr uint32_t ID_S2 = instr_desc_bf16(128, 32, true, false);
+    constexpr uint32_t ID_S2I = instr_desc_bf16(128, 32, false, false);
+    constexpr uint32_t ID_S1I = instr_desc_bf16(128, 64, true, false);
+    const int n1_valid = n / 16;
+    const int k1steps = (n1_valid + 15) / 16;   // causal input: digits n1 >= n/16 are zero -> skipped
+
+    uint32_t ph_x = 0, ph_m = 0;
+    bool ok = true, aborted = false;
+    // Units beyond the first two are handed out by a device-wide counter (sched[0]): pipelines that finish early take more.
+    // The last pipeline to leave (sched[1] counts them) zeroes both words for the next launch on this plan.
+    int un = u + ustride;   // the second unit is static too
+    int un2 = units;        // thread 0: the unit after next, claimed one whole unit ahead so the atomic's latency is never waited for
+    while (u < units) {
+        const int h = u % H;
+        const int b0 = (u / H) * 2 * kRows;
+        // ---- S1 ---------------------------------------------------------------------------------
+        if (leader) {
+            ok = mbar_wait(bar_x, ph_x);
+            x_pending = false;
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < 2; ++c)   // K = (re | im part of the input) x n1
+#pragma unroll 1
+                    for (int s = 0; s < k1steps; ++s)
+                        umma_f16(tmem + T1, smem_desc(s_base + P_G_X + c * 8192 + s * 256, 128, 512),
+                                 smem_desc(s_all + P_OFF_B1 + (2 * c + s) * 256, 128, 1024), ID_S1, (c | s) > 0);
+                umma_commit(bar_mma);
+            }
+        }
+        ph_x ^= 1;
+        // ---- h1: twiddle, A2 ---------------------------------------------------------------------
+        ok = ok && mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (leader) un2 = 2 * ustride + atomicAdd(sched, 1);   // consumed at the end of this unit
+        if (leader && ok && un < units) {   // the x tile is free: fetch the next unit's
+            load_unit(un);
+        }
+        if (ok) {
+            const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
+            const float4* twA = reinterpret_cast<const float4*>(smem_all + P_OFF_TWA) + n2;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {   // two batches of 16 complex values keep the register count down
+                float re[16], im[16];
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    tmem_ld8(t_lane + T1 + 16 * hh + 8 * jj, re + 8 * jj);
+                    tmem_ld8(t_lane + T1 + 32 + 16 * hh + 8 * jj, im + 8 * jj);
+                }
+                tmem_ld_wait();
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    tmem_ld_fence8(re + 8 * jj);
+                    tmem_ld_fence8(im + 8 * jj);
+                }
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int j = 2 * hh + jj;
+                    float4 w[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) w[q] = twA[(4 * j + q) * 16];
+                    uint4 pr, pi;
+                    cmul_pack8(re + 8 * jj, im + 8 * jj, w, pr, pi);
+                    unsigned char* base = smem + P_G_A + (r * 4 + j) * 512 + n2lo * 16;
+                    *reinterpret_cast<uint4*>(base + (0 + n2hi) * 128) = pr;
+                    *reinterpret_cast<uint4*>(base + (2 + n2hi) * 128) = pi;
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (group_sync_or(wg, !ok, abort_flag)) {
+            aborted = true;
+            break;
+        }
+        // ---- S2 ---------------------------------------------------------------------------------
+        if (leader) {
+            tc_fence_after();
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int s = 0; s < 2; ++s)
+                    umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 512),
+                             smem_desc(s_all + P_OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+            umma_commit(bar_mma);
+        }
+        // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
+        float4 kw[8];   // this thread's 16 spectrum values (k1 fixed), requested before the accumulator is waited for
+#pragma unroll
+        for (int q = 0; q < 8; ++q) kw[q] = __ldg(kfu_k1 + (size_t)h * 256 + q * 32);
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (ok) {
+            // both row halves (hf) of a thread share k1, hence the spectrum values
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                float re[16], im[16];
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld8(t_lane + T2 + hf * 32 + 8 * g, re + 8 * hf);
+                    tmem_ld8(t_lane + T2 + hf * 32 + 16 + 8 * g, im + 8 * hf);
+                }
+                float4 w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = kw[g * 4 + q];
+                tmem_ld_wait();
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld_fence8(re + 8 * hf);
+                    tmem_ld_fence8(im + 8 * hf);
+                }
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int m = hf * 128 + tid;
+                    unsigned char* rowp = smem + P_G_A + (m >> 3) * 512 + (m & 7) * 16;
+                    uint4 pr, pi;
+                    cmul_pack8(re + 8 * hf, im + 8 * hf, w, pr, pi);
+                    *reinterpret_cast<uint4*>(rowp + g * 128) = pr;
+                    *reinterpret_cast<uint4*>(rowp + (2 + g) * 128) = pi;
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (group_sync_or(wg, !ok, abort_flag)) {
+            aborted = true;
+            break;
+        }
+        // ---- S2' --------------------------------------------------------------------------------
+        if (leader) {
+            tc_fence_after();
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int s = 0; s < 2; ++s)
+                    umma_f16(tmem + T1 + hf * 32, smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 512),
+                             smem_desc(s_all + P_OFF_B3 + s * 256, 128, 512), ID_S2I, s > 0);
+            umma_commit(bar_mma);
+        }
+        // ---- h3: conjugate twiddle, A4 --------------------------------------------------------------
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (ok) {
+            const int k1 = tid & 31;
+            const float4* twB = reinterpret_cast<const float4*>(smem_all + P_OFF_TWB) + k1;
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {   // the twiddles depend on (k1, n2) only: shared by both row halves
+                float re[16], im[16];
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld8(t_lane + T1 + hf * 32 + 8 * g, re + 8 * hf);
+                    tmem_ld8(t_lane + T1 + hf * 32 + 16 + 8 * g, im + 8 * hf);
+                }
+                float4 w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = twB[(4 * g + q) * 32];
+                tmem_ld_wait();
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld_fence8(re + 8 * hf);
+                    tmem_ld_fence8(im + 8 * hf);
+                }
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int r = hf * 4 + (tid >> 5);
+                    uint4 pr, pi;
+                    cmul_pack8(re + 8 * hf, im + 8 * hf, w, pr, pi);
+                    unsigned char* base = smem + P_G_A + (r * 2 + g) * 1024 + (k1 >> 3) * 128 + (k1 & 7) * 16;
+                    *reinterpret_cast<uint4*>(base) = pr;
+                    *reinterpret_cast<uint4*>(base + 512) = pi;
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        if (group_sync_or(wg, !ok, abort_flag)) {
+            aborted = true;
+            break;
+        }
+        // ---- S1' --------------------------------------------------------------------------------
+        if (leader) {
+            tc_fence_after();
+#pragma unroll
+            for (int s = 0; s < 4; ++s)
+                umma_f16(tmem + T2, smem_desc(s_base + P_G_A + s * 256, 128, 1024),
+                         smem_desc(s_all + P_OFF_B4 + s * 256, 128, 1024), ID_S1I, s > 0);
+            umma_commit(bar_mma);
+        }
+        // ---- h4: round and store: lane (r, n2) holds y[r][n1*16 + n2] for all n1; a warp writes two full
+        //      32-byte sectors per instruction --------------------------------------------------------
+        ok = mbar_wait(bar_mma, ph_m);
+        ph_m ^= 1;
+        tc_fence_after();
+        if (ok) {
+            const int r = tid >> 4, n2 = tid & 15;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {   // real part: row b0 + r; imaginary part: row b0 + 8 + r
+                float v[32];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) tmem_ld8(t_lane + T2 + 32 * c + 8 * g, v + 8 * g);
+                tmem_ld_wait();
+#pragma unroll
+                for (int g = 0; g < 4; ++g) tmem_ld_fence8(v + 8 * g);
+                if (b0 + kRows * c + r < B) {
+                    __nv_bfloat16* yr = y + ((size_t)(b0 + kRows * c + r) * H + h) * n + n2;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < n1_valid) yr[i * 16] = __float2bfloat16_rn(v[i]);
+                }
+            }
+        }
+        if (leader) *next_slot = un2;
+        tc_fence_before();
+        if (group_sync_or(wg, !ok, abort_flag)) {
+            aborted = true;
+            break;
+        }
+        u = un;
+        un = *next_slot;   // written by thread 0 before the barrier above
+    }
+    // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
+    if (leader) {
+        if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+        if (x_pending) mbar_wait(bar_x, ph_x);
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == ustride - 1) {   // last pipeline out: reset the scheduler words
+            sched[0] = 0;
+            sched[1] = 0;
+            __threadfence();
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_dealloc(tmem_cta, kTmemCols);
+}
+
 // ---- gradient with respect to the kernel k ---------------------------------------------------------------------------
 //
 //   dk[h] = M^-1 ( sum_b conj(M x_b) (.) M g_b ) [0:n)          (the transpose of Eq. 2 with respect to k)
@@ -437,7 +768,7 @@ convwgrad512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     const int bgroups = (B + kRows - 1) / kRows;
     const int units = H * bgroups;
     const int ustride = gridDim.x * kGroupsW;
-    int u = blockIdx.x * kGroupsW + wg;
+    int u = wg * gridDim.x + blockIdx.x;   // pipeline-major: a partial last round spreads over all CTAs
     if (leader) {
         mbar_init(bar_x, 1);
         mbar_init(bar_mma, 1);
@@ -705,8 +1036,30 @@ cudaError_t create_tables(m2_plan* pl) {
     std::memcpy(blob.data() + 8192, B4.data(), 4096);
     std::memcpy(blob.data() + 12288, twA.data(), 4096);
     std::memcpy(blob.data() + 16384, twB.data(), 4096);
+    // row-pair kernel: B1p [N = (c,k1) 64][K = (c',n1) 64] = F32 on complex input; B4p [N = (c',n1) 64][K = (c,k1) 64] = conj(F32)
+    std::vector<uint16_t> B1p(4096), B4p(4096);
+    for (int co = 0; co < 2; ++co)
+        for (int o = 0; o < N1; ++o)
+            for (int ci = 0; ci < 2; ++ci)
+                for (int i = 0; i < N1; ++i) {
+                    const double th = 2.0 * M_PI * ((o * i) % N1) / N1;
+                    const double cs = std::cos(th), sn = sg * std::sin(th);
+                    // (a + ib)(cs + i sn): re = cs a - sn b, im = sn a + cs b;   conjugate: re = cs a + sn b, im = -sn a + cs b
+                    put_kmajor(B1p, 64, co * 32 + o, ci * 32 + i, co == 0 ? (ci == 0 ? cs : -sn) : (ci == 0 ? sn : cs));
+                    put_kmajor(B4p, 64, co * 32 + o, ci * 32 + i, co == 0 ? (ci == 0 ? cs : sn) : (ci == 0 ? -sn : cs));
+                }
+    std::vector<unsigned char> blob_p(P_CONST_BYTES);
+    std::memcpy(blob_p.data() + P_OFF_B1, B1p.data(), 8192);
+    std::memcpy(blob_p.data() + P_OFF_B2, B2.data(), 2048);
+    std::memcpy(blob_p.data() + P_OFF_B3, B3.data(), 2048);
+    std::memcpy(blob_p.data() + P_OFF_B4, B4p.data(), 8192);
+    std::memcpy(blob_p.data() + P_OFF_TWA, twA.data(), 4096);
+    std::memcpy(blob_p.data() + P_OFF_TWB, twB.data(), 4096);
     Tables* t = new Tables();
     cudaError_t e = cudaMalloc(&t->d_const, CONST_BYTES);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_const_p, P_CONST_BYTES);
+    if (e == cudaSuccess) e = cudaMemcpy(t->d_const_p, blob_p.data(), P_CONST_BYTES, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_sched, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(t->d_sched, 0, 2 * sizeof(int));
@@ -714,6 +1067,7 @@ cudaError_t create_tables(m2_plan* pl) {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(convwgrad512_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, W_SMEM_BYTES);
     if (e != cudaSuccess) {
         if (t->d_const) cudaFree(t->d_const);
+        if (t->d_const_p) cudaFree(t->d_const_p);
         if (t->d_sched) cudaFree(t->d_sched);
         delete t;
         return e;
@@ -726,6 +1080,7 @@ void destroy_tables(m2_plan* pl) {
     if (!pl->umma || !covered(pl)) return;
     Tables* t = reinterpret_cast<Tables*>(pl->umma);
     if (t->d_const) cudaFree(t->d_const);
+    if (t->d_const_p) cudaFree(t->d_const_p);
     if (t->d_sched) cudaFree(t->d_sched);
     delete t;
     pl->umma = nullptr;
@@ -739,6 +1094,15 @@ static bool make_map(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, in
     return tma_host::encode_bf16(map, ptr, 4, gdim, gstr, box);
 }
 
+// development switch: M2_CONV512_PAIRS=0 in the environment selects the one-row-per-lane kernel for every batch size
+static bool pair_kernel_enabled() {
+    static const bool on = [] {
+        const char* v = std::getenv("M2_CONV512_PAIRS");
+        return !(v && v[0] == '0');
+    }();
+    return on;
+}
+
 int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
                  cudaStream_t stream) {
     if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
@@ -750,24 +1114,26 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long units = H * ((B + kRows - 1) / kRows);
-    const long long ctas = (units + kGroups - 1) / kGroups;
+    const bool pairs = B > kRows && pair_kernel_enabled();   // two batch rows per complex row once there are more than 8
+    const long long units = pairs ? H * ((B + 2 * kRows - 1) / (2 * kRows)) : H * ((B + kRows - 1) / kRows);
+    const int groups = pairs ? kGroupsP : kGroups;
+    const long long ctas = (units + groups - 1) / groups;
     const int grid = (int)(ctas < sms ? ctas : sms);
     const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * 512 * 8);
     // launched with programmatic stream serialization: its CTAs may take over SMs that the previous kernel's CTAs
     // have left while that kernel's last CTAs still run (the kernel waits for it before touching its data)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.blockDim = dim3(pairs ? kThreadsP : kThreads);
+    cfg.dynamicSmemBytes = pairs ? P_SMEM_BYTES : SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n,
-                           pl->d_status, t->d_sched) != cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, pairs ? conv512p_kernel : conv512_kernel, mx, (__nv_bfloat16*)y, kfu,
+                           (const uint4*)(pairs ? t->d_const_p : t->d_const), (int)B, (int)H, (int)n, pl->d_status, t->d_sched) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o2_512";
     pl->launches += 1;

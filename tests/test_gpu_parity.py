@@ -107,8 +107,8 @@ def test_fp32_conv_sign_minus_matches():
 
 # ---- config 2: bf16 circular, N = 512 = 32 x 16 ----------------------------------------------
 
-@pytest.mark.parametrize("B,H", [(4, 24), (3, 5), (1, 1), (32, 9)])
-def test_config2_small_full_compare(B, H):
+@pytest.mark.parametrize("B,H", [(4, 24), (3, 5), (1, 1), (32, 9), (9, 5), (16, 3), (19, 6), (40, 150)])
+def test_config2_small_full_compare(B, H):   # more than 8 batch rows: the kernel that packs row pairs as complex rows
     c = synth.config2(B=B, H=H)
     y, name = run_conv(c["dims"], c["x"], c["k"], False, M.M2_BF16)
     ref = O.monarch_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64), c["dims"], causal=False)
@@ -127,9 +127,10 @@ def test_config2_full_size():
         check(y[b, h][None], d[None], TOL_BF16 / 2, f"config2 row ({b},{h}) direct")
 
 
-def test_bf16_causal_order2_and_ragged():
-    for n in (256, 100):
-        B, H = 5, 7
+@pytest.mark.parametrize("B", [5, 19])
+def test_bf16_causal_order2_and_ragged(B):
+    for n in (256, 100, 48):
+        H = 7
         x = synth.round_bf16(synth.normal(800 + n, (B, H, n)))
         k = synth.decay_kernel(2, H, n, 0.005, float(np.sqrt(512.0)))
         y, name = run_conv((32, 16), x, k, True, M.M2_BF16)

@@ -178,7 +178,7 @@ def time_launches(fn, n, torch):
     return e0.elapsed_time(e1)
 
 
-def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5", "operator"), reps=None):
+def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5", "operator", "backward"), reps=None):
     """Config 3 (Monarch matmul), config 4 (order-3 causal conv) and config 5 (M2 block forward): time per call,
     throughput and roofline fraction, outside the headline timed region."""
     out = {}
@@ -192,6 +192,46 @@ def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "confi
         out.update(_side_config5(torch, M, synth, peaks, reps, bf))
     if "operator" in which:
         out.update(_side_operator(torch, M, synth, peaks, reps, bf))
+    if "backward" in which:
+        out.update(_side_backward(torch, M, synth, peaks, reps, bf))
+    return out
+
+
+def _side_backward(torch, M, synth, peaks, reps, bf):
+    """Gradient kernels on the config-2 and config-3 shapes: time per call (CUDA events), upstream gradients synthetic."""
+    out = {}
+    c = synth.config2(B=B2, H=H2)
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=torch.cuda.current_device())
+    kf = M.m2_kernel_spectrum(plan, torch.from_numpy(c["k"]).cuda())
+    kfc = M.m2_spectrum_conjugate(plan, kf, H2)
+    x = bf(c["x"])
+    g = bf(synth.round_bf16(synth.normal(synth.stream_id(12, 0), c["x"].shape)))
+    dx = torch.empty_like(x)
+    ws = torch.empty(int(M.lib().m2_conv_bwd_workspace_bytes(plan.handle, B2, H2)), dtype=torch.uint8, device="cuda")
+    f_dx = lambda i: M.m2_monarch_conv_fwd(plan, g, kfc, M.M2_CIRCULAR, y=dx)  # noqa: E731
+    f_dk = lambda i: M.m2_monarch_conv_bwd_kernel(plan, x, g, M.M2_CIRCULAR, ws=ws)  # noqa: E731
+    res = {}
+    for name, f in (("dx", f_dx), ("dk", f_dk)):
+        time_launches(f, 3, torch)
+        res[name + "_ms"] = time_launches(f, reps, torch) / reps
+        res[name + "_kernel"] = plan.last_kernel()
+    out["config2_backward"] = res
+    plan.close()
+    T, b = 16384, 64
+    c = synth.config3(T=T, b=b)
+    plan = M.Plan((b, b), dtype=M.M2_BF16, device=torch.cuda.current_device())
+    L, R, X = bf(c["L"]), bf(c["R"]), bf(c["X"])
+    G = bf(synth.round_bf16(synth.normal(synth.stream_id(12, 1), c["X"].shape)))
+    ws = torch.empty(int(M.lib().m2_matmul_bwd_workspace_bytes(plan.handle, T)), dtype=torch.uint8, device="cuda")
+    f_dX = lambda i: M.m2_monarch_matmul_bwd_input(plan, G, L, R, ws=ws)  # noqa: E731
+    f_dW = lambda i: M.m2_monarch_matmul_bwd_weights(plan, X, G, L, R, ws=ws)  # noqa: E731
+    res = {}
+    for name, f in (("dX", f_dX), ("dL_dR", f_dW)):
+        time_launches(f, 3, torch)
+        res[name + "_ms"] = time_launches(f, reps, torch) / reps
+        res[name + "_kernel"] = plan.last_kernel()
+    out["config3_backward"] = res
+    plan.close()
     return out
 
 
@@ -423,7 +463,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-side", action="store_true", help="skip the config-3 / config-4 side measurements")
     ap.add_argument("--quick", action="store_true", help="fewer repetitions of the side measurements")
-    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5", "operator"],
+    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5", "operator", "backward"],
                     help="run just this side workload (--steps launches after 2 warm-ups) and print its JSON; used for profiling")
     args = ap.parse_args()
     if args.impl == "reference":

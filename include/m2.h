@@ -171,6 +171,19 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
                      float eps, void* y_dev, int64_t B, void* scratch_dev, int64_t scratch_bytes, void* ws_dev,
                      int64_t ws_bytes, void* stream);
 
+/* The Monarch product on matrices whose COLUMNS are the vectors -- Eq. 2's M X with X in R^{N x d} stored row-major, the
+ * layout of the paper's operator benchmark (Table 2: N = 4K .. 256K, block size sqrt(N), 768 columns):
+ *   Y[bt] = sigma(K (.) (M X[bt])),  M = P L P^T R P,  bt < Bt,  sigma = identity or ReLU (M2_ACT_*).
+ * X_dev, Y_dev: [Bt, N, d] in the plan dtype, d contiguous (Y_dev must not overlap X_dev); K_dev: [N, d], shared by the
+ * batch, or NULL (then sigma is not applied either: Y = M X).  L_dev, R_dev as in m2_monarch_matmul.  ws_dev: caller-owned,
+ * at least Bt N d elements of the plan dtype (the intermediate between the two factors), 16-byte aligned.
+ * The M2 operator M_b (K (.) M_a X) is two calls, the first with K, the second without.
+ * With the columns contiguous both factors are batched GEMMs over rows and the stride permutations are strides of TMA
+ * tensor maps: square bf16 plans with blocks of 64, 128, 256 or 512 and d a multiple of 64 run on the tensor cores, two
+ * launches per call; everything else on a CUDA-core kernel (N <= 65535, else M2_ERR_UNSUPPORTED). */
+int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev,
+                        int32_t act, void* Y_dev, int64_t Bt, int64_t d, void* ws_dev, int64_t ws_bytes, void* stream);
+
 /* W_out[b][c][r] = W_in[b][r][c]: block-wise transpose of a block-diagonal factor of nblocks blocks of rows x cols
  * elements of the plan dtype (W_out must not overlap W_in).  It gives the gradient of the Monarch matmul with
  * respect to its input: M^T = P^T R^T P L^T P^T (Sec. 3.1 transposed) is again an order-2 Monarch product, so for an

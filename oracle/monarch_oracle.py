@@ -218,6 +218,17 @@ def monarch_mix(La, Ra, Lb, Rb, K: np.ndarray, x: np.ndarray, act: str = "none")
     return monarch_apply(Lb, Rb, mid)
 
 
+def monarch_cols(L, R, X: np.ndarray, K: np.ndarray | None = None, act: str = "none") -> np.ndarray:
+    """Y = sigma(K (.) M X) for X [.., N, d] whose COLUMNS are the vectors (Eq. 2's M X with X in R^{N x d}); K: [N, d]
+    or None (then no sigma either).  The Monarch apply itself is monarch_apply along axis -2."""
+    Y = np.swapaxes(monarch_apply(L, R, np.swapaxes(X, -1, -2)), -1, -2)
+    if K is not None:
+        Y = K * Y
+        if act == "relu":
+            Y = np.maximum(Y, 0.0)
+    return Y
+
+
 def layer_norm(v: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float = 1e-5) -> np.ndarray:
     """LayerNorm over the last axis: (v - mean) / sqrt(var + eps) * gamma + beta with the biased variance."""
     mu = v.mean(axis=-1, keepdims=True)

@@ -38,6 +38,7 @@ SIGNATURES = {
     "m2_monarch_mix": (_i32, [_vp, _vp, _vp, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_layer_scratch_bytes": (_i64, [_vp, _vp, _i64]),
     "m2_layer_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
+    "m2_monarch_cols": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_conv_bwd_workspace_bytes": (_i64, [_vp, _i64, _i64]),
     "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]),
@@ -266,6 +267,23 @@ def m2_layer_fwd(plan_n: Plan, plan_d: Plan, x: torch.Tensor, factors, n_kernel:
                               _ptr(y), B, _ptr(scratch), scratch.numel(), _ptr(ws), 0 if ws is None else ws.numel(), _stream()),
            "m2_layer_fwd")
     return y
+
+
+def m2_monarch_cols(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tensor, K: torch.Tensor | None = None, act: int = M2_ACT_NONE,
+                    Y: torch.Tensor | None = None, ws: torch.Tensor | None = None) -> torch.Tensor:
+    """Y[bt] = sigma(K (.) M X[bt]) for X [Bt, N, d] (the columns are the vectors); K: [N, d] or None."""
+    for a in (X, L, R) + ((K,) if K is not None else ()):
+        assert a.is_cuda and a.dtype == plan.torch_dtype and a.is_contiguous()
+    assert X.dim() == 3 and X.shape[1] == plan.N
+    Bt, N, d = X.shape
+    assert K is None or tuple(K.shape) == (N, d)
+    if Y is None:
+        Y = torch.empty_like(X)
+    if ws is None:
+        ws = torch.empty_like(X)
+    _check(lib().m2_monarch_cols(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(K), act, _ptr(Y), Bt, d, _ptr(ws),
+                                 ws.numel() * ws.element_size(), _stream()), "m2_monarch_cols")
+    return Y
 
 
 def m2_blocks_transpose(plan: Plan, W: torch.Tensor) -> torch.Tensor:

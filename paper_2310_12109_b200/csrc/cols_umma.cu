@@ -1,0 +1,235 @@
+// Monarch matrix times a matrix whose COLUMNS are the vectors:  Y = sigma(K (.) M X),  X, Y, K: [N][d] row-major,
+// M = P L P^T R P with N = b * b (Sec. 3.1; this is Eq. 2's M X with X in R^{N x d} as the paper writes it, and the layout
+// of its operator benchmark, Table 2: N = 4K .. 256K, block size sqrt(N), d = 768 columns).
+//
+// With the d columns contiguous, both block-diagonal factors are plain batched GEMMs over rows and no element ever has
+// to be transposed:
+//   stage(W, V)[row o*b + j][c] = sum_i W[j][o][i] * V[row(i, j)][c]
+//   z = stage(R, x) with row(i, j) = i*b + j   (block j = n2 reads the rows n1*b + n2: a strided set of rows)
+//   y = stage(L, z) with row(i, j) = j*b + i   (block j = k1 reads the rows k1*b + n2: b consecutive rows)
+// so the stride permutations are nothing but the strides of two TMA tensor maps.  One kernel serves both stages:
+// a CTA computes the tile [128 outputs o][NC columns] of one block j:  A = W[j] rows (K-major, 128B-swizzled TMA boxes
+// of 64 inputs), B = 64 input rows x NC columns (N-major: a row of the operand is a row of V), accumulator in TMEM
+// (M = 128, or 64 when b = 64; N = NC <= 256), K = b walked in chunks of 64 through a two-stage TMA ring; the
+// epilogue applies the optional factor K (.) and ReLU in fp32, rounds to bf16, stages the tile in the swizzled image of
+// the TMA store boxes and stores it to the rows o*b + j.  About 100 KB of shared memory and NC TMEM columns per CTA:
+// two CTAs per SM overlap each other's load, UMMA and epilogue phases.  All waits are bounded.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <cstring>
+
+#include "cols_umma.h"
+#include "ptx_sm100.cuh"
+#include "tma_host.h"
+
+namespace m2c {
+
+using namespace sm100;
+
+constexpr int kThreads = 128;
+constexpr int kStages = 2;
+constexpr int STAGE_BYTES = 49152;          // A chunk [128][64] 16384 | B chunk [64][256] 32768
+constexpr int OFF_BAR = kStages * STAGE_BYTES;   // full[2], empty[2], done, tmem ptr
+constexpr int SMEM_BYTES = OFF_BAR + 64;
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+                 "l"(map), "r"(c0), "r"(c1), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// grid: x = column tile, y = j * otiles + output tile, z = matrix of the batch
+__global__ void __launch_bounds__(kThreads, 2)
+monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_v,
+                          const __grid_constant__ CUtensorMap map_o, const __nv_bfloat16* __restrict__ Kmul, int relu, int b, int d, int nc,
+                          int m, int32_t* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t bar_full = s_base + OFF_BAR, bar_empty = bar_full + 16, bar_done = bar_full + 32, s_tptr = bar_full + 40;
+    const int otiles = (b + 127) / 128;
+    const int c0 = blockIdx.x * nc, j = blockIdx.y / otiles, ot = blockIdx.y % otiles, bt = blockIdx.z;
+    const int chunks = b / 64, nq = nc / 64;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_done, 1);
+        fence_barrier_init();
+        prefetch_tensormap(&map_w);
+        prefetch_tensormap(&map_v);
+        prefetch_tensormap(&map_o);
+    }
+    if (warp == 0) tmem_alloc(s_tptr, (uint32_t)nc);   // 64, 128 or 256 columns
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // V may have been written by the kernel before this one
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 40);
+    bool ok = true;
+
+    if (tid == 0) {
+        const uint32_t stage_tx = (uint32_t)(m * 128 + nq * 8192);
+        auto load = [&](int kc) {
+            const int s = kc & 1;
+            const uint32_t sb = s_base + s * STAGE_BYTES, bf = bar_full + 8 * s;
+            mbar_expect_tx(bf, stage_tx);
+            tma_load_2d(sb, &map_w, kc * 64, j * b + ot * 128, bf);                                      // W[j][o tile][64 inputs]
+            for (int q = 0; q < nq; ++q) tma_load_4d(sb + 16384 + q * 8192, &map_v, c0 + 64 * q, kc * 64, j, bt, bf);   // 64 input rows
+        };
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(nc >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+        for (int kc = 0; kc < kStages && kc < chunks; ++kc) load(kc);
+#pragma unroll 1
+        for (int kc = 0; kc < chunks && ok; ++kc) {
+            const int s = kc & 1;
+            const uint32_t sb = s_base + s * STAGE_BYTES;
+            ok = mbar_wait(bar_full + 8 * s, (kc >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)   // 16 inputs per instruction
+                umma_f16(tmem, smem_desc_sw128(sb + ks * 32, 16, 1024), smem_desc_sw128(sb + 16384 + ks * 2048, 8192, 1024), idesc,
+                         (kc | ks) != 0);
+            umma_commit(bar_empty + 8 * s);
+            if (kc >= 1 && kc - 1 + kStages < chunks) {   // refill the other buffer once the previous chunk's UMMAs have read it
+                ok = mbar_wait(bar_empty + 8 * (s ^ 1), ((kc - 1) >> 1) & 1);
+                if (ok) load(kc - 1 + kStages);
+            }
+        }
+        umma_commit(bar_done);   // completes when every UMMA above has (at once if none was issued)
+        if (!ok) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    }
+    ok = mbar_wait(bar_done, 0);
+    tc_fence_after();
+    ok = __syncthreads_and(ok);   // the ring buffers become the output staging area
+
+    // epilogue: accumulator row r = output o; M = 128: lane r; M = 64: lane (r % 16) + 32 (r / 16)
+    const bool valid = m == 128 || lane < 16;
+    const int r = m == 128 ? tid : warp * 16 + (lane & 15);
+    const int o = ot * 128 + r;
+    if (ok) {
+        const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+        const __nv_bfloat16* krow = Kmul ? Kmul + ((size_t)o * b + j) * d + c0 : nullptr;   // K is shared by the batch
+#pragma unroll 1
+        for (int q = 0; q < nq; ++q) {
+            unsigned char* box = smem + q * (m * 128);   // [m rows][64 columns], 128-byte rows, 16-byte chunks XOR (row % 8)
+#pragma unroll 2
+            for (int c8 = 0; c8 < 8; ++c8) {
+                float v[8];
+                tmem_ld8(t_lane + q * 64 + c8 * 8, v);
+                tmem_ld_wait();
+                tmem_ld_fence8(v);
+                if (valid) {
+                    if (krow) {
+                        const uint4 kp = *reinterpret_cast<const uint4*>(krow + q * 64 + c8 * 8);
+                        const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            v[2 * e] *= __uint_as_float(kw[e] << 16);
+                            v[2 * e + 1] *= __uint_as_float(kw[e] & 0xffff0000u);
+                        }
+                        if (relu) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) v[e] = fmaxf(v[e], 0.f);
+                        }
+                    }
+                    *reinterpret_cast<uint4*>(box + (r >> 3) * 1024 + (r & 7) * 128 + ((c8 ^ (r & 7)) << 4)) =
+                        make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+                }
+            }
+        }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && ok) {
+        for (int q = 0; q < nq; ++q) tma_store_4d(&map_o, s_base + q * (m * 128), c0 + 64 * q, ot * 128, j, bt);
+        tma_store_commit();
+        tma_store_wait_read0();   // the staging area dies with the CTA
+    }
+    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, (uint32_t)nc);
+}
+
+bool covered(const m2_plan* pl, int64_t d) {
+    if (pl->dtype != M2_BF16 || pl->p != 2 || pl->dims[0] != pl->dims[1]) return false;
+    const int b = pl->dims[0];
+    return (b == 64 || b == 128 || b == 256 || b == 512) && d > 0 && d % 64 == 0;
+}
+
+cudaError_t prepare() {
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(monarch_cols_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    return e;
+}
+
+// one stage: out rows o*b + j = W[j] applied to the rows row(i, j) = i*si + j*sj of V
+static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, const void* Kmul, int relu, int64_t Bt, int64_t d,
+                     int64_t si, int64_t sj, cudaStream_t stream) {
+    const int b = pl->dims[0];
+    const int m = b == 64 ? 64 : 128;
+    const int nc = d % 256 == 0 ? 256 : d % 128 == 0 ? 128 : 64;
+    alignas(64) CUtensorMap mw, mv, mo;
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)b, (cuuint64_t)b * b}, gstr[1] = {(cuuint64_t)b * 2};
+        const cuuint32_t box[2] = {64, (cuuint32_t)m};
+        if (!tma_host::encode_sw128_bf16(&mw, W, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    }
+    {
+        const cuuint64_t gdim[4] = {(cuuint64_t)d, (cuuint64_t)b, (cuuint64_t)b, (cuuint64_t)Bt};
+        const cuuint64_t gstr[3] = {(cuuint64_t)(si * d * 2), (cuuint64_t)(sj * d * 2), (cuuint64_t)b * b * d * 2};
+        const cuuint32_t box[4] = {64, 64, 1, 1};
+        if (!tma_host::encode_sw128_bf16(&mv, V, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    }
+    {
+        const cuuint64_t gdim[4] = {(cuuint64_t)d, (cuuint64_t)b, (cuuint64_t)b, (cuuint64_t)Bt};
+        const cuuint64_t gstr[3] = {(cuuint64_t)b * d * 2, (cuuint64_t)d * 2, (cuuint64_t)b * b * d * 2};
+        const cuuint32_t box[4] = {64, (cuuint32_t)m, 1, 1};
+        if (!tma_host::encode_sw128_bf16(&mo, O, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(d / nc), (unsigned)(b * ((b + 127) / 128)), (unsigned)Bt);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, monarch_cols_stage_kernel, mw, mv, mo, (const __nv_bfloat16*)Kmul, relu, b, (int)d, nc, m, pl->d_status) !=
+        cudaSuccess)
+        return M2_ERR_CUDA;
+    return M2_OK;
+}
+
+int32_t apply(const m2_plan* pl, const void* X, const void* L, const void* R, const void* Kmul, int relu, void* Y, int64_t Bt, int64_t d,
+              void* ws, cudaStream_t stream) {
+    if (!covered(pl, d)) return M2_ERR_UNSUPPORTED;
+    if (Bt > 65535) return M2_ERR_UNSUPPORTED;
+    if (Bt == 0) return M2_OK;
+    if (prepare() != cudaSuccess) return M2_ERR_CUDA;
+    const int b = pl->dims[0];
+    int32_t st = stage(pl, R, X, ws, nullptr, 0, Bt, d, b, 1, stream);          // z[k1*b + n2] from the rows n1*b + n2
+    if (st != M2_OK) return st;
+    st = stage(pl, L, ws, Y, Kmul, relu, Bt, d, 1, b, stream);                   // y[k2*b + k1] from the rows k1*b + n2
+    if (st != M2_OK) return st;
+    pl->last_kernel = "monarch_cols_umma";
+    pl->launches += 2;
+    return M2_OK;
+}
+
+}  // namespace m2c

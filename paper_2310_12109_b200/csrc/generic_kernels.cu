@@ -890,4 +890,45 @@ cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamm
     return cudaGetLastError();
 }
 
+// One block-diagonal factor applied to a matrix whose columns are the vectors (V, O: [Bt][N][d], d contiguous):
+//   O[row o*so + j*sjo][c] = sigma(K[that row][c] * sum_i W[j][o][i] * V[row i*si + j*sj][c]),  one thread per output element
+template <typename IO>
+__global__ void __launch_bounds__(128) cols_stage_kernel(const IO* __restrict__ W, const IO* __restrict__ V, IO* __restrict__ O,
+                                                         const IO* __restrict__ Kmul, int relu, int nin, int nout, long long N, int d, long long si,
+                                                         long long sj, long long so, long long sjo) {
+    const int c = blockIdx.x * 128 + threadIdx.x;
+    if (c >= d) return;
+    const int j = blockIdx.y / nout, o = blockIdx.y % nout;
+    const long long bt = blockIdx.z;
+    const IO* w = W + ((long long)j * nout + o) * nin;
+    const IO* v = V + (bt * N + j * sj) * d + c;
+    float acc = 0.f;
+    for (int i = 0; i < nin; ++i) acc = fmaf(to_f32<IO>(w[i]), to_f32<IO>(v[(long long)i * si * d]), acc);
+    const long long row = o * so + j * sjo;
+    if (Kmul) {
+        acc *= to_f32<IO>(Kmul[row * d + c]);
+        if (relu) acc = fmaxf(acc, 0.f);
+    }
+    O[(bt * N + row) * d + c] = from_f32<IO>(acc);
+}
+
+// Y = sigma(K (.) P L P^T R P X) on [Bt][N][d] through the intermediate ws ([Bt][N][d], rows k1*N2 + n2)
+cudaError_t launch_monarch_cols(int N1, int N2, long long Bt, int d, bool bf16_io, const void* X, const void* L, const void* R, const void* Kmul,
+                                int relu, void* Y, void* ws, cudaStream_t st) {
+    const long long N = (long long)N1 * N2;
+    if (Bt == 0 || d == 0) return cudaSuccess;
+    if (Bt > 65535 || N > 65535) return cudaErrorInvalidValue;   // grid limits of this simple kernel
+    const dim3 grid((d + 127) / 128, (unsigned)N, (unsigned)Bt);
+    if (bf16_io) {
+        using T = __nv_bfloat16;
+        cols_stage_kernel<T><<<grid, 128, 0, st>>>((const T*)R, (const T*)X, (T*)ws, nullptr, 0, N1, N1, N, d, N2, 1, N2, 1);
+        cols_stage_kernel<T><<<grid, 128, 0, st>>>((const T*)L, (const T*)ws, (T*)Y, (const T*)Kmul, relu, N2, N2, N, d, 1, N2, N1, 1);
+    } else {
+        cols_stage_kernel<float><<<grid, 128, 0, st>>>((const float*)R, (const float*)X, (float*)ws, nullptr, 0, N1, N1, N, d, N2, 1, N2, 1);
+        cols_stage_kernel<float><<<grid, 128, 0, st>>>((const float*)L, (const float*)ws, (float*)Y, (const float*)Kmul, relu, N2, N2, N, d, 1, N2,
+                                                       N1, 1);
+    }
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

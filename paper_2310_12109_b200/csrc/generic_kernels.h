@@ -42,6 +42,9 @@ cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamm
                                  float eps, bool bf16, cudaStream_t st);
 // dk[h] = Re M^-1(sum_p partial[p][h][:])[0:n) / N with partial [parts][H][N] complex fp32 in plan order
 cudaError_t launch_spectrum_sum_inverse(const ConvShape& s, const void* partial, int parts, float* dk, cudaStream_t st);
+// Y = sigma(K (.) M X) for Bt matrices [N][d] whose columns are the vectors (CUDA cores; ws: Bt*N*d values of the I/O type)
+cudaError_t launch_monarch_cols(int N1, int N2, long long Bt, int d, bool bf16_io, const void* X, const void* L, const void* R, const void* Kmul,
+                                int relu, void* Y, void* ws, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -10,6 +10,7 @@
 
 #include "conv_umma.h"
 #include "generic_kernels.h"
+#include "cols_umma.h"
 #include "matmul_umma.h"
 #include "mlp_umma.h"
 #include "m2_plan.h"
@@ -385,6 +386,33 @@ int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev
 }
 
 static int64_t round256(int64_t v) { return (v + 255) / 256 * 256; }
+
+int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev, int32_t act,
+                        void* Y_dev, int64_t Bt, int64_t d, void* ws_dev, int64_t ws_bytes, void* stream) {
+    if (!plan || Bt < 0 || d < 0) return M2_ERR_INVALID_ARG;
+    if (act != M2_ACT_NONE && act != M2_ACT_RELU) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (plan->p != 2) return M2_ERR_UNSUPPORTED;
+    const int64_t elems = Bt * plan->N * d;
+    if (elems == 0) return M2_OK;
+    if (!X_dev || !L_dev || !R_dev || !Y_dev || !ws_dev) return M2_ERR_INVALID_ARG;
+    if (!aligned16(X_dev) || !aligned16(L_dev) || !aligned16(R_dev) || !aligned16(K_dev) || !aligned16(Y_dev) || !aligned16(ws_dev))
+        return M2_ERR_ALIGNMENT;
+    const bool bf = plan->dtype == M2_BF16;
+    if (ws_bytes < elems * (bf ? 2 : 4)) return M2_ERR_INVALID_ARG;
+    if (d > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    int32_t st = m2c::apply(plan, X_dev, L_dev, R_dev, K_dev, act == M2_ACT_RELU, Y_dev, Bt, d, ws_dev, (cudaStream_t)stream);
+    if (st != M2_ERR_UNSUPPORTED) return st;
+    const cudaError_t e = m2g::launch_monarch_cols(plan->dims[0], plan->dims[1], Bt, (int)d, bf, X_dev, L_dev, R_dev, K_dev, act == M2_ACT_RELU,
+                                                   Y_dev, ws_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "monarch_cols_generic";
+    plan->launches += 2;
+    return M2_OK;
+}
 
 int64_t m2_layer_scratch_bytes(const m2_plan* plan_n, const m2_plan* plan_d, int64_t B) {
     if (!plan_n || !plan_d || B < 0) return -1;

@@ -441,6 +441,29 @@ def test_m2_layer_fwd(B, sn, sd, dtype):
     plan_d.close()
 
 
+@pytest.mark.parametrize("b,Bt,d,dtype,withK", [(64, 2, 192, M.M2_BF16, True), (128, 1, 256, M.M2_BF16, True), (256, 1, 64, M.M2_BF16, False),
+                                                 (64, 1, 768, M.M2_BF16, False), (8, 3, 40, M.M2_BF16, True), (6, 2, 33, M.M2_FP32, True)])
+def test_monarch_cols(b, Bt, d, dtype, withK):
+    """Y = sigma(K (.) M X) with the columns of X [Bt, N, d] as the vectors (the layout of the operator benchmark)."""
+    N = b * b
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    L = rnd(synth.normal(synth.stream_id(13, 0), (b, b, b)) / np.sqrt(b))
+    R = rnd(synth.normal(synth.stream_id(13, 1), (b, b, b)) / np.sqrt(b))
+    X = rnd(synth.normal(synth.stream_id(13, 2), (Bt, N, d)))
+    K = rnd(synth.normal(synth.stream_id(13, 3), (N, d))) if withK else None
+    plan = M.Plan((b, b), dtype=dtype, device=0)
+    dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
+    Y = M.m2_monarch_cols(plan, dv(X), dv(L), dv(R), None if K is None else dv(K), act=M.M2_ACT_RELU if withK else M.M2_ACT_NONE)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    umma = dtype == M.M2_BF16 and b in (64, 128, 256, 512) and d % 64 == 0
+    assert plan.last_kernel() == ("monarch_cols_umma" if umma else "monarch_cols_generic")
+    ref = O.monarch_cols(L, R, X, K, "relu" if withK else "none")
+    check(host(Y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, f"monarch cols b={b}")
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -376,6 +376,17 @@ def test_monarch_mix_operator():
     assert np.allclose(y.imag, 0) and np.allclose(y.real, np.stack([O.direct_circular_conv(k[t % Hk], x[t]) for t in range(T)]))
 
 
+def test_monarch_cols_oracle():
+    """Columns as vectors: the dense matrix times X, and the factor / ReLU applied afterwards."""
+    N1, N2, d = 3, 4, 5
+    L, R = rng.standard_normal((N1, N2, N2)), rng.standard_normal((N2, N1, N1))
+    X, K = rng.standard_normal((2, N1 * N2, d)), rng.standard_normal((N1 * N2, d))
+    Md = O.monarch_dense(L, R)
+    assert np.allclose(O.monarch_cols(L, R, X), Md @ X)
+    assert np.allclose(O.monarch_cols(L, R, X, K, "relu"), np.where(K * (Md @ X) > 0, K * (Md @ X), 0.0))
+    assert np.allclose(O.monarch_cols(L, R, X, K), K * (Md @ X))
+
+
 def test_m2_layer_oracle():
     """The layer against the same computation with dense matrices and einsum over the un-transposed [B, n, d] tensor;
     LayerNorm against torch's routine and its invariants (zero mean, unit variance, shift/scale invariance)."""

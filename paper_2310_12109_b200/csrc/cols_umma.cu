@@ -10,10 +10,11 @@
 // so the stride permutations are nothing but the strides of two TMA tensor maps.  One kernel serves both stages:
 // a CTA computes the tile [128 outputs o][NC columns] of one block j:  A = W[j] rows (K-major, 128B-swizzled TMA boxes
 // of 64 inputs), B = 64 input rows x NC columns (N-major: a row of the operand is a row of V), accumulator in TMEM
-// (M = 128, or 64 when b = 64; N = NC <= 256), K = b walked in chunks of 64 through a two-stage TMA ring; the
+// (M = 128, or 64 when b = 64; N = NC <= 256), K = b walked in chunks of 64 through a three-stage TMA ring; the
 // epilogue applies the optional factor K (.) and ReLU in fp32, rounds to bf16, stages the tile in the swizzled image of
-// the TMA store boxes and stores it to the rows o*b + j.  About 100 KB of shared memory and NC TMEM columns per CTA:
-// two CTAs per SM overlap each other's load, UMMA and epilogue phases.  All waits are bounded.
+// the TMA store boxes and stores it to the rows o*b + j.  One persistent CTA per SM with a producer warp, an issuing warp
+// and four epilogue warps; two accumulators in TMEM, so a tile's epilogue overlaps the next tile's UMMAs.  All waits are
+// bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -27,11 +28,13 @@ namespace m2c {
 
 using namespace sm100;
 
-constexpr int kThreads = 128;
-constexpr int kStages = 2;
+constexpr int kThreads = 192;               // warps 0..3: epilogue (the four TMEM lane quarters); warp 4: TMA producer; warp 5: UMMA issuer
+constexpr int kStages = 3;
 constexpr int STAGE_BYTES = 49152;          // A chunk [128][64] 16384 | B chunk [64][256] 32768
-constexpr int OFF_BAR = kStages * STAGE_BYTES;   // full[2], empty[2], done, tmem ptr
-constexpr int SMEM_BYTES = OFF_BAR + 64;
+constexpr int OFF_OUT = kStages * STAGE_BYTES;   // output staging: up to 4 boxes [128][64] bf16   65536
+constexpr int OFF_BAR = OFF_OUT + 65536;    // full[3], empty[3], acc_full[2], acc_empty[2], tmem ptr, abort flag
+constexpr int SMEM_BYTES = OFF_BAR + 128;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
@@ -43,120 +46,197 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// grid: x = column tile, y = j * otiles + output tile, z = matrix of the batch
-__global__ void __launch_bounds__(kThreads, 2)
+// barrier among the 128 epilogue threads that also ANDs a predicate (every thread gets the same answer)
+__device__ __forceinline__ bool epilogue_sync_and(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return r != 0;
+}
+
+// Persistent: CTA p works on tiles p, p + gridDim.x, ...; tile index = ((bt * b + j) * otiles + ot) * ctiles + ct, so the
+// CTAs running at the same time share the block's weights or its input rows in L2.  The producer runs ahead through the
+// three-stage ring across tile boundaries; the accumulator is double-buffered in TMEM, so a tile's epilogue overlaps the
+// next tile's UMMAs.
+__global__ void __launch_bounds__(kThreads, 1)
 monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_v,
                           const __grid_constant__ CUtensorMap map_o, const __nv_bfloat16* __restrict__ Kmul, int relu, int b, int d, int nc,
-                          int m, int32_t* __restrict__ status) {
+                          int m, int tiles, int32_t* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
-    const uint32_t bar_full = s_base + OFF_BAR, bar_empty = bar_full + 16, bar_done = bar_full + 32, s_tptr = bar_full + 40;
-    const int otiles = (b + 127) / 128;
-    const int c0 = blockIdx.x * nc, j = blockIdx.y / otiles, ot = blockIdx.y % otiles, bt = blockIdx.z;
+    const uint32_t bar_full = s_base + OFF_BAR, bar_empty = bar_full + 24, bar_accf = bar_full + 48, bar_acce = bar_full + 64;
+    const uint32_t s_tptr = bar_full + 80;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + 88);
+    const int otiles = (b + 127) / 128, ctiles = d / nc;
     const int chunks = b / 64, nq = nc / 64;
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        mbar_init(bar_done, 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_accf + 8 * a, 1);
+            mbar_init(bar_acce + 8 * a, 4);   // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_w);
         prefetch_tensormap(&map_v);
         prefetch_tensormap(&map_o);
     }
-    if (warp == 0) tmem_alloc(s_tptr, (uint32_t)nc);   // 64, 128 or 256 columns
+    if (warp == 5) tmem_alloc(s_tptr, (uint32_t)(2 * nc));   // 128, 256 or 512 columns: two accumulators
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     asm volatile("griddepcontrol.wait;" ::: "memory");   // V may have been written by the kernel before this one
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 40);
-    bool ok = true;
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + 80);
 
-    if (tid == 0) {
-        const uint32_t stage_tx = (uint32_t)(m * 128 + nq * 8192);
-        auto load = [&](int kc) {
-            const int s = kc & 1;
-            const uint32_t sb = s_base + s * STAGE_BYTES, bf = bar_full + 8 * s;
-            mbar_expect_tx(bf, stage_tx);
-            tma_load_2d(sb, &map_w, kc * 64, j * b + ot * 128, bf);                                      // W[j][o tile][64 inputs]
-            for (int q = 0; q < nq; ++q) tma_load_4d(sb + 16384 + q * 8192, &map_v, c0 + 64 * q, kc * 64, j, bt, bf);   // 64 input rows
-        };
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(nc >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-        for (int kc = 0; kc < kStages && kc < chunks; ++kc) load(kc);
-#pragma unroll 1
-        for (int kc = 0; kc < chunks && ok; ++kc) {
-            const int s = kc & 1;
-            const uint32_t sb = s_base + s * STAGE_BYTES;
-            ok = mbar_wait(bar_full + 8 * s, (kc >> 1) & 1);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)   // 16 inputs per instruction
-                umma_f16(tmem, smem_desc_sw128(sb + ks * 32, 16, 1024), smem_desc_sw128(sb + 16384 + ks * 2048, 8192, 1024), idesc,
-                         (kc | ks) != 0);
-            umma_commit(bar_empty + 8 * s);
-            if (kc >= 1 && kc - 1 + kStages < chunks) {   // refill the other buffer once the previous chunk's UMMAs have read it
-                ok = mbar_wait(bar_empty + 8 * (s ^ 1), ((kc - 1) >> 1) & 1);
-                if (ok) load(kc - 1 + kStages);
-            }
-        }
-        umma_commit(bar_done);   // completes when every UMMA above has (at once if none was issued)
-        if (!ok) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-    }
-    ok = mbar_wait(bar_done, 0);
-    tc_fence_after();
-    ok = __syncthreads_and(ok);   // the ring buffers become the output staging area
-
-    // epilogue: accumulator row r = output o; M = 128: lane r; M = 64: lane (r % 16) + 32 (r / 16)
-    const bool valid = m == 128 || lane < 16;
-    const int r = m == 128 ? tid : warp * 16 + (lane & 15);
-    const int o = ot * 128 + r;
-    if (ok) {
-        const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-        const __nv_bfloat16* krow = Kmul ? Kmul + ((size_t)o * b + j) * d + c0 : nullptr;   // K is shared by the batch
-#pragma unroll 1
-        for (int q = 0; q < nq; ++q) {
-            unsigned char* box = smem + q * (m * 128);   // [m rows][64 columns], 128-byte rows, 16-byte chunks XOR (row % 8)
-#pragma unroll 2
-            for (int c8 = 0; c8 < 8; ++c8) {
-                float v[8];
-                tmem_ld8(t_lane + q * 64 + c8 * 8, v);
-                tmem_ld_wait();
-                tmem_ld_fence8(v);
-                if (valid) {
-                    if (krow) {
-                        const uint4 kp = *reinterpret_cast<const uint4*>(krow + q * 64 + c8 * 8);
-                        const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            v[2 * e] *= __uint_as_float(kw[e] << 16);
-                            v[2 * e + 1] *= __uint_as_float(kw[e] & 0xffff0000u);
-                        }
-                        if (relu) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) v[e] = fmaxf(v[e], 0.f);
-                        }
+    if (warp == 4) {
+        // ---- TMA producer ----------------------------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t stage_tx = (uint32_t)(m * 128 + nq * 8192);
+            uint32_t n = 0;   // chunks issued so far
+            bool ok = true;
+            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+                const int ct = t % ctiles, ot = (t / ctiles) % otiles, j = (t / (ctiles * otiles)) % b, bt = t / (ctiles * otiles * b);
+                for (int kc = 0; kc < chunks; ++kc, ++n) {
+                    const int s = n % kStages;
+                    if (n >= kStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kStages) - 1) & 1);   // the UMMAs have read the buffer
+                    if (!ok || *abort_flag) {
+                        ok = false;
+                        break;
                     }
-                    *reinterpret_cast<uint4*>(box + (r >> 3) * 1024 + (r & 7) * 128 + ((c8 ^ (r & 7)) << 4)) =
-                        make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+                    const uint32_t sb = s_base + s * STAGE_BYTES, bf = bar_full + 8 * s;
+                    mbar_expect_tx(bf, stage_tx);
+                    tma_load_2d(sb, &map_w, kc * 64, j * b + ot * 128, bf);                                          // W[j][o tile][64 inputs]
+                    for (int q = 0; q < nq; ++q) tma_load_4d(sb + 16384 + q * 8192, &map_v, ct * nc + 64 * q, kc * 64, j, bt, bf);   // 64 input rows
                 }
             }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+            }
+        }
+    } else if (warp == 5) {
+        // ---- UMMA issuer -----------------------------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(nc >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+            uint32_t n = 0;
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+                const int acc = it & 1;
+                if (it >= 2) ok = mbar_wait(bar_acce + 8 * acc, ((it >> 1) - 1) & 1);   // the epilogue has read this accumulator
+                if (!ok) break;
+                tc_fence_after();
+                for (int kc = 0; kc < chunks; ++kc, ++n) {
+                    const int s = n % kStages;
+                    ok = mbar_wait(bar_full + 8 * s, (n / kStages) & 1);
+                    if (!ok || *abort_flag) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sb = s_base + s * STAGE_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)   // 16 inputs per instruction
+                        umma_f16(tmem + acc * nc, smem_desc_sw128(sb + ks * 32, 16, 1024), smem_desc_sw128(sb + 16384 + ks * 2048, 8192, 1024),
+                                 idesc, (kc | ks) != 0);
+                    umma_commit(bar_empty + 8 * s);
+                }
+                if (ok) umma_commit(bar_accf + 8 * acc);
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+            }
+        }
+    } else {
+        // ---- epilogue warps: accumulator row r = output o; M = 128: lane r; M = 64: lane (r % 16) + 32 (r / 16) -------------------
+        const bool valid = m == 128 || lane < 16;
+        const int r = m == 128 ? tid : warp * 16 + (lane & 15);
+        const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+        unsigned char* stg = smem + OFF_OUT;
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+            const int ct = t % ctiles, ot = (t / ctiles) % otiles, j = (t / (ctiles * otiles)) % b, bt = t / (ctiles * otiles * b);
+            const int acc = it & 1, o = ot * 128 + r, c0 = ct * nc;
+            // the factor K (.) for this thread's row, requested while the tile's UMMAs still run
+            uint4 kreg[32];
+            if (Kmul != nullptr && valid) {
+                const uint4* krow = reinterpret_cast<const uint4*>(Kmul + ((size_t)o * b + j) * d + c0);   // K is shared by the batch
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    if (e < nq * 8) kreg[e] = __ldg(krow + e);
+            }
+            ok = mbar_wait(bar_accf + 8 * acc, (it >> 1) & 1);
+            tc_fence_after();
+            if (tid == 0) tma_store_wait_read0();   // the previous tile's stores have read the staging area
+            ok = epilogue_sync_and(ok && *abort_flag == 0);
+            if (!ok) break;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q >= nq) break;
+                unsigned char* box = stg + q * (m * 128);   // [m rows][64 columns], 128-byte rows, 16-byte chunks XOR (row % 8)
+#pragma unroll
+                for (int hq = 0; hq < 2; ++hq) {
+                    float v[32];
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) tmem_ld8(t_lane + acc * nc + q * 64 + (hq * 4 + c8) * 8, v + 8 * c8);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) tmem_ld_fence8(v + 8 * c8);
+                    if (valid) {
+#pragma unroll
+                        for (int c8 = 0; c8 < 4; ++c8) {
+                            float* w = v + 8 * c8;
+                            if (Kmul != nullptr) {
+                                const uint4 kp = kreg[q * 8 + hq * 4 + c8];
+                                const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    w[2 * e] *= __uint_as_float(kw[e] << 16);
+                                    w[2 * e + 1] *= __uint_as_float(kw[e] & 0xffff0000u);
+                                }
+                                if (relu) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) w[e] = fmaxf(w[e], 0.f);
+                                }
+                            }
+                            *reinterpret_cast<uint4*>(box + (r >> 3) * 1024 + (r & 7) * 128 + (((hq * 4 + c8) ^ (r & 7)) << 4)) =
+                                make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]), pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7]));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acce + 8 * acc);   // this warp has read its part of the accumulator
+            fence_proxy_async();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (tid == 0) {
+                for (int q = 0; q < nq; ++q) tma_store_4d(&map_o, s_base + OFF_OUT + q * (m * 128), c0 + 64 * q, ot * 128, j, bt);
+                tma_store_commit();
+            }
+        }
+        if (tid == 0) tma_store_wait_read0();   // the staging area dies with the CTA
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
         }
     }
-    fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    if (tid == 0 && ok) {
-        for (int q = 0; q < nq; ++q) tma_store_4d(&map_o, s_base + q * (m * 128), c0 + 64 * q, ot * 128, j, bt);
-        tma_store_commit();
-        tma_store_wait_read0();   // the staging area dies with the CTA
-    }
-    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, (uint32_t)nc);
+    if (warp == 5) tmem_dealloc(tmem, (uint32_t)(2 * nc));
 }
 
 bool covered(const m2_plan* pl, int64_t d) {
@@ -200,8 +280,13 @@ static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, c
         const cuuint32_t box[4] = {64, (cuuint32_t)m, 1, 1};
         if (!tma_host::encode_sw128_bf16(&mo, O, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
     }
+    const long long tiles = Bt * b * ((b + 127) / 128) * (d / nc);
+    if (tiles > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(d / nc), (unsigned)(b * ((b + 127) / 128)), (unsigned)Bt);
+    cfg.gridDim = dim3((unsigned)(tiles < sms ? tiles : sms));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = stream;
@@ -210,7 +295,7 @@ static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, monarch_cols_stage_kernel, mw, mv, mo, (const __nv_bfloat16*)Kmul, relu, b, (int)d, nc, m, pl->d_status) !=
+    if (cudaLaunchKernelEx(&cfg, monarch_cols_stage_kernel, mw, mv, mo, (const __nv_bfloat16*)Kmul, relu, b, (int)d, nc, m, (int)tiles, pl->d_status) !=
         cudaSuccess)
         return M2_ERR_CUDA;
     return M2_OK;

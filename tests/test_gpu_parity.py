@@ -442,7 +442,7 @@ def test_m2_layer_fwd(B, sn, sd, dtype):
 
 
 @pytest.mark.parametrize("b,Bt,d,dtype,withK", [(64, 2, 192, M.M2_BF16, True), (128, 1, 256, M.M2_BF16, True), (256, 1, 64, M.M2_BF16, False),
-                                                 (64, 1, 768, M.M2_BF16, False), (8, 3, 40, M.M2_BF16, True), (6, 2, 33, M.M2_FP32, True)])
+                                                 (256, 2, 256, M.M2_BF16, True), (64, 1, 768, M.M2_BF16, False), (8, 3, 40, M.M2_BF16, True), (6, 2, 33, M.M2_FP32, True)])
 def test_monarch_cols(b, Bt, d, dtype, withK):
     """Y = sigma(K (.) M X) with the columns of X [Bt, N, d] as the vectors (the layout of the operator benchmark)."""
     N = b * b

@@ -163,8 +163,10 @@ int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev
  * (R is applied first; the listing's parameter called L is the one applied first, i.e. this library's R).
  * y_dev: [B, n, d] (must not overlap x_dev).  scratch_dev: m2_layer_scratch_bytes(plan_n, plan_d, B) bytes, caller-owned.
  * ws_dev / ws_bytes: optional matmul workspace, at least the larger of m2_matmul_workspace_bytes(plan_n, B d) and
- * m2_matmul_workspace_bytes(plan_d, B n); NULL selects the kernels that need none.  9 launches with a workspace
- * for both products, fewer on the generic path. */
+ * m2_matmul_workspace_bytes(plan_d, B n); NULL selects the kernels that need none.
+ * The sequence mix runs through the columns-as-vectors kernels (m2_monarch_cols: x is [n, d] per batch entry with the
+ * channels contiguous, so nothing but the [d, n] kernel parameter is transposed); the feature mix through the
+ * rows-as-vectors kernels (m2_monarch_mix); the residual add and the normalisation are one kernel. */
 int64_t m2_layer_scratch_bytes(const m2_plan* plan_n, const m2_plan* plan_d, int64_t B);
 int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x_dev, const void* const* factors,
                      const void* n_kernel_dev, const void* d_kernel_dev, const float* gamma_dev, const float* beta_dev,

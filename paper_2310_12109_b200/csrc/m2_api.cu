@@ -387,6 +387,20 @@ int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev
 
 static int64_t round256(int64_t v) { return (v + 255) / 256 * 256; }
 
+// Y[bt] = sigma(K (.) M X[bt]) on [Bt][N][d]; arguments already checked, device already current
+static int32_t cols_impl(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev, int relu, void* Y_dev,
+                         int64_t Bt, int64_t d, void* ws_dev, cudaStream_t stream) {
+    int32_t st = m2c::apply(plan, X_dev, L_dev, R_dev, K_dev, relu, Y_dev, Bt, d, ws_dev, stream);
+    if (st != M2_ERR_UNSUPPORTED) return st;
+    const cudaError_t e = m2g::launch_monarch_cols(plan->dims[0], plan->dims[1], Bt, (int)d, plan->dtype == M2_BF16, X_dev, L_dev, R_dev, K_dev,
+                                                   relu, Y_dev, ws_dev, stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "monarch_cols_generic";
+    plan->launches += 2;
+    return M2_OK;
+}
+
 int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev, int32_t act,
                         void* Y_dev, int64_t Bt, int64_t d, void* ws_dev, int64_t ws_bytes, void* stream) {
     if (!plan || Bt < 0 || d < 0) return M2_ERR_INVALID_ARG;
@@ -403,20 +417,13 @@ int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_de
     if (d > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
-    int32_t st = m2c::apply(plan, X_dev, L_dev, R_dev, K_dev, act == M2_ACT_RELU, Y_dev, Bt, d, ws_dev, (cudaStream_t)stream);
-    if (st != M2_ERR_UNSUPPORTED) return st;
-    const cudaError_t e = m2g::launch_monarch_cols(plan->dims[0], plan->dims[1], Bt, (int)d, bf, X_dev, L_dev, R_dev, K_dev, act == M2_ACT_RELU,
-                                                   Y_dev, ws_dev, (cudaStream_t)stream);
-    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
-    if (e != cudaSuccess) return M2_ERR_CUDA;
-    plan->last_kernel = "monarch_cols_generic";
-    plan->launches += 2;
-    return M2_OK;
+    return cols_impl(plan, X_dev, L_dev, R_dev, K_dev, act == M2_ACT_RELU, Y_dev, Bt, d, ws_dev, (cudaStream_t)stream);
 }
 
 int64_t m2_layer_scratch_bytes(const m2_plan* plan_n, const m2_plan* plan_d, int64_t B) {
     if (!plan_n || !plan_d || B < 0) return -1;
-    return 2 * round256(B * plan_n->N * plan_d->N * (plan_n->dtype == M2_BF16 ? 2 : 4));
+    const int64_t es = plan_n->dtype == M2_BF16 ? 2 : 4;
+    return 3 * round256(B * plan_n->N * plan_d->N * es) + round256(plan_n->N * plan_d->N * es);
 }
 
 int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x_dev, const void* const* factors, const void* n_kernel_dev,
@@ -437,22 +444,35 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
         return M2_ERR_ALIGNMENT;
     const bool bf = plan_n->dtype == M2_BF16;
     const int64_t tensor_bytes = B * n * d * (bf ? 2 : 4);
-    if (scratch_bytes < 2 * round256(tensor_bytes)) return M2_ERR_INVALID_ARG;
+    if (scratch_bytes < m2_layer_scratch_bytes(plan_n, plan_d, B)) return M2_ERR_INVALID_ARG;
     DeviceGuard g(plan_n->device);
     if (!g.ok) return M2_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    void* s1 = scratch_dev;                                                  // [B, d, n]: x^T, then the sequence mix
-    void* s2 = static_cast<unsigned char*>(scratch_dev) + round256(tensor_bytes);   // [B, n, d]: x~
-    if (m2g::launch_transpose_any(x_dev, s1, B, (int)n, (int)d, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    int32_t rc = matmul_impl(plan_n, s1, factors[0], factors[1], s1, B * d, ws_dev, ws_bytes, n_kernel_dev, d, 1, st);
-    if (rc == M2_OK) rc = matmul_impl(plan_n, s1, factors[2], factors[3], s1, B * d, ws_dev, ws_bytes, nullptr, 1, 0, st);
+    unsigned char* sc = static_cast<unsigned char*>(scratch_dev);
+    void* s1 = sc;                                   // [B, n, d]: relu(K_n (.) M1 x)      (or [B, d, n] on the transposing route)
+    void* s2 = sc + round256(tensor_bytes);          // [B, n, d]: x~
+    void* s3 = sc + 2 * round256(tensor_bytes);      // [B, n, d]: the intermediate between the two factors of M1 / M2
+    void* kt = sc + 3 * round256(tensor_bytes);      // [n, d]: the sequence kernel with the channels contiguous
+    // Sequence mix.  x is [B, n, d] with the channels contiguous, i.e. the COLUMNS of each [n, d] matrix are the vectors M1, M2
+    // act on: no transposition of the activations, only of the [d, n] kernel parameter.
+    if (m2g::launch_transpose_any(n_kernel_dev, kt, 1, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    int32_t rc = cols_impl(plan_n, x_dev, factors[0], factors[1], kt, 1, s1, B, d, s3, st);
+    if (rc == M2_OK) rc = cols_impl(plan_n, s1, factors[2], factors[3], nullptr, 0, s2, B, d, s3, st);
+    int extra = 2;   // launches beyond the products: kernel transpose + normalisation
+    if (rc == M2_ERR_UNSUPPORTED) {   // n too large for the CUDA-core column kernel: transpose the activations instead
+        if (m2g::launch_transpose_any(x_dev, s1, B, (int)n, (int)d, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+        rc = matmul_impl(plan_n, s1, factors[0], factors[1], s1, B * d, ws_dev, ws_bytes, n_kernel_dev, d, 1, st);
+        if (rc == M2_OK) rc = matmul_impl(plan_n, s1, factors[2], factors[3], s1, B * d, ws_dev, ws_bytes, nullptr, 1, 0, st);
+        if (rc != M2_OK) return rc;
+        if (m2g::launch_transpose_any(s1, s2, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+        extra = 4;
+    }
     if (rc != M2_OK) return rc;
-    if (m2g::launch_transpose_any(s1, s2, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
     rc = matmul_impl(plan_d, s2, factors[4], factors[5], y_dev, B * n, ws_dev, ws_bytes, d_kernel_dev, 1, 1, st);
     if (rc == M2_OK) rc = matmul_impl(plan_d, y_dev, factors[6], factors[7], y_dev, B * n, ws_dev, ws_bytes, nullptr, 1, 0, st);
     if (rc != M2_OK) return rc;
     if (m2g::launch_add_layernorm(y_dev, s2, gamma_dev, beta_dev, y_dev, B * n, (int)d, eps, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    plan_n->launches += 3;   // the two transposes and the normalisation (the products count themselves on their plans)
+    plan_n->launches += extra;   // (the products count themselves on their plans)
     plan_n->last_kernel = "layer_fwd";
     return M2_OK;
 }

@@ -487,6 +487,49 @@ def test_empty_batches_and_error_codes():
     plan.close()
 
 
+def test_error_codes_of_the_operator_and_gradient_calls():
+    """Bad arguments are refused on the host, before anything is launched."""
+    lib = M.lib()
+    s = torch.cuda.current_stream().cuda_stream
+    plan = M.Plan((64, 64), dtype=M.M2_BF16, device=0)
+    plan3 = M.Plan((4, 4, 4), dtype=M.M2_BF16, device=0)
+    T, N = 4, 4096
+    X = torch.zeros((T, N), dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros((64, 64, 64), dtype=torch.bfloat16, device="cuda")
+    Y = torch.empty_like(X)
+    dW = torch.empty((64, 64, 64), dtype=torch.float32, device="cuda")
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    p, w, y = X.data_ptr(), W.data_ptr(), Y.data_ptr()
+    # m2_monarch_mix: unknown activation, missing kernel, Hk < 1, misaligned kernel, order-3 plan
+    assert lib.m2_monarch_mix(plan.handle, p, p, 1, 7, w, w, w, w, y, T, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_mix(plan.handle, p, None, 1, 0, w, w, w, w, y, T, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_mix(plan.handle, p, p, 0, 0, w, w, w, w, y, T, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_mix(plan.handle, p, p + 2, 1, 0, w, w, w, w, y, T, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_ALIGNMENT
+    assert lib.m2_monarch_mix(plan3.handle, p, p, 1, 0, w, w, w, w, y, T, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_UNSUPPORTED
+    # m2_monarch_cols: workspace too small, missing workspace, unknown activation
+    assert lib.m2_monarch_cols(plan.handle, p, w, w, None, 0, y, 1, 4, ws.data_ptr(), 16, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_cols(plan.handle, p, w, w, None, 0, y, 1, 4, None, 0, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_cols(plan.handle, p, w, w, None, 5, y, 1, 4, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_cols(plan.handle, p, w, w, None, 0, y, 0, 4, None, 0, s) == M.M2_OK          # empty batch
+    # m2_monarch_matmul_bwd_weights: workspace too small, missing gradient buffers
+    assert lib.m2_monarch_matmul_bwd_weights(plan.handle, p, p, w, w, dW.data_ptr(), dW.data_ptr(), T, ws.data_ptr(), 16, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_matmul_bwd_weights(plan.handle, p, p, w, w, None, dW.data_ptr(), T, ws.data_ptr(), ws.numel(), s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_matmul_bwd_workspace_bytes(plan3.handle, T) == -1
+    # m2_blocks_transpose: non-positive block shape
+    assert lib.m2_blocks_transpose(plan.handle, w, dW.data_ptr(), 64, 0, 64, s) == M.M2_ERR_INVALID_ARG
+    # m2_layer_fwd: plans of different dtypes, scratch too small
+    pf = M.Plan((8, 8), dtype=M.M2_FP32, device=0)
+    pb = M.Plan((8, 8), dtype=M.M2_BF16, device=0)
+    fac = (ctypes.c_void_p * 8)(*([w] * 8))
+    g = torch.ones(64, dtype=torch.float32, device="cuda")
+    assert lib.m2_layer_fwd(pb.handle, pf.handle, p, fac, p, p, g.data_ptr(), g.data_ptr(), 1e-5, y, 1, ws.data_ptr(), ws.numel(), None, 0, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_layer_fwd(pb.handle, pb.handle, p, fac, p, p, g.data_ptr(), g.data_ptr(), 1e-5, y, 1, ws.data_ptr(), 64, None, 0, s) == M.M2_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    for q in (plan, plan3, pf, pb):
+        assert q.device_status() == 0
+        q.close()
+
+
 def test_runs_are_bit_identical_and_stay_in_bounds():
     c = synth.config2(B=8, H=16)
     plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)

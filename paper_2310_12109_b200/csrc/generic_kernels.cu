@@ -177,15 +177,17 @@ __global__ void __launch_bounds__(1024) conv_row_kernel(const IO* __restrict__ x
 }
 
 // Gradient with respect to the kernel: dk[h] = M^-1 ( sum_b conj(M x'_b) (.) M g'_b ) [0:n) / N, one block per channel,
-// the batch walked sequentially; x, g rows and the accumulated product stay in shared memory (3 complex fp32 rows).
+// the batch walked sequentially; x, g rows and the accumulated product stay in shared memory (3 complex fp32 rows) -- or, for
+// N too large for that, in a per-block slice of a global scratch buffer (gscratch != nullptr; blocks then walk the channels).
 template <typename IO, int ITEMS>
 __global__ void __launch_bounds__(1024) conv_wgrad_kernel(const IO* __restrict__ x, const IO* __restrict__ g, float* __restrict__ dk, Dims D,
-                                                          Roots R, int B, int H, int n) {
+                                                          Roots R, int B, int H, int n, float2* gscratch) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float2* bx = reinterpret_cast<float2*>(smem_raw);
+    float2* bx = gscratch ? gscratch + (size_t)blockIdx.x * 3 * D.N : reinterpret_cast<float2*>(smem_raw);
     float2* bg = bx + D.N;
     float2* acc = bg + D.N;
-    const int h = blockIdx.x;
+    for (int h = blockIdx.x; h < H; h += gridDim.x) {
+    __syncthreads();   // the previous channel's result has been read
     for (int i = threadIdx.x; i < D.N; i += blockDim.x) acc[i] = make_float2(0.f, 0.f);
     for (int b = 0; b < B; ++b) {
         const IO* xr = x + ((long long)b * H + h) * n;
@@ -206,6 +208,7 @@ __global__ void __launch_bounds__(1024) conv_wgrad_kernel(const IO* __restrict__
     for (int a = D.p - 1; a >= 0; --a) stage<float2, ITEMS, true>(acc, D, a, R.r[a]);
     const float inv = 1.0f / (float)D.N;
     for (int i = threadIdx.x; i < n; i += blockDim.x) dk[(long long)h * n + i] = acc[i].x * inv;
+    }
 }
 
 // k_f = F_N pad(k) / N per channel, in plan order, computed in place in the output buffer (global
@@ -653,20 +656,34 @@ cudaError_t launch_spectrum_sum_inverse(const ConvShape& s, const void* partial,
     return cudaGetLastError();
 }
 
-cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, cudaStream_t st) {
+long long conv_wgrad_scratch_bytes(long long N, long long H) {
+    if ((size_t)N * sizeof(float2) * 3 <= 200 * 1024) return 0;   // fits in shared memory
+    return (H < kWgradScratchBlocks ? H : kWgradScratchBlocks) * 3 * N * (long long)sizeof(float2);
+}
+
+cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, void* scratch, long long scratch_bytes,
+                              cudaStream_t st) {
     Dims D = make_dims(s);
     Roots R{{s.roots[0], s.roots[1], s.roots[2]}};
     int items, threads;
     if (!pick_launch(D, items, threads)) return cudaErrorInvalidValue;
-    const size_t smem = (size_t)D.N * sizeof(float2) * 3;
-    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    size_t smem = (size_t)D.N * sizeof(float2) * 3;
+    unsigned grid = (unsigned)s.H;
+    float2* gs = nullptr;
+    const long long need = conv_wgrad_scratch_bytes(D.N, s.H);
+    if (need > 0) {   // rows too long for shared memory: per-block slices of the caller's scratch buffer
+        if (!scratch || scratch_bytes < need) return cudaErrorInvalidValue;
+        gs = reinterpret_cast<float2*>(scratch);
+        smem = 0;
+        grid = (unsigned)(s.H < kWgradScratchBlocks ? s.H : kWgradScratchBlocks);
+    }
     if (s.H == 0) return cudaSuccess;
 #define M2_LAUNCH_WGRAD(IO, IT)                                                                                   \
     {                                                                                                             \
         auto kern = conv_wgrad_kernel<IO, IT>;                                                                    \
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);       \
         if (e != cudaSuccess) return e;                                                                           \
-        kern<<<(unsigned)s.H, threads, smem, st>>>((const IO*)x, (const IO*)g, dk, D, R, (int)s.B, (int)s.H, (int)s.n); \
+        kern<<<grid, threads, smem, st>>>((const IO*)x, (const IO*)g, dk, D, R, (int)s.B, (int)s.H, (int)s.n, gs); \
     }
     if (bf16_io) {
         switch (items) {

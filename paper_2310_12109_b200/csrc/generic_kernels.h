@@ -29,7 +29,11 @@ cudaError_t launch_transpose_btc(const void* x, void* xT, long long B, int T, in
 cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w, void* z, long long B, int T, int C, cudaStream_t st);
 
 // dk[H, n] (fp32) = gradient of sum_b <conv(k, x_b), g_b> with respect to k; x, g: [B, H, n] contiguous
-cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, cudaStream_t st);
+constexpr long long kWgradScratchBlocks = 296;   // blocks (two per SM) that walk the channels when rows do not fit in shared memory
+// bytes of global scratch launch_conv_wgrad needs (0 when three complex rows of N fit in shared memory)
+long long conv_wgrad_scratch_bytes(long long N, long long H);
+cudaError_t launch_conv_wgrad(const ConvShape& s, bool bf16_io, const void* x, const void* g, float* dk, void* scratch, long long scratch_bytes,
+                              cudaStream_t st);
 // out[b][c][r] = in[b][r][c] for nblocks blocks of rows x cols elements (fp32 or bf16)
 cudaError_t launch_blocks_transpose(const void* in, void* out, long long nblocks, int rows, int cols, bool bf16, cudaStream_t st);
 // dL[N1][N2][N2], dR[N2][N1][N1] (fp32) of sum_t <M x_t, g_t>; ws: T*N floats (4 launches)

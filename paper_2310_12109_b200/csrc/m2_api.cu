@@ -240,7 +240,8 @@ int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t 
 
 int64_t m2_conv_bwd_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H) {
     if (!plan || B < 0 || H < 0) return -1;
-    return m2u::conv_wgrad_workspace_bytes(plan, B, H);
+    const int64_t umma = m2u::conv_wgrad_workspace_bytes(plan, B, H), generic = m2g::conv_wgrad_scratch_bytes(plan->N, H);
+    return umma > generic ? umma : generic;
 }
 
 int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const void* g_dev, float* dk_dev, int64_t B, int64_t H,
@@ -266,7 +267,7 @@ int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const
         }
         if (st != M2_ERR_UNSUPPORTED) return st;
     }
-    const cudaError_t e = m2g::launch_conv_wgrad(s, plan->dtype == M2_BF16, x_dev, g_dev, dk_dev, (cudaStream_t)stream);
+    const cudaError_t e = m2g::launch_conv_wgrad(s, plan->dtype == M2_BF16, x_dev, g_dev, dk_dev, ws_dev, ws_bytes, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;
     plan->last_kernel = "conv_wgrad_generic";

@@ -217,6 +217,19 @@ def _side_backward(torch, M, synth, peaks, reps, bf):
         res[name + "_kernel"] = plan.last_kernel()
     out["config2_backward"] = res
     plan.close()
+    del x, g, dx, ws
+    B4, H4, n4 = 4, 1024, 16384
+    c = synth.config4(B=B4, H=H4, n=n4)
+    plan = M.Plan((32, 32, 32), dtype=M.M2_BF16, device=torch.cuda.current_device())
+    x = bf(c["x"])
+    g = bf(synth.round_bf16(synth.normal(synth.stream_id(12, 2), c["x"].shape)))
+    ws = torch.empty(int(M.lib().m2_conv_bwd_workspace_bytes(plan.handle, B4, H4)), dtype=torch.uint8, device="cuda")
+    f_dk = lambda i: M.m2_monarch_conv_bwd_kernel(plan, x, g, M.M2_CAUSAL, ws=ws)  # noqa: E731
+    time_launches(f_dk, 2, torch)
+    out["config4_backward"] = {"dk_ms": time_launches(f_dk, reps, torch) / reps, "dk_kernel": plan.last_kernel(),
+                               "note": "dx = the forward kernel with the conjugated spectrum (same time as the forward pass)"}
+    plan.close()
+    del x, g, ws
     T, b = 16384, 64
     c = synth.config3(T=T, b=b)
     plan = M.Plan((b, b), dtype=M.M2_BF16, device=torch.cuda.current_device())

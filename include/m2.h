@@ -105,9 +105,12 @@ int32_t m2_spectrum_conjugate(const m2_plan* plan, const void* kf_in_dev, int64_
  * means this plan has no kernel that uses one).  With it, plans the tensor-core path covers (bf16, N = 512 = 32 x 16)
  * run both forward transforms and the products conj(M x) (.) M g on the tensor cores (intermediates rounded to bf16
  * like the forward pass), 8 batch rows at a time, and a CUDA-core kernel adds the groups in order and applies M^-1 in
- * fp32.  Otherwise everything runs on the CUDA cores in fp32, one thread block per channel with its three complex rows in
- * shared memory (N up to 8192) or, for longer rows (e.g. N = 32768), in the workspace, which is then required
- * (M2_ERR_UNSUPPORTED without it).  All paths are deterministic.  (The paper trains through the operator, Sec. 5, without writing the
+ * fp32; for N = 32768 = 32^3 (causal, n = 16384) the order-3 convolution kernel is run twice (the row pairs' conjugated
+ * spectra, then the convolution of the g pairs with them) and the pairs' rows are added.  Otherwise, or with a workspace
+ * too small for those, everything runs on the CUDA cores in fp32, one thread block per channel with its three complex
+ * rows in shared memory (N up to 8192) or, for longer rows, in the workspace (at least 24 N bytes per channel for up to
+ * 296 channels; M2_ERR_UNSUPPORTED without it).  m2_conv_bwd_workspace_bytes returns the largest of these needs.  All
+ * paths are deterministic.  (The paper trains through the operator, Sec. 5, without writing the
  * backward pass out.) */
 int64_t m2_conv_bwd_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H);
 int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const void* g_dev, float* dk_dev, int64_t B,

@@ -31,6 +31,11 @@ void destroy_tables(m2_plan* plan);
 cudaError_t relayout_spectrum(const m2_plan* plan, void* kf, int64_t H, cudaStream_t stream);
 int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
                  int32_t mode, cudaStream_t stream);
+// kernel gradient dk[H][16384] (fp32) through the same kernel: the row pairs' conjugated spectra, then the convolution of the
+// g pairs with them, then the sum over a channel's pairs; ws: conv_wgrad_workspace_bytes(plan, B, H) bytes
+int64_t conv_wgrad_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H);
+int32_t conv_wgrad(const m2_plan* plan, const void* x, const void* g, float* dk, int64_t B, int64_t H, int64_t n, int32_t mode, void* ws,
+                   cudaStream_t stream);
 }  // namespace m2u3
 
 namespace m2u {

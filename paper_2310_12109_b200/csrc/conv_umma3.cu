@@ -153,9 +153,15 @@ __device__ __forceinline__ void load_pair(uint32_t s_x, const __nv_bfloat16* xa,
     cp_async_commit();
 }
 
+// MODE 0: the convolution.  kf_per_pair != 0: the spectrum block is selected by the row pair instead of by the channel (the
+//         kernel-gradient path: every pair is multiplied by its own conj(M x) / N).
+// MODE 1: only the forward transform: conj(M (xa + i xb)) / N of every row pair is written to spec_out in the layout hand-off 3
+//         reads (pair index in place of the channel); no output rows.
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* __restrict__ x, const float4* __restrict__ kfu,
-               const uint4* __restrict__ consts, const float2* __restrict__ tn, int B, int H, int32_t* __restrict__ status) {
+               const uint4* __restrict__ consts, const float2* __restrict__ tn, int B, int H, int32_t* __restrict__ status,
+               int kf_per_pair, float4* __restrict__ spec_out) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x;
     const int wg = tid >> 7, t = tid & 127, warp = t >> 5;
@@ -224,11 +230,12 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
         // the pair's input has landed (every thread waits for its own copies, then the block syncs)
         cp_async_wait_all();
         M2_STAGE_SYNC()
+        const int kidx = kf_per_pair ? pr_i : h;   // which 256 KB spectrum block this pair is multiplied by
         // pull this pair's 256 KB of spectrum towards L2 now; hand-off 3 reads it five stages later
-        if ((t & 7) == 0) {
+        if (MODE == 0 && (t & 7) == 0) {
 #pragma unroll 1
             for (int jj = 0; jj < 2; ++jj) {
-                const float4* kp = kfu + ((size_t)(h * 8 + wg + 4 * jj) * 16) * 128 + t;
+                const float4* kp = kfu + ((size_t)(kidx * 8 + wg + 4 * jj) * 16) * 128 + t;
 #pragma unroll
                 for (int q = 0; q < 16; ++q) asm volatile("prefetch.global.L2 [%0];" ::"l"(kp + q * 128));
             }
@@ -326,8 +333,26 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
         }
         // ---- h3: spectrum multiply (k_f holds 1/N); A4 K-major: row = lane, K = (c, k3).  All of a tile's spectrum
         //      values are requested before the wait for the UMMAs, the second tile's while the first is worked on. ------
+        if constexpr (MODE == 1) {
+            // the spectrum of the pair, conjugated and scaled by 1 / N, in the layout hand-off 3 reads it back in
+            M2_WAIT_MMA()
+            if (ok) {
+                const float inv = 1.0f / (float)kN;
+#pragma unroll 1
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int j = wg + 4 * jj;
+                    float4* dst = spec_out + ((size_t)(pr_i * 8 + j) * 16) * 128 + t;
+                    float re[32], im[32];
+                    load_tile(t_lane + j * 64, re, im);
+#pragma unroll
+                    for (int q = 0; q < 16; ++q)
+                        dst[q * 128] = make_float4(re[2 * q] * inv, re[2 * q + 1] * inv, -im[2 * q] * inv, -im[2 * q + 1] * inv);
+                }
+            }
+            continue;   // the next pair's first barrier orders these accumulator reads before its UMMAs
+        }
         {
-            const float4* kp0 = kfu + ((size_t)(h * 8 + wg) * 16) * 128 + t;
+            const float4* kp0 = kfu + ((size_t)(kidx * 8 + wg) * 16) * 128 + t;
             float4 w[16];
 #pragma unroll
             for (int q = 0; q < 16; ++q) w[q] = __ldg(kp0 + q * 128);
@@ -564,7 +589,8 @@ cudaError_t create_tables(m2_plan* pl) {
     if (e == cudaSuccess) e = cudaMemcpy(tb->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMalloc(&tb->d_tn, tn.size() * sizeof(float));
     if (e == cudaSuccess) e = cudaMemcpy(tb->d_tn, tn.data(), tn.size() * sizeof(float), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv32k_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv32k_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv32k_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) {
         if (tb->d_const) cudaFree(tb->d_const);
         if (tb->d_tn) cudaFree(tb->d_tn);
@@ -620,11 +646,74 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, conv32k_kernel, my, (const __nv_bfloat16*)x, kfu, (const uint4*)tb->d_const, (const float2*)tb->d_tn,
-                           (int)B, (int)H, pl->d_status) != cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, conv32k_kernel<0>, my, (const __nv_bfloat16*)x, kfu, (const uint4*)tb->d_const, (const float2*)tb->d_tn,
+                           (int)B, (int)H, pl->d_status, 0, (float4*)nullptr) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o3_32k";
     pl->launches += 1;
+    return M2_OK;
+}
+
+// dk[h][i] = sum over the row pairs of channel h of the pair's first output row (fp32 sum of bf16 values, pairs in index order)
+__global__ void wgrad_pair_sum_kernel(const __nv_bfloat16* __restrict__ rows, float* __restrict__ dk, int B, int H, long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 16384
+    if (e >= total) return;
+    const long long h = e >> 14, i = e & 16383;
+    float acc = 0.f;
+    for (int b = 0; b < B; b += 2) acc += __bfloat162float(rows[((long long)b * H + h) * 16384 + i]);
+    dk[e] = acc;
+}
+
+// Kernel gradient on the tensor cores: with z_p = xa + i xb and w_p = ga + i gb for the row pairs p of a channel,
+//   M^-1( conj(M z_p) (.) M w_p ) = (corr(xa, ga) + corr(xb, gb)) + i (corr(xa, gb) - corr(xb, ga)),
+// both parts real sequences, so the first output row of the convolution kernel run on the g pairs with the spectrum
+// conj(M z_p) / N is the pair's contribution to dk; the pairs of a channel are then added.
+// ws: spectra [pairs][256 KB] | output rows [B][H][16384] bf16.
+int64_t conv_wgrad_workspace_bytes(const m2_plan* pl, int64_t B, int64_t H) {
+    if (!pl->umma || !covered(pl)) return 0;
+    return H * ((B + 1) / 2) * 262144 + B * H * 16384 * 2;
+}
+
+int32_t conv_wgrad(const m2_plan* pl, const void* x, const void* g, float* dk, int64_t B, int64_t H, int64_t n, int32_t mode, void* ws,
+                   cudaStream_t stream) {
+    if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (mode != M2_CAUSAL || n != 16384 || B == 0) return M2_ERR_UNSUPPORTED;
+    Tables* tb = reinterpret_cast<Tables*>(pl->umma);
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long pairs = H * ((B + 1) / 2);
+    if (pairs > 0x7ffffff) return M2_ERR_UNSUPPORTED;
+    float4* spec = reinterpret_cast<float4*>(ws);
+    __nv_bfloat16* rows = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(ws) + pairs * 262144);
+    alignas(64) CUtensorMap my;
+    {
+        const cuuint64_t gdim[2] = {32, (cuuint64_t)(B * H * 512)};
+        const cuuint64_t gstr[1] = {64};
+        const cuuint32_t box[2] = {32, 256};
+        if (!tma_host::encode_sw64_bf16(&my, rows, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(pairs < sms ? pairs : sms));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, conv32k_kernel<1>, my, (const __nv_bfloat16*)x, (const float4*)nullptr, (const uint4*)tb->d_const,
+                           (const float2*)tb->d_tn, (int)B, (int)H, pl->d_status, 1, spec) != cudaSuccess)
+        return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, conv32k_kernel<0>, my, (const __nv_bfloat16*)g, (const float4*)spec, (const uint4*)tb->d_const,
+                           (const float2*)tb->d_tn, (int)B, (int)H, pl->d_status, 1, (float4*)nullptr) != cudaSuccess)
+        return M2_ERR_CUDA;
+    const long long total = H * 16384;
+    wgrad_pair_sum_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(rows, dk, (int)B, (int)H, total);
+    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
+    pl->last_kernel = "conv_wgrad_umma_o3_32k";
+    pl->launches += 3;
     return M2_OK;
 }
 

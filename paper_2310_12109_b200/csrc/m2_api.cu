@@ -240,7 +240,8 @@ int32_t m2_spectrum_to_natural(const m2_plan* plan, const void* kf_dev, int64_t 
 
 int64_t m2_conv_bwd_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H) {
     if (!plan || B < 0 || H < 0) return -1;
-    const int64_t umma = m2u::conv_wgrad_workspace_bytes(plan, B, H), generic = m2g::conv_wgrad_scratch_bytes(plan->N, H);
+    const int64_t u2 = m2u::conv_wgrad_workspace_bytes(plan, B, H), u3 = m2u3::conv_wgrad_workspace_bytes(plan, B, H);
+    const int64_t umma = u2 > u3 ? u2 : u3, generic = m2g::conv_wgrad_scratch_bytes(plan->N, H);
     return umma > generic ? umma : generic;
 }
 
@@ -265,6 +266,11 @@ int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const
             plan->launches += 1;
             return M2_OK;
         }
+        if (st != M2_ERR_UNSUPPORTED) return st;
+    }
+    const int64_t need3 = m2u3::conv_wgrad_workspace_bytes(plan, B, H);
+    if (need3 > 0 && B > 0 && ws_dev && ws_bytes >= need3) {   // N = 32768: the order-3 tensor-core kernel, three launches
+        st = m2u3::conv_wgrad(plan, x_dev, g_dev, dk_dev, B, H, n, mode, ws_dev, (cudaStream_t)stream);
         if (st != M2_ERR_UNSUPPORTED) return st;
     }
     const cudaError_t e = m2g::launch_conv_wgrad(s, plan->dtype == M2_BF16, x_dev, g_dev, dk_dev, ws_dev, ws_bytes, (cudaStream_t)stream);

@@ -303,7 +303,7 @@ def test_conv_input_gradient(cfg, kernel):
 
 
 @pytest.mark.parametrize("cfg,use_ws", [("c1", True), ("c2", False), ("c2", True), ("c2big", True), ("c2causal", True),
-                                        ("c2causal256", True), ("small3", True), ("c4small", True)])
+                                        ("c2causal256", True), ("small3", True), ("c4small", True), ("c4odd", True), ("c4cuda", True)])
 def test_conv_kernel_gradient(cfg, use_ws):
     if cfg == "c1":
         c, causal, dtype, tol = synth.config1(), True, M.M2_FP32, 1e-5
@@ -319,8 +319,12 @@ def test_conv_kernel_gradient(cfg, use_ws):
         c = synth.config2(B=5, H=7)
         c = dict(c, x=c["x"][..., :256].copy(), k=c["k"][..., :256].copy())
         causal, dtype, tol = True, M.M2_BF16, 1e-5
-    elif cfg == "c4small":   # N = 32768: rows too long for shared memory, the CUDA-core kernel works in the workspace
-        c, causal, dtype, tol = synth.config4(B=2, H=3), True, M.M2_BF16, 1e-5
+    elif cfg == "c4small":   # N = 32768 on the tensor cores: pair spectra, convolution of the g pairs, sum over the pairs
+        c, causal, dtype, tol = synth.config4(B=4, H=3), True, M.M2_BF16, 1e-5
+    elif cfg == "c4odd":     # an odd batch: the last pair has one row
+        c, causal, dtype, tol = synth.config4(B=3, H=2), True, M.M2_BF16, 1e-5
+    elif cfg == "c4cuda":    # N = 32768 with a workspace that only the CUDA-core kernel can use (rows too long for shared memory)
+        c, causal, dtype, tol = synth.config4(B=8, H=1), True, M.M2_BF16, 1e-5
     else:
         c = dict(x=synth.round_bf16(synth.normal(synth.stream_id(9, 0), (3, 4, 32))), dims=(4, 4, 4))
         causal, dtype, tol = True, M.M2_BF16, 1e-5
@@ -328,11 +332,15 @@ def test_conv_kernel_gradient(cfg, use_ws):
     tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
     x = c["x"].astype(np.float64)
     gup = synth.round_bf16(synth.normal(synth.stream_id(9, 1), x.shape)).astype(np.float64)   # upstream gradient
+    ws = None
+    if cfg == "c4cuda":   # 3 complex rows of one channel: less than the tensor-core path needs for 4 pairs
+        ws = torch.empty(3 * 32768 * 8, dtype=torch.uint8, device="cuda")
     dk = M.m2_monarch_conv_bwd_kernel(plan, dev(x.astype(np.float32), tdt), dev(gup.astype(np.float32), tdt),
-                                      M.M2_CAUSAL if causal else M.M2_CIRCULAR, use_workspace=use_ws)
+                                      M.M2_CAUSAL if causal else M.M2_CIRCULAR, ws=ws, use_workspace=use_ws)
     torch.cuda.synchronize()
-    umma = use_ws and cfg in ("c2", "c2big", "c2causal256")
-    assert plan.device_status() == 0 and plan.last_kernel() == ("conv_wgrad_umma_o2_512" if umma else "conv_wgrad_generic")
+    umma = use_ws and cfg in ("c2", "c2big", "c2causal256", "c4small", "c4odd")
+    want = "conv_wgrad_generic" if not umma else "conv_wgrad_umma_o3_32k" if cfg.startswith("c4") else "conv_wgrad_umma_o2_512"
+    assert plan.device_status() == 0 and plan.last_kernel() == want
     ref = O.monarch_conv_kernel_grad(x, gup, c["dims"], causal)
     check(host(dk), ref, TOL_BF16 if umma else tol, "kernel gradient " + cfg)   # tensor-core path: bf16 intermediates
     plan.close()

@@ -558,6 +558,47 @@ def test_runs_are_bit_identical_and_stay_in_bounds():
     plan.close()
 
 
+def test_new_kernels_are_bit_identical_and_stay_in_bounds():
+    """Column-layout Monarch, weight gradients and kernel gradient: two runs give the same bits; nothing is written outside the outputs."""
+    torch.manual_seed(7)
+    b, d, Bt = 128, 192, 2
+    N = b * b
+    plan = M.Plan((b, b), dtype=M.M2_BF16, device=0)
+    L = (torch.randn(b, b, b, device="cuda") / b ** 0.5).to(torch.bfloat16)
+    R = (torch.randn(b, b, b, device="cuda") / b ** 0.5).to(torch.bfloat16)
+    X = torch.randn(Bt, N, d, device="cuda").to(torch.bfloat16)
+    K = torch.randn(N, d, device="cuda").to(torch.bfloat16)
+    pad = 8192
+    buf = torch.full((X.numel() + 2 * pad,), 7.0, dtype=torch.bfloat16, device="cuda")
+    Y = buf[pad:pad + X.numel()].view_as(X)
+    M.m2_monarch_cols(plan, X, L, R, K, M.M2_ACT_RELU, Y=Y)
+    Y1 = Y.clone()
+    M.m2_monarch_cols(plan, X, L, R, K, M.M2_ACT_RELU, Y=Y)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and torch.equal(Y1, Y)
+    assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + X.numel():] == 7.0).all())
+    plan.close()
+    plan = M.Plan((64, 64), dtype=M.M2_BF16, device=0)
+    T = 700
+    X = torch.randn(T, 4096, device="cuda").to(torch.bfloat16)
+    G = torch.randn(T, 4096, device="cuda").to(torch.bfloat16)
+    L = (torch.randn(64, 64, 64, device="cuda") / 8).to(torch.bfloat16)
+    R = (torch.randn(64, 64, 64, device="cuda") / 8).to(torch.bfloat16)
+    a = M.m2_monarch_matmul_bwd_weights(plan, X, G, L, R)
+    b2 = M.m2_monarch_matmul_bwd_weights(plan, X, G, L, R)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and torch.equal(a[0], b2[0]) and torch.equal(a[1], b2[1])
+    plan.close()
+    plan = M.Plan((32, 16), dtype=M.M2_BF16, device=0)
+    x = torch.randn(24, 40, 512, device="cuda").to(torch.bfloat16)
+    g = torch.randn(24, 40, 512, device="cuda").to(torch.bfloat16)
+    d1 = M.m2_monarch_conv_bwd_kernel(plan, x, g, M.M2_CIRCULAR)
+    d2 = M.m2_monarch_conv_bwd_kernel(plan, x, g, M.M2_CIRCULAR)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "conv_wgrad_umma_o2_512" and torch.equal(d1, d2)
+    plan.close()
+
+
 def test_host_buffer_entry_points():
     c = synth.config2(B=2, H=8)
     plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)

@@ -428,7 +428,7 @@ static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols 
               "per-CTA budgets");
 
 __global__ void __launch_bounds__(kThreadsP, 1)
-conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restrict__ y,
+conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
                int32_t* __restrict__ status, int* __restrict__ sched) {
     extern __shared__ __align__(1024) unsigned char smem_all[];
@@ -457,6 +457,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __rest
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_x);
+        prefetch_tensormap(&map_y);
     }
     // Programmatic dependent launch: the next kernel on the stream may start its CTAs as this grid's CTAs leave
     // their SMs; everything above the wait below touches only plan-owned constants and this CTA's own resources.
@@ -516,6 +517,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __rest
         if (leader) {
             ok = mbar_wait(bar_x, ph_x);
             x_pending = false;
+            tma_store_wait_read0();   // the previous unit's output stores have read the operand buffer (their staging area)
             if (ok) {
                 tc_fence_after();
 #pragma unroll
@@ -688,8 +690,9 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __rest
                          smem_desc(s_all + P_OFF_B4 + s * 256, 128, 1024), ID_S1I, s > 0);
             umma_commit(bar_mma);
         }
-        // ---- h4: round and store: lane (r, n2) holds y[r][n1*16 + n2] for all n1; a warp writes two full
-        //      32-byte sectors per instruction --------------------------------------------------------
+        // ---- h4: round and stage: lane (r, n2) holds y[r][n1*16 + n2] for all n1 of the real-part row and of the
+        //      imaginary-part row; the operand buffer (free now) takes the two boxes [8 rows][32 n1][16 n2] in the
+        //      32-byte-swizzled image of the TMA stores (16-byte chunk XOR bit 7 of the address) ---------------
         ok = mbar_wait(bar_mma, ph_m);
         ph_m ^= 1;
         tc_fence_after();
@@ -703,19 +706,23 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __rest
                 tmem_ld_wait();
 #pragma unroll
                 for (int g = 0; g < 4; ++g) tmem_ld_fence8(v + 8 * g);
-                if (b0 + kRows * c + r < B) {
-                    __nv_bfloat16* yr = y + ((size_t)(b0 + kRows * c + r) * H + h) * n + n2;
+                unsigned char* st = smem + P_G_A + c * 8192 + r * 1024 + (n2 & 7) * 2;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (i < n1_valid) yr[i * 16] = __float2bfloat16_rn(v[i]);
-                }
+                for (int i = 0; i < 32; ++i)
+                    *reinterpret_cast<__nv_bfloat16*>(st + i * 32 + (((n2 >> 3) ^ ((i >> 2) & 1)) << 4)) = __float2bfloat16_rn(v[i]);
             }
         }
         if (leader) *next_slot = un2;
+        fence_proxy_async();   // the staged rows are read by the TMA stores
         tc_fence_before();
         if (group_sync_or(wg, !ok, abort_flag)) {
             aborted = true;
             break;
+        }
+        if (leader) {   // rows past the batch and positions past n are clipped by the tensor map
+            tma_store_4d(&map_y, s_base + P_G_A, 0, 0, h, b0);
+            if (b0 + kRows < B) tma_store_4d(&map_y, s_base + P_G_A + 8192, 0, 0, h, b0 + kRows);
+            tma_store_commit();
         }
         u = un;
         un = *next_slot;   // written by thread 0 before the barrier above
@@ -724,6 +731,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __rest
     if (leader) {
         if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
         if (x_pending) mbar_wait(bar_x, ph_x);
+        tma_store_wait_read0();
         __threadfence();
         if (atomicAdd(sched + 1, 1) == ustride - 1) {   // last pipeline out: reset the scheduler words
             sched[0] = 0;
@@ -1087,6 +1095,14 @@ void destroy_tables(m2_plan* pl) {
 }
 
 // x / y viewed as [b][h][n1][n2] with n2 innermost; box = 8 of the 16 n2, all 32 n1, one h, 8 b.
+// y viewed the same way, whole rows of 16 n2: box = 16 n2 (32 bytes, 32-byte swizzle), 32 n1, one h, 8 b
+static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
+    const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
+    const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
+    const cuuint32_t box[4] = {16, 32, 1, (cuuint32_t)kRows};
+    return tma_host::encode_sw32_bf16(map, ptr, 4, gdim, gstr, box);
+}
+
 static bool make_map(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
     const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
     const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
@@ -1132,8 +1148,14 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, pairs ? conv512p_kernel : conv512_kernel, mx, (__nv_bfloat16*)y, kfu,
-                           (const uint4*)(pairs ? t->d_const_p : t->d_const), (int)B, (int)H, (int)n, pl->d_status, t->d_sched) != cudaSuccess)
+    if (pairs) {
+        alignas(64) CUtensorMap my;
+        if (!make_map_rows32(&my, y, B, H, n)) return M2_ERR_UNSUPPORTED;
+        if (cudaLaunchKernelEx(&cfg, conv512p_kernel, mx, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H, (int)n,
+                               pl->d_status, t->d_sched) != cudaSuccess)
+            return M2_ERR_CUDA;
+    } else if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n,
+                                  pl->d_status, t->d_sched) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "conv_umma_o2_512";
     pl->launches += 1;

@@ -517,7 +517,6 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         if (leader) {
             ok = mbar_wait(bar_x, ph_x);
             x_pending = false;
-            tma_store_wait_read0();   // the previous unit's output stores have read the operand buffer (their staging area)
             if (ok) {
                 tc_fence_after();
 #pragma unroll
@@ -526,6 +525,9 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     for (int s = 0; s < k1steps; ++s)
                         umma_f16(tmem + T1, smem_desc(s_base + P_G_X + c * 8192 + s * 256, 128, 512),
                                  smem_desc(s_all + P_OFF_B1 + (2 * c + s) * 256, 128, 1024), ID_S1, (c | s) > 0);
+                // S1 does not touch the operand buffer, hand-off 1 (which waits for this commit) overwrites it: the previous
+                // unit's output stores must have read their staging area by then, and they do so while S1 runs
+                tma_store_wait_read0();
                 umma_commit(bar_mma);
             }
         }

@@ -420,7 +420,7 @@ constexpr int P_OFF_B1 = 0, P_OFF_B2 = 8192, P_OFF_B3 = 10240, P_OFF_B4 = 12288,
 constexpr int P_CONST_BYTES = 28672;
 constexpr int P_OFF_BAR = P_CONST_BYTES;          // per group 32 B; tmem ptr at +512
 constexpr int P_OFF_GROUP = P_OFF_BAR + 1024;
-constexpr int P_G_X = 0;                          // re tile 8192 | im tile 8192 (2 boxes [n2hi][r][n1][8] each)
+constexpr int P_G_X = 0;                          // re tile 8192 | im tile 8192 (one box [r][n1][16 n2] each, 32-byte swizzled)
 constexpr int P_G_A = 16384;                      // A2 / A3 / A4   16384
 constexpr int P_GROUP_BYTES = 32768;
 constexpr int P_SMEM_BYTES = P_OFF_GROUP + kGroupsP * P_GROUP_BYTES;
@@ -473,14 +473,13 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // reset of the scheduler words, readers of y) is complete and visible from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // rows b0 .. b0+7 are the real parts and rows b0+8 .. b0+15 the imaginary parts of the unit's 8 complex rows (boxes
-    // past the end of the batch read zeros)
+    // past the end of the batch read zeros).  A box is [8 rows][32 n1][16 n2] with 32-byte rows, 32-byte swizzled: as it lies
+    // it is the M-major operand of S1 with M = (row, n2) -- 16-element M blocks 1 KB apart, groups of 8 n1 256 B apart.
     auto load_unit = [&](int v) {
         mbar_expect_tx(bar_x, 16384);
         const int hh = v % H, bb = (v / H) * 2 * kRows;
         tma_load_4d(s_base + P_G_X, &map_x, 0, 0, hh, bb, bar_x);
-        tma_load_4d(s_base + P_G_X + 4096, &map_x, 8, 0, hh, bb, bar_x);
         tma_load_4d(s_base + P_G_X + 8192, &map_x, 0, 0, hh, bb + kRows, bar_x);
-        tma_load_4d(s_base + P_G_X + 12288, &map_x, 8, 0, hh, bb + kRows, bar_x);
         x_pending = true;
     };
     if (leader && u < units0) {   // first loads
@@ -523,7 +522,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 for (int c = 0; c < 2; ++c)   // K = (re | im part of the input) x n1
 #pragma unroll 1
                     for (int s = 0; s < k1steps; ++s)
-                        umma_f16(tmem + T1, smem_desc(s_base + P_G_X + c * 8192 + s * 256, 128, 512),
+                        umma_f16(tmem + T1, smem_desc_sw32(s_base + P_G_X + c * 8192 + s * 512, 1024, 256),
                                  smem_desc(s_all + P_OFF_B1 + (2 * c + s) * 256, 128, 1024), ID_S1, (c | s) > 0);
                 // S1 does not touch the operand buffer, hand-off 1 (which waits for this commit) overwrites it: the previous
                 // unit's output stores must have read their staging area by then, and they do so while S1 runs
@@ -541,7 +540,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             load_unit(un);
         }
         if (ok) {
-            const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
+            const int r = tid >> 4, n2 = tid & 15, n2hi = n2 >> 3, n2lo = n2 & 7;   // lane = r * 16 + n2: the row order of the input boxes
             const float4* twA = reinterpret_cast<const float4*>(smem_all + P_OFF_TWA) + n2;
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {   // two batches of 16 complex values keep the register count down
@@ -757,7 +756,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 // kernel adds the b groups in order and applies M^-1 in fp32 (one block per channel).
 constexpr int kGroupsW = 4;
 constexpr int kThreadsW = 128 * kGroupsW;
-constexpr int WG_X = 0;              // x tile 8192 | g tile 8192 (2 boxes [n2hi][r][n1][8] each)
+constexpr int WG_X = 0;              // x tile 8192 | g tile 8192 (one box [r][n1][16 n2] each, 32-byte swizzled)
 constexpr int WG_A = 16384;          // A2 of x 16384 | A2 of g 16384; afterwards the four warps' sums [warp][k2][33 k1] float2
 constexpr int W_GROUP_BYTES = 49152;
 constexpr int W_SMEM_BYTES = OFF_GROUP + kGroupsW * W_GROUP_BYTES;
@@ -798,10 +797,8 @@ convwgrad512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     auto load_unit = [&](int v) {   // both tiles of unit v, one barrier phase
         mbar_expect_tx(bar_x, 16384);
         const int hh = v % H, bb = (v / H) * kRows;
-        tma_load_4d(s_base + WG_X, &map_x, 0, 0, hh, bb, bar_x);
-        tma_load_4d(s_base + WG_X + 4096, &map_x, 8, 0, hh, bb, bar_x);
+        tma_load_4d(s_base + WG_X, &map_x, 0, 0, hh, bb, bar_x);          // boxes [8 rows][32 n1][16 n2], 32-byte swizzled
         tma_load_4d(s_base + WG_X + 8192, &map_g, 0, 0, hh, bb, bar_x);
-        tma_load_4d(s_base + WG_X + 12288, &map_g, 8, 0, hh, bb, bar_x);
         x_pending = true;
     };
     if (leader && u < units) load_unit(u);
@@ -830,7 +827,7 @@ convwgrad512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 for (int tt = 0; tt < 2; ++tt)
 #pragma unroll 1
                     for (int s = 0; s < k1steps; ++s)
-                        umma_f16(tmem + 64 * tt, smem_desc(s_base + WG_X + tt * 8192 + s * 256, 128, 512),
+                        umma_f16(tmem + 64 * tt, smem_desc_sw32(s_base + WG_X + tt * 8192 + s * 512, 1024, 256),
                                  smem_desc(s_all + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
                 umma_commit(bar_mma);
             }
@@ -842,7 +839,7 @@ convwgrad512_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         if (leader && ok && un < units) load_unit(un);   // the tiles are free
         // ---- h1: twiddle, A2 of x and of g ---------------------------------------------------------------
         if (ok) {
-            const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
+            const int r = tid >> 4, n2 = tid & 15, n2hi = n2 >> 3, n2lo = n2 & 7;   // lane = r * 16 + n2: the row order of the input boxes
             const float4* twA = reinterpret_cast<const float4*>(smem_all + OFF_TWA) + n2;
 #pragma unroll 1
             for (int tt = 0; tt < 2; ++tt)
@@ -1097,7 +1094,7 @@ void destroy_tables(m2_plan* pl) {
 }
 
 // x / y viewed as [b][h][n1][n2] with n2 innermost; box = 8 of the 16 n2, all 32 n1, one h, 8 b.
-// y viewed the same way, whole rows of 16 n2: box = 16 n2 (32 bytes, 32-byte swizzle), 32 n1, one h, 8 b
+// x / y viewed the same way, whole rows of 16 n2: box = 16 n2 (32 bytes, 32-byte swizzle), 32 n1, one h, 8 b
 static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
     const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
     const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
@@ -1127,8 +1124,6 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
     Tables* t = reinterpret_cast<Tables*>(pl->umma);
-    alignas(64) CUtensorMap mx;
-    if (!make_map(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -1153,12 +1148,18 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     if (pairs) {
         alignas(64) CUtensorMap my;
         if (!make_map_rows32(&my, y, B, H, n)) return M2_ERR_UNSUPPORTED;
-        if (cudaLaunchKernelEx(&cfg, conv512p_kernel, mx, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H, (int)n,
+        alignas(64) CUtensorMap mx32;   // the row-pair kernel reads whole 32-byte rows of 16 n2
+        if (!make_map_rows32(&mx32, x, B, H, n)) return M2_ERR_UNSUPPORTED;
+        if (cudaLaunchKernelEx(&cfg, conv512p_kernel, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H, (int)n,
                                pl->d_status, t->d_sched) != cudaSuccess)
             return M2_ERR_CUDA;
-    } else if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n,
-                                  pl->d_status, t->d_sched) != cudaSuccess)
-        return M2_ERR_CUDA;
+    } else {
+        alignas(64) CUtensorMap mx;
+        if (!make_map(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
+        if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n, pl->d_status,
+                               t->d_sched) != cudaSuccess)
+            return M2_ERR_CUDA;
+    }
     pl->last_kernel = "conv_umma_o2_512";
     pl->launches += 1;
     return M2_OK;
@@ -1175,7 +1176,7 @@ int32_t conv_wgrad_partials(const m2_plan* pl, const void* x, const void* g, voi
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
     Tables* t = reinterpret_cast<Tables*>(pl->umma);
     alignas(64) CUtensorMap mx, mg;
-    if (!make_map(&mx, x, B, H, n) || !make_map(&mg, g, B, H, n)) return M2_ERR_UNSUPPORTED;
+    if (!make_map_rows32(&mx, x, B, H, n) || !make_map_rows32(&mg, g, B, H, n)) return M2_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

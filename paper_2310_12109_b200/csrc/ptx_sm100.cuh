@@ -170,6 +170,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     return smem_desc(addr, lbo_bytes, sbo_bytes) | ((uint64_t)2 << 61);
 }
+// Same with the 32-byte swizzle (16-byte chunk index XOR bit 7 of the address, atoms of 8 rows x 32 B), MN-major: a row = 16
+// consecutive M/N elements of one K index; LBO = step between 16-element M/N blocks, SBO = step between groups of 8 K indices.
+__device__ __forceinline__ uint64_t smem_desc_sw32(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return smem_desc(addr, lbo_bytes, sbo_bytes) | ((uint64_t)6 << 61);
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, dense.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
     return (1u << 4)                          // D format: fp32

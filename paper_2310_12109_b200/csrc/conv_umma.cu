@@ -10,7 +10,7 @@
 // digit that is NOT being contracted, so each thread owns whole complex numbers (re and im sit in
 // different TMEM columns of its lane) and the twiddle / spectrum multiplies are thread-local fp32:
 //
-//   S1   D1[(r,n2)][(c,k1)]   = sum_n1  x[r][n1][n2] * F32[(c,k1)][n1]           A: M-major (TMA tile)
+//   S1   D1[(r,n2)][(c,k1)]   = sum_n1  x[r][n1][n2] * F32[(c,k1)][n1]           A: M-major, 32B-swizzled (the TMA box as it lies)
 //   h1   twiddle w_N^{n2 k1} (fp32), round to bf16, write A2[(r,k1)][(c,n2)]         M-major
 //   S2   D2[(r,k1)][(c,k2)]   = sum_(c,n2) A2 * F16                              two M=128 halves
 //   h2   multiply by k_f[h][k1][k2] (fp32, 1/N folded in), write A3[(r,k1)][(c,k2)]  K-major
@@ -52,7 +52,7 @@ constexpr int OFF_B1 = OFF_CONST, OFF_B2 = OFF_B1 + 4096, OFF_B3 = OFF_B2 + 2048
 constexpr int OFF_TWA = OFF_B4 + 4096, OFF_TWB = OFF_TWA + 4096;
 constexpr int OFF_BAR = OFF_CONST + CONST_BYTES;   // per group: bar_x, bar_mma, bar_k, flag (32 B each, up to 16 groups); tmem ptr at +512
 constexpr int OFF_GROUP = OFF_BAR + 1024;   // keeps every group slice 1024-byte aligned
-constexpr int G_X = 0;               // 2 boxes [n2hi][r][n1][8]            8192
+constexpr int G_X = 0;               // one box [r][n1][16 n2], 32-byte swizzled   8192
 constexpr int G_A = 8192;            // A2 / A3 / A4                        16384
 constexpr int G_KF = 24576;          // spectrum row of the unit's channel  4096
 constexpr int GROUP_BYTES = 28672;
@@ -145,7 +145,6 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
     if (leader && u < units0) {   // first loads
         mbar_expect_tx(bar_x, 8192);
         tma_load_4d(s_base + G_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
-        tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, u % H, (u / H) * kRows, bar_x);
         x_pending = true;
         mbar_expect_tx(bar_k, 4096);
         bulk_load(s_base + G_KF, kfu + (size_t)(u % H) * 256, 4096, bar_k);
@@ -185,7 +184,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
                 tc_fence_after();
 #pragma unroll 1
                 for (int s = 0; s < k1steps; ++s)
-                    umma_f16(tmem + T1, smem_desc(s_base + G_X + s * 256, 128, 512),
+                    umma_f16(tmem + T1, smem_desc_sw32(s_base + G_X + s * 512, 1024, 256),
                              smem_desc(s_all + OFF_B1 + s * 256, 128, 512), ID_S1, s > 0);
                 umma_commit(bar_mma);
             }
@@ -199,11 +198,10 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         if (leader && ok && un < units) {   // the x tile is free: fetch the next unit's
             mbar_expect_tx(bar_x, 8192);
             tma_load_4d(s_base + G_X, &map_x, 0, 0, un % H, (un / H) * kRows, bar_x);
-            tma_load_4d(s_base + G_X + 4096, &map_x, 8, 0, un % H, (un / H) * kRows, bar_x);
             x_pending = true;
         }
         if (ok) {
-            const int n2hi = tid >> 6, r = (tid >> 3) & 7, n2lo = tid & 7, n2 = n2hi * 8 + n2lo;
+            const int r = tid >> 4, n2 = tid & 15, n2hi = n2 >> 3, n2lo = n2 & 7;   // lane = r * 16 + n2: the row order of the input box
             const float4* twA = reinterpret_cast<const float4*>(smem_all + OFF_TWA) + n2;
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {   // two batches of 16 complex values keep the register count down
@@ -1093,8 +1091,7 @@ void destroy_tables(m2_plan* pl) {
     pl->umma = nullptr;
 }
 
-// x / y viewed as [b][h][n1][n2] with n2 innermost; box = 8 of the 16 n2, all 32 n1, one h, 8 b.
-// x / y viewed the same way, whole rows of 16 n2: box = 16 n2 (32 bytes, 32-byte swizzle), 32 n1, one h, 8 b
+// x / y viewed as [b][h][n1][n2] with n2 innermost; box = the 16 n2 of a row (32 bytes, 32-byte swizzle), all 32 n1, one h, 8 b
 static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
     const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
     const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
@@ -1102,12 +1099,6 @@ static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_
     return tma_host::encode_sw32_bf16(map, ptr, 4, gdim, gstr, box);
 }
 
-static bool make_map(CUtensorMap* map, const void* ptr, int64_t B, int64_t H, int64_t n) {
-    const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)H, (cuuint64_t)B};
-    const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)H * n * 2};
-    const cuuint32_t box[4] = {8, 32, 1, (cuuint32_t)kRows};
-    return tma_host::encode_bf16(map, ptr, 4, gdim, gstr, box);
-}
 
 // development switch: M2_CONV512_PAIRS=0 in the environment selects the one-row-per-lane kernel for every batch size
 static bool pair_kernel_enabled() {
@@ -1155,7 +1146,7 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
             return M2_ERR_CUDA;
     } else {
         alignas(64) CUtensorMap mx;
-        if (!make_map(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
+        if (!make_map_rows32(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
         if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n, pl->d_status,
                                t->d_sched) != cudaSuccess)
             return M2_ERR_CUDA;

@@ -270,6 +270,23 @@ def _side_operator(torch, M, synth, peaks, reps, bf):
         time_launches(f, 3, torch)
         r = max(reps, 20) if b <= 128 else max(reps, 5)
         ms = time_launches(f, r, torch) / r
+        ms_graph = None
+        if b <= 128:   # the four launches are host-bound at these sizes: also time them replayed from a CUDA graph
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                f(0)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=st):
+                    for _ in range(10):
+                        f(0)
+                g.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(st)
+                for _ in range(10):
+                    g.replay()
+                e1.record(st)
+            torch.cuda.synchronize()
+            ms_graph = e0.elapsed_time(e1) / 100
         fl = 8.0 * N * b * d
         by = 4 * (2 * N * d * 2 + b * b * b * 2) + N * d * 2   # per stage: rows in, rows out, one factor; + the kernel K once
         t_roof = max(fl / (peaks["bf16_tflops_sustained"] * 1e12), by / (peaks["hbm_gbs"] * 1e9))
@@ -277,6 +294,8 @@ def _side_operator(torch, M, synth, peaks, reps, bf):
             "kernel": plan.last_kernel(), "ms": ms, "TFLOPs": fl / (ms * 1e9), "launches_per_call": 4,
             "flop_utilisation_pct": 100 * fl / (ms * 1e9) / peaks["bf16_tflops"], "roofline_frac": t_roof / (ms * 1e-3),
             "paper_flop_utilisation_pct": {"A100": paper[N][0], "RTX4090": paper[N][1]}}
+        if ms_graph is not None:
+            out[f"operator_N{N}"].update({"ms_cuda_graph": ms_graph, "flop_utilisation_pct_cuda_graph": 100 * fl / (ms_graph * 1e9) / peaks["bf16_tflops"]})
         plan.close()
         del W, X, K, Y1, Y2, ws
     # the same operator at N = 4096 with the vectors as rows (tokens contiguous in N): m2_monarch_mix

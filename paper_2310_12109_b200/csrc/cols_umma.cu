@@ -74,7 +74,7 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
     const uint32_t bar_full = s_base + OFF_BAR, bar_empty = bar_full + 24, bar_accf = bar_full + 48, bar_acce = bar_full + 64;
     const uint32_t s_tptr = bar_full + 80;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + 88);
-    const int otiles = (b + 127) / 128, ctiles = d / nc;
+    const int otiles = (b + 127) / 128, ctiles = (d + nc - 1) / nc;   // the last column tile may be ragged: TMA zero-fills / clips it
     const int chunks = b / 64, nq = nc / 64;
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -176,7 +176,7 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
                 const uint4* krow = reinterpret_cast<const uint4*>(Kmul + ((size_t)o * b + j) * d + c0);   // K is shared by the batch
 #pragma unroll
                 for (int e = 0; e < 32; ++e)
-                    if (e < nq * 8) kreg[e] = __ldg(krow + e);
+                    if (e < nq * 8) kreg[e] = c0 + 8 * e < d ? __ldg(krow + e) : make_uint4(0u, 0u, 0u, 0u);   // d is a multiple of 8
             }
             ok = mbar_wait(bar_accf + 8 * acc, (it >> 1) & 1);
             tc_fence_after();
@@ -242,7 +242,7 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
 bool covered(const m2_plan* pl, int64_t d) {
     if (pl->dtype != M2_BF16 || pl->p != 2 || pl->dims[0] != pl->dims[1]) return false;
     const int b = pl->dims[0];
-    return (b == 64 || b == 128 || b == 256 || b == 512) && d > 0 && d % 64 == 0;
+    return (b == 64 || b == 128 || b == 256 || b == 512) && d > 0 && d % 8 == 0;   // rows of whole 16-byte pieces
 }
 
 cudaError_t prepare() {
@@ -261,7 +261,7 @@ static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, c
                      int64_t si, int64_t sj, cudaStream_t stream) {
     const int b = pl->dims[0];
     const int m = b == 64 ? 64 : 128;
-    const int nc = d % 256 == 0 ? 256 : d % 128 == 0 ? 128 : 64;
+    const int nc = d > 128 ? 256 : d > 64 ? 128 : 64;   // columns per tile
     alignas(64) CUtensorMap mw, mv, mo;
     {
         const cuuint64_t gdim[2] = {(cuuint64_t)b, (cuuint64_t)b * b}, gstr[1] = {(cuuint64_t)b * 2};
@@ -280,7 +280,7 @@ static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, c
         const cuuint32_t box[4] = {64, (cuuint32_t)m, 1, 1};
         if (!tma_host::encode_sw128_bf16(&mo, O, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
     }
-    const long long tiles = Bt * b * ((b + 127) / 128) * (d / nc);
+    const long long tiles = Bt * b * ((b + 127) / 128) * ((d + nc - 1) / nc);
     if (tiles > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);

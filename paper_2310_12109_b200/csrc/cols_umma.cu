@@ -242,7 +242,9 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
 bool covered(const m2_plan* pl, int64_t d) {
     if (pl->dtype != M2_BF16 || pl->p != 2 || pl->dims[0] != pl->dims[1]) return false;
     const int b = pl->dims[0];
-    return (b == 64 || b == 128 || b == 256 || b == 512) && d > 0 && d % 8 == 0;   // rows of whole 16-byte pieces
+    // blocks of whole 64-input chunks (an output tile past the end of a block computes rows that the store's tensor map clips),
+    // rows of whole 16-byte pieces
+    return b >= 64 && b <= 1024 && b % 64 == 0 && d > 0 && d % 8 == 0;
 }
 
 cudaError_t prepare() {

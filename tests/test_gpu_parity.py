@@ -453,7 +453,7 @@ def test_m2_layer_fwd(B, sn, sd, dtype):
 
 @pytest.mark.parametrize("b,Bt,d,dtype,withK", [(64, 2, 192, M.M2_BF16, True), (128, 1, 256, M.M2_BF16, True), (256, 1, 64, M.M2_BF16, False),
                                                  (256, 2, 256, M.M2_BF16, True), (64, 1, 768, M.M2_BF16, False), (64, 2, 200, M.M2_BF16, True),
-                                                 (128, 1, 328, M.M2_BF16, True), (64, 1, 8, M.M2_BF16, False), (8, 3, 40, M.M2_BF16, True), (6, 2, 33, M.M2_FP32, True)])
+                                                 (128, 1, 328, M.M2_BF16, True), (64, 1, 8, M.M2_BF16, False), (192, 1, 72, M.M2_BF16, True), (8, 3, 40, M.M2_BF16, True), (6, 2, 33, M.M2_FP32, True)])
 def test_monarch_cols(b, Bt, d, dtype, withK):
     """Y = sigma(K (.) M X) with the columns of X [Bt, N, d] as the vectors (the layout of the operator benchmark)."""
     N = b * b
@@ -468,7 +468,7 @@ def test_monarch_cols(b, Bt, d, dtype, withK):
     Y = M.m2_monarch_cols(plan, dv(X), dv(L), dv(R), None if K is None else dv(K), act=M.M2_ACT_RELU if withK else M.M2_ACT_NONE)
     torch.cuda.synchronize()
     assert plan.device_status() == 0
-    umma = dtype == M.M2_BF16 and b in (64, 128, 256, 512) and d % 8 == 0
+    umma = dtype == M.M2_BF16 and b % 64 == 0 and d % 8 == 0
     assert plan.last_kernel() == ("monarch_cols_umma" if umma else "monarch_cols_generic")
     ref = O.monarch_cols(L, R, X, K, "relu" if withK else "none")
     check(host(Y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, f"monarch cols b={b}")

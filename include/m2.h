@@ -185,7 +185,7 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
  * at least Bt N d elements of the plan dtype (the intermediate between the two factors), 16-byte aligned.
  * The M2 operator M_b (K (.) M_a X) is two calls, the first with K, the second without.
  * With the columns contiguous both factors are batched GEMMs over rows and the stride permutations are strides of TMA
- * tensor maps: square bf16 plans whose block size is a multiple of 64 (up to 1024) with d a multiple of 8 run on the tensor cores, two
+ * tensor maps: bf16 plans whose factors N1, N2 are multiples of 64 (up to 1024) with d a multiple of 8 run on the tensor cores, two
  * launches per call; everything else on a CUDA-core kernel (N <= 65535, else M2_ERR_UNSUPPORTED). */
 int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev,
                         int32_t act, void* Y_dev, int64_t Bt, int64_t d, void* ws_dev, int64_t ws_bytes, void* stream);

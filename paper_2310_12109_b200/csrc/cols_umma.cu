@@ -1,20 +1,21 @@
 // Monarch matrix times a matrix whose COLUMNS are the vectors:  Y = sigma(K (.) M X),  X, Y, K: [N][d] row-major,
-// M = P L P^T R P with N = b * b (Sec. 3.1; this is Eq. 2's M X with X in R^{N x d} as the paper writes it, and the layout
+// M = P L P^T R P with N = N1 * N2 (Sec. 3.1; this is Eq. 2's M X with X in R^{N x d} as the paper writes it, and the layout
 // of its operator benchmark, Table 2: N = 4K .. 256K, block size sqrt(N), d = 768 columns).
 //
 // With the d columns contiguous, both block-diagonal factors are plain batched GEMMs over rows and no element ever has
 // to be transposed:
-//   stage(W, V)[row o*b + j][c] = sum_i W[j][o][i] * V[row(i, j)][c]
-//   z = stage(R, x) with row(i, j) = i*b + j   (block j = n2 reads the rows n1*b + n2: a strided set of rows)
-//   y = stage(L, z) with row(i, j) = j*b + i   (block j = k1 reads the rows k1*b + n2: b consecutive rows)
+//   stage(W, V)[row o*so + j][c] = sum_i W[j][o][i] * V[row i*si + j*sj][c]
+//   z = stage(R, x): N2 blocks of N1 x N1, block j = n2 reads the rows n1*N2 + n2 (a strided set) and writes the rows k1*N2 + n2
+//   y = stage(L, z): N1 blocks of N2 x N2, block j = k1 reads the rows k1*N2 + n2 (consecutive) and writes the rows k2*N1 + k1
 // so the stride permutations are nothing but the strides of two TMA tensor maps.  One kernel serves both stages:
 // a CTA computes the tile [128 outputs o][NC columns] of one block j:  A = W[j] rows (K-major, 128B-swizzled TMA boxes
 // of 64 inputs), B = 64 input rows x NC columns (N-major: a row of the operand is a row of V), accumulator in TMEM
-// (M = 128, or 64 when b = 64; N = NC <= 256), K = b walked in chunks of 64 through a three-stage TMA ring; the
-// epilogue applies the optional factor K (.) and ReLU in fp32, rounds to bf16, stages the tile in the swizzled image of
-// the TMA store boxes and stores it to the rows o*b + j.  One persistent CTA per SM with a producer warp, an issuing warp
-// and four epilogue warps; two accumulators in TMEM, so a tile's epilogue overlaps the next tile's UMMAs.  All waits are
-// bounded.
+// (M = 128, or 64 for blocks of 64; N = NC <= 256), K = the block size walked in chunks of 64 through a three-stage TMA ring;
+// the epilogue applies the optional factor K (.) and ReLU in fp32, rounds to bf16, stages the tile in the swizzled image of
+// the TMA store boxes and stores it to its rows.  One persistent CTA per SM with a producer warp, an issuing warp
+// and four epilogue warps; two accumulators in TMEM, so a tile's epilogue overlaps the next tile's UMMAs.  Block sizes are
+// multiples of 64 (an output tile past the end of a block is clipped by the store's tensor map), d a multiple of 8 (a ragged
+// last column tile is zero-filled on the way in and clipped on the way out).  All waits are bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -66,8 +67,8 @@ __device__ __forceinline__ bool epilogue_sync_and(bool pred) {
 // next tile's UMMAs.
 __global__ void __launch_bounds__(kThreads, 1)
 monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_v,
-                          const __grid_constant__ CUtensorMap map_o, const __nv_bfloat16* __restrict__ Kmul, int relu, int b, int d, int nc,
-                          int m, int tiles, int32_t* __restrict__ status) {
+                          const __grid_constant__ CUtensorMap map_o, const __nv_bfloat16* __restrict__ Kmul, int relu, int b, int nb, int krs_o, int d,
+                          int nc, int m, int tiles, int32_t* __restrict__ status) {   // b: block size, nb: number of blocks
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
@@ -106,7 +107,7 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
             uint32_t n = 0;   // chunks issued so far
             bool ok = true;
             for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
-                const int ct = t % ctiles, ot = (t / ctiles) % otiles, j = (t / (ctiles * otiles)) % b, bt = t / (ctiles * otiles * b);
+                const int ct = t % ctiles, ot = (t / ctiles) % otiles, j = (t / (ctiles * otiles)) % nb, bt = t / (ctiles * otiles * nb);
                 for (int kc = 0; kc < chunks; ++kc, ++n) {
                     const int s = n % kStages;
                     if (n >= kStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kStages) - 1) & 1);   // the UMMAs have read the buffer
@@ -168,12 +169,12 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
         int it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
-            const int ct = t % ctiles, ot = (t / ctiles) % otiles, j = (t / (ctiles * otiles)) % b, bt = t / (ctiles * otiles * b);
+            const int ct = t % ctiles, ot = (t / ctiles) % otiles, j = (t / (ctiles * otiles)) % nb, bt = t / (ctiles * otiles * nb);
             const int acc = it & 1, o = ot * 128 + r, c0 = ct * nc;
             // the factor K (.) for this thread's row, requested while the tile's UMMAs still run
             uint4 kreg[32];
             if (Kmul != nullptr && valid) {
-                const uint4* krow = reinterpret_cast<const uint4*>(Kmul + ((size_t)o * b + j) * d + c0);   // K is shared by the batch
+                const uint4* krow = reinterpret_cast<const uint4*>(Kmul + ((size_t)o * krs_o + j) * d + c0);   // K is shared by the batch
 #pragma unroll
                 for (int e = 0; e < 32; ++e)
                     if (e < nq * 8) kreg[e] = c0 + 8 * e < d ? __ldg(krow + e) : make_uint4(0u, 0u, 0u, 0u);   // d is a multiple of 8
@@ -240,11 +241,12 @@ monarch_cols_stage_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
 }
 
 bool covered(const m2_plan* pl, int64_t d) {
-    if (pl->dtype != M2_BF16 || pl->p != 2 || pl->dims[0] != pl->dims[1]) return false;
-    const int b = pl->dims[0];
+    if (pl->dtype != M2_BF16 || pl->p != 2) return false;
     // blocks of whole 64-input chunks (an output tile past the end of a block computes rows that the store's tensor map clips),
     // rows of whole 16-byte pieces
-    return b >= 64 && b <= 1024 && b % 64 == 0 && d > 0 && d % 8 == 0;
+    for (int a = 0; a < 2; ++a)
+        if (pl->dims[a] < 64 || pl->dims[a] > 1024 || pl->dims[a] % 64 != 0) return false;
+    return d > 0 && d % 8 == 0;
 }
 
 cudaError_t prepare() {
@@ -258,31 +260,31 @@ cudaError_t prepare() {
     return e;
 }
 
-// one stage: out rows o*b + j = W[j] applied to the rows row(i, j) = i*si + j*sj of V
-static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, const void* Kmul, int relu, int64_t Bt, int64_t d,
-                     int64_t si, int64_t sj, cudaStream_t stream) {
-    const int b = pl->dims[0];
+// one stage: nb blocks of b x b; out rows o*so + j = W[j] applied to the rows i*si + j*sj of V (N = rows per matrix)
+static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, const void* Kmul, int relu, int64_t Bt, int64_t d, int b,
+                     int nb, int64_t si, int64_t sj, int64_t so, cudaStream_t stream) {
+    const int64_t N = pl->N;
     const int m = b == 64 ? 64 : 128;
     const int nc = d > 128 ? 256 : d > 64 ? 128 : 64;   // columns per tile
     alignas(64) CUtensorMap mw, mv, mo;
     {
-        const cuuint64_t gdim[2] = {(cuuint64_t)b, (cuuint64_t)b * b}, gstr[1] = {(cuuint64_t)b * 2};
+        const cuuint64_t gdim[2] = {(cuuint64_t)b, (cuuint64_t)nb * b}, gstr[1] = {(cuuint64_t)b * 2};
         const cuuint32_t box[2] = {64, (cuuint32_t)m};
         if (!tma_host::encode_sw128_bf16(&mw, W, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
     }
     {
-        const cuuint64_t gdim[4] = {(cuuint64_t)d, (cuuint64_t)b, (cuuint64_t)b, (cuuint64_t)Bt};
-        const cuuint64_t gstr[3] = {(cuuint64_t)(si * d * 2), (cuuint64_t)(sj * d * 2), (cuuint64_t)b * b * d * 2};
+        const cuuint64_t gdim[4] = {(cuuint64_t)d, (cuuint64_t)b, (cuuint64_t)nb, (cuuint64_t)Bt};
+        const cuuint64_t gstr[3] = {(cuuint64_t)(si * d * 2), (cuuint64_t)(sj * d * 2), (cuuint64_t)N * d * 2};
         const cuuint32_t box[4] = {64, 64, 1, 1};
         if (!tma_host::encode_sw128_bf16(&mv, V, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
     }
     {
-        const cuuint64_t gdim[4] = {(cuuint64_t)d, (cuuint64_t)b, (cuuint64_t)b, (cuuint64_t)Bt};
-        const cuuint64_t gstr[3] = {(cuuint64_t)b * d * 2, (cuuint64_t)d * 2, (cuuint64_t)b * b * d * 2};
+        const cuuint64_t gdim[4] = {(cuuint64_t)d, (cuuint64_t)b, (cuuint64_t)nb, (cuuint64_t)Bt};
+        const cuuint64_t gstr[3] = {(cuuint64_t)(so * d * 2), (cuuint64_t)d * 2, (cuuint64_t)N * d * 2};
         const cuuint32_t box[4] = {64, (cuuint32_t)m, 1, 1};
         if (!tma_host::encode_sw128_bf16(&mo, O, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
     }
-    const long long tiles = Bt * b * ((b + 127) / 128) * ((d + nc - 1) / nc);
+    const long long tiles = Bt * nb * ((b + 127) / 128) * ((d + nc - 1) / nc);
     if (tiles > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
@@ -297,8 +299,8 @@ static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, monarch_cols_stage_kernel, mw, mv, mo, (const __nv_bfloat16*)Kmul, relu, b, (int)d, nc, m, (int)tiles, pl->d_status) !=
-        cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, monarch_cols_stage_kernel, mw, mv, mo, (const __nv_bfloat16*)Kmul, relu, b, nb, (int)so, (int)d, nc, m,
+                           (int)tiles, pl->d_status) != cudaSuccess)
         return M2_ERR_CUDA;
     return M2_OK;
 }
@@ -309,10 +311,10 @@ int32_t apply(const m2_plan* pl, const void* X, const void* L, const void* R, co
     if (Bt > 65535) return M2_ERR_UNSUPPORTED;
     if (Bt == 0) return M2_OK;
     if (prepare() != cudaSuccess) return M2_ERR_CUDA;
-    const int b = pl->dims[0];
-    int32_t st = stage(pl, R, X, ws, nullptr, 0, Bt, d, b, 1, stream);          // z[k1*b + n2] from the rows n1*b + n2
+    const int N1 = pl->dims[0], N2 = pl->dims[1];
+    int32_t st = stage(pl, R, X, ws, nullptr, 0, Bt, d, N1, N2, N2, 1, N2, stream);   // z[k1*N2 + n2]: N2 blocks R[n2] on the rows n1*N2 + n2
     if (st != M2_OK) return st;
-    st = stage(pl, L, ws, Y, Kmul, relu, Bt, d, 1, b, stream);                   // y[k2*b + k1] from the rows k1*b + n2
+    st = stage(pl, L, ws, Y, Kmul, relu, Bt, d, N2, N1, 1, N2, N1, stream);           // y[k2*N1 + k1]: N1 blocks L[k1] on the rows k1*N2 + n2
     if (st != M2_OK) return st;
     pl->last_kernel = "monarch_cols_umma";
     pl->launches += 2;

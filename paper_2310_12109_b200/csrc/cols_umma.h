@@ -5,7 +5,7 @@
 #include "m2_plan.h"
 
 namespace m2c {
-// square order-2 bf16 plans with blocks of 64, 128, 192, ... 1024 and d a multiple of 8
+// order-2 bf16 plans whose two factors are multiples of 64 (up to 1024), d a multiple of 8
 bool covered(const m2_plan* plan, int64_t d);
 // Y[bt] = sigma(K (.) M X[bt]) for Bt matrices [N][d]; Kmul: [N][d] (shared by the batch) or nullptr; ws: Bt * N * d bf16 values
 int32_t apply(const m2_plan* plan, const void* X, const void* L, const void* R, const void* Kmul, int relu, void* Y, int64_t Bt,

@@ -456,22 +456,32 @@ def test_m2_layer_fwd(B, sn, sd, dtype):
                                                  (128, 1, 328, M.M2_BF16, True), (64, 1, 8, M.M2_BF16, False), (192, 1, 72, M.M2_BF16, True), (8, 3, 40, M.M2_BF16, True), (6, 2, 33, M.M2_FP32, True)])
 def test_monarch_cols(b, Bt, d, dtype, withK):
     """Y = sigma(K (.) M X) with the columns of X [Bt, N, d] as the vectors (the layout of the operator benchmark)."""
-    N = b * b
+    run_monarch_cols(b, b, Bt, d, dtype, withK)
+
+
+@pytest.mark.parametrize("N1,N2,d", [(64, 128, 72), (128, 64, 256), (192, 64, 64)])
+def test_monarch_cols_rectangular(N1, N2, d):
+    run_monarch_cols(N1, N2, 2, d, M.M2_BF16, True)
+
+
+def run_monarch_cols(N1, N2, Bt, d, dtype, withK):
+    b = N1
+    N = N1 * N2
     tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
     rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
-    L = rnd(synth.normal(synth.stream_id(13, 0), (b, b, b)) / np.sqrt(b))
-    R = rnd(synth.normal(synth.stream_id(13, 1), (b, b, b)) / np.sqrt(b))
+    L = rnd(synth.normal(synth.stream_id(13, 0), (N1, N2, N2)) / np.sqrt(N2))
+    R = rnd(synth.normal(synth.stream_id(13, 1), (N2, N1, N1)) / np.sqrt(N1))
     X = rnd(synth.normal(synth.stream_id(13, 2), (Bt, N, d)))
     K = rnd(synth.normal(synth.stream_id(13, 3), (N, d))) if withK else None
-    plan = M.Plan((b, b), dtype=dtype, device=0)
+    plan = M.Plan((N1, N2), dtype=dtype, device=0)
     dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
     Y = M.m2_monarch_cols(plan, dv(X), dv(L), dv(R), None if K is None else dv(K), act=M.M2_ACT_RELU if withK else M.M2_ACT_NONE)
     torch.cuda.synchronize()
     assert plan.device_status() == 0
-    umma = dtype == M.M2_BF16 and b % 64 == 0 and d % 8 == 0
+    umma = dtype == M.M2_BF16 and N1 % 64 == 0 and N2 % 64 == 0 and d % 8 == 0
     assert plan.last_kernel() == ("monarch_cols_umma" if umma else "monarch_cols_generic")
     ref = O.monarch_cols(L, R, X, K, "relu" if withK else "none")
-    check(host(Y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, f"monarch cols b={b}")
+    check(host(Y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, f"monarch cols {N1}x{N2}")
     plan.close()
 
 

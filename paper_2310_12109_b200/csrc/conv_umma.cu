@@ -1156,6 +1156,52 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     return M2_OK;
 }
 
+// dk[h] = Re M^-1 ( sum_p partial[p][h][:] ) [0:n) / 512 for N = 512 = 32 x 16: the parts added in index order, then the two
+// inverse stages in fp32 (conj F_16 over k2 with the conjugated twiddle, conj F_32 over k1, real part); one block per channel
+__global__ void __launch_bounds__(256) wgrad512_finish_kernel(const float2* __restrict__ partial, int parts, float* __restrict__ dk,
+                                                              const float2* __restrict__ roots32, const float2* __restrict__ roots16, int H, int n,
+                                                              float sgn) {
+    __shared__ float2 a[512], bb[512], r32[32], r16[16];
+    const int h = blockIdx.x, tid = threadIdx.x;
+    if (tid < 32) r32[tid] = roots32[tid];
+    if (tid < 16) r16[tid] = roots16[tid];
+    for (int i = tid; i < 512; i += 256) {
+        float2 v = make_float2(0.f, 0.f);
+        for (int p = 0; p < parts; ++p) {
+            const float2 w = partial[((size_t)p * H + h) * 512 + i];
+            v.x += w.x;
+            v.y += w.y;
+        }
+        a[i] = v;
+    }
+    __syncthreads();
+    for (int o = tid; o < 512; o += 256) {   // (k1, n2) = sum_k2 conj(w_16^{k2 n2}) a[k1][k2], times conj(w_512^{n2 k1})
+        const int k1 = o >> 4, n2 = o & 15;
+        float sr = 0.f, si = 0.f;
+#pragma unroll
+        for (int k2 = 0; k2 < 16; ++k2) {
+            const float2 w = r16[(k2 * n2) & 15], v = a[k1 * 16 + k2];   // conj(w) v = (wx vx + wy vy) + i (wx vy - wy vx)
+            sr = fmaf(w.x, v.x, fmaf(w.y, v.y, sr));
+            si = fmaf(w.x, v.y, fmaf(-w.y, v.x, si));
+        }
+        float ts, tc;
+        sincospif(2.0f * (float)((n2 * k1) & 511) / 512.0f, &ts, &tc);
+        ts *= sgn;   // w_512^{n2 k1} = tc + i ts; multiply by its conjugate
+        bb[o] = make_float2(sr * tc + si * ts, si * tc - sr * ts);
+    }
+    __syncthreads();
+    for (int t = tid; t < 512; t += 256) {   // y[n1*16 + n2] = Re sum_k1 conj(w_32^{k1 n1}) bb[k1][n2]
+        const int n1 = t >> 4, n2 = t & 15;
+        float acc = 0.f;
+#pragma unroll
+        for (int k1 = 0; k1 < 32; ++k1) {
+            const float2 w = r32[(k1 * n1) & 31], v = bb[k1 * 16 + n2];
+            acc = fmaf(w.x, v.x, fmaf(w.y, v.y, acc));
+        }
+        if (t < n) dk[(size_t)h * n + t] = acc * (1.0f / 512.0f);
+    }
+}
+
 int64_t conv_wgrad_workspace_bytes(const m2_plan* pl, int64_t B, int64_t H) {
     return pl->umma && covered(pl) ? ((B + kRows - 1) / kRows) * H * 512 * 8 : 0;
 }
@@ -1187,6 +1233,17 @@ int32_t conv_wgrad_partials(const m2_plan* pl, const void* x, const void* g, voi
                            pl->d_status) != cudaSuccess)
         return M2_ERR_CUDA;
     *parts = (int)bgroups;
+    pl->launches += 1;
+    return M2_OK;
+}
+
+// the second launch of the kernel gradient: dk from the partial sums
+int32_t conv_wgrad_finish(const m2_plan* pl, const void* partial, int parts, float* dk, int64_t H, int64_t n, cudaStream_t stream) {
+    if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (H == 0) return M2_OK;
+    wgrad512_finish_kernel<<<(unsigned)H, 256, 0, stream>>>((const float2*)partial, parts, dk, pl->d_roots[0], pl->d_roots[1], (int)H, (int)n,
+                                                            pl->sign >= 0 ? 1.0f : -1.0f);
+    if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
     pl->launches += 1;
     return M2_OK;
 }

@@ -20,6 +20,8 @@ int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, in
 int64_t conv_wgrad_workspace_bytes(const m2_plan* plan, int64_t B, int64_t H);
 int32_t conv_wgrad_partials(const m2_plan* plan, const void* x, const void* g, void* partial, int64_t B, int64_t H, int64_t n,
                             int32_t mode, int* parts, cudaStream_t stream);
+// ... and dk[H][n] (fp32) = Re M^-1(sum of the parts)[0:n) / N from them (CUDA cores, fp32)
+int32_t conv_wgrad_finish(const m2_plan* plan, const void* partial, int parts, float* dk, int64_t H, int64_t n, cudaStream_t stream);
 
 }  // namespace m2u
 

@@ -609,53 +609,6 @@ cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order
     return cudaGetLastError();
 }
 
-// dk[h] = Re M^-1 ( sum_p partial[p][h][:] ) [0:n) / N: the parts added in index order, the inverse stages in fp32
-template <int ITEMS>
-__global__ void __launch_bounds__(1024) spectrum_sum_inverse_kernel(const float2* __restrict__ partial, int parts, float* __restrict__ dk, Dims D,
-                                                                    Roots R, int H, int n) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float2* acc = reinterpret_cast<float2*>(smem_raw);
-    const int h = blockIdx.x;
-    for (int i = threadIdx.x; i < D.N; i += blockDim.x) {
-        float2 a = make_float2(0.f, 0.f);
-        for (int p = 0; p < parts; ++p) {
-            const float2 v = partial[((long long)p * H + h) * D.N + i];
-            a.x += v.x;
-            a.y += v.y;
-        }
-        acc[i] = a;
-    }
-    __syncthreads();
-    for (int a = D.p - 1; a >= 0; --a) stage<float2, ITEMS, true>(acc, D, a, R.r[a]);
-    const float inv = 1.0f / (float)D.N;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) dk[(long long)h * n + i] = acc[i].x * inv;
-}
-
-cudaError_t launch_spectrum_sum_inverse(const ConvShape& s, const void* partial, int parts, float* dk, cudaStream_t st) {
-    Dims D = make_dims(s);
-    Roots R{{s.roots[0], s.roots[1], s.roots[2]}};
-    int items, threads;
-    if (!pick_launch(D, items, threads)) return cudaErrorInvalidValue;
-    const size_t smem = (size_t)D.N * sizeof(float2);
-    if (smem > 200 * 1024) return cudaErrorInvalidValue;
-    if (s.H == 0) return cudaSuccess;
-#define M2_LAUNCH_SSI(IT)                                                                                       \
-    {                                                                                                           \
-        auto kern = spectrum_sum_inverse_kernel<IT>;                                                            \
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
-        if (e != cudaSuccess) return e;                                                                         \
-        kern<<<(unsigned)s.H, threads, smem, st>>>((const float2*)partial, parts, dk, D, R, (int)s.H, (int)s.n); \
-    }
-    switch (items) {
-        case 1: M2_LAUNCH_SSI(1) break;
-        case 2: M2_LAUNCH_SSI(2) break;
-        case 4: M2_LAUNCH_SSI(4) break;
-        default: return cudaErrorInvalidValue;
-    }
-#undef M2_LAUNCH_SSI
-    return cudaGetLastError();
-}
-
 long long conv_wgrad_scratch_bytes(long long N, long long H) {
     if ((size_t)N * sizeof(float2) * 3 <= 200 * 1024) return 0;   // fits in shared memory
     return (H < kWgradScratchBlocks ? H : kWgradScratchBlocks) * 3 * N * (long long)sizeof(float2);

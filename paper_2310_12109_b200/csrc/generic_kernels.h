@@ -44,8 +44,6 @@ cudaError_t launch_transpose_any(const void* in, void* out, long long B, int R, 
 // y[row] = LayerNorm(a[row] + b[row]) * gamma + beta over d values (y may alias a or b)
 cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamma, const float* beta, void* y, long long rows, int d,
                                  float eps, bool bf16, cudaStream_t st);
-// dk[h] = Re M^-1(sum_p partial[p][h][:])[0:n) / N with partial [parts][H][N] complex fp32 in plan order
-cudaError_t launch_spectrum_sum_inverse(const ConvShape& s, const void* partial, int parts, float* dk, cudaStream_t st);
 // Y = sigma(K (.) M X) for Bt matrices [N][d] whose columns are the vectors (CUDA cores; ws: Bt*N*d values of the I/O type)
 cudaError_t launch_monarch_cols(int N1, int N2, long long Bt, int d, bool bf16_io, const void* X, const void* L, const void* R, const void* Kmul,
                                 int relu, void* Y, void* ws, cudaStream_t st);

@@ -261,9 +261,9 @@ int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const
         int parts = 0;
         st = m2u::conv_wgrad_partials(plan, x_dev, g_dev, ws_dev, B, H, n, mode, &parts, (cudaStream_t)stream);
         if (st == M2_OK) {
-            if (m2g::launch_spectrum_sum_inverse(s, ws_dev, parts, dk_dev, (cudaStream_t)stream) != cudaSuccess) return M2_ERR_CUDA;
+            st = m2u::conv_wgrad_finish(plan, ws_dev, parts, dk_dev, H, n, (cudaStream_t)stream);
+            if (st != M2_OK) return st;
             plan->last_kernel = "conv_wgrad_umma_o2_512";
-            plan->launches += 1;
             return M2_OK;
         }
         if (st != M2_ERR_UNSUPPORTED) return st;

@@ -654,14 +654,25 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     return M2_OK;
 }
 
-// dk[h][i] = sum over the row pairs of channel h of the pair's first output row (fp32 sum of bf16 values, pairs in index order)
-__global__ void wgrad_pair_sum_kernel(const __nv_bfloat16* __restrict__ rows, float* __restrict__ dk, int B, int H, long long total) {
-    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 16384
-    if (e >= total) return;
-    const long long h = e >> 14, i = e & 16383;
-    float acc = 0.f;
-    for (int b = 0; b < B; b += 2) acc += __bfloat162float(rows[((long long)b * H + h) * 16384 + i]);
-    dk[e] = acc;
+// dk[h][i] = sum over the row pairs of channel h of the pair's first output row (fp32 sum of bf16 values, pairs in index order);
+// 8 consecutive positions per thread
+__global__ void wgrad_pair_sum_kernel(const __nv_bfloat16* __restrict__ rows, float* __restrict__ dk, int B, int H, long long total8) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over H * 16384 / 8
+    if (e >= total8) return;
+    const long long h = e >> 11, i = (e & 2047) * 8;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int b = 0; b < B; b += 2) {
+        const uint4 v = *reinterpret_cast<const uint4*>(rows + ((long long)b * H + h) * 16384 + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            acc[2 * q] += __uint_as_float(w[q] << 16);
+            acc[2 * q + 1] += __uint_as_float(w[q] & 0xffff0000u);
+        }
+    }
+    float4* dst = reinterpret_cast<float4*>(dk + h * 16384 + i);
+    dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
 }
 
 // Kernel gradient on the tensor cores: with z_p = xa + i xb and w_p = ga + i gb for the row pairs p of a channel,
@@ -709,8 +720,8 @@ int32_t conv_wgrad(const m2_plan* pl, const void* x, const void* g, float* dk, i
     if (cudaLaunchKernelEx(&cfg, conv32k_kernel<0>, my, (const __nv_bfloat16*)g, (const float4*)spec, (const uint4*)tb->d_const,
                            (const float2*)tb->d_tn, (int)B, (int)H, pl->d_status, 1, (float4*)nullptr) != cudaSuccess)
         return M2_ERR_CUDA;
-    const long long total = H * 16384;
-    wgrad_pair_sum_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(rows, dk, (int)B, (int)H, total);
+    const long long total8 = H * 2048;
+    wgrad_pair_sum_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, stream>>>(rows, dk, (int)B, (int)H, total8);
     if (cudaGetLastError() != cudaSuccess) return M2_ERR_CUDA;
     pl->last_kernel = "conv_wgrad_umma_o3_32k";
     pl->launches += 3;

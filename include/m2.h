@@ -190,6 +190,22 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
 int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev,
                         int32_t act, void* Y_dev, int64_t Bt, int64_t d, void* ws_dev, int64_t ws_bytes, void* stream);
 
+/* The M2 Hyena layer with heads (App. "GPT Causal Language Modeling", the algorithm of that name), u: [B, n, d]:
+ *   X1, X2, V = u W_X1, u W_X2, u W_V;  X1~, X2~, V~ = causal Monarch convolution of every channel with a short kernel;
+ *   per head of dh channels: XV[t] = X2~[t] V~[t]^T, each of its dh^2 sequences through the causal Monarch convolution with
+ *   the head's long kernel; O[t] = X1~[t] XV[t];  y = concat(O) W_O.
+ * plan: the convolution plan, N >= 2 n (the convolutions are m2_monarch_conv_fwd in M2_CAUSAL mode on channel-first rows).
+ * W: HOST array of 4 device pointers {W_X1, W_X2, W_V, W_O}, each [d][d] stored outputs x inputs (y[o] = sum_i W[o][i] u[i]).
+ * kf1_dev, kf2_dev, kf3_dev: m2_kernel_spectrum of the short kernels [d, n];  kf_long_dev: m2_kernel_spectrum of the long
+ * kernel with one row per (head, i, j) channel, i.e. [d dh, n] with the head's kernel repeated dh^2 times.
+ * y_dev: [B, n, d] (must not overlap u_dev).  scratch_dev: m2_hyena_scratch_bytes(plan, B, n, d, dh) bytes, caller-owned.
+ * The projections are the single-block case of the column-layout Monarch kernel (tensor cores for d a multiple of 64 up
+ * to 4096 and n a multiple of 8, bf16), so after one transposition everything runs channel-first. */
+int64_t m2_hyena_scratch_bytes(const m2_plan* plan, int64_t B, int64_t n, int64_t d, int64_t dh);
+int32_t m2_hyena_heads_fwd(const m2_plan* plan, const void* u_dev, const void* const* W, const void* kf1_dev,
+                           const void* kf2_dev, const void* kf3_dev, const void* kf_long_dev, void* y_dev, int64_t B,
+                           int64_t n, int64_t d, int64_t dh, void* scratch_dev, int64_t scratch_bytes, void* stream);
+
 /* W_out[b][c][r] = W_in[b][r][c]: block-wise transpose of a block-diagonal factor of nblocks blocks of rows x cols
  * elements of the plan dtype (W_out must not overlap W_in).  It gives the gradient of the Monarch matmul with
  * respect to its input: M^T = P^T R^T P L^T P^T (Sec. 3.1 transposed) is again an order-2 Monarch product, so for an

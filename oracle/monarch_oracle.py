@@ -254,6 +254,33 @@ def m2_layer(x: np.ndarray, p: dict, eps: float = 1e-5, stages: dict | None = No
     return out
 
 
+def m2_hyena_heads(u: np.ndarray, p: dict, dims: tuple, dh: int, stages: dict | None = None) -> np.ndarray:
+    """The M2 Hyena layer with heads (App. "GPT Causal Language Modeling", the algorithm of that name), u: [B, n, d]:
+        X1, X2, V = u W_X1, u W_X2, u W_V                                     (dense projections)
+        X1~, X2~, V~ = causal Monarch convolution of each channel with the short kernels K1, K2, K3 [d, n]
+        per head h (d_h channels): XV[t] = X2~[t] V~[t]^T (d_h x d_h per position), each of its d_h^2 sequences through the
+        causal Monarch convolution with the head's long kernel K_long[h]; O[t] = X1~[t] XV[t]  (row vector times matrix)
+        y = concat_h(O) W_O.
+    Weights act as u @ W with W: [d_in, d_out].  The convolutions are monarch_conv with the plan's factorisation `dims`
+    (N = prod(dims) >= 2 n)."""
+    B, n, d = u.shape
+    Hh = d // dh
+    assert Hh * dh == d
+    cm = lambda a: np.swapaxes(a, 1, 2)                                       # [B, n, d] <-> [B, d, n]
+    X1, X2, V = u @ p["W_x1"], u @ p["W_x2"], u @ p["W_v"]
+    X1c = monarch_conv(p["K1"][None], cm(X1), dims, causal=True)             # [B, d, n]
+    X2c = monarch_conv(p["K2"][None], cm(X2), dims, causal=True)
+    Vc = monarch_conv(p["K3"][None], cm(V), dims, causal=True)
+    x2h, vh, x1h = (a.reshape(B, Hh, dh, n) for a in (X2c, Vc, X1c))
+    XV = np.einsum("bhit,bhjt->bhijt", x2h, vh)                              # outer product per position
+    XVc = monarch_conv(p["K_long"][None, :, None, None, :], XV, dims, causal=True)
+    O = np.einsum("bhit,bhijt->bhjt", x1h, XVc).reshape(B, d, n)
+    y = cm(O) @ p["W_o"]
+    if stages is not None:
+        stages.update(X1c=X1c, X2c=X2c, Vc=Vc, XVc=XVc, O=O)
+    return y
+
+
 def monarch_weight_grads(L: np.ndarray, R: np.ndarray, x: np.ndarray, g: np.ndarray):
     """Gradients of sum_t <M x_t, g_t> with respect to the blocks of L and R for M = P L P^T R P (Sec. 3.1), by the
     chain rule through the stages of monarch_apply: with v0 = P x ([n2][n1]), v1 = R v0 ([n2][k1]) and the upstream

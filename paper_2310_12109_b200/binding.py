@@ -39,6 +39,8 @@ SIGNATURES = {
     "m2_layer_scratch_bytes": (_i64, [_vp, _vp, _i64]),
     "m2_layer_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_cols": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _i64, _vp, _i64, _vp]),
+    "m2_hyena_scratch_bytes": (_i64, [_vp, _i64, _i64, _i64, _i64]),
+    "m2_hyena_heads_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_conv_bwd_workspace_bytes": (_i64, [_vp, _i64, _i64]),
     "m2_monarch_conv_bwd_kernel": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]),
@@ -284,6 +286,23 @@ def m2_monarch_cols(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tenso
     _check(lib().m2_monarch_cols(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(K), act, _ptr(Y), Bt, d, _ptr(ws),
                                  ws.numel() * ws.element_size(), _stream()), "m2_monarch_cols")
     return Y
+
+
+def m2_hyena_heads_fwd(plan: Plan, u: torch.Tensor, W, kf1, kf2, kf3, kf_long, dh: int) -> torch.Tensor:
+    """The M2 Hyena layer with heads on u [B, n, d]; W = (W_X1, W_X2, W_V, W_O), each [d, d] stored outputs x inputs;
+    kf1..kf3 = m2_kernel_spectrum of the short kernels [d, n]; kf_long = m2_kernel_spectrum of the long kernel repeated
+    to one row per (head, i, j) channel: K_long.repeat_interleave(dh * dh, dim=0)."""
+    B, n, d = u.shape
+    assert len(W) == 4 and d % dh == 0
+    for a in (u, *W):
+        assert a.is_cuda and a.dtype == plan.torch_dtype and a.is_contiguous()
+    y = torch.empty_like(u)
+    sb = int(lib().m2_hyena_scratch_bytes(plan.handle, B, n, d, dh))
+    scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=u.device)
+    wp = (ctypes.c_void_p * 4)(*[w.data_ptr() for w in W])
+    _check(lib().m2_hyena_heads_fwd(plan.handle, _ptr(u), wp, _ptr(kf1), _ptr(kf2), _ptr(kf3), _ptr(kf_long), _ptr(y), B, n, d, dh,
+                                    _ptr(scratch), scratch.numel(), _stream()), "m2_hyena_heads_fwd")
+    return y
 
 
 def m2_blocks_transpose(plan: Plan, W: torch.Tensor) -> torch.Tensor:

@@ -260,10 +260,9 @@ cudaError_t prepare() {
     return e;
 }
 
-// one stage: nb blocks of b x b; out rows o*so + j = W[j] applied to the rows i*si + j*sj of V (N = rows per matrix)
-static int32_t stage(const m2_plan* pl, const void* W, const void* V, void* O, const void* Kmul, int relu, int64_t Bt, int64_t d, int b,
-                     int nb, int64_t si, int64_t sj, int64_t so, cudaStream_t stream) {
-    const int64_t N = pl->N;
+// one stage: nb blocks of b x b; out rows o*so + j = W[j] applied to the rows i*si + j*sj of V (N = rows per matrix of the batch)
+static int32_t stage(const m2_plan* pl, int64_t N, const void* W, const void* V, void* O, const void* Kmul, int relu, int64_t Bt, int64_t d,
+                     int b, int nb, int64_t si, int64_t sj, int64_t so, cudaStream_t stream) {
     const int m = b == 64 ? 64 : 128;
     const int nc = d > 128 ? 256 : d > 64 ? 128 : 64;   // columns per tile
     alignas(64) CUtensorMap mw, mv, mo;
@@ -312,13 +311,28 @@ int32_t apply(const m2_plan* pl, const void* X, const void* L, const void* R, co
     if (Bt == 0) return M2_OK;
     if (prepare() != cudaSuccess) return M2_ERR_CUDA;
     const int N1 = pl->dims[0], N2 = pl->dims[1];
-    int32_t st = stage(pl, R, X, ws, nullptr, 0, Bt, d, N1, N2, N2, 1, N2, stream);   // z[k1*N2 + n2]: N2 blocks R[n2] on the rows n1*N2 + n2
+    int32_t st = stage(pl, pl->N, R, X, ws, nullptr, 0, Bt, d, N1, N2, N2, 1, N2, stream);   // z[k1*N2 + n2]: N2 blocks R[n2] on the rows n1*N2 + n2
     if (st != M2_OK) return st;
-    st = stage(pl, L, ws, Y, Kmul, relu, Bt, d, N2, N1, 1, N2, N1, stream);           // y[k2*N1 + k1]: N1 blocks L[k1] on the rows k1*N2 + n2
+    st = stage(pl, pl->N, L, ws, Y, Kmul, relu, Bt, d, N2, N1, 1, N2, N1, stream);           // y[k2*N1 + k1]: N1 blocks L[k1] on the rows k1*N2 + n2
     if (st != M2_OK) return st;
     pl->last_kernel = "monarch_cols_umma";
     pl->launches += 2;
     return M2_OK;
+}
+
+// A dense matrix is a block-diagonal one with a single block: O[bt] = W V[bt] for Bt matrices V [c][cols] (cols contiguous),
+// W: [c][c] row-major (outputs x inputs).  pl only lends its status word and launch counter.
+bool dense_covered(const m2_plan* pl, int64_t c, int64_t cols) {
+    return pl->dtype == M2_BF16 && c >= 64 && c <= 4096 && c % 64 == 0 && cols > 0 && cols % 8 == 0;
+}
+
+int32_t dense(const m2_plan* pl, const void* W, const void* V, void* O, int64_t Bt, int64_t c, int64_t cols, cudaStream_t stream) {
+    if (!dense_covered(pl, c, cols) || Bt > 65535) return M2_ERR_UNSUPPORTED;
+    if (Bt == 0) return M2_OK;
+    if (prepare() != cudaSuccess) return M2_ERR_CUDA;
+    const int32_t st = stage(pl, c, W, V, O, nullptr, 0, Bt, cols, (int)c, 1, 1, c, 1, stream);   // (the block stride is never used: one block)
+    if (st == M2_OK) pl->launches += 1;
+    return st;
 }
 
 }  // namespace m2c

@@ -901,4 +901,70 @@ cudaError_t launch_monarch_cols(int N1, int N2, long long Bt, int d, bool bf16_i
     return cudaGetLastError();
 }
 
+// Heads of the M2 Hyena layer, channel-first tensors [B][channels][n] (n contiguous):
+//   outer : XV[b][(h dh + i) dh + j][t] = X2[b][h dh + i][t] * V[b][h dh + j][t]
+//   reduce: O[b][h dh + j][t] = sum_i X1[b][h dh + i][t] * XVc[b][(h dh + i) dh + j][t]
+// one thread per output element (fp32 arithmetic, one rounding on the way out)
+template <typename IO>
+__global__ void heads_outer_kernel(const IO* __restrict__ X2, const IO* __restrict__ V, IO* __restrict__ XV, int d, int dh, int n,
+                                   long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * dh * n
+    if (e >= total) return;
+    const int t = (int)(e % n);
+    const long long ch = (e / n) % ((long long)d * dh), b = e / ((long long)n * d * dh);
+    const int j = (int)(ch % dh), hi = (int)(ch / dh);   // hi = h dh + i
+    const int hj = (hi / dh) * dh + j;
+    XV[e] = from_f32<IO>(to_f32<IO>(X2[(b * d + hi) * n + t]) * to_f32<IO>(V[(b * d + hj) * n + t]));
+}
+
+template <typename IO>
+__global__ void heads_reduce_kernel(const IO* __restrict__ X1, const IO* __restrict__ XVc, IO* __restrict__ O, int d, int dh, int n,
+                                    long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n
+    if (e >= total) return;
+    const int t = (int)(e % n);
+    const int c = (int)((e / n) % d);
+    const long long b = e / ((long long)n * d);
+    const int h = c / dh, j = c % dh;
+    float acc = 0.f;
+    for (int i = 0; i < dh; ++i)
+        acc = fmaf(to_f32<IO>(X1[(b * d + h * dh + i) * n + t]), to_f32<IO>(XVc[((b * d + h * dh + i) * dh + j) * n + t]), acc);
+    O[e] = from_f32<IO>(acc);
+}
+
+cudaError_t launch_heads_outer(const void* X2, const void* V, void* XV, long long B, int d, int dh, int n, bool bf16, cudaStream_t st) {
+    const long long total = B * d * dh * n;
+    if (total == 0) return cudaSuccess;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (bf16)
+        heads_outer_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X2, (const __nv_bfloat16*)V, (__nv_bfloat16*)XV, d, dh, n, total);
+    else
+        heads_outer_kernel<float><<<grid, 256, 0, st>>>((const float*)X2, (const float*)V, (float*)XV, d, dh, n, total);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_heads_reduce(const void* X1, const void* XVc, void* O, long long B, int d, int dh, int n, bool bf16, cudaStream_t st) {
+    const long long total = B * d * n;
+    if (total == 0) return cudaSuccess;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (bf16)
+        heads_reduce_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X1, (const __nv_bfloat16*)XVc, (__nv_bfloat16*)O, d, dh, n, total);
+    else
+        heads_reduce_kernel<float><<<grid, 256, 0, st>>>((const float*)X1, (const float*)XVc, (float*)O, d, dh, n, total);
+    return cudaGetLastError();
+}
+
+// O[bt] = W V[bt] on the CUDA cores: W [c][c] (outputs x inputs), V, O [Bt][c][cols] (one block-diagonal stage with a single block)
+cudaError_t launch_dense_cols(const void* W, const void* V, void* O, long long Bt, int c, int cols, bool bf16, cudaStream_t st) {
+    if (Bt == 0 || c == 0 || cols == 0) return cudaSuccess;
+    if (Bt > 65535 || c > 65535) return cudaErrorInvalidValue;
+    const dim3 grid((cols + 127) / 128, (unsigned)c, (unsigned)Bt);
+    if (bf16)
+        cols_stage_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>((const __nv_bfloat16*)W, (const __nv_bfloat16*)V, (__nv_bfloat16*)O, nullptr, 0, c, c, c,
+                                                               cols, 1, 0, 1, 0);
+    else
+        cols_stage_kernel<float><<<grid, 128, 0, st>>>((const float*)W, (const float*)V, (float*)O, nullptr, 0, c, c, c, cols, 1, 0, 1, 0);
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

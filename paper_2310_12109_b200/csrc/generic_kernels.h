@@ -47,6 +47,11 @@ cudaError_t launch_add_layernorm(const void* a, const void* b, const float* gamm
 // Y = sigma(K (.) M X) for Bt matrices [N][d] whose columns are the vectors (CUDA cores; ws: Bt*N*d values of the I/O type)
 cudaError_t launch_monarch_cols(int N1, int N2, long long Bt, int d, bool bf16_io, const void* X, const void* L, const void* R, const void* Kmul,
                                 int relu, void* Y, void* ws, cudaStream_t st);
+// heads of the M2 Hyena layer on channel-first tensors [B][channels][n]: outer product per position and its contraction with X1
+cudaError_t launch_heads_outer(const void* X2, const void* V, void* XV, long long B, int d, int dh, int n, bool bf16, cudaStream_t st);
+cudaError_t launch_heads_reduce(const void* X1, const void* XVc, void* O, long long B, int d, int dh, int n, bool bf16, cudaStream_t st);
+// O[bt] = W V[bt]: W [c][c] (outputs x inputs), V, O [Bt][c][cols], CUDA cores
+cudaError_t launch_dense_cols(const void* W, const void* V, void* O, long long Bt, int c, int cols, bool bf16, cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

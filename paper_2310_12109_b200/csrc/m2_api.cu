@@ -484,6 +484,62 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
     return M2_OK;
 }
 
+int64_t m2_hyena_scratch_bytes(const m2_plan* plan, int64_t B, int64_t n, int64_t d, int64_t dh) {
+    if (!plan || B < 0 || n < 0 || d < 0 || dh <= 0) return -1;
+    return (7 + 2 * dh) * round256(B * d * n * (plan->dtype == M2_BF16 ? 2 : 4));
+}
+
+int32_t m2_hyena_heads_fwd(const m2_plan* plan, const void* u_dev, const void* const* W, const void* kf1_dev, const void* kf2_dev,
+                           const void* kf3_dev, const void* kf_long_dev, void* y_dev, int64_t B, int64_t n, int64_t d, int64_t dh,
+                           void* scratch_dev, int64_t scratch_bytes, void* stream) {
+    if (!plan || !W || B < 0 || n <= 0 || d <= 0 || dh <= 0 || d % dh != 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (2 * n > plan->N) return M2_ERR_INVALID_ARG;   // causal: N >= 2 n
+    if (B > 65535 || B * d * dh * n > 0x7fffffffffLL || d > 65535) return M2_ERR_UNSUPPORTED;
+    if (B == 0) return M2_OK;
+    for (int i = 0; i < 4; ++i)
+        if (!W[i] || !aligned16(W[i])) return W[i] ? M2_ERR_ALIGNMENT : M2_ERR_INVALID_ARG;
+    if (!u_dev || !kf1_dev || !kf2_dev || !kf3_dev || !kf_long_dev || !y_dev || !scratch_dev) return M2_ERR_INVALID_ARG;
+    if (!aligned16(u_dev) || !aligned16(y_dev) || !aligned16(scratch_dev)) return M2_ERR_ALIGNMENT;
+    if (scratch_bytes < m2_hyena_scratch_bytes(plan, B, n, d, dh)) return M2_ERR_INVALID_ARG;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf = plan->dtype == M2_BF16;
+    const int64_t tb = round256(B * d * n * (bf ? 2 : 4));
+    unsigned char* sc = static_cast<unsigned char*>(scratch_dev);
+    void *uT = sc, *P1 = sc + tb, *P2 = sc + 2 * tb, *P3 = sc + 3 * tb, *C1 = sc + 4 * tb, *C2 = sc + 5 * tb, *C3 = sc + 6 * tb;
+    void *XV = sc + 7 * tb, *XVc = sc + (7 + dh) * tb;
+    auto dense = [&](const void* Wm, const void* V, void* O) -> int32_t {   // O[b] = Wm V[b] on [B][d][n]
+        int32_t rc = m2c::dense(plan, Wm, V, O, B, d, n, st);
+        if (rc != M2_ERR_UNSUPPORTED) return rc;
+        const cudaError_t e = m2g::launch_dense_cols(Wm, V, O, B, (int)d, (int)n, bf, st);
+        if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+        if (e != cudaSuccess) return M2_ERR_CUDA;
+        plan->launches += 1;
+        return M2_OK;
+    };
+    // channel-first from here on: every projection, convolution and head product works on rows of n positions
+    if (m2g::launch_transpose_any(u_dev, uT, B, (int)n, (int)d, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    int32_t rc = dense(W[0], uT, P1);
+    if (rc == M2_OK) rc = dense(W[1], uT, P2);
+    if (rc == M2_OK) rc = dense(W[2], uT, P3);
+    if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, P1, kf1_dev, C1, B, d, n, M2_CAUSAL, stream);
+    if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, P2, kf2_dev, C2, B, d, n, M2_CAUSAL, stream);
+    if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, P3, kf3_dev, C3, B, d, n, M2_CAUSAL, stream);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_heads_outer(C2, C3, XV, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    rc = m2_monarch_conv_fwd(plan, XV, kf_long_dev, XVc, B, d * dh, n, M2_CAUSAL, stream);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_heads_reduce(C1, XVc, P1, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    rc = dense(W[3], P1, P2);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_transpose_any(P2, y_dev, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    plan->launches += 4;   // two transposes and the two head kernels (the products and convolutions count themselves)
+    plan->last_kernel = "hyena_heads_fwd";
+    return M2_OK;
+}
+
 int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows, int64_t cols,
                             void* stream) {
     if (!plan || nblocks < 0 || rows <= 0 || cols <= 0 || rows > 65536 || cols > 65536) return M2_ERR_INVALID_ARG;

@@ -485,6 +485,43 @@ def run_monarch_cols(N1, N2, Bt, d, dtype, withK):
     plan.close()
 
 
+@pytest.mark.parametrize("B,n,d,dh,dims,dtype", [(9, 256, 128, 16, (32, 16), M.M2_BF16), (2, 100, 64, 4, (32, 16), M.M2_BF16),
+                                                  (2, 24, 12, 3, (8, 8), M.M2_FP32)])
+def test_m2_hyena_heads_fwd(B, n, d, dh, dims, dtype):
+    """The M2 Hyena layer with heads: projections, short convolutions, head outer products through the long convolution, output
+    projection (all channel-first after one transposition)."""
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    p = {k: rnd(synth.normal(synth.stream_id(14, i), (d, d)) / np.sqrt(d)) for i, k in enumerate(("W_x1", "W_x2", "W_v", "W_o"))}
+    dec = np.exp(-0.05 * np.arange(n))[None]
+    for i, k in enumerate(("K1", "K2", "K3")):
+        p[k] = (synth.normal(synth.stream_id(14, 4 + i), (d, n)) * dec / 4).astype(np.float32).astype(np.float64)
+    p["K_long"] = (synth.normal(synth.stream_id(14, 7), (d // dh, n)) * dec / 4).astype(np.float32).astype(np.float64)
+    u = rnd(synth.normal(synth.stream_id(14, 8), (B, n, d)))
+    plan = M.Plan(dims, dtype=dtype, device=0)
+    f32 = lambda a: torch.from_numpy(a.astype(np.float32)).cuda()   # noqa: E731
+    kfs = [M.m2_kernel_spectrum(plan, f32(p[k])) for k in ("K1", "K2", "K3")]
+    kfl = M.m2_kernel_spectrum(plan, f32(np.repeat(p["K_long"], dh * dh, axis=0)))
+    dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
+    W = [dv(np.ascontiguousarray(p[k].T)) for k in ("W_x1", "W_x2", "W_v", "W_o")]   # stored outputs x inputs
+    y = M.m2_hyena_heads_fwd(plan, dv(u), W, kfs[0], kfs[1], kfs[2], kfl, dh)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "hyena_heads_fwd"
+    ref = O.m2_hyena_heads(u, p, dims, dh)
+    # The first positions of a causal layer have tiny outputs (one term of every convolution), so their rows are judged
+    # against the typical row norm: an absolute error bound of 2 tol x the RMS row norm, plus the global relative bound.
+    tol = TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32
+    got = host(y).reshape(B * n, d)
+    want = ref.reshape(B * n, d)
+    assert np.isfinite(got).all()
+    gl = np.linalg.norm(got - want) / np.linalg.norm(want)
+    rms_row = np.sqrt(np.mean(np.sum(want ** 2, axis=1)))
+    worst = np.max(np.linalg.norm(got - want, axis=1)) / rms_row
+    assert gl <= tol, f"global rel-L2 {gl:.3e} > {tol}"
+    assert worst <= 2 * tol, f"worst row error {worst:.3e} of the RMS row norm > {2 * tol}"
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -387,6 +387,47 @@ def test_monarch_cols_oracle():
     assert np.allclose(O.monarch_cols(L, R, X, K), K * (Md @ X))
 
 
+def test_m2_hyena_heads_oracle():
+    """The layer against the same computation spelled out with explicit loops over heads and positions and the direct
+    O(n^2) causal convolution; causality of the whole layer; head dimension 1 = a gated double convolution."""
+    B, n, d, dh = 2, 8, 6, 2
+    dims = (4, 4)
+    p = {k: rng.standard_normal((d, d)) for k in ("W_x1", "W_x2", "W_v", "W_o")}
+    for k in ("K1", "K2", "K3"):
+        p[k] = rng.standard_normal((d, n))
+    p["K_long"] = rng.standard_normal((d // dh, n))
+    u = rng.standard_normal((B, n, d))
+    y = O.m2_hyena_heads(u, p, dims, dh)
+    conv = lambda k, x: O.direct_causal_conv(k, x)   # noqa: E731
+    want = np.zeros((B, n, d))
+    for b in range(B):
+        X1, X2, V = u[b] @ p["W_x1"], u[b] @ p["W_x2"], u[b] @ p["W_v"]     # [n, d]
+        X1c = np.stack([conv(p["K1"][c], X1[:, c]) for c in range(d)], 1)
+        X2c = np.stack([conv(p["K2"][c], X2[:, c]) for c in range(d)], 1)
+        Vc = np.stack([conv(p["K3"][c], V[:, c]) for c in range(d)], 1)
+        Oc = np.zeros((n, d))
+        for h in range(d // dh):
+            sl = slice(h * dh, (h + 1) * dh)
+            XV = np.einsum("ti,tj->tij", X2c[:, sl], Vc[:, sl])               # [n, dh, dh]
+            XVc = np.zeros_like(XV)
+            for i in range(dh):
+                for j in range(dh):
+                    XVc[:, i, j] = conv(p["K_long"][h], XV[:, i, j])
+            for t_ in range(n):
+                Oc[t_, sl] = X1c[t_, sl] @ XVc[t_]
+        want[b] = Oc @ p["W_o"]
+    assert np.allclose(y, want)
+    u2 = u.copy()
+    u2[:, 5:] += rng.standard_normal((B, 3, d))      # perturbing positions >= 5 leaves outputs < 5 unchanged
+    assert np.allclose(O.m2_hyena_heads(u2, p, dims, dh)[:, :5], y[:, :5])
+    p1 = dict(p, K_long=rng.standard_normal((d, n)))
+    y1 = O.m2_hyena_heads(u, p1, dims, 1)           # d_h = 1: y = (X1~ (.) conv(K_long, X2~ (.) V~)) W_o
+    st = {}
+    O.m2_hyena_heads(u, p1, dims, 1, stages=st)
+    inner = O.direct_causal_conv(p1["K_long"][None], st["X2c"] * st["Vc"])
+    assert np.allclose(y1, np.swapaxes(st["X1c"] * inner, 1, 2) @ p["W_o"])
+
+
 def test_m2_layer_oracle():
     """The layer against the same computation with dense matrices and einsum over the un-transposed [B, n, d] tensor;
     LayerNorm against torch's routine and its invariants (zero mean, unit variance, shift/scale invariance)."""

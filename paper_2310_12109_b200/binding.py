@@ -288,7 +288,13 @@ def m2_monarch_cols(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tenso
     return Y
 
 
-def m2_hyena_heads_fwd(plan: Plan, u: torch.Tensor, W, kf1, kf2, kf3, kf_long, dh: int) -> torch.Tensor:
+def m2_hyena_scratch(plan: Plan, B: int, n: int, d: int, dh: int, device=None) -> torch.Tensor:
+    sb = int(lib().m2_hyena_scratch_bytes(plan.handle, B, n, d, dh))
+    return torch.empty(max(sb, 16), dtype=torch.uint8, device=device if device is not None else f"cuda:{plan.device}")
+
+
+def m2_hyena_heads_fwd(plan: Plan, u: torch.Tensor, W, kf1, kf2, kf3, kf_long, dh: int, scratch: torch.Tensor | None = None,
+                       y: torch.Tensor | None = None) -> torch.Tensor:
     """The M2 Hyena layer with heads on u [B, n, d]; W = (W_X1, W_X2, W_V, W_O), each [d, d] stored outputs x inputs;
     kf1..kf3 = m2_kernel_spectrum of the short kernels [d, n]; kf_long = m2_kernel_spectrum of the long kernel repeated
     to one row per (head, i, j) channel: K_long.repeat_interleave(dh * dh, dim=0)."""
@@ -296,9 +302,10 @@ def m2_hyena_heads_fwd(plan: Plan, u: torch.Tensor, W, kf1, kf2, kf3, kf_long, d
     assert len(W) == 4 and d % dh == 0
     for a in (u, *W):
         assert a.is_cuda and a.dtype == plan.torch_dtype and a.is_contiguous()
-    y = torch.empty_like(u)
-    sb = int(lib().m2_hyena_scratch_bytes(plan.handle, B, n, d, dh))
-    scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=u.device)
+    if y is None:
+        y = torch.empty_like(u)
+    if scratch is None:   # hundreds of MB at model sizes: callers in a loop should pass one buffer (m2_hyena_scratch)
+        scratch = m2_hyena_scratch(plan, B, n, d, dh, u.device)
     wp = (ctypes.c_void_p * 4)(*[w.data_ptr() for w in W])
     _check(lib().m2_hyena_heads_fwd(plan.handle, _ptr(u), wp, _ptr(kf1), _ptr(kf2), _ptr(kf3), _ptr(kf_long), _ptr(y), B, n, d, dh,
                                     _ptr(scratch), scratch.numel(), _stream()), "m2_hyena_heads_fwd")

@@ -932,9 +932,70 @@ __global__ void heads_reduce_kernel(const IO* __restrict__ X1, const IO* __restr
     O[e] = from_f32<IO>(acc);
 }
 
+// The same on bf16 rows whose length is a multiple of 8: 16-byte accesses, one thread per (b, h dh + i, 8 positions) for the
+// outer product (its X2 piece is reused for all j) and per (b, h dh + j, 8 positions) for the contraction.
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        f[2 * q] = __uint_as_float(w[q] << 16);
+        f[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
+    }
+}
+__device__ __forceinline__ uint4 f32_to_bf16x8(const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
+        w[q] = *reinterpret_cast<uint32_t*>(&p);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__global__ void __launch_bounds__(256) heads_outer_bf16x8_kernel(const uint4* __restrict__ X2, const uint4* __restrict__ V, uint4* __restrict__ XV,
+                                                                 int d, int dh, int n8, long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n8
+    if (e >= total) return;
+    const int t8 = (int)(e % n8);
+    const int hi = (int)((e / n8) % d);
+    const long long b = e / ((long long)n8 * d);
+    float a[8], v[8], o[8];
+    bf16x8_to_f32(X2[e], a);
+    const int h0 = (hi / dh) * dh;
+    for (int j = 0; j < dh; ++j) {
+        bf16x8_to_f32(V[(b * d + h0 + j) * n8 + t8], v);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) o[q] = a[q] * v[q];
+        XV[((b * d + hi) * dh + j) * n8 + t8] = f32_to_bf16x8(o);
+    }
+}
+
+__global__ void __launch_bounds__(256) heads_reduce_bf16x8_kernel(const uint4* __restrict__ X1, const uint4* __restrict__ XVc, uint4* __restrict__ O,
+                                                                  int d, int dh, int n8, long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n8
+    if (e >= total) return;
+    const int t8 = (int)(e % n8);
+    const int c = (int)((e / n8) % d);
+    const long long b = e / ((long long)n8 * d);
+    const int h0 = (c / dh) * dh, j = c % dh;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, a[8], v[8];
+    for (int i = 0; i < dh; ++i) {
+        bf16x8_to_f32(X1[(b * d + h0 + i) * n8 + t8], a);
+        bf16x8_to_f32(XVc[((b * d + h0 + i) * dh + j) * n8 + t8], v);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc[q] = fmaf(a[q], v[q], acc[q]);
+    }
+    O[e] = f32_to_bf16x8(acc);
+}
+
 cudaError_t launch_heads_outer(const void* X2, const void* V, void* XV, long long B, int d, int dh, int n, bool bf16, cudaStream_t st) {
     const long long total = B * d * dh * n;
     if (total == 0) return cudaSuccess;
+    if (bf16 && n % 8 == 0) {
+        const long long t8 = B * d * (n / 8);
+        heads_outer_bf16x8_kernel<<<(unsigned)((t8 + 255) / 256), 256, 0, st>>>((const uint4*)X2, (const uint4*)V, (uint4*)XV, d, dh, n / 8, t8);
+        return cudaGetLastError();
+    }
     const unsigned grid = (unsigned)((total + 255) / 256);
     if (bf16)
         heads_outer_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X2, (const __nv_bfloat16*)V, (__nv_bfloat16*)XV, d, dh, n, total);
@@ -946,6 +1007,11 @@ cudaError_t launch_heads_outer(const void* X2, const void* V, void* XV, long lon
 cudaError_t launch_heads_reduce(const void* X1, const void* XVc, void* O, long long B, int d, int dh, int n, bool bf16, cudaStream_t st) {
     const long long total = B * d * n;
     if (total == 0) return cudaSuccess;
+    if (bf16 && n % 8 == 0) {
+        const long long t8 = B * d * (n / 8);
+        heads_reduce_bf16x8_kernel<<<(unsigned)((t8 + 255) / 256), 256, 0, st>>>((const uint4*)X1, (const uint4*)XVc, (uint4*)O, d, dh, n / 8, t8);
+        return cudaGetLastError();
+    }
     const unsigned grid = (unsigned)((total + 255) / 256);
     if (bf16)
         heads_reduce_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)X1, (const __nv_bfloat16*)XVc, (__nv_bfloat16*)O, d, dh, n, total);

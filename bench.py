@@ -178,7 +178,7 @@ def time_launches(fn, n, torch):
     return e0.elapsed_time(e1)
 
 
-def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5", "operator", "backward"), reps=None):
+def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "config4", "config5", "operator", "backward", "hyena"), reps=None):
     """Config 3 (Monarch matmul), config 4 (order-3 causal conv) and config 5 (M2 block forward): time per call,
     throughput and roofline fraction, outside the headline timed region."""
     out = {}
@@ -194,6 +194,28 @@ def side_workloads(torch, M, synth, peaks, quick: bool, which=("config3", "confi
         out.update(_side_operator(torch, M, synth, peaks, reps, bf))
     if "backward" in which:
         out.update(_side_backward(torch, M, synth, peaks, reps, bf))
+    if "hyena" in which:
+        out.update(_side_hyena(torch, M, synth, peaks, reps, bf))
+    return out
+
+
+def _side_hyena(torch, M, synth, peaks, reps, bf):
+    """The M2 Hyena layer with heads at B = 32, n = 256, d = 768, head dimension 16 (convolution plan N = 512): time per call."""
+    B, n, d, dh = 32, 256, 768, 16
+    torch.manual_seed(231012109)
+    plan = M.Plan((32, 16), dtype=M.M2_BF16, device=torch.cuda.current_device())
+    W = [(torch.randn(d, d, device="cuda") / d ** 0.5).to(torch.bfloat16) for _ in range(4)]
+    kfs = [M.m2_kernel_spectrum(plan, torch.randn(d, n, device="cuda") * 0.05) for _ in range(3)]
+    kfl = M.m2_kernel_spectrum(plan, (torch.randn(d // dh, n, device="cuda") * 0.05).repeat_interleave(dh * dh, dim=0).contiguous())
+    u = torch.randn(B, n, d, device="cuda").to(torch.bfloat16)
+    y = torch.empty_like(u)
+    scratch = M.m2_hyena_scratch(plan, B, n, d, dh)
+    f = lambda i: M.m2_hyena_heads_fwd(plan, u, W, kfs[0], kfs[1], kfs[2], kfl, dh, scratch=scratch, y=y)  # noqa: E731
+    time_launches(f, 2, torch)
+    ms = time_launches(f, reps, torch) / reps
+    out = {"hyena_heads_layer": {"kernel": plan.last_kernel(), "ms": ms, "tokens_per_s": B * n / (ms * 1e-3),
+                                 "shape": {"B": B, "n": n, "d": d, "head_dim": dh}, "scratch_MB": scratch.numel() / 1e6}}
+    plan.close()
     return out
 
 
@@ -520,7 +542,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-baseline leg")
     ap.add_argument("--no-side", action="store_true", help="skip the config-3 / config-4 side measurements")
     ap.add_argument("--quick", action="store_true", help="fewer repetitions of the side measurements")
-    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5", "operator", "backward"],
+    ap.add_argument("--only", default=None, choices=["config3", "config4", "config5", "operator", "backward", "hyena"],
                     help="run just this side workload (--steps launches after 2 warm-ups) and print its JSON; used for profiling")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -215,6 +215,19 @@ def _side_hyena(torch, M, synth, peaks, reps, bf):
     ms = time_launches(f, reps, torch) / reps
     out = {"hyena_heads_layer": {"kernel": plan.last_kernel(), "ms": ms, "tokens_per_s": B * n / (ms * 1e-3),
                                  "shape": {"B": B, "n": n, "d": d, "head_dim": dh}, "scratch_MB": scratch.numel() / 1e6}}
+    del scratch, kfl
+    # the gated bidirectional M2-BERT sequence mixer at the M2-BERT-base shape (circular, n = N = 512)
+    n = 512
+    kf, kfr = (M.m2_kernel_spectrum(plan, torch.randn(d, n, device="cuda") * 0.05) for _ in range(2))
+    ws = [torch.randn(d, 3, device="cuda") / 3 ** 0.5 for _ in range(3)]
+    x = torch.randn(B, n, d, device="cuda").to(torch.bfloat16)
+    y = torch.empty_like(x)
+    scratch = torch.empty(int(M.lib().m2_bert_mixer_scratch_bytes(plan.handle, B, d)), dtype=torch.uint8, device="cuda")
+    f = lambda i: M.m2_bert_mixer_fwd(plan, x, W, ws, kf, kfr, scratch=scratch, y=y)  # noqa: E731
+    time_launches(f, 2, torch)
+    ms = time_launches(f, reps, torch) / reps
+    out["bert_gated_mixer"] = {"kernel": plan.last_kernel(), "ms": ms, "tokens_per_s": B * n / (ms * 1e-3), "shape": {"B": B, "n": n, "d": d},
+                               "scratch_MB": scratch.numel() / 1e6}
     plan.close()
     return out
 

@@ -190,6 +190,23 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
 int32_t m2_monarch_cols(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, const void* K_dev,
                         int32_t act, void* Y_dev, int64_t Bt, int64_t d, void* ws_dev, int64_t ws_bytes, void* stream);
 
+/* The gated bidirectional sequence mixer of M2-BERT (Sec. 5.1 in words; Sec. 3.2's V (.) M2 (K1 (.) M1 (Q (.) K)) with M1, M2
+ * the DFT and its inverse), x: [B, n, d] with n = the plan length (circular convolutions):
+ *   Q, K, V = DW3(x W_q), DW3(x W_k), DW3(x W_v)    dense projections, then width-3 depthwise filters along the sequence
+ *                                                   (DW3(a)[t] = w0 a[t-1] + w1 a[t] + w2 a[t+1], zero padded)
+ *   y = ( V (.) conv(k, Q (.) K) + conv(k_res, x) ) W_o
+ * (the paper gives this block in words and a figure: where the residual convolution taps the input and the output
+ * projection are this library's reading).
+ * W: HOST array of 4 device pointers {W_q, W_k, W_v, W_o}, each [d][d] stored outputs x inputs; w_short: HOST array of 3
+ * device pointers to fp32 [d][3] filters (q, k, v); kf_dev, kf_res_dev: m2_kernel_spectrum of k and k_res [d, n].
+ * y_dev: [B, n, d] (must not overlap x_dev); scratch_dev: m2_bert_mixer_scratch_bytes(plan, B, d) bytes, caller-owned.
+ * After one transposition everything runs channel-first: projections = the single-block column-layout kernel, the two
+ * convolutions = m2_monarch_conv_fwd, two elementwise kernels for the filters and gates. */
+int64_t m2_bert_mixer_scratch_bytes(const m2_plan* plan, int64_t B, int64_t d);
+int32_t m2_bert_mixer_fwd(const m2_plan* plan, const void* x_dev, const void* const* W, const float* const* w_short,
+                          const void* kf_dev, const void* kf_res_dev, void* y_dev, int64_t B, int64_t d, void* scratch_dev,
+                          int64_t scratch_bytes, void* stream);
+
 /* The M2 Hyena layer with heads (App. "GPT Causal Language Modeling", the algorithm of that name), u: [B, n, d]:
  *   X1, X2, V = u W_X1, u W_X2, u W_V;  X1~, X2~, V~ = causal Monarch convolution of every channel with a short kernel;
  *   per head of dh channels: XV[t] = X2~[t] V~[t]^T, each of its dh^2 sequences through the causal Monarch convolution with

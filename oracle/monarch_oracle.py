@@ -254,6 +254,26 @@ def m2_layer(x: np.ndarray, p: dict, eps: float = 1e-5, stages: dict | None = No
     return out
 
 
+def m2_bert_mixer(x: np.ndarray, p: dict, dims: tuple, stages: dict | None = None) -> np.ndarray:
+    """The gated bidirectional sequence mixer of M2-BERT (Sec. 5.1 in words; Sec. 3.2's "more expressive layer"
+    V (.) M2 (K1 (.) M1 (Q (.) K)) with M1, M2 the DFT and its inverse), x: [B, n, d], n = prod(dims):
+        Q, K, V = DW3(x W_q), DW3(x W_k), DW3(x W_v)          dense projections, then the short depthwise convolutions
+        y = ( V (.) circconv(k, Q (.) K) + circconv(k_res, x) ) W_o     gated convolution + residual convolution, output projection
+    Weights act as x @ W ([d_in, d_out]); k, k_res: [d, n]; w_q, w_k, w_v: [d, 3].
+    (The paper gives this block in words and a figure only: where the residual convolution taps the input and the output
+    projection are this build's reading -- parity of the composition unpinned.)"""
+    cm = lambda a: np.swapaxes(a, 1, 2)
+    Q = depthwise_conv3_same(x @ p["W_q"], p["w_q"])
+    K = depthwise_conv3_same(x @ p["W_k"], p["w_k"])
+    V = depthwise_conv3_same(x @ p["W_v"], p["w_v"])
+    C = monarch_conv(p["k"][None], cm(Q * K), dims, causal=False)            # [B, d, n]
+    Cr = monarch_conv(p["k_res"][None], cm(x), dims, causal=False)
+    Z = V * cm(C) + cm(Cr)
+    if stages is not None:
+        stages.update(Q=Q, K=K, V=V, C=C, Cr=Cr, Z=Z)
+    return Z @ p["W_o"]
+
+
 def m2_hyena_heads(u: np.ndarray, p: dict, dims: tuple, dh: int, stages: dict | None = None) -> np.ndarray:
     """The M2 Hyena layer with heads (App. "GPT Causal Language Modeling", the algorithm of that name), u: [B, n, d]:
         X1, X2, V = u W_X1, u W_X2, u W_V                                     (dense projections)

@@ -39,6 +39,8 @@ SIGNATURES = {
     "m2_layer_scratch_bytes": (_i64, [_vp, _vp, _i64]),
     "m2_layer_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_cols": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _vp, _i64, _i64, _vp, _i64, _vp]),
+    "m2_bert_mixer_scratch_bytes": (_i64, [_vp, _i64, _i64]),
+    "m2_bert_mixer_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _vp, _i64, _vp]),
     "m2_hyena_scratch_bytes": (_i64, [_vp, _i64, _i64, _i64, _i64]),
     "m2_hyena_heads_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp, _i64, _vp]),
     "m2_blocks_transpose": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, _vp]),
@@ -286,6 +288,28 @@ def m2_monarch_cols(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tenso
     _check(lib().m2_monarch_cols(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(K), act, _ptr(Y), Bt, d, _ptr(ws),
                                  ws.numel() * ws.element_size(), _stream()), "m2_monarch_cols")
     return Y
+
+
+def m2_bert_mixer_fwd(plan: Plan, x: torch.Tensor, W, w_short, kf, kf_res, scratch: torch.Tensor | None = None,
+                      y: torch.Tensor | None = None) -> torch.Tensor:
+    """The gated bidirectional M2-BERT sequence mixer on x [B, n, d], n = plan.N; W = (W_q, W_k, W_v, W_o), each [d, d] stored
+    outputs x inputs; w_short = three fp32 [d, 3] filters; kf, kf_res = m2_kernel_spectrum of the long and residual kernels."""
+    B, n, d = x.shape
+    assert n == plan.N and len(W) == 4 and len(w_short) == 3
+    for a in (x, *W):
+        assert a.is_cuda and a.dtype == plan.torch_dtype and a.is_contiguous()
+    for a in w_short:
+        assert a.is_cuda and a.dtype == torch.float32 and a.is_contiguous() and tuple(a.shape) == (d, 3)
+    if y is None:
+        y = torch.empty_like(x)
+    if scratch is None:
+        sb = int(lib().m2_bert_mixer_scratch_bytes(plan.handle, B, d))
+        scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=x.device)
+    wp = (ctypes.c_void_p * 4)(*[w.data_ptr() for w in W])
+    sp = (ctypes.c_void_p * 3)(*[w.data_ptr() for w in w_short])
+    _check(lib().m2_bert_mixer_fwd(plan.handle, _ptr(x), wp, sp, _ptr(kf), _ptr(kf_res), _ptr(y), B, d, _ptr(scratch), scratch.numel(),
+                                   _stream()), "m2_bert_mixer_fwd")
+    return y
 
 
 def m2_hyena_scratch(plan: Plan, B: int, n: int, d: int, dh: int, device=None) -> torch.Tensor:

@@ -1033,4 +1033,117 @@ cudaError_t launch_dense_cols(const void* W, const void* V, void* O, long long B
     return cudaGetLastError();
 }
 
+// Gated mixer pieces on channel-first tensors [B][d][n] (n contiguous); DW3(a; w)[t] = w0 a[t-1] + w1 a[t] + w2 a[t+1], zero padded:
+//   gate_in : QK[b][c][t] = DW3(Pq[b][c]; wq[c])[t] * DW3(Pk[b][c]; wk[c])[t]
+//   gate_out: Z[b][c][t]  = DW3(Pv[b][c]; wv[c])[t] * C[b][c][t] + Cr[b][c][t]
+// one thread per element, fp32 arithmetic, one rounding on the way out (Z may alias Pv's buffer only if it does not: it reads
+// neighbours, so the output must be a different buffer)
+template <typename IO>
+__device__ __forceinline__ float dw3_at(const IO* __restrict__ row, const float* __restrict__ w, int t, int n) {
+    float g = w[1] * to_f32<IO>(row[t]);
+    if (t > 0) g = fmaf(w[0], to_f32<IO>(row[t - 1]), g);
+    if (t + 1 < n) g = fmaf(w[2], to_f32<IO>(row[t + 1]), g);
+    return g;
+}
+
+template <typename IO>
+__global__ void gate_in_kernel(const IO* __restrict__ Pq, const IO* __restrict__ Pk, const float* __restrict__ wq, const float* __restrict__ wk,
+                               IO* __restrict__ QK, int d, int n, long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n
+    if (e >= total) return;
+    const int t = (int)(e % n);
+    const long long rowi = e / n;
+    const int c = (int)(rowi % d);
+    QK[e] = from_f32<IO>(dw3_at<IO>(Pq + rowi * n, wq + 3 * c, t, n) * dw3_at<IO>(Pk + rowi * n, wk + 3 * c, t, n));
+}
+
+template <typename IO>
+__global__ void gate_out_kernel(const IO* __restrict__ Pv, const float* __restrict__ wv, const IO* __restrict__ C, const IO* __restrict__ Cr,
+                                IO* __restrict__ Z, int d, int n, long long total) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (e >= total) return;
+    const int t = (int)(e % n);
+    const long long rowi = e / n;
+    const int c = (int)(rowi % d);
+    Z[e] = from_f32<IO>(fmaf(dw3_at<IO>(Pv + rowi * n, wv + 3 * c, t, n), to_f32<IO>(C[e]), to_f32<IO>(Cr[e])));
+}
+
+// bf16 rows whose length is a multiple of 8: 8 positions per thread (one 16-byte piece plus the two neighbours)
+__device__ __forceinline__ void dw3_x8(const __nv_bfloat16* __restrict__ row, const float* __restrict__ w, int t0, int n, float* g) {
+    float a[10];
+    bf16x8_to_f32(*reinterpret_cast<const uint4*>(row + t0), a + 1);
+    a[0] = t0 > 0 ? __bfloat162float(row[t0 - 1]) : 0.f;
+    a[9] = t0 + 8 < n ? __bfloat162float(row[t0 + 8]) : 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) g[q] = fmaf(w[0], a[q], fmaf(w[1], a[q + 1], w[2] * a[q + 2]));
+}
+
+__global__ void __launch_bounds__(256) gate_in_bf16x8_kernel(const __nv_bfloat16* __restrict__ Pq, const __nv_bfloat16* __restrict__ Pk,
+                                                             const float* __restrict__ wq, const float* __restrict__ wk,
+                                                             __nv_bfloat16* __restrict__ QK, int d, int n, long long total8) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n / 8
+    if (e >= total8) return;
+    const int n8 = n / 8, t0 = (int)(e % n8) * 8;
+    const long long rowi = e / n8;
+    const int c = (int)(rowi % d);
+    float gq[8], gk[8];
+    dw3_x8(Pq + rowi * n, wq + 3 * c, t0, n, gq);
+    dw3_x8(Pk + rowi * n, wk + 3 * c, t0, n, gk);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) gq[q] *= gk[q];
+    *reinterpret_cast<uint4*>(QK + rowi * n + t0) = f32_to_bf16x8(gq);
+}
+
+__global__ void __launch_bounds__(256) gate_out_bf16x8_kernel(const __nv_bfloat16* __restrict__ Pv, const float* __restrict__ wv,
+                                                              const __nv_bfloat16* __restrict__ C, const __nv_bfloat16* __restrict__ Cr,
+                                                              __nv_bfloat16* __restrict__ Z, int d, int n, long long total8) {
+    const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (e >= total8) return;
+    const int n8 = n / 8, t0 = (int)(e % n8) * 8;
+    const long long rowi = e / n8;
+    const int c = (int)(rowi % d);
+    float gv[8], cv[8], rv[8];
+    dw3_x8(Pv + rowi * n, wv + 3 * c, t0, n, gv);
+    bf16x8_to_f32(*reinterpret_cast<const uint4*>(C + rowi * n + t0), cv);
+    bf16x8_to_f32(*reinterpret_cast<const uint4*>(Cr + rowi * n + t0), rv);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) gv[q] = fmaf(gv[q], cv[q], rv[q]);
+    *reinterpret_cast<uint4*>(Z + rowi * n + t0) = f32_to_bf16x8(gv);
+}
+
+cudaError_t launch_gate_in(const void* Pq, const void* Pk, const float* wq, const float* wk, void* QK, long long B, int d, int n, bool bf16,
+                           cudaStream_t st) {
+    const long long total = B * d * n;
+    if (total == 0) return cudaSuccess;
+    if (bf16 && n % 8 == 0) {
+        gate_in_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16*)Pq, (const __nv_bfloat16*)Pk, wq, wk,
+                                                                                  (__nv_bfloat16*)QK, d, n, total / 8);
+        return cudaGetLastError();
+    }
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (bf16)
+        gate_in_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Pq, (const __nv_bfloat16*)Pk, wq, wk, (__nv_bfloat16*)QK, d, n, total);
+    else
+        gate_in_kernel<float><<<grid, 256, 0, st>>>((const float*)Pq, (const float*)Pk, wq, wk, (float*)QK, d, n, total);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gate_out(const void* Pv, const float* wv, const void* C, const void* Cr, void* Z, long long B, int d, int n, bool bf16,
+                            cudaStream_t st) {
+    const long long total = B * d * n;
+    if (total == 0) return cudaSuccess;
+    if (bf16 && n % 8 == 0) {
+        gate_out_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16*)Pv, wv, (const __nv_bfloat16*)C,
+                                                                                   (const __nv_bfloat16*)Cr, (__nv_bfloat16*)Z, d, n, total / 8);
+        return cudaGetLastError();
+    }
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (bf16)
+        gate_out_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Pv, wv, (const __nv_bfloat16*)C, (const __nv_bfloat16*)Cr,
+                                                             (__nv_bfloat16*)Z, d, n, total);
+    else
+        gate_out_kernel<float><<<grid, 256, 0, st>>>((const float*)Pv, wv, (const float*)C, (const float*)Cr, (float*)Z, d, n, total);
+    return cudaGetLastError();
+}
+
 }  // namespace m2g

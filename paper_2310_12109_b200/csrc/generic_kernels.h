@@ -52,6 +52,12 @@ cudaError_t launch_heads_outer(const void* X2, const void* V, void* XV, long lon
 cudaError_t launch_heads_reduce(const void* X1, const void* XVc, void* O, long long B, int d, int dh, int n, bool bf16, cudaStream_t st);
 // O[bt] = W V[bt]: W [c][c] (outputs x inputs), V, O [Bt][c][cols], CUDA cores
 cudaError_t launch_dense_cols(const void* W, const void* V, void* O, long long Bt, int c, int cols, bool bf16, cudaStream_t st);
+// gated mixer pieces on channel-first tensors [B][d][n]; DW3 = width-3 depthwise filter, zero padded, weights [d][3] fp32:
+// QK = DW3(Pq) * DW3(Pk);  Z = DW3(Pv) * C + Cr  (Z must not be one of its inputs)
+cudaError_t launch_gate_in(const void* Pq, const void* Pk, const float* wq, const float* wk, void* QK, long long B, int d, int n, bool bf16,
+                           cudaStream_t st);
+cudaError_t launch_gate_out(const void* Pv, const float* wv, const void* C, const void* Cr, void* Z, long long B, int d, int n, bool bf16,
+                            cudaStream_t st);
 // conjugates a spectrum buffer: plan-order part (interleaved re, im) followed by the tensor-core kernels' private part
 cudaError_t launch_spectrum_conj(const void* in, void* out, long long plan_order_values, long long private_values, cudaStream_t st);
 

@@ -484,6 +484,59 @@ int32_t m2_layer_fwd(const m2_plan* plan_n, const m2_plan* plan_d, const void* x
     return M2_OK;
 }
 
+int64_t m2_bert_mixer_scratch_bytes(const m2_plan* plan, int64_t B, int64_t d) {
+    if (!plan || B < 0 || d < 0) return -1;
+    return 8 * round256(B * d * plan->N * (plan->dtype == M2_BF16 ? 2 : 4));
+}
+
+int32_t m2_bert_mixer_fwd(const m2_plan* plan, const void* x_dev, const void* const* W, const float* const* w_short, const void* kf_dev,
+                          const void* kf_res_dev, void* y_dev, int64_t B, int64_t d, void* scratch_dev, int64_t scratch_bytes, void* stream) {
+    if (!plan || !W || !w_short || B < 0 || d <= 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    const int64_t n = plan->N;   // bidirectional: circular convolution over the whole plan length
+    if (B > 65535 || d > 65535 || B * d * n > 0x7fffffffffLL) return M2_ERR_UNSUPPORTED;
+    if (B == 0) return M2_OK;
+    for (int i = 0; i < 4; ++i)
+        if (!W[i] || !aligned16(W[i])) return W[i] ? M2_ERR_ALIGNMENT : M2_ERR_INVALID_ARG;
+    for (int i = 0; i < 3; ++i)
+        if (!w_short[i]) return M2_ERR_INVALID_ARG;
+    if (!x_dev || !kf_dev || !kf_res_dev || !y_dev || !scratch_dev) return M2_ERR_INVALID_ARG;
+    if (!aligned16(x_dev) || !aligned16(y_dev) || !aligned16(scratch_dev)) return M2_ERR_ALIGNMENT;
+    if (scratch_bytes < m2_bert_mixer_scratch_bytes(plan, B, d)) return M2_ERR_INVALID_ARG;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool bf = plan->dtype == M2_BF16;
+    const int64_t tb = round256(B * d * n * (bf ? 2 : 4));
+    unsigned char* sc = static_cast<unsigned char*>(scratch_dev);
+    void *xT = sc, *Pq = sc + tb, *Pk = sc + 2 * tb, *Pv = sc + 3 * tb, *QK = sc + 4 * tb, *C = sc + 5 * tb, *Cr = sc + 6 * tb, *Z = sc + 7 * tb;
+    auto dense = [&](const void* Wm, const void* V, void* O) -> int32_t {   // O[b] = Wm V[b] on [B][d][n]
+        int32_t rc = m2c::dense(plan, Wm, V, O, B, d, n, st);
+        if (rc != M2_ERR_UNSUPPORTED) return rc;
+        const cudaError_t e = m2g::launch_dense_cols(Wm, V, O, B, (int)d, (int)n, bf, st);
+        if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+        if (e != cudaSuccess) return M2_ERR_CUDA;
+        plan->launches += 1;
+        return M2_OK;
+    };
+    if (m2g::launch_transpose_any(x_dev, xT, B, (int)n, (int)d, bf, st) != cudaSuccess) return M2_ERR_CUDA;   // channel-first from here on
+    int32_t rc = dense(W[0], xT, Pq);
+    if (rc == M2_OK) rc = dense(W[1], xT, Pk);
+    if (rc == M2_OK) rc = dense(W[2], xT, Pv);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_gate_in(Pq, Pk, w_short[0], w_short[1], QK, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    rc = m2_monarch_conv_fwd(plan, QK, kf_dev, C, B, d, n, M2_CIRCULAR, stream);
+    if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, xT, kf_res_dev, Cr, B, d, n, M2_CIRCULAR, stream);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_gate_out(Pv, w_short[2], C, Cr, Z, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    rc = dense(W[3], Z, Pq);
+    if (rc != M2_OK) return rc;
+    if (m2g::launch_transpose_any(Pq, y_dev, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    plan->launches += 4;
+    plan->last_kernel = "bert_mixer_fwd";
+    return M2_OK;
+}
+
 int64_t m2_hyena_scratch_bytes(const m2_plan* plan, int64_t B, int64_t n, int64_t d, int64_t dh) {
     if (!plan || B < 0 || n < 0 || d < 0 || dh <= 0) return -1;
     return (7 + 2 * dh) * round256(B * d * n * (plan->dtype == M2_BF16 ? 2 : 4));

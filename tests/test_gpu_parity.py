@@ -522,6 +522,33 @@ def test_m2_hyena_heads_fwd(B, n, d, dh, dims, dtype):
     plan.close()
 
 
+@pytest.mark.parametrize("B,d,dims,dtype", [(12, 128, (32, 16), M.M2_BF16), (3, 24, (32, 16), M.M2_BF16), (2, 10, (6, 4), M.M2_FP32)])
+def test_m2_bert_mixer_fwd(B, d, dims, dtype):
+    """The gated bidirectional M2-BERT sequence mixer: projections, short filters, gated long convolution + residual convolution,
+    output projection."""
+    n = int(np.prod(dims))
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    p = {k: rnd(synth.normal(synth.stream_id(15, i), (d, d)) / np.sqrt(d)) for i, k in enumerate(("W_q", "W_k", "W_v", "W_o"))}
+    for i, k in enumerate(("w_q", "w_k", "w_v")):
+        p[k] = (synth.normal(synth.stream_id(15, 4 + i), (d, 3)) / np.sqrt(3.0)).astype(np.float32).astype(np.float64)
+    dec = np.exp(-0.02 * np.arange(n))[None]
+    p["k"] = (synth.normal(synth.stream_id(15, 7), (d, n)) * dec / 4).astype(np.float32).astype(np.float64)
+    p["k_res"] = (synth.normal(synth.stream_id(15, 8), (d, n)) * dec / 4).astype(np.float32).astype(np.float64)
+    x = rnd(synth.normal(synth.stream_id(15, 9), (B, n, d)))
+    plan = M.Plan(dims, dtype=dtype, device=0)
+    f32 = lambda a: torch.from_numpy(a.astype(np.float32)).cuda()   # noqa: E731
+    kf, kfr = M.m2_kernel_spectrum(plan, f32(p["k"])), M.m2_kernel_spectrum(plan, f32(p["k_res"]))
+    dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
+    W = [dv(np.ascontiguousarray(p[k].T)) for k in ("W_q", "W_k", "W_v", "W_o")]
+    y = M.m2_bert_mixer_fwd(plan, dv(x), W, [f32(p[k]) for k in ("w_q", "w_k", "w_v")], kf, kfr)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "bert_mixer_fwd"
+    ref = O.m2_bert_mixer(x, p, dims)
+    check(host(y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, "M2-BERT gated mixer")
+    plan.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

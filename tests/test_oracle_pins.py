@@ -387,6 +387,41 @@ def test_monarch_cols_oracle():
     assert np.allclose(O.monarch_cols(L, R, X, K), K * (Md @ X))
 
 
+def test_m2_bert_mixer_oracle():
+    """The gated mixer against explicit per-channel loops with the direct O(n^2) circular convolution; with identity
+    projections and the pass-through short filter (0, 1, 0) it is x (.) conv(k, x (.) x) + conv(k_res, x); circular-shift
+    equivariance along the sequence does not hold with zero-padded short filters unless they are pass-through, where it does."""
+    B, dims, d = 2, (4, 4), 5
+    n = 16
+    p = {k: rng.standard_normal((d, d)) for k in ("W_q", "W_k", "W_v", "W_o")}
+    for k in ("w_q", "w_k", "w_v"):
+        p[k] = rng.standard_normal((d, 3))
+    p["k"], p["k_res"] = rng.standard_normal((d, n)), rng.standard_normal((d, n))
+    x = rng.standard_normal((B, n, d))
+    y = O.m2_bert_mixer(x, p, dims)
+    want = np.zeros_like(y)
+    for b in range(B):
+        def dw(a, w):   # [n, d], zero padded, centred
+            g = np.zeros_like(a)
+            for t_ in range(n):
+                for c in range(d):
+                    g[t_, c] = w[c, 1] * a[t_, c] + (w[c, 0] * a[t_ - 1, c] if t_ > 0 else 0.0) + (w[c, 2] * a[t_ + 1, c] if t_ + 1 < n else 0.0)
+            return g
+        Q, K, V = dw(x[b] @ p["W_q"], p["w_q"]), dw(x[b] @ p["W_k"], p["w_k"]), dw(x[b] @ p["W_v"], p["w_v"])
+        Z = np.zeros((n, d))
+        for c in range(d):
+            Z[:, c] = V[:, c] * O.direct_circular_conv(p["k"][c], Q[:, c] * K[:, c]) + O.direct_circular_conv(p["k_res"][c], x[b][:, c])
+        want[b] = Z @ p["W_o"]
+    assert np.allclose(y, want)
+    eye = np.eye(d)
+    thru = np.tile(np.array([0.0, 1.0, 0.0]), (d, 1))
+    p2 = dict(p, W_q=eye, W_k=eye, W_v=eye, W_o=eye, w_q=thru, w_k=thru, w_v=thru)
+    xc = np.swapaxes(x, 1, 2)
+    want2 = xc * O.direct_circular_conv(p["k"][None], xc * xc) + O.direct_circular_conv(p["k_res"][None], xc)
+    assert np.allclose(O.m2_bert_mixer(x, p2, dims), np.swapaxes(want2, 1, 2))
+    assert np.allclose(O.m2_bert_mixer(np.roll(x, 3, axis=1), p2, dims), np.roll(O.m2_bert_mixer(x, p2, dims), 3, axis=1))
+
+
 def test_m2_hyena_heads_oracle():
     """The layer against the same computation spelled out with explicit loops over heads and positions and the direct
     O(n^2) causal convolution; causality of the whole layer; head dimension 1 = a gated double convolution."""

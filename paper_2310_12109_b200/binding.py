@@ -336,6 +336,12 @@ def m2_hyena_heads_fwd(plan: Plan, u: torch.Tensor, W, kf1, kf2, kf3, kf_long, d
     return y
 
 
+def m2_monarch_cols_bwd_input(plan_t: Plan, G: torch.Tensor, L: torch.Tensor, R: torch.Tensor, ws: torch.Tensor | None = None):
+    """dX = M^T G for Y = M X in the column layout (X, G: [Bt, N, d]): the forward call with the block-wise transposed factors
+    in swapped roles.  plan_t: a plan with the factors (N2, N1) (the forward plan itself when N1 == N2)."""
+    return m2_monarch_cols(plan_t, G, m2_blocks_transpose(plan_t, R), m2_blocks_transpose(plan_t, L), ws=ws)
+
+
 def m2_blocks_transpose(plan: Plan, W: torch.Tensor) -> torch.Tensor:
     """W: [nblocks, rows, cols] CUDA tensor of the plan dtype; returns [nblocks, cols, rows]."""
     assert W.is_cuda and W.dtype == plan.torch_dtype and W.is_contiguous() and W.dim() == 3

@@ -464,6 +464,24 @@ def test_monarch_cols_rectangular(N1, N2, d):
     run_monarch_cols(N1, N2, 2, d, M.M2_BF16, True)
 
 
+@pytest.mark.parametrize("N1,N2,d,dtype", [(64, 64, 72, M.M2_BF16), (64, 128, 64, M.M2_BF16), (5, 3, 7, M.M2_FP32)])
+def test_monarch_cols_input_gradient(N1, N2, d, dtype):
+    """dX = M^T G in the column layout: the forward kernels with swapped, block-transposed factors on the (N2, N1) plan."""
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    L = rnd(synth.normal(synth.stream_id(16, 0), (N1, N2, N2)) / np.sqrt(N2))
+    R = rnd(synth.normal(synth.stream_id(16, 1), (N2, N1, N1)) / np.sqrt(N1))
+    G = rnd(synth.normal(synth.stream_id(16, 2), (2, N1 * N2, d)))
+    plan_t = M.Plan((N2, N1), dtype=dtype, device=0)
+    dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
+    dX = M.m2_monarch_cols_bwd_input(plan_t, dv(G), dv(L), dv(R))
+    torch.cuda.synchronize()
+    assert plan_t.device_status() == 0
+    ref = np.swapaxes(O.monarch_apply_transpose(L, R, np.swapaxes(G, 1, 2)), 1, 2)   # M^T applied down the columns
+    check(host(dX), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, "cols input gradient")
+    plan_t.close()
+
+
 def run_monarch_cols(N1, N2, Bt, d, dtype, withK):
     b = N1
     N = N1 * N2

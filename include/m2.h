@@ -60,12 +60,17 @@ enum m2_table {
 
 /* Creates a plan for length N = factors[0]*..*factors[p-1] (p = 2 or 3 for the convolution; the
  * matmul uses p = 2).  dtype is the storage type of x / y (M2_FP32: float, M2_BF16: bfloat16);
- * accumulation is always fp32.  sign = +1 (paper) or -1.  device >= 0: CUDA device ordinal, tables
+ * every sum is accumulated in fp32.  (Between stages bf16 plans round: the tensor-core kernels re-round the
+ * operands of every stage to bf16, and the general-shape convolution kernel, for 20480 < N <= 51200 where
+ * a complex fp32 row no longer fits in shared memory, keeps the row between its stages as bf16 pairs.)  sign = +1 (paper) or -1.  device >= 0: CUDA device ordinal, tables
  * are uploaded (the call synchronises).  device < 0: host-only plan, usable only with
  * m2_plan_get_table.  (Eq. 1: the factorisation N = N1..Np with block size N^(1/p); Corollary
  * "DFT is M": the twiddles.)  A plan carries a little device state of its own (a status word, work
  * counters of its kernels): calls on one plan must be ordered on the GPU -- one stream, or events
- * between streams; use one plan per stream for calls that may overlap. */
+ * between streams; use one plan per stream for calls that may overlap.  A plan also carries host-side
+ * bookkeeping (launch count, name of the last kernel) that is not synchronised: do not use one plan from
+ * two host threads at the same time (give each thread its own plan; the library's global state -- the
+ * per-device kernel attributes and the static scratch address -- is safe to reach from several threads). */
 int32_t m2_plan_create(m2_plan** out, int64_t N, int32_t p, const int32_t* factors, int32_t dtype,
                        int32_t sign, int32_t device);
 int32_t m2_plan_destroy(m2_plan* plan);
@@ -238,9 +243,12 @@ int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_o
  *   dR[n2][k1][n1] = sum_t dv[t][n2][k1] X[t][n1 N2 + n2],          dv = L^T-stage applied to G.
  * X_dev, G_dev: [T, N], L_dev, R_dev as in m2_monarch_matmul (plan dtype); dL_dev [N1][N2][N2] and dR_dev [N2][N1][N1]
  * are fp32 and overwritten (zeros for T == 0).  ws_dev: caller-owned, at least m2_matmul_bwd_workspace_bytes(plan, T)
- * = 4 T N bytes (holds v, then dv), 16-byte aligned; too small or NULL with T > 0: M2_ERR_INVALID_ARG.  fp32
- * CUDA-core kernels with a fixed summation order (deterministic).  (The paper trains through the operator, Sec. 5,
- * without writing the backward pass out.) */
+ * bytes (at least 4 T N: it holds v, then dv; bf16 plans with 64 x 64 blocks add room for the partial sums of the
+ * token shares and one transposed factor), 16-byte aligned; too small or NULL with T > 0: M2_ERR_INVALID_ARG.
+ * bf16 plans with 64 x 64 blocks run on the tensor cores with the tokens as the contraction dimension (v and dv pass
+ * through bf16 like the forward intermediate; partial sums per token share in fp32, added in a fixed order); every
+ * other plan runs four fp32 CUDA-core kernels with a fixed summation order.  Both are deterministic.  (The paper
+ * trains through the operator, Sec. 5, without writing the backward pass out.) */
 int64_t m2_matmul_bwd_workspace_bytes(const m2_plan* plan, int64_t T);
 int32_t m2_monarch_matmul_bwd_weights(const m2_plan* plan, const void* X_dev, const void* G_dev, const void* L_dev,
                                       const void* R_dev, float* dL_dev, float* dR_dev, int64_t T, void* ws_dev,
@@ -278,6 +286,18 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
 int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
                             const void* W_up_dev, const void* W_down_dev, void* y_dev, int64_t B, int64_t T,
                             int64_t C, int32_t nblk, int32_t expand, void* stream);
+
+/* Self-test of the device-side bounded waits (the paper has no counterpart; a test and diagnosis aid).  Every wait
+ * inside the tensor-core kernels -- for a TMA copy, for a tensor-core commit -- gives up after a fixed number of
+ * polls; the pipeline that gave up sets M2_ERR_TIMEOUT in the plan's status word, waits (again bounded) for its own
+ * copies in flight, releases its tensor memory and returns, so that the context stays usable.  This call launches the
+ * row-pair N = 512 convolution kernel with the arguments of m2_monarch_conv_fwd in a mode where no input copy is issued
+ * and every wait gives up after a few polls: each pipeline's first wait runs out with nothing in flight and the kernel
+ * leaves through that abort path.  y_dev is not written.  Afterwards m2_last_device_status reports M2_ERR_TIMEOUT
+ * (and resets it) and the plan serves ordinary calls as before.  Needs a bf16 plan with N = 512 = 32 x 16 and B > 8;
+ * M2_ERR_UNSUPPORTED otherwise. */
+int32_t m2_selftest_bounded_wait(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
+                                 int64_t H, int64_t n, int32_t mode, void* stream);
 
 const char* m2_status_string(int32_t status);
 

@@ -160,12 +160,16 @@ def gelu_erf(v: np.ndarray) -> np.ndarray:
 
 
 def blockdiag_apply(W: np.ndarray, x: np.ndarray) -> np.ndarray:
-    """out[..., b, n] = sum_m W[b, n, m] x[..., b, m] on the last axis split into
-    nblocks groups (the blockdiag_matmul listing, App. A)."""
+    """Multiplication by the block-diagonal matrix diag(W[0], .., W[nb-1]) of Sec. 3.1 along the last axis: the vector
+    is cut into nb consecutive segments and segment b is multiplied by its own block W[b] (out x in), one block after
+    the other."""
     nb, o, i = W.shape
-    xs = x.reshape(*x.shape[:-1], nb, i)
-    out = np.einsum("bnm,...bm->...bn", W, xs)
-    return out.reshape(*x.shape[:-1], nb * o)
+    assert x.shape[-1] == nb * i
+    out = np.empty(x.shape[:-1] + (nb * o,), dtype=np.result_type(W.dtype, x.dtype))
+    for b in range(nb):
+        seg = x[..., b * i:(b + 1) * i]                       # the inputs of block b
+        out[..., b * o:(b + 1) * o] = seg @ W[b].T            # (W[b] seg) for every leading index
+    return out
 
 
 # ----------------------------------------------------------------------------

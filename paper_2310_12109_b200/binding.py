@@ -50,6 +50,7 @@ SIGNATURES = {
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
     "m2_block_fwd_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
+    "m2_selftest_bounded_wait": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_status_string": (ctypes.c_char_p, [_i32]),
     "m2_last_device_status": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "m2_last_kernel_name": (ctypes.c_char_p, [_vp]),
@@ -195,6 +196,15 @@ def m2_monarch_conv_fwd(plan: Plan, x: torch.Tensor, kf: torch.Tensor, mode: int
     _check(lib().m2_monarch_conv_fwd(plan.handle, _ptr(x), _ptr(kf), _ptr(y), B, H, n, mode, _stream()),
            "m2_monarch_conv_fwd")
     return y
+
+
+def m2_selftest_bounded_wait(plan: Plan, x: torch.Tensor, kf: torch.Tensor, mode: int, y: torch.Tensor):
+    """Launches the row-pair convolution kernel so that its first bounded wait runs out; y is left untouched and the
+    plan's device status reads M2_ERR_TIMEOUT afterwards."""
+    assert x.is_cuda and x.dtype == plan.torch_dtype and x.is_contiguous() and x.dim() == 3
+    B, H, n = x.shape
+    _check(lib().m2_selftest_bounded_wait(plan.handle, _ptr(x), _ptr(kf), _ptr(y), B, H, n, mode, _stream()),
+           "m2_selftest_bounded_wait")
 
 
 def m2_monarch_conv_fwd_host(plan: Plan, x_host: torch.Tensor, kf: torch.Tensor, y_host: torch.Tensor,

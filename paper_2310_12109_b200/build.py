@@ -16,7 +16,7 @@ OBJ_DIR = os.path.join(HERE, "build")
 SOURCES = ["m2_api.cu", "generic_kernels.cu", "conv_umma.cu", "conv_umma3.cu", "matmul_umma.cu", "mlp_umma.cu", "cols_umma.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "--use_fast_math=false",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -40,7 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     os.makedirs(OBJ_DIR, exist_ok=True)
     nvcc = _nvcc()
-    flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
+    flags = list(NVCC_FLAGS)
     if verbose:
         flags = flags + ["-Xptxas", "-v"]
 

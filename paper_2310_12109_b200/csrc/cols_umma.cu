@@ -17,6 +17,8 @@
 // multiples of 64 (an output tile past the end of a block is clipped by the store's tensor map), d a multiple of 8 (a ragged
 // last column tile is zero-filled on the way in and clipped on the way out).  All waits are bounded.
 #include <cuda.h>
+
+#include <atomic>
 #include <cuda_bf16.h>
 
 #include <cstring>
@@ -250,13 +252,14 @@ bool covered(const m2_plan* pl, int64_t d) {
 }
 
 cudaError_t prepare() {
-    static bool done[64] = {};
+    // per-device opt-in; setting the attribute twice is harmless, so host threads only need the flag itself to be race-free
+    static std::atomic<bool> done[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+    if (dev >= 0 && dev < 64 && done[dev].load(std::memory_order_acquire)) return cudaSuccess;
     e = cudaFuncSetAttribute(monarch_cols_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+    if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev].store(true, std::memory_order_release);
     return e;
 }
 

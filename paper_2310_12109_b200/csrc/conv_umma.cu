@@ -428,7 +428,7 @@ static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols 
 __global__ void __launch_bounds__(kThreadsP, 1)
 conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
-               int32_t* __restrict__ status, int* __restrict__ sched) {
+               int32_t* __restrict__ status, int* __restrict__ sched, int selftest) {
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
@@ -461,6 +461,10 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // their SMs; everything above the wait below touches only plan-owned constants and this CTA's own resources.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool x_pending = false;
+    // Self-test of the bounded waits (selftest != 0): no input copy is ever issued and every wait gives up after a few polls,
+    // so each pipeline's first wait -- on a barrier nothing will arrive on, with nothing in flight -- runs out and the pipeline
+    // leaves through the abort path below exactly as it would after a lost copy.
+    const uint32_t wlim = selftest ? 16u : (1u << 22);
     // constants -> shared memory
     {
         uint4* dst = reinterpret_cast<uint4*>(smem_all);
@@ -474,6 +478,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // past the end of the batch read zeros).  A box is [8 rows][32 n1][16 n2] with 32-byte rows, 32-byte swizzled: as it lies
     // it is the M-major operand of S1 with M = (row, n2) -- 16-element M blocks 1 KB apart, groups of 8 n1 256 B apart.
     auto load_unit = [&](int v) {
+        if (selftest) return;
         mbar_expect_tx(bar_x, 16384);
         const int hh = v % H, bb = (v / H) * 2 * kRows;
         tma_load_4d(s_base + P_G_X, &map_x, 0, 0, hh, bb, bar_x);
@@ -512,7 +517,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int b0 = (u / H) * 2 * kRows;
         // ---- S1 ---------------------------------------------------------------------------------
         if (leader) {
-            ok = mbar_wait(bar_x, ph_x);
+            ok = mbar_wait(bar_x, ph_x, wlim);
             x_pending = false;
             if (ok) {
                 tc_fence_after();
@@ -530,7 +535,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         }
         ph_x ^= 1;
         // ---- h1: twiddle, A2 ---------------------------------------------------------------------
-        ok = ok && mbar_wait(bar_mma, ph_m);
+        ok = ok && mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
         if (leader) un2 = 2 * ustride + atomicAdd(sched, 1);   // consumed at the end of this unit
@@ -589,7 +594,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         float4 kw[8];   // this thread's 16 spectrum values (k1 fixed), requested before the accumulator is waited for
 #pragma unroll
         for (int q = 0; q < 8; ++q) kw[q] = __ldg(kfu_k1 + (size_t)h * 256 + q * 32);
-        ok = mbar_wait(bar_mma, ph_m);
+        ok = mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
         if (ok) {
@@ -640,7 +645,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             umma_commit(bar_mma);
         }
         // ---- h3: conjugate twiddle, A4 --------------------------------------------------------------
-        ok = mbar_wait(bar_mma, ph_m);
+        ok = mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
         if (ok) {
@@ -692,7 +697,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ---- h4: round and stage: lane (r, n2) holds y[r][n1*16 + n2] for all n1 of the real-part row and of the
         //      imaginary-part row; the operand buffer (free now) takes the two boxes [8 rows][32 n1][16 n2] in the
         //      32-byte-swizzled image of the TMA stores (16-byte chunk XOR bit 7 of the address) ---------------
-        ok = mbar_wait(bar_mma, ph_m);
+        ok = mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
         if (ok) {
@@ -729,7 +734,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // ---- teardown: nothing of ours may still be in flight when the TMEM and the CTA go away ----------
     if (leader) {
         if (aborted) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-        if (x_pending) mbar_wait(bar_x, ph_x);
+        if (x_pending) mbar_wait(bar_x, ph_x, wlim);
         tma_store_wait_read0();
         __threadfence();
         if (atomicAdd(sched + 1, 1) == ustride - 1) {   // last pipeline out: reset the scheduler words
@@ -1099,18 +1104,8 @@ static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_
     return tma_host::encode_sw32_bf16(map, ptr, 4, gdim, gstr, box);
 }
 
-
-// development switch: M2_CONV512_PAIRS=0 in the environment selects the one-row-per-lane kernel for every batch size
-static bool pair_kernel_enabled() {
-    static const bool on = [] {
-        const char* v = std::getenv("M2_CONV512_PAIRS");
-        return !(v && v[0] == '0');
-    }();
-    return on;
-}
-
-int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
-                 cudaStream_t stream) {
+static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
+                             cudaStream_t stream, int selftest) {
     if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
     // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
@@ -1118,7 +1113,8 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const bool pairs = B > kRows && pair_kernel_enabled();   // two batch rows per complex row once there are more than 8
+    const bool pairs = B > kRows;   // two batch rows per complex row once there are more than 8
+    if (selftest && !pairs) return M2_ERR_UNSUPPORTED;
     const long long units = pairs ? H * ((B + 2 * kRows - 1) / (2 * kRows)) : H * ((B + kRows - 1) / kRows);
     const int groups = pairs ? kGroupsP : kGroups;
     const long long ctas = (units + groups - 1) / groups;
@@ -1142,7 +1138,7 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
         alignas(64) CUtensorMap mx32;   // the row-pair kernel reads whole 32-byte rows of 16 n2
         if (!make_map_rows32(&mx32, x, B, H, n)) return M2_ERR_UNSUPPORTED;
         if (cudaLaunchKernelEx(&cfg, conv512p_kernel, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H, (int)n,
-                               pl->d_status, t->d_sched) != cudaSuccess)
+                               pl->d_status, t->d_sched, selftest) != cudaSuccess)
             return M2_ERR_CUDA;
     } else {
         alignas(64) CUtensorMap mx;
@@ -1151,9 +1147,19 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
                                t->d_sched) != cudaSuccess)
             return M2_ERR_CUDA;
     }
-    pl->last_kernel = "conv_umma_o2_512";
+    pl->last_kernel = pairs ? "conv_umma_o2_512_pairs" : "conv_umma_o2_512_rows";
     pl->launches += 1;
     return M2_OK;
+}
+
+int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
+                 cudaStream_t stream) {
+    return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 0);
+}
+
+int32_t conv_fwd_wait_selftest(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
+                               cudaStream_t stream) {
+    return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 1);
 }
 
 // dk[h] = Re M^-1 ( sum_p partial[p][h][:] ) [0:n) / 512 for N = 512 = 32 x 16: the parts added in index order, then the two

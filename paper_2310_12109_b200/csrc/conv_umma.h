@@ -14,6 +14,11 @@ void destroy_tables(m2_plan* plan);
 // the CUDA-core kernels), M2_OK after enqueueing, another status on failure.
 int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
                  int32_t mode, cudaStream_t stream);
+// The row-pair kernel launched so that every pipeline's first bounded wait runs out with nothing in flight (no copy is
+// issued, a few polls per wait): the kernel leaves through its abort path, sets M2_ERR_TIMEOUT in the plan's status
+// word, writes nothing to y.  Needs B > 8 (the row-pair kernel); M2_ERR_UNSUPPORTED otherwise.
+int32_t conv_fwd_wait_selftest(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
+                               int32_t mode, cudaStream_t stream);
 
 // Kernel gradient, tensor-core part: partial[b group][h][512] = sum over the group's 8 rows of conj(M x) (.) M g in plan
 // order (complex fp32, conv_wgrad_workspace_bytes(plan, B, H) bytes); *parts = number of b groups.

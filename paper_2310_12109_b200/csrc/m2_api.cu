@@ -317,6 +317,16 @@ int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* 
     return M2_OK;
 }
 
+int32_t m2_selftest_bounded_wait(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B, int64_t H, int64_t n,
+                                 int32_t mode, void* stream) {
+    int32_t st = check_conv_args(plan, x_dev, kf_dev, y_dev, B, H, n, mode);
+    if (st != M2_OK) return st;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (B * H == 0) return M2_ERR_UNSUPPORTED;
+    return m2u::conv_fwd_wait_selftest(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
+}
+
 int32_t m2_monarch_conv_fwd_host(const m2_plan* plan, const void* x_host, const void* kf_dev, void* y_host,
                                  void* x_dev_scratch, void* y_dev_scratch, int64_t B, int64_t H, int64_t n, int32_t mode,
                                  void* stream) {
@@ -689,6 +699,7 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
     if (plan->device < 0) return M2_ERR_NO_DEVICE;
     if (B < 0 || C <= 0 || nblk <= 0 || expand <= 0 || C % nblk != 0 || T != plan->N) return M2_ERR_INVALID_ARG;
     if (plan->dtype != M2_BF16 || plan->p < 2 || plan->p > 3) return M2_ERR_UNSUPPORTED;
+    if (B > 0x7fffffffLL / T || B * T > 0x7fffffffffLL / C) return M2_ERR_UNSUPPORTED;   // token and element counts stay far from wrapping
     if (!aligned16(x_dev) || !aligned16(kf_dev) || !aligned16(W_up_dev) || !aligned16(W_down_dev) || !aligned16(z_dev) ||
         !aligned16(y_dev))
         return M2_ERR_ALIGNMENT;
@@ -720,7 +731,7 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
     if (plan->device < 0) return M2_ERR_NO_DEVICE;
     if (B < 0 || C <= 0 || nblk <= 0 || expand <= 0 || C % nblk != 0 || T != plan->N) return M2_ERR_INVALID_ARG;
     if (plan->dtype != M2_BF16 || plan->p < 2 || plan->p > 3) return M2_ERR_UNSUPPORTED;
-    if (B * T * C * 2 > (int64_t)M2_STATIC_SCRATCH_BYTES) return M2_ERR_UNSUPPORTED;   // z would not fit the fixed array
+    if (B > (int64_t)M2_STATIC_SCRATCH_BYTES / 2 / T / C) return M2_ERR_UNSUPPORTED;   // z would not fit the fixed array (no product that could wrap)
     if (!aligned16(x_dev) || !aligned16(kf_dev) || !aligned16(W_up_dev) || !aligned16(W_down_dev) || !aligned16(y_dev))
         return M2_ERR_ALIGNMENT;
     if (plan->device >= kMaxDevices) return M2_ERR_UNSUPPORTED;
@@ -750,12 +761,13 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
     if (m2mlp::covered((int)C, nblk, expand)) {
         const int32_t st = m2mlp::launch(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
         if (st != M2_OK) return st;
+        plan->last_kernel = tc_mix ? "block_conv_umma_mlp_umma_static" : "block_conv_generic_mlp_umma_static";
     } else {
         e = m2g::launch_mlp(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, expand, B * T, (cudaStream_t)stream);
         if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
         if (e != cudaSuccess) return M2_ERR_CUDA;
+        plan->last_kernel = tc_mix ? "block_conv_umma_mlp_generic_static" : "block_generic_static";
     }
-    plan->last_kernel = "block_generic_static_scratch";
     plan->launches += nl + 1;
     return M2_OK;
 }

@@ -12,6 +12,8 @@
 // are the GELU warps (lane quarter = warp % 4, 32 of the 128 chunk columns each).  All operands are K-major with the
 // 128-byte swizzle, written by TMA (Z, weights) or by the GELU warps (G).  Every wait is bounded.
 #include <cuda.h>
+
+#include <atomic>
 #include <cuda_bf16.h>
 
 #include "mlp_umma.h"
@@ -258,13 +260,13 @@ cudaError_t prepare() { return cudaFuncSetAttribute(mlp_umma_kernel, cudaFuncAtt
 int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, long long tokens, int32_t* status,
                cudaStream_t stream) {
     if (tokens == 0) return M2_OK;
-    {   // the shared-memory opt-in is per device
-        static bool prepared[64] = {};
+    {   // the shared-memory opt-in is per device (setting it twice is harmless; the flag itself is race-free)
+        static std::atomic<bool> prepared[64];
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return M2_ERR_CUDA;
-        if (!prepared[dev]) {
+        if (!prepared[dev].load(std::memory_order_acquire)) {
             if (prepare() != cudaSuccess) return M2_ERR_CUDA;
-            prepared[dev] = true;
+            prepared[dev].store(true, std::memory_order_release);
         }
     }
     alignas(64) CUtensorMap mz, mw1, mw2, my;

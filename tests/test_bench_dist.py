@@ -46,3 +46,15 @@ def test_reference_arm_prints_one_json_line():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
     assert d["value"] > 0 and d["unit"] == "tokens*ch/s"
+
+
+def test_gpus_flag_without_launcher_never_reports_one_gpu():
+    """`bench.py --gpus 2` started without a launcher must start two ranks itself or refuse; on a box with fewer GPUs it
+    refuses with a non-zero exit code and prints no result line."""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "2", "--warmup", "1"],
+                       capture_output=True, text=True, timeout=300, env={k: v for k, v in os.environ.items() if k != "WORLD_SIZE"})
+    import torch
+    if torch.cuda.device_count() < 2:
+        assert r.returncode != 0 and "n_gpus" not in r.stdout
+    else:
+        assert r.returncode == 0 and '"n_gpus": 2' in r.stdout

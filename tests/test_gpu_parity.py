@@ -113,6 +113,8 @@ def test_config2_small_full_compare(B, H):   # more than 8 batch rows: the kerne
     y, name = run_conv(c["dims"], c["x"], c["k"], False, M.M2_BF16)
     ref = O.monarch_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64), c["dims"], causal=False)
     check(y, ref, TOL_BF16, f"config2 B={B} H={H} {name}")
+    # up to 8 batch rows: one row per lane; more: two batch rows packed as one complex row
+    assert name == ("conv_umma_o2_512_pairs" if B > 8 else "conv_umma_o2_512_rows")
 
 
 def test_config2_full_size():
@@ -121,6 +123,7 @@ def test_config2_full_size():
     x64, k64 = c["x"].astype(np.float64), c["k"].astype(np.float64)
     ref = O.monarch_conv(k64[None], x64, c["dims"], causal=False)
     check(y, ref, TOL_BF16, "config2 full " + name)
+    assert name == "conv_umma_o2_512_pairs"
     # sampled rows against the direct O(N^2) sum
     for b, h in [(0, 0), (31, 767), (7, 100), (16, 384), (1, 766), (30, 1), (12, 511), (5, 513)]:
         d = O.direct_circular_conv(k64[h], x64[b, h])
@@ -172,15 +175,20 @@ def test_matmul_fp32_rectangular_vs_dense():
     plan.close()
 
 
-def test_config3_full_size_sampled():
+def test_config3_full_size_every_token():
+    """Config 3 at full size, every one of the 16384 tokens against the oracle, row by row (the oracle runs in chunks of
+    2048 tokens to bound host memory)."""
     c = synth.config3()
     Y, name = run_matmul(c)
-    idx = np.array([0, 1, 127, 128, 4095, 8191, 8192, 12345, 16382, 16383])
-    ref = O.monarch_apply(c["L"].astype(np.float64), c["R"].astype(np.float64), c["X"][idx].astype(np.float64))
-    check(Y[idx], ref, TOL_BF16, "config3 full sampled " + name)
-    # property over every token: no row is garbage (norms agree with the sampled ratio)
-    ratio = np.linalg.norm(Y, axis=1) / np.linalg.norm(c["X"].astype(np.float64), axis=1)
-    assert np.isfinite(Y).all() and ratio.min() > 0.5 and ratio.max() < 2.0
+    assert name == "matmul_umma_64x64"
+    L64, R64 = c["L"].astype(np.float64), c["R"].astype(np.float64)
+    num = den = 0.0
+    for t0 in range(0, c["X"].shape[0], 2048):
+        ref = O.monarch_apply(L64, R64, c["X"][t0:t0 + 2048].astype(np.float64))
+        check(Y[t0:t0 + 2048], ref, TOL_BF16, f"config3 full, tokens {t0}..{t0 + 2047} " + name)
+        num += float(np.sum((Y[t0:t0 + 2048] - ref) ** 2))
+        den += float(np.sum(ref ** 2))
+    assert np.sqrt(num / den) <= TOL_BF16
 
 
 # ---- config 4: order-3 causal, N = 32768 ------------------------------------------------------------
@@ -196,21 +204,44 @@ def test_config4_small_full_rows(B, H):
 def test_config4_full_size_sampled():
     c = synth.config4()
     y, name = run_conv(c["dims"], c["x"], c["k"], True, M.M2_BF16)
-    assert np.isfinite(y).all()
-    rows = [(0, 0), (3, 1023), (1, 512), (2, 77), (0, 1022), (3, 1), (2, 1000), (1, 300)]
+    assert np.isfinite(y).all() and name == "conv_umma_o3_32k"
+    # The kernel walks row pairs p = h * 2 + b0 / 2 (rows b0, b0 + 1 of channel h), CTA c of 148 taking p = c, c + 148, ...:
+    # one row of every CTA's first pair and of its last pair, plus pairs spread over the whole range; the row within the
+    # pair alternates, so every batch index occurs and the channels span 0 .. 1023.
+    B4, H4, ctas = 4, 1024, 148
+    npairs = H4 * (B4 // 2)
+    first = list(range(ctas))
+    last = [cta + ctas * ((npairs - 1 - cta) // ctas) for cta in range(ctas)]
+    spread = list(range(7, npairs, 41))
+    rows = [(3, 1023), (0, 0)]   # rows[0] is also checked against the direct sum below
+    for i, p in enumerate(first + last + spread):
+        rows.append((2 * (p % 2) + (i % 2), p // 2))
+    rows = list(dict.fromkeys(rows))
+    assert len(rows) >= 300 and {b for b, _ in rows} == {0, 1, 2, 3}
     xs = np.stack([c["x"][b, h] for b, h in rows]).astype(np.float64)
     ks = np.stack([c["k"][h] for b, h in rows]).astype(np.float64)
     ref = O.monarch_conv(ks, xs, c["dims"], causal=True)
     got = np.stack([y[b, h] for b, h in rows])
     check(got, ref, TOL_BF16, "config4 full sampled " + name)
     # direct sum at sampled outputs of one row
-    b, h = rows[1]
     for t in (0, 1, 1024, 9999, 16383):
-        d = float(np.dot(ks[1][: t + 1], xs[1][t::-1]))
-        assert abs(got[1][t] - d) <= 4e-2 * max(abs(d), np.abs(ref[1]).mean())
+        d = float(np.dot(ks[0][: t + 1], xs[0][t::-1]))
+        assert abs(got[0][t] - d) <= 4e-2 * max(abs(d), np.abs(ref[0]).mean())
     # every row is sane: output energy within the range of the checked rows
     e = np.linalg.norm(y.reshape(-1, y.shape[-1]), axis=1)
     assert e.min() > 0.2 * np.median(e) and e.max() < 5 * np.median(e)
+
+
+@pytest.mark.parametrize("B,H,n,causal", [(2, 3, 32768, False), (1, 2, 8192, True)])
+def test_bf16_general_shape_kernel_on_long_rows(B, H, n, causal):
+    """(32, 32, 32) bf16 requests the order-3 tensor-core kernel does not cover (circular, or causal with n != 16384) run on the
+    general-shape kernel, which for rows this long keeps the row between its stages as bf16 pairs."""
+    x = synth.round_bf16(synth.normal(synth.stream_id(17, n), (B, H, n)))
+    k = synth.decay_kernel(17, H, n, 0.0005, 128.0)
+    y, name = run_conv((32, 32, 32), x, k, causal, M.M2_BF16)
+    assert name == "conv_generic_bf16io"
+    ref = O.monarch_conv(k.astype(np.float64)[None], x.astype(np.float64), (32, 32, 32), causal=causal)
+    check(y, ref, TOL_BF16, f"bf16 general-shape kernel n={n} causal={causal}")
 
 
 # ---- config 5: the M2 block -------------------------------------------------------------------------
@@ -270,12 +301,15 @@ def test_config5_full_size_sampled():
 
 # ---- gradient with respect to the input: the same kernels with the conjugated spectrum ---------------------
 
-@pytest.mark.parametrize("cfg,kernel", [("c1", None), ("c2", "conv_umma_o2_512"), ("c2causal", "conv_umma_o2_512"), ("c4", "conv_umma_o3_32k")])
+@pytest.mark.parametrize("cfg,kernel", [("c1", None), ("c2", "conv_umma_o2_512_rows"), ("c2causal", "conv_umma_o2_512_rows"), ("c2pairs", "conv_umma_o2_512_pairs"),
+                                         ("c4", "conv_umma_o3_32k")])
 def test_conv_input_gradient(cfg, kernel):
     if cfg == "c1":
         c, causal, dtype, tol = synth.config1(), True, M.M2_FP32, TOL_FP32
     elif cfg == "c2":
         c, causal, dtype, tol = synth.config2(B=8, H=12), False, M.M2_BF16, TOL_BF16
+    elif cfg == "c2pairs":
+        c, causal, dtype, tol = synth.config2(B=11, H=12), False, M.M2_BF16, TOL_BF16
     elif cfg == "c2causal":
         c = synth.config2(B=8, H=12)
         c = dict(c, x=c["x"][..., :256].copy(), k=c["k"][..., :256].copy())
@@ -689,6 +723,32 @@ def test_new_kernels_are_bit_identical_and_stay_in_bounds():
     d2 = M.m2_monarch_conv_bwd_kernel(plan, x, g, M.M2_CIRCULAR)
     torch.cuda.synchronize()
     assert plan.device_status() == 0 and plan.last_kernel() == "conv_wgrad_umma_o2_512" and torch.equal(d1, d2)
+    plan.close()
+
+
+def test_bounded_wait_runs_out_and_the_plan_recovers():
+    """A device-side wait that runs out: the row-pair kernel is launched in its self-test mode (no copy issued, a few polls per
+    wait), must come back by itself through its abort path with nothing in flight, report M2_ERR_TIMEOUT in the plan's status
+    word and leave y alone; the next ordinary calls on the same plan are correct and clean."""
+    c = synth.config2(B=19, H=40)     # more pipelines than one CTA holds, a ragged last batch group
+    plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)
+    kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+    x = dev(c["x"], torch.bfloat16)
+    y = torch.full_like(x, 7.0)
+    M.m2_selftest_bounded_wait(plan, x, kf, M.M2_CIRCULAR, y)
+    torch.cuda.synchronize()
+    assert plan.device_status() == M.M2_ERR_TIMEOUT
+    assert plan.device_status() == 0                      # reading the word resets it
+    assert bool((y == 7.0).all())                         # nothing was written
+    ref = O.monarch_conv(c["k"].astype(np.float64)[None], c["x"].astype(np.float64), c["dims"], causal=False)
+    for _ in range(2):                                    # the scheduler words were reset: two ordinary calls in a row
+        M.m2_monarch_conv_fwd(plan, x, kf, M.M2_CIRCULAR, y=y)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0 and plan.last_kernel() == "conv_umma_o2_512_pairs"
+        check(host(y), ref, TOL_BF16, "after the timed-out launch")
+    # up to 8 batch rows there is no row-pair kernel to test
+    lib, s = M.lib(), torch.cuda.current_stream().cuda_stream
+    assert lib.m2_selftest_bounded_wait(plan.handle, x.data_ptr(), kf.data_ptr(), y.data_ptr(), 8, 40, 512, M.M2_CIRCULAR, s) == M.M2_ERR_UNSUPPORTED
     plan.close()
 
 

@@ -531,3 +531,75 @@ def m2_block_forward(x, k, w_short, W_up, W_down, dims=(32, 16)):
     z = g * np.transpose(v, (0, 2, 1))
     h = gelu_erf(blockdiag_apply(W_up, z))
     return blockdiag_apply(W_down, h), z
+
+
+# ----------------------------------------------------------------------------
+# Learnable (causal) Monarch matrices from polynomial coefficients (App. D.5, block size sqrt N)
+# ----------------------------------------------------------------------------
+
+
+def blocky_monarch(Lt: np.ndarray, Rt: np.ndarray, sign: int = +1):
+    """Alg. BlockyMonarch: coefficient matrices -> the block-diagonal factors of M = P L P R P, N = b^2.
+
+    Lt: [N, b], column j holds the N coefficients of l_j(Z) = sum_a Lt[a, j] Z^a.
+    Rt: [N, b] = b stacked blocks Rt_c [b, b]; column j of block c holds the coefficients of
+        r~_{c,j}(Y) = sum_a Rt_c[a, j] Y^a.
+    Returns (L [b, b, b], R [b, b, b]) in this module's weight layout [block][out][in], complex.
+
+    Steps, in the algorithm's order: F_N is taken as the Monarch matrix of the corollary "DFT is M";
+    L' = P F_N Lt and block c of L is rows c b .. c b + b - 1 of L'; block c of R is F_b Rt_c.
+    Reading (the appendix prints two formulas for the blocks of L that cannot both hold): the one used in the
+    proof of the theorem on BlockyMonarch's return value, block i0 of L has entry [i1, j] = l_j(omega_N^{i1 b + i0});
+    only this one makes the corollary true (pinned: identity coefficients give monarch_dft_factors).
+    With it, M[i1 b + i0, j1 b + j0] = l_{j0}(w) r~_{j0,j1}(w^b), w = omega_N^{i1 b + i0}: column j of M is the basis
+    polynomial l_{j0}(Z) r~_{j0,j1}(Z^b) at the N-th roots of unity."""
+    N, b = Lt.shape
+    assert b * b == N and Rt.shape == (N, b)
+    FL, FR = monarch_dft_factors(b, b, sign)
+    L2 = monarch_apply(FL, FR, Lt.T.astype(np.complex128)).T      # F_N Lt, column by column, by the factored apply
+    L1 = apply_perm(b, N, L2.T).T                                 # P (F_N Lt): the rows permuted
+    L = L1.reshape(b, b, b).copy()                                # block c = rows c b .. c b + b - 1
+    Fb = dft_matrix(b, sign)
+    R = np.stack([Fb @ Rt[c * b:(c + 1) * b, :] for c in range(b)])
+    return L, R
+
+
+def causal_coefficient_masks(b: int):
+    """The zero patterns of the lemma on masking and basis degree (App. D.5): returns (mask_L [N, b], mask_R [N, b])
+    of zeros and ones, N = b^2.
+      Lt': only the top b x b block survives, and there only entries [i0, j] with i0 >= j  (l_j has minimum degree j
+           and degree < b);
+      Rt'_c[i0, j0] is zeroed where i0 < j0 (minimum degree j0) or where i0 >= floor(b/2) and j0 < floor(b/2)
+           (degree < floor(b/2) for the first half of the columns)."""
+    N = b * b
+    mL = np.zeros((N, b))
+    i0 = np.arange(b)[:, None]
+    j = np.arange(b)[None, :]
+    mL[:b, :] = (i0 >= j)
+    h = b // 2
+    blockR = ((i0 >= j) & ~((i0 >= h) & (j < h))).astype(np.float64)
+    mR = np.tile(blockR, (b, 1))
+    return mL, mR
+
+
+def blocky_monarch_conv(Lt: np.ndarray, Rt: np.ndarray, k: np.ndarray, u: np.ndarray, sign: int = +1,
+                        stages: dict | None = None) -> np.ndarray:
+    """Alg. BlockMonarchConv with the padding of the theorem on causal block Monarch convolution:
+    f = M^-1 ((M k') (.) (M u'))[0:n], k' = (k, 0), u' = (u, 0) of length N = b^2, M = P L P R P from
+    blocky_monarch(Lt, Rt).  k: [..., n], u: [..., n] (broadcast against each other), n <= N/2.
+    M^-1 is applied through the block inverses of L and R.  With the masked coefficient matrices
+    (causal_coefficient_masks, non-zero diagonals) the map u -> f is causal and f is real up to rounding; the complex
+    result is returned so that tests can check that."""
+    N, b = Lt.shape
+    n = u.shape[-1]
+    assert k.shape[-1] == n and 2 * n <= N
+    L, R = blocky_monarch(Lt, Rt, sign)
+    Linv, Rinv = monarch_inverse_factors(L, R)
+    kp = np.concatenate([k, np.zeros((*k.shape[:-1], N - n))], axis=-1).astype(np.complex128)
+    up = np.concatenate([u, np.zeros((*u.shape[:-1], N - n))], axis=-1).astype(np.complex128)
+    k_f = monarch_apply(L, R, kp)
+    u_f = monarch_apply(L, R, up)
+    f = monarch_inverse_apply(Linv, Rinv, k_f * u_f)
+    if stages is not None:
+        stages.update(L=L, R=R, Linv=Linv, Rinv=Rinv, k_f=k_f, u_f=u_f, f=f)
+    return f[..., :n]

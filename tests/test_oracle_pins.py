@@ -583,3 +583,141 @@ def test_table2_flop_convention():
         # printed with 3 significant digits (two entries differ in the last printed digit)
         assert abs(dense_model - float(dense)) <= 0.012 * float(dense) + 6e-4
         assert abs(m2_model - float(m2)) <= 0.012 * float(m2) + 6e-4
+
+
+# ---- learnable / causal Monarch from polynomial coefficients (App. D.5) -----------------------------------
+
+def _basis_coefficients(Lt, Rt):
+    """Coefficient vectors (length N, ascending powers) of the basis polynomials b_j(Z) = l_{j0}(Z) r~_{j0,j1}(Z^b) mod (Z^N - 1),
+    j = j1 b + j0, by explicit polynomial products -- no DFT, no Monarch factor anywhere."""
+    N, b = Lt.shape
+    Bc = np.zeros((N, N))
+    for j1 in range(b):
+        for j0 in range(b):
+            l = Lt[:, j0]
+            r = np.zeros(b * (b - 1) + 1)
+            r[::b] = Rt[j0 * b:(j0 + 1) * b, j1]          # r~(Z^b): coefficient a sits at power a b
+            prod = np.convolve(l, r)
+            col = np.zeros(N)
+            for d, c in enumerate(prod):
+                col[d % N] += c                            # reduction mod Z^N - 1
+            Bc[:, j1 * b + j0] = col
+    return Bc
+
+
+@pytest.mark.parametrize("b", [2, 3, 4, 6])
+def test_blocky_monarch_columns_are_the_basis_polynomials_on_the_roots_of_unity(b):
+    """Theorem on BlockyMonarch's return value: M[i, j1 b + j0] = l_{j0}(w_N^i) r~_{j0,j1}(w_N^{i b}), evaluated here by
+    Horner's rule on the raw coefficients."""
+    N = b * b
+    rng = np.random.default_rng(100 + b)
+    Lt, Rt = rng.standard_normal((N, b)), rng.standard_normal((N, b))
+    for sign in (+1, -1):
+        L, R = O.blocky_monarch(Lt, Rt, sign)
+        Md = O.monarch_dense(L, R)
+        w = np.exp(sign * 2j * np.pi / N)
+        for i in range(N):
+            z = w ** i
+            for j1 in range(b):
+                for j0 in range(b):
+                    want = np.polyval(Lt[::-1, j0], z) * np.polyval(Rt[j0 * b:(j0 + 1) * b, j1][::-1], z ** b)
+                    assert abs(Md[i, j1 * b + j0] - want) < 1e-9 * max(1.0, abs(want))
+        # the same statement through the coefficient matrix of the basis: M = F_N B
+        assert np.allclose(Md, O.dft_matrix(N, sign) @ _basis_coefficients(Lt, Rt), atol=1e-9)
+
+
+@pytest.mark.parametrize("b", [2, 4, 8, 16])
+def test_blocky_monarch_with_identity_coefficients_is_the_dft(b):
+    """Corollary "DFT is M": identity blocks in Rt, identity top block in Lt -> the factors of monarch_dft_factors."""
+    N = b * b
+    Lt = np.zeros((N, b))
+    Lt[:b] = np.eye(b)
+    Rt = np.tile(np.eye(b), (b, 1))
+    for sign in (+1, -1):
+        L, R = O.blocky_monarch(Lt, Rt, sign)
+        FL, FR = O.monarch_dft_factors(b, b, sign)
+        assert np.allclose(L, FL, atol=1e-12) and np.allclose(R, FR, atol=1e-12)
+        assert np.allclose(O.monarch_dense(L, R), O.dft_matrix(N, sign), atol=1e-10)
+
+
+def test_causal_masks_literal_b4():
+    mL, mR = O.causal_coefficient_masks(4)
+    assert mL.shape == (16, 4) and mR.shape == (16, 4)
+    assert (mL[:4] == np.array([[1, 0, 0, 0], [1, 1, 0, 0], [1, 1, 1, 0], [1, 1, 1, 1]])).all() and (mL[4:] == 0).all()
+    blk = np.array([[1, 0, 0, 0], [1, 1, 0, 0], [0, 0, 1, 0], [0, 0, 1, 1]])   # rows >= 2 of columns < 2 are cut (degree < 2)
+    for c in range(4):
+        assert (mR[4 * c:4 * c + 4] == blk).all()
+
+
+@pytest.mark.parametrize("b", [4, 5, 6])
+def test_masked_basis_has_the_degrees_the_lemma_states(b):
+    """Lemma on masking: basis polynomial j = j1 b + j0 of M has minimum degree j; for j < b floor(b/2) its degree is < N/2."""
+    N = b * b
+    rng = np.random.default_rng(7 + b)
+    mL, mR = O.causal_coefficient_masks(b)
+    Lt = (np.eye(N, b) + rng.standard_normal((N, b))) * mL
+    Rt = (np.tile(np.eye(b), (b, 1)) + rng.standard_normal((N, b))) * mR
+    Bc = _basis_coefficients(Lt, Rt)
+    for j in range(N):
+        nz = np.nonzero(np.abs(Bc[:, j]) > 1e-12)[0]
+        assert nz.min() == j
+        if j < b * (b // 2):
+            assert nz.max() <= N // 2 - 1
+
+
+@pytest.mark.parametrize("b,n", [(4, 8), (4, 5), (6, 18), (5, 12), (8, 32)])
+def test_blocky_monarch_conv_is_the_polynomial_product_in_the_basis(b, n):
+    """Alg. BlockMonarchConv against its plain definition (the theorem on the univariate convolution): with k(Z) = sum k_j b_j,
+    u(Z) = sum u_j b_j, f holds the coefficients of k(Z) u(Z) mod (Z^N - 1) in the basis (b_i) -- computed here with explicit
+    polynomial products and one dense solve."""
+    N = b * b
+    rng = np.random.default_rng(50 + b + n)
+    mL, mR = O.causal_coefficient_masks(b)
+    Lt = (np.eye(N, b) + 0.4 * rng.standard_normal((N, b))) * mL
+    Rt = (np.tile(np.eye(b), (b, 1)) + 0.4 * rng.standard_normal((N, b))) * mR
+    k, u = rng.standard_normal((3, n)), rng.standard_normal((2, 3, n))
+    f = O.blocky_monarch_conv(Lt, Rt, k, u)
+    assert np.abs(f.imag).max() < 1e-9
+    Bc = _basis_coefficients(Lt, Rt)
+    for bi in range(2):
+        for h in range(3):
+            kz, uz = Bc[:, :n] @ k[h], Bc[:, :n] @ u[bi, h]
+            prod = np.zeros(N)
+            for d, c in enumerate(np.convolve(kz, uz)):
+                prod[d % N] += c
+            want = np.linalg.solve(Bc, prod)[:n]
+            assert np.allclose(f[bi, h].real, want, atol=1e-8 * max(1.0, np.abs(want).max()))
+
+
+@pytest.mark.parametrize("b", [4, 6, 8])
+def test_masked_blocky_monarch_conv_is_causal_and_unmasked_is_not(b):
+    """Theorem on causal block Monarch convolution: with the masked coefficients, f[:t0] does not change when u[t0:] does."""
+    N = b * b
+    n = N // 2
+    rng = np.random.default_rng(9 + b)
+    mL, mR = O.causal_coefficient_masks(b)
+    Lt0, Rt0 = np.eye(N, b) + 0.3 * rng.standard_normal((N, b)), np.tile(np.eye(b), (b, 1)) + 0.3 * rng.standard_normal((N, b))
+    k, u = rng.standard_normal(n), rng.standard_normal(n)
+    f = O.blocky_monarch_conv(Lt0 * mL, Rt0 * mR, k, u)
+    for t0 in (1, 2, n // 2, n - 1):
+        u2 = u.copy()
+        u2[t0:] += rng.standard_normal(n - t0)
+        f2 = O.blocky_monarch_conv(Lt0 * mL, Rt0 * mR, k, u2)
+        assert np.abs(f2[:t0] - f[:t0]).max() < 1e-9 * max(1.0, np.abs(f).max())
+        assert np.abs(f2[t0:] - f[t0:]).max() > 1e-6
+    g = O.blocky_monarch_conv(Lt0, Rt0, k, u)
+    u2 = u.copy()
+    u2[-1] += 1.0
+    assert abs(O.blocky_monarch_conv(Lt0, Rt0, k, u2)[0] - g[0]) > 1e-6     # without the masks the future leaks
+
+
+def test_blocky_monarch_conv_with_dft_coefficients_is_the_causal_convolution():
+    b, n = 8, 32
+    N = b * b
+    Lt = np.zeros((N, b))
+    Lt[:b] = np.eye(b)
+    Rt = np.tile(np.eye(b), (b, 1))
+    rng = np.random.default_rng(3)
+    k, u = rng.standard_normal((2, n)), rng.standard_normal((3, 2, n))
+    f = O.blocky_monarch_conv(Lt, Rt, k, u)
+    assert np.allclose(f.real, O.direct_causal_conv(k[None], u), atol=1e-10) and np.abs(f.imag).max() < 1e-10

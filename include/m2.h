@@ -42,7 +42,8 @@ enum m2_status {
     M2_ERR_ALIGNMENT = 3,   /* a device pointer is not 16-byte aligned */
     M2_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed */
     M2_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (read via m2_last_device_status) */
-    M2_ERR_NO_DEVICE = 6    /* the plan was created host-only (device < 0) */
+    M2_ERR_NO_DEVICE = 6,   /* the plan was created host-only (device < 0) */
+    M2_ERR_SINGULAR = 7     /* a block of a learnable Monarch factor could not be inverted (read via m2_last_device_status) */
 };
 
 enum m2_dtype { M2_FP32 = 0, M2_BF16 = 1 };
@@ -286,6 +287,34 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
 int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
                             const void* W_up_dev, const void* W_down_dev, void* y_dev, int64_t B, int64_t T,
                             int64_t C, int32_t nblk, int32_t expand, void* stream);
+
+/* Learnable (causal) Monarch matrices from polynomial coefficients, block size b = sqrt(N) (App. D.5: Alg. BlockyMonarch; the
+ * lemma on masking and basis degrees; Alg. BlockMonarchConv; the theorem on causal block Monarch convolution).  `plan` is an
+ * order-2 plan with N1 = N2 = b, 2 <= b <= 64 (M2_ERR_UNSUPPORTED otherwise).
+ *
+ * m2_blocky_monarch: Lt_dev, Rt_dev are float32 [N][b] coefficient matrices: column j of Lt holds the coefficients of
+ *   l_j(Z) = sum_a Lt[a][j] Z^a; Rt is b stacked [b][b] blocks, column j of block c holds r~_{c,j}(Y) = sum_a Rt[c b + a][j] Y^a.
+ *   It writes the factor set of M = P L P R P into factors_dev (m2_blocky_factors_bytes(plan) bytes, caller-owned, 16-byte
+ *   aligned, opaque): L[k1][k2][n2] = l_{n2}(w_N^{k2 b + k1}), R[n2][k1][n1] = r~_{n2,n1}(w_b^{k1}) -- so that column
+ *   j1 b + j0 of M is the basis polynomial l_{j0}(Z) r~_{j0,j1}(Z^b) on the N-th roots of unity -- and the block inverses of
+ *   both (M^-1 = P R^-1 P L^-1 P).  Of the two formulas App. D.5 prints for the blocks of L this is the one used in the proof
+ *   that the DFT is such an M.  causal_mask != 0 applies the lemma's zero patterns while reading: of Lt only entries
+ *   [a][j] with j <= a < b survive; of every block of Rt entry [a][j] is dropped where a < j, or a >= b/2 and j < b/2; the
+ *   diagonals must be non-zero.  Evaluation and inversion run in fp64, the results are stored as complex fp32.  A block that
+ *   cannot be inverted sets M2_ERR_SINGULAR in the plan's status word (m2_last_device_status) and leaves zeros as its inverse.
+ *   Meant to run once per weight update.
+ * m2_blocky_kernel_spectrum: kf_dev[h] = M (k[h], 0) in plan order, complex fp32 [H][N] (k_dev float32 [H][n], n <= N).
+ * m2_blocky_monarch_conv_fwd: y = Re( M^-1 ( kf[h] (.) M (x, 0) ) )[0:n) per row; x_dev, y_dev [B][H][n] in the plan dtype,
+ *   2 n <= N.  With masked factors the map x -> y is causal (f[i] depends on x[0..i] only) and its imaginary part vanishes;
+ *   with the DFT's coefficients (identity blocks in Rt, identity on top of Lt) it is the causal convolution.  CUDA-core
+ *   kernels, fp32 arithmetic: a general M has no fast structure beyond its two block-diagonal factors. */
+int64_t m2_blocky_factors_bytes(const m2_plan* plan);
+int32_t m2_blocky_monarch(const m2_plan* plan, const float* Lt_dev, const float* Rt_dev, int32_t causal_mask, void* factors_dev,
+                          void* stream);
+int32_t m2_blocky_kernel_spectrum(const m2_plan* plan, const void* factors_dev, const float* k_dev, int64_t H, int64_t n,
+                                  void* kf_dev, void* stream);
+int32_t m2_blocky_monarch_conv_fwd(const m2_plan* plan, const void* factors_dev, const void* x_dev, const void* kf_dev,
+                                   void* y_dev, int64_t B, int64_t H, int64_t n, void* stream);
 
 /* Self-test of the device-side bounded waits (the paper has no counterpart; a test and diagnosis aid).  Every wait
  * inside the tensor-core kernels -- for a TMA copy, for a tensor-core commit -- gives up after a fixed number of

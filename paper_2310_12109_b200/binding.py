@@ -18,7 +18,7 @@ M2_FP32, M2_BF16 = 0, 1
 M2_CAUSAL, M2_CIRCULAR = 0, 1
 M2_STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 M2_TABLE_PERM, M2_TABLE_PERM_INV, M2_TABLE_DIGIT_REV, M2_TABLE_TW_EXP = 0, 1, 2, 16
-M2_OK, M2_ERR_INVALID_ARG, M2_ERR_UNSUPPORTED, M2_ERR_ALIGNMENT, M2_ERR_CUDA, M2_ERR_TIMEOUT, M2_ERR_NO_DEVICE = range(7)
+M2_OK, M2_ERR_INVALID_ARG, M2_ERR_UNSUPPORTED, M2_ERR_ALIGNMENT, M2_ERR_CUDA, M2_ERR_TIMEOUT, M2_ERR_NO_DEVICE, M2_ERR_SINGULAR = range(8)
 
 # every symbol include/m2.h declares: (name, restype, argtypes)
 _vp, _i32, _i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
@@ -50,6 +50,10 @@ SIGNATURES = {
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
     "m2_block_fwd_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
+    "m2_blocky_factors_bytes": (_i64, [_vp]),
+    "m2_blocky_monarch": (_i32, [_vp, _vp, _vp, _i32, _vp, _vp]),
+    "m2_blocky_kernel_spectrum": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp, _vp]),
+    "m2_blocky_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_selftest_bounded_wait": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_status_string": (ctypes.c_char_p, [_i32]),
     "m2_last_device_status": (_i32, [_vp, ctypes.POINTER(_i32)]),
@@ -417,4 +421,37 @@ def m2_block_fwd_static(plan: Plan, x: torch.Tensor, kf: torch.Tensor, w_short: 
     B, T, C = x.shape
     _check(lib().m2_block_fwd_static(plan.handle, _ptr(x), _ptr(kf), _ptr(w_short), _ptr(W_up), _ptr(W_down), _ptr(y),
                                      B, T, C, nblk, expand, _stream()), "m2_block_fwd_static")
+    return y
+
+
+def m2_blocky_monarch(plan: Plan, Lt: torch.Tensor, Rt: torch.Tensor, causal_mask: bool = True):
+    """Lt, Rt: float32 CUDA tensors [N, b] of polynomial coefficients.  Returns the opaque factor set (uint8 tensor)."""
+    b = plan.dims[0]
+    for t in (Lt, Rt):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (plan.N, b)
+    nbytes = int(lib().m2_blocky_factors_bytes(plan.handle))
+    if nbytes < 0:
+        raise M2Error(M2_ERR_UNSUPPORTED, "m2_blocky_factors_bytes")
+    fac = torch.empty(nbytes, dtype=torch.uint8, device=Lt.device)
+    _check(lib().m2_blocky_monarch(plan.handle, _ptr(Lt), _ptr(Rt), 1 if causal_mask else 0, _ptr(fac), _stream()), "m2_blocky_monarch")
+    return fac
+
+
+def m2_blocky_kernel_spectrum(plan: Plan, factors: torch.Tensor, k: torch.Tensor):
+    """k: float32 CUDA tensor [H, n].  Returns kf: float32 [H, N, 2] (complex, plan order)."""
+    assert k.is_cuda and k.dtype == torch.float32 and k.is_contiguous() and k.dim() == 2
+    H, n = k.shape
+    kf = torch.empty((H, plan.N, 2), dtype=torch.float32, device=k.device)
+    _check(lib().m2_blocky_kernel_spectrum(plan.handle, _ptr(factors), _ptr(k), H, n, _ptr(kf), _stream()), "m2_blocky_kernel_spectrum")
+    return kf
+
+
+def m2_blocky_monarch_conv_fwd(plan: Plan, factors: torch.Tensor, x: torch.Tensor, kf: torch.Tensor, y: torch.Tensor | None = None):
+    """x: [B, H, n] CUDA tensor of the plan dtype, 2 n <= N; returns y of the same shape."""
+    assert x.is_cuda and x.dtype == plan.torch_dtype and x.is_contiguous() and x.dim() == 3
+    B, H, n = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _check(lib().m2_blocky_monarch_conv_fwd(plan.handle, _ptr(factors), _ptr(x), _ptr(kf), _ptr(y), B, H, n, _stream()),
+           "m2_blocky_monarch_conv_fwd")
     return y

@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libm2.so")
 OBJ_DIR = os.path.join(HERE, "build")
-SOURCES = ["m2_api.cu", "generic_kernels.cu", "conv_umma.cu", "conv_umma3.cu", "matmul_umma.cu", "mlp_umma.cu", "cols_umma.cu"]
+SOURCES = ["m2_api.cu", "generic_kernels.cu", "conv_umma.cu", "conv_umma3.cu", "matmul_umma.cu", "mlp_umma.cu", "cols_umma.cu", "blocky_monarch.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

@@ -8,6 +8,7 @@
 #include <new>
 #include <vector>
 
+#include "blocky_monarch.h"
 #include "conv_umma.h"
 #include "generic_kernels.h"
 #include "cols_umma.h"
@@ -772,6 +773,47 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
     return M2_OK;
 }
 
+int64_t m2_blocky_factors_bytes(const m2_plan* plan) { return plan ? m2b::factors_bytes(plan) : -1; }
+
+int32_t m2_blocky_monarch(const m2_plan* plan, const float* Lt_dev, const float* Rt_dev, int32_t causal_mask, void* factors_dev,
+                          void* stream) {
+    if (!plan || !Lt_dev || !Rt_dev || !factors_dev) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (!m2b::covered(plan)) return M2_ERR_UNSUPPORTED;
+    if (!aligned16(factors_dev)) return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    return m2b::build(plan, Lt_dev, Rt_dev, causal_mask != 0, factors_dev, (cudaStream_t)stream);
+}
+
+int32_t m2_blocky_kernel_spectrum(const m2_plan* plan, const void* factors_dev, const float* k_dev, int64_t H, int64_t n,
+                                  void* kf_dev, void* stream) {
+    if (!plan || !factors_dev || H < 0 || n <= 0) return M2_ERR_INVALID_ARG;
+    if ((!k_dev || !kf_dev) && H > 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (!m2b::covered(plan)) return M2_ERR_UNSUPPORTED;
+    if (n > plan->N) return M2_ERR_INVALID_ARG;
+    if (!aligned16(factors_dev) || !aligned16(kf_dev)) return M2_ERR_ALIGNMENT;
+    if (H > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    return m2b::spectrum(plan, factors_dev, k_dev, H, n, kf_dev, (cudaStream_t)stream);
+}
+
+int32_t m2_blocky_monarch_conv_fwd(const m2_plan* plan, const void* factors_dev, const void* x_dev, const void* kf_dev,
+                                   void* y_dev, int64_t B, int64_t H, int64_t n, void* stream) {
+    if (!plan || !factors_dev || B < 0 || H < 0 || n <= 0) return M2_ERR_INVALID_ARG;
+    if ((!x_dev || !kf_dev || !y_dev) && B * H != 0) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (!m2b::covered(plan)) return M2_ERR_UNSUPPORTED;
+    if (2 * n > plan->N) return M2_ERR_INVALID_ARG;   // the theorem's padding: N >= 2 n
+    if (!aligned16(factors_dev) || !aligned16(x_dev) || !aligned16(kf_dev) || !aligned16(y_dev)) return M2_ERR_ALIGNMENT;
+    if (B * H > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    return m2b::conv_fwd(plan, factors_dev, x_dev, kf_dev, y_dev, B, H, n, (cudaStream_t)stream);
+}
+
 const char* m2_status_string(int32_t status) {
     switch (status) {
         case M2_OK: return "ok";
@@ -781,6 +823,7 @@ const char* m2_status_string(int32_t status) {
         case M2_ERR_CUDA: return "CUDA call failed";
         case M2_ERR_TIMEOUT: return "device-side wait timed out";
         case M2_ERR_NO_DEVICE: return "plan has no device";
+        case M2_ERR_SINGULAR: return "a block of a learnable Monarch factor is singular";
         default: return "unknown status";
     }
 }

@@ -601,6 +601,92 @@ def test_m2_bert_mixer_fwd(B, d, dims, dtype):
     plan.close()
 
 
+# ---- learnable (causal) Monarch from polynomial coefficients (App. D.5) --------------------------------------------------
+
+def _blocky_coefficients(b, seed, noise):
+    """Near-identity coefficient matrices (the DFT's plus noise), rounded to fp32: what a learnable layer starts from."""
+    N = b * b
+    Lt = np.zeros((N, b))
+    Lt[:b] = np.eye(b)
+    Rt = np.tile(np.eye(b), (b, 1))
+    Lt = Lt + noise * synth.normal(synth.stream_id(18, seed), (N, b)) / np.sqrt(b)
+    Rt = Rt + noise * synth.normal(synth.stream_id(18, seed + 1), (N, b)) / np.sqrt(b)
+    return Lt.astype(np.float32).astype(np.float64), Rt.astype(np.float32).astype(np.float64)
+
+
+@pytest.mark.parametrize("b,n,dtype,masked,noise", [(8, 32, M.M2_FP32, True, 0.3), (16, 128, M.M2_FP32, True, 0.3), (16, 100, M.M2_BF16, True, 0.3),
+                                                     (32, 512, M.M2_BF16, True, 0.2), (6, 11, M.M2_FP32, True, 0.3), (8, 30, M.M2_FP32, False, 0.3),
+                                                     (16, 128, M.M2_FP32, True, 0.0), (64, 2048, M.M2_BF16, True, 0.1)])
+def test_blocky_monarch_conv(b, n, dtype, masked, noise):
+    """Alg. BlockyMonarch + Alg. BlockMonarchConv on the device against the oracle: factors from coefficient matrices (with the
+    causal zero patterns applied on the device), kernel spectrum, convolution; the masked operator is causal on the device too."""
+    N = b * b
+    Bn, H = 3, 4
+    Lt, Rt = _blocky_coefficients(b, 10 * b, noise)
+    k = synth.decay_kernel(18, H, n, 2.0 / n, 4.0).astype(np.float64)
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    x = rnd(synth.normal(synth.stream_id(18, 3), (Bn, H, n)))
+    plan = M.Plan((b, b), dtype=dtype, device=0)
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    fac = M.m2_blocky_monarch(plan, dev(Lt.astype(np.float32)), dev(Rt.astype(np.float32)), causal_mask=masked)
+    kf = M.m2_blocky_kernel_spectrum(plan, fac, dev(k.astype(np.float32)))
+    y = M.m2_blocky_monarch_conv_fwd(plan, fac, dev(x.astype(np.float32), tdt), kf)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "blocky_monarch_conv"
+    mL, mR = O.causal_coefficient_masks(b) if masked else (1.0, 1.0)
+    st = {}
+    f = O.blocky_monarch_conv(Lt * mL, Rt * mR, k[None], x, stages=st)
+    if masked:
+        assert np.abs(f.imag).max() <= 1e-8 * np.abs(f.real).max()
+    tol = TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32
+    # factors and the kernel spectrum against the oracle's, as complex arrays
+    per = N * b
+    fv = fac.view(torch.float32).cpu().numpy().astype(np.float64).reshape(4, per, 2)
+    got = [(fv[i, :, 0] + 1j * fv[i, :, 1]).reshape(b, b, b) for i in range(4)]
+    # (the device inverts its fp32-rounded factors in fp64, the oracle the fp64 factors: the inverses differ by cond x 6e-8)
+    for name, g, want, ftol in zip(("L", "R", "Linv", "Rinv"), got, (st["L"], st["R"], st["Linv"], st["Rinv"]), (1e-6, 1e-6, 2e-5, 2e-5)):
+        assert np.linalg.norm(g - want) <= ftol * np.linalg.norm(want), name
+    kfg = host(kf)
+    kfg = kfg[..., 0] + 1j * kfg[..., 1]
+    want_kf = st["k_f"][0].reshape(H, b, b).transpose(0, 2, 1).reshape(H, N)      # natural [k2][k1] -> plan order [k1][k2]
+    assert np.linalg.norm(kfg - want_kf) <= 1e-5 * np.linalg.norm(want_kf)
+    check(host(y), f.real, tol, f"blocky Monarch conv b={b} n={n}")
+    if masked:     # causality on the device: changing x[t0:] leaves y[:t0] as it was, up to rounding
+        t0 = n // 3 + 1
+        x2 = x.copy()
+        x2[..., t0:] = rnd(synth.normal(synth.stream_id(18, 4), (Bn, H, n - t0)))
+        y2 = M.m2_blocky_monarch_conv_fwd(plan, fac, dev(x2.astype(np.float32), tdt), kf)
+        torch.cuda.synchronize()
+        d = (host(y2) - host(y))[..., :t0]
+        assert np.abs(d).max() <= tol * np.abs(host(y)).max()
+    if noise == 0.0:   # the DFT's coefficients: the plain causal convolution
+        check(host(y), O.direct_causal_conv(k[None], x), tol, "blocky Monarch with the DFT's coefficients")
+    plan.close()
+
+
+def test_blocky_monarch_singular_block_and_bad_arguments():
+    b = 8
+    N = b * b
+    plan = M.Plan((b, b), dtype=M.M2_FP32, device=0)
+    Lt, Rt = _blocky_coefficients(b, 5, 0.2)
+    Rt[3 * b:4 * b] = 0.0                                    # block 3 of R becomes the zero matrix
+    fac = M.m2_blocky_monarch(plan, dev(Lt.astype(np.float32)), dev(Rt.astype(np.float32)), causal_mask=True)
+    torch.cuda.synchronize()
+    assert plan.device_status() == M.M2_ERR_SINGULAR and plan.device_status() == 0
+    lib, s = M.lib(), torch.cuda.current_stream().cuda_stream
+    rect = M.Plan((8, 4), dtype=M.M2_FP32, device=0)
+    assert lib.m2_blocky_factors_bytes(rect.handle) == -1
+    x = torch.zeros((1, 1, 40), dtype=torch.float32, device="cuda")
+    kf = torch.zeros((1, N, 2), dtype=torch.float32, device="cuda")
+    assert lib.m2_blocky_monarch(rect.handle, x.data_ptr(), x.data_ptr(), 1, fac.data_ptr(), s) == M.M2_ERR_UNSUPPORTED
+    assert lib.m2_blocky_monarch_conv_fwd(plan.handle, fac.data_ptr(), x.data_ptr(), kf.data_ptr(), x.data_ptr(), 1, 1, 40, s) == M.M2_ERR_INVALID_ARG   # 2 n > N
+    assert lib.m2_blocky_monarch_conv_fwd(plan.handle, fac.data_ptr(), None, kf.data_ptr(), x.data_ptr(), 1, 1, 32, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_blocky_monarch_conv_fwd(plan.handle, fac.data_ptr(), None, None, None, 0, 1, 32, s) == M.M2_OK      # empty batch
+    torch.cuda.synchronize()
+    plan.close()
+    rect.close()
+
+
 # ---- edge cases, error paths, determinism -------------------------------------------------------------
 
 def test_empty_batches_and_error_codes():

@@ -456,6 +456,14 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         fence_barrier_init();
         prefetch_tensormap(&map_x);
         prefetch_tensormap(&map_y);
+        // Pull this pipeline's first input tiles towards L2 now, while the previous kernel on the stream is still finishing:
+        // a prefetch returns no data, and L2 is where that kernel's writes land, so the copies issued after the wait below
+        // see them whatever it wrote.
+        if (!selftest && u < units0) {
+            const int hh = u % H, bb = (u / H) * 2 * kRows;
+            tma_prefetch_4d(&map_x, 0, 0, hh, bb);
+            tma_prefetch_4d(&map_x, 0, 0, hh, bb + kRows);
+        }
     }
     // Programmatic dependent launch: the next kernel on the stream may start its CTAs as this grid's CTAs leave
     // their SMs; everything above the wait below touches only plan-owned constants and this CTA's own resources.
@@ -710,10 +718,19 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 tmem_ld_wait();
 #pragma unroll
                 for (int g = 0; g < 4; ++g) tmem_ld_fence8(v + 8 * g);
-                unsigned char* st = smem + P_G_A + c * 8192 + r * 1024 + (n2 & 7) * 2;
+                // Neighbouring lanes hold neighbouring n2: the even lane collects the pair (n2, n2 + 1) of row n1 = 2j, the odd lane
+                // the pair of row 2j + 1 -- one word exchange per two values -- so the staging stores are whole 32-bit words.
+                const int odd = n2 & 1;
+                unsigned char* st = smem + P_G_A + c * 8192 + r * 1024 + odd * 32 + ((n2 & 7) >> 1) * 4;
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    *reinterpret_cast<__nv_bfloat16*>(st + i * 32 + (((n2 >> 3) ^ ((i >> 2) & 1)) << 4)) = __float2bfloat16_rn(v[i]);
+                for (int j = 0; j < 16; ++j) {
+                    const uint32_t mine = pack_bf16(v[2 * j], v[2 * j + 1]);           // (row 2j, row 2j+1) of this lane's n2
+                    const uint32_t theirs = __shfl_xor_sync(0xffffffffu, mine, 1);
+                    // even lane: (own row 2j, partner row 2j); odd lane: (partner row 2j+1, own row 2j+1)
+                    const uint32_t w = odd ? __byte_perm(theirs, mine, 0x7632) : __byte_perm(mine, theirs, 0x5410);
+                    const int i = 2 * j + odd;
+                    *reinterpret_cast<uint32_t*>(st + (2 * j) * 32 + (((n2 >> 3) ^ ((i >> 2) & 1)) << 4)) = w;
+                }
             }
         }
         if (leader) *next_slot = un2;

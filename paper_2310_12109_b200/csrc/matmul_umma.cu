@@ -225,6 +225,202 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
 bool covered(const m2_plan* pl);
 int64_t workspace_bytes(const m2_plan* pl, int64_t T);
 
+// ---- the forward passes: 64 tokens x 16 blocks per CTA ------------------------------------------------------------------
+//
+// The cost of both passes is the number of memory requests for the pieces of x (pass 1) and of y (pass 2) that a CTA owning
+// g consecutive blocks touches: 2 g bytes of every 128-byte line.  With g = 16 a piece is a whole 32-byte sector -- half as
+// many requests as with g = 8 -- and the tile shrinks to 64 tokens so that the 16 operands still fill 128 KB:
+//
+//   UMMA         M = 64 (tokens), N = 64, K = 64 per block; row r of an accumulator lives in TMEM lane (r % 16) + 32 (r / 16),
+//                so the accumulators of blocks 8..15 sit at lane offset 16 in the columns of blocks 0..7: 16 accumulators in
+//                512 columns, and in the epilogue lanes 0..15 of a warp hold blocks 0..7 and lanes 16..31 blocks 8..15 of
+//                the same 16 tokens.
+//   weights      16 blocks of 8 KB do not fit beside the operands: they stream through a ring of kSlots buffers, one TMA
+//                tile per block (128-byte swizzle = the K-major operand image), re-filled as the UMMAs release them.
+//   workspace    z[64-token tile][k1][n2 / 8][t % 64][n2 % 8]: per (tile, k1) 8 KB that ARE the K-major operand of block k1
+//                in pass 2 without swizzle (core matrix = 8 tokens x 16 bytes; next K chunk 1 KB further).  The pass-1 CTA
+//                (tile, n2 group) writes 2 KB of each of them straight from registers; the pass-2 CTA (tile, k1 group)
+//                fetches its 16 operands as 128 contiguous KB.
+//   pass 1 in    one (token, 8 consecutive n1) per thread: 8 loads of 32 bytes, a 16 x 8 transpose in registers (PRMT; this
+//                is P), 16 stores of 16 bytes into the swizzled operands A_{n2}[t][n1].
+//   pass 2 out   y[t][k2][16 k1]: a thread's 8 accumulators of one k2 are 16 bytes, the lane 16 further holds the other half
+//                of the sector; stored from registers (the last P).
+constexpr int kTile2 = 64;                    // tokens per CTA
+constexpr int kGroup2 = 16;                   // blocks per CTA
+constexpr int kSlots = 11;                    // weight ring
+constexpr int kIssuers = 4;                   // UMMA-issuing threads
+constexpr int F_OFF_A = 0;                    // 16 operands [64 t][64] bf16                         131072
+constexpr int F_OFF_W = 131072;               // kSlots weight blocks [64][64] bf16, swizzled         90112
+constexpr int F_OFF_BAR = F_OFF_W + kSlots * 8192;   // full[kSlots], empty[kSlots], bar_mma, bar_in, tmem ptr
+constexpr int F_SMEM_BYTES = F_OFF_BAR + 256;
+static_assert(F_SMEM_BYTES <= 232448 && (2 * kSlots + 3) * 8 <= 256, "shared-memory budget of the forward passes");
+
+// PASS 1: in = x[T][64 n1][64 n2], weights R[n2][k1][n1], out = workspace z
+// PASS 2: in = workspace z, weights L[k1][k2][n2], out = y[T][64 k2][64 k1] (optionally sigma(K (.) y))
+template <int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant__ CUtensorMap map_w, __nv_bfloat16* __restrict__ out,
+                     long long T, int32_t* __restrict__ status, const __nv_bfloat16* __restrict__ Kmul, long long Hk, int relu) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t s_base = smem_u32(smem);
+    const uint32_t bar_full = s_base + F_OFF_BAR, bar_empty = bar_full + 8 * kSlots, bar_mma = bar_empty + 8 * kSlots;
+    const uint32_t bar_in = bar_mma + 8, s_tptr = bar_mma + 16;
+    // the 4 CTAs that share the lines of one token tile are neighbours in launch order: the other sectors of a line are
+    // fetched / written while the line is still in L2
+    const int grp = blockIdx.x;                              // which 16 consecutive blocks (n2 in pass 1, k1 in pass 2)
+    const long long tile = blockIdx.y, t0 = tile * kTile2;
+    if (tid == 0) {
+        for (int i = 0; i < 2 * kSlots + 2; ++i) mbar_init(bar_full + 8 * i, i == 2 * kSlots ? kIssuers : 1);   // bar_mma: one arrival per issuing thread
+        fence_barrier_init();
+        prefetch_tensormap(&map_w);
+    }
+    if (warp == 2) tmem_alloc(s_tptr, 512);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __syncthreads();   // barriers initialised before anyone arms them
+    // The weights are the caller's and were complete before this call: the first ring-full of blocks is requested at once.
+    auto load_block = [&](int b) {
+        const uint32_t slot = (uint32_t)(b % kSlots);
+        mbar_expect_tx(bar_full + 8 * slot, 8192);
+        tma_load_2d(s_base + F_OFF_W + slot * 8192, &map_w, 0, (grp * kGroup2 + b) * 64, bar_full + 8 * slot);
+    };
+    if (tid == 32)
+        for (int b = 0; b < kSlots; ++b) load_block(b);
+    if (PASS == 1 && tid == 64 && t0 < T) {   // pull this CTA's share of the tile's lines towards L2 while the previous kernel finishes
+        const long long rows = T - t0 < kTile2 ? T - t0 : kTile2;
+        const long long share = rows * 8192 / 4;   // the 4 sibling CTAs prefetch a quarter each
+        bulk_prefetch_l2(reinterpret_cast<const unsigned char*>(in) + t0 * 8192 + grp * share, (uint32_t)share);
+    }
+    // everything else (pass 1's z for pass 2, the producer of x, earlier readers of the buffers written here) is awaited now
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (PASS == 1) {
+        const int g = tid & 7, tt = tid >> 3;   // 8 consecutive n1 of one token
+        uint32_t w[8][8];                        // w[i][j]: n1 = 8 g + i, n2 = 16 grp + 2 j, 2 j + 1
+        const bool live = t0 + tt < T;
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(in) + (size_t)(t0 + tt) * 8192 + (size_t)(8 * g) * 128 + grp * 32;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {   // cached in L2 only: the rest of every line belongs to other SMs
+            if (live) {
+                asm volatile("ld.global.cg.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                             : "=r"(w[i][0]), "=r"(w[i][1]), "=r"(w[i][2]), "=r"(w[i][3]), "=r"(w[i][4]), "=r"(w[i][5]), "=r"(w[i][6]), "=r"(w[i][7])
+                             : "l"(src + i * 128));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w[i][j] = 0u;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint4 lo, hi;
+            lo.x = prmt(w[0][j], w[1][j], 0x5410); hi.x = prmt(w[0][j], w[1][j], 0x7632);
+            lo.y = prmt(w[2][j], w[3][j], 0x5410); hi.y = prmt(w[2][j], w[3][j], 0x7632);
+            lo.z = prmt(w[4][j], w[5][j], 0x5410); hi.z = prmt(w[4][j], w[5][j], 0x7632);
+            lo.w = prmt(w[6][j], w[7][j], 0x5410); hi.w = prmt(w[6][j], w[7][j], 0x7632);
+            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j) * 8192 + sw_off(tt, g)) = lo;
+            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j + 1) * 8192 + sw_off(tt, g)) = hi;
+        }
+    } else if (tid == 0) {
+        // the 16 operands of this (tile, k1 group): 128 contiguous KB of the workspace
+        mbar_expect_tx(bar_in, kGroup2 * 8192);
+        const unsigned char* zb = reinterpret_cast<const unsigned char*>(in) + ((size_t)tile * 64 + (size_t)grp * kGroup2) * 8192;
+        for (int b = 0; b < kGroup2; ++b) bulk_load(s_base + F_OFF_A + b * 8192, zb + (size_t)b * 8192, 8192, bar_in);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + F_OFF_BAR + (2 * kSlots + 2) * 8);
+    // UMMA issue.  One thread issues an instruction of this size every ~57 cycles while the tensor core can take one every ~32:
+    // four threads (lane 0 of warps 4..7, one per scheduler) issue the blocks b = i, i + 4, .. concurrently, each as soon as the
+    // block's weights have landed; a block's ring slot is released by a commit of the thread that used it.
+    if (lane == 0 && warp >= 4 && warp < 4 + kIssuers) {
+        constexpr uint32_t IDESC = instr_desc_bf16(64, 64, false, false);
+        bool ok_in = true;
+        if (PASS == 2) ok_in = mbar_wait(bar_in, 0);
+        tc_fence_after();
+#pragma unroll 1
+        for (int b = warp - 4; b < kGroup2 && ok_in; b += kIssuers) {
+            const uint32_t slot = (uint32_t)(b % kSlots);
+            ok_in = mbar_wait(bar_full + 8 * slot, (uint32_t)((b / kSlots) & 1));
+            if (!ok_in) break;
+            tc_fence_after();
+            const uint32_t d = tmem + ((uint32_t)(16 * (b >> 3)) << 16) + (uint32_t)(b & 7) * 64;
+            const uint64_t ad = PASS == 1 ? smem_desc_sw128(s_base + F_OFF_A + b * 8192, 16, 1024) : smem_desc(s_base + F_OFF_A + b * 8192, 1024, 128);
+            const uint64_t bd = smem_desc_sw128(s_base + F_OFF_W + slot * 8192, 16, 1024);
+            constexpr uint64_t a_step = PASS == 1 ? 2 : 128;   // per K step of 16: 32 bytes of a swizzled row, or two 1 KB chunks (in 16-byte units)
+#pragma unroll
+            for (int s = 0; s < 4; ++s) umma_f16(d, ad + s * a_step, bd + s * 2, IDESC, s > 0);
+            if (b + kSlots < kGroup2) umma_commit(bar_empty + 8 * slot);
+        }
+        umma_commit(bar_mma);   // (with nothing issued it completes at once; the missing input is reported here)
+        if (!ok_in) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    } else if (tid == 32) {   // the blocks that did not fit the ring at the start
+#pragma unroll 1
+        for (int b = kSlots; b < kGroup2; ++b) {
+            if (!mbar_wait(bar_empty + 8 * (b % kSlots), 0)) {
+                atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+                break;
+            }
+            load_block(b);
+        }
+    }
+    const bool ok = mbar_wait(bar_mma, 0);
+    tc_fence_after();
+    // epilogue: lane l of lane quarter q holds token 16 q + (l & 15) of block set l >> 4 (blocks 8 set .. 8 set + 7); the four warps
+    // of a quarter split the 64 output columns.  For every output index the 8 accumulators of a thread are 8 consecutive block
+    // indices: one 16-byte piece.
+    if (ok) {
+        const int q = warp & 3, c4 = warp >> 2, tt = 16 * q + (lane & 15), set = lane >> 4;
+        const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
+        const bool live = t0 + tt < T;
+        unsigned char* dst;
+        if (PASS == 1)   // z[tile][k1][octet 2 grp + set][tt][16 B]
+            dst = reinterpret_cast<unsigned char*>(out) + (size_t)tile * (64 * 8192) + (size_t)(2 * grp + set) * 1024 + tt * 16;
+        else             // y[t][k2][16 grp + 8 set ..]
+            dst = reinterpret_cast<unsigned char*>(out) + (size_t)(t0 + tt) * 8192 + (size_t)(16 * grp + 8 * set) * 2;
+#pragma unroll 1
+        for (int gk = 0; gk < 2; ++gk) {
+            const int o0 = 16 * c4 + 8 * gk;
+            float v[8][8];
+#pragma unroll
+            for (int bl = 0; bl < 8; ++bl) tmem_ld8(t_lane + bl * 64 + o0, v[bl]);
+            tmem_ld_wait();
+#pragma unroll
+            for (int bl = 0; bl < 8; ++bl) tmem_ld_fence8(v[bl]);
+            if (PASS == 2 && Kmul != nullptr && live) {
+                // y = sigma(K (.) M x) (first half of the M2 operator, Eq. 2): the 8 accumulators of one output index are 8
+                // consecutive k1 -> one 16-byte piece of the kernel row
+                const __nv_bfloat16* krow = Kmul + (size_t)((t0 + tt) % Hk) * 4096 + 16 * grp + 8 * set;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint4 kp = *reinterpret_cast<const uint4*>(krow + (o0 + kk) * 64);
+                    const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        float a = v[2 * p][kk] * __uint_as_float(kw[p] << 16);
+                        float b = v[2 * p + 1][kk] * __uint_as_float(kw[p] & 0xffff0000u);
+                        v[2 * p][kk] = relu ? fmaxf(a, 0.f) : a;
+                        v[2 * p + 1][kk] = relu ? fmaxf(b, 0.f) : b;
+                    }
+                }
+            }
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
+                                           pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
+                if (PASS == 1)   // whole tiles of the workspace are written (rows past T are zeros)
+                    *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 8192) = p;
+                else if (live)
+                    *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 128) = p;
+            }
+        }
+    }
+    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
 // ---- gradients with respect to the weight blocks ------------------------------------------------------------------
 //
 //   D_b[m][a] = sum_t Z_b[t][m] * V_b[t][a]        for the 64 blocks b, contraction over ALL tokens
@@ -431,10 +627,13 @@ cudaError_t prepare(const m2_plan* pl) {
     cudaError_t e = cudaFuncSetAttribute(monarch64_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(monarch64_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM_BYTES);
     return e;
 }
 
-int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
+// 128 tokens x 8 blocks per CTA (16-byte pieces): serves inputs that are only 16-byte aligned
+static int32_t matmul_g8(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
                int64_t Hk, int relu, cudaStream_t stream) {
     if (!covered(pl)) return M2_ERR_UNSUPPORTED;
     if (T == 0) return M2_OK;
@@ -460,6 +659,39 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     if (cudaLaunchKernelEx(&cfg, monarch64_pass_kernel<2>, (const __nv_bfloat16*)ws, (const __nv_bfloat16*)L, my,
                            (__nv_bfloat16*)nullptr, (long long)T, pl->d_status, (const __nv_bfloat16*)Kmul, (long long)(Hk > 0 ? Hk : 1),
                            relu) != cudaSuccess)
+        return M2_ERR_CUDA;
+    pl->last_kernel = "matmul_umma_64x64_g8";
+    pl->launches += 2;
+    return M2_OK;
+}
+
+int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
+               int64_t Hk, int relu, cudaStream_t stream) {
+    if (!covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (T == 0) return M2_OK;
+    // the 32-byte loads of pass 1 want x on a 32-byte boundary (torch allocations are; a view need not be)
+    if ((reinterpret_cast<uintptr_t>(X) & 31u) != 0) return matmul_g8(pl, X, L, R, Y, T, ws, Kmul, Hk, relu, stream);
+    // weight blocks as TMA tiles: [64 blocks x 64 rows][64] bf16, one box = one block, 128-byte swizzle
+    alignas(64) CUtensorMap mr, ml;
+    const cuuint64_t gdim[2] = {64, 64 * 64}, gstr[1] = {128};
+    const cuuint32_t box[2] = {64, 64};
+    if (!tma_host::encode_sw128_bf16(&mr, R, 2, gdim, gstr, box) || !tma_host::encode_sw128_bf16(&ml, L, 2, gdim, gstr, box))
+        return M2_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(64 / kGroup2, (unsigned)((T + kTile2 - 1) / kTile2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = F_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<1>, (const __nv_bfloat16*)X, mr, (__nv_bfloat16*)ws, (long long)T, pl->d_status,
+                           (const __nv_bfloat16*)nullptr, 1LL, 0) != cudaSuccess)
+        return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<2>, (const __nv_bfloat16*)ws, ml, (__nv_bfloat16*)Y, (long long)T, pl->d_status,
+                           (const __nv_bfloat16*)Kmul, (long long)(Hk > 0 ? Hk : 1), relu) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "matmul_umma_64x64";
     pl->launches += 2;

@@ -253,10 +253,17 @@ constexpr int F_OFF_A = 0;                    // 16 operands [64 t][64] bf16    
 constexpr int F_OFF_W = 131072;               // kSlots weight blocks [64][64] bf16, swizzled         90112
 constexpr int F_OFF_BAR = F_OFF_W + kSlots * 8192;   // full[kSlots], empty[kSlots], bar_mma, bar_in, tmem ptr
 constexpr int F_SMEM_BYTES = F_OFF_BAR + 256;
-static_assert(F_SMEM_BYTES <= 232448 && (2 * kSlots + 3) * 8 <= 256, "shared-memory budget of the forward passes");
+static_assert(F_SMEM_BYTES <= 232448 && (2 * kSlots + 4) * 8 + 24 <= 256, "shared-memory budget of the forward passes");
 
 // PASS 1: in = x[T][64 n1][64 n2], weights R[n2][k1][n1], out = workspace z
 // PASS 2: in = workspace z, weights L[k1][k2][n2], out = y[T][64 k2][64 k1] (optionally sigma(K (.) y))
+//
+// Persistent: CTA c of a grid that is a multiple of 4 walks the items c, c + grid, .. of (token tile, block group) pairs numbered
+// group-fastest, so its block group is c % 4 for good (the weights stay) and the 4 CTAs that share a tile's lines work on it at
+// the same time.  Of the 16 weight blocks, 5..10 own ring slots 5..10; blocks 0..4 and 11..15 take turns in slots 0..4: a tile
+// runs the blocks that are resident first (0..10 on even iterations, 15..5 on odd ones) and the other five as their slots are
+// re-filled -- 5 block loads per tile.  The phases of consecutive tiles overlap: the loads of tile i + 1 are in flight (in
+// registers in pass 1, as bulk copies into the operand buffer in pass 2) while the accumulators of tile i are drained.
 template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
 monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant__ CUtensorMap map_w, __nv_bfloat16* __restrict__ out,
@@ -265,39 +272,56 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
     const uint32_t bar_full = s_base + F_OFF_BAR, bar_empty = bar_full + 8 * kSlots, bar_mma = bar_empty + 8 * kSlots;
-    const uint32_t bar_in = bar_mma + 8, s_tptr = bar_mma + 16;
-    // the 4 CTAs that share the lines of one token tile are neighbours in launch order: the other sectors of a line are
-    // fetched / written while the line is still in L2
-    const int grp = blockIdx.x;                              // which 16 consecutive blocks (n2 in pass 1, k1 in pass 2)
-    const long long tile = blockIdx.y, t0 = tile * kTile2;
+    const uint32_t bar_in = bar_mma + 8, s_tptr = bar_mma + 16, bar_go = bar_mma + 48;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + F_OFF_BAR + (2 * kSlots + 2) * 8 + 8);
+    const int grp = blockIdx.x & 3;                                   // which 16 consecutive blocks (n2 in pass 1, k1 in pass 2)
+    const long long ntiles = (T + kTile2 - 1) / kTile2, nitems = 4 * ntiles;
+    long long item = blockIdx.x;
     if (tid == 0) {
-        for (int i = 0; i < 2 * kSlots + 2; ++i) mbar_init(bar_full + 8 * i, i == 2 * kSlots ? kIssuers : 1);   // bar_mma: one arrival per issuing thread
+        for (int i = 0; i < 2 * kSlots + 2; ++i) mbar_init(bar_full + 8 * i, i == 2 * kSlots ? kIssuers : 1);   // bar_mma: one arrival per issuer
+        *abort_flag = 0;
+        mbar_init(bar_go, 1);
         fence_barrier_init();
         prefetch_tensormap(&map_w);
     }
     if (warp == 2) tmem_alloc(s_tptr, 512);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __syncthreads();   // barriers initialised before anyone arms them
-    // The weights are the caller's and were complete before this call: the first ring-full of blocks is requested at once.
+    // weight block b -> ring slot b % kSlots (the weights are the caller's and were complete before this call)
     auto load_block = [&](int b) {
         const uint32_t slot = (uint32_t)(b % kSlots);
         mbar_expect_tx(bar_full + 8 * slot, 8192);
         tma_load_2d(s_base + F_OFF_W + slot * 8192, &map_w, 0, (grp * kGroup2 + b) * 64, bar_full + 8 * slot);
     };
+    volatile int* fills = abort_flag + 1;   // thread 32: fills requested so far for slots 0..4
     if (tid == 32)
-        for (int b = 0; b < kSlots; ++b) load_block(b);
-    if (PASS == 1 && tid == 64 && t0 < T) {   // pull this CTA's share of the tile's lines towards L2 while the previous kernel finishes
-        const long long rows = T - t0 < kTile2 ? T - t0 : kTile2;
-        const long long share = rows * 8192 / 4;   // the 4 sibling CTAs prefetch a quarter each
-        bulk_prefetch_l2(reinterpret_cast<const unsigned char*>(in) + t0 * 8192 + grp * share, (uint32_t)share);
+        for (int b = 0; b < kSlots; ++b) {
+            load_block(b);
+            if (b < 5) fills[b] = 1;
+        }
+    // this CTA's quarter of a tile's lines, pulled towards L2 as whole lines well before the 32-byte pieces are read
+    auto prefetch_item = [&](long long it) {
+        if (PASS == 1 && it < nitems) {
+            const long long t0p = (it >> 2) * kTile2;
+            const long long rows = T - t0p < kTile2 ? T - t0p : kTile2;
+            const long long share = rows * 8192 / 4;
+            bulk_prefetch_l2(reinterpret_cast<const unsigned char*>(in) + t0p * 8192 + grp * share, (uint32_t)share);
+        }
+    };
+    if (tid == 64) {
+        prefetch_item(item);
+        prefetch_item(item + gridDim.x);
     }
     // everything else (pass 1's z for pass 2, the producer of x, earlier readers of the buffers written here) is awaited now
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (PASS == 1) {
-        const int g = tid & 7, tt = tid >> 3;   // 8 consecutive n1 of one token
-        uint32_t w[8][8];                        // w[i][j]: n1 = 8 g + i, n2 = 16 grp + 2 j, 2 j + 1
-        const bool live = t0 + tt < T;
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(in) + (size_t)(t0 + tt) * 8192 + (size_t)(8 * g) * 128 + grp * 32;
+
+    // pass 1: one (token, 8 consecutive n1) per thread, 8 loads of 32 bytes
+    const int g = tid & 7, tt_in = tid >> 3;
+    uint32_t w[8][8];   // w[i][j]: n1 = 8 g + i, n2 = 16 grp + 2 j, 2 j + 1
+    auto load_x = [&](long long it) {
+        const long long t0l = (it >> 2) * kTile2;
+        const bool live = t0l + tt_in < T;
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(in) + (size_t)(t0l + tt_in) * 8192 + (size_t)(8 * g) * 128 + grp * 32;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {   // cached in L2 only: the rest of every line belongs to other SMs
             if (live) {
@@ -309,6 +333,9 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
                 for (int j = 0; j < 8; ++j) w[i][j] = 0u;
             }
         }
+    };
+    // the 16 x 8 transpose in registers (this is P) and the 16 stores into the swizzled operands A_{n2}[t][n1]
+    auto store_a = [&]() {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint4 lo, hi;
@@ -316,109 +343,175 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
             lo.y = prmt(w[2][j], w[3][j], 0x5410); hi.y = prmt(w[2][j], w[3][j], 0x7632);
             lo.z = prmt(w[4][j], w[5][j], 0x5410); hi.z = prmt(w[4][j], w[5][j], 0x7632);
             lo.w = prmt(w[6][j], w[7][j], 0x5410); hi.w = prmt(w[6][j], w[7][j], 0x7632);
-            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j) * 8192 + sw_off(tt, g)) = lo;
-            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j + 1) * 8192 + sw_off(tt, g)) = hi;
+            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j) * 8192 + sw_off(tt_in, g)) = lo;
+            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j + 1) * 8192 + sw_off(tt_in, g)) = hi;
         }
-    } else if (tid == 0) {
-        // the 16 operands of this (tile, k1 group): 128 contiguous KB of the workspace
+    };
+    // pass 2: the 16 operands of (tile, k1 group) are 128 contiguous KB of the workspace
+    auto load_z = [&](long long it) {
         mbar_expect_tx(bar_in, kGroup2 * 8192);
-        const unsigned char* zb = reinterpret_cast<const unsigned char*>(in) + ((size_t)tile * 64 + (size_t)grp * kGroup2) * 8192;
+        const unsigned char* zb = reinterpret_cast<const unsigned char*>(in) + ((size_t)(it >> 2) * 64 + (size_t)grp * kGroup2) * 8192;
         for (int b = 0; b < kGroup2; ++b) bulk_load(s_base + F_OFF_A + b * 8192, zb + (size_t)b * 8192, 8192, bar_in);
+    };
+    bool z_pending = false;
+    uint32_t z_par = 0;   // thread 0: parity of the operand copy in flight
+    if (item < nitems) {
+        if (PASS == 1) {
+            load_x(item);
+            store_a();
+        } else if (tid == 0) {
+            load_z(item);
+            z_pending = true;
+        }
     }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + F_OFF_BAR + (2 * kSlots + 2) * 8);
-    // UMMA issue.  One thread issues an instruction of this size every ~57 cycles while the tensor core can take one every ~32:
-    // four threads (lane 0 of warps 4..7, one per scheduler) issue the blocks b = i, i + 4, .. concurrently, each as soon as the
-    // block's weights have landed; a block's ring slot is released by a commit of the thread that used it.
-    if (lane == 0 && warp >= 4 && warp < 4 + kIssuers) {
-        constexpr uint32_t IDESC = instr_desc_bf16(64, 64, false, false);
-        bool ok_in = true;
-        if (PASS == 2) ok_in = mbar_wait(bar_in, 0);
+    const uint32_t tmem_slot = F_OFF_BAR + (2 * kSlots + 2) * 8;
+    uint32_t it_n = 0;   // iterations done: parities of bar_mma, bar_in and of the alternating ring slots
+    bool ok = true;
+#pragma unroll 1
+    for (; item < nitems; item += gridDim.x, ++it_n) {
+        const long long tile = item >> 2, t0 = tile * kTile2, next = item + gridDim.x;
+        // the operands of this tile are complete (pass 1) and the previous tile's accumulators have been read
+        fence_proxy_async();
+        tc_fence_before();
+        if (__syncthreads_or(*abort_flag)) break;   // a wait ran out somewhere: every thread leaves here, together
         tc_fence_after();
-#pragma unroll 1
-        for (int b = warp - 4; b < kGroup2 && ok_in; b += kIssuers) {
-            const uint32_t slot = (uint32_t)(b % kSlots);
-            ok_in = mbar_wait(bar_full + 8 * slot, (uint32_t)((b / kSlots) & 1));
-            if (!ok_in) break;
+        const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + tmem_slot);
+        const bool odd = (it_n & 1u) != 0;
+        // UMMA issue.  One thread issues an instruction of this size every ~57 cycles while the tensor core can take one every ~32:
+        // four threads (lane 0 of warps 4..7, one per scheduler) issue the positions p = i, i + 4, .. concurrently.  Position p
+        // runs block p on even iterations and 15 - p on odd ones: first the blocks whose weights are resident, then the five
+        // whose slots are re-filled meanwhile; a slot is released by a commit of the thread that used it.
+        if (lane == 0 && warp >= 4 && warp < 4 + kIssuers) {
+            constexpr uint32_t IDESC = instr_desc_bf16(64, 64, false, false);
+            bool ok_in = true;
+            if (PASS == 2) ok_in = mbar_wait(bar_in, it_n & 1u);
             tc_fence_after();
-            const uint32_t d = tmem + ((uint32_t)(16 * (b >> 3)) << 16) + (uint32_t)(b & 7) * 64;
-            const uint64_t ad = PASS == 1 ? smem_desc_sw128(s_base + F_OFF_A + b * 8192, 16, 1024) : smem_desc(s_base + F_OFF_A + b * 8192, 1024, 128);
-            const uint64_t bd = smem_desc_sw128(s_base + F_OFF_W + slot * 8192, 16, 1024);
-            constexpr uint64_t a_step = PASS == 1 ? 2 : 128;   // per K step of 16: 32 bytes of a swizzled row, or two 1 KB chunks (in 16-byte units)
-#pragma unroll
-            for (int s = 0; s < 4; ++s) umma_f16(d, ad + s * a_step, bd + s * 2, IDESC, s > 0);
-            if (b + kSlots < kGroup2) umma_commit(bar_empty + 8 * slot);
-        }
-        umma_commit(bar_mma);   // (with nothing issued it completes at once; the missing input is reported here)
-        if (!ok_in) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-    } else if (tid == 32) {   // the blocks that did not fit the ring at the start
 #pragma unroll 1
-        for (int b = kSlots; b < kGroup2; ++b) {
-            if (!mbar_wait(bar_empty + 8 * (b % kSlots), 0)) {
-                atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-                break;
+            for (int p = warp - 4; p < kGroup2 && ok_in; p += kIssuers) {
+                const int b = odd ? kGroup2 - 1 - p : p;
+                const uint32_t slot = (uint32_t)(b % kSlots);
+                // Slots 5..10 are filled once (waited for on the first iteration).  Slots 0..4 are filled once before the loop and once
+                // in every iteration: the first five positions use fill number it_n (there since the previous iteration), the last
+                // five fill number it_n + 1 (requested in this iteration).
+                if (p >= 5 && p < kSlots) {
+                    if (it_n == 0) ok_in = mbar_wait(bar_full + 8 * slot, 0);
+                } else {
+                    ok_in = mbar_wait(bar_full + 8 * slot, (p < 5 ? it_n : it_n + 1u) & 1u);
+                }
+                if (!ok_in) break;
+                tc_fence_after();
+                const uint32_t d = tmem + ((uint32_t)(16 * (b >> 3)) << 16) + (uint32_t)(b & 7) * 64;
+                const uint64_t ad = PASS == 1 ? smem_desc_sw128(s_base + F_OFF_A + b * 8192, 16, 1024) : smem_desc(s_base + F_OFF_A + b * 8192, 1024, 128);
+                const uint64_t bd = smem_desc_sw128(s_base + F_OFF_W + slot * 8192, 16, 1024);
+                constexpr uint64_t a_step = PASS == 1 ? 2 : 128;   // per K step of 16: 32 bytes of a swizzled row, or two 1 KB chunks (in 16-byte units)
+#pragma unroll
+                for (int s = 0; s < 4; ++s) umma_f16(d, ad + s * a_step, bd + s * 2, IDESC, s > 0);
+                if (p < 5) umma_commit(bar_empty + 8 * slot);   // the slot's other block may come in
             }
-            load_block(b);
-        }
-    }
-    const bool ok = mbar_wait(bar_mma, 0);
-    tc_fence_after();
-    // epilogue: lane l of lane quarter q holds token 16 q + (l & 15) of block set l >> 4 (blocks 8 set .. 8 set + 7); the four warps
-    // of a quarter split the 64 output columns.  For every output index the 8 accumulators of a thread are 8 consecutive block
-    // indices: one 16-byte piece.
-    if (ok) {
-        const int q = warp & 3, c4 = warp >> 2, tt = 16 * q + (lane & 15), set = lane >> 4;
-        const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
-        const bool live = t0 + tt < T;
-        unsigned char* dst;
-        if (PASS == 1)   // z[tile][k1][octet 2 grp + set][tt][16 B]
-            dst = reinterpret_cast<unsigned char*>(out) + (size_t)tile * (64 * 8192) + (size_t)(2 * grp + set) * 1024 + tt * 16;
-        else             // y[t][k2][16 grp + 8 set ..]
-            dst = reinterpret_cast<unsigned char*>(out) + (size_t)(t0 + tt) * 8192 + (size_t)(16 * grp + 8 * set) * 2;
+            umma_commit(bar_mma);   // (with nothing issued it completes at once; the missing input is reported here)
+            if (!ok_in) {
+                atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+                *abort_flag = 1;
+            }
+        } else if (tid == 32) {   // re-fill slots 0..4 with the blocks this tile runs last: 11..15 on even iterations, 4..0 on odd ones
 #pragma unroll 1
-        for (int gk = 0; gk < 2; ++gk) {
-            const int o0 = 16 * c4 + 8 * gk;
-            float v[8][8];
+            for (int p = kSlots; p < kGroup2; ++p) {
+                const int b = odd ? kGroup2 - 1 - p : p;
+                if (!mbar_wait(bar_empty + 8 * (b % kSlots), it_n & 1u)) {
+                    atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+                    *abort_flag = 1;
+                    break;
+                }
+                load_block(b);
+                ++fills[b % kSlots];
+            }
+            if (PASS == 1) mbar_arrive(bar_go);   // (also after a failed wait: nobody is left waiting for this)
+        } else if (tid == 64) {
+            prefetch_item(next + gridDim.x);
+        }
+        __syncwarp();   // the lanes that share a warp with an issuing or producing thread must not spin on a barrier while it works
+        // pass 1: the next tile's pieces are requested now and arrive while this tile's accumulators are computed and drained --
+        // but only once the five weight blocks this tile still needs have been requested: behind 64 K piece requests they would
+        // arrive thousands of cycles late, and the last UMMAs wait for them
+        if (PASS == 1 && next < nitems) {
+            if (tid != 32 && !mbar_wait(bar_go, it_n & 1u)) *abort_flag = 1;
+            load_x(next);
+        }
+        ok = mbar_wait(bar_mma, it_n & 1u);
+        tc_fence_after();
+        // pass 2: the operand buffer is free again: the next tile's operands come in while this tile is stored
+        if (PASS == 2 && tid == 0) {
+            z_pending = false;
+            if (ok && next < nitems) {
+                load_z(next);
+                z_pending = true;
+                z_par = (it_n + 1u) & 1u;
+            }
+        }
+        // epilogue: lane l of lane quarter q holds token 16 q + (l & 15) of block set l >> 4 (blocks 8 set .. 8 set + 7); the four warps
+        // of a quarter split the 64 output columns.  For every output index the 8 accumulators of a thread are 8 consecutive block
+        // indices: one 16-byte piece.
+        if (ok) {
+            const int q = warp & 3, c4 = warp >> 2, tt = 16 * q + (lane & 15), set = lane >> 4;
+            const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
+            const bool live = t0 + tt < T;
+            unsigned char* dst;
+            if (PASS == 1)   // z[tile][k1][octet 2 grp + set][tt][16 B]
+                dst = reinterpret_cast<unsigned char*>(out) + (size_t)tile * (64 * 8192) + (size_t)(2 * grp + set) * 1024 + tt * 16;
+            else             // y[t][k2][16 grp + 8 set ..]
+                dst = reinterpret_cast<unsigned char*>(out) + (size_t)(t0 + tt) * 8192 + (size_t)(16 * grp + 8 * set) * 2;
+#pragma unroll 1
+            for (int gk = 0; gk < 4; ++gk) {
+                const int o0 = 16 * c4 + 4 * gk;
+                float v[8][4];
 #pragma unroll
-            for (int bl = 0; bl < 8; ++bl) tmem_ld8(t_lane + bl * 64 + o0, v[bl]);
-            tmem_ld_wait();
+                for (int bl = 0; bl < 8; ++bl) tmem_ld4(t_lane + bl * 64 + o0, v[bl]);
+                tmem_ld_wait();
 #pragma unroll
-            for (int bl = 0; bl < 8; ++bl) tmem_ld_fence8(v[bl]);
-            if (PASS == 2 && Kmul != nullptr && live) {
-                // y = sigma(K (.) M x) (first half of the M2 operator, Eq. 2): the 8 accumulators of one output index are 8
-                // consecutive k1 -> one 16-byte piece of the kernel row
-                const __nv_bfloat16* krow = Kmul + (size_t)((t0 + tt) % Hk) * 4096 + 16 * grp + 8 * set;
+                for (int bl = 0; bl < 8; ++bl) tmem_ld_fence4(v[bl]);
+                if (PASS == 2 && Kmul != nullptr && live) {
+                    // y = sigma(K (.) M x) (first half of the M2 operator, Eq. 2): the 8 accumulators of one output index are 8
+                    // consecutive k1 -> one 16-byte piece of the kernel row
+                    const __nv_bfloat16* krow = Kmul + (size_t)((t0 + tt) % Hk) * 4096 + 16 * grp + 8 * set;
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint4 kp = *reinterpret_cast<const uint4*>(krow + (o0 + kk) * 64);
-                    const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint4 kp = *reinterpret_cast<const uint4*>(krow + (o0 + kk) * 64);
+                        const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
 #pragma unroll
-                    for (int p = 0; p < 4; ++p) {
-                        float a = v[2 * p][kk] * __uint_as_float(kw[p] << 16);
-                        float b = v[2 * p + 1][kk] * __uint_as_float(kw[p] & 0xffff0000u);
-                        v[2 * p][kk] = relu ? fmaxf(a, 0.f) : a;
-                        v[2 * p + 1][kk] = relu ? fmaxf(b, 0.f) : b;
+                        for (int pp = 0; pp < 4; ++pp) {
+                            float a = v[2 * pp][kk] * __uint_as_float(kw[pp] << 16);
+                            float bb = v[2 * pp + 1][kk] * __uint_as_float(kw[pp] & 0xffff0000u);
+                            v[2 * pp][kk] = relu ? fmaxf(a, 0.f) : a;
+                            v[2 * pp + 1][kk] = relu ? fmaxf(bb, 0.f) : bb;
+                        }
                     }
                 }
-            }
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint4 p = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
-                                           pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
-                if (PASS == 1)   // whole tiles of the workspace are written (rows past T are zeros)
-                    *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 8192) = p;
-                else if (live)
-                    *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 128) = p;
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint4 pk = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
+                                                pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
+                    if (PASS == 1)   // whole tiles of the workspace are written (rows past T are zeros)
+                        *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 8192) = pk;
+                    else if (live)
+                        *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 128) = pk;
+                }
             }
         }
+        if (!ok && tid == 0) {
+            atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+            *abort_flag = 1;
+        }
+        // pass 1: the operand buffer is free (this tile's UMMAs are complete): the next tile's operands go in
+        if (PASS == 1 && ok && next < nitems) store_a();
     }
-    if (!ok && tid == 0) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+    // teardown: nothing of ours may be in flight when the CTA goes away (only after a wait ran out can anything be left)
+    if (PASS == 2 && tid == 0 && z_pending) mbar_wait(bar_in, z_par);
+    if (tid == 32)
+        for (int sl = 0; sl < 5; ++sl)
+            if (fills[sl] > 0) mbar_wait(bar_full + 8 * sl, (uint32_t)(fills[sl] - 1) & 1u);
     tc_fence_before();
     __syncthreads();
-    if (warp == 2) tmem_dealloc(tmem, 512);
+    if (warp == 2) tmem_dealloc(*reinterpret_cast<volatile uint32_t*>(smem + tmem_slot), 512);
 }
 
 // ---- gradients with respect to the weight blocks ------------------------------------------------------------------
@@ -678,7 +771,12 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     if (!tma_host::encode_sw128_bf16(&mr, R, 2, gdim, gstr, box) || !tma_host::encode_sw128_bf16(&ml, L, 2, gdim, gstr, box))
         return M2_ERR_UNSUPPORTED;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(64 / kGroup2, (unsigned)((T + kTile2 - 1) / kTile2));
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long nitems = 4 * ((T + kTile2 - 1) / kTile2);
+    const long long ctas = (sms / 4) * 4 > 4 ? (sms / 4) * 4 : 4;   // a multiple of 4: a CTA keeps its block group
+    cfg.gridDim = dim3((unsigned)(nitems < ctas ? nitems : ctas));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = F_SMEM_BYTES;
     cfg.stream = stream;

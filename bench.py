@@ -224,7 +224,7 @@ def _side_hyena(torch, M, synth, peaks, reps, bf):
     plan = M.Plan((32, 16), dtype=M.M2_BF16, device=torch.cuda.current_device())
     W = [(torch.randn(d, d, device="cuda") / d ** 0.5).to(torch.bfloat16) for _ in range(4)]
     kfs = [M.m2_kernel_spectrum(plan, torch.randn(d, n, device="cuda") * 0.05) for _ in range(3)]
-    kfl = M.m2_kernel_spectrum(plan, (torch.randn(d // dh, n, device="cuda") * 0.05).repeat_interleave(dh * dh, dim=0).contiguous())
+    kfl = M.m2_kernel_spectrum(plan, torch.randn(d // dh, n, device="cuda") * 0.05)   # one long kernel per head
     u = torch.randn(B, n, d, device="cuda").to(torch.bfloat16)
     y = torch.empty_like(u)
     scratch = M.m2_hyena_scratch(plan, B, n, d, dh)

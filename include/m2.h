@@ -129,6 +129,13 @@ int32_t m2_monarch_conv_bwd_kernel(const m2_plan* plan, const void* x_dev, const
 int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
                             int64_t H, int64_t n, int32_t mode, void* stream);
 
+/* The same convolution with one kernel shared by kf_group consecutive channels: channel h is multiplied by row h / kf_group
+ * of the spectrum, which m2_kernel_spectrum computed for H / kf_group kernels (H must be a multiple of kf_group).  This is how
+ * the heads of the M2 Hyena layer (App. "GPT Causal Language Modeling") use one long kernel for the dh^2 sequences of a head's
+ * outer product without the spectrum being repeated dh^2 times. */
+int32_t m2_monarch_conv_fwd_grouped(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
+                                    int64_t H, int64_t n, int32_t mode, int64_t kf_group, void* stream);
+
 /* Same operation from host buffers: copies x_host -> x_dev (scratch the caller provides), runs the
  * convolution, copies y_dev -> y_host, all on `stream`; returns without synchronising.  x_host and
  * y_host should be pinned for the copies to be asynchronous. */
@@ -220,7 +227,7 @@ int32_t m2_bert_mixer_fwd(const m2_plan* plan, const void* x_dev, const void* co
  * plan: the convolution plan, N >= 2 n (the convolutions are m2_monarch_conv_fwd in M2_CAUSAL mode on channel-first rows).
  * W: HOST array of 4 device pointers {W_X1, W_X2, W_V, W_O}, each [d][d] stored outputs x inputs (y[o] = sum_i W[o][i] u[i]).
  * kf1_dev, kf2_dev, kf3_dev: m2_kernel_spectrum of the short kernels [d, n];  kf_long_dev: m2_kernel_spectrum of the long
- * kernel with one row per (head, i, j) channel, i.e. [d dh, n] with the head's kernel repeated dh^2 times.
+ * kernels, one row per head: [d / dh, n] (the dh^2 sequences of a head share its row: m2_monarch_conv_fwd_grouped).
  * y_dev: [B, n, d] (must not overlap u_dev).  scratch_dev: m2_hyena_scratch_bytes(plan, B, n, d, dh) bytes, caller-owned.
  * The projections are the single-block case of the column-layout Monarch kernel (tensor cores for d a multiple of 64 up
  * to 4096 and n a multiple of 8, bf16), so after one transposition everything runs channel-first. */

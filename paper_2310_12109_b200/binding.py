@@ -30,6 +30,7 @@ SIGNATURES = {
     "m2_kernel_spectrum": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp]),
     "m2_spectrum_to_natural": (_i32, [_vp, _vp, _i64, _vp, _vp]),
     "m2_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
+    "m2_monarch_conv_fwd_grouped": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i64, _vp]),
     "m2_monarch_conv_fwd_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_matmul_workspace_bytes": (_i64, [_vp, _i64]),
     "m2_spectrum_conjugate": (_i32, [_vp, _vp, _i64, _vp, _vp]),
@@ -202,6 +203,17 @@ def m2_monarch_conv_fwd(plan: Plan, x: torch.Tensor, kf: torch.Tensor, mode: int
     return y
 
 
+def m2_monarch_conv_fwd_grouped(plan: Plan, x: torch.Tensor, kf: torch.Tensor, mode: int, kf_group: int, y: torch.Tensor | None = None):
+    """Like m2_monarch_conv_fwd with channel h using spectrum row h // kf_group (kf computed for H // kf_group kernels)."""
+    assert x.is_cuda and x.dtype == plan.torch_dtype and x.is_contiguous() and x.dim() == 3
+    B, H, n = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _check(lib().m2_monarch_conv_fwd_grouped(plan.handle, _ptr(x), _ptr(kf), _ptr(y), B, H, n, mode, kf_group, _stream()),
+           "m2_monarch_conv_fwd_grouped")
+    return y
+
+
 def m2_selftest_bounded_wait(plan: Plan, x: torch.Tensor, kf: torch.Tensor, mode: int, y: torch.Tensor):
     """Launches the row-pair convolution kernel so that its first bounded wait runs out; y is left untouched and the
     plan's device status reads M2_ERR_TIMEOUT afterwards."""
@@ -334,8 +346,8 @@ def m2_hyena_scratch(plan: Plan, B: int, n: int, d: int, dh: int, device=None) -
 def m2_hyena_heads_fwd(plan: Plan, u: torch.Tensor, W, kf1, kf2, kf3, kf_long, dh: int, scratch: torch.Tensor | None = None,
                        y: torch.Tensor | None = None) -> torch.Tensor:
     """The M2 Hyena layer with heads on u [B, n, d]; W = (W_X1, W_X2, W_V, W_O), each [d, d] stored outputs x inputs;
-    kf1..kf3 = m2_kernel_spectrum of the short kernels [d, n]; kf_long = m2_kernel_spectrum of the long kernel repeated
-    to one row per (head, i, j) channel: K_long.repeat_interleave(dh * dh, dim=0)."""
+    kf1..kf3 = m2_kernel_spectrum of the short kernels [d, n]; kf_long = m2_kernel_spectrum of the long kernels
+    [d // dh, n], one row per head (its dh^2 outer-product sequences share it)."""
     B, n, d = u.shape
     assert len(W) == 4 and d % dh == 0
     for a in (u, *W):

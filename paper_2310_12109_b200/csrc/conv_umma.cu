@@ -101,7 +101,7 @@ __device__ __forceinline__ bool group_sync_or(int wg, bool pred, volatile int* f
 __global__ void __launch_bounds__(kThreads, 1)
 conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
-               int32_t* __restrict__ status, int* __restrict__ sched) {
+               int32_t* __restrict__ status, int* __restrict__ sched, int kf_group) {
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
@@ -147,7 +147,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
         tma_load_4d(s_base + G_X, &map_x, 0, 0, u % H, (u / H) * kRows, bar_x);
         x_pending = true;
         mbar_expect_tx(bar_k, 4096);
-        bulk_load(s_base + G_KF, kfu + (size_t)(u % H) * 256, 4096, bar_k);
+        bulk_load(s_base + G_KF, kfu + (size_t)((u % H) / kf_group) * 256, 4096, bar_k);
         k_pending = true;
     }
     fence_proxy_async();   // the constant matrices are read by the async proxy (UMMA)
@@ -305,7 +305,7 @@ conv512_kernel(const __grid_constant__ CUtensorMap map_x, __nv_bfloat16* __restr
             umma_commit(bar_mma);
             if (un < units) {                 // the spectrum tile is free: fetch the next unit's
                 mbar_expect_tx(bar_k, 4096);
-                bulk_load(s_base + G_KF, kfu + (size_t)(un % H) * 256, 4096, bar_k);
+                bulk_load(s_base + G_KF, kfu + (size_t)((un % H) / kf_group) * 256, 4096, bar_k);
                 k_pending = true;
             }
         }
@@ -428,7 +428,7 @@ static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols 
 __global__ void __launch_bounds__(kThreadsP, 1)
 conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
-               int32_t* __restrict__ status, int* __restrict__ sched, int selftest) {
+               int32_t* __restrict__ status, int* __restrict__ sched, int selftest, int kf_group) {
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
@@ -601,7 +601,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
         float4 kw[8];   // this thread's 16 spectrum values (k1 fixed), requested before the accumulator is waited for
 #pragma unroll
-        for (int q = 0; q < 8; ++q) kw[q] = __ldg(kfu_k1 + (size_t)h * 256 + q * 32);
+        for (int q = 0; q < 8; ++q) kw[q] = __ldg(kfu_k1 + (size_t)(h / kf_group) * 256 + q * 32);
         ok = mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
@@ -1122,7 +1122,7 @@ static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_
 }
 
 static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
-                             cudaStream_t stream, int selftest) {
+                             cudaStream_t stream, int selftest, int kf_group) {
     if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
     // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
@@ -1136,7 +1136,8 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
     const int groups = pairs ? kGroupsP : kGroups;
     const long long ctas = (units + groups - 1) / groups;
     const int grid = (int)(ctas < sms ? ctas : sms);
-    const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)H * 512 * 8);
+    // the kernels' own spectrum layout follows the plan-order copy of the H / kf_group spectrum rows
+    const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf) + (size_t)(H / kf_group) * 512 * 8);
     // launched with programmatic stream serialization: its CTAs may take over SMs that the previous kernel's CTAs
     // have left while that kernel's last CTAs still run (the kernel waits for it before touching its data)
     cudaLaunchConfig_t cfg = {};
@@ -1155,13 +1156,13 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
         alignas(64) CUtensorMap mx32;   // the row-pair kernel reads whole 32-byte rows of 16 n2
         if (!make_map_rows32(&mx32, x, B, H, n)) return M2_ERR_UNSUPPORTED;
         if (cudaLaunchKernelEx(&cfg, conv512p_kernel, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H, (int)n,
-                               pl->d_status, t->d_sched, selftest) != cudaSuccess)
+                               pl->d_status, t->d_sched, selftest, kf_group) != cudaSuccess)
             return M2_ERR_CUDA;
     } else {
         alignas(64) CUtensorMap mx;
         if (!make_map_rows32(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
         if (cudaLaunchKernelEx(&cfg, conv512_kernel, mx, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const, (int)B, (int)H, (int)n, pl->d_status,
-                               t->d_sched) != cudaSuccess)
+                               t->d_sched, kf_group) != cudaSuccess)
             return M2_ERR_CUDA;
     }
     pl->last_kernel = pairs ? "conv_umma_o2_512_pairs" : "conv_umma_o2_512_rows";
@@ -1170,13 +1171,13 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
 }
 
 int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
-                 cudaStream_t stream) {
-    return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 0);
+                 cudaStream_t stream, int kf_group) {
+    return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 0, kf_group);
 }
 
 int32_t conv_fwd_wait_selftest(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
                                cudaStream_t stream) {
-    return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 1);
+    return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 1, 1);
 }
 
 // dk[h] = Re M^-1 ( sum_p partial[p][h][:] ) [0:n) / 512 for N = 512 = 32 x 16: the parts added in index order, then the two

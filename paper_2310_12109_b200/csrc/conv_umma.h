@@ -12,8 +12,9 @@ void destroy_tables(m2_plan* plan);
 
 // Returns M2_ERR_UNSUPPORTED when no tensor-core kernel covers the request (caller falls back to
 // the CUDA-core kernels), M2_OK after enqueueing, another status on failure.
+// kf_group: channel h is multiplied by spectrum row h / kf_group (the buffer then holds H / kf_group rows).
 int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
-                 int32_t mode, cudaStream_t stream);
+                 int32_t mode, cudaStream_t stream, int kf_group = 1);
 // The row-pair kernel launched so that every pipeline's first bounded wait runs out with nothing in flight (no copy is
 // issued, a few polls per wait): the kernel leaves through its abort path, sets M2_ERR_TIMEOUT in the plan's status
 // word, writes nothing to y.  Needs B > 8 (the row-pair kernel); M2_ERR_UNSUPPORTED otherwise.

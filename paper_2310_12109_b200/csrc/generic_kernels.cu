@@ -145,7 +145,7 @@ struct Roots {
 template <typename IO, typename ST, int ITEMS>
 __global__ void __launch_bounds__(1024) conv_row_kernel(const IO* __restrict__ x, const float2* __restrict__ kf, IO* __restrict__ y, Dims D,
                                 Roots R, int H, int n, long long row_stride_b, long long row_stride_h,
-                                long long elem_stride, const float* __restrict__ gate_w) {
+                                long long elem_stride, const float* __restrict__ gate_w, int kf_group) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     ST* buf = reinterpret_cast<ST*>(smem_raw);
     const int row = blockIdx.x;
@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(1024) conv_row_kernel(const IO* __restrict__ x
     }
     __syncthreads();
     for (int a = 0; a < D.p; ++a) stage<ST, ITEMS, false>(buf, D, a, R.r[a]);
-    const float2* kr = kf + (long long)h * D.N;
+    const float2* kr = kf + (long long)(h / kf_group) * D.N;
     for (int i = threadIdx.x; i < D.N; i += blockDim.x) Store<ST>::st(buf + i, cmul(Store<ST>::ld(buf + i), kr[i]));
     __syncthreads();
     for (int a = D.p - 1; a >= 0; --a) stage<ST, ITEMS, true>(buf, D, a, R.r[a]);
@@ -404,7 +404,8 @@ static cudaError_t launch_conv_t(const ConvShape& s, const void* x, const void* 
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);        \
         if (e != cudaSuccess) return e;                                                                            \
         kern<<<(unsigned)rows, threads, smem, st>>>((const IO*)x, (const float2*)kf, (IO*)y, D, R, (int)s.H,       \
-                                                    (int)s.n, s.stride_b, s.stride_h, s.stride_e, gate_w);         \
+                                                    (int)s.n, s.stride_b, s.stride_h, s.stride_e, gate_w,          \
+                                                    s.kf_group > 0 ? s.kf_group : 1);                              \
     }
     switch (items) {
         case 1: M2_LAUNCH_CONV(1) break;

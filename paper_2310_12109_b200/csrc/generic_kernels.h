@@ -12,6 +12,7 @@ struct ConvShape {
     // element (b, h, i) of x / y lives at b*stride_b + h*stride_h + i*stride_e
     long long stride_b, stride_h, stride_e;
     const float2* roots[3];  // device: omega_{Na}^j per stage
+    int kf_group = 1;        // channel h is multiplied by spectrum row h / kf_group
 };
 
 cudaError_t launch_conv(const ConvShape& s, bool bf16_io, const void* x, const void* kf, void* y, const float* gate_w,

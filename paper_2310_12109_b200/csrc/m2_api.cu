@@ -297,25 +297,38 @@ int32_t m2_spectrum_conjugate(const m2_plan* plan, const void* kf_in_dev, int64_
     return M2_OK;
 }
 
-int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
-                            int64_t H, int64_t n, int32_t mode, void* stream) {
+// y = conv(k[h / kf_group], x[b][h]); arguments beyond kf_group checked here
+static int32_t conv_fwd_grouped(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B, int64_t H, int64_t n,
+                                int32_t mode, int64_t kf_group, void* stream) {
     int32_t st = check_conv_args(plan, x_dev, kf_dev, y_dev, B, H, n, mode);
     if (st != M2_OK) return st;
+    if (kf_group < 1 || kf_group > 0x7fffffffLL || H % kf_group != 0) return M2_ERR_INVALID_ARG;
     DeviceGuard g(plan->device);
     if (!g.ok) return M2_ERR_CUDA;
     if (B * H == 0) return M2_OK;
     // tensor-core path where a kernel exists for the shape, CUDA-core path otherwise
-    int32_t ust = m2u::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
-    if (ust == M2_ERR_UNSUPPORTED) ust = m2u3::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
+    int32_t ust = m2u::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream, (int)kf_group);
+    if (ust == M2_ERR_UNSUPPORTED && kf_group == 1) ust = m2u3::conv_fwd(plan, x_dev, kf_dev, y_dev, B, H, n, mode, (cudaStream_t)stream);
     if (ust == M2_OK) return M2_OK;
     if (ust != M2_ERR_UNSUPPORTED) return ust;
     m2g::ConvShape s = conv_shape(plan, B, H, n);
+    s.kf_group = (int)kf_group;
     cudaError_t e = m2g::launch_conv(s, plan->dtype == M2_BF16, x_dev, kf_dev, y_dev, nullptr, (cudaStream_t)stream);
     if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
     if (e != cudaSuccess) return M2_ERR_CUDA;
     plan->last_kernel = plan->dtype == M2_BF16 ? "conv_generic_bf16io" : "conv_generic_fp32";
     plan->launches += 1;
     return M2_OK;
+}
+
+int32_t m2_monarch_conv_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
+                            int64_t H, int64_t n, int32_t mode, void* stream) {
+    return conv_fwd_grouped(plan, x_dev, kf_dev, y_dev, B, H, n, mode, 1, stream);
+}
+
+int32_t m2_monarch_conv_fwd_grouped(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B, int64_t H,
+                                    int64_t n, int32_t mode, int64_t kf_group, void* stream) {
+    return conv_fwd_grouped(plan, x_dev, kf_dev, y_dev, B, H, n, mode, kf_group, stream);
 }
 
 int32_t m2_selftest_bounded_wait(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B, int64_t H, int64_t n,
@@ -593,7 +606,7 @@ int32_t m2_hyena_heads_fwd(const m2_plan* plan, const void* u_dev, const void* c
     if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, P3, kf3_dev, C3, B, d, n, M2_CAUSAL, stream);
     if (rc != M2_OK) return rc;
     if (m2g::launch_heads_outer(C2, C3, XV, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    rc = m2_monarch_conv_fwd(plan, XV, kf_long_dev, XVc, B, d * dh, n, M2_CAUSAL, stream);
+    rc = conv_fwd_grouped(plan, XV, kf_long_dev, XVc, B, d * dh, n, M2_CAUSAL, dh * dh, stream);   // dh^2 channels share a head's kernel
     if (rc != M2_OK) return rc;
     if (m2g::launch_heads_reduce(C1, XVc, P1, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
     rc = dense(W[3], P1, P2);

@@ -130,6 +130,32 @@ def test_config2_full_size():
         check(y[b, h][None], d[None], TOL_BF16 / 2, f"config2 row ({b},{h}) direct")
 
 
+@pytest.mark.parametrize("B,dims,n,causal,dtype,group", [(19, (32, 16), 512, False, M.M2_BF16, 4), (5, (32, 16), 256, True, M.M2_BF16, 3),
+                                                          (3, (8, 4, 2), 30, True, M.M2_FP32, 2), (2, (32, 16), 100, True, M.M2_BF16, 6)])
+def test_conv_with_a_kernel_shared_by_channel_groups(B, dims, n, causal, dtype, group):
+    """m2_monarch_conv_fwd_grouped: channel h uses spectrum row h // group (both N = 512 tensor-core kernels and the
+    general-shape kernel); same result as the plain call with the kernels repeated."""
+    Hk = 5
+    H = Hk * group
+    rnd = (lambda a: synth.round_bf16(a)) if dtype == M.M2_BF16 else (lambda a: a.astype(np.float32).astype(np.float64))
+    x = rnd(synth.normal(synth.stream_id(19, n), (B, H, n)))
+    k = synth.decay_kernel(19, Hk, n, 0.01, 8.0)
+    plan = M.Plan(dims, dtype=dtype, device=0)
+    tdt = torch.bfloat16 if dtype == M.M2_BF16 else torch.float32
+    kf = M.m2_kernel_spectrum(plan, dev(k))
+    y = M.m2_monarch_conv_fwd_grouped(plan, dev(x.astype(np.float32), tdt), kf, M.M2_CAUSAL if causal else M.M2_CIRCULAR, group)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    krep = np.repeat(k.astype(np.float64), group, axis=0)
+    ref = O.direct_causal_conv(krep[None], x) if causal else O.direct_circular_conv(krep[None], x)
+    check(host(y), ref, TOL_BF16 if dtype == M.M2_BF16 else TOL_FP32, "grouped conv " + plan.last_kernel())
+    lib, s = M.lib(), torch.cuda.current_stream().cuda_stream
+    xd = dev(x.astype(np.float32), tdt)
+    assert lib.m2_monarch_conv_fwd_grouped(plan.handle, xd.data_ptr(), kf.data_ptr(), y.data_ptr(), B, H, n, M.M2_CAUSAL if causal else M.M2_CIRCULAR, 0, s) == M.M2_ERR_INVALID_ARG
+    assert lib.m2_monarch_conv_fwd_grouped(plan.handle, xd.data_ptr(), kf.data_ptr(), y.data_ptr(), B, H, n, M.M2_CAUSAL if causal else M.M2_CIRCULAR, H + 1, s) == M.M2_ERR_INVALID_ARG
+    plan.close()
+
+
 @pytest.mark.parametrize("B", [5, 19])
 def test_bf16_causal_order2_and_ragged(B):
     for n in (256, 100, 48):
@@ -553,7 +579,7 @@ def test_m2_hyena_heads_fwd(B, n, d, dh, dims, dtype):
     plan = M.Plan(dims, dtype=dtype, device=0)
     f32 = lambda a: torch.from_numpy(a.astype(np.float32)).cuda()   # noqa: E731
     kfs = [M.m2_kernel_spectrum(plan, f32(p[k])) for k in ("K1", "K2", "K3")]
-    kfl = M.m2_kernel_spectrum(plan, f32(np.repeat(p["K_long"], dh * dh, axis=0)))
+    kfl = M.m2_kernel_spectrum(plan, f32(p["K_long"]))       # one row per head; its dh^2 sequences share it
     dv = lambda a: dev(a.astype(np.float32), tdt)   # noqa: E731
     W = [dv(np.ascontiguousarray(p[k].T)) for k in ("W_x1", "W_x2", "W_v", "W_o")]   # stored outputs x inputs
     y = M.m2_hyena_heads_fwd(plan, dv(u), W, kfs[0], kfs[1], kfs[2], kfl, dh)

@@ -150,7 +150,9 @@ int32_t m2_monarch_conv_fwd_host(const m2_plan* plan, const void* x_host, const 
  * R is applied first.  (The listing's parameter called L is applied first and so plays R's role.)
  * ws_dev: caller-owned device workspace of at least m2_matmul_workspace_bytes(plan, T) bytes for the
  * intermediate between the two factors (16-byte aligned); with ws_dev == NULL or ws_bytes too small the
- * call uses the slower kernels that need none. */
+ * call uses the slower kernels that need none.  bf16 plans with 64 x 64 blocks run on the tensor cores; their fastest
+ * kernels read X in 32-byte pieces and want X_dev on a 32-byte boundary (any fresh allocation is; a view at an odd
+ * 16-byte offset falls back to kernels with 16-byte pieces, same results). */
 int64_t m2_matmul_workspace_bytes(const m2_plan* plan, int64_t T);
 int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev,
                           void* Y_dev, int64_t T, void* ws_dev, int64_t ws_bytes, void* stream);

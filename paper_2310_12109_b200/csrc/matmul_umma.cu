@@ -225,293 +225,293 @@ monarch64_pass_kernel(const __nv_bfloat16* __restrict__ in, const __nv_bfloat16*
 bool covered(const m2_plan* pl);
 int64_t workspace_bytes(const m2_plan* pl, int64_t T);
 
-// ---- the forward passes: 64 tokens x 16 blocks per CTA ------------------------------------------------------------------
+// ---- the forward passes: 32 tokens x 16 blocks per item ------------------------------------------------------------------
 //
 // The cost of both passes is the number of memory requests for the pieces of x (pass 1) and of y (pass 2) that a CTA owning
-// g consecutive blocks touches: 2 g bytes of every 128-byte line.  With g = 16 a piece is a whole 32-byte sector -- half as
-// many requests as with g = 8 -- and the tile shrinks to 64 tokens so that the 16 operands still fill 128 KB:
+// g consecutive blocks touches: 2 g bytes of every 128-byte line.  With g = 16 a piece is a whole 32-byte sector.  An SM takes
+// such requests at a fixed rate (and a warp that issues them is blocked while they queue), so everything else a tile needs
+// runs underneath them, in other warps:
 //
-//   UMMA         M = 64 (tokens), N = 64, K = 64 per block; row r of an accumulator lives in TMEM lane (r % 16) + 32 (r / 16),
-//                so the accumulators of blocks 8..15 sit at lane offset 16 in the columns of blocks 0..7: 16 accumulators in
-//                512 columns, and in the epilogue lanes 0..15 of a warp hold blocks 0..7 and lanes 16..31 blocks 8..15 of
-//                the same 16 tokens.
-//   weights      16 blocks of 8 KB do not fit beside the operands: they stream through a ring of kSlots buffers, one TMA
-//                tile per block (128-byte swizzle = the K-major operand image), re-filled as the UMMAs release them.
-//   workspace    z[64-token tile][k1][n2 / 8][t % 64][n2 % 8]: per (tile, k1) 8 KB that ARE the K-major operand of block k1
-//                in pass 2 without swizzle (core matrix = 8 tokens x 16 bytes; next K chunk 1 KB further).  The pass-1 CTA
-//                (tile, n2 group) writes 2 KB of each of them straight from registers; the pass-2 CTA (tile, k1 group)
-//                fetches its 16 operands as 128 contiguous KB.
-//   pass 1 in    one (token, 8 consecutive n1) per thread: 8 loads of 32 bytes, a 16 x 8 transpose in registers (PRMT; this
-//                is P), 16 stores of 16 bytes into the swizzled operands A_{n2}[t][n1].
-//   pass 2 out   y[t][k2][16 k1]: a thread's 8 accumulators of one k2 are 16 bytes, the lane 16 further holds the other half
-//                of the sector; stored from registers (the last P).
-constexpr int kTile2 = 64;                    // tokens per CTA
+//   UMMA         the WEIGHT block is the A operand (M = 64 output indices, K = 64) and the tile's data the B operand (N = 32
+//                tokens): D_b[out][t].  Row r of an M = 64 accumulator lives in TMEM lane (r % 16) + 32 (r / 16), so blocks
+//                8..15 sit at lane offset 16 in the columns of blocks 0..7: a tile's 16 accumulators take 256 columns, and
+//                the 512 columns hold TWO tiles -- the UMMAs of tile i run while the accumulators of tile i - 1 are drained.
+//   weights      all 16 blocks of the CTA's group stay in shared memory (128 KB, one TMA tile per block, 128-byte swizzle =
+//                the K-major operand image); the 16 operands of a 32-token tile take the other 64 KB.
+//   roles        warps 0..7 load (global -> registers -> operand buffer), warps 8..15 drain (TMEM -> registers -> global),
+//                lane 0 of warps 16 and 17 issues 8 blocks each (32 UMMAs, ~60 cycles of the thread's time per instruction,
+//                about what the tensor core needs for them).  They meet only through mbarriers.
+//   workspace    z[32-token tile][n2 / 16][t % 32][k1][n2 % 16]: 32-byte pieces with k1 running fastest.  In pass 1 lane l of a
+//                draining warp holds output index k1 = 16 q + l % 16 of blocks 8 (l / 16) .. + 7, i.e. 16 bytes of a piece, and a
+//                warp store is 512 contiguous bytes; in pass 2 the CTA (tile, k1 group) reads, for every (n2 / 16, t), 16 pieces
+//                = 512 contiguous bytes, and a piece is 32 bytes of row t of the K-major operand of its block as it lies.
+//   pass 1 in    one (token, 8 consecutive n1) per loading thread: 8 loads of 32 bytes, a 16 x 8 transpose in registers (PRMT;
+//                this is P), 16 stores of 16 bytes into the swizzled operands B_{n2}[t][n1].
+//   pass 2 out   y[t][k2][16 k1]: a thread's 8 accumulators of one token are 16 bytes, the lane 16 further holds the other half
+//                of the sector.  Each draining warp stages [4 tokens][its 16 k2][32 B] in shared memory (the 32-byte-swizzled
+//                image of a TMA box: no bank conflicts) and lane 0 sends it off with one tensor store (the last P): the 2048
+//                sectors a tile scatters over 2048 lines never pass through the load/store unit, whose request rate is
+//                what the loads need; rows past T are clipped by the tensor map.
+constexpr int kTok = 32;                      // tokens per item
 constexpr int kGroup2 = 16;                   // blocks per CTA
-constexpr int kSlots = 11;                    // weight ring
-constexpr int kIssuers = 4;                   // UMMA-issuing threads
-constexpr int F_OFF_A = 0;                    // 16 operands [64 t][64] bf16                         131072
-constexpr int F_OFF_W = 131072;               // kSlots weight blocks [64][64] bf16, swizzled         90112
-constexpr int F_OFF_BAR = F_OFF_W + kSlots * 8192;   // full[kSlots], empty[kSlots], bar_mma, bar_in, tmem ptr
-constexpr int F_SMEM_BYTES = F_OFF_BAR + 256;
-static_assert(F_SMEM_BYTES <= 232448 && (2 * kSlots + 4) * 8 + 24 <= 256, "shared-memory budget of the forward passes");
+constexpr int F_OFF_A = 0;                    // 16 operands [32 t][64] bf16, swizzled rows of 128 bytes      65536
+constexpr int F_OFF_W = 65536;                // 16 weight blocks [64][64] bf16, swizzled                     131072
+constexpr int kLoadWarps = 8, kDrainWarps = 8, kIssueWarps = 2;
+constexpr int F_OFF_ST = F_OFF_W + kGroup2 * 8192;    // pass 2: per draining warp two staging buffers [4 t][16 k2][32 B]  32768
+constexpr int F_OFF_BAR = F_OFF_ST + kDrainWarps * 4096;   // bar_w, bar_mma[2], tmem ptr, abort flag, bar_opnd, bar_tfree[2]
+constexpr int F_SMEM_BYTES = F_OFF_BAR + 64;
+constexpr int kFwdThreads = 32 * (kLoadWarps + kDrainWarps + kIssueWarps);
+constexpr size_t kTileBytes = (size_t)kTok * 8192;    // a tile of x, z or y
+static_assert(F_SMEM_BYTES <= 232448, "shared-memory budget of the forward passes");
 
 // PASS 1: in = x[T][64 n1][64 n2], weights R[n2][k1][n1], out = workspace z
 // PASS 2: in = workspace z, weights L[k1][k2][n2], out = y[T][64 k2][64 k1] (optionally sigma(K (.) y))
 //
 // Persistent: CTA c of a grid that is a multiple of 4 walks the items c, c + grid, .. of (token tile, block group) pairs numbered
 // group-fastest, so its block group is c % 4 for good (the weights stay) and the 4 CTAs that share a tile's lines work on it at
-// the same time.  Of the 16 weight blocks, 5..10 own ring slots 5..10; blocks 0..4 and 11..15 take turns in slots 0..4: a tile
-// runs the blocks that are resident first (0..10 on even iterations, 15..5 on odd ones) and the other five as their slots are
-// re-filled -- 5 block loads per tile.  The phases of consecutive tiles overlap: the loads of tile i + 1 are in flight (in
-// registers in pass 1, as bulk copies into the operand buffer in pass 2) while the accumulators of tile i are drained.
+// the same time.  Tile i of a CTA uses accumulator set i % 2:
+//   loading warps   wait for the UMMAs of tile i - 1 (operand buffer free), write tile i's operands from their registers, arrive on
+//                   bar_opnd, request tile i + 1;
+//   issuing threads wait for bar_opnd (operands of tile i) and bar_tfree[i % 2] (set drained of tile i - 2), issue, commit to
+//                   bar_mma[i % 2];
+//   draining warps  wait for bar_mma[i % 2], move the set to global memory, arrive on bar_tfree[i % 2].
 template <int PASS>
-__global__ void __launch_bounds__(kThreads, 1)
-monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant__ CUtensorMap map_w, __nv_bfloat16* __restrict__ out,
-                     long long T, int32_t* __restrict__ status, const __nv_bfloat16* __restrict__ Kmul, long long Hk, int relu) {
+__global__ void __launch_bounds__(kFwdThreads, 1)
+monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant__ CUtensorMap map_w,
+                     const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ out, long long T, int32_t* __restrict__ status, const __nv_bfloat16* __restrict__ Kmul, long long Hk, int relu) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
-    const uint32_t bar_full = s_base + F_OFF_BAR, bar_empty = bar_full + 8 * kSlots, bar_mma = bar_empty + 8 * kSlots;
-    const uint32_t bar_in = bar_mma + 8, s_tptr = bar_mma + 16, bar_go = bar_mma + 48;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + F_OFF_BAR + (2 * kSlots + 2) * 8 + 8);
+    const uint32_t bar_w = s_base + F_OFF_BAR, bar_mma = bar_w + 8, s_tptr = bar_w + 24, bar_opnd = bar_w + 40, bar_tfree = bar_w + 48;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + F_OFF_BAR + 32);
     const int grp = blockIdx.x & 3;                                   // which 16 consecutive blocks (n2 in pass 1, k1 in pass 2)
-    const long long ntiles = (T + kTile2 - 1) / kTile2, nitems = 4 * ntiles;
+    const long long ntiles = (T + kTok - 1) / kTok, nitems = 4 * ntiles;
     long long item = blockIdx.x;
     if (tid == 0) {
-        for (int i = 0; i < 2 * kSlots + 2; ++i) mbar_init(bar_full + 8 * i, i == 2 * kSlots ? kIssuers : 1);   // bar_mma: one arrival per issuer
+        mbar_init(bar_w, 1);
+        mbar_init(bar_mma, kIssueWarps);       // one arrival per issuing thread
+        mbar_init(bar_mma + 8, kIssueWarps);
+        mbar_init(bar_opnd, kLoadWarps);       // one arrival per loading warp
+        mbar_init(bar_tfree, kDrainWarps);     // one arrival per draining warp
+        mbar_init(bar_tfree + 8, kDrainWarps);
         *abort_flag = 0;
-        mbar_init(bar_go, 1);
         fence_barrier_init();
         prefetch_tensormap(&map_w);
+        if (PASS == 2) prefetch_tensormap(&map_y);
     }
     if (warp == 2) tmem_alloc(s_tptr, 512);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __syncthreads();   // barriers initialised before anyone arms them
-    // weight block b -> ring slot b % kSlots (the weights are the caller's and were complete before this call)
-    auto load_block = [&](int b) {
-        const uint32_t slot = (uint32_t)(b % kSlots);
-        mbar_expect_tx(bar_full + 8 * slot, 8192);
-        tma_load_2d(s_base + F_OFF_W + slot * 8192, &map_w, 0, (grp * kGroup2 + b) * 64, bar_full + 8 * slot);
-    };
-    volatile int* fills = abort_flag + 1;   // thread 32: fills requested so far for slots 0..4
-    if (tid == 32)
-        for (int b = 0; b < kSlots; ++b) {
-            load_block(b);
-            if (b < 5) fills[b] = 1;
-        }
-    // this CTA's quarter of a tile's lines, pulled towards L2 as whole lines well before the 32-byte pieces are read
+    // the weights are the caller's and were complete before this call
+    if (tid == 32) {
+        mbar_expect_tx(bar_w, kGroup2 * 8192);
+        for (int b = 0; b < kGroup2; ++b) tma_load_2d(s_base + F_OFF_W + b * 8192, &map_w, 0, (grp * kGroup2 + b) * 64, bar_w);
+    }
+    // this CTA's quarter of a tile's lines, pulled towards L2 as whole lines well before the pieces are read (the four CTAs that
+    // share a tile ask for a quarter each).  L2 is where the previous kernel's writes land, so nothing stale can be fetched.
     auto prefetch_item = [&](long long it) {
-        if (PASS == 1 && it < nitems) {
-            const long long t0p = (it >> 2) * kTile2;
-            const long long rows = T - t0p < kTile2 ? T - t0p : kTile2;
+        if (it < nitems) {
+            const long long t0p = (it >> 2) * kTok;
+            const long long rows = PASS == 2 || T - t0p >= kTok ? kTok : T - t0p;   // (whole tiles of the workspace exist)
             const long long share = rows * 8192 / 4;
             bulk_prefetch_l2(reinterpret_cast<const unsigned char*>(in) + t0p * 8192 + grp * share, (uint32_t)share);
         }
     };
-    if (tid == 64) {
+    if (tid == 33) {
         prefetch_item(item);
         prefetch_item(item + gridDim.x);
     }
     // everything else (pass 1's z for pass 2, the producer of x, earlier readers of the buffers written here) is awaited now
     asm volatile("griddepcontrol.wait;" ::: "memory");
-
-    // pass 1: one (token, 8 consecutive n1) per thread, 8 loads of 32 bytes
-    const int g = tid & 7, tt_in = tid >> 3;
-    uint32_t w[8][8];   // w[i][j]: n1 = 8 g + i, n2 = 16 grp + 2 j, 2 j + 1
-    auto load_x = [&](long long it) {
-        const long long t0l = (it >> 2) * kTile2;
-        const bool live = t0l + tt_in < T;
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(in) + (size_t)(t0l + tt_in) * 8192 + (size_t)(8 * g) * 128 + grp * 32;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {   // cached in L2 only: the rest of every line belongs to other SMs
-            if (live) {
-                asm volatile("ld.global.cg.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                             : "=r"(w[i][0]), "=r"(w[i][1]), "=r"(w[i][2]), "=r"(w[i][3]), "=r"(w[i][4]), "=r"(w[i][5]), "=r"(w[i][6]), "=r"(w[i][7])
-                             : "l"(src + i * 128));
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) w[i][j] = 0u;
-            }
-        }
-    };
-    // the 16 x 8 transpose in registers (this is P) and the 16 stores into the swizzled operands A_{n2}[t][n1]
-    auto store_a = [&]() {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint4 lo, hi;
-            lo.x = prmt(w[0][j], w[1][j], 0x5410); hi.x = prmt(w[0][j], w[1][j], 0x7632);
-            lo.y = prmt(w[2][j], w[3][j], 0x5410); hi.y = prmt(w[2][j], w[3][j], 0x7632);
-            lo.z = prmt(w[4][j], w[5][j], 0x5410); hi.z = prmt(w[4][j], w[5][j], 0x7632);
-            lo.w = prmt(w[6][j], w[7][j], 0x5410); hi.w = prmt(w[6][j], w[7][j], 0x7632);
-            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j) * 8192 + sw_off(tt_in, g)) = lo;
-            *reinterpret_cast<uint4*>(smem + F_OFF_A + (2 * j + 1) * 8192 + sw_off(tt_in, g)) = hi;
-        }
-    };
-    // pass 2: the 16 operands of (tile, k1 group) are 128 contiguous KB of the workspace
-    auto load_z = [&](long long it) {
-        mbar_expect_tx(bar_in, kGroup2 * 8192);
-        const unsigned char* zb = reinterpret_cast<const unsigned char*>(in) + ((size_t)(it >> 2) * 64 + (size_t)grp * kGroup2) * 8192;
-        for (int b = 0; b < kGroup2; ++b) bulk_load(s_base + F_OFF_A + b * 8192, zb + (size_t)b * 8192, 8192, bar_in);
-    };
-    bool z_pending = false;
-    uint32_t z_par = 0;   // thread 0: parity of the operand copy in flight
-    if (item < nitems) {
-        if (PASS == 1) {
-            load_x(item);
-            store_a();
-        } else if (tid == 0) {
-            load_z(item);
-            z_pending = true;
-        }
-    }
-    const uint32_t tmem_slot = F_OFF_BAR + (2 * kSlots + 2) * 8;
-    uint32_t it_n = 0;   // iterations done: parities of bar_mma, bar_in and of the alternating ring slots
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + F_OFF_BAR + 24);
+    uint32_t it_n = 0;        // tiles begun: tile it_n of this CTA uses accumulator set it_n % 2 and phase it_n / 2 of that set's barriers
     bool ok = true;
-#pragma unroll 1
-    for (; item < nitems; item += gridDim.x, ++it_n) {
-        const long long tile = item >> 2, t0 = tile * kTile2, next = item + gridDim.x;
-        // the operands of this tile are complete (pass 1) and the previous tile's accumulators have been read
-        fence_proxy_async();
-        tc_fence_before();
-        if (__syncthreads_or(*abort_flag)) break;   // a wait ran out somewhere: every thread leaves here, together
-        tc_fence_after();
-        const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem + tmem_slot);
-        const bool odd = (it_n & 1u) != 0;
-        // UMMA issue.  One thread issues an instruction of this size every ~57 cycles while the tensor core can take one every ~32:
-        // four threads (lane 0 of warps 4..7, one per scheduler) issue the positions p = i, i + 4, .. concurrently.  Position p
-        // runs block p on even iterations and 15 - p on odd ones: first the blocks whose weights are resident, then the five
-        // whose slots are re-filled meanwhile; a slot is released by a commit of the thread that used it.
-        if (lane == 0 && warp >= 4 && warp < 4 + kIssuers) {
-            constexpr uint32_t IDESC = instr_desc_bf16(64, 64, false, false);
-            bool ok_in = true;
-            if (PASS == 2) ok_in = mbar_wait(bar_in, it_n & 1u);
-            tc_fence_after();
-#pragma unroll 1
-            for (int p = warp - 4; p < kGroup2 && ok_in; p += kIssuers) {
-                const int b = odd ? kGroup2 - 1 - p : p;
-                const uint32_t slot = (uint32_t)(b % kSlots);
-                // Slots 5..10 are filled once (waited for on the first iteration).  Slots 0..4 are filled once before the loop and once
-                // in every iteration: the first five positions use fill number it_n (there since the previous iteration), the last
-                // five fill number it_n + 1 (requested in this iteration).
-                if (p >= 5 && p < kSlots) {
-                    if (it_n == 0) ok_in = mbar_wait(bar_full + 8 * slot, 0);
-                } else {
-                    ok_in = mbar_wait(bar_full + 8 * slot, (p < 5 ? it_n : it_n + 1u) & 1u);
-                }
-                if (!ok_in) break;
-                tc_fence_after();
-                const uint32_t d = tmem + ((uint32_t)(16 * (b >> 3)) << 16) + (uint32_t)(b & 7) * 64;
-                const uint64_t ad = PASS == 1 ? smem_desc_sw128(s_base + F_OFF_A + b * 8192, 16, 1024) : smem_desc(s_base + F_OFF_A + b * 8192, 1024, 128);
-                const uint64_t bd = smem_desc_sw128(s_base + F_OFF_W + slot * 8192, 16, 1024);
-                constexpr uint64_t a_step = PASS == 1 ? 2 : 128;   // per K step of 16: 32 bytes of a swizzled row, or two 1 KB chunks (in 16-byte units)
+    auto timed_out = [&]() {
+        atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
+        *abort_flag = 1;
+    };
+
+    if (warp < kLoadWarps) {
+        // ---- loading warps: the 2048 pieces of an item, 8 per thread ----
+        // Pass 1: (token tid / 8, n1 = 8 (tid % 8) + i), a piece = 16 consecutive n2; the quarter-warp that shared memory serves a
+        // 16-byte store in writes the 8 chunks of one row: no bank conflicts.
+        // Pass 2: (token 16 (warp / 4) + 8 (i / 4) + lane % 8, k1 = 4 (warp % 4) + lane / 8 of the group, n2 / 16 = i % 4): a warp reads 8
+        // whole lines, and a quarter-warp stores to 8 different rows.
+        const int t_in = PASS == 1 ? tid >> 3 : 16 * (warp >> 2) + (lane & 7);
+        const int sub = PASS == 1 ? tid & 7 : 4 * (warp & 3) + (lane >> 3);
+        uint32_t w[8][8];
+        auto load_in = [&](long long it) {
+            const long long tile = it >> 2;
+            if (PASS == 1) {
+                const bool live = tile * kTok + t_in < T;
+                const unsigned char* src =
+                    reinterpret_cast<const unsigned char*>(in) + (size_t)(tile * kTok + t_in) * 8192 + (size_t)(8 * sub) * 128 + grp * 32;
 #pragma unroll
-                for (int s = 0; s < 4; ++s) umma_f16(d, ad + s * a_step, bd + s * 2, IDESC, s > 0);
-                if (p < 5) umma_commit(bar_empty + 8 * slot);   // the slot's other block may come in
-            }
-            umma_commit(bar_mma);   // (with nothing issued it completes at once; the missing input is reported here)
-            if (!ok_in) {
-                atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-                *abort_flag = 1;
-            }
-        } else if (tid == 32) {   // re-fill slots 0..4 with the blocks this tile runs last: 11..15 on even iterations, 4..0 on odd ones
-#pragma unroll 1
-            for (int p = kSlots; p < kGroup2; ++p) {
-                const int b = odd ? kGroup2 - 1 - p : p;
-                if (!mbar_wait(bar_empty + 8 * (b % kSlots), it_n & 1u)) {
-                    atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-                    *abort_flag = 1;
-                    break;
+                for (int i = 0; i < 8; ++i) {   // cached in L2 only: the rest of every line belongs to other SMs
+                    if (live) {
+                        asm volatile("ld.global.cg.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                     : "=r"(w[i][0]), "=r"(w[i][1]), "=r"(w[i][2]), "=r"(w[i][3]), "=r"(w[i][4]), "=r"(w[i][5]), "=r"(w[i][6]), "=r"(w[i][7])
+                                     : "l"(src + i * 128));
+                    } else {
+#pragma unroll
+                        for (int m = 0; m < 8; ++m) w[i][m] = 0u;
+                    }
                 }
-                load_block(b);
-                ++fills[b % kSlots];
+            } else {   // whole tiles of the workspace were written
+                const unsigned char* src =
+                    reinterpret_cast<const unsigned char*>(in) + (size_t)tile * kTileBytes + (size_t)t_in * 2048 + (size_t)(16 * grp + sub) * 32;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    asm volatile("ld.global.cg.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                 : "=r"(w[i][0]), "=r"(w[i][1]), "=r"(w[i][2]), "=r"(w[i][3]), "=r"(w[i][4]), "=r"(w[i][5]), "=r"(w[i][6]), "=r"(w[i][7])
+                                 : "l"(src + (size_t)(i & 3) * 65536 + (size_t)(i >> 2) * (8 * 2048)));
             }
-            if (PASS == 1) mbar_arrive(bar_go);   // (also after a failed wait: nobody is left waiting for this)
-        } else if (tid == 64) {
-            prefetch_item(next + gridDim.x);
-        }
-        __syncwarp();   // the lanes that share a warp with an issuing or producing thread must not spin on a barrier while it works
-        // pass 1: the next tile's pieces are requested now and arrive while this tile's accumulators are computed and drained --
-        // but only once the five weight blocks this tile still needs have been requested: behind 64 K piece requests they would
-        // arrive thousands of cycles late, and the last UMMAs wait for them
-        if (PASS == 1 && next < nitems) {
-            if (tid != 32 && !mbar_wait(bar_go, it_n & 1u)) *abort_flag = 1;
-            load_x(next);
-        }
-        ok = mbar_wait(bar_mma, it_n & 1u);
-        tc_fence_after();
-        // pass 2: the operand buffer is free again: the next tile's operands come in while this tile is stored
-        if (PASS == 2 && tid == 0) {
-            z_pending = false;
-            if (ok && next < nitems) {
-                load_z(next);
-                z_pending = true;
-                z_par = (it_n + 1u) & 1u;
+        };
+        auto store_opnd = [&]() {
+            if (PASS == 1) {   // the 16 x 8 transpose in registers (this is P): 16 bytes = 8 consecutive n1 of one (t, n2)
+                unsigned char* dst = smem + F_OFF_A + sw_off(t_in, sub);
+#pragma unroll
+                for (int m = 0; m < 8; ++m) {
+                    uint4 lo, hi;
+                    lo.x = prmt(w[0][m], w[1][m], 0x5410); hi.x = prmt(w[0][m], w[1][m], 0x7632);
+                    lo.y = prmt(w[2][m], w[3][m], 0x5410); hi.y = prmt(w[2][m], w[3][m], 0x7632);
+                    lo.z = prmt(w[4][m], w[5][m], 0x5410); hi.z = prmt(w[4][m], w[5][m], 0x7632);
+                    lo.w = prmt(w[6][m], w[7][m], 0x5410); hi.w = prmt(w[6][m], w[7][m], 0x7632);
+                    *reinterpret_cast<uint4*>(dst + (2 * m) * 4096) = lo;
+                    *reinterpret_cast<uint4*>(dst + (2 * m + 1) * 4096) = hi;
+                }
+            } else {           // a piece is 32 bytes of row t of block k1's operand as it lies
+                unsigned char* dst = smem + F_OFF_A + sub * 4096;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int t = t_in + 8 * (i >> 2), c = 2 * (i & 3);
+                    *reinterpret_cast<uint4*>(dst + sw_off(t, c)) = make_uint4(w[i][0], w[i][1], w[i][2], w[i][3]);
+                    *reinterpret_cast<uint4*>(dst + sw_off(t, c + 1)) = make_uint4(w[i][4], w[i][5], w[i][6], w[i][7]);
+                }
             }
-        }
-        // epilogue: lane l of lane quarter q holds token 16 q + (l & 15) of block set l >> 4 (blocks 8 set .. 8 set + 7); the four warps
-        // of a quarter split the 64 output columns.  For every output index the 8 accumulators of a thread are 8 consecutive block
-        // indices: one 16-byte piece.
-        if (ok) {
-            const int q = warp & 3, c4 = warp >> 2, tt = 16 * q + (lane & 15), set = lane >> 4;
-            const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
-            const bool live = t0 + tt < T;
-            unsigned char* dst;
-            if (PASS == 1)   // z[tile][k1][octet 2 grp + set][tt][16 B]
-                dst = reinterpret_cast<unsigned char*>(out) + (size_t)tile * (64 * 8192) + (size_t)(2 * grp + set) * 1024 + tt * 16;
-            else             // y[t][k2][16 grp + 8 set ..]
-                dst = reinterpret_cast<unsigned char*>(out) + (size_t)(t0 + tt) * 8192 + (size_t)(16 * grp + 8 * set) * 2;
+        };
+        if (item < nitems) load_in(item);
 #pragma unroll 1
-            for (int gk = 0; gk < 4; ++gk) {
-                const int o0 = 16 * c4 + 4 * gk;
+        for (; item < nitems; item += gridDim.x, ++it_n) {
+            if (__any_sync(~0u, *abort_flag != 0)) break;
+            // the UMMAs of the previous tile have read the operand buffer
+            if (it_n > 0) ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * ((it_n - 1u) & 1u), ((it_n - 1u) >> 1) & 1u));
+            if (!ok) break;
+            store_opnd();
+            fence_proxy_async();   // operands visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_opnd);
+            // the next tile's pieces are requested now and arrive while this one is computed
+            if (item + gridDim.x < nitems) load_in(item + gridDim.x);
+            if (tid == 33) prefetch_item(item + 2 * (long long)gridDim.x);
+        }
+        if (!ok && lane == 0) timed_out();
+    } else if (warp < kLoadWarps + kDrainWarps) {
+        // ---- draining warps: lane l of lane quarter q = warp % 4 holds output index 16 q + (l & 15) of blocks 8 (l >> 4) .. + 7; the two
+        // warps of a quarter split the 32 tokens.  For every token the 8 accumulators of a thread are 8 consecutive block indices:
+        // one 16-byte piece. ----
+        const int q = warp & 3, c2 = (warp - kLoadWarps) >> 2, r = 16 * q + (lane & 15), set = lane >> 4;
+#pragma unroll 1
+        for (; item < nitems; item += gridDim.x, ++it_n) {
+            if (__any_sync(~0u, *abort_flag != 0)) break;
+            const uint32_t p = it_n & 1u;
+            const long long tile = item >> 2, t0 = tile * kTok + 16 * c2;
+            ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * p, (it_n >> 1) & 1u));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16) + p * 256u + 16u * c2;
+            // pass 1: z[tile][grp][t][k1][32 B], straight from registers, 512 contiguous bytes per warp store
+            unsigned char* dst = reinterpret_cast<unsigned char*>(out) + (size_t)tile * kTileBytes + (size_t)grp * 65536 + (size_t)(16 * c2) * 2048 + r * 32 + set * 16;
+            // pass 2: this warp's staging buffers; chunk (16 bytes) index XOR bit 7 of the address = the 32-byte swizzle of the box
+            const uint32_t st_warp = F_OFF_ST + (uint32_t)(warp - kLoadWarps) * 4096u;
+            const uint32_t st_lane = (uint32_t)(lane & 15) * 32u + (uint32_t)((set ^ ((lane >> 2) & 1)) << 4);
+#pragma unroll 1
+            for (int h = 0; h < 4; ++h) {
                 float v[8][4];
 #pragma unroll
-                for (int bl = 0; bl < 8; ++bl) tmem_ld4(t_lane + bl * 64 + o0, v[bl]);
+                for (int bl = 0; bl < 8; ++bl) tmem_ld4(t_lane + bl * 32 + 4 * h, v[bl]);
+                if (PASS == 2) {   // the buffer of two rounds ago has been read by its store
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                }
                 tmem_ld_wait();
 #pragma unroll
                 for (int bl = 0; bl < 8; ++bl) tmem_ld_fence4(v[bl]);
-                if (PASS == 2 && Kmul != nullptr && live) {
-                    // y = sigma(K (.) M x) (first half of the M2 operator, Eq. 2): the 8 accumulators of one output index are 8
-                    // consecutive k1 -> one 16-byte piece of the kernel row
-                    const __nv_bfloat16* krow = Kmul + (size_t)((t0 + tt) % Hk) * 4096 + 16 * grp + 8 * set;
+                if (PASS == 2 && Kmul != nullptr) {
+                    // y = sigma(K (.) M x) (first half of the M2 operator, Eq. 2): the 8 accumulators of one token are 8 consecutive k1
+                    // -> one 16-byte piece of the kernel row
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        const uint4 kp = *reinterpret_cast<const uint4*>(krow + (o0 + kk) * 64);
-                        const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
+                        const long long t = t0 + 4 * h + kk;
+                        if (t < T) {
+                            const uint4 kp = *reinterpret_cast<const uint4*>(Kmul + (size_t)(t % Hk) * 4096 + r * 64 + 16 * grp + 8 * set);
+                            const uint32_t kw[4] = {kp.x, kp.y, kp.z, kp.w};
 #pragma unroll
-                        for (int pp = 0; pp < 4; ++pp) {
-                            float a = v[2 * pp][kk] * __uint_as_float(kw[pp] << 16);
-                            float bb = v[2 * pp + 1][kk] * __uint_as_float(kw[pp] & 0xffff0000u);
-                            v[2 * pp][kk] = relu ? fmaxf(a, 0.f) : a;
-                            v[2 * pp + 1][kk] = relu ? fmaxf(bb, 0.f) : bb;
+                            for (int pp = 0; pp < 4; ++pp) {
+                                float a = v[2 * pp][kk] * __uint_as_float(kw[pp] << 16);
+                                float bb = v[2 * pp + 1][kk] * __uint_as_float(kw[pp] & 0xffff0000u);
+                                v[2 * pp][kk] = relu ? fmaxf(a, 0.f) : a;
+                                v[2 * pp + 1][kk] = relu ? fmaxf(bb, 0.f) : bb;
+                            }
                         }
                     }
                 }
+                unsigned char* stg = smem + st_warp + (uint32_t)(h & 1) * 2048u + st_lane;
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
                     const uint4 pk = make_uint4(pack_bf16(v[0][kk], v[1][kk]), pack_bf16(v[2][kk], v[3][kk]),
                                                 pack_bf16(v[4][kk], v[5][kk]), pack_bf16(v[6][kk], v[7][kk]));
                     if (PASS == 1)   // whole tiles of the workspace are written (rows past T are zeros)
-                        *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 8192) = pk;
-                    else if (live)
-                        *reinterpret_cast<uint4*>(dst + (size_t)(o0 + kk) * 128) = pk;
+                        *reinterpret_cast<uint4*>(dst + (size_t)(4 * h + kk) * 2048) = pk;
+                    else
+                        *reinterpret_cast<uint4*>(stg + kk * 512) = pk;
+                }
+                if (PASS == 2) {
+                    fence_proxy_async();   // staged rows visible to the copy engine
+                    __syncwarp();
+                    if (lane == 0 && t0 + 4 * h < T) {   // (a box that starts past T has nothing to store)
+                        tma_store_3d(&map_y, s_base + st_warp + (uint32_t)(h & 1) * 2048u, 16 * grp, 16 * q, (int)(t0 + 4 * h));
+                        tma_store_commit();
+                    }
                 }
             }
+            // the set may be overwritten: this warp's TMEM loads are complete
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tfree + 8 * p);
         }
-        if (!ok && tid == 0) {
-            atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
-            *abort_flag = 1;
+        if (PASS == 2 && lane == 0) tma_store_wait_all0();   // this thread's stores are complete before shared memory goes away
+        if (!ok && lane == 0) timed_out();
+    } else if (lane == 0) {
+        // ---- issuing threads ----
+        constexpr uint32_t IDESC = instr_desc_bf16(64, kTok, false, false);
+        constexpr int kPer = kGroup2 / kIssueWarps;
+        const int b0 = (warp - kLoadWarps - kDrainWarps) * kPer;
+        ok = mbar_wait(bar_w, 0);
+#pragma unroll 1
+        for (; item < nitems && ok && *abort_flag == 0; item += gridDim.x, ++it_n) {
+            const uint32_t p = it_n & 1u;
+            ok = mbar_wait(bar_opnd, p);
+            if (ok && it_n >= 2) ok = mbar_wait(bar_tfree + 8 * p, ((it_n - 2u) >> 1) & 1u);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int b = b0; b < b0 + kPer; ++b) {
+                const uint32_t d = tmem + ((uint32_t)(16 * (b >> 3)) << 16) + p * 256u + (uint32_t)(b & 7) * kTok;
+                const uint64_t ad = smem_desc_sw128(s_base + F_OFF_W + b * 8192, 16, 1024);
+                const uint64_t bd = smem_desc_sw128(s_base + F_OFF_A + b * 4096, 16, 1024);
+#pragma unroll
+                for (int s = 0; s < 4; ++s) umma_f16(d, ad + s * 2, bd + s * 2, IDESC, s > 0);   // K step of 16: 32 bytes of a swizzled row
+            }
+            umma_commit(bar_mma + 8 * p);
         }
-        // pass 1: the operand buffer is free (this tile's UMMAs are complete): the next tile's operands go in
-        if (PASS == 1 && ok && next < nitems) store_a();
+        if (!ok) timed_out();
     }
-    // teardown: nothing of ours may be in flight when the CTA goes away (only after a wait ran out can anything be left)
-    if (PASS == 2 && tid == 0 && z_pending) mbar_wait(bar_in, z_par);
-    if (tid == 32)
-        for (int sl = 0; sl < 5; ++sl)
-            if (fills[sl] > 0) mbar_wait(bar_full + 8 * sl, (uint32_t)(fills[sl] - 1) & 1u);
+    // teardown: the weight copy is the only thing that can still be in flight (after a wait ran out)
+    if (tid == 32) mbar_wait(bar_w, 0);
     tc_fence_before();
     __syncthreads();
-    if (warp == 2) tmem_dealloc(*reinterpret_cast<volatile uint32_t*>(smem + tmem_slot), 512);
+    if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
 // ---- gradients with respect to the weight blocks ------------------------------------------------------------------
@@ -765,19 +765,23 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     // the 32-byte loads of pass 1 want x on a 32-byte boundary (torch allocations are; a view need not be)
     if ((reinterpret_cast<uintptr_t>(X) & 31u) != 0) return matmul_g8(pl, X, L, R, Y, T, ws, Kmul, Hk, relu, stream);
     // weight blocks as TMA tiles: [64 blocks x 64 rows][64] bf16, one box = one block, 128-byte swizzle
-    alignas(64) CUtensorMap mr, ml;
+    alignas(64) CUtensorMap mr, ml, my;
     const cuuint64_t gdim[2] = {64, 64 * 64}, gstr[1] = {128};
     const cuuint32_t box[2] = {64, 64};
     if (!tma_host::encode_sw128_bf16(&mr, R, 2, gdim, gstr, box) || !tma_host::encode_sw128_bf16(&ml, L, 2, gdim, gstr, box))
         return M2_ERR_UNSUPPORTED;
+    // y[t][k2][k1] seen as (k1 64 | k2, stride 128 B | t, stride 8 KB); box = 16 k1 x 16 k2 x 4 tokens, 32-byte swizzle
+    const cuuint64_t ydim[3] = {64, 64, (cuuint64_t)T}, ystr[2] = {128, 8192};
+    const cuuint32_t ybox[3] = {16, 16, 4};
+    if (!tma_host::encode_sw32_bf16(&my, Y, 3, ydim, ystr, ybox)) return M2_ERR_UNSUPPORTED;
     cudaLaunchConfig_t cfg = {};
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long nitems = 4 * ((T + kTile2 - 1) / kTile2);
+    const long long nitems = 4 * ((T + kTok - 1) / kTok);
     const long long ctas = (sms / 4) * 4 > 4 ? (sms / 4) * 4 : 4;   // a multiple of 4: a CTA keeps its block group
     cfg.gridDim = dim3((unsigned)(nitems < ctas ? nitems : ctas));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(kFwdThreads);
     cfg.dynamicSmemBytes = F_SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -785,10 +789,10 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<1>, (const __nv_bfloat16*)X, mr, (__nv_bfloat16*)ws, (long long)T, pl->d_status,
+    if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<1>, (const __nv_bfloat16*)X, mr, my, (__nv_bfloat16*)ws, (long long)T, pl->d_status,
                            (const __nv_bfloat16*)nullptr, 1LL, 0) != cudaSuccess)
         return M2_ERR_CUDA;
-    if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<2>, (const __nv_bfloat16*)ws, ml, (__nv_bfloat16*)Y, (long long)T, pl->d_status,
+    if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<2>, (const __nv_bfloat16*)ws, ml, my, (__nv_bfloat16*)Y, (long long)T, pl->d_status,
                            (const __nv_bfloat16*)Kmul, (long long)(Hk > 0 ? Hk : 1), relu) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "matmul_umma_64x64";

@@ -189,6 +189,22 @@ def test_config3_small_full_compare(T, b):
     check(Y, ref, TOL_BF16, f"config3 T={T} b={b} {name}")
 
 
+def test_matmul_input_at_an_odd_16_byte_offset():
+    """X that is only 16-byte aligned (a view into a larger buffer) takes the kernels with 16-byte pieces: same result."""
+    c = synth.config3(T=200, b=64)
+    plan = M.Plan((64, 64), dtype=M.M2_BF16, device=0)
+    buf = torch.zeros(200 * 4096 + 8, dtype=torch.bfloat16, device="cuda")
+    X = buf[8:].view(200, 4096)
+    X.copy_(dev(c["X"], torch.bfloat16))
+    assert X.data_ptr() % 32 == 16
+    Y = M.m2_monarch_matmul(plan, X, dev(c["L"], torch.bfloat16), dev(c["R"], torch.bfloat16))
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "matmul_umma_64x64_g8"
+    ref = O.monarch_apply(c["L"].astype(np.float64), c["R"].astype(np.float64), c["X"].astype(np.float64))
+    check(host(Y), ref, TOL_BF16, "matmul, 16-byte aligned input")
+    plan.close()
+
+
 def test_matmul_fp32_rectangular_vs_dense():
     N1, N2, T = 8, 4, 9
     X = synth.normal(31, (T, N1 * N2)).astype(np.float32)

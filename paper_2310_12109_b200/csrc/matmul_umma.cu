@@ -287,6 +287,8 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
     const int grp = blockIdx.x & 3;                                   // which 16 consecutive blocks (n2 in pass 1, k1 in pass 2)
     const long long ntiles = (T + kTok - 1) / kTok, nitems = 4 * ntiles;
     long long item = blockIdx.x;
+    // pass 2 walks the tiles from the last to the first: what pass 1 wrote last is what the L2 still holds
+    auto tile_of = [&](long long it) { return PASS == 1 ? it >> 2 : ntiles - 1 - (it >> 2); };
     if (tid == 0) {
         mbar_init(bar_w, 1);
         mbar_init(bar_mma, kIssueWarps);       // one arrival per issuing thread
@@ -311,7 +313,7 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
     // share a tile ask for a quarter each).  L2 is where the previous kernel's writes land, so nothing stale can be fetched.
     auto prefetch_item = [&](long long it) {
         if (it < nitems) {
-            const long long t0p = (it >> 2) * kTok;
+            const long long t0p = tile_of(it) * kTok;
             const long long rows = PASS == 2 || T - t0p >= kTok ? kTok : T - t0p;   // (whole tiles of the workspace exist)
             const long long share = rows * 8192 / 4;
             bulk_prefetch_l2(reinterpret_cast<const unsigned char*>(in) + t0p * 8192 + grp * share, (uint32_t)share);
@@ -341,7 +343,7 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
         const int sub = PASS == 1 ? tid & 7 : 4 * (warp & 3) + (lane >> 3);
         uint32_t w[8][8];
         auto load_in = [&](long long it) {
-            const long long tile = it >> 2;
+            const long long tile = tile_of(it);
             if (PASS == 1) {
                 const bool live = tile * kTok + t_in < T;
                 const unsigned char* src =
@@ -415,7 +417,7 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
         for (; item < nitems; item += gridDim.x, ++it_n) {
             if (__any_sync(~0u, *abort_flag != 0)) break;
             const uint32_t p = it_n & 1u;
-            const long long tile = item >> 2, t0 = tile * kTok + 16 * c2;
+            const long long tile = tile_of(item), t0 = tile * kTok + 16 * c2;
             ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * p, (it_n >> 1) & 1u));
             if (!ok) break;
             tc_fence_after();

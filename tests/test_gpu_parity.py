@@ -189,6 +189,31 @@ def test_config3_small_full_compare(T, b):
     check(Y, ref, TOL_BF16, f"config3 T={T} b={b} {name}")
 
 
+def test_matmul_token_counts_around_the_tile_boundaries():
+    """Token counts on both sides of the 32-token tile and of the 148 x 4 item boundaries, one plan and ONE workspace for
+    all calls, no synchronisation between them (a call's pass 1 may only overwrite the workspace after the previous call's
+    pass 2 has read it); rows past T of the output buffer must stay untouched."""
+    c = synth.config3(T=4800, b=64)
+    plan = M.Plan((64, 64), dtype=M.M2_BF16, device=0)
+    L, R = dev(c["L"], torch.bfloat16), dev(c["R"], torch.bfloat16)
+    Xall = dev(c["X"], torch.bfloat16)
+    ws = M.m2_matmul_workspace(plan, 4800)
+    counts = (31, 32, 33, 63, 64, 65, 1183, 1184, 1185, 4735, 4737, 4800, 2, 95)
+    outs = []
+    for T in counts:
+        Y = torch.full((T + 3, 4096), 5.0, dtype=torch.bfloat16, device="cuda")
+        M.m2_monarch_matmul(plan, Xall[:T], L, R, Y[:T], ws=ws)
+        outs.append(Y)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0
+    L64, R64 = c["L"].astype(np.float64), c["R"].astype(np.float64)
+    ref = O.monarch_apply(L64, R64, c["X"].astype(np.float64))
+    for T, Y in zip(counts, outs):
+        assert bool((Y[T:] == 5.0).all()), f"T={T}: rows past T were written"
+        check(host(Y[:T]), ref[:T], TOL_BF16, f"matmul T={T}")
+    plan.close()
+
+
 def test_matmul_input_at_an_odd_16_byte_offset():
     """X that is only 16-byte aligned (a view into a larger buffer) takes the kernels with 16-byte pieces: same result."""
     c = synth.config3(T=200, b=64)

@@ -337,6 +337,15 @@ int32_t m2_blocky_monarch_conv_fwd(const m2_plan* plan, const void* factors_dev,
 int32_t m2_selftest_bounded_wait(const m2_plan* plan, const void* x_dev, const void* kf_dev, void* y_dev, int64_t B,
                                  int64_t H, int64_t n, int32_t mode, void* stream);
 
+/* The same self-test for the tensor-core Monarch matmul (bf16 plans with 64 x 64 blocks): launches the two passes of
+ * m2_monarch_matmul with its arguments in a mode where the issuing threads give the tensor core nothing and every wait
+ * for it gives up after a few polls, so that the loading, draining and issuing warps of every CTA leave through their
+ * abort paths.  Y_dev and ws_dev are not written.  Afterwards m2_last_device_status reports M2_ERR_TIMEOUT (and resets
+ * it) and the plan serves ordinary calls as before.  Needs T > 0, X_dev on a 32-byte boundary and a workspace of
+ * m2_matmul_workspace_bytes(plan, T) bytes; M2_ERR_UNSUPPORTED otherwise. */
+int32_t m2_selftest_bounded_wait_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev,
+                                        void* Y_dev, int64_t T, void* ws_dev, int64_t ws_bytes, void* stream);
+
 const char* m2_status_string(int32_t status);
 
 /* Reads (synchronously) the device status word kernels set when a bounded wait expires or a

@@ -56,6 +56,7 @@ SIGNATURES = {
     "m2_blocky_kernel_spectrum": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp, _vp]),
     "m2_blocky_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_selftest_bounded_wait": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
+    "m2_selftest_bounded_wait_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_status_string": (ctypes.c_char_p, [_i32]),
     "m2_last_device_status": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "m2_last_kernel_name": (ctypes.c_char_p, [_vp]),
@@ -255,6 +256,14 @@ def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Ten
     _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _ptr(ws),
                                    0 if ws is None else ws.numel(), _stream()), "m2_monarch_matmul")
     return Y
+
+
+def m2_selftest_bounded_wait_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Tensor, Y: torch.Tensor, ws: torch.Tensor):
+    """The two matmul passes in the mode where every wait for the tensor core runs out; Y and ws are not written."""
+    for t in (X, L, R, Y):
+        assert t.is_cuda and t.dtype == plan.torch_dtype and t.is_contiguous()
+    _check(lib().m2_selftest_bounded_wait_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _ptr(ws), ws.numel(),
+                                                 _stream()), "m2_selftest_bounded_wait_matmul")
 
 
 M2_ACT_NONE, M2_ACT_RELU = 0, 1

@@ -400,6 +400,17 @@ int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_
     return matmul_impl(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, ws_bytes, nullptr, 1, 0, (cudaStream_t)stream);
 }
 
+int32_t m2_selftest_bounded_wait_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, void* Y_dev,
+                                        int64_t T, void* ws_dev, int64_t ws_bytes, void* stream) {
+    int32_t st = check_matmul_args(plan, X_dev, L_dev, R_dev, Y_dev, T);
+    if (st != M2_OK) return st;
+    if (ws_dev && !aligned16(ws_dev)) return M2_ERR_ALIGNMENT;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    if (T == 0 || !m2mm::covered(plan) || !ws_dev || ws_bytes < m2mm::workspace_bytes(plan, T)) return M2_ERR_UNSUPPORTED;
+    return m2mm::matmul_wait_selftest(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, (cudaStream_t)stream);
+}
+
 int32_t m2_monarch_mix(const m2_plan* plan, const void* X_dev, const void* K_dev, int64_t Hk, int32_t act, const void* La_dev,
                        const void* Ra_dev, const void* Lb_dev, const void* Rb_dev, void* Y_dev, int64_t T, void* ws_dev,
                        int64_t ws_bytes, void* stream) {

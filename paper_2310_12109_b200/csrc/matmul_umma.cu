@@ -278,11 +278,15 @@ static_assert(F_SMEM_BYTES <= 232448, "shared-memory budget of the forward passe
 template <int PASS>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant__ CUtensorMap map_w,
-                     const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ out, long long T, int32_t* __restrict__ status, const __nv_bfloat16* __restrict__ Kmul, long long Hk, int relu) {
+                     const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ out, long long T,
+                     int32_t* __restrict__ status, const __nv_bfloat16* __restrict__ Kmul, long long Hk, int relu, int selftest) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
     const uint32_t bar_w = s_base + F_OFF_BAR, bar_mma = bar_w + 8, s_tptr = bar_w + 24, bar_opnd = bar_w + 40, bar_tfree = bar_w + 48;
+    // selftest: the issuing threads issue and commit nothing and every wait for them gives up after a few polls, so that all
+    // roles leave through their abort paths with nothing of theirs in flight
+    const uint32_t wlim = selftest ? 64u : (1u << 22);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + F_OFF_BAR + 32);
     const int grp = blockIdx.x & 3;                                   // which 16 consecutive blocks (n2 in pass 1, k1 in pass 2)
     const long long ntiles = (T + kTok - 1) / kTok, nitems = 4 * ntiles;
@@ -397,7 +401,7 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
         for (; item < nitems; item += gridDim.x, ++it_n) {
             if (__any_sync(~0u, *abort_flag != 0)) break;
             // the UMMAs of the previous tile have read the operand buffer
-            if (it_n > 0) ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * ((it_n - 1u) & 1u), ((it_n - 1u) >> 1) & 1u));
+            if (it_n > 0) ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * ((it_n - 1u) & 1u), ((it_n - 1u) >> 1) & 1u, wlim));
             if (!ok) break;
             store_opnd();
             fence_proxy_async();   // operands visible to the tensor core
@@ -418,7 +422,7 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
             if (__any_sync(~0u, *abort_flag != 0)) break;
             const uint32_t p = it_n & 1u;
             const long long tile = tile_of(item), t0 = tile * kTok + 16 * c2;
-            ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * p, (it_n >> 1) & 1u));
+            ok = __all_sync(~0u, mbar_wait(bar_mma + 8 * p, (it_n >> 1) & 1u, wlim));
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16) + p * 256u + 16u * c2;
@@ -493,9 +497,10 @@ monarch64_fwd_kernel(const __nv_bfloat16* __restrict__ in, const __grid_constant
 #pragma unroll 1
         for (; item < nitems && ok && *abort_flag == 0; item += gridDim.x, ++it_n) {
             const uint32_t p = it_n & 1u;
-            ok = mbar_wait(bar_opnd, p);
-            if (ok && it_n >= 2) ok = mbar_wait(bar_tfree + 8 * p, ((it_n - 2u) >> 1) & 1u);
+            ok = mbar_wait(bar_opnd, p, wlim);
+            if (ok && it_n >= 2) ok = mbar_wait(bar_tfree + 8 * p, ((it_n - 2u) >> 1) & 1u, wlim);
             if (!ok) break;
+            if (selftest) continue;
             tc_fence_after();
 #pragma unroll 1
             for (int b = b0; b < b0 + kPer; ++b) {
@@ -760,12 +765,13 @@ static int32_t matmul_g8(const m2_plan* pl, const void* X, const void* L, const 
     return M2_OK;
 }
 
-int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
-               int64_t Hk, int relu, cudaStream_t stream) {
+static int32_t matmul_impl(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
+                           int64_t Hk, int relu, int selftest, cudaStream_t stream) {
     if (!covered(pl)) return M2_ERR_UNSUPPORTED;
-    if (T == 0) return M2_OK;
+    if (T == 0) return selftest ? M2_ERR_UNSUPPORTED : M2_OK;
     // the 32-byte loads of pass 1 want x on a 32-byte boundary (torch allocations are; a view need not be)
-    if ((reinterpret_cast<uintptr_t>(X) & 31u) != 0) return matmul_g8(pl, X, L, R, Y, T, ws, Kmul, Hk, relu, stream);
+    if ((reinterpret_cast<uintptr_t>(X) & 31u) != 0)
+        return selftest ? M2_ERR_UNSUPPORTED : matmul_g8(pl, X, L, R, Y, T, ws, Kmul, Hk, relu, stream);
     // weight blocks as TMA tiles: [64 blocks x 64 rows][64] bf16, one box = one block, 128-byte swizzle
     alignas(64) CUtensorMap mr, ml, my;
     const cuuint64_t gdim[2] = {64, 64 * 64}, gstr[1] = {128};
@@ -792,14 +798,24 @@ int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, v
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<1>, (const __nv_bfloat16*)X, mr, my, (__nv_bfloat16*)ws, (long long)T, pl->d_status,
-                           (const __nv_bfloat16*)nullptr, 1LL, 0) != cudaSuccess)
+                           (const __nv_bfloat16*)nullptr, 1LL, 0, selftest) != cudaSuccess)
         return M2_ERR_CUDA;
     if (cudaLaunchKernelEx(&cfg, monarch64_fwd_kernel<2>, (const __nv_bfloat16*)ws, ml, my, (__nv_bfloat16*)Y, (long long)T, pl->d_status,
-                           (const __nv_bfloat16*)Kmul, (long long)(Hk > 0 ? Hk : 1), relu) != cudaSuccess)
+                           (const __nv_bfloat16*)Kmul, (long long)(Hk > 0 ? Hk : 1), relu, selftest) != cudaSuccess)
         return M2_ERR_CUDA;
     pl->last_kernel = "matmul_umma_64x64";
     pl->launches += 2;
     return M2_OK;
+}
+
+int32_t matmul(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws, const void* Kmul,
+               int64_t Hk, int relu, cudaStream_t stream) {
+    return matmul_impl(pl, X, L, R, Y, T, ws, Kmul, Hk, relu, 0, stream);
+}
+
+int32_t matmul_wait_selftest(const m2_plan* pl, const void* X, const void* L, const void* R, void* Y, int64_t T, void* ws,
+                             cudaStream_t stream) {
+    return matmul_impl(pl, X, L, R, Y, T, ws, nullptr, 1, 0, 1, stream);
 }
 
 }  // namespace m2mm

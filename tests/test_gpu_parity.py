@@ -905,6 +905,34 @@ def test_bounded_wait_runs_out_and_the_plan_recovers():
     plan.close()
 
 
+def test_bounded_wait_runs_out_in_the_matmul_and_the_plan_recovers():
+    """The same for the tensor-core matmul: both passes are launched in the mode where the issuing threads give the tensor
+    core nothing and every wait for it runs out after a few polls; the loading, draining and issuing warps of every CTA
+    must leave through their abort paths, report M2_ERR_TIMEOUT and write neither Y nor the workspace; ordinary calls on
+    the same plan are correct afterwards."""
+    c = synth.config3(T=5000, b=64)                       # more items than CTAs: every CTA has a next tile in flight when it gives up
+    plan = M.Plan((64, 64), dtype=M.M2_BF16, device=0)
+    X, L, R = dev(c["X"], torch.bfloat16), dev(c["L"], torch.bfloat16), dev(c["R"], torch.bfloat16)
+    ws = M.m2_matmul_workspace(plan, 5000)
+    ws.fill_(3)
+    Y = torch.full_like(X, 7.0)
+    M.m2_selftest_bounded_wait_matmul(plan, X, L, R, Y, ws)
+    torch.cuda.synchronize()
+    assert plan.device_status() == M.M2_ERR_TIMEOUT
+    assert plan.device_status() == 0                      # reading the word resets it
+    assert bool((Y == 7.0).all()) and bool((ws == 3).all())
+    ref = O.monarch_apply(c["L"].astype(np.float64), c["R"].astype(np.float64), c["X"].astype(np.float64))
+    for _ in range(2):
+        M.m2_monarch_matmul(plan, X, L, R, Y, ws=ws)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0 and plan.last_kernel() == "matmul_umma_64x64"
+        check(host(Y), ref, TOL_BF16, "after the timed-out launches")
+    # no workspace, no self-test
+    lib, st = M.lib(), torch.cuda.current_stream().cuda_stream
+    assert lib.m2_selftest_bounded_wait_matmul(plan.handle, X.data_ptr(), L.data_ptr(), R.data_ptr(), Y.data_ptr(), 5000, None, 0, st) == M.M2_ERR_UNSUPPORTED
+    plan.close()
+
+
 def test_host_buffer_entry_points():
     c = synth.config2(B=2, H=8)
     plan = M.Plan(c["dims"], dtype=M.M2_BF16, device=0)

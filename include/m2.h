@@ -248,6 +248,18 @@ int32_t m2_hyena_heads_fwd(const m2_plan* plan, const void* u_dev, const void* c
 int32_t m2_blocks_transpose(const m2_plan* plan, const void* W_in_dev, void* W_out_dev, int64_t nblocks, int64_t rows,
                             int64_t cols, void* stream);
 
+/* Order-p Monarch product Y_t = M X_t in the direct form (Eq. 1; App. D.6, "p-variate Monarch") for a plan of any order
+ * p = 1..3 with arbitrary (learnable) blocks.  With the input index n = (n_1, .., n_p), n_1 most significant, stage
+ * a = 1..p contracts the digit n_a into the output digit k_a with the block chosen by (k_1, .., k_{a-1}, n_{a+1}, .., n_p);
+ * the output index is k = k_1 + N_1 k_2 + .. (natural order).  W_dev: HOST array of p DEVICE pointers; W_dev[a-1] is
+ * [N / N_a][N_a out][N_a in] of the plan dtype, the block id being the row-major flattening of
+ * (k_1, .., k_{a-1}, n_{a+1}, .., n_p).  (For p >= 3 the paper gives the block index as a tuple only: this linear order is
+ * this library's reading.)  For p = 2, W_dev = {R, L} gives exactly m2_monarch_matmul.  X_dev, Y_dev: [T, N] of the plan
+ * dtype, must not overlap; fp32 accumulation, the row stays in fp32 between the stages.  One CUDA-core kernel; needs
+ * every N_a <= 256 and N <= 51200 (M2_ERR_UNSUPPORTED otherwise).  T == 0 is a no-op. */
+int32_t m2_monarch_apply_order_p(const m2_plan* plan, const void* X_dev, const void* const* W_dev, void* Y_dev, int64_t T,
+                                 void* stream);
+
 /* Gradients of sum_t <Y_t, G_t>, Y = M X with M = P L P^T R P (Sec. 3.1), with respect to the blocks of L and R:
  *   dL[k1][k2][n2] = sum_t G[t][k2 N1 + k1] v[t][n2][k1],           v  = R-stage of the forward pass,
  *   dR[n2][k1][n1] = sum_t dv[t][n2][k1] X[t][n1 N2 + n2],          dv = L^T-stage applied to G.

@@ -57,6 +57,7 @@ SIGNATURES = {
     "m2_blocky_monarch_conv_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "m2_selftest_bounded_wait": (_i32, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp]),
     "m2_selftest_bounded_wait_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
+    "m2_monarch_apply_order_p": (_i32, [_vp, _vp, ctypes.POINTER(ctypes.c_void_p), _vp, _i64, _vp]),
     "m2_status_string": (ctypes.c_char_p, [_i32]),
     "m2_last_device_status": (_i32, [_vp, ctypes.POINTER(_i32)]),
     "m2_last_kernel_name": (ctypes.c_char_p, [_vp]),
@@ -255,6 +256,21 @@ def m2_monarch_matmul(plan: Plan, X: torch.Tensor, L: torch.Tensor, R: torch.Ten
         ws = m2_matmul_workspace(plan, X.shape[0], X.device)
     _check(lib().m2_monarch_matmul(plan.handle, _ptr(X), _ptr(L), _ptr(R), _ptr(Y), X.shape[0], _ptr(ws),
                                    0 if ws is None else ws.numel(), _stream()), "m2_monarch_matmul")
+    return Y
+
+
+def m2_monarch_apply_order_p(plan: Plan, X: torch.Tensor, W, Y: torch.Tensor | None = None) -> torch.Tensor:
+    """Order-p product in the direct form; W: list of p tensors, W[a] of shape [N / N_a, N_a, N_a] (plan dtype)."""
+    assert len(W) == len(plan.dims)
+    for t in [X] + list(W):
+        assert t.is_cuda and t.dtype == plan.torch_dtype and t.is_contiguous()
+    for a, w in enumerate(W):
+        assert tuple(w.shape) == (plan.N // plan.dims[a], plan.dims[a], plan.dims[a])
+    assert X.dim() == 2 and X.shape[1] == plan.N
+    if Y is None:
+        Y = torch.empty_like(X)
+    ptrs = (ctypes.c_void_p * len(W))(*[w.data_ptr() for w in W])
+    _check(lib().m2_monarch_apply_order_p(plan.handle, _ptr(X), ptrs, _ptr(Y), X.shape[0], _stream()), "m2_monarch_apply_order_p")
     return Y
 
 

@@ -476,6 +476,120 @@ cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void*
                    : launch_matmul_t<float>(N1, N2, T, X, L, R, Y, Kmul, Hk, relu, st);
 }
 
+// Order-p Monarch product in the direct form (Eq. 1; App. D.6, "p-variate Monarch"), TT tokens per block, fp32 accumulate:
+// stage a = 1..p contracts the input digit n_a into the output digit k_a with the block chosen by
+// (k_1..k_{a-1}, n_{a+1}..n_p) -- its id is the row-major flattening of that tuple, W[a-1] is [N / N_a][N_a out][N_a in].
+// The row stays in shared memory as an array with axes (k_1..k_{a-1}, n_a..n_p), first axis most significant; a stage
+// works in place: the elements of one block differ only in axis a (stride s_a = N_{a+1} .. N_p), a warp owns a block,
+// reads its N_a inputs (broadcast reads) into up to 8 outputs per lane and writes them back after the warp has
+// finished reading.  The result leaves in natural order k = k_1 + N_1 k_2 + ...
+struct OrderPArgs {
+    const void* W[4];
+    int dims[4];
+    int p;
+};
+
+template <typename IO, int TT>
+__global__ void __launch_bounds__(512) monarch_order_p_kernel(const IO* __restrict__ X, IO* __restrict__ Y, OrderPArgs A, int N, long long T) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* v = reinterpret_cast<float*>(smem_raw);   // [TT][N]
+    const long long t0 = (long long)blockIdx.x * TT;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int i = threadIdx.x; i < TT * N; i += blockDim.x) {
+        const long long t = t0 + i / N;
+        v[i] = (t < T) ? to_f32<IO>(X[t * N + (i % N)]) : 0.f;
+    }
+    __syncthreads();
+    int sa = N;
+    for (int a = 0; a < A.p; ++a) {
+        const int Na = A.dims[a];
+        sa /= Na;                                    // stride of axis a
+        const IO* Wa = reinterpret_cast<const IO*>(A.W[a]);
+        const int nblocks = N / Na;
+        for (int b = warp; b < nblocks; b += nwarps) {
+            const int base = (b / sa) * (Na * sa) + (b % sa);
+            const IO* wb = Wa + (long long)b * Na * Na;
+            float acc[8][TT];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+#pragma unroll
+                for (int t = 0; t < TT; ++t) acc[j][t] = 0.f;
+            for (int i = 0; i < Na; ++i) {
+                float xv[TT];
+#pragma unroll
+                for (int t = 0; t < TT; ++t) xv[t] = v[t * N + base + i * sa];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int o = lane + 32 * j;
+                    if (o < Na) {
+                        const float wv = to_f32<IO>(wb[(long long)o * Na + i]);
+#pragma unroll
+                        for (int t = 0; t < TT; ++t) acc[j][t] = fmaf(wv, xv[t], acc[j][t]);
+                    }
+                }
+            }
+            __syncwarp();   // every lane has read the block's inputs
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int o = lane + 32 * j;
+                if (o < Na)
+#pragma unroll
+                    for (int t = 0; t < TT; ++t) v[t * N + base + o * sa] = acc[j][t];
+            }
+        }
+        __syncthreads();
+    }
+    // axes (k_1..k_p), first most significant  ->  natural order, k_1 least significant
+    for (int i = threadIdx.x; i < N; i += blockDim.x) {
+        int rest = i, nat = 0, w = N;
+        for (int a = 0, mul = 1; a < A.p; ++a) {
+            w /= A.dims[a];
+            const int k = rest / w;
+            rest -= k * w;
+            nat += k * mul;
+            mul *= A.dims[a];
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t)
+            if (t0 + t < T) Y[(t0 + t) * N + nat] = from_f32<IO>(v[t * N + i]);
+    }
+}
+
+template <typename IO>
+static cudaError_t launch_order_p_t(const OrderPArgs& A, int N, long long T, const void* X, void* Y, cudaStream_t st) {
+    if (T == 0) return cudaSuccess;
+    const bool four = (size_t)4 * N * sizeof(float) <= 160 * 1024;
+    const size_t smem = (size_t)(four ? 4 : 1) * N * sizeof(float);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    const int threads = N < 512 * 8 ? 128 : 512;
+    cudaError_t e;
+    if (four) {
+        auto kern = monarch_order_p_kernel<IO, 4>;
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        kern<<<(unsigned)((T + 3) / 4), threads, smem, st>>>((const IO*)X, (IO*)Y, A, N, T);
+    } else {
+        auto kern = monarch_order_p_kernel<IO, 1>;
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        kern<<<(unsigned)T, threads, smem, st>>>((const IO*)X, (IO*)Y, A, N, T);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_order_p(const int* dims, int p, long long T, bool bf16_io, const void* X, const void* const* W, void* Y, cudaStream_t st) {
+    if (p < 1 || p > 4) return cudaErrorInvalidValue;
+    OrderPArgs A;
+    long long N = 1;
+    for (int a = 0; a < 4; ++a) {
+        A.W[a] = a < p ? W[a] : nullptr;
+        A.dims[a] = a < p ? dims[a] : 1;
+        if (a < p && (dims[a] < 1 || dims[a] > 256)) return cudaErrorInvalidValue;   // 8 outputs per lane
+        N *= A.dims[a];
+    }
+    A.p = p;
+    if (N > (1 << 20)) return cudaErrorInvalidValue;
+    return bf16_io ? launch_order_p_t<__nv_bfloat16>(A, (int)N, T, X, Y, st) : launch_order_p_t<float>(A, (int)N, T, X, Y, st);
+}
+
 cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,
                        long long tokens, cudaStream_t st) {
     constexpr int TT = 8;

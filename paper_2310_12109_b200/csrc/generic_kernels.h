@@ -22,6 +22,8 @@ cudaError_t launch_spectrum_to_natural(const ConvShape& s, const void* kf, float
 // Kmul != nullptr: Y = sigma(K (.) M X), K [Hk][N] of the I/O type, row t uses K[t % Hk], sigma = ReLU if relu else identity
 cudaError_t launch_matmul(int N1, int N2, long long T, bool bf16_io, const void* X, const void* L, const void* R, void* Y,
                           const void* Kmul, long long Hk, int relu, cudaStream_t st);
+// order-p product in the direct form: W[a] = [N / dims[a]][dims[a]][dims[a]], block id = row-major (k_1..k_{a-1}, n_{a+1}..n_p)
+cudaError_t launch_order_p(const int* dims, int p, long long T, bool bf16_io, const void* X, const void* const* W, void* Y, cudaStream_t st);
 cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, int expand,
                        long long tokens, cudaStream_t st);
 

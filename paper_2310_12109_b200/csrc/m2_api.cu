@@ -400,6 +400,28 @@ int32_t m2_monarch_matmul(const m2_plan* plan, const void* X_dev, const void* L_
     return matmul_impl(plan, X_dev, L_dev, R_dev, Y_dev, T, ws_dev, ws_bytes, nullptr, 1, 0, (cudaStream_t)stream);
 }
 
+int32_t m2_monarch_apply_order_p(const m2_plan* plan, const void* X_dev, const void* const* W_dev, void* Y_dev, int64_t T, void* stream) {
+    if (!plan || T < 0 || !W_dev) return M2_ERR_INVALID_ARG;
+    if (plan->device < 0) return M2_ERR_NO_DEVICE;
+    if (plan->p < 1 || plan->p > 4) return M2_ERR_UNSUPPORTED;
+    if ((!X_dev || !Y_dev) && T != 0) return M2_ERR_INVALID_ARG;
+    for (int a = 0; a < plan->p; ++a) {
+        if (!W_dev[a] && T != 0) return M2_ERR_INVALID_ARG;
+        if (!aligned16(W_dev[a])) return M2_ERR_ALIGNMENT;
+    }
+    if (!aligned16(X_dev) || !aligned16(Y_dev)) return M2_ERR_ALIGNMENT;
+    if (T > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    if (T == 0) return M2_OK;
+    DeviceGuard g(plan->device);
+    if (!g.ok) return M2_ERR_CUDA;
+    cudaError_t e = m2g::launch_order_p(plan->dims, plan->p, T, plan->dtype == M2_BF16, X_dev, W_dev, Y_dev, (cudaStream_t)stream);
+    if (e == cudaErrorInvalidValue) return M2_ERR_UNSUPPORTED;
+    if (e != cudaSuccess) return M2_ERR_CUDA;
+    plan->last_kernel = "monarch_order_p_generic";
+    plan->launches += 1;
+    return M2_OK;
+}
+
 int32_t m2_selftest_bounded_wait_matmul(const m2_plan* plan, const void* X_dev, const void* L_dev, const void* R_dev, void* Y_dev,
                                         int64_t T, void* ws_dev, int64_t ws_bytes, void* stream) {
     int32_t st = check_matmul_args(plan, X_dev, L_dev, R_dev, Y_dev, T);

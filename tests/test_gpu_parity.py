@@ -230,6 +230,51 @@ def test_matmul_input_at_an_odd_16_byte_offset():
     plan.close()
 
 
+@pytest.mark.parametrize("dims,T,dtype", [((4, 3, 5), 7, "fp32"), ((8, 8, 8), 9, "fp32"), ((2, 9, 5), 5, "fp32"), ((7,), 3, "fp32"),
+                                          ((16, 16, 16), 33, "bf16"), ((32, 32, 32), 6, "bf16"), ((12, 40), 10, "bf16")])
+def test_monarch_apply_order_p(dims, T, dtype):
+    """Order-p product with arbitrary blocks (Eq. 1; App. D.6) against the oracle's direct form: orders 1 to 3, mixed digit
+    sizes, the tokens-per-block variants of the kernel (4 for N <= 10240, 1 beyond)."""
+    N = int(np.prod(dims))
+    bf = dtype == "bf16"
+    rnd = (lambda a: synth.round_bf16(a)) if bf else (lambda a: a.astype(np.float32))
+    X = rnd(synth.normal(900 + N, (T, N)))
+    W = [rnd(synth.normal(901 + N + a, (N // Na, Na, Na)) / np.sqrt(Na)) for a, Na in enumerate(dims)]
+    plan = M.Plan(dims, dtype=M.M2_BF16 if bf else M.M2_FP32, device=0)
+    tdt = torch.bfloat16 if bf else torch.float32
+    Y = M.m2_monarch_apply_order_p(plan, dev(X, tdt), [dev(w, tdt) for w in W])
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "monarch_order_p_generic"
+    ref = O.monarch_apply_order_p([w.astype(np.float64) for w in W], tuple(dims), X.astype(np.float64))
+    check(host(Y), ref, TOL_BF16 if bf else TOL_FP32, f"order-p product {dims} {dtype}")
+    plan.close()
+
+
+def test_monarch_apply_order_p_is_the_matmul_for_p_2():
+    """For p = 2 the direct form with W = (R, L) is M = P L P^T R P (Sec. 3.1): same result as m2_monarch_matmul."""
+    c = synth.config3(T=40, b=16)
+    plan = M.Plan((16, 16), dtype=M.M2_FP32, device=0)
+    X, L, R = dev(c["X"].astype(np.float32)), dev(c["L"].astype(np.float32)), dev(c["R"].astype(np.float32))
+    Y2 = M.m2_monarch_matmul(plan, X, L, R)
+    Yp = M.m2_monarch_apply_order_p(plan, X, [R, L])
+    torch.cuda.synchronize()
+    check(host(Yp), host(Y2).astype(np.float64), 1e-6, "order-p product, p = 2, against the order-2 kernel")
+    ref = O.monarch_apply(c["L"].astype(np.float64), c["R"].astype(np.float64), c["X"].astype(np.float64))
+    check(host(Yp), ref, TOL_FP32, "order-p product, p = 2, against the oracle")
+    # bad arguments: a missing factor, a digit beyond 256
+    lib, st = M.lib(), torch.cuda.current_stream().cuda_stream
+    import ctypes
+    ptrs = (ctypes.c_void_p * 2)(R.data_ptr(), None)
+    assert lib.m2_monarch_apply_order_p(plan.handle, X.data_ptr(), ptrs, Yp.data_ptr(), 40, st) == M.M2_ERR_INVALID_ARG
+    plan.close()
+    big = M.Plan((512, 8), dtype=M.M2_FP32, device=0)
+    Xb = torch.zeros(1, 4096, device="cuda")
+    Wb = [torch.zeros(8, 512, 512, device="cuda"), torch.zeros(512, 8, 8, device="cuda")]
+    ptrs = (ctypes.c_void_p * 2)(Wb[0].data_ptr(), Wb[1].data_ptr())
+    assert lib.m2_monarch_apply_order_p(big.handle, Xb.data_ptr(), ptrs, Xb.clone().data_ptr(), 1, st) == M.M2_ERR_UNSUPPORTED
+    big.close()
+
+
 def test_matmul_fp32_rectangular_vs_dense():
     N1, N2, T = 8, 4, 9
     X = synth.normal(31, (T, N1 * N2)).astype(np.float32)

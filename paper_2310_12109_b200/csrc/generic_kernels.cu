@@ -606,6 +606,26 @@ cudaError_t launch_mlp(const void* z, const void* Wup, const void* Wdn, void* y,
     return cudaGetLastError();
 }
 
+// Launch with programmatic stream serialization (the kernel starts with griddepcontrol.launch_dependents / .wait): its CTAs
+// may be placed while the previous kernel's last CTAs still run, and the next kernel's while this one's do.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+__device__ __forceinline__ void pdl_prologue() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // everything the stream produced before is complete
+}
+
 // ---- channel-last <-> channel-first helpers of the M2 block (Sec. 5.1; Eq. 2 runs along the sequence) -----------------
 // 64 x 64 bf16 tile transposes through shared memory.  The tile is kept as 32-bit words (two neighbouring columns of one
 // row) with a row pitch of 33 words: the 16-byte global loads land as four conflict-free word stores, and the transposed
@@ -635,6 +655,7 @@ __device__ __forceinline__ uint4 tr_get(const uint32_t* tile, int rb, int col) {
 // x[B][T][C] -> xT[B][C][T]; both sides move 16 bytes per thread and whole 128-byte rows per 8 threads.
 __global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ xT, int T, int C) {
     __shared__ uint32_t tile[64 * kTrPitch];   // [t][c pair]
+    pdl_prologue();
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const long long b = blockIdx.z;
     const __nv_bfloat16* src = x + (b * T + t0) * (long long)C + c0;
@@ -657,6 +678,7 @@ __global__ void __launch_bounds__(256) transpose_btc_kernel(const __nv_bfloat16*
 __global__ void __launch_bounds__(256) gate_transpose_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ vT,
                                                              const float* __restrict__ w, __nv_bfloat16* __restrict__ z, int T, int C) {
     __shared__ uint32_t tile[64 * kTrPitch];   // [c][t pair]: v as it arrives
+    pdl_prologue();   // the convolution's output is complete
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const long long b = blockIdx.z;
     const __nv_bfloat16* src = vT + (b * C + c0) * (long long)T + t0;
@@ -695,16 +717,14 @@ __global__ void __launch_bounds__(256) gate_transpose_kernel(const __nv_bfloat16
 cudaError_t launch_transpose_btc(const void* x, void* xT, long long B, int T, int C, cudaStream_t st) {
     if (T % 64 != 0 || C % 64 != 0) return cudaErrorInvalidValue;
     if (B == 0) return cudaSuccess;
-    transpose_btc_kernel<<<dim3(T / 64, C / 64, (unsigned)B), 256, 0, st>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)xT, T, C);
-    return cudaGetLastError();
+    return launch_pdl(transpose_btc_kernel, dim3(T / 64, C / 64, (unsigned)B), dim3(256), st, (const __nv_bfloat16*)x, (__nv_bfloat16*)xT, T, C);
 }
 
 cudaError_t launch_gate_transpose(const void* x, const void* vT, const float* w, void* z, long long B, int T, int C, cudaStream_t st) {
     if (T % 64 != 0 || C % 64 != 0) return cudaErrorInvalidValue;
     if (B == 0) return cudaSuccess;
-    gate_transpose_kernel<<<dim3(T / 64, C / 64, (unsigned)B), 256, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)vT, w,
-                                                                              (__nv_bfloat16*)z, T, C);
-    return cudaGetLastError();
+    return launch_pdl(gate_transpose_kernel, dim3(T / 64, C / 64, (unsigned)B), dim3(256), st, (const __nv_bfloat16*)x, (const __nv_bfloat16*)vT, w,
+                      (__nv_bfloat16*)z, T, C);
 }
 
 // conj of a spectrum buffer: `pairs` interleaved complex values (re, im), then `quads` values of the tensor-core
@@ -1069,6 +1089,7 @@ __device__ __forceinline__ uint4 f32_to_bf16x8(const float* f) {
 
 __global__ void __launch_bounds__(256) heads_outer_bf16x8_kernel(const uint4* __restrict__ X2, const uint4* __restrict__ V, uint4* __restrict__ XV,
                                                                  int d, int dh, int n8, long long total) {
+    pdl_prologue();
     const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n8
     if (e >= total) return;
     const int t8 = (int)(e % n8);
@@ -1087,6 +1108,7 @@ __global__ void __launch_bounds__(256) heads_outer_bf16x8_kernel(const uint4* __
 
 __global__ void __launch_bounds__(256) heads_reduce_bf16x8_kernel(const uint4* __restrict__ X1, const uint4* __restrict__ XVc, uint4* __restrict__ O,
                                                                   int d, int dh, int n8, long long total) {
+    pdl_prologue();
     const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n8
     if (e >= total) return;
     const int t8 = (int)(e % n8);
@@ -1108,8 +1130,8 @@ cudaError_t launch_heads_outer(const void* X2, const void* V, void* XV, long lon
     if (total == 0) return cudaSuccess;
     if (bf16 && n % 8 == 0) {
         const long long t8 = B * d * (n / 8);
-        heads_outer_bf16x8_kernel<<<(unsigned)((t8 + 255) / 256), 256, 0, st>>>((const uint4*)X2, (const uint4*)V, (uint4*)XV, d, dh, n / 8, t8);
-        return cudaGetLastError();
+        return launch_pdl(heads_outer_bf16x8_kernel, dim3((unsigned)((t8 + 255) / 256)), dim3(256), st, (const uint4*)X2, (const uint4*)V, (uint4*)XV, d, dh,
+                          n / 8, t8);
     }
     const unsigned grid = (unsigned)((total + 255) / 256);
     if (bf16)
@@ -1124,8 +1146,8 @@ cudaError_t launch_heads_reduce(const void* X1, const void* XVc, void* O, long l
     if (total == 0) return cudaSuccess;
     if (bf16 && n % 8 == 0) {
         const long long t8 = B * d * (n / 8);
-        heads_reduce_bf16x8_kernel<<<(unsigned)((t8 + 255) / 256), 256, 0, st>>>((const uint4*)X1, (const uint4*)XVc, (uint4*)O, d, dh, n / 8, t8);
-        return cudaGetLastError();
+        return launch_pdl(heads_reduce_bf16x8_kernel, dim3((unsigned)((t8 + 255) / 256)), dim3(256), st, (const uint4*)X1, (const uint4*)XVc, (uint4*)O, d,
+                          dh, n / 8, t8);
     }
     const unsigned grid = (unsigned)((total + 255) / 256);
     if (bf16)
@@ -1196,6 +1218,7 @@ __device__ __forceinline__ void dw3_x8(const __nv_bfloat16* __restrict__ row, co
 __global__ void __launch_bounds__(256) gate_in_bf16x8_kernel(const __nv_bfloat16* __restrict__ Pq, const __nv_bfloat16* __restrict__ Pk,
                                                              const float* __restrict__ wq, const float* __restrict__ wk,
                                                              __nv_bfloat16* __restrict__ QK, int d, int n, long long total8) {
+    pdl_prologue();
     const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;   // over B * d * n / 8
     if (e >= total8) return;
     const int n8 = n / 8, t0 = (int)(e % n8) * 8;
@@ -1212,6 +1235,7 @@ __global__ void __launch_bounds__(256) gate_in_bf16x8_kernel(const __nv_bfloat16
 __global__ void __launch_bounds__(256) gate_out_bf16x8_kernel(const __nv_bfloat16* __restrict__ Pv, const float* __restrict__ wv,
                                                               const __nv_bfloat16* __restrict__ C, const __nv_bfloat16* __restrict__ Cr,
                                                               __nv_bfloat16* __restrict__ Z, int d, int n, long long total8) {
+    pdl_prologue();
     const long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (e >= total8) return;
     const int n8 = n / 8, t0 = (int)(e % n8) * 8;
@@ -1231,9 +1255,8 @@ cudaError_t launch_gate_in(const void* Pq, const void* Pk, const float* wq, cons
     const long long total = B * d * n;
     if (total == 0) return cudaSuccess;
     if (bf16 && n % 8 == 0) {
-        gate_in_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16*)Pq, (const __nv_bfloat16*)Pk, wq, wk,
-                                                                                  (__nv_bfloat16*)QK, d, n, total / 8);
-        return cudaGetLastError();
+        return launch_pdl(gate_in_bf16x8_kernel, dim3((unsigned)((total / 8 + 255) / 256)), dim3(256), st, (const __nv_bfloat16*)Pq,
+                          (const __nv_bfloat16*)Pk, wq, wk, (__nv_bfloat16*)QK, d, n, total / 8);
     }
     const unsigned grid = (unsigned)((total + 255) / 256);
     if (bf16)
@@ -1248,9 +1271,8 @@ cudaError_t launch_gate_out(const void* Pv, const float* wv, const void* C, cons
     const long long total = B * d * n;
     if (total == 0) return cudaSuccess;
     if (bf16 && n % 8 == 0) {
-        gate_out_bf16x8_kernel<<<(unsigned)((total / 8 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16*)Pv, wv, (const __nv_bfloat16*)C,
-                                                                                   (const __nv_bfloat16*)Cr, (__nv_bfloat16*)Z, d, n, total / 8);
-        return cudaGetLastError();
+        return launch_pdl(gate_out_bf16x8_kernel, dim3((unsigned)((total / 8 + 255) / 256)), dim3(256), st, (const __nv_bfloat16*)Pv, wv,
+                          (const __nv_bfloat16*)C, (const __nv_bfloat16*)Cr, (__nv_bfloat16*)Z, d, n, total / 8);
     }
     const unsigned grid = (unsigned)((total + 255) / 256);
     if (bf16)

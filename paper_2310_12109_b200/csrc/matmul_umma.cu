@@ -5,10 +5,14 @@
 // Both block-diagonal factors are batches of 64 independent GEMMs [tokens x 64] x [64 x 64]; the batch
 // index is the CONTIGUOUS index of the data each factor reads (n2 for R, k1 for L after the middle
 // permutation), so neither operand of a tensor-core GEMM can be taken from memory as it lies.  The two
-// factors therefore run as two passes of one kernel that exchange the intermediate through a workspace
-// laid out in 16 KB blocks z[token tile][n2 / 8][k1][t % 128][n2 % 8] (it mostly stays in the 126 MB L2): what the
-// pass-1 CTA (token tile, n2 group) writes is one contiguous 128 KB slab, and what the pass-2 CTA (token tile, k1
-// group) reads are eight contiguous 16 KB pieces of eight such slabs:
+// factors therefore run as two passes that exchange the intermediate through a caller workspace.  Two
+// generations of pass kernels live in this file:
+//
+//   monarch64_fwd_kernel<1|2>   the forward path (further down): 32 tokens x 16 blocks per item, 32-byte pieces,
+//                               weights resident, loading / draining / issuing warps.
+//   monarch64_pass_kernel<1|2>  128 tokens x 8 blocks per CTA, 16-byte pieces (described next): serves inputs that are
+//                               only 16-byte aligned, and the weight gradients, whose kernel reads its workspace layout
+//                               z[token tile][n2 / 8][k1][t % 128][n2 % 8]:
 //
 //   pass 1 (R): a CTA owns 128 tokens x 8 consecutive n2.  Threads read 16-byte pieces of x (8 values of
 //               n2 for one (t, n1)), transpose 8 x 8 blocks in registers (the permutation P) and write the

@@ -3,14 +3,20 @@
 // for blocks of 192 inputs / 768 hidden / 192 outputs (d = 768, 4 blocks, expansion 4).  bf16 operands, fp32
 // accumulation in TMEM, the hidden activations are rounded to bf16 and never leave the SM.
 //
-// One CTA = 128 tokens x one block.  The hidden dimension is walked in 6 chunks of 128:
+// An item = 128 tokens x one block.  The hidden dimension is walked in 6 chunks of 128:
 //   S1(c)  D1[c % 2][128 tok][128 hid] = Z[128][192] * W_up[j][chunk c]^T        12 UMMAs (M128 N128 K16)
-//   E1(c)  TMEM -> registers -> GELU -> bf16 -> G[128 tok][128 hid] (UMMA operand, shared memory)
-//   S2(c)  D2[128 tok][192 out] += G * W_down[j][:, chunk c]^T                     8 UMMAs (M128 N192 K16)
-// and at the end D2 -> bf16 -> staging -> TMA store.  Warp roles: warp 0 feeds the weight chunks by TMA (W_up
-// chunks double-buffered), warp 1 issues the UMMAs and runs S1(c + 1) ahead of E1(c) (two D1 buffers), warps 2..17
-// are the GELU warps (lane quarter = warp % 4, 32 of the 128 chunk columns each).  All operands are K-major with the
-// 128-byte swizzle, written by TMA (Z, weights) or by the GELU warps (G).  Every wait is bounded.
+//   E1(c)  TMEM -> registers -> GELU -> bf16 -> back into TMEM, over the first 64 columns of the D1 buffer it came from
+//          (two values per column): G[128 tok][128 hid] is the A operand of S2 and never touches shared memory
+//   S2(c)  D2[128 tok][192 out] += G * W_down[j][:, chunk c]^T                     8 UMMAs (M128 N192 K16, A from TMEM)
+// and at the end of an item D2 -> bf16 -> staging -> TMA stores.
+//
+// Persistent: one CTA per SM walks the items c, c + grid, ..; all barriers count chunks across items, so the weight
+// chunks, the activations and the first UMMAs of the next item are under way while the GELU warps finish and store the
+// current one (a CTA per item spent a third of its time launching, setting up and draining).  Warp roles: warp 0 feeds
+// the activation tiles and the weight chunks by TMA (W_up chunks double-buffered), warp 1 issues the UMMAs and runs
+// S1(c + 1) ahead of E1(c) (two D1 buffers), warps 2..17 are the GELU warps (lane quarter = warp % 4, 32 of the 128
+// chunk columns each).  Shared-memory operands are K-major with the 128-byte swizzle, written by TMA.  Every wait is
+// bounded; a role that gave up keeps arriving at the GELU warps' block barriers so that nobody is left behind.
 #include <cuda.h>
 
 #include <atomic>
@@ -26,15 +32,15 @@ using namespace sm100;
 
 constexpr int kCI = 192, kHID = 768, kCO = 192, kChunk = 128, kChunks = kHID / kChunk, kTileT = 128;
 constexpr int kEpiWarps = 16, kThreads = 64 + 32 * kEpiWarps;
-constexpr int OFF_Z = 0;                    // 3 K-blocks [128][64] bf16 (also the output staging)   49152
+constexpr int OFF_Z = 0;                    // 3 K-blocks [128][64] bf16                               49152
 constexpr int OFF_W1 = 49152;               // 2 buffers x 3 K-blocks [128 hid][64]                   98304
 constexpr int OFF_W2 = 147456;              // 2 K-blocks [192 out][64]                               49152
-constexpr int OFF_G = 196608;               // 2 K-blocks [128 tok][64]                               32768
+constexpr int OFF_ST = 196608;              // output staging: 2 buffers [128 tok][64]                32768
 constexpr int OFF_BAR = 229376;
 constexpr int SMEM_BYTES = OFF_BAR + 192;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 // mbarriers (8 bytes each) from OFF_BAR
-enum { B_Z = 0, B_W1F = 1, B_W1E = 3, B_W2F = 5, B_W2E = 6, B_D1F = 7, B_D1E = 9, B_GF = 11, B_GE = 12, B_D2F = 13, B_COUNT = 14 };
+enum { B_Z = 0, B_W1F = 1, B_W1E = 3, B_W2F = 5, B_W2E = 6, B_D1F = 7, B_D1E = 9, B_GF = 11, B_ZE = 12, B_D2F = 13, B_D2E = 14, B_COUNT = 15 };
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
@@ -77,17 +83,22 @@ __device__ __forceinline__ uint32_t sw_off(int r, int kc) { return (uint32_t)((r
 
 __global__ void __launch_bounds__(kThreads, 1)
 mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_w1,
-                const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_y, int32_t* __restrict__ status) {
+                const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_y, int32_t* __restrict__ status,
+                int nblk, int nitems) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
     const uint32_t bars = s_base + OFF_BAR, s_tptr = s_base + OFF_BAR + 8 * B_COUNT;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
-    const int j = blockIdx.y;                      // block of the block-diagonal factors
-    const int t0 = blockIdx.x * kTileT;            // first token of the tile
+    // this CTA's items: item(q) = blockIdx.x + q * gridDim.x  ->  block j = item % nblk, token tile = item / nblk
+    const int nq = ((int)blockIdx.x < nitems) ? (nitems - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total = nq * kChunks;                // chunks of all items, counted through by every role
+    auto item_j = [&](int q) { return (int)((blockIdx.x + (unsigned)q * gridDim.x) % (unsigned)nblk); };
+    auto item_t0 = [&](int q) { return (int)((blockIdx.x + (unsigned)q * gridDim.x) / (unsigned)nblk) * kTileT; };
 
     if (tid == 0) {
         mbar_init(bar(B_Z), 1);
+        mbar_init(bar(B_ZE), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar(B_W1F + i), 1);
             mbar_init(bar(B_W1E + i), 1);
@@ -97,8 +108,8 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
         mbar_init(bar(B_W2F), 1);
         mbar_init(bar(B_W2E), 1);
         mbar_init(bar(B_GF), kEpiWarps);
-        mbar_init(bar(B_GE), 1);
         mbar_init(bar(B_D2F), 1);
+        mbar_init(bar(B_D2E), kEpiWarps);
         fence_barrier_init();
         prefetch_tensormap(&map_z);
         prefetch_tensormap(&map_w1);
@@ -116,43 +127,48 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     bool ok = true;
 
     if (warp == 0) {
-        // ---- TMA producer ------------------------------------------------------------------------------------------
+        // ---- TMA producer: three streams that advance independently (activation tiles, W_up chunks two ahead of the
+        //      UMMAs, the single W_down buffer as soon as S2 has read it), so none waits behind another's barrier ----
         if (lane == 0) {
-            mbar_expect_tx(bar(B_Z), 49152);
-            for (int kb = 0; kb < 3; ++kb) tma_load_2d(s_base + OFF_Z + kb * 16384, &map_z, j * kCI + kb * 64, t0, bar(B_Z));
-            // The two weight streams advance independently (a W_up chunk two ahead of the UMMAs, the single W_down
-            // buffer as soon as S2 has read it), so neither waits behind the other's barrier.
-            int c1 = 0, c2 = 0;
+            int zq = 0, g1 = 0, g2 = 0;
             uint32_t idle = 0;
-            while ((c1 < kChunks || c2 < kChunks) && idle < (1u << 22)) {
+            while ((zq < nq || g1 < total || g2 < total) && idle < (1u << 22)) {
                 bool progressed = false;
-                if (c1 < kChunks && (c1 < 2 || mbar_try_wait(bar(B_W1E + (c1 & 1)), ((c1 >> 1) - 1) & 1))) {   // S1(c1 - 2) has read the buffer
-                    const int bb = c1 & 1;
-                    mbar_expect_tx(bar(B_W1F + bb), 49152);
+                if (zq < nq && (zq < 1 || mbar_try_wait(bar(B_ZE), (zq - 1) & 1))) {                                  // the last S1 of item zq - 1 has read Z
+                    mbar_expect_tx(bar(B_Z), 49152);
                     for (int kb = 0; kb < 3; ++kb)
-                        tma_load_2d(s_base + OFF_W1 + bb * 49152 + kb * 16384, &map_w1, kb * 64, j * kHID + c1 * kChunk, bar(B_W1F + bb));
-                    ++c1;
+                        tma_load_2d(s_base + OFF_Z + kb * 16384, &map_z, item_j(zq) * kCI + kb * 64, item_t0(zq), bar(B_Z));
+                    ++zq;
                     progressed = true;
                 }
-                if (c2 < kChunks && (c2 < 1 || mbar_try_wait(bar(B_W2E), (c2 - 1) & 1))) {                        // S2(c2 - 1) has read the chunk
+                if (g1 < total && (g1 < 2 || mbar_try_wait(bar(B_W1E + (g1 & 1)), ((g1 >> 1) - 1) & 1))) {            // S1(g1 - 2) has read the buffer
+                    const int bb = g1 & 1, c = g1 % kChunks, jj = item_j(g1 / kChunks);
+                    mbar_expect_tx(bar(B_W1F + bb), 49152);
+                    for (int kb = 0; kb < 3; ++kb)
+                        tma_load_2d(s_base + OFF_W1 + bb * 49152 + kb * 16384, &map_w1, kb * 64, jj * kHID + c * kChunk, bar(B_W1F + bb));
+                    ++g1;
+                    progressed = true;
+                }
+                if (g2 < total && (g2 < 1 || mbar_try_wait(bar(B_W2E), (g2 - 1) & 1))) {                               // S2(g2 - 1) has read the chunk
+                    const int c = g2 % kChunks, jj = item_j(g2 / kChunks);
                     mbar_expect_tx(bar(B_W2F), 49152);
                     for (int kb = 0; kb < 2; ++kb)
-                        tma_load_2d(s_base + OFF_W2 + kb * 24576, &map_w2, c2 * kChunk + kb * 64, j * kCO, bar(B_W2F));
-                    ++c2;
+                        tma_load_2d(s_base + OFF_W2 + kb * 24576, &map_w2, c * kChunk + kb * 64, jj * kCO, bar(B_W2F));
+                    ++g2;
                     progressed = true;
                 }
                 idle = progressed ? 0 : idle + 1;
             }
-            if (c1 < kChunks || c2 < kChunks) ok = false;
+            if (zq < nq || g1 < total || g2 < total) ok = false;
         }
     } else if (warp == 1) {
         // ---- UMMA issuer ---------------------------------------------------------------------------------------------
         if (lane == 0) {
             constexpr uint32_t ID1 = instr_desc_bf16(128, 128, false, false), ID2 = instr_desc_bf16(128, 192, false, false);
-            auto s1 = [&](int c) {   // D1[c % 2] = Z * W_up chunk c
-                const int b = c & 1;
-                ok = mbar_wait(bar(B_W1F + b), (c >> 1) & 1);
-                if (ok && c >= 2) ok = mbar_wait(bar(B_D1E + b), ((c >> 1) - 1) & 1);   // the GELU warps have read D1[b]
+            auto s1 = [&](int g) {   // D1[g % 2] = Z * W_up chunk g
+                const int b = g & 1;
+                ok = mbar_wait(bar(B_W1F + b), (g >> 1) & 1);
+                if (ok && g >= 2) ok = mbar_wait(bar(B_D1E + b), ((g >> 1) - 1) & 1);   // the GELU warps have read D1[b]
                 if (!ok) return;
                 tc_fence_after();
 #pragma unroll 1
@@ -163,89 +179,130 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                                  smem_desc_sw128(s_base + OFF_W1 + b * 49152 + kb * 16384 + s * 32, 16, 1024), ID1, (kb | s) != 0);
                 umma_commit(bar(B_D1F + b));
                 umma_commit(bar(B_W1E + b));
+                if (g % kChunks == kChunks - 1) umma_commit(bar(B_ZE));   // the item's last S1: its activation tile is free after it
             };
-            ok = mbar_wait(bar(B_Z), 0);
-            if (ok) s1(0);
-            for (int c = 0; c < kChunks && ok; ++c) {
-                if (c + 1 < kChunks) s1(c + 1);
+            if (total > 0) {
+                ok = mbar_wait(bar(B_Z), 0);
+                if (ok) s1(0);
+            }
+            for (int g = 0; g < total && ok; ++g) {
+                const int c = g % kChunks, q = g / kChunks;
+                if (c + 1 < kChunks) s1(g + 1);
                 if (!ok) break;
-                ok = mbar_wait(bar(B_GF), c & 1) && mbar_wait(bar(B_W2F), c & 1);
+                ok = mbar_wait(bar(B_GF), g & 1) && mbar_wait(bar(B_W2F), g & 1);
+                if (ok && c == 0 && q > 0) ok = mbar_wait(bar(B_D2E), (q - 1) & 1);   // the previous item's D2 has been read
                 if (!ok) break;
                 tc_fence_after();
+                // A = G in tensor memory: the first 64 columns of D1[g % 2], 8 columns per K step of 16
 #pragma unroll 1
                 for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
                     for (int s = 0; s < 4; ++s)
-                        umma_f16(D2, smem_desc_sw128(s_base + OFF_G + kb * 16384 + s * 32, 16, 1024),
-                                 smem_desc_sw128(s_base + OFF_W2 + kb * 24576 + s * 32, 16, 1024), ID2, (c | kb | s) != 0);
-                umma_commit(bar(B_GE));
+                        umma_f16_ta(D2, D1 + (g & 1) * 128 + (kb * 4 + s) * 8,
+                                    smem_desc_sw128(s_base + OFF_W2 + kb * 24576 + s * 32, 16, 1024), ID2, (c | kb | s) != 0);
                 umma_commit(bar(B_W2E));
-                if (c == kChunks - 1) umma_commit(bar(B_D2F));
+                if (c == kChunks - 1) {
+                    umma_commit(bar(B_D2F));
+                    if (g + 1 < total) {   // the next item's first S1 follows this item's last S2
+                        ok = mbar_wait(bar(B_Z), (q + 1) & 1);
+                        if (ok) s1(g + 1);
+                    }
+                }
             }
         }
     } else {
-        // ---- GELU warps: lane quarter q = warp % 4 (a TMEM rule), column slice sl = 32 of the chunk's 128 columns ----
-        const int ew = warp - 2, q = warp & 3, sl = ew >> 2;
-        const int row = q * 32 + lane;                                   // token within the tile
-        const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
-        for (int c = 0; c < kChunks && ok; ++c) {
-            const int b = c & 1;
-            ok = mbar_wait(bar(B_D1F + b), (c >> 1) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            float v[32];
+        // ---- GELU warps: lane quarter qq = warp % 4 (a TMEM rule), column slice sl = 32 of the chunk's 128 columns ----
+        const int ew = warp - 2, qq = warp & 3, sl = ew >> 2;
+        const int row = qq * 32 + lane;                                   // token within the tile
+        const uint32_t t_lane = tmem + ((uint32_t)(qq * 32) << 16);
+        const bool storer = ew == 0 && lane == 0;                         // issues the output stores
+        for (int g = 0; g < total; ++g) {
+            const int b = g & 1, c = g % kChunks, q = g / kChunks;
+            if (ok) ok = mbar_wait(bar(B_D1F + b), (g >> 1) & 1);
+            if (ok) {
+                tc_fence_after();
+                float v[32];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) tmem_ld8(t_lane + b * 128 + sl * 32 + 8 * i, v + 8 * i);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 4; ++i) tmem_ld_fence8(v + 8 * i);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_D1E + b));                  // this warp has read its part of D1[b]
-            uint4 pk[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                pk[i] = make_uint4(gelu2_pack(v[8 * i], v[8 * i + 1]), gelu2_pack(v[8 * i + 2], v[8 * i + 3]),
-                                   gelu2_pack(v[8 * i + 4], v[8 * i + 5]), gelu2_pack(v[8 * i + 6], v[8 * i + 7]));
-            if (c >= 1) ok = mbar_wait(bar(B_GE), (c - 1) & 1);          // S2(c - 1) has read G
-            if (!ok) break;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int kc = sl * 4 + i;                               // 16-byte chunk of the 128-column row
-                *reinterpret_cast<uint4*>(smem + OFF_G + (kc >> 3) * 16384 + sw_off(row, kc & 7)) = pk[i];
-            }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(B_GF));
-        }
-        // ---- output: D2 -> bf16 -> staging (the Z buffer, free since the last S1) -> TMA store ---------------------
-        if (ok) ok = mbar_wait(bar(B_D2F), 0);
-        if (ok) {
-            tc_fence_after();
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {                                // 48 of the 192 output columns per slice: 6 chunks
-                float w[24];
-#pragma unroll
-                for (int i = 0; i < 3; ++i) tmem_ld8(t_lane + 256 + sl * 48 + h * 24 + 8 * i, w + 8 * i);
+                for (int i = 0; i < 4; ++i) tmem_ld8(t_lane + b * 128 + sl * 32 + 8 * i, v + 8 * i);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 3; ++i) tmem_ld_fence8(w + 8 * i);
+                for (int i = 0; i < 4; ++i) tmem_ld_fence8(v + 8 * i);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_D1E + b));                  // this warp has read its part of D1[b]
+                uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 3; ++i) {
-                    const int kc = sl * 6 + h * 3 + i;                   // 16-byte chunk of the 192-column row: 24 of them
-                    *reinterpret_cast<uint4*>(smem + OFF_Z + (kc >> 3) * 16384 + sw_off(row, kc & 7)) =
-                        make_uint4(pack_bf16(w[8 * i], w[8 * i + 1]), pack_bf16(w[8 * i + 2], w[8 * i + 3]),
-                                   pack_bf16(w[8 * i + 4], w[8 * i + 5]), pack_bf16(w[8 * i + 6], w[8 * i + 7]));
+                for (int i = 0; i < 16; ++i) pk[i] = gelu2_pack(v[2 * i], v[2 * i + 1]);
+                // G goes back into tensor memory over the first 64 columns of D1[b]: every GELU warp must have read the buffer
+                ok = mbar_wait(bar(B_D1E + b), (g >> 1) & 1);
+                if (ok) {
+                    tc_fence_after();
+                    tmem_st8(t_lane + b * 128 + sl * 16, pk);
+                    tmem_st8(t_lane + b * 128 + sl * 16 + 8, pk + 8);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(B_GF));
                 }
             }
-            fence_proxy_async();
+            if (c != kChunks - 1) continue;
+            // ---- output of item q: D2 -> bf16 -> staging -> TMA stores.  The 24 chunks (16 bytes) of a 192-column row
+            //      belong to three K-blocks of 64 columns; K-blocks 0 and 1 are staged in the two 16 KB buffers and sent,
+            //      K-block 2 follows in the first buffer once its store has read it.  The block barriers are passed by
+            //      every GELU warp whatever happened before. ----
+            if (ok) ok = mbar_wait(bar(B_D2F), q & 1);
+            uint4 keep[6];
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {                                // 48 of the 192 output columns per slice: 6 chunks
+                    float w[24];
+#pragma unroll
+                    for (int i = 0; i < 3; ++i) tmem_ld8(t_lane + 256 + sl * 48 + h * 24 + 8 * i, w + 8 * i);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 3; ++i) tmem_ld_fence8(w + 8 * i);
+#pragma unroll
+                    for (int i = 0; i < 3; ++i)
+                        keep[h * 3 + i] = make_uint4(pack_bf16(w[8 * i], w[8 * i + 1]), pack_bf16(w[8 * i + 2], w[8 * i + 3]),
+                                                     pack_bf16(w[8 * i + 4], w[8 * i + 5]), pack_bf16(w[8 * i + 6], w[8 * i + 7]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_D2E));                      // D2 may be overwritten by the next item
+            }
+            if (storer) tma_store_wait_read0();                              // the previous item's stores have read the staging buffers
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+            if (ok) {
+#pragma unroll
+                for (int i = 0; i < 6; ++i) {
+                    const int kc = sl * 6 + i;                               // 16-byte chunk of the 192-column row
+                    if (kc < 16) *reinterpret_cast<uint4*>(smem + OFF_ST + (kc >> 3) * 16384 + sw_off(row, kc & 7)) = keep[i];
+                }
+                fence_proxy_async();
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+            if (storer && ok) {
+                for (int kb = 0; kb < 2; ++kb) tma_store_2d(&map_y, s_base + OFF_ST + kb * 16384, item_j(q) * kCO + kb * 64, item_t0(q));
+                tma_store_commit();
+                tma_store_wait_read0();
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+            if (ok) {
+#pragma unroll
+                for (int i = 0; i < 6; ++i) {
+                    const int kc = sl * 6 + i;
+                    if (kc >= 16) *reinterpret_cast<uint4*>(smem + OFF_ST + sw_off(row, kc & 7)) = keep[i];
+                }
+                fence_proxy_async();
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+            if (storer && ok) {
+                tma_store_2d(&map_y, s_base + OFF_ST, item_j(q) * kCO + 128, item_t0(q));
+                tma_store_commit();
+            }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
-        if (ok && ew == 0 && lane == 0) {
-            for (int kb = 0; kb < 3; ++kb) tma_store_2d(&map_y, s_base + OFF_Z + kb * 16384, j * kCO + kb * 64, t0);
-            tma_store_commit();
-            tma_store_wait_all0();
-        }
+        if (storer) tma_store_wait_all0();                                   // complete before shared memory goes away
     }
     if (!ok) atomicExch(status, (int32_t)M2_ERR_TIMEOUT);
     tc_fence_before();
@@ -260,6 +317,7 @@ cudaError_t prepare() { return cudaFuncSetAttribute(mlp_umma_kernel, cudaFuncAtt
 int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, long long tokens, int32_t* status,
                cudaStream_t stream) {
     if (tokens == 0) return M2_OK;
+    int dev_id = 0;
     {   // the shared-memory opt-in is per device (setting it twice is harmless; the flag itself is race-free)
         static std::atomic<bool> prepared[64];
         int dev = 0;
@@ -268,6 +326,7 @@ int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, 
             if (prepare() != cudaSuccess) return M2_ERR_CUDA;
             prepared[dev].store(true, std::memory_order_release);
         }
+        dev_id = dev;
     }
     alignas(64) CUtensorMap mz, mw1, mw2, my;
     {   // activations [tokens][C]: box = 64 columns x 128 tokens, 128B swizzle (rows past the end: zero-filled / clipped)
@@ -285,7 +344,10 @@ int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, 
             return M2_ERR_UNSUPPORTED;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((tokens + kTileT - 1) / kTileT), (unsigned)nblk);
+    const long long nitems = ((tokens + kTileT - 1) / kTileT) * nblk;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev_id) != cudaSuccess || sms < 1 || nitems > 0x7fffffffLL) return M2_ERR_CUDA;
+    cfg.gridDim = dim3((unsigned)(nitems < sms ? nitems : sms));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = stream;
@@ -294,7 +356,7 @@ int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, mlp_umma_kernel, mz, mw1, mw2, my, status) != cudaSuccess) return M2_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, mlp_umma_kernel, mz, mw1, mw2, my, status, nblk, (int)nitems) != cudaSuccess) return M2_ERR_CUDA;
     return M2_OK;
 }
 

@@ -33,33 +33,34 @@ inline bool encode_bf16(CUtensorMap* map, const void* ptr, int rank, const cuuin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// same with the 128-byte swizzle (inner box extent must be 128 bytes)
+// same with the 128-byte swizzle.  The inner box extent must be exactly the swizzle span (refused otherwise): the copy engine
+// pads a narrower inner row to the span, so the box would take more shared memory than its element count says.
 inline bool encode_sw128_bf16(CUtensorMap* map, const void* ptr, int rank, const cuuint64_t* gdim, const cuuint64_t* gstr,
                               const cuuint32_t* box) {
     EncodeTiledFn enc = encode_fn();
-    if (!enc) return false;
+    if (!enc || box[0] * 2 != 128) return false;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), gdim, gstr, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// same with the 64-byte swizzle (inner box extent must be 64 bytes): 16-byte chunk index XOR bits 7..8 of the address
+// same with the 64-byte swizzle (inner box extent exactly 64 bytes, see above): 16-byte chunk index XOR bits 7..8 of the address
 inline bool encode_sw64_bf16(CUtensorMap* map, const void* ptr, int rank, const cuuint64_t* gdim, const cuuint64_t* gstr,
                              const cuuint32_t* box) {
     EncodeTiledFn enc = encode_fn();
-    if (!enc) return false;
+    if (!enc || box[0] * 2 != 64) return false;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), gdim, gstr, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// same with the 32-byte swizzle (inner box extent must be 32 bytes): 16-byte chunk index XOR bit 7 of the address
+// same with the 32-byte swizzle (inner box extent exactly 32 bytes, see above): 16-byte chunk index XOR bit 7 of the address
 inline bool encode_sw32_bf16(CUtensorMap* map, const void* ptr, int rank, const cuuint64_t* gdim, const cuuint64_t* gstr,
                              const cuuint32_t* box) {
     EncodeTiledFn enc = encode_fn();
-    if (!enc) return false;
+    if (!enc || box[0] * 2 != 32) return false;
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), gdim, gstr, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,

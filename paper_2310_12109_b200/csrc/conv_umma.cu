@@ -510,7 +510,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     constexpr uint32_t ID_S1 = instr_desc_bf16(128, 64, true, false);
     constexpr uint32_t ID_S2 = instr_desc_bf16(128, 32, true, false);
     constexpr uint32_t ID_S2I = instr_desc_bf16(128, 32, false, false);
-    constexpr uint32_t ID_S1I = instr_desc_bf16(128, 64, true, false);
+    constexpr uint32_t ID_S1I = instr_desc_bf16(64, 64, false, true);
     const int n1_valid = n / 16;
     const int k1steps = (n1_valid + 15) / 16;   // causal input: digits n1 >= n/16 are zero -> skipped
 
@@ -696,40 +696,42 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ---- S1' --------------------------------------------------------------------------------
         if (leader) {
             tc_fence_after();
+            // the conjugated F_32 image is the A operand here (M = (re | im) x n1 = 64) and the data the B operand (N = 4 rows x 16 n2),
+            // so that a thread of the last hand-off owns whole 32-byte runs of the output; the second half of the rows goes to
+            // lanes 16..31 of every lane quarter (an M = 64 accumulator keeps row m in lane m % 16 + 32 (m / 16))
 #pragma unroll
-            for (int s = 0; s < 4; ++s)
-                umma_f16(tmem + T2, smem_desc(s_base + P_G_A + s * 256, 128, 1024),
-                         smem_desc(s_all + P_OFF_B4 + s * 256, 128, 1024), ID_S1I, s > 0);
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    umma_f16(tmem + T2 + ((uint32_t)(16 * hf) << 16), smem_desc(s_all + P_OFF_B4 + s * 256, 128, 1024),
+                             smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 1024), ID_S1I, s > 0);
             umma_commit(bar_mma);
         }
-        // ---- h4: round and stage: lane (r, n2) holds y[r][n1*16 + n2] for all n1 of the real-part row and of the
-        //      imaginary-part row; the operand buffer (free now) takes the two boxes [8 rows][32 n1][16 n2] in the
-        //      32-byte-swizzled image of the TMA stores (16-byte chunk XOR bit 7 of the address) ---------------
+        // ---- h4: round and stage: a lane holds, for one n1 of the real-part rows or of the imaginary-part rows, the 16 n2 of
+        //      four rows: 32-byte runs of y[r][n1*16 + n2].  The operand buffer (free now) takes the two boxes
+        //      [8 rows][32 n1][16 n2] in the 32-byte-swizzled image of the TMA stores (16-byte chunk XOR bit 7 of the address):
+        //      a quarter-warp's eight 16-byte stores fall into eight different bank groups ---------------
         ok = mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
         if (ok) {
-            const int r = tid >> 4, n2 = tid & 15;
+            // lane l of warp w holds output row m = 16 w + l % 16 = (c, n1) for the rows r = 4 (l / 16) .. + 3: 16 n2 per row
+            const int m = 16 * warp + (tid & 15), c = m >> 5, n1 = m & 31, rh = (tid >> 4) & 1;
+            unsigned char* st = smem + P_G_A + c * 8192 + (4 * rh) * 1024 + n1 * 32;
+            const int sw = (n1 >> 2) & 1;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {   // real part: row b0 + r; imaginary part: row b0 + 8 + r
+            for (int g = 0; g < 2; ++g) {   // two rows at a time
                 float v[32];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) tmem_ld8(t_lane + T2 + 32 * c + 8 * g, v + 8 * g);
+                for (int q = 0; q < 4; ++q) tmem_ld8(t_lane + T2 + 32 * g + 8 * q, v + 8 * q);
                 tmem_ld_wait();
 #pragma unroll
-                for (int g = 0; g < 4; ++g) tmem_ld_fence8(v + 8 * g);
-                // Neighbouring lanes hold neighbouring n2: the even lane collects the pair (n2, n2 + 1) of row n1 = 2j, the odd lane
-                // the pair of row 2j + 1 -- one word exchange per two values -- so the staging stores are whole 32-bit words.
-                const int odd = n2 & 1;
-                unsigned char* st = smem + P_G_A + c * 8192 + r * 1024 + odd * 32 + ((n2 & 7) >> 1) * 4;
+                for (int q = 0; q < 4; ++q) tmem_ld_fence8(v + 8 * q);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const uint32_t mine = pack_bf16(v[2 * j], v[2 * j + 1]);           // (row 2j, row 2j+1) of this lane's n2
-                    const uint32_t theirs = __shfl_xor_sync(0xffffffffu, mine, 1);
-                    // even lane: (own row 2j, partner row 2j); odd lane: (partner row 2j+1, own row 2j+1)
-                    const uint32_t w = odd ? __byte_perm(theirs, mine, 0x7632) : __byte_perm(mine, theirs, 0x5410);
-                    const int i = 2 * j + odd;
-                    *reinterpret_cast<uint32_t*>(st + (2 * j) * 32 + (((n2 >> 3) ^ ((i >> 2) & 1)) << 4)) = w;
+                for (int q = 0; q < 4; ++q) {   // q = (row, half of the n2 range): one 16-byte chunk of the row's 32-byte run
+                    const uint4 pk = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                                                pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+                    *reinterpret_cast<uint4*>(st + (2 * g + (q >> 1)) * 1024 + (((q & 1) ^ sw) << 4)) = pk;
                 }
             }
         }

@@ -299,6 +299,10 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                              smem_desc(s_base + OFF_BF + s * 256, 128, 1024), ID_MM, s > 0);
             umma_commit(bar_mma);
         }
+        // (the first factor of hand-off 2 comes from L2: the first tile's is asked for before the wait for the UMMAs, the second
+        // tile's while the first is worked on; tile wg + 4 has the same k1 and n3 larger by 16)
+        const float2* tn_h2 = tn + (((wg >> 1) << 3) + ((t >> 3) & 7)) * 32 + ((2 * (wg & 1) + (t >> 6)) << 3) + (t & 7);
+        float2 f0_next = __ldg(tn_h2);
         M2_WAIT_MMA()
         // ---- h2: w_N^{n3 (k1 + 32 k2)} = w_N^{n3 k1} (w_1024^{n3})^{k2}; A3[(k1, k2)][(c, n3)] --------------------
         if (ok) {
@@ -306,9 +310,11 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
             for (int jj = 0; jj < 2; ++jj) {
                 const int j = wg + 4 * jj;
                 const int k1 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), n3 = ((j >> 1) << 3) + ((t >> 3) & 7);
+                const float2 f0 = f0_next;
+                if (jj == 0) f0_next = __ldg(tn_h2 + 16 * 32);
                 float re[32], im[32];
                 load_tile(t_lane + j * 64, re, im);
-                const float2 f0 = __ldg(tn + n3 * 32 + k1), rho = tw_at(n3, 1);
+                const float2 rho = tw_at(n3, 1);
 #pragma unroll
                 for (int hi = 0; hi < 4; ++hi) {
                     uint4 pr, pi;
@@ -395,6 +401,12 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
                              smem_desc(s_base + OFF_BI + s * 256, 128, 1024), ID_KM, s > 0);
             umma_commit(bar_mma);
         }
+        // (hand-off 4's factors w_N^{m k1}, m = 1, 8, 16, 24: the same way; tile wg + 4 has k1 larger by 16)
+        const float2* tn_h4 = tn + ((wg >> 1) << 3) + ((t >> 3) & 7);
+        float2 g_next[4];
+        g_next[0] = __ldg(tn_h4 + 32);
+#pragma unroll
+        for (int hi = 1; hi < 4; ++hi) g_next[hi] = __ldg(tn_h4 + 8 * hi * 32);
         M2_WAIT_MMA()
         // ---- h4: conj w_N^{n3 (k1 + 32 k2)}; A5[(k1, n3)][(c, k2)] -----------------------------------------------------
         if (ok) {
@@ -402,14 +414,22 @@ conv32k_kernel(const __grid_constant__ CUtensorMap map_y, const __nv_bfloat16* _
             for (int jj = 0; jj < 2; ++jj) {
                 const int j = wg + 4 * jj;
                 const int k2 = ((2 * (j & 1) + (t >> 6)) << 3) + (t & 7), k1 = ((j >> 1) << 3) + ((t >> 3) & 7);
+                float2 g[4];
+#pragma unroll
+                for (int hi = 0; hi < 4; ++hi) g[hi] = g_next[hi];
+                if (jj == 0) {
+                    g_next[0] = __ldg(tn_h4 + 16 + 32);
+#pragma unroll
+                    for (int hi = 1; hi < 4; ++hi) g_next[hi] = __ldg(tn_h4 + 16 + 8 * hi * 32);
+                }
                 float re[32], im[32];
                 load_tile(t_lane + j * 64, re, im);
                 // rho^m = conj( w_N^{m k1} w_1024^{m k2} )
-                const float2 rho = conjf(cmul(__ldg(tn + 1 * 32 + k1), tw_at(1, k2)));
+                const float2 rho = conjf(cmul(g[0], tw_at(1, k2)));
 #pragma unroll
                 for (int hi = 0; hi < 4; ++hi) {
                     float2 f = make_float2(1.f, 0.f);
-                    if (hi > 0) f = conjf(cmul(__ldg(tn + 8 * hi * 32 + k1), tw_at(8 * hi, k2)));
+                    if (hi > 0) f = conjf(cmul(g[hi], tw_at(8 * hi, k2)));
                     uint4 pr, pi;
                     geometric8_pack(re + 8 * hi, im + 8 * hi, f, rho, pr, pi);
                     const int mb = (k1 >> 3) * 4 + hi;

@@ -426,7 +426,7 @@ def _side_config4(torch, M, synth, peaks, reps, bf):
 
 
 def _side_config5(torch, M, synth, peaks, reps, bf):
-    """M2 block forward [32, 512, 768]: sequence mix + gate + block-diagonal MLP (4 launches + the conv)."""
+    """M2 block forward [32, 512, 768]: sequence mix + gate + block-diagonal MLP (3 launches: transpose, gated conv, MLP)."""
     out = {}
     B, T, C = 32, 512, 768
     c = synth.config5(B=B, T=T, C=C)
@@ -443,7 +443,7 @@ def _side_config5(torch, M, synth, peaks, reps, bf):
     t_tc = fl / (peaks["bf16_tflops_sustained"] * 1e12)
     out["config5_block"] = {
         "kernel": plan.last_kernel(), "ms": ms, "tokens_ch_per_s": B * T * C / (ms * 1e-3), "mlp_TFLOPs_if_all_time_were_mlp": fl / (ms * 1e9),
-        "note": "whole block (transpose, conv, gate, MLP); roofline = the MLP's tensor time plus the conv's HBM time",
+        "note": "whole block (transpose, conv with the gate in its last hand-off, MLP); roofline = the MLP's tensor time plus the conv's HBM time",
         "roofline": {"bound": "tensor", "achieved": fl / (ms * 1e9), "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": (t_tc + by / (peaks["hbm_gbs"] * 1e9)) / (ms * 1e-3)}}
     plan.close()

@@ -281,9 +281,14 @@ int32_t m2_monarch_matmul_bwd_weights(const m2_plan* plan, const void* X_dev, co
  * (centred, zero padded); z = g (.) v; then the block-diagonal MLP y = bd(W_down) GELU(bd(W_up) z)
  * with nblk blocks (exact erf GELU).  x_dev, y_dev: [B, T, C] bf16 with T == N of the plan;
  * kf_dev: spectrum of k[C, T]; w_short_dev: [C, 3] float32; W_up_dev: [nblk, E*C/nblk, C/nblk] bf16;
- * W_down_dev: [nblk, C/nblk, E*C/nblk] bf16; z_dev: [B, T, C] bf16 scratch that receives z.  z_dev and y_dev
- * must not overlap x_dev or each other; both are also used as scratch while the call runs (y_dev holds the
- * convolution output before it receives y). */
+ * W_down_dev: [nblk, C/nblk, E*C/nblk] bf16; z_dev: B*T*C bf16 of scratch that receives z.  z_dev and y_dev
+ * must not overlap x_dev or each other; both are also used as scratch while the call runs.
+ * Layout of z on return: [B, T, C] like x, except where m2_block_z_channel_first(plan, T, C, nblk, E) returns 1: there
+ * z is left channel-first, [B, C, T], the layout the tensor-core sequence mixer works in and the tensor-core MLP reads
+ * as it lies (bf16 plans with N = 512 = 32 x 16 and blocks of 192 -> 768 -> 192; x is transposed once on the way in,
+ * convolution and gate are one kernel, nothing is transposed back).  The query is host-only arithmetic on the plan and
+ * the shape; it returns 0 for bad arguments. */
+int32_t m2_block_z_channel_first(const m2_plan* plan, int64_t T, int64_t C, int32_t nblk, int32_t expand);
 int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
                      const void* W_up_dev, const void* W_down_dev, void* z_dev, void* y_dev, int64_t B,
                      int64_t T, int64_t C, int32_t nblk, int32_t expand, void* stream);

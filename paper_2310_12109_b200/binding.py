@@ -50,6 +50,7 @@ SIGNATURES = {
     "m2_monarch_matmul": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_monarch_matmul_host": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64, _vp]),
     "m2_block_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
+    "m2_block_z_channel_first": (_i32, [_vp, _i64, _i64, _i32, _i32]),
     "m2_block_fwd_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _i32, _vp]),
     "m2_blocky_factors_bytes": (_i64, [_vp]),
     "m2_blocky_monarch": (_i32, [_vp, _vp, _vp, _i32, _vp, _vp]),
@@ -437,15 +438,17 @@ def m2_monarch_matmul_host(plan: Plan, X_host, L, R, Y_host, X_scratch, Y_scratc
 
 def m2_block_fwd(plan: Plan, x: torch.Tensor, kf: torch.Tensor, w_short: torch.Tensor, W_up: torch.Tensor,
                  W_down: torch.Tensor, nblk: int = 4, expand: int = 4):
-    """x: [B, T, C] bf16.  Returns (y, z)."""
+    """x: [B, T, C] bf16.  Returns (y, z), both indexed [b, t, c]; where the library leaves z channel-first
+    (m2_block_z_channel_first) the returned z is a transposed view of that buffer."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 3
     assert w_short.dtype == torch.float32 and W_up.dtype == torch.bfloat16 and W_down.dtype == torch.bfloat16
     B, T, C = x.shape
-    z = torch.empty_like(x)
+    zcf = int(lib().m2_block_z_channel_first(plan.handle, T, C, nblk, expand)) == 1
+    z = torch.empty((B, C, T) if zcf else (B, T, C), dtype=x.dtype, device=x.device)
     y = torch.empty_like(x)
     _check(lib().m2_block_fwd(plan.handle, _ptr(x), _ptr(kf), _ptr(w_short), _ptr(W_up), _ptr(W_down), _ptr(z), _ptr(y),
                               B, T, C, nblk, expand, _stream()), "m2_block_fwd")
-    return y, z
+    return y, (z.transpose(1, 2) if zcf else z)
 
 
 def m2_block_fwd_static(plan: Plan, x: torch.Tensor, kf: torch.Tensor, w_short: torch.Tensor, W_up: torch.Tensor,

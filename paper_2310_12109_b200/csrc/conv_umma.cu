@@ -425,10 +425,18 @@ constexpr int P_SMEM_BYTES = P_OFF_GROUP + kGroupsP * P_GROUP_BYTES;
 static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols && P_SMEM_BYTES <= 232448 && P_OFF_GROUP % 1024 == 0,
               "per-CTA budgets");
 
+//
+// GATE (the M2 block's sequence mixer, Eq. 2 with the depthwise gate of Sec. 5.1): the rows leave multiplied by the width-3
+// depthwise convolution of the INPUT row, y[t] <- y[t] (w[h][0] x[t-1] + w[h][1] x[t] + w[h][2] x[t+1]), zero padded at both ends
+// of the row.  xg = the input rows again ([B][H][512], read from L2 in the last hand-off: the unit's tile in shared memory has
+// long been replaced by the next unit's), w_gate = [H][3] fp32.  The output may be written over the input (map_y over the same rows
+// as map_x): a unit's rows are read for the last time before its stores are issued, and no other unit touches them.
+template <bool GATE>
 __global__ void __launch_bounds__(kThreadsP, 1)
 conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
-               int32_t* __restrict__ status, int* __restrict__ sched, int selftest, int kf_group) {
+               int32_t* __restrict__ status, int* __restrict__ sched, int selftest, int kf_group,
+               const __nv_bfloat16* __restrict__ xg, const float* __restrict__ w_gate) {
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
@@ -719,14 +727,55 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const int m = 16 * warp + (tid & 15), c = m >> 5, n1 = m & 31, rh = (tid >> 4) & 1;
             unsigned char* st = smem + P_G_A + c * 8192 + (4 * rh) * 1024 + n1 * 32;
             const int sw = (n1 >> 2) & 1;
+            float w0 = 0.f, w1 = 0.f, w2 = 0.f;
+            if (GATE) {
+                w0 = __ldg(w_gate + 3 * h);
+                w1 = __ldg(w_gate + 3 * h + 1);
+                w2 = __ldg(w_gate + 3 * h + 2);
+            }
 #pragma unroll
             for (int g = 0; g < 2; ++g) {   // two rows at a time
+                // GATE: the 16 input values under this thread's run and their two neighbours, for both rows (requested before the
+                // accumulator is read so that the two latencies overlap)
+                uint4 xa[2], xb[2];
+                unsigned short xl[2], xr[2];
+                if (GATE) {
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const int brow = b0 + kRows * c + 4 * rh + 2 * g + rr;
+                        xa[rr] = xb[rr] = make_uint4(0u, 0u, 0u, 0u);
+                        xl[rr] = xr[rr] = 0;
+                        if (brow < B) {
+                            const __nv_bfloat16* xrow = xg + ((size_t)brow * H + h) * 512 + 16 * n1;
+                            xa[rr] = __ldg(reinterpret_cast<const uint4*>(xrow));
+                            xb[rr] = __ldg(reinterpret_cast<const uint4*>(xrow) + 1);
+                            if (n1 > 0) xl[rr] = __ldg(reinterpret_cast<const unsigned short*>(xrow) - 1);
+                            if (n1 < 31) xr[rr] = __ldg(reinterpret_cast<const unsigned short*>(xrow) + 16);
+                        }
+                    }
+                }
                 float v[32];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) tmem_ld8(t_lane + T2 + 32 * g + 8 * q, v + 8 * q);
                 tmem_ld_wait();
 #pragma unroll
                 for (int q = 0; q < 4; ++q) tmem_ld_fence8(v + 8 * q);
+                if (GATE) {
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const uint32_t xw[8] = {xa[rr].x, xa[rr].y, xa[rr].z, xa[rr].w, xb[rr].x, xb[rr].y, xb[rr].z, xb[rr].w};
+                        float xv[18];   // x[t0 - 1 .. t0 + 16]; a bf16 is the upper half of its fp32
+                        xv[0] = __uint_as_float((uint32_t)xl[rr] << 16);
+                        xv[17] = __uint_as_float((uint32_t)xr[rr] << 16);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            xv[1 + 2 * j] = __uint_as_float(xw[j] << 16);
+                            xv[2 + 2 * j] = __uint_as_float(xw[j] & 0xffff0000u);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[16 * rr + j] *= fmaf(w2, xv[j + 2], fmaf(w1, xv[j + 1], w0 * xv[j]));
+                    }
+                }
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {   // q = (row, half of the n2 range): one 16-byte chunk of the row's 32-byte run
                     const uint4 pk = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
@@ -1088,7 +1137,8 @@ cudaError_t create_tables(m2_plan* pl) {
     cudaError_t e = cudaMalloc(&t->d_const, CONST_BYTES);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_const_p, P_CONST_BYTES);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_const_p, blob_p.data(), P_CONST_BYTES, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_sched, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(t->d_sched, 0, 2 * sizeof(int));
@@ -1124,7 +1174,7 @@ static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_
 }
 
 static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
-                             cudaStream_t stream, int selftest, int kf_group) {
+                             cudaStream_t stream, int selftest, int kf_group, const float* w_gate = nullptr) {
     if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
     // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
@@ -1132,7 +1182,8 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const bool pairs = B > kRows;   // two batch rows per complex row once there are more than 8
+    const bool pairs = B > kRows || w_gate != nullptr;   // two batch rows per complex row once there are more than 8 (the gated form has this kernel only)
+    if (w_gate != nullptr && (mode != M2_CIRCULAR || kf_group != 1)) return M2_ERR_UNSUPPORTED;
     if (selftest && !pairs) return M2_ERR_UNSUPPORTED;
     const long long units = pairs ? H * ((B + 2 * kRows - 1) / (2 * kRows)) : H * ((B + kRows - 1) / kRows);
     const int groups = pairs ? kGroupsP : kGroups;
@@ -1157,9 +1208,13 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
         if (!make_map_rows32(&my, y, B, H, n)) return M2_ERR_UNSUPPORTED;
         alignas(64) CUtensorMap mx32;   // the row-pair kernel reads whole 32-byte rows of 16 n2
         if (!make_map_rows32(&mx32, x, B, H, n)) return M2_ERR_UNSUPPORTED;
-        if (cudaLaunchKernelEx(&cfg, conv512p_kernel, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H, (int)n,
-                               pl->d_status, t->d_sched, selftest, kf_group) != cudaSuccess)
-            return M2_ERR_CUDA;
+        const cudaError_t le =
+            w_gate != nullptr
+                ? cudaLaunchKernelEx(&cfg, conv512p_kernel<true>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
+                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)x, w_gate)
+                : cudaLaunchKernelEx(&cfg, conv512p_kernel<false>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
+                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)nullptr, (const float*)nullptr);
+        if (le != cudaSuccess) return M2_ERR_CUDA;
     } else {
         alignas(64) CUtensorMap mx;
         if (!make_map_rows32(&mx, x, B, H, n)) return M2_ERR_UNSUPPORTED;
@@ -1167,7 +1222,7 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
                                t->d_sched, kf_group) != cudaSuccess)
             return M2_ERR_CUDA;
     }
-    pl->last_kernel = pairs ? "conv_umma_o2_512_pairs" : "conv_umma_o2_512_rows";
+    pl->last_kernel = w_gate != nullptr ? "conv_umma_o2_512_pairs_gated" : pairs ? "conv_umma_o2_512_pairs" : "conv_umma_o2_512_rows";
     pl->launches += 1;
     return M2_OK;
 }
@@ -1175,6 +1230,12 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
 int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
                  cudaStream_t stream, int kf_group) {
     return conv_fwd_impl(pl, x, kf, y, B, H, n, mode, stream, 0, kf_group);
+}
+
+int32_t conv_gate_fwd(const m2_plan* pl, const void* x, const void* kf, const float* w_gate, void* y, int64_t B, int64_t H,
+                      cudaStream_t stream) {
+    if (w_gate == nullptr) return M2_ERR_INVALID_ARG;
+    return conv_fwd_impl(pl, x, kf, y, B, H, 512, M2_CIRCULAR, stream, 0, 1, w_gate);
 }
 
 int32_t conv_fwd_wait_selftest(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,

@@ -15,6 +15,11 @@ void destroy_tables(m2_plan* plan);
 // kf_group: channel h is multiplied by spectrum row h / kf_group (the buffer then holds H / kf_group rows).
 int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n,
                  int32_t mode, cudaStream_t stream, int kf_group = 1);
+// The circular convolution of [B][H][512] rows followed by the M2 block's depthwise gate, in one kernel:
+//   y[b][h][t] = conv(x[b][h], k[h])[t] * (w_gate[h][0] x[b][h][t-1] + w_gate[h][1] x[b][h][t] + w_gate[h][2] x[b][h][t+1])
+// (zero padded at both ends of a row; w_gate [H][3] fp32).  y may be x: the rows are then replaced in place.
+int32_t conv_gate_fwd(const m2_plan* plan, const void* x, const void* kf, const float* w_gate, void* y, int64_t B, int64_t H,
+                      cudaStream_t stream);
 // The row-pair kernel launched so that every pipeline's first bounded wait runs out with nothing in flight (no copy is
 // issued, a few polls per wait): the kernel leaves through its abort path, sets M2_ERR_TIMEOUT in the plan's status
 // word, writes nothing to y.  Needs B > 8 (the row-pair kernel); M2_ERR_UNSUPPORTED otherwise.

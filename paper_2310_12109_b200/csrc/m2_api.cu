@@ -715,9 +715,23 @@ namespace {
 // order-2 kernel covers take the channel-first route: x -> xT[B][C][T] (in z), long convolution on the tensor cores
 // (into y, which the MLP overwrites afterwards), then the gate kernel transposes back into z.  Other plans run the
 // strided CUDA-core kernel.  Returns the number of launches to add to the plan's count or a negative status.
+// true when the block forward keeps z channel-first, [B][C][T]: the tensor-core sequence mixer (N = 512) feeding the tensor-core
+// MLP.  One transposition (x to channel-first) is then all that stands between the caller's layout and the kernels'.
+bool block_z_channel_first(const m2_plan* plan, int64_t T, int64_t C, int32_t nblk, int32_t expand) {
+    return plan->dtype == M2_BF16 && m2u::has_private_spectrum(plan) && !m2u3::covered(plan) && T == 512 && C % 64 == 0 &&
+           m2mlp::covered((int)C, nblk, expand);
+}
+
 int32_t block_mix_gate(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev, void* z, void* y_scratch,
-                       int64_t B, int64_t T, int64_t C, cudaStream_t stream, bool* tensor_core) {
+                       int64_t B, int64_t T, int64_t C, cudaStream_t stream, bool* tensor_core, bool channel_first) {
     *tensor_core = false;
+    if (channel_first) {   // x -> channel-first in z; convolution and gate in one kernel, in place
+        if (m2g::launch_transpose_btc(x_dev, z, B, (int)T, (int)C, stream) != cudaSuccess) return -M2_ERR_CUDA;
+        const int32_t st = m2u::conv_gate_fwd(plan, z, kf_dev, w_short_dev, z, B, C, stream);
+        if (st != M2_OK) return -st;
+        *tensor_core = true;
+        return 1;   // (the convolution counts its own launch)
+    }
     if (m2u::has_private_spectrum(plan) && !m2u3::covered(plan) && T == 512 && C % 64 == 0) {
         if (m2g::launch_transpose_btc(x_dev, z, B, (int)T, (int)C, stream) != cudaSuccess) return -M2_ERR_CUDA;
         const int32_t st = m2u::conv_fwd(plan, z, kf_dev, y_scratch, B, C, T, M2_CIRCULAR, stream);
@@ -738,6 +752,11 @@ int32_t block_mix_gate(const m2_plan* plan, const void* x_dev, const void* kf_de
 
 }  // namespace
 
+int32_t m2_block_z_channel_first(const m2_plan* plan, int64_t T, int64_t C, int32_t nblk, int32_t expand) {
+    if (!plan || C <= 0 || nblk <= 0 || expand <= 0 || C % nblk != 0) return 0;
+    return block_z_channel_first(plan, T, C, nblk, expand) ? 1 : 0;
+}
+
 int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev, const float* w_short_dev,
                      const void* W_up_dev, const void* W_down_dev, void* z_dev, void* y_dev, int64_t B, int64_t T,
                      int64_t C, int32_t nblk, int32_t expand, void* stream) {
@@ -754,11 +773,12 @@ int32_t m2_block_fwd(const m2_plan* plan, const void* x_dev, const void* kf_dev,
     if (!g.ok) return M2_ERR_CUDA;
     if (B == 0) return M2_OK;
     bool tc_mix = false;
-    const int32_t nl = block_mix_gate(plan, x_dev, kf_dev, w_short_dev, z_dev, y_dev, B, T, C, (cudaStream_t)stream, &tc_mix);
+    const bool zcf = block_z_channel_first(plan, T, C, nblk, expand);
+    const int32_t nl = block_mix_gate(plan, x_dev, kf_dev, w_short_dev, z_dev, y_dev, B, T, C, (cudaStream_t)stream, &tc_mix, zcf);
     if (nl < 0) return -nl;
     cudaError_t e = cudaSuccess;
     if (m2mlp::covered((int)C, nblk, expand)) {   // tensor-core MLP for 192 -> 768 -> 192 blocks
-        const int32_t st = m2mlp::launch(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
+        const int32_t st = m2mlp::launch(z_dev, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream, zcf ? T : 0);
         if (st != M2_OK) return st;
         plan->last_kernel = tc_mix ? "block_conv_umma_mlp_umma" : "block_conv_generic_mlp_umma";
     } else {
@@ -802,11 +822,12 @@ int32_t m2_block_fwd_static(const m2_plan* plan, const void* x_dev, const void* 
     // Same launches as m2_block_fwd; every element of z[B, T, C] is written before it is read, so the array's
     // previous contents never matter.
     bool tc_mix = false;
-    const int32_t nl = block_mix_gate(plan, x_dev, kf_dev, w_short_dev, z, y_dev, B, T, C, (cudaStream_t)stream, &tc_mix);
+    const bool zcf = block_z_channel_first(plan, T, C, nblk, expand);
+    const int32_t nl = block_mix_gate(plan, x_dev, kf_dev, w_short_dev, z, y_dev, B, T, C, (cudaStream_t)stream, &tc_mix, zcf);
     if (nl < 0) return -nl;
     cudaError_t e = cudaSuccess;
     if (m2mlp::covered((int)C, nblk, expand)) {
-        const int32_t st = m2mlp::launch(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream);
+        const int32_t st = m2mlp::launch(z, W_up_dev, W_down_dev, y_dev, (int)C, nblk, B * T, plan->d_status, (cudaStream_t)stream, zcf ? T : 0);
         if (st != M2_OK) return st;
         plan->last_kernel = tc_mix ? "block_conv_umma_mlp_umma_static" : "block_conv_generic_mlp_umma_static";
     } else {

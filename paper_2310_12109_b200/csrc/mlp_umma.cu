@@ -47,6 +47,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
                  "l"(map), "r"(c0), "r"(c1), "r"(bar)
                  : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+                 "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+                 : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -81,10 +86,14 @@ __device__ __forceinline__ uint32_t gelu2_pack(float v0, float v1) {
 // byte offset of 16-byte chunk kc of row r in a K-major block with 128-byte rows and the 128B swizzle
 __device__ __forceinline__ uint32_t sw_off(int r, int kc) { return (uint32_t)((r >> 3) * 1024 + (r & 7) * 128 + ((kc ^ (r & 7)) << 4)); }
 
+// ZCF: the activations arrive channel-first, z[b][c][t] (T positions per batch entry, a multiple of 128), as the sequence mixer
+// leaves them: an item's tile is then two boxes [192 channels][64 tokens], the tokens contiguous -- as they lie the two 64-token
+// blocks of an M-major A operand (K = the channels) -- and nothing has to be transposed between the mixer and the MLP.
+template <bool ZCF>
 __global__ void __launch_bounds__(kThreads, 1)
 mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_w1,
                 const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_y, int32_t* __restrict__ status,
-                int nblk, int nitems) {
+                int nblk, int nitems, int T) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t s_base = smem_u32(smem);
@@ -136,8 +145,14 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 bool progressed = false;
                 if (zq < nq && (zq < 1 || mbar_try_wait(bar(B_ZE), (zq - 1) & 1))) {                                  // the last S1 of item zq - 1 has read Z
                     mbar_expect_tx(bar(B_Z), 49152);
-                    for (int kb = 0; kb < 3; ++kb)
-                        tma_load_2d(s_base + OFF_Z + kb * 16384, &map_z, item_j(zq) * kCI + kb * 64, item_t0(zq), bar(B_Z));
+                    if (ZCF) {
+                        const int tt = item_t0(zq);
+                        for (int mb = 0; mb < 2; ++mb)
+                            tma_load_3d(s_base + OFF_Z + mb * 24576, &map_z, tt % T + 64 * mb, item_j(zq) * kCI, tt / T, bar(B_Z));
+                    } else {
+                        for (int kb = 0; kb < 3; ++kb)
+                            tma_load_2d(s_base + OFF_Z + kb * 16384, &map_z, item_j(zq) * kCI + kb * 64, item_t0(zq), bar(B_Z));
+                    }
                     ++zq;
                     progressed = true;
                 }
@@ -164,7 +179,7 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
     } else if (warp == 1) {
         // ---- UMMA issuer ---------------------------------------------------------------------------------------------
         if (lane == 0) {
-            constexpr uint32_t ID1 = instr_desc_bf16(128, 128, false, false), ID2 = instr_desc_bf16(128, 192, false, false);
+            constexpr uint32_t ID1 = instr_desc_bf16(128, 128, ZCF, false), ID2 = instr_desc_bf16(128, 192, false, false);
             auto s1 = [&](int g) {   // D1[g % 2] = Z * W_up chunk g
                 const int b = g & 1;
                 ok = mbar_wait(bar(B_W1F + b), (g >> 1) & 1);
@@ -175,7 +190,9 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
                 for (int kb = 0; kb < 3; ++kb)
 #pragma unroll
                     for (int s = 0; s < 4; ++s)
-                        umma_f16(D1 + b * 128, smem_desc_sw128(s_base + OFF_Z + kb * 16384 + s * 32, 16, 1024),
+                        umma_f16(D1 + b * 128,
+                                 ZCF ? smem_desc_sw128(s_base + OFF_Z + (kb * 4 + s) * 2048, 24576, 1024)   // 16 channels = 16 rows of 128 bytes
+                                     : smem_desc_sw128(s_base + OFF_Z + kb * 16384 + s * 32, 16, 1024),
                                  smem_desc_sw128(s_base + OFF_W1 + b * 49152 + kb * 16384 + s * 32, 16, 1024), ID1, (kb | s) != 0);
                 umma_commit(bar(B_D1F + b));
                 umma_commit(bar(B_W1E + b));
@@ -312,11 +329,17 @@ mlp_umma_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant
 
 bool covered(int C, int nblk, int expand) { return nblk > 0 && C / nblk == kCI && C % nblk == 0 && expand * kCI == kHID; }
 
-cudaError_t prepare() { return cudaFuncSetAttribute(mlp_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES); }
+cudaError_t prepare() {
+    cudaError_t e = cudaFuncSetAttribute(mlp_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(mlp_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    return e;
+}
 
 int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, int nblk, long long tokens, int32_t* status,
-               cudaStream_t stream) {
+               cudaStream_t stream, long long z_channel_first_T) {
     if (tokens == 0) return M2_OK;
+    const long long T = z_channel_first_T;
+    if (T != 0 && (T < 0 || T % kTileT != 0 || tokens % T != 0 || T > 0x7fffffffLL)) return M2_ERR_INVALID_ARG;
     int dev_id = 0;
     {   // the shared-memory opt-in is per device (setting it twice is harmless; the flag itself is race-free)
         static std::atomic<bool> prepared[64];
@@ -332,8 +355,14 @@ int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, 
     {   // activations [tokens][C]: box = 64 columns x 128 tokens, 128B swizzle (rows past the end: zero-filled / clipped)
         const cuuint64_t gdim[2] = {(cuuint64_t)C, (cuuint64_t)tokens}, gstr[1] = {(cuuint64_t)C * 2};
         const cuuint32_t box[2] = {64, (cuuint32_t)kTileT};
-        if (!tma_host::encode_sw128_bf16(&mz, z, 2, gdim, gstr, box) || !tma_host::encode_sw128_bf16(&my, y, 2, gdim, gstr, box))
-            return M2_ERR_UNSUPPORTED;
+        if (!tma_host::encode_sw128_bf16(&my, y, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+        if (T == 0) {
+            if (!tma_host::encode_sw128_bf16(&mz, z, 2, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+        } else {   // z[b][c][t]: box = 64 tokens x the block's 192 channels of one batch entry
+            const cuuint64_t zdim[3] = {(cuuint64_t)T, (cuuint64_t)C, (cuuint64_t)(tokens / T)}, zstr[2] = {(cuuint64_t)T * 2, (cuuint64_t)C * T * 2};
+            const cuuint32_t zbox[3] = {64, (cuuint32_t)kCI, 1};
+            if (!tma_host::encode_sw128_bf16(&mz, z, 3, zdim, zstr, zbox)) return M2_ERR_UNSUPPORTED;
+        }
     }
     {   // W_up [nblk * 768 hidden][192 in]: box = 64 x 128 rows;  W_down [nblk * 192 out][768 hidden]: box = 64 x 192 rows
         const cuuint64_t g1[2] = {(cuuint64_t)kCI, (cuuint64_t)nblk * kHID}, s1[1] = {(cuuint64_t)kCI * 2};
@@ -356,7 +385,9 @@ int32_t launch(const void* z, const void* Wup, const void* Wdn, void* y, int C, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, mlp_umma_kernel, mz, mw1, mw2, my, status, nblk, (int)nitems) != cudaSuccess) return M2_ERR_CUDA;
+    const cudaError_t le = T != 0 ? cudaLaunchKernelEx(&cfg, mlp_umma_kernel<true>, mz, mw1, mw2, my, status, nblk, (int)nitems, (int)T)
+                                  : cudaLaunchKernelEx(&cfg, mlp_umma_kernel<false>, mz, mw1, mw2, my, status, nblk, (int)nitems, 1);
+    if (le != cudaSuccess) return M2_ERR_CUDA;
     return M2_OK;
 }
 

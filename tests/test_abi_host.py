@@ -86,6 +86,9 @@ def test_argument_validation_without_device():
     assert lib.m2_monarch_matmul(h, 16, 16, 16, 16, 4, None, 0, None) == M.M2_ERR_NO_DEVICE
     assert lib.m2_kernel_spectrum(h, 16, 1, 256, 16, None) == M.M2_ERR_NO_DEVICE
     assert lib.m2_spectrum_bytes(h, 3) == 3 * 512 * 8
+    # a host-only plan has no tensor-core route, so its block forward would leave z channel-last; bad arguments answer 0 too
+    assert lib.m2_block_z_channel_first(h, 512, 768, 4, 4) == 0
+    assert lib.m2_block_z_channel_first(None, 512, 768, 4, 4) == 0 and lib.m2_block_z_channel_first(h, 512, 768, 5, 4) == 0
     assert lib.m2_plan_destroy(h) == M.M2_OK
     assert lib.m2_plan_destroy(None) == M.M2_ERR_INVALID_ARG
     assert lib.m2_status_string(M.M2_ERR_TIMEOUT) == b"device-side wait timed out"

@@ -401,6 +401,45 @@ def test_block_other_shapes(T, C, nblk, expand, dims, kernel):
     check(y.reshape(-1, C), yr.reshape(-1, C), TOL_BF16, "block y")
 
 
+@pytest.mark.parametrize("B", [1, 9, 17])
+def test_config5_ragged_batches(B):
+    """Batch sizes that leave the last 16-row unit of the gated convolution partly empty (rows past B are never read or written)."""
+    c = synth.config5(B=B)
+    y, z = run_block(c, "block_conv_umma_mlp_umma")
+    sel = sorted({0, B // 2, B - 1})
+    yr, zr = block_ref(c, sel)
+    check(z[sel].reshape(-1, 768), zr.reshape(-1, 768), TOL_BF16, "config5 ragged z")
+    check(y[sel].reshape(-1, 768), yr.reshape(-1, 768), TOL_BF16, "config5 ragged y")
+
+
+def test_block_z_layout_query_matches_the_buffer():
+    """Where the query says so, the z buffer is channel-first [B, C, T]; elsewhere [B, T, C].  Called through the C ABI with the
+    caller's own buffers, canaries behind both."""
+    lib = M.lib()
+    s = torch.cuda.current_stream().cuda_stream
+    for (T, C, nblk, expand, dims, want) in ((512, 768, 4, 4, (32, 16), 1), (512, 128, 4, 2, (32, 16), 0), (64, 32, 4, 2, (8, 8), 0)):
+        c = synth.config5(B=3, T=T, C=C, nblk=nblk, expand=expand)
+        c["dims"] = dims
+        plan = M.Plan(dims, dtype=M.M2_BF16, device=0)
+        assert lib.m2_block_z_channel_first(plan.handle, T, C, nblk, expand) == want
+        assert lib.m2_block_z_channel_first(plan.handle, T, C, 0, expand) == 0 and lib.m2_block_z_channel_first(None, T, C, nblk, expand) == 0
+        kf = M.m2_kernel_spectrum(plan, dev(c["k"]))
+        x, w, wu, wd = dev(c["x"], torch.bfloat16), dev(c["w_short"]), dev(c["W_up"], torch.bfloat16), dev(c["W_down"], torch.bfloat16)
+        n = 3 * T * C
+        zbuf = torch.full((n + 64,), 7.0, dtype=torch.bfloat16, device="cuda")
+        ybuf = torch.full((n + 64,), 7.0, dtype=torch.bfloat16, device="cuda")
+        assert lib.m2_block_fwd(plan.handle, x.data_ptr(), kf.data_ptr(), w.data_ptr(), wu.data_ptr(), wd.data_ptr(), zbuf.data_ptr(),
+                                ybuf.data_ptr(), 3, T, C, nblk, expand, s) == M.M2_OK
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        assert (zbuf[n:] == 7).all().item() and (ybuf[n:] == 7).all().item()
+        yr, zr = block_ref(c)
+        z = zbuf[:n].view(3, C, T).transpose(1, 2) if want else zbuf[:n].view(3, T, C)
+        check(host(z).reshape(-1, C), zr.reshape(-1, C), TOL_BF16, f"block z buffer layout T={T} C={C}")
+        check(host(ybuf[:n].view(3, T, C)).reshape(-1, C), yr.reshape(-1, C), TOL_BF16, f"block y T={T} C={C}")
+        plan.close()
+
+
 def test_config5_full_size_sampled():
     c = synth.config5()
     y, z = run_block(c)

@@ -444,6 +444,8 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // the thread that issues this pipeline's UMMAs and copies; its warp differs from group to group so that
     // the extra work spreads over the SM's four schedulers
     const bool leader = tid == 32 * (wg & 3);
+    // a second issuing thread, two schedulers further on, takes the second half of the stages that have two independent halves
+    const bool leader2 = tid == 32 * ((wg + 2) & 3);
     const uint32_t s_all = smem_u32(smem_all);
     unsigned char* smem = smem_all + P_OFF_GROUP + wg * P_GROUP_BYTES;   // this group's slice
     const uint32_t s_base = s_all + P_OFF_GROUP + wg * P_GROUP_BYTES;
@@ -459,7 +461,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const int ustride = gridDim.x * kGroupsP;
     if (leader) {
         mbar_init(bar_x, 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_mma, 2);   // both issuing threads commit in every stage
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_x);
@@ -549,6 +551,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 umma_commit(bar_mma);
             }
         }
+        if (leader2) umma_commit(bar_mma);   // (nothing of its own to track in this stage)
         ph_x ^= 1;
         // ---- h1: twiddle, A2 ---------------------------------------------------------------------
         ok = ok && mbar_wait(bar_mma, ph_m, wlim);
@@ -596,14 +599,13 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             break;
         }
         // ---- S2 ---------------------------------------------------------------------------------
-        if (leader) {
+        if (leader || leader2) {
             tc_fence_after();
+            const int hf = leader ? 0 : 1;
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                for (int s = 0; s < 2; ++s)
-                    umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 512),
-                             smem_desc(s_all + P_OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
+            for (int s = 0; s < 2; ++s)
+                umma_f16(tmem + T2 + hf * 32, smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 512),
+                         smem_desc(s_all + P_OFF_B2 + s * 256, 128, 512), ID_S2, s > 0);
             umma_commit(bar_mma);
         }
         // ---- h2: spectrum multiply, A3 -------------------------------------------------------------
@@ -650,14 +652,13 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             break;
         }
         // ---- S2' --------------------------------------------------------------------------------
-        if (leader) {
+        if (leader || leader2) {
             tc_fence_after();
+            const int hf = leader ? 0 : 1;
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                for (int s = 0; s < 2; ++s)
-                    umma_f16(tmem + T1 + hf * 32, smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 512),
-                             smem_desc(s_all + P_OFF_B3 + s * 256, 128, 512), ID_S2I, s > 0);
+            for (int s = 0; s < 2; ++s)
+                umma_f16(tmem + T1 + hf * 32, smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 512),
+                         smem_desc(s_all + P_OFF_B3 + s * 256, 128, 512), ID_S2I, s > 0);
             umma_commit(bar_mma);
         }
         // ---- h3: conjugate twiddle, A4 --------------------------------------------------------------
@@ -702,17 +703,16 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             break;
         }
         // ---- S1' --------------------------------------------------------------------------------
-        if (leader) {
+        if (leader || leader2) {
             tc_fence_after();
             // the conjugated F_32 image is the A operand here (M = (re | im) x n1 = 64) and the data the B operand (N = 4 rows x 16 n2),
             // so that a thread of the last hand-off owns whole 32-byte runs of the output; the second half of the rows goes to
             // lanes 16..31 of every lane quarter (an M = 64 accumulator keeps row m in lane m % 16 + 32 (m / 16))
+            const int hf = leader ? 0 : 1;
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                for (int s = 0; s < 4; ++s)
-                    umma_f16(tmem + T2 + ((uint32_t)(16 * hf) << 16), smem_desc(s_all + P_OFF_B4 + s * 256, 128, 1024),
-                             smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 1024), ID_S1I, s > 0);
+            for (int s = 0; s < 4; ++s)
+                umma_f16(tmem + T2 + ((uint32_t)(16 * hf) << 16), smem_desc(s_all + P_OFF_B4 + s * 256, 128, 1024),
+                         smem_desc(s_base + P_G_A + hf * 8192 + s * 256, 128, 1024), ID_S1I, s > 0);
             umma_commit(bar_mma);
         }
         // ---- h4: round and stage: a lane holds, for one n1 of the real-part rows or of the imaginary-part rows, the 16 n2 of

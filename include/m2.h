@@ -230,7 +230,9 @@ int32_t m2_bert_mixer_fwd(const m2_plan* plan, const void* x_dev, const void* co
  * W: HOST array of 4 device pointers {W_X1, W_X2, W_V, W_O}, each [d][d] stored outputs x inputs (y[o] = sum_i W[o][i] u[i]).
  * kf1_dev, kf2_dev, kf3_dev: m2_kernel_spectrum of the short kernels [d, n];  kf_long_dev: m2_kernel_spectrum of the long
  * kernels, one row per head: [d / dh, n] (the dh^2 sequences of a head share its row: m2_monarch_conv_fwd_grouped).
- * y_dev: [B, n, d] (must not overlap u_dev).  scratch_dev: m2_hyena_scratch_bytes(plan, B, n, d, dh) bytes, caller-owned.
+ * y_dev: [B, n, d] (must not overlap u_dev).  scratch_dev: m2_hyena_scratch_bytes(plan, B, n, d, dh) bytes, caller-owned
+ * ((7 + 2 dh) tensors of B d n elements; 7 for heads of dh = 16 on the bf16 N = 512 plan with n a multiple of 16 up to 256, where
+ * outer product, long convolution and contraction are one tensor-core kernel and the dh-times larger tensors do not exist).
  * The projections are the single-block case of the column-layout Monarch kernel (tensor cores for d a multiple of 64 up
  * to 4096 and n a multiple of 8, bf16), so after one transposition everything runs channel-first. */
 int64_t m2_hyena_scratch_bytes(const m2_plan* plan, int64_t B, int64_t n, int64_t d, int64_t dh);

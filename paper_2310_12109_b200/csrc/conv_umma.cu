@@ -431,12 +431,21 @@ static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols 
 // of the row.  xg = the input rows again ([B][H][512], read from L2 in the last hand-off: the unit's tile in shared memory has
 // long been replaced by the next unit's), w_gate = [H][3] fp32.  The output may be written over the input (map_y over the same rows
 // as map_x): a unit's rows are read for the last time before its stores are issued, and no other unit touches them.
-template <bool GATE>
+//
+// HEADS (MODE 2; the core of the M2 Hyena layer with heads of dh = 16 channels, GPT appendix): a unit is one (batch entry b, channel
+// hj = head * 16 + j) and its 16 rows are the sequences X2[b][head * 16 + i][t] V[b][hj][t], i = 0 .. 15, of the head's outer
+// product -- formed in shared memory from the TMA-loaded X2 rows (map_x boxes span 8 CHANNELS of one batch entry) and the V row
+// (vh) before the first stage -- and what leaves is their causal convolution with the head's kernel contracted with X1 (xg):
+//   y[b][hj][t] = sum_i X1[b][head * 16 + i][t] (k_head * (X2_i V_j))[t],   t < n <= 256.
+// The d_h-times larger tensor of the outer product and of its convolution never exists in memory.  kf_group = dh selects the
+// head's spectrum row.  Nothing is staged or stored by TMA in this mode: a unit's result is one row of n values.
+template <int MODE>
 __global__ void __launch_bounds__(kThreadsP, 1)
 conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y, __nv_bfloat16* __restrict__ y,
                const float4* __restrict__ kfu, const uint4* __restrict__ consts, int B, int H, int n,
                int32_t* __restrict__ status, int* __restrict__ sched, int selftest, int kf_group,
-               const __nv_bfloat16* __restrict__ xg, const float* __restrict__ w_gate) {
+               const __nv_bfloat16* __restrict__ xg, const float* __restrict__ w_gate, const __nv_bfloat16* __restrict__ vh) {
+    constexpr bool GATE = MODE == 1, HEADS = MODE == 2;
     extern __shared__ __align__(1024) unsigned char smem_all[];
     const int wg = threadIdx.x >> 7;          // warpgroup = independent unit pipeline
     const int tid = threadIdx.x & 127;
@@ -454,7 +463,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     volatile int* next_slot = reinterpret_cast<volatile int*>(smem_all + P_OFF_BAR + wg * 32 + 28);
     const uint32_t s_tptr = s_all + P_OFF_BAR + 512;
 
-    const int bgroups0 = (B + 2 * kRows - 1) / (2 * kRows);   // 16 batch rows = 8 complex rows per unit
+    const int bgroups0 = HEADS ? B : (B + 2 * kRows - 1) / (2 * kRows);   // 16 batch rows = 8 complex rows per unit (HEADS: 16 channels of one entry)
     const int units0 = H * bgroups0;
     // pipeline-major numbering: a partial last round of units spreads over all CTAs instead of filling the first ones
     int u = wg * gridDim.x + blockIdx.x;
@@ -470,9 +479,15 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // a prefetch returns no data, and L2 is where that kernel's writes land, so the copies issued after the wait below
         // see them whatever it wrote.
         if (!selftest && u < units0) {
-            const int hh = u % H, bb = (u / H) * 2 * kRows;
-            tma_prefetch_4d(&map_x, 0, 0, hh, bb);
-            tma_prefetch_4d(&map_x, 0, 0, hh, bb + kRows);
+            if (HEADS) {
+                const int hb = ((u % H) / kf_group) * kf_group, bb = u / H;
+                tma_prefetch_4d(&map_x, 0, 0, hb, bb);
+                tma_prefetch_4d(&map_x, 0, 0, hb + kRows, bb);
+            } else {
+                const int hh = u % H, bb = (u / H) * 2 * kRows;
+                tma_prefetch_4d(&map_x, 0, 0, hh, bb);
+                tma_prefetch_4d(&map_x, 0, 0, hh, bb + kRows);
+            }
         }
     }
     // Programmatic dependent launch: the next kernel on the stream may start its CTAs as this grid's CTAs leave
@@ -498,9 +513,15 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     auto load_unit = [&](int v) {
         if (selftest) return;
         mbar_expect_tx(bar_x, 16384);
-        const int hh = v % H, bb = (v / H) * 2 * kRows;
-        tma_load_4d(s_base + P_G_X, &map_x, 0, 0, hh, bb, bar_x);
-        tma_load_4d(s_base + P_G_X + 8192, &map_x, 0, 0, hh, bb + kRows, bar_x);
+        if (HEADS) {   // the head's 16 X2 rows of batch entry v / H: two boxes of 8 channels
+            const int hb = ((v % H) / kf_group) * kf_group, bb = v / H;
+            tma_load_4d(s_base + P_G_X, &map_x, 0, 0, hb, bb, bar_x);
+            tma_load_4d(s_base + P_G_X + 8192, &map_x, 0, 0, hb + kRows, bb, bar_x);
+        } else {
+            const int hh = v % H, bb = (v / H) * 2 * kRows;
+            tma_load_4d(s_base + P_G_X, &map_x, 0, 0, hh, bb, bar_x);
+            tma_load_4d(s_base + P_G_X + 8192, &map_x, 0, 0, hh, bb + kRows, bar_x);
+        }
         x_pending = true;
     };
     if (leader && u < units0) {   // first loads
@@ -532,10 +553,49 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     int un2 = units;        // thread 0: the unit after next, claimed one whole unit ahead so the atomic's latency is never waited for
     while (u < units) {
         const int h = u % H;
-        const int b0 = (u / H) * 2 * kRows;
+        const int b0 = HEADS ? u / H : (u / H) * 2 * kRows;
+        if (HEADS) {
+            // ---- h0: the X2 rows have landed; every row times the V row of this unit's channel, in place.  Thread (row r, n1) owns
+            //      the 32-byte run of 16 positions t = 16 n1 .. of its row in both boxes (rows i = r and i = 8 + r). ----
+            const int r = tid >> 4, n1 = tid & 15, sw = (n1 >> 2) & 1;
+            uint4 va = make_uint4(0u, 0u, 0u, 0u), vb = va;
+            if (16 * n1 < n) {   // (asked for before the wait for the tile: the two latencies overlap)
+                const uint4* vrow = reinterpret_cast<const uint4*>(vh + ((size_t)b0 * H + h) * n + 16 * n1);
+                va = __ldg(vrow);
+                vb = __ldg(vrow + 1);
+            }
+            ok = mbar_wait(bar_x, ph_x, wlim);
+            x_pending = false;
+            if (ok) {
+                if (16 * n1 < n) {
+                    const uint32_t vw[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        unsigned char* row = smem + P_G_X + c * 8192 + r * 1024 + n1 * 32;
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {   // q = half of the run: positions 8 q .. 8 q + 7
+                            uint4* cell = reinterpret_cast<uint4*>(row + ((q ^ sw) << 4));
+                            const uint4 xv = *cell;
+                            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+                            uint32_t o[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                o[k] = pack_bf16(__uint_as_float(xw[k] << 16) * __uint_as_float(vw[4 * q + k] << 16),
+                                                 __uint_as_float(xw[k] & 0xffff0000u) * __uint_as_float(vw[4 * q + k] & 0xffff0000u));
+                            *cell = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                }
+            }
+            fence_proxy_async();   // the products are read by the tensor core
+            if (group_sync_or(wg, !ok, abort_flag)) {
+                aborted = true;
+                break;
+            }
+        }
         // ---- S1 ---------------------------------------------------------------------------------
         if (leader) {
-            ok = mbar_wait(bar_x, ph_x, wlim);
+            if (!HEADS) ok = mbar_wait(bar_x, ph_x, wlim);
             x_pending = false;
             if (ok) {
                 tc_fence_after();
@@ -719,14 +779,66 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         //      four rows: 32-byte runs of y[r][n1*16 + n2].  The operand buffer (free now) takes the two boxes
         //      [8 rows][32 n1][16 n2] in the 32-byte-swizzled image of the TMA stores (16-byte chunk XOR bit 7 of the address):
         //      a quarter-warp's eight 16-byte stores fall into eight different bank groups ---------------
+        // (HEADS: the X1 values this thread will need -- its four rows at its 16 positions -- come from L2 and are asked for before
+        // the wait for the last stage)
+        uint4 x1v[HEADS ? 8 : 1];
+        if (HEADS) {
+            const int m = 16 * warp + (tid & 15), c = m >> 5, n1 = m & 31, rh = (tid >> 4) & 1;
+#pragma unroll
+            for (int rl = 0; rl < 8; ++rl) x1v[rl] = make_uint4(0u, 0u, 0u, 0u);
+            if ((warp & 1) == 0 && 16 * n1 < n) {
+                const int hb = (h / kf_group) * kf_group;
+#pragma unroll
+                for (int rl = 0; rl < 4; ++rl) {
+                    const uint4* xrow = reinterpret_cast<const uint4*>(xg + ((size_t)b0 * H + hb + kRows * c + 4 * rh + rl) * n + 16 * n1);
+                    x1v[2 * rl] = __ldg(xrow);
+                    x1v[2 * rl + 1] = __ldg(xrow + 1);
+                }
+            }
+        }
         ok = mbar_wait(bar_mma, ph_m, wlim);
         ph_m ^= 1;
         tc_fence_after();
+        float hacc[HEADS ? 16 : 1];
         if (ok) {
             // lane l of warp w holds output row m = 16 w + l % 16 = (c, n1) for the rows r = 4 (l / 16) .. + 3: 16 n2 per row
             const int m = 16 * warp + (tid & 15), c = m >> 5, n1 = m & 31, rh = (tid >> 4) & 1;
             unsigned char* st = smem + P_G_A + c * 8192 + (4 * rh) * 1024 + n1 * 32;
             const int sw = (n1 >> 2) & 1;
+            if (HEADS) {
+                // contraction with X1: this thread's four rows i = 8 c + 4 rh + (0 .. 3) at its 16 positions; positions past n do not exist
+#pragma unroll
+                for (int j = 0; j < 16; ++j) hacc[j] = 0.f;
+                // (a warp holds n1 = 0 .. 15 or 16 .. 31: the second kind has nothing below position 256 and skips the tensor-memory
+                // loads as a whole warp; a single lane whose positions lie past n only skips its own global loads)
+                const bool lane_live = 16 * n1 < n;
+                if ((warp & 1) == 0) {
+#pragma unroll
+                    for (int rl = 0; rl < 4; ++rl) {   // one row at a time
+                        const uint4 xa = x1v[2 * rl], xb = x1v[2 * rl + 1];
+                        float v[16];
+                        tmem_ld8(t_lane + T2 + 16 * rl, v);
+                        tmem_ld8(t_lane + T2 + 16 * rl + 8, v + 8);
+                        tmem_ld_wait();
+                        tmem_ld_fence8(v);
+                        tmem_ld_fence8(v + 8);
+                        const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            hacc[2 * j] = fmaf(v[2 * j], __uint_as_float(xw[j] << 16), hacc[2 * j]);
+                            hacc[2 * j + 1] = fmaf(v[2 * j + 1], __uint_as_float(xw[j] & 0xffff0000u), hacc[2 * j + 1]);
+                        }
+                    }
+                }
+                // the other four rows of this half sit 16 lanes further on; the half c = 1 hands its sums over through the operand buffer
+#pragma unroll
+                for (int j = 0; j < 16; ++j) hacc[j] += __shfl_xor_sync(0xffffffffu, hacc[j], 16);
+                if (c == 1 && rh == 0 && lane_live) {
+                    float4* xch = reinterpret_cast<float4*>(smem + P_G_A) + n1 * 4;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) xch[j] = make_float4(hacc[4 * j], hacc[4 * j + 1], hacc[4 * j + 2], hacc[4 * j + 3]);
+                }
+            }
             float w0 = 0.f, w1 = 0.f, w2 = 0.f;
             if (GATE) {
                 w0 = __ldg(w_gate + 3 * h);
@@ -734,7 +846,7 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 w2 = __ldg(w_gate + 3 * h + 2);
             }
 #pragma unroll
-            for (int g = 0; g < 2; ++g) {   // two rows at a time
+            for (int g = 0; g < (HEADS ? 0 : 2); ++g) {   // two rows at a time
                 // GATE: the 16 input values under this thread's run and their two neighbours, for both rows (requested before the
                 // accumulator is read so that the two latencies overlap)
                 uint4 xa[2], xb[2];
@@ -791,7 +903,21 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             aborted = true;
             break;
         }
-        if (leader) {   // rows past the batch and positions past n are clipped by the tensor map
+        if (HEADS) {
+            if (tid < 16 && 16 * tid < n) {   // rows 0 .. 7 summed: add the other half's sums, round, store this lane's 16 positions
+                const float4* xch = reinterpret_cast<const float4*>(smem + P_G_A) + tid * 4;
+                uint32_t o[8];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float4 t4 = xch[j];
+                    o[2 * j] = pack_bf16(hacc[4 * j] + t4.x, hacc[4 * j + 1] + t4.y);
+                    o[2 * j + 1] = pack_bf16(hacc[4 * j + 2] + t4.z, hacc[4 * j + 3] + t4.w);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(y + ((size_t)b0 * H + h) * n + 16 * tid);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+        } else if (leader) {   // rows past the batch and positions past n are clipped by the tensor map
             tma_store_4d(&map_y, s_base + P_G_A, 0, 0, h, b0);
             if (b0 + kRows < B) tma_store_4d(&map_y, s_base + P_G_A + 8192, 0, 0, h, b0 + kRows);
             tma_store_commit();
@@ -1137,8 +1263,9 @@ cudaError_t create_tables(m2_plan* pl) {
     cudaError_t e = cudaMalloc(&t->d_const, CONST_BYTES);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_const_p, P_CONST_BYTES);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_const_p, blob_p.data(), P_CONST_BYTES, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(conv512p_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM_BYTES);
     if (e == cudaSuccess) e = cudaMemcpy(t->d_const, blob.data(), CONST_BYTES, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_sched, 2 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(t->d_sched, 0, 2 * sizeof(int));
@@ -1210,10 +1337,12 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
         if (!make_map_rows32(&mx32, x, B, H, n)) return M2_ERR_UNSUPPORTED;
         const cudaError_t le =
             w_gate != nullptr
-                ? cudaLaunchKernelEx(&cfg, conv512p_kernel<true>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
-                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)x, w_gate)
-                : cudaLaunchKernelEx(&cfg, conv512p_kernel<false>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
-                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)nullptr, (const float*)nullptr);
+                ? cudaLaunchKernelEx(&cfg, conv512p_kernel<1>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
+                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)x, w_gate,
+                                     (const __nv_bfloat16*)nullptr)
+                : cudaLaunchKernelEx(&cfg, conv512p_kernel<0>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
+                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)nullptr, (const float*)nullptr,
+                                     (const __nv_bfloat16*)nullptr);
         if (le != cudaSuccess) return M2_ERR_CUDA;
     } else {
         alignas(64) CUtensorMap mx;
@@ -1236,6 +1365,44 @@ int32_t conv_gate_fwd(const m2_plan* pl, const void* x, const void* kf, const fl
                       cudaStream_t stream) {
     if (w_gate == nullptr) return M2_ERR_INVALID_ARG;
     return conv_fwd_impl(pl, x, kf, y, B, H, 512, M2_CIRCULAR, stream, 0, 1, w_gate);
+}
+
+int32_t conv_heads_fwd(const m2_plan* pl, const void* X1, const void* X2, const void* V, const void* kf_heads, void* y, int64_t B,
+                       int64_t d, int64_t dh, int64_t n, cudaStream_t stream) {
+    if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
+    if (dh != 2 * kRows || d % dh != 0 || n % 16 != 0 || n > 256 || n <= 0) return M2_ERR_UNSUPPORTED;
+    if (B == 0) return M2_OK;
+    if (B * d > 0x7fffffffLL) return M2_ERR_UNSUPPORTED;
+    Tables* t = reinterpret_cast<Tables*>(pl->umma);
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long units = B * d, ctas = (units + kGroupsP - 1) / kGroupsP;
+    // X2 [B][d][n] as (16 n2 | n1 | channel | batch entry); a box takes 8 channels of one entry, digits n1 >= n / 16 read zeros
+    alignas(64) CUtensorMap mx, my;
+    const cuuint64_t gdim[4] = {16, (cuuint64_t)(n / 16), (cuuint64_t)d, (cuuint64_t)B};
+    const cuuint64_t gstr[3] = {32, (cuuint64_t)n * 2, (cuuint64_t)d * n * 2};
+    const cuuint32_t box[4] = {16, 32, (cuuint32_t)kRows, 1};
+    if (!tma_host::encode_sw32_bf16(&mx, X2, 4, gdim, gstr, box)) return M2_ERR_UNSUPPORTED;
+    if (!make_map_rows32(&my, y, B, d, n)) return M2_ERR_UNSUPPORTED;   // (not used by this mode; a valid map all the same)
+    const float4* kfu = reinterpret_cast<const float4*>(static_cast<const unsigned char*>(kf_heads) + (size_t)(d / dh) * 512 * 8);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(ctas < sms ? ctas : sms));
+    cfg.blockDim = dim3(kThreadsP);
+    cfg.dynamicSmemBytes = P_SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, conv512p_kernel<2>, mx, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)d, (int)n,
+                           pl->d_status, t->d_sched, 0, (int)dh, (const __nv_bfloat16*)X1, (const float*)nullptr,
+                           (const __nv_bfloat16*)V) != cudaSuccess)
+        return M2_ERR_CUDA;
+    pl->last_kernel = "conv_umma_o2_512_heads";
+    pl->launches += 1;
+    return M2_OK;
 }
 
 int32_t conv_fwd_wait_selftest(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,

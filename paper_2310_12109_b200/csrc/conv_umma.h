@@ -20,6 +20,11 @@ int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, in
 // (zero padded at both ends of a row; w_gate [H][3] fp32).  y may be x: the rows are then replaced in place.
 int32_t conv_gate_fwd(const m2_plan* plan, const void* x, const void* kf, const float* w_gate, void* y, int64_t B, int64_t H,
                       cudaStream_t stream);
+// The core of the M2 Hyena layer with heads of dh = 16 channels, in one kernel (no d_h-times larger tensor in memory):
+//   y[b][h dh + j][t] = sum_i X1[b][h dh + i][t] (k_h * (X2[b][h dh + i] V[b][h dh + j]))[t],   causal, t < n <= 256,
+// X1, X2, V, y: [B][d][n] bf16; kf_heads: the spectrum of the d / dh head kernels.  M2_ERR_UNSUPPORTED for other shapes.
+int32_t conv_heads_fwd(const m2_plan* plan, const void* X1, const void* X2, const void* V, const void* kf_heads, void* y, int64_t B,
+                       int64_t d, int64_t dh, int64_t n, cudaStream_t stream);
 // The row-pair kernel launched so that every pipeline's first bounded wait runs out with nothing in flight (no copy is
 // issued, a few polls per wait): the kernel leaves through its abort path, sets M2_ERR_TIMEOUT in the plan's status
 // word, writes nothing to y.  Needs B > 8 (the row-pair kernel); M2_ERR_UNSUPPORTED otherwise.

@@ -594,9 +594,17 @@ int32_t m2_bert_mixer_fwd(const m2_plan* plan, const void* x_dev, const void* co
     return M2_OK;
 }
 
+// heads of 16 channels on the N = 512 tensor-core plan: outer product, long convolution and contraction are one kernel and the
+// dh-times larger tensors do not exist
+static bool hyena_heads_fused(const m2_plan* plan, int64_t n, int64_t d, int64_t dh) {
+    return plan->dtype == M2_BF16 && m2u::has_private_spectrum(plan) && !m2u3::covered(plan) && dh == 16 && d % 16 == 0 && n % 16 == 0 &&
+           n <= 256;
+}
+
 int64_t m2_hyena_scratch_bytes(const m2_plan* plan, int64_t B, int64_t n, int64_t d, int64_t dh) {
     if (!plan || B < 0 || n < 0 || d < 0 || dh <= 0) return -1;
-    return (7 + 2 * dh) * round256(B * d * n * (plan->dtype == M2_BF16 ? 2 : 4));
+    const int64_t big = hyena_heads_fused(plan, n, d, dh) ? 0 : 2 * dh;
+    return (7 + big) * round256(B * d * n * (plan->dtype == M2_BF16 ? 2 : 4));
 }
 
 int32_t m2_hyena_heads_fwd(const m2_plan* plan, const void* u_dev, const void* const* W, const void* kf1_dev, const void* kf2_dev,
@@ -638,15 +646,21 @@ int32_t m2_hyena_heads_fwd(const m2_plan* plan, const void* u_dev, const void* c
     if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, P2, kf2_dev, C2, B, d, n, M2_CAUSAL, stream);
     if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, P3, kf3_dev, C3, B, d, n, M2_CAUSAL, stream);
     if (rc != M2_OK) return rc;
-    if (m2g::launch_heads_outer(C2, C3, XV, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    rc = conv_fwd_grouped(plan, XV, kf_long_dev, XVc, B, d * dh, n, M2_CAUSAL, dh * dh, stream);   // dh^2 channels share a head's kernel
-    if (rc != M2_OK) return rc;
-    if (m2g::launch_heads_reduce(C1, XVc, P1, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    if (hyena_heads_fused(plan, n, d, dh)) {
+        rc = m2u::conv_heads_fwd(plan, C1, C2, C3, kf_long_dev, P1, B, d, dh, n, st);
+        if (rc != M2_OK) return rc;
+    } else {
+        if (m2g::launch_heads_outer(C2, C3, XV, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+        rc = conv_fwd_grouped(plan, XV, kf_long_dev, XVc, B, d * dh, n, M2_CAUSAL, dh * dh, stream);   // dh^2 channels share a head's kernel
+        if (rc != M2_OK) return rc;
+        if (m2g::launch_heads_reduce(C1, XVc, P1, B, (int)d, (int)dh, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+        plan->launches += 2;
+    }
     rc = dense(W[3], P1, P2);
     if (rc != M2_OK) return rc;
     if (m2g::launch_transpose_any(P2, y_dev, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    plan->launches += 4;   // two transposes and the two head kernels (the products and convolutions count themselves)
-    plan->last_kernel = "hyena_heads_fwd";
+    plan->launches += 2;   // the two transposes (the products, convolutions and head kernels count themselves)
+    plan->last_kernel = hyena_heads_fused(plan, n, d, dh) ? "hyena_heads_fwd_fused" : "hyena_heads_fwd";
     return M2_OK;
 }
 

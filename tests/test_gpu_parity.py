@@ -688,7 +688,9 @@ def run_monarch_cols(N1, N2, Bt, d, dtype, withK):
     plan.close()
 
 
-@pytest.mark.parametrize("B,n,d,dh,dims,dtype", [(9, 256, 128, 16, (32, 16), M.M2_BF16), (2, 100, 64, 4, (32, 16), M.M2_BF16),
+@pytest.mark.parametrize("B,n,d,dh,dims,dtype", [(9, 256, 128, 16, (32, 16), M.M2_BF16),   # heads of 16: one fused tensor-core kernel
+                                                  (3, 112, 64, 16, (32, 16), M.M2_BF16),    # the same with a ragged sequence length
+                                                  (2, 100, 64, 4, (32, 16), M.M2_BF16),     # other head sizes: three kernels
                                                   (2, 24, 12, 3, (8, 8), M.M2_FP32)])
 def test_m2_hyena_heads_fwd(B, n, d, dh, dims, dtype):
     """The M2 Hyena layer with heads: projections, short convolutions, head outer products through the long convolution, output
@@ -709,7 +711,8 @@ def test_m2_hyena_heads_fwd(B, n, d, dh, dims, dtype):
     W = [dv(np.ascontiguousarray(p[k].T)) for k in ("W_x1", "W_x2", "W_v", "W_o")]   # stored outputs x inputs
     y = M.m2_hyena_heads_fwd(plan, dv(u), W, kfs[0], kfs[1], kfs[2], kfl, dh)
     torch.cuda.synchronize()
-    assert plan.device_status() == 0 and plan.last_kernel() == "hyena_heads_fwd"
+    fused = dtype == M.M2_BF16 and dims == (32, 16) and dh == 16 and n % 16 == 0 and n <= 256
+    assert plan.device_status() == 0 and plan.last_kernel() == ("hyena_heads_fwd_fused" if fused else "hyena_heads_fwd")
     ref = O.m2_hyena_heads(u, p, dims, dh)
     # The first positions of a causal layer have tiny outputs (one term of every convolution), so their rows are judged
     # against the typical row norm: an absolute error bound of 2 tol x the RMS row norm, plus the global relative bound.

@@ -430,7 +430,9 @@ static_assert(kGroupsP * 32 <= 512 && kGroupsP * kTmemColsPerGroup <= kTmemCols 
 // depthwise convolution of the INPUT row, y[t] <- y[t] (w[h][0] x[t-1] + w[h][1] x[t] + w[h][2] x[t+1]), zero padded at both ends
 // of the row.  xg = the input rows again ([B][H][512], read from L2 in the last hand-off: the unit's tile in shared memory has
 // long been replaced by the next unit's), w_gate = [H][3] fp32.  The output may be written over the input (map_y over the same rows
-// as map_x): a unit's rows are read for the last time before its stores are issued, and no other unit touches them.
+// as map_x): a unit's rows are read for the last time before its stores are issued, and no other unit touches them.  The gate may
+// also be taken from other rows than the convolution's input (xg need not be what map_x covers), and vh != nullptr names rows
+// [B][H][512] that are added after the gate: y <- y gate + vh (the gated M2-BERT sequence mixer: V (.) conv(k, Q (.) K) + conv(k_res, x)).
 //
 // HEADS (MODE 2; the core of the M2 Hyena layer with heads of dh = 16 channels, GPT appendix): a unit is one (batch entry b, channel
 // hj = head * 16 + j) and its 16 rows are the sequences X2[b][head * 16 + i][t] V[b][hj][t], i = 0 .. 15, of the head's outer
@@ -849,13 +851,13 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             for (int g = 0; g < (HEADS ? 0 : 2); ++g) {   // two rows at a time
                 // GATE: the 16 input values under this thread's run and their two neighbours, for both rows (requested before the
                 // accumulator is read so that the two latencies overlap)
-                uint4 xa[2], xb[2];
+                uint4 xa[2], xb[2], aa[2], ab[2];
                 unsigned short xl[2], xr[2];
                 if (GATE) {
 #pragma unroll
                     for (int rr = 0; rr < 2; ++rr) {
                         const int brow = b0 + kRows * c + 4 * rh + 2 * g + rr;
-                        xa[rr] = xb[rr] = make_uint4(0u, 0u, 0u, 0u);
+                        xa[rr] = xb[rr] = aa[rr] = ab[rr] = make_uint4(0u, 0u, 0u, 0u);
                         xl[rr] = xr[rr] = 0;
                         if (brow < B) {
                             const __nv_bfloat16* xrow = xg + ((size_t)brow * H + h) * 512 + 16 * n1;
@@ -863,6 +865,11 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                             xb[rr] = __ldg(reinterpret_cast<const uint4*>(xrow) + 1);
                             if (n1 > 0) xl[rr] = __ldg(reinterpret_cast<const unsigned short*>(xrow) - 1);
                             if (n1 < 31) xr[rr] = __ldg(reinterpret_cast<const unsigned short*>(xrow) + 16);
+                            if (vh != nullptr) {
+                                const uint4* arow = reinterpret_cast<const uint4*>(vh + ((size_t)brow * H + h) * 512 + 16 * n1);
+                                aa[rr] = __ldg(arow);
+                                ab[rr] = __ldg(arow + 1);
+                            }
                         }
                     }
                 }
@@ -884,8 +891,12 @@ conv512p_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                             xv[1 + 2 * j] = __uint_as_float(xw[j] << 16);
                             xv[2 + 2 * j] = __uint_as_float(xw[j] & 0xffff0000u);
                         }
+                        const uint32_t aw[8] = {aa[rr].x, aa[rr].y, aa[rr].z, aa[rr].w, ab[rr].x, ab[rr].y, ab[rr].z, ab[rr].w};
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) v[16 * rr + j] *= fmaf(w2, xv[j + 2], fmaf(w1, xv[j + 1], w0 * xv[j]));
+                        for (int j = 0; j < 16; ++j) {
+                            const float add = (j & 1) ? __uint_as_float(aw[j >> 1] & 0xffff0000u) : __uint_as_float(aw[j >> 1] << 16);
+                            v[16 * rr + j] = fmaf(v[16 * rr + j], fmaf(w2, xv[j + 2], fmaf(w1, xv[j + 1], w0 * xv[j])), add);
+                        }
                     }
                 }
 #pragma unroll
@@ -1301,7 +1312,8 @@ static bool make_map_rows32(CUtensorMap* map, const void* ptr, int64_t B, int64_
 }
 
 static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, void* y, int64_t B, int64_t H, int64_t n, int32_t mode,
-                             cudaStream_t stream, int selftest, int kf_group, const float* w_gate = nullptr) {
+                             cudaStream_t stream, int selftest, int kf_group, const float* w_gate = nullptr, const void* gate_rows = nullptr,
+                             const void* addend = nullptr) {
     if (!pl->umma || !covered(pl)) return M2_ERR_UNSUPPORTED;
     // rows must be whole multiples of the inner digit and 16-byte pitched for TMA
     if (n % 16 != 0 || (mode == M2_CIRCULAR && n != 512) || n > 512) return M2_ERR_UNSUPPORTED;
@@ -1338,8 +1350,8 @@ static int32_t conv_fwd_impl(const m2_plan* pl, const void* x, const void* kf, v
         const cudaError_t le =
             w_gate != nullptr
                 ? cudaLaunchKernelEx(&cfg, conv512p_kernel<1>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
-                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)x, w_gate,
-                                     (const __nv_bfloat16*)nullptr)
+                                     (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)(gate_rows ? gate_rows : x), w_gate,
+                                     (const __nv_bfloat16*)addend)
                 : cudaLaunchKernelEx(&cfg, conv512p_kernel<0>, mx32, my, (__nv_bfloat16*)y, kfu, (const uint4*)t->d_const_p, (int)B, (int)H,
                                      (int)n, pl->d_status, t->d_sched, selftest, kf_group, (const __nv_bfloat16*)nullptr, (const float*)nullptr,
                                      (const __nv_bfloat16*)nullptr);
@@ -1362,9 +1374,9 @@ int32_t conv_fwd(const m2_plan* pl, const void* x, const void* kf, void* y, int6
 }
 
 int32_t conv_gate_fwd(const m2_plan* pl, const void* x, const void* kf, const float* w_gate, void* y, int64_t B, int64_t H,
-                      cudaStream_t stream) {
+                      cudaStream_t stream, const void* gate_rows, const void* addend) {
     if (w_gate == nullptr) return M2_ERR_INVALID_ARG;
-    return conv_fwd_impl(pl, x, kf, y, B, H, 512, M2_CIRCULAR, stream, 0, 1, w_gate);
+    return conv_fwd_impl(pl, x, kf, y, B, H, 512, M2_CIRCULAR, stream, 0, 1, w_gate, gate_rows, addend);
 }
 
 int32_t conv_heads_fwd(const m2_plan* pl, const void* X1, const void* X2, const void* V, const void* kf_heads, void* y, int64_t B,

@@ -18,8 +18,10 @@ int32_t conv_fwd(const m2_plan* plan, const void* x, const void* kf, void* y, in
 // The circular convolution of [B][H][512] rows followed by the M2 block's depthwise gate, in one kernel:
 //   y[b][h][t] = conv(x[b][h], k[h])[t] * (w_gate[h][0] x[b][h][t-1] + w_gate[h][1] x[b][h][t] + w_gate[h][2] x[b][h][t+1])
 // (zero padded at both ends of a row; w_gate [H][3] fp32).  y may be x: the rows are then replaced in place.
+// gate_rows != nullptr: the gate is formed from these rows [B][H][512] instead of x; addend != nullptr: rows [B][H][512] added
+// after the gate, y = conv(x, k) * gate + addend (neither may be y).
 int32_t conv_gate_fwd(const m2_plan* plan, const void* x, const void* kf, const float* w_gate, void* y, int64_t B, int64_t H,
-                      cudaStream_t stream);
+                      cudaStream_t stream, const void* gate_rows = nullptr, const void* addend = nullptr);
 // The core of the M2 Hyena layer with heads of dh = 16 channels, in one kernel (no d_h-times larger tensor in memory):
 //   y[b][h dh + j][t] = sum_i X1[b][h dh + i][t] (k_h * (X2[b][h dh + i] V[b][h dh + j]))[t],   causal, t < n <= 256,
 // X1, X2, V, y: [B][d][n] bf16; kf_heads: the spectrum of the d / dh head kernels.  M2_ERR_UNSUPPORTED for other shapes.

@@ -582,15 +582,27 @@ int32_t m2_bert_mixer_fwd(const m2_plan* plan, const void* x_dev, const void* co
     if (rc == M2_OK) rc = dense(W[2], xT, Pv);
     if (rc != M2_OK) return rc;
     if (m2g::launch_gate_in(Pq, Pk, w_short[0], w_short[1], QK, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    rc = m2_monarch_conv_fwd(plan, QK, kf_dev, C, B, d, n, M2_CIRCULAR, stream);
-    if (rc == M2_OK) rc = m2_monarch_conv_fwd(plan, xT, kf_res_dev, Cr, B, d, n, M2_CIRCULAR, stream);
+    // the residual convolution first; on the N = 512 tensor-core plan the main convolution then applies the gate and adds the
+    // residual in its last hand-off (one kernel less and one tensor less through memory)
+    rc = m2_monarch_conv_fwd(plan, xT, kf_res_dev, Cr, B, d, n, M2_CIRCULAR, stream);
     if (rc != M2_OK) return rc;
-    if (m2g::launch_gate_out(Pv, w_short[2], C, Cr, Z, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+    bool fused_out = false;
+    if (bf && n == 512 && m2u::has_private_spectrum(plan) && !m2u3::covered(plan)) {
+        rc = m2u::conv_gate_fwd(plan, QK, kf_dev, w_short[2], Z, B, d, st, Pv, Cr);
+        if (rc == M2_OK) fused_out = true;
+        else if (rc != M2_ERR_UNSUPPORTED) return rc;
+    }
+    if (!fused_out) {
+        rc = m2_monarch_conv_fwd(plan, QK, kf_dev, C, B, d, n, M2_CIRCULAR, stream);
+        if (rc != M2_OK) return rc;
+        if (m2g::launch_gate_out(Pv, w_short[2], C, Cr, Z, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
+        plan->launches += 1;
+    }
     rc = dense(W[3], Z, Pq);
     if (rc != M2_OK) return rc;
     if (m2g::launch_transpose_any(Pq, y_dev, B, (int)d, (int)n, bf, st) != cudaSuccess) return M2_ERR_CUDA;
-    plan->launches += 4;
-    plan->last_kernel = "bert_mixer_fwd";
+    plan->launches += 3;   // the two transposes and the input gate (the products, convolutions and the output gate count themselves)
+    plan->last_kernel = fused_out ? "bert_mixer_fwd_fused_gate" : "bert_mixer_fwd";
     return M2_OK;
 }
 

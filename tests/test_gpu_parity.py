@@ -728,6 +728,39 @@ def test_m2_hyena_heads_fwd(B, n, d, dh, dims, dtype):
     plan.close()
 
 
+def test_m2_hyena_heads_full_size_sampled():
+    """The layer at the benchmark shape (B = 32, n = 256, d = 768, heads of 16: 24 576 units of the fused kernel, many rounds per
+    pipeline); batch entries are independent, so the first and the last one are compared with the oracle run on them alone."""
+    B, n, d, dh, dims = 32, 256, 768, 16, (32, 16)
+    rnd = synth.round_bf16
+    p = {k: rnd(synth.normal(synth.stream_id(16, i), (d, d)) / np.sqrt(d)) for i, k in enumerate(("W_x1", "W_x2", "W_v", "W_o"))}
+    dec = np.exp(-0.05 * np.arange(n))[None]
+    for i, k in enumerate(("K1", "K2", "K3")):
+        p[k] = (synth.normal(synth.stream_id(16, 4 + i), (d, n)) * dec / 4).astype(np.float32).astype(np.float64)
+    p["K_long"] = (synth.normal(synth.stream_id(16, 7), (d // dh, n)) * dec / 4).astype(np.float32).astype(np.float64)
+    u = rnd(synth.normal(synth.stream_id(16, 8), (B, n, d)))
+    plan = M.Plan(dims, dtype=M.M2_BF16, device=0)
+    f32 = lambda a: torch.from_numpy(a.astype(np.float32)).cuda()   # noqa: E731
+    kfs = [M.m2_kernel_spectrum(plan, f32(p[k])) for k in ("K1", "K2", "K3")]
+    kfl = M.m2_kernel_spectrum(plan, f32(p["K_long"]))
+    dv = lambda a: dev(a.astype(np.float32), torch.bfloat16)   # noqa: E731
+    W = [dv(np.ascontiguousarray(p[k].T)) for k in ("W_x1", "W_x2", "W_v", "W_o")]
+    y = M.m2_hyena_heads_fwd(plan, dv(u), W, kfs[0], kfs[1], kfs[2], kfl, dh)
+    torch.cuda.synchronize()
+    assert plan.device_status() == 0 and plan.last_kernel() == "hyena_heads_fwd_fused"
+    got_all = host(y)
+    assert np.isfinite(got_all).all()
+    sel = [0, B - 1]
+    ref = O.m2_hyena_heads(u[sel], p, dims, dh)
+    got, want = got_all[sel].reshape(-1, d), ref.reshape(-1, d)
+    gl = np.linalg.norm(got - want) / np.linalg.norm(want)
+    rms_row = np.sqrt(np.mean(np.sum(want * want, axis=1)))
+    worst = np.max(np.linalg.norm(got - want, axis=1)) / rms_row   # (first causal positions are tiny: judged against the typical row)
+    assert gl <= TOL_BF16, f"global rel-L2 {gl:.3e}"
+    assert worst <= 2 * TOL_BF16, f"worst row error {worst:.3e} of the RMS row norm"
+    plan.close()
+
+
 @pytest.mark.parametrize("B,d,dims,dtype", [(12, 128, (32, 16), M.M2_BF16), (3, 24, (32, 16), M.M2_BF16), (2, 10, (6, 4), M.M2_FP32)])
 def test_m2_bert_mixer_fwd(B, d, dims, dtype):
     """The gated bidirectional M2-BERT sequence mixer: projections, short filters, gated long convolution + residual convolution,
